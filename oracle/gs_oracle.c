@@ -1,0 +1,460 @@
+/*
+ * CPU oracle for the random-walk + skip-gram-with-negative-sampling (SGNS)
+ * path of GraphScale-style node-embedding training.
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is a plain, slow, single-threaded
+ * restatement of what the path computes, in fp64 for every floating-point
+ * quantity, written so that it can be checked against the definitions by eye.
+ * It shares no code, header, table or helper with the CUDA library and must
+ * never be called from the product path.
+ *
+ * What the paper fixes (Section 2.2 "Node embedding training", Section 3.2
+ * "Node Embedding Training", Section 4 "Configuration"):
+ *   - DeepWalk = random walks from every node fed to skip-gram; node2vec = the
+ *     same with a biased second-order walk (Section 2.2);
+ *   - training uses skip-gram with negative sampling (Section 2.2);
+ *   - a mini-batch of B source nodes touches at most B x walk_len nodes,
+ *     sources included, so walk_len counts NODES (Section 3.2);
+ *   - updates of a mini-batch are written as increments, and trainers may race
+ *     on the same rows, Hogwild style (Section 3.2 "Synchronization").
+ * Everything the paper leaves open (RNG, index mapping, negative distribution,
+ * masking, gradient scaling) follows the readings listed in the design notes
+ * of this repository; each function below states the reading it implements.
+ *
+ * Parity pins (see tests, "not gpu"): Philox known answers; walks follow
+ * edges; degree-proportional stationarity; node2vec closed-form transition
+ * weights; pair-count identity; alias-table mass identity; finite-difference
+ * gradients; closed form of the first step from zero output vectors;
+ * pair-order independence of the synchronous step.
+ * gso_sgns_seq_from_lists (sequential per-pair SGD, the reference point for
+ * the racy Hogwild mode) has no exact counterpart on the GPU: parity unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------
+ * Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as
+ * easy as 1, 2, 3", SC'11).  Ten rounds; each round multiplies two counter
+ * words by fixed odd constants, mixes high halves with the other two words
+ * and the key, and the key is bumped by Weyl constants between rounds.
+ * ---------------------------------------------------------------------- */
+void gso_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* Stream tags: which consumer of random words a counter belongs to. */
+enum { TAG_UNIFORM_WALK = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4 };
+
+/* Keying shared (as a published convention, not as code) with the GPU path:
+ * key = 64-bit seed; counter = (id low, id high, step, tag<<24 | sub). */
+static void draw4(uint64_t seed, uint64_t id, uint32_t step, uint32_t tag, uint32_t sub,
+                  uint32_t out[4])
+{
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t ctr[4] = { (uint32_t)id, (uint32_t)(id >> 32), step, (tag << 24) | sub };
+    gso_philox4x32_10(ctr, key, out);
+}
+
+/* Map a 32-bit word to [0, n) by multiply-high (bias <= n / 2^32, no rejection). */
+static uint64_t scale32(uint32_t r, uint64_t n)
+{
+    return ((uint64_t)r * n) >> 32;
+}
+
+/* ------------------------------------------------------------------------
+ * Uniform (DeepWalk) walks.  Section 2.2: "random walks from each node".
+ * walk[0] = start; each transition picks a uniformly random out-neighbour.
+ * A node without out-neighbours ends the walk; the remaining entries are -1.
+ * starts == NULL means start node = walk id mod n_nodes.
+ * Returns the number of transitions taken over all walks.
+ * ---------------------------------------------------------------------- */
+int64_t gso_uniform_walks(int64_t n_nodes, const int64_t *off, const int32_t *col,
+                          const int32_t *starts, int64_t n_walks, int64_t walk_id_base,
+                          int32_t L, uint64_t seed, int32_t *walks)
+{
+    int64_t steps = 0;
+    for (int64_t i = 0; i < n_walks; ++i) {
+        uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t *W = walks + i * (int64_t)L;
+        int32_t cur = starts ? starts[i] : (int32_t)(id % (uint64_t)n_nodes);
+        W[0] = cur;
+        int32_t t = 0;
+        for (; t + 1 < L; ++t) {
+            int64_t deg = off[cur + 1] - off[cur];
+            if (deg == 0) break;
+            uint32_t r[4];
+            draw4(seed, id, (uint32_t)t, TAG_UNIFORM_WALK, 0, r);
+            cur = col[off[cur] + (int64_t)scale32(r[0], (uint64_t)deg)];
+            W[t + 1] = cur;
+            ++steps;
+        }
+        for (int32_t s = t + 1; s < L; ++s) W[s] = -1;
+    }
+    return steps;
+}
+
+/* ------------------------------------------------------------------------
+ * node2vec second-order walks (Grover & Leskovec, KDD'16; named in Section
+ * 2.2).  Unnormalised weight of candidate x after the move prev -> cur:
+ *   1/p if x == prev;  1 if x is a neighbour of prev;  1/q otherwise.
+ * Sampled by rejection: propose x uniformly from adj(cur), accept with
+ * probability weight / max(1/p, 1, 1/q).  Acceptance compares a 32-bit word
+ * with an integer threshold T[class] = floor(weight/max * 2^32).
+ * ---------------------------------------------------------------------- */
+void gso_node2vec_thresholds(double p, double q, uint64_t T[3])
+{
+    double a_prev = 1.0 / p, a_near = 1.0, a_far = 1.0 / q;
+    double m = a_prev;
+    if (a_near > m) m = a_near;
+    if (a_far > m) m = a_far;
+    double a[3] = { a_prev, a_near, a_far };
+    for (int c = 0; c < 3; ++c) {
+        double v = floor(a[c] / m * 4294967296.0);
+        if (v > 4294967296.0) v = 4294967296.0;
+        T[c] = (uint64_t)v;
+    }
+}
+
+/* membership test in a strictly increasing adjacency list */
+static int is_neighbour(const int64_t *off, const int32_t *col, int32_t u, int32_t x)
+{
+    int64_t lo = off[u], hi = off[u + 1];
+    while (lo < hi) {
+        int64_t mid = lo + (hi - lo) / 2;
+        if (col[mid] < x) lo = mid + 1; else hi = mid;
+    }
+    return lo < off[u + 1] && col[lo] == x;
+}
+
+int64_t gso_node2vec_walks(int64_t n_nodes, const int64_t *off, const int32_t *col,
+                           const int32_t *starts, int64_t n_walks, int64_t walk_id_base,
+                           int32_t L, uint64_t seed, double p, double q, int32_t max_rounds,
+                           int32_t *walks, int64_t *cap_hits)
+{
+    uint64_t T[3];
+    gso_node2vec_thresholds(p, q, T);
+    int64_t steps = 0, caps = 0;
+    for (int64_t i = 0; i < n_walks; ++i) {
+        uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t *W = walks + i * (int64_t)L;
+        int32_t cur = starts ? starts[i] : (int32_t)(id % (uint64_t)n_nodes);
+        int32_t prev = -1;
+        W[0] = cur;
+        int32_t t = 0;
+        for (; t + 1 < L; ++t) {
+            int64_t deg = off[cur + 1] - off[cur];
+            if (deg == 0) break;
+            int32_t nxt = -1;
+            if (t == 0) {
+                /* no predecessor yet: plain uniform choice */
+                uint32_t r[4];
+                draw4(seed, id, 0u, TAG_NODE2VEC, 0, r);
+                nxt = col[off[cur] + (int64_t)scale32(r[0], (uint64_t)deg)];
+            } else {
+                int accepted = 0;
+                for (int32_t s = 0; s < max_rounds && !accepted; ++s) {
+                    uint32_t r[4];
+                    draw4(seed, id, (uint32_t)t, TAG_NODE2VEC, (uint32_t)s, r);
+                    int32_t x = col[off[cur] + (int64_t)scale32(r[0], (uint64_t)deg)];
+                    int cls = (x == prev) ? 0 : (is_neighbour(off, col, prev, x) ? 1 : 2);
+                    nxt = x;
+                    if ((uint64_t)r[1] < T[cls]) accepted = 1;
+                }
+                if (!accepted) ++caps;   /* keeps the last proposal */
+            }
+            prev = cur;
+            cur = nxt;
+            W[t + 1] = cur;
+            ++steps;
+        }
+        for (int32_t s = t + 1; s < L; ++s) W[s] = -1;
+    }
+    if (cap_hits) *cap_hits = caps;
+    return steps;
+}
+
+/* ------------------------------------------------------------------------
+ * Window expansion and negative draws.
+ * For position i of a walk and every j with 0 < |i-j| <= w inside the walk,
+ * both entries present: pair (center = W[i], context = W[j]) in slot
+ * sigma = j - i + w - (j > i), 0 <= sigma < 2w.  (Fixed window; Section 4
+ * gives only "window-size".)
+ * For each pair, K negatives from the alias table (thr, alias) over n_alias
+ * nodes: word pair (a, b) -> cell jj = mulhi(a, n_alias); keep jj if
+ * b < thr[jj] else alias[jj].  Negatives 2m and 2m+1 use words (0,1) and
+ * (2,3) of the Philox block with step = i*2w + sigma, sub = m.
+ *
+ * Output lists are laid out by slot: entry e = (walk*L + i)*2w + sigma;
+ * centers[e] = contexts[e] = -1 and negs[e*K..] = -1 where no pair exists.
+ * Returns the number of pairs.
+ * ---------------------------------------------------------------------- */
+int64_t gso_expand_lists(const int32_t *walks, int64_t n_walks, int64_t walk_id_base,
+                         int32_t L, int32_t w, int32_t K,
+                         const uint32_t *thr, const int32_t *alias, int64_t n_alias,
+                         uint64_t seed,
+                         int32_t *centers, int32_t *contexts, int32_t *negs)
+{
+    int64_t n_pairs = 0;
+    const int32_t S = 2 * w;
+    for (int64_t a = 0; a < n_walks; ++a) {
+        const int32_t *W = walks + a * (int64_t)L;
+        uint64_t id = (uint64_t)(walk_id_base + a);
+        for (int32_t i = 0; i < L; ++i) {
+            for (int32_t sg = 0; sg < S; ++sg) {
+                int64_t e = (a * (int64_t)L + i) * S + sg;
+                /* invert sigma = j - i + w - (j > i) */
+                int32_t j = (sg < w) ? (i - w + sg) : (i - w + sg + 1);
+                int ok = (W[i] >= 0) && (j >= 0) && (j < L) && (W[j] >= 0);
+                centers[e] = ok ? W[i] : -1;
+                contexts[e] = ok ? W[j] : -1;
+                for (int32_t k = 0; k < K; ++k) negs[e * K + k] = -1;
+                if (!ok) continue;
+                ++n_pairs;
+                for (int32_t m = 0; 2 * m < K; ++m) {
+                    uint32_t r[4];
+                    draw4(seed, id, (uint32_t)(i * S + sg), TAG_NEGATIVE, (uint32_t)m, r);
+                    for (int h = 0; h < 2 && 2 * m + h < K; ++h) {
+                        uint32_t ra = r[2 * h], rb = r[2 * h + 1];
+                        int64_t jj = (int64_t)scale32(ra, (uint64_t)n_alias);
+                        negs[e * K + 2 * m + h] = (rb < thr[jj]) ? (int32_t)jj : alias[jj];
+                    }
+                }
+            }
+        }
+    }
+    return n_pairs;
+}
+
+/* ------------------------------------------------------------------------
+ * Alias table (Walker / Vose) for p(v) proportional to weight(v)^power;
+ * zero-weight entries get probability zero.  Cells are processed through
+ * two first-in-first-out queues filled in increasing node order, so the
+ * table is a deterministic function of the weights.
+ * thr[v] = floor(keep_probability * 2^32) capped at 2^32 - 1; a cell whose
+ * keep probability is one aliases to itself, which makes the cap harmless.
+ * Returns 0, or -1 when no weight is positive / allocation fails.
+ * ---------------------------------------------------------------------- */
+int gso_build_alias(const double *weights, int64_t n, double power,
+                    uint32_t *thr, int32_t *alias)
+{
+    double *s = (double *)malloc(sizeof(double) * (size_t)n);
+    int64_t *small = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
+    int64_t *large = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
+    if (!s || !small || !large) { free(s); free(small); free(large); return -1; }
+    double total = 0.0;
+    for (int64_t v = 0; v < n; ++v) {
+        s[v] = weights[v] > 0.0 ? pow(weights[v], power) : 0.0;
+        total += s[v];
+    }
+    if (!(total > 0.0)) { free(s); free(small); free(large); return -1; }
+    int64_t sh = 0, st = 0, lh = 0, lt = 0;   /* queue heads and tails */
+    for (int64_t v = 0; v < n; ++v) {
+        s[v] = s[v] * (double)n / total;
+        if (s[v] < 1.0) small[st++] = v; else large[lt++] = v;
+    }
+    for (int64_t v = 0; v < n; ++v) { thr[v] = 0xFFFFFFFFu; alias[v] = (int32_t)v; }
+    while (sh < st && lh < lt) {
+        int64_t l = small[sh++];
+        int64_t g = large[lh];
+        double keep = floor(s[l] * 4294967296.0);
+        thr[l] = keep >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)keep;
+        alias[l] = (int32_t)g;
+        s[g] = (s[g] + s[l]) - 1.0;
+        if (s[g] < 1.0) { ++lh; small[st++] = g; }
+    }
+    /* whatever is left keeps its whole cell (thr = max, alias = self) */
+    free(s); free(small); free(large);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Table initialisation: input vectors uniform in [-0.5/d, 0.5/d), output
+ * vectors zero (the word2vec convention).  Entry (row, j) uses word j%4 of
+ * the Philox block (id = row, step = j/4, TAG_INIT): u = (word>>8) * 2^-24,
+ * value = (u - 0.5)/d.  Fills rows rows[0..n_rows) of a compact table.
+ * ---------------------------------------------------------------------- */
+void gso_init_rows(const int64_t *rows, int64_t n_rows, int32_t d, uint64_t seed, double *U)
+{
+    for (int64_t a = 0; a < n_rows; ++a) {
+        for (int32_t j = 0; j < d; ++j) {
+            uint32_t r[4];
+            draw4(seed, (uint64_t)rows[a], (uint32_t)(j / 4), TAG_INIT, 0, r);
+            double u = (double)(r[j % 4] >> 8) * (1.0 / 16777216.0);
+            U[a * (int64_t)d + j] = (u - 0.5) / (double)d;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------
+ * SGNS objective for one pair (c, o) with negatives n_1..n_K:
+ *   loss = softplus(-<U_c,V_o>) + sum_k softplus(<U_c,V_nk>)
+ * (Mikolov et al. 2013, the "skip-gram and negative sampling" of Section
+ * 2.2).  A negative equal to the pair's context is masked: no loss term and
+ * no gradient.
+ * ---------------------------------------------------------------------- */
+static double softplus(double x)
+{
+    return (x > 0.0 ? x : 0.0) + log1p(exp(-fabs(x)));
+}
+static double sigmoid(double x)
+{
+    return 1.0 / (1.0 + exp(-x));
+}
+static double dot(const double *a, const double *b, int32_t d)
+{
+    double s = 0.0;
+    for (int32_t j = 0; j < d; ++j) s += a[j] * b[j];
+    return s;
+}
+
+/* Loss of a list of pairs at fixed tables (used for finite differences). */
+double gso_sgns_loss_from_lists(const double *U, const double *V, int32_t d,
+                                int64_t n_slots, int32_t K,
+                                const int32_t *centers, const int32_t *contexts,
+                                const int32_t *negs)
+{
+    double loss = 0.0;
+    for (int64_t e = 0; e < n_slots; ++e) {
+        if (centers[e] < 0) continue;
+        const double *u = U + (int64_t)centers[e] * d;
+        loss += softplus(-dot(u, V + (int64_t)contexts[e] * d, d));
+        for (int32_t k = 0; k < K; ++k) {
+            int32_t nk = negs[e * K + k];
+            if (nk < 0 || nk == contexts[e]) continue;
+            loss += softplus(dot(u, V + (int64_t)nk * d, d));
+        }
+    }
+    return loss;
+}
+
+/* ------------------------------------------------------------------------
+ * Deterministic synchronous mini-batch step (Section 3.2: gradients of the
+ * mini-batch are computed from the embeddings fetched at the start of the
+ * iteration and written back as increments, with a barrier after the write).
+ * All gradients use the tables as they are on entry; the increments of every
+ * pair are summed (not averaged) and applied once:
+ *   g_o = sigmoid(f_o) - 1, g_k = sigmoid(f_k)
+ *   GU[c] += g_o V_o + sum_k g_k V_nk ;  GV[o] += g_o U_c ;  GV[nk] += g_k U_c
+ *   U -= lr GU ; V -= lr GV
+ * order == NULL visits slots 0..n_slots-1; otherwise in the given order (the
+ * result must not depend on it beyond rounding).
+ * Row indices in the lists address rows of U and V directly (the caller may
+ * have remapped node ids to a compact table; masking compares the indices,
+ * which a one-to-one remap preserves).
+ * ---------------------------------------------------------------------- */
+int gso_sgns_det_from_lists(double *U, double *V, int64_t n_rows, int32_t d,
+                            int64_t n_slots, int32_t K,
+                            const int32_t *centers, const int32_t *contexts,
+                            const int32_t *negs, const int64_t *order,
+                            double lr, double *loss_sum, int64_t *pair_count)
+{
+    double *GU = (double *)calloc((size_t)(n_rows * d), sizeof(double));
+    double *GV = (double *)calloc((size_t)(n_rows * d), sizeof(double));
+    if (!GU || !GV) { free(GU); free(GV); return -1; }
+    double loss = 0.0;
+    int64_t pairs = 0;
+    for (int64_t a = 0; a < n_slots; ++a) {
+        int64_t e = order ? order[a] : a;
+        if (centers[e] < 0) continue;
+        int64_t c = centers[e], o = contexts[e];
+        const double *u = U + c * d;
+        ++pairs;
+        {
+            const double *v = V + o * d;
+            double f = dot(u, v, d);
+            double g = sigmoid(f) - 1.0;
+            loss += softplus(-f);
+            for (int32_t j = 0; j < d; ++j) {
+                GU[c * d + j] += g * v[j];
+                GV[o * d + j] += g * u[j];
+            }
+        }
+        for (int32_t k = 0; k < K; ++k) {
+            int64_t nk = negs[e * K + k];
+            if (nk < 0 || nk == o) continue;
+            const double *v = V + nk * d;
+            double f = dot(u, v, d);
+            double g = sigmoid(f);
+            loss += softplus(f);
+            for (int32_t j = 0; j < d; ++j) {
+                GU[c * d + j] += g * v[j];
+                GV[nk * d + j] += g * u[j];
+            }
+        }
+    }
+    for (int64_t x = 0; x < n_rows * d; ++x) {
+        U[x] -= lr * GU[x];
+        V[x] -= lr * GV[x];
+    }
+    free(GU); free(GV);
+    if (loss_sum) *loss_sum = loss;
+    if (pair_count) *pair_count = pairs;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Sequential per-pair SGD (each pair sees all earlier updates): the
+ * race-free limit of the lock-free mode of Section 3.2 "Synchronization".
+ * For each center position the center row is held fixed while its pairs
+ * update the output rows, and the accumulated center gradient is applied
+ * after the position's last pair (the word2vec order).  Slots must be laid
+ * out position-major as gso_expand_lists writes them, S slots per position.
+ * parity unpinned: the GPU's lock-free mode is racy by design.
+ * ---------------------------------------------------------------------- */
+int gso_sgns_seq_from_lists(double *U, double *V, int32_t d,
+                            int64_t n_slots, int32_t S, int32_t K,
+                            const int32_t *centers, const int32_t *contexts,
+                            const int32_t *negs, double lr,
+                            double *loss_sum, int64_t *pair_count)
+{
+    double *acc = (double *)malloc(sizeof(double) * (size_t)d);
+    if (!acc) return -1;
+    double loss = 0.0;
+    int64_t pairs = 0;
+    for (int64_t base = 0; base < n_slots; base += S) {
+        int64_t c = -1;
+        for (int32_t j = 0; j < d; ++j) acc[j] = 0.0;
+        for (int32_t sg = 0; sg < S && base + sg < n_slots; ++sg) {
+            int64_t e = base + sg;
+            if (centers[e] < 0) continue;
+            c = centers[e];
+            const double *u = U + c * d;
+            int64_t o = contexts[e];
+            ++pairs;
+            for (int32_t k = -1; k < K; ++k) {
+                int64_t t = (k < 0) ? o : negs[e * K + k];
+                if (k >= 0 && (t < 0 || t == o)) continue;
+                double *v = V + t * d;
+                double f = dot(u, v, d);
+                double g = (k < 0) ? sigmoid(f) - 1.0 : sigmoid(f);
+                loss += (k < 0) ? softplus(-f) : softplus(f);
+                for (int32_t j = 0; j < d; ++j) {
+                    acc[j] += g * v[j];
+                    v[j] -= lr * g * u[j];
+                }
+            }
+        }
+        if (c >= 0)
+            for (int32_t j = 0; j < d; ++j) U[c * d + j] -= lr * acc[j];
+    }
+    free(acc);
+    if (loss_sum) *loss_sum = loss;
+    if (pair_count) *pair_count = pairs;
+    return 0;
+}

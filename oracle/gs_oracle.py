@@ -1,0 +1,246 @@
+"""ctypes front end of the CPU oracle (gs_oracle.c).
+
+TEST INFRASTRUCTURE ONLY.  Nothing on the product path may import this module;
+it exists so that tests, the smoke check and the benchmark's CPU-baseline leg
+can call the plain C restatement of the walk + SGNS path.  It shares no code
+with the CUDA library and takes every input (CSR arrays, alias table, walks,
+tables) as plain numpy data.
+
+Array conventions: CSR offsets are passed as int64 (int32 offsets are widened
+here), columns / walks / lists as int32, tables as C-contiguous float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "gs_oracle.c"
+_LIB = _HERE / "libgs_oracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile gs_oracle.c with gcc (-O2, no fast-math) if the library is stale."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".{os.getpid()}.tmp")
+        subprocess.run(
+            ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-ffp-contract=off",
+             "-o", str(tmp), str(_SRC), "-lm"],
+            check=True,
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _p(a, ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(str(_LIB))
+        L.gso_uniform_walks.restype = ctypes.c_int64
+        L.gso_node2vec_walks.restype = ctypes.c_int64
+        L.gso_expand_lists.restype = ctypes.c_int64
+        L.gso_sgns_loss_from_lists.restype = ctypes.c_double
+        _lib = L
+    return _lib
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def _i32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.int32)
+
+
+def philox4x32_10(ctr, key):
+    """Philox4x32-10 block for a 4-word counter and 2-word key (SC'11)."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().gso_philox4x32_10(_p(c, ctypes.c_uint32), _p(k, ctypes.c_uint32),
+                            _p(out, ctypes.c_uint32))
+    return out
+
+
+def uniform_walks(off, col, starts, n_walks, walk_id_base, L, seed):
+    """DeepWalk walks (Section 2.2).  Returns (walks[n_walks, L], steps)."""
+    off = _i64(off)
+    col = _i32(col)
+    starts = _i32(starts)
+    walks = np.empty((n_walks, L), dtype=np.int32)
+    steps = lib().gso_uniform_walks(
+        ctypes.c_int64(len(off) - 1), _p(off, ctypes.c_int64), _p(col, ctypes.c_int32),
+        _p(starts, ctypes.c_int32), ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base),
+        ctypes.c_int32(L), ctypes.c_uint64(seed), _p(walks, ctypes.c_int32))
+    return walks, int(steps)
+
+
+def node2vec_thresholds(p, q):
+    T = np.zeros(3, dtype=np.uint64)
+    lib().gso_node2vec_thresholds(ctypes.c_double(p), ctypes.c_double(q),
+                                  _p(T, ctypes.c_uint64))
+    return T
+
+
+def node2vec_walks(off, col, starts, n_walks, walk_id_base, L, seed, p, q, max_rounds=1024):
+    """node2vec walks (Section 2.2).  Returns (walks, steps, cap_hits)."""
+    off = _i64(off)
+    col = _i32(col)
+    starts = _i32(starts)
+    walks = np.empty((n_walks, L), dtype=np.int32)
+    caps = ctypes.c_int64(0)
+    steps = lib().gso_node2vec_walks(
+        ctypes.c_int64(len(off) - 1), _p(off, ctypes.c_int64), _p(col, ctypes.c_int32),
+        _p(starts, ctypes.c_int32), ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base),
+        ctypes.c_int32(L), ctypes.c_uint64(seed), ctypes.c_double(p), ctypes.c_double(q),
+        ctypes.c_int32(max_rounds), _p(walks, ctypes.c_int32), ctypes.byref(caps))
+    return walks, int(steps), int(caps.value)
+
+
+def expand_lists(walks, walk_id_base, w, K, thr, alias, seed):
+    """Window pairs and negative draws, slot layout [(walk, i, sigma)].
+
+    Returns (centers[n_slots], contexts[n_slots], negs[n_slots, K], n_pairs).
+    """
+    walks = _i32(walks)
+    n_walks, L = walks.shape
+    thr = np.ascontiguousarray(thr, dtype=np.uint32)
+    alias = _i32(alias)
+    n_slots = n_walks * L * 2 * w
+    centers = np.empty(n_slots, dtype=np.int32)
+    contexts = np.empty(n_slots, dtype=np.int32)
+    negs = np.empty((n_slots, K), dtype=np.int32)
+    n_pairs = lib().gso_expand_lists(
+        _p(walks, ctypes.c_int32), ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base),
+        ctypes.c_int32(L), ctypes.c_int32(w), ctypes.c_int32(K),
+        _p(thr, ctypes.c_uint32), _p(alias, ctypes.c_int32), ctypes.c_int64(len(thr)),
+        ctypes.c_uint64(seed),
+        _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32))
+    return centers, contexts, negs, int(n_pairs)
+
+
+def build_alias(weights, power=0.75):
+    """Alias table for p(v) ~ weight(v)**power.  Returns (thr uint32, alias int32)."""
+    wgt = np.ascontiguousarray(weights, dtype=np.float64)
+    n = len(wgt)
+    thr = np.empty(n, dtype=np.uint32)
+    alias = np.empty(n, dtype=np.int32)
+    rc = lib().gso_build_alias(_p(wgt, ctypes.c_double), ctypes.c_int64(n),
+                               ctypes.c_double(power), _p(thr, ctypes.c_uint32),
+                               _p(alias, ctypes.c_int32))
+    if rc != 0:
+        raise ValueError("alias table needs at least one positive weight")
+    return thr, alias
+
+
+def init_rows(rows, d, seed):
+    """Initial input vectors of the given node ids (uniform in [-0.5/d, 0.5/d))."""
+    rows = _i64(rows)
+    U = np.empty((len(rows), d), dtype=np.float64)
+    lib().gso_init_rows(_p(rows, ctypes.c_int64), ctypes.c_int64(len(rows)),
+                        ctypes.c_int32(d), ctypes.c_uint64(seed), _p(U, ctypes.c_double))
+    return U
+
+
+def sgns_loss_from_lists(U, V, centers, contexts, negs):
+    d = U.shape[1]
+    negs = _i32(negs)
+    K = negs.shape[1]
+    return float(lib().gso_sgns_loss_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int32(d),
+        ctypes.c_int64(len(centers)), ctypes.c_int32(K),
+        _p(_i32(centers), ctypes.c_int32), _p(_i32(contexts), ctypes.c_int32),
+        _p(negs, ctypes.c_int32)))
+
+
+def sgns_det_from_lists(U, V, centers, contexts, negs, lr, order=None):
+    """Synchronous mini-batch step in place on float64 tables U, V.
+
+    Returns (loss_sum, pair_count); the loss is taken at the entry tables.
+    """
+    assert U.dtype == np.float64 and V.dtype == np.float64
+    assert U.flags.c_contiguous and V.flags.c_contiguous and U.shape == V.shape
+    n_rows, d = U.shape
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    K = negs.shape[1]
+    order = None if order is None else _i64(order)
+    loss = ctypes.c_double(0.0)
+    cnt = ctypes.c_int64(0)
+    rc = lib().gso_sgns_det_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int64(n_rows),
+        ctypes.c_int32(d), ctypes.c_int64(len(centers)), ctypes.c_int32(K),
+        _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32),
+        _p(order, ctypes.c_int64), ctypes.c_double(lr), ctypes.byref(loss), ctypes.byref(cnt))
+    if rc != 0:
+        raise MemoryError("oracle gradient buffers")
+    return float(loss.value), int(cnt.value)
+
+
+def sgns_seq_from_lists(U, V, centers, contexts, negs, S, lr):
+    """Sequential per-pair SGD in place (race-free limit of the lock-free mode)."""
+    assert U.dtype == np.float64 and V.dtype == np.float64
+    d = U.shape[1]
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    K = negs.shape[1]
+    loss = ctypes.c_double(0.0)
+    cnt = ctypes.c_int64(0)
+    rc = lib().gso_sgns_seq_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int32(d),
+        ctypes.c_int64(len(centers)), ctypes.c_int32(S), ctypes.c_int32(K),
+        _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32),
+        ctypes.c_double(lr), ctypes.byref(loss), ctypes.byref(cnt))
+    if rc != 0:
+        raise MemoryError("oracle accumulator")
+    return float(loss.value), int(cnt.value)
+
+
+def lr_at(schedule, lr0, b, num_batches):
+    """Learning rate of mini-batch b: 'constant', or 'linear' decay floored at 1e-4 lr0."""
+    if schedule == "constant":
+        return lr0
+    if schedule == "linear":
+        return lr0 * max(1.0 - b / num_batches, 1e-4)
+    raise ValueError(schedule)
+
+
+def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, schedule,
+               batch_walks, seed, mode="det", kind="uniform", p=1.0, q=1.0,
+               first_batch=0, num_batches=None):
+    """One pass over walk ids rep*N + v in order, batch by batch (dense tables).
+
+    Each batch: generate its walks, expand pairs and negatives, apply one step.
+    Returns dict(loss_sum, pairs, steps).  Tables are updated in place.
+    """
+    n_nodes = len(off) - 1
+    total = n_nodes * walks_per_node
+    nb_total = (total + batch_walks - 1) // batch_walks
+    if num_batches is None:
+        num_batches = nb_total - first_batch
+    loss_sum, pairs, steps = 0.0, 0, 0
+    for b in range(first_batch, first_batch + num_batches):
+        base = b * batch_walks
+        n = min(batch_walks, total - base)
+        if kind == "uniform":
+            walks, st = uniform_walks(off, col, None, n, base, L, seed)
+        else:
+            walks, st, _ = node2vec_walks(off, col, None, n, base, L, seed, p, q)
+        c, o, ng, _ = expand_lists(walks, base, w, K, thr, alias, seed)
+        lr = lr_at(schedule, lr0, b, nb_total)
+        if mode == "det":
+            ls, pc = sgns_det_from_lists(U, V, c, o, ng, lr)
+        else:
+            ls, pc = sgns_seq_from_lists(U, V, c, o, ng, 2 * w, lr)
+        loss_sum += ls
+        pairs += pc
+        steps += st
+    return {"loss_sum": loss_sum, "pairs": pairs, "steps": steps}

@@ -1,0 +1,258 @@
+/*
+ * gs.h - C ABI of the B200 random-walk + SGNS library.
+ *
+ * The library implements, on one GPU, the data-parallel hot path of
+ * unsupervised node-embedding training as GraphScale runs it (paper Section
+ * 2.2 "Node embedding training" and Section 3.2 "Node Embedding Training"):
+ * random walks over a CSR graph (DeepWalk: uniform; node2vec: second-order
+ * biased) and the skip-gram-with-negative-sampling (SGNS) update of an input
+ * and an output embedding table, either as a synchronous mini-batch step
+ * whose result does not depend on thread scheduling, or lock-free (Section
+ * 3.2 "Synchronization": trainers write increments to the same rows without
+ * locking).
+ *
+ * Conventions
+ *  - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  Every
+ *    buffer is allocated and freed by the caller; the library borrows it for
+ *    the duration of the call (a graph handle borrows the CSR arrays until
+ *    gs_graph_free).  The library allocates only its own scratch memory
+ *    (cached per device, released by gs_release_workspace).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *    Calls enqueue work on it and return without waiting unless stated.
+ *  - Every function returns a gs_status; nothing throws, aborts or traps.
+ *    gs_last_error() gives a thread-local description of the last failure.
+ *  - Random numbers are Philox4x32-10 blocks with key = seed and counter =
+ *    (id low, id high, step, tag << 24 | sub): a result depends on
+ *    (seed, walk id, position), never on launch shape or batching.
+ *      tag 1 uniform walk : id = walk id, step = transition index t
+ *      tag 2 node2vec     : id = walk id, step = t, sub = rejection round
+ *      tag 3 negatives    : id = walk id, step = i * 2w + slot, sub = m
+ *      tag 4 table init   : id = row, step = column / 4
+ *  - A 32-bit word r is mapped to [0, n) as (r * n) >> 32.
+ */
+#ifndef GS_H
+#define GS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define GS_API __attribute__((visibility("default")))
+#else
+#define GS_API
+#endif
+
+typedef int32_t gs_status;
+#define GS_OK                 0
+#define GS_ERR_INVALID_ARG   (-1)  /* null pointer, negative size, bad enum          */
+#define GS_ERR_BAD_CSR       (-2)  /* offsets not monotone / column out of range     */
+#define GS_ERR_UNSORTED_ADJ  (-3)  /* a row is not strictly increasing               */
+#define GS_ERR_CUDA          (-4)  /* a CUDA call failed; text in gs_last_error()    */
+#define GS_ERR_OOM           (-5)  /* scratch allocation failed                      */
+#define GS_ERR_UNSUPPORTED   (-6)  /* shape outside the supported range              */
+
+/* Thread-local, library-owned, NUL-terminated; valid until the next call. */
+GS_API const char *gs_last_error(void);
+
+/* ---------------------------------------------------------------- graph */
+typedef struct gs_graph gs_graph;
+
+#define GS_VALIDATE        1u   /* check offsets and column range on the device    */
+#define GS_REQUIRE_SORTED  2u   /* additionally require strictly increasing rows   */
+
+/*
+ * Wraps a CSR graph that already lives in device memory (the whole topology
+ * stays resident next to the sampler, as each trainer keeps it in Section 3.1).
+ *   d_offsets : n_nodes+1 entries, int64 if offsets_are_64bit else int32
+ *   d_cols    : n_edges int32 neighbour ids
+ * With GS_VALIDATE the call checks offsets[0] = 0, offsets[n] = n_edges,
+ * monotone offsets and 0 <= col < n_nodes, records the maximum degree, and
+ * WAITS for the result (one small device-to-host read).  node2vec needs
+ * GS_REQUIRE_SORTED rows.  On error *out is NULL; GS_ERR_BAD_CSR /
+ * GS_ERR_UNSORTED_ADJ name the first offending row in gs_last_error().
+ */
+GS_API gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges,
+                            const void *d_offsets, int32_t offsets_are_64bit,
+                            const int32_t *d_cols, uint32_t flags,
+                            void *stream, gs_graph **out);
+
+/* Frees the handle only; the CSR arrays stay the caller's. NULL is allowed. */
+GS_API void gs_graph_free(gs_graph *g);
+
+/* max_degree is -1 if the graph was loaded without GS_VALIDATE. */
+GS_API gs_status gs_graph_info(const gs_graph *g, int64_t *n_nodes, int64_t *n_edges,
+                        int64_t *max_degree, int32_t *rows_sorted);
+
+/* ---------------------------------------------------------------- alias table */
+/*
+ * HOST function.  Builds the alias table of p(v) ~ h_weights[v]^power (the
+ * word2vec unigram^0.75 negative distribution when weights are node
+ * frequencies or degrees; the paper only says nodes are "negatively sampled",
+ * Section 3.2).  Zero weights get probability zero.  Entry v of h_table_out
+ * packs thr (low 32 bits) and alias (high 32 bits): a draw with words (a, b)
+ * picks cell j = (a * n) >> 32 and returns j if b < thr[j], else alias[j].
+ * The caller uploads the table.  Deterministic: small and large cells are
+ * paired through two first-in-first-out queues filled in increasing v.
+ * Errors: GS_ERR_INVALID_ARG (null, n <= 0, n >= 2^31, no positive weight,
+ * negative or non-finite weight), GS_ERR_OOM.
+ */
+GS_API gs_status gs_build_alias(const double *h_weights, int64_t n, double power,
+                         uint64_t *h_table_out);
+
+/* ---------------------------------------------------------------- tables */
+/*
+ * Fills d_w_in[n_nodes][dim] with (u - 0.5)/dim, u = (word >> 8) * 2^-24 drawn
+ * with tag 4, and d_w_out[n_nodes][dim] with zeros (either may be NULL to
+ * skip it).  Row-major fp32, rows contiguous.
+ */
+GS_API gs_status gs_init_embeddings(float *d_w_in, float *d_w_out, int64_t n_nodes,
+                             int32_t dim, uint64_t seed, void *stream);
+
+/* ---------------------------------------------------------------- walks */
+/*
+ * DeepWalk walks (Section 2.2: "random walks from each node").
+ *   d_starts     : n_walks start nodes, or NULL for start = walk id mod n_nodes
+ *   walk id      : walk_id_base + index; selects the random stream
+ *   walk_len     : number of NODES per walk (Section 3.2 counts a batch as
+ *                  B x walk_len nodes, sources included); >= 1
+ *   d_walks_out  : [n_walks][walk_len] int32, walk-major.  A walk that reaches
+ *                  a node without out-edges stops; remaining entries are -1.
+ *   d_steps      : if not NULL, the number of transitions taken is ADDED to it.
+ * Transition t: next = cols[off[cur] + ((word0 * deg) >> 32)], tag 1.
+ */
+GS_API gs_status gs_random_walks(const gs_graph *g, const int32_t *d_starts,
+                          int64_t n_walks, int64_t walk_id_base, int32_t walk_len,
+                          uint64_t seed, int32_t *d_walks_out,
+                          uint64_t *d_steps, void *stream);
+
+/*
+ * node2vec walks (Section 2.2: "biased random walk to balance between
+ * breadth-first and depth-first traversals"; Grover & Leskovec 2016).  After
+ * the move prev -> cur, neighbour x of cur has weight 1/p if x = prev, 1 if x
+ * is a neighbour of prev, 1/q otherwise.  Sampled by rejection with tag 2:
+ * round s proposes x = cols[off[cur] + ((word0 * deg) >> 32)] and accepts iff
+ * word1 < floor(weight / max(1/p, 1, 1/q) * 2^32).  The first transition is
+ * uniform (round 0, word 0).  If max_rounds rounds reject, the last proposal
+ * is taken and *d_cap_hits (nullable) is incremented.  Needs a graph loaded
+ * with GS_REQUIRE_SORTED (GS_ERR_UNSORTED_ADJ otherwise); p, q > 0;
+ * 1 <= max_rounds <= 65536.
+ */
+GS_API gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts,
+                            int64_t n_walks, int64_t walk_id_base, int32_t walk_len,
+                            uint64_t seed, double p, double q, int32_t max_rounds,
+                            int32_t *d_walks_out, uint64_t *d_steps,
+                            uint64_t *d_cap_hits, void *stream);
+
+/* ---------------------------------------------------------------- SGNS */
+#define GS_DETERMINISTIC  0   /* synchronous mini-batch step, bitwise reproducible */
+#define GS_HOGWILD        1   /* lock-free: plain loads and stores, rows may race   */
+#define GS_HOGWILD_RED    2   /* lock-free: increments sent as reductions (no lost  */
+                              /* updates, gradients may still be stale)             */
+
+/*
+ * One SGNS update over a batch of walks.
+ *
+ * Pairs: for position i of a walk and j with 0 < |i-j| <= window inside the
+ * walk, both entries >= 0: center = walk[i], context = walk[j], slot
+ * sigma = j - i + window - (j > i) in [0, 2*window).
+ * Negatives: n_neg draws per pair from d_alias (n_nodes packed entries, see
+ * gs_build_alias), tag 3, block m gives draws 2m and 2m+1 from words (0,1)
+ * and (2,3).  A negative equal to the pair's context is masked (no term).
+ * Objective per pair: softplus(-<u_c, v_o>) + sum_k softplus(<u_c, v_nk>),
+ * u rows of d_w_in, v rows of d_w_out; g = sigmoid(f) - label.
+ *
+ * GS_DETERMINISTIC: every gradient uses the tables as they are on entry;
+ * increments are grouped by destination row, summed in a fixed order without
+ * atomics and applied once: U -= lr * GU, V -= lr * GV (sum over pairs, not
+ * mean).  Two runs give identical bits.  Scratch grows with
+ * n_walks * walk_len * 2 * window * (1 + n_neg) (20 bytes per slot);
+ * GS_ERR_UNSUPPORTED beyond 2^30 slots.
+ * GS_HOGWILD / GS_HOGWILD_RED: one warp per walk runs positions in order;
+ * per position the center row is read once, every target row is read,
+ * updated from the current center row and written back at once, and the
+ * center row receives its accumulated increment after the last pair.
+ * Results depend on scheduling.
+ *
+ *   d_w_in, d_w_out : [n_nodes][dim] fp32 row-major, 16-byte aligned,
+ *                     dim in {32, 64, 128, 256}
+ *   d_walks         : [n_walks][walk_len] int32 (as written by the walk calls)
+ *   d_loss_sum      : the batch's summed loss is ADDED (nullable)
+ *   d_pair_count    : the number of pairs is ADDED (nullable)
+ *   d_pairs_dump    : nullable; [n_walks][walk_len][2*window][2] int32
+ *                     (center, context) or (-1,-1) where no pair exists
+ *   d_negs_dump     : nullable; [n_walks][walk_len][2*window][n_neg] int32, the
+ *                     drawn ids (masked ones included), -1 where no pair exists
+ * Limits: 1 <= window <= 32, 0 <= n_neg <= 32, 1 <= walk_len <= 1024,
+ * 2*window*(1+n_neg) <= 512.
+ */
+GS_API gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t dim,
+                       const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                       int32_t walk_len, int32_t window, int32_t n_neg,
+                       const uint64_t *d_alias, float lr, uint64_t seed, int32_t mode,
+                       double *d_loss_sum, int64_t *d_pair_count,
+                       int32_t *d_pairs_dump, int32_t *d_negs_dump, void *stream);
+
+#define GS_WALK_UNIFORM   0
+#define GS_WALK_NODE2VEC  1
+#define GS_LR_CONSTANT    0
+#define GS_LR_LINEAR      1   /* lr_b = lr0 * max(1 - b / total_batches, 1e-4) */
+
+typedef struct gs_sgns_config {
+    int32_t dim;
+    int32_t walks_per_node;   /* walk ids are rep * n_nodes + v, start node v   */
+    int32_t walk_len;
+    int32_t window;
+    int32_t n_neg;
+    int32_t walk_kind;        /* GS_WALK_*                                       */
+    int32_t lr_schedule;      /* GS_LR_*                                         */
+    int32_t mode;             /* GS_DETERMINISTIC | GS_HOGWILD | GS_HOGWILD_RED  */
+    int32_t max_rounds;       /* node2vec rejection cap                          */
+    int32_t reserved;
+    double  p, q;             /* node2vec parameters                             */
+    double  lr0;
+    int64_t batch_walks;      /* walks per mini-batch (512 in the paper's runs)  */
+    int64_t first_batch;      /* resume point; batches are numbered over the     */
+    int64_t num_batches;      /* whole epoch; <= 0 means "to the end"            */
+    uint64_t seed;
+} gs_sgns_config;
+
+typedef struct gs_epoch_stats {
+    double  loss_sum;         /* sum of per-pair losses, each at its batch start */
+    int64_t pairs;
+    int64_t steps;            /* walk transitions taken                          */
+    int64_t cap_hits;         /* node2vec rejection cap hits                     */
+    int64_t batches;
+    float   ms_walk;          /* device time of the walk kernels                 */
+    float   ms_sgns;          /* device time of the SGNS kernels                 */
+    float   ms_total;
+} gs_epoch_stats;
+
+/*
+ * One pass (or a range of mini-batches of one pass) over all walks: for batch
+ * b = walk ids [b*batch_walks, (b+1)*batch_walks): generate the walks, then
+ * one gs_sgns_step with lr_b (the paper's loop: sample, fetch rows, compute,
+ * write back, barrier - Section 3.2).  Walk generation of batch b+1 overlaps
+ * the SGNS step of batch b on a second stream.  WAITS for completion and
+ * fills *h_out (host struct).  Epoch defaults of the paper: batch 512.
+ */
+GS_API gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias,
+                        float *d_w_in, float *d_w_out, const gs_sgns_config *cfg,
+                        gs_epoch_stats *h_out, void *stream);
+
+/* Frees the cached scratch memory of the current device (waits for the device). */
+GS_API gs_status gs_release_workspace(void);
+
+/*
+ * Tuning knob: lanes that cooperate on one node2vec walk (1, 2, 4, 8 or 32;
+ * default 4).  Lane k of a group evaluates rejection round base + k and the
+ * first accepted round wins, so walks do not depend on this setting.
+ */
+GS_API gs_status gs_tune_node2vec_group(int32_t lanes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GS_H */

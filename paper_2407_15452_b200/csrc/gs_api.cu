@@ -1,0 +1,531 @@
+// C ABI entry points (see include/gs.h): argument checks, the graph handle,
+// the host-side alias-table builder, the cached scratch memory and the epoch
+// driver.  Kernels live in gs_walks.cu, gs_sgns.cu and gs_sort.cu.
+#include <math.h>
+#include <stdarg.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "gs_common.cuh"
+
+namespace gs {
+
+// ---- implemented in the kernel files ------------------------------------------
+gs_status validate_csr(const gs_graph *g, bool check_sorted, cudaStream_t st, int64_t *bad_row,
+                       int64_t *unsorted_row, int64_t *max_degree, bool *ends_bad);
+gs_status init_embeddings(float *w_in, float *w_out, int64_t n, int32_t dim, uint64_t seed,
+                          cudaStream_t st);
+gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
+                               int64_t base, int32_t L, uint64_t seed, int32_t *walks,
+                               unsigned long long *steps, cudaStream_t st);
+gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
+                                int64_t base, int32_t L, uint64_t seed, double p, double q,
+                                int32_t max_rounds, int group, int32_t *walks,
+                                unsigned long long *steps, unsigned long long *caps,
+                                cudaStream_t st);
+gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                    int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                    const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
+                    int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st);
+
+// ---- errors ----------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+gs_status cuda_fail(cudaError_t e, const char *what)
+{
+    set_error("CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
+    return GS_ERR_CUDA;
+}
+
+static gs_status invalid(const char *msg)
+{
+    set_error("invalid argument: %s", msg);
+    return GS_ERR_INVALID_ARG;
+}
+
+// ---- per-device state ----------------------------------------------------------------
+struct DeviceState {
+    void *ws[WS_SLOTS] = { nullptr, nullptr, nullptr, nullptr };
+    size_t ws_bytes[WS_SLOTS] = { 0, 0, 0, 0 };
+    int sms = 0;
+};
+static std::mutex g_mu;
+static DeviceState g_dev[64];
+
+static DeviceState *current_state()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    return &g_dev[dev];
+}
+
+int sm_count()
+{
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceState *d = current_state();
+    if (!d) return 148;
+    if (d->sms == 0) {
+        int dev = 0, n = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+        d->sms = n;
+    }
+    return d->sms;
+}
+
+gs_status workspace_get(int slot, size_t bytes, void **out)
+{
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceState *d = current_state();
+    if (!d) { set_error("no current CUDA device"); return GS_ERR_CUDA; }
+    if (d->ws_bytes[slot] < bytes) {
+        if (d->ws[slot]) {
+            cudaError_t e = cudaFree(d->ws[slot]);       // waits for work that may still use it
+            d->ws[slot] = nullptr;
+            d->ws_bytes[slot] = 0;
+            if (e != cudaSuccess) return cuda_fail(e, "cudaFree(scratch)");
+        }
+        size_t want = bytes + bytes / 4;                  // head room against regrowth
+        want = (want + 255) & ~(size_t)255;
+        void *p = nullptr;
+        cudaError_t e = cudaMalloc(&p, want);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            set_error("scratch allocation of %zu bytes failed: %s", want, cudaGetErrorString(e));
+            return GS_ERR_OOM;
+        }
+        d->ws[slot] = p;
+        d->ws_bytes[slot] = want;
+    }
+    *out = d->ws[slot];
+    return GS_OK;
+}
+
+static bool dim_ok(int32_t dim) { return dim == 32 || dim == 64 || dim == 128 || dim == 256; }
+
+}  // namespace gs
+
+using namespace gs;
+
+extern "C" {
+
+const char *gs_last_error(void) { return g_err; }
+
+gs_status gs_release_workspace(void)
+{
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceState *d = current_state();
+    if (!d) return GS_OK;
+    for (int s = 0; s < WS_SLOTS; ++s) {
+        if (d->ws[s]) {
+            cudaError_t e = cudaFree(d->ws[s]);
+            d->ws[s] = nullptr;
+            d->ws_bytes[s] = 0;
+            if (e != cudaSuccess) return cuda_fail(e, "cudaFree(scratch)");
+        }
+    }
+    return GS_OK;
+}
+
+// ------------------------------------------------------------------ graph
+gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offsets,
+                            int32_t offsets_are_64bit, const int32_t *d_cols, uint32_t flags,
+                            void *stream, gs_graph **out)
+{
+    if (!out) return invalid("out is NULL");
+    *out = nullptr;
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
+    if (n_edges < 0) return invalid("n_edges < 0");
+    if (!d_offsets) return invalid("d_offsets is NULL");
+    if (n_edges > 0 && !d_cols) return invalid("d_cols is NULL");
+    if (!offsets_are_64bit && n_edges >= ((int64_t)1 << 31))
+        return invalid("int32 offsets cannot address 2^31 or more edges");
+    if (flags & ~(GS_VALIDATE | GS_REQUIRE_SORTED)) return invalid("unknown flag");
+    gs_graph *g = new (std::nothrow) gs_graph;
+    if (!g) { set_error("out of host memory"); return GS_ERR_OOM; }
+    g->n_nodes = n_nodes;
+    g->n_edges = n_edges;
+    g->d_offsets = d_offsets;
+    g->d_cols = d_cols;
+    g->offsets64 = offsets_are_64bit ? 1 : 0;
+    g->sorted = 0;
+    g->max_degree = -1;
+    g->device = 0;
+    cudaGetDevice(&g->device);
+    if (flags & (GS_VALIDATE | GS_REQUIRE_SORTED)) {
+        int64_t bad = -1, unsorted = -1, maxdeg = 0;
+        bool ends_bad = false;
+        const bool want_sorted = (flags & GS_REQUIRE_SORTED) != 0;
+        gs_status s = validate_csr(g, want_sorted, (cudaStream_t)stream, &bad, &unsorted, &maxdeg,
+                                   &ends_bad);
+        if (s != GS_OK) { delete g; return s; }
+        if (ends_bad) {
+            delete g;
+            set_error("bad CSR: offsets[0] must be 0 and offsets[n_nodes] must equal n_edges");
+            return GS_ERR_BAD_CSR;
+        }
+        if (bad >= 0) {
+            delete g;
+            set_error("bad CSR: row %lld has decreasing/out-of-range offsets or a column outside [0, n_nodes)",
+                      (long long)bad);
+            return GS_ERR_BAD_CSR;
+        }
+        if (unsorted >= 0) {
+            delete g;
+            set_error("row %lld is not strictly increasing", (long long)unsorted);
+            return GS_ERR_UNSORTED_ADJ;
+        }
+        g->max_degree = maxdeg;
+        g->sorted = want_sorted ? 1 : 0;
+    }
+    *out = g;
+    return GS_OK;
+}
+
+void gs_graph_free(gs_graph *g) { delete g; }
+
+gs_status gs_graph_info(const gs_graph *g, int64_t *n_nodes, int64_t *n_edges, int64_t *max_degree,
+                        int32_t *rows_sorted)
+{
+    if (!g) return invalid("graph is NULL");
+    if (n_nodes) *n_nodes = g->n_nodes;
+    if (n_edges) *n_edges = g->n_edges;
+    if (max_degree) *max_degree = g->max_degree;
+    if (rows_sorted) *rows_sorted = g->sorted;
+    return GS_OK;
+}
+
+// ------------------------------------------------------------------ alias table (host)
+gs_status gs_build_alias(const double *h_weights, int64_t n, double power, uint64_t *h_table_out)
+{
+    if (!h_weights || !h_table_out) return invalid("null pointer");
+    if (n <= 0 || n >= ((int64_t)1 << 31)) return invalid("n must be in [1, 2^31)");
+    std::vector<double> mass;
+    std::vector<int64_t> lo_q, hi_q;
+    try {
+        mass.resize((size_t)n);
+        lo_q.resize((size_t)n);
+        hi_q.resize((size_t)n);
+    } catch (const std::bad_alloc &) {
+        set_error("out of host memory building the alias table");
+        return GS_ERR_OOM;
+    }
+    double total = 0.0;
+    for (int64_t v = 0; v < n; ++v) {
+        const double x = h_weights[v];
+        if (!(x >= 0.0) || !isfinite(x)) return invalid("weights must be finite and >= 0");
+        mass[v] = x > 0.0 ? pow(x, power) : 0.0;
+        total += mass[v];
+    }
+    if (!(total > 0.0)) return invalid("no positive weight");
+    // cells scaled so that the average cell holds mass 1; under-full cells queue in lo_q,
+    // the others in hi_q, both in increasing node order
+    int64_t lo_head = 0, lo_tail = 0, hi_head = 0, hi_tail = 0;
+    for (int64_t v = 0; v < n; ++v) {
+        mass[v] = mass[v] * (double)n / total;
+        if (mass[v] < 1.0) lo_q[lo_tail++] = v; else hi_q[hi_tail++] = v;
+        h_table_out[v] = ((uint64_t)(uint32_t)v << 32) | 0xFFFFFFFFull;   // keep whole cell
+    }
+    while (lo_head < lo_tail && hi_head < hi_tail) {
+        const int64_t under = lo_q[lo_head++];
+        const int64_t donor = hi_q[hi_head];
+        const double keep = floor(mass[under] * 4294967296.0);
+        const uint32_t thr = keep >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)keep;
+        h_table_out[under] = ((uint64_t)(uint32_t)donor << 32) | (uint64_t)thr;
+        mass[donor] = (mass[donor] + mass[under]) - 1.0;
+        if (mass[donor] < 1.0) { ++hi_head; lo_q[lo_tail++] = donor; }
+    }
+    return GS_OK;
+}
+
+// ------------------------------------------------------------------ tables
+gs_status gs_init_embeddings(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t dim,
+                             uint64_t seed, void *stream)
+{
+    if (n_nodes < 0) return invalid("n_nodes < 0");
+    if (!dim_ok(dim)) { set_error("dim %d not supported (32, 64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
+    return init_embeddings(d_w_in, d_w_out, n_nodes, dim, seed, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------ walks
+static gs_status check_walk_args(const gs_graph *g, int64_t n_walks, int64_t base, int32_t L,
+                                 const int32_t *out)
+{
+    if (!g) return invalid("graph is NULL");
+    if (n_walks < 0 || base < 0) return invalid("negative n_walks or walk_id_base");
+    if (L < 1 || L > 1024) { set_error("walk_len %d outside [1, 1024]", L); return GS_ERR_UNSUPPORTED; }
+    if (n_walks > 0 && !out) return invalid("d_walks_out is NULL");
+    return GS_OK;
+}
+
+gs_status gs_random_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_walks,
+                          int64_t walk_id_base, int32_t walk_len, uint64_t seed,
+                          int32_t *d_walks_out, uint64_t *d_steps, void *stream)
+{
+    gs_status s = check_walk_args(g, n_walks, walk_id_base, walk_len, d_walks_out);
+    if (s != GS_OK) return s;
+    return launch_uniform_walks(g, d_starts, n_walks, walk_id_base, walk_len, seed, d_walks_out,
+                                (unsigned long long *)d_steps, (cudaStream_t)stream);
+}
+
+static int g_n2v_group = 4;   // lanes per walk in the node2vec sampler
+
+gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_walks,
+                            int64_t walk_id_base, int32_t walk_len, uint64_t seed, double p,
+                            double q, int32_t max_rounds, int32_t *d_walks_out, uint64_t *d_steps,
+                            uint64_t *d_cap_hits, void *stream)
+{
+    gs_status s = check_walk_args(g, n_walks, walk_id_base, walk_len, d_walks_out);
+    if (s != GS_OK) return s;
+    if (!(p > 0.0) || !(q > 0.0) || !isfinite(p) || !isfinite(q)) return invalid("p and q must be positive");
+    if (max_rounds < 1 || max_rounds > 65536) return invalid("max_rounds outside [1, 65536]");
+    if (!g->sorted) {
+        set_error("node2vec needs a graph loaded with GS_REQUIRE_SORTED");
+        return GS_ERR_UNSORTED_ADJ;
+    }
+    return launch_node2vec_walks(g, d_starts, n_walks, walk_id_base, walk_len, seed, p, q,
+                                 max_rounds, g_n2v_group, d_walks_out,
+                                 (unsigned long long *)d_steps, (unsigned long long *)d_cap_hits,
+                                 (cudaStream_t)stream);
+}
+
+// Tuning knob used by the benchmarks: lanes per walk (1, 2, 4, 8, 32) of the node2vec sampler.
+// Results do not depend on it.
+gs_status gs_tune_node2vec_group(int32_t lanes)
+{
+    if (lanes != 1 && lanes != 2 && lanes != 4 && lanes != 8 && lanes != 32)
+        return invalid("lanes per walk must be 1, 2, 4, 8 or 32");
+    g_n2v_group = lanes;
+    return GS_OK;
+}
+
+// ------------------------------------------------------------------ SGNS
+static gs_status check_sgns_shape(int32_t dim, int32_t L, int32_t w, int32_t K, int32_t mode)
+{
+    if (!dim_ok(dim)) { set_error("dim %d not supported (32, 64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
+    if (L < 1 || L > 1024) { set_error("walk_len %d outside [1, 1024]", L); return GS_ERR_UNSUPPORTED; }
+    if (w < 1 || w > 32) { set_error("window %d outside [1, 32]", w); return GS_ERR_UNSUPPORTED; }
+    if (K < 0 || K > 32) { set_error("n_neg %d outside [0, 32]", K); return GS_ERR_UNSUPPORTED; }
+    if (2 * w * (1 + K) > 512) { set_error("2*window*(1+n_neg) = %d exceeds 512", 2 * w * (1 + K)); return GS_ERR_UNSUPPORTED; }
+    if (mode != GS_DETERMINISTIC && mode != GS_HOGWILD && mode != GS_HOGWILD_RED) return invalid("unknown mode");
+    return GS_OK;
+}
+
+gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t dim,
+                       const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                       int32_t walk_len, int32_t window, int32_t n_neg, const uint64_t *d_alias,
+                       float lr, uint64_t seed, int32_t mode, double *d_loss_sum,
+                       int64_t *d_pair_count, int32_t *d_pairs_dump, int32_t *d_negs_dump,
+                       void *stream)
+{
+    if (!d_w_in || !d_w_out) return invalid("table pointer is NULL");
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
+    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
+    if (n_walks > 0 && !d_walks) return invalid("d_walks is NULL");
+    gs_status s = check_sgns_shape(dim, walk_len, window, n_neg, mode);
+    if (s != GS_OK) return s;
+    if (n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
+    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out) & 15) return invalid("tables must be 16-byte aligned");
+    return sgns_step(d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len,
+                     window, n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count,
+                     d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------ epoch driver
+struct EpochCounters {
+    double loss;
+    long long pairs;
+    unsigned long long steps;
+    unsigned long long caps;
+};
+
+namespace {
+// A small ring of event pairs that accumulates device time of one kind of work.
+struct TimerRing {
+    static const int N = 8;
+    cudaEvent_t beg[N], end[N];
+    bool used[N];
+    int next = 0;
+    double total_ms = 0.0;
+    bool ok = false;
+    bool init()
+    {
+        for (int i = 0; i < N; ++i) {
+            used[i] = false;
+            if (cudaEventCreate(&beg[i]) != cudaSuccess || cudaEventCreate(&end[i]) != cudaSuccess)
+                return false;
+        }
+        ok = true;
+        return true;
+    }
+    void collect(int i)
+    {
+        if (!used[i]) return;
+        float ms = 0.f;
+        if (cudaEventSynchronize(end[i]) == cudaSuccess &&
+            cudaEventElapsedTime(&ms, beg[i], end[i]) == cudaSuccess)
+            total_ms += ms;
+        used[i] = false;
+    }
+    int start(cudaStream_t st)
+    {
+        const int i = next;
+        next = (next + 1) % N;
+        collect(i);
+        cudaEventRecord(beg[i], st);
+        return i;
+    }
+    void stop(int i, cudaStream_t st) { cudaEventRecord(end[i], st); used[i] = true; }
+    void finish() { for (int i = 0; i < N; ++i) collect(i); }
+    void destroy()
+    {
+        if (!ok) return;
+        for (int i = 0; i < N; ++i) { cudaEventDestroy(beg[i]); cudaEventDestroy(end[i]); }
+    }
+};
+}  // namespace
+
+gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, float *d_w_in, float *d_w_out,
+                        const gs_sgns_config *cfg, gs_epoch_stats *h_out, void *stream)
+{
+    if (!g || !cfg || !h_out) return invalid("null pointer");
+    if (!d_w_in || !d_w_out) return invalid("table pointer is NULL");
+    gs_status s = check_sgns_shape(cfg->dim, cfg->walk_len, cfg->window, cfg->n_neg, cfg->mode);
+    if (s != GS_OK) return s;
+    if (cfg->n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
+    if (cfg->walks_per_node < 1 || cfg->batch_walks < 1) return invalid("walks_per_node and batch_walks must be >= 1");
+    if (cfg->walk_kind != GS_WALK_UNIFORM && cfg->walk_kind != GS_WALK_NODE2VEC) return invalid("unknown walk_kind");
+    if (cfg->lr_schedule != GS_LR_CONSTANT && cfg->lr_schedule != GS_LR_LINEAR) return invalid("unknown lr_schedule");
+    if (cfg->first_batch < 0) return invalid("first_batch < 0");
+    if (cfg->walk_kind == GS_WALK_NODE2VEC) {
+        if (!g->sorted) { set_error("node2vec needs a graph loaded with GS_REQUIRE_SORTED"); return GS_ERR_UNSORTED_ADJ; }
+        if (!(cfg->p > 0.0) || !(cfg->q > 0.0)) return invalid("p and q must be positive");
+        if (cfg->max_rounds < 1 || cfg->max_rounds > 65536) return invalid("max_rounds outside [1, 65536]");
+    }
+    memset(h_out, 0, sizeof(*h_out));
+    const int64_t total_walks = g->n_nodes * (int64_t)cfg->walks_per_node;
+    const int64_t nb_total = (total_walks + cfg->batch_walks - 1) / cfg->batch_walks;
+    int64_t b_end = cfg->num_batches > 0 ? cfg->first_batch + cfg->num_batches : nb_total;
+    if (b_end > nb_total) b_end = nb_total;
+    if (cfg->first_batch >= b_end) return GS_OK;
+
+    cudaStream_t s_sgns = (cudaStream_t)stream;
+    cudaStream_t s_walk = nullptr;
+    cudaEvent_t ev_walk[2] = { nullptr, nullptr }, ev_sgns[2] = { nullptr, nullptr };
+    cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
+    TimerRing t_walk, t_sgns;
+    gs_status rc = GS_OK;
+    int32_t *wbuf[2] = { nullptr, nullptr };
+    EpochCounters *ctr = nullptr;
+    EpochCounters host_ctr;
+    memset(&host_ctr, 0, sizeof(host_ctr));
+
+#define EP_TRY(expr)                                                   \
+    do {                                                               \
+        cudaError_t _e = (expr);                                       \
+        if (_e != cudaSuccess) { rc = cuda_fail(_e, #expr); goto done; } \
+    } while (0)
+#define EP_CALL(expr)                                                  \
+    do { rc = (expr); if (rc != GS_OK) goto done; } while (0)
+
+    {
+        const size_t wbytes = sizeof(int32_t) * (size_t)cfg->batch_walks * (size_t)cfg->walk_len;
+        void *p = nullptr;
+        EP_CALL(workspace_get(WS_WALKS0, wbytes, &p)); wbuf[0] = (int32_t *)p;
+        EP_CALL(workspace_get(WS_WALKS1, wbytes, &p)); wbuf[1] = (int32_t *)p;
+        EP_CALL(workspace_get(WS_COUNTERS, 256, &p)); ctr = (EpochCounters *)p;
+    }
+    EP_TRY(cudaStreamCreateWithFlags(&s_walk, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+        EP_TRY(cudaEventCreateWithFlags(&ev_walk[i], cudaEventDisableTiming));
+        EP_TRY(cudaEventCreateWithFlags(&ev_sgns[i], cudaEventDisableTiming));
+    }
+    EP_TRY(cudaEventCreate(&ev_begin));
+    EP_TRY(cudaEventCreate(&ev_end));
+    if (!t_walk.init() || !t_sgns.init()) { rc = cuda_fail(cudaGetLastError(), "cudaEventCreate"); goto done; }
+
+    EP_TRY(cudaMemsetAsync(ctr, 0, sizeof(EpochCounters), s_sgns));
+    EP_TRY(cudaEventRecord(ev_begin, s_sgns));
+    EP_TRY(cudaStreamWaitEvent(s_walk, ev_begin, 0));        // the walk stream starts after prior work
+
+    for (int64_t b = cfg->first_batch; b < b_end; ++b) {
+        const int buf = (int)((b - cfg->first_batch) & 1);
+        const int64_t base = b * cfg->batch_walks;
+        const int64_t n = (base + cfg->batch_walks <= total_walks) ? cfg->batch_walks : total_walks - base;
+        // this walk buffer was last read by the SGNS step two batches ago
+        if (b - cfg->first_batch >= 2) EP_TRY(cudaStreamWaitEvent(s_walk, ev_sgns[buf], 0));
+        {
+            const int tk = t_walk.start(s_walk);
+            if (cfg->walk_kind == GS_WALK_UNIFORM)
+                EP_CALL(launch_uniform_walks(g, nullptr, n, base, cfg->walk_len, cfg->seed, wbuf[buf],
+                                             &ctr->steps, s_walk));
+            else
+                EP_CALL(launch_node2vec_walks(g, nullptr, n, base, cfg->walk_len, cfg->seed, cfg->p,
+                                              cfg->q, cfg->max_rounds, g_n2v_group, wbuf[buf],
+                                              &ctr->steps, &ctr->caps, s_walk));
+            t_walk.stop(tk, s_walk);
+        }
+        EP_TRY(cudaEventRecord(ev_walk[buf], s_walk));
+        EP_TRY(cudaStreamWaitEvent(s_sgns, ev_walk[buf], 0));
+        {
+            double lr = cfg->lr0;
+            if (cfg->lr_schedule == GS_LR_LINEAR) {
+                double f = 1.0 - (double)b / (double)nb_total;
+                lr = cfg->lr0 * (f > 1e-4 ? f : 1e-4);
+            }
+            const int tk = t_sgns.start(s_sgns);
+            EP_CALL(sgns_step(d_w_in, d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n, base, cfg->walk_len,
+                              cfg->window, cfg->n_neg, d_alias, (float)lr, cfg->seed, cfg->mode,
+                              &ctr->loss, (int64_t *)&ctr->pairs, nullptr, nullptr, s_sgns));
+            t_sgns.stop(tk, s_sgns);
+        }
+        EP_TRY(cudaEventRecord(ev_sgns[buf], s_sgns));
+        ++h_out->batches;
+    }
+    EP_TRY(cudaEventRecord(ev_end, s_sgns));
+    EP_TRY(cudaMemcpyAsync(&host_ctr, ctr, sizeof(host_ctr), cudaMemcpyDeviceToHost, s_sgns));
+    EP_TRY(cudaStreamSynchronize(s_sgns));
+    EP_TRY(cudaStreamSynchronize(s_walk));
+    t_walk.finish();
+    t_sgns.finish();
+    h_out->loss_sum = host_ctr.loss;
+    h_out->pairs = (int64_t)host_ctr.pairs;
+    h_out->steps = (int64_t)host_ctr.steps;
+    h_out->cap_hits = (int64_t)host_ctr.caps;
+    h_out->ms_walk = (float)t_walk.total_ms;
+    h_out->ms_sgns = (float)t_sgns.total_ms;
+    EP_TRY(cudaEventElapsedTime(&h_out->ms_total, ev_begin, ev_end));
+
+done:
+    if (rc != GS_OK) {                       // let queued work drain before buffers are reused
+        if (s_walk) cudaStreamSynchronize(s_walk);
+        cudaStreamSynchronize(s_sgns);
+    }
+    t_walk.destroy();
+    t_sgns.destroy();
+    for (int i = 0; i < 2; ++i) {
+        if (ev_walk[i]) cudaEventDestroy(ev_walk[i]);
+        if (ev_sgns[i]) cudaEventDestroy(ev_sgns[i]);
+    }
+    if (ev_begin) cudaEventDestroy(ev_begin);
+    if (ev_end) cudaEventDestroy(ev_end);
+    if (s_walk) cudaStreamDestroy(s_walk);
+#undef EP_TRY
+#undef EP_CALL
+    return rc;
+}
+
+}  // extern "C"

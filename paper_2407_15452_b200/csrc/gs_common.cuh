@@ -1,0 +1,80 @@
+// Shared device/host helpers of the CUDA library: status plumbing, the Philox
+// block function and the counter layout that gs.h documents.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "gs.h"
+
+namespace gs {
+
+// ---- error plumbing ------------------------------------------------------
+void set_error(const char *fmt, ...);
+gs_status cuda_fail(cudaError_t e, const char *what);
+
+#define GS_CUDA_TRY(expr)                                              \
+    do {                                                               \
+        cudaError_t _e = (expr);                                       \
+        if (_e != cudaSuccess) return ::gs::cuda_fail(_e, #expr);      \
+    } while (0)
+
+// ---- per-device scratch (grow-only, cached) --------------------------------
+// Returns a 256-byte aligned scratch block of at least `bytes` for slot `slot`
+// (independent blocks so that kernels on different streams do not share one).
+gs_status workspace_get(int slot, size_t bytes, void **out);
+enum { WS_WALKS0 = 0, WS_WALKS1 = 1, WS_SGNS = 2, WS_COUNTERS = 3, WS_SLOTS = 4 };
+
+int sm_count();
+
+// ---- graph handle --------------------------------------------------------------
+}  // namespace gs
+
+struct gs_graph {
+    int64_t n_nodes;
+    int64_t n_edges;
+    const void *d_offsets;
+    const int32_t *d_cols;
+    int32_t offsets64;
+    int32_t sorted;       // rows verified strictly increasing
+    int64_t max_degree;   // -1 when not validated
+    int device;
+};
+
+namespace gs {
+
+// ---- Philox4x32-10 ---------------------------------------------------------------
+enum : uint32_t { TAG_UNIFORM = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4 };
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x);
+        const uint32_t lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z);
+        const uint32_t lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+        k.x += 0x9E3779B9u;
+        k.y += 0xBB67AE85u;
+    }
+    return c;
+}
+
+// counter = (id low, id high, step, tag << 24 | sub), key = seed
+__device__ __forceinline__ uint4 draw(uint64_t seed, uint64_t id, uint32_t step,
+                                      uint32_t tag, uint32_t sub)
+{
+    return philox4x32_10(make_uint4((uint32_t)id, (uint32_t)(id >> 32), step, (tag << 24) | sub),
+                         make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)));
+}
+
+// CSR offset of node v for either offset width
+template <typename OffT>
+__device__ __forceinline__ int64_t load_off(const OffT *off, int64_t v)
+{
+    return (int64_t)__ldg(off + v);
+}
+
+}  // namespace gs

@@ -1,0 +1,611 @@
+// Skip-gram-with-negative-sampling update kernels.
+//
+// A row of an embedding table is dim fp32 values; a warp holds one row as
+// FPL = dim/32 values per lane (16-byte vector accesses for dim >= 128), so a
+// row read or write is one fully coalesced request.  Dot products are
+// butterfly shuffles.  The path is bound by row traffic in HBM/L2, not by
+// arithmetic, so there is no tensor-core work here.
+//
+// Lock-free mode: one warp per walk, positions in order.  For each position
+// the center row sits in registers, the targets of all its pairs (context +
+// negatives, slot by slot) are listed in shared memory, and the list is
+// consumed in chunks of TCH rows whose loads are all in flight together.
+//
+// Synchronous mode: one warp per position computes the coefficients g and the
+// center-row gradient from the entry tables and emits one (destination row,
+// contribution index) key per target; the keys are radix-sorted, and one warp
+// per distinct row sums that row's contributions in index order and writes the
+// row once.  No floating-point atomics anywhere on this path.
+#include "gs_common.cuh"
+
+namespace gs {
+
+int radix_sort_pairs(uint32_t *keysA, uint32_t *valsA, uint32_t *keysB, uint32_t *valsB,
+                     uint32_t n, int bits, uint32_t *counts, cudaStream_t st,
+                     uint32_t **keys_sorted, uint32_t **vals_sorted);
+size_t sort_counts_bytes(uint32_t n);
+
+constexpr int TCH = 6;            // target rows in flight per warp
+constexpr int SGNS_WARPS = 4;     // warps per block
+
+// ---------------------------------------------------------------- row vectors
+template <int FPL> struct Row { float v[FPL]; };
+
+template <int FPL>
+__device__ __forceinline__ Row<FPL> row_load(const float *__restrict__ tab, int64_t r, int lane)
+{
+    Row<FPL> out;
+    const float *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 1) {
+        out.v[0] = p[lane];
+    } else if constexpr (FPL == 2) {
+        const float2 t = reinterpret_cast<const float2 *>(p)[lane];
+        out.v[0] = t.x; out.v[1] = t.y;
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q) {
+            const float4 t = reinterpret_cast<const float4 *>(p)[q * 32 + lane];
+            out.v[4 * q] = t.x; out.v[4 * q + 1] = t.y; out.v[4 * q + 2] = t.z; out.v[4 * q + 3] = t.w;
+        }
+    }
+    return out;
+}
+
+template <int FPL>
+__device__ __forceinline__ void row_store(float *__restrict__ tab, int64_t r, int lane,
+                                          const Row<FPL> &x)
+{
+    float *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 1) {
+        p[lane] = x.v[0];
+    } else if constexpr (FPL == 2) {
+        reinterpret_cast<float2 *>(p)[lane] = make_float2(x.v[0], x.v[1]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q)
+            reinterpret_cast<float4 *>(p)[q * 32 + lane] =
+                make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]);
+    }
+}
+
+// row += x, sent as reductions (no value returned)
+template <int FPL>
+__device__ __forceinline__ void row_red_add(float *__restrict__ tab, int64_t r, int lane,
+                                            const Row<FPL> &x)
+{
+    float *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 1) {
+        atomicAdd(p + lane, x.v[0]);
+    } else if constexpr (FPL == 2) {
+        atomicAdd(reinterpret_cast<float2 *>(p) + lane, make_float2(x.v[0], x.v[1]));
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q)
+            atomicAdd(reinterpret_cast<float4 *>(p) + q * 32 + lane,
+                      make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
+    }
+}
+
+template <int FPL>
+__device__ __forceinline__ float row_dot(const Row<FPL> &a, const Row<FPL> &b)
+{
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < FPL; ++j) s = fmaf(a.v[j], b.v[j], s);
+    return s;
+}
+
+__device__ __forceinline__ float warp_sum(float s)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return s;                       // identical bits on every lane (commutative pairs)
+}
+
+__device__ __forceinline__ float sigmoidf_exact(float x) { return 1.0f / (1.0f + expf(-x)); }
+__device__ __forceinline__ float softplusf(float x)
+{
+    return fmaxf(x, 0.f) + log1pf(expf(-fabsf(x)));
+}
+
+// ---------------------------------------------------------------- target list of one position
+// Slot layout: tgt[s * (1 + K) + 0] = context of slot s, tgt[s * (1 + K) + 1 + k] = negative k;
+// -1 where the pair does not exist or the negative equals the context (masked).
+// W points at the walk (global or shared), c = W[i] >= 0.  Returns the number of pairs
+// (identical on every lane).  dump_* (nullable) are this position's rows of the dump arrays.
+__device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_t i, int32_t w,
+                                             int32_t K, uint64_t seed, uint64_t id,
+                                             const uint64_t *__restrict__ alias, uint32_t n_alias,
+                                             int32_t c, int32_t *tgt, int lane,
+                                             int32_t *dump_pairs, int32_t *dump_negs)
+{
+    const int S = 2 * w, T1 = 1 + K;
+    const int hp = K > 0 ? (K + 1) / 2 : 1;          // Philox blocks per slot (>= 1 work item)
+    int pairs = 0;
+    __syncwarp();                                    // earlier readers of tgt are done
+    for (int it0 = 0; it0 < S * hp; it0 += 32) {
+        const int it = it0 + lane;
+        bool valid = false;
+        if (it < S * hp) {
+            const int s = it / hp, m = it - s * hp;
+            const int j = i - w + s + (s >= w ? 1 : 0);
+            const int32_t ctx = (j >= 0 && j < L) ? W[j] : -1;
+            valid = ctx >= 0;
+            if (m == 0) {
+                tgt[s * T1] = ctx;
+                if (dump_pairs) {
+                    dump_pairs[2 * s] = valid ? c : -1;
+                    dump_pairs[2 * s + 1] = ctx;
+                }
+            }
+            if (K > 0) {
+                int32_t n0 = -1, n1 = -1;
+                const bool two = 2 * m + 1 < K;
+                if (valid) {
+                    const uint4 r = draw(seed, id, (uint32_t)(i * S + s), TAG_NEGATIVE, (uint32_t)m);
+                    const uint32_t j0 = __umulhi(r.x, n_alias);
+                    const uint64_t e0 = __ldg(alias + j0);
+                    n0 = r.y < (uint32_t)e0 ? (int32_t)j0 : (int32_t)(e0 >> 32);
+                    if (two) {
+                        const uint32_t j1 = __umulhi(r.z, n_alias);
+                        const uint64_t e1 = __ldg(alias + j1);
+                        n1 = r.w < (uint32_t)e1 ? (int32_t)j1 : (int32_t)(e1 >> 32);
+                    }
+                }
+                if (dump_negs) {
+                    dump_negs[s * K + 2 * m] = n0;
+                    if (two) dump_negs[s * K + 2 * m + 1] = n1;
+                }
+                tgt[s * T1 + 1 + 2 * m] = (n0 == ctx) ? -1 : n0;
+                if (two) tgt[s * T1 + 2 + 2 * m] = (n1 == ctx) ? -1 : n1;
+            }
+            valid = valid && m == 0;
+        }
+        pairs += __popc(__ballot_sync(0xffffffffu, valid));
+    }
+    __syncwarp();
+    return pairs;
+}
+
+__device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int lane,
+                                                    int32_t *dump_pairs, int32_t *dump_negs)
+{
+    if (dump_pairs) for (int x = lane; x < 2 * S; x += 32) dump_pairs[x] = -1;
+    if (dump_negs) for (int x = lane; x < S * K; x += 32) dump_negs[x] = -1;
+}
+
+// ---------------------------------------------------------------- lock-free kernel
+template <int FPL, bool RED>
+__global__ void __launch_bounds__(SGNS_WARPS * 32)
+sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
+                    const int32_t *__restrict__ walks, int64_t n_walks, int64_t walk_id_base,
+                    int32_t L, int32_t w, int32_t K, const uint64_t *__restrict__ alias,
+                    uint32_t n_alias, float lr, uint64_t seed, double *loss_out,
+                    unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs)
+{
+    extern __shared__ int32_t smem[];
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    const int S = 2 * w, T1 = 1 + K, SL = S * T1;
+    int32_t *W = smem + wi * (L + SL);
+    int32_t *tgt = W + L;
+    const int64_t n_warps = (int64_t)gridDim.x * SGNS_WARPS;
+    double loss_acc = 0.0;
+    unsigned long long pair_acc = 0;
+
+    for (int64_t a = (int64_t)blockIdx.x * SGNS_WARPS + wi; a < n_walks; a += n_warps) {
+        const uint64_t id = (uint64_t)(walk_id_base + a);
+        __syncwarp();
+        for (int x = lane; x < L; x += 32) W[x] = walks[a * L + x];
+        __syncwarp();
+        for (int32_t i = 0; i < L; ++i) {
+            const int32_t c = W[i];
+            int32_t *dp = dump_pairs ? dump_pairs + ((a * L + i) * S) * 2 : nullptr;
+            int32_t *dn = dump_negs ? dump_negs + ((a * L + i) * S) * (int64_t)K : nullptr;
+            if (c < 0) { dump_empty_position(S, K, lane, dp, dn); continue; }
+            const int pairs = build_targets(W, L, i, w, K, seed, id, alias, n_alias, c, tgt, lane,
+                                            dp, dn);
+            if (pairs == 0) continue;
+            pair_acc += (unsigned long long)pairs;
+            const Row<FPL> u = row_load<FPL>(w_in, c, lane);
+            Row<FPL> acc;
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+            float loss = 0.f;
+            int kk = 0;                                  // (base + k) mod T1, tracked incrementally
+            for (int base = 0; base < SL; base += TCH) {
+                int32_t ids[TCH];
+                bool any = false;
+#pragma unroll
+                for (int k = 0; k < TCH; ++k) {
+                    ids[k] = base + k < SL ? tgt[base + k] : -1;
+                    any |= ids[k] >= 0;
+                }
+                if (any) {
+                    Row<FPL> rows[TCH];
+                    float f[TCH];
+#pragma unroll
+                    for (int k = 0; k < TCH; ++k)
+                        if (ids[k] >= 0) rows[k] = row_load<FPL>(w_out, ids[k], lane);
+#pragma unroll
+                    for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
+#pragma unroll
+                    for (int k = 0; k < TCH; ++k) f[k] = warp_sum(f[k]);
+#pragma unroll
+                    for (int k = 0; k < TCH; ++k) {
+                        int kt = kk + k;
+                        while (kt >= T1) kt -= T1;
+                        if (ids[k] >= 0) {
+                            const bool is_ctx = kt == 0;
+                            const float g = sigmoidf_exact(f[k]) - (is_ctx ? 1.f : 0.f);
+                            loss += softplusf(is_ctx ? -f[k] : f[k]);
+                            const float step = -lr * g;
+                            Row<FPL> delta;
+#pragma unroll
+                            for (int j = 0; j < FPL; ++j) {
+                                acc.v[j] = fmaf(g, rows[k].v[j], acc.v[j]);
+                                delta.v[j] = step * u.v[j];
+                                rows[k].v[j] += delta.v[j];
+                            }
+                            if (RED) row_red_add<FPL>(w_out, ids[k], lane, delta);
+                            else row_store<FPL>(w_out, ids[k], lane, rows[k]);
+                        }
+                    }
+                }
+                kk += TCH;
+                while (kk >= T1) kk -= T1;
+            }
+            // center row: add the accumulated increment to the row as it is now
+            Row<FPL> delta;
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) delta.v[j] = -lr * acc.v[j];
+            if (RED) {
+                row_red_add<FPL>(w_in, c, lane, delta);
+            } else {
+                Row<FPL> now = row_load<FPL>(w_in, c, lane);
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) now.v[j] += delta.v[j];
+                row_store<FPL>(w_in, c, lane, now);
+            }
+            loss_acc += (double)loss;
+        }
+    }
+    if (lane == 0) {
+        if (loss_out && pair_acc) atomicAdd(loss_out, loss_acc);
+        if (pairs_out && pair_acc) atomicAdd(pairs_out, pair_acc);
+    }
+}
+
+// ---------------------------------------------------------------- synchronous mode
+// Pass 1: one warp per position.  Writes, for slot index x = pos * SL + slot:
+//   keys[x] = destination row of w_out (or `invalid`), gbuf[x] = coefficient g,
+// and per position: keys[n_slots + pos] = n_nodes + center (or `invalid`),
+// GU[pos] = sum g * v (gradient of the center row), loss_pos, pairs_pos.
+template <int FPL>
+__global__ void __launch_bounds__(SGNS_WARPS * 32)
+sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out,
+                 const int32_t *__restrict__ walks, int64_t n_pos, int64_t walk_id_base, int32_t L,
+                 int32_t w, int32_t K, const uint64_t *__restrict__ alias, uint32_t n_alias,
+                 uint32_t n_nodes, uint64_t seed, uint32_t *__restrict__ keys,
+                 float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos,
+                 int32_t *__restrict__ pairs_pos, int32_t *dump_pairs, int32_t *dump_negs)
+{
+    extern __shared__ int32_t smem[];
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    const int S = 2 * w, T1 = 1 + K, SL = S * T1;
+    int32_t *tgt = smem + wi * SL;
+    const uint32_t invalid = 2u * n_nodes;
+    const int64_t n_slots = n_pos * SL;
+    const int64_t n_warps = (int64_t)gridDim.x * SGNS_WARPS;
+
+    for (int64_t pos = (int64_t)blockIdx.x * SGNS_WARPS + wi; pos < n_pos; pos += n_warps) {
+        const int64_t a = pos / L;
+        const int32_t i = (int32_t)(pos - a * L);
+        const int32_t *W = walks + a * L;
+        const int32_t c = W[i];
+        int32_t *dp = dump_pairs ? dump_pairs + (pos * S) * 2 : nullptr;
+        int32_t *dn = dump_negs ? dump_negs + (pos * S) * (int64_t)K : nullptr;
+        uint32_t *kp = keys + pos * SL;
+        float *gp = gbuf + pos * SL;
+        Row<FPL> acc;
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+        float loss = 0.f;
+        int pairs = 0;
+        __syncwarp();
+        if (c >= 0)
+            pairs = build_targets(W, L, i, w, K, seed, (uint64_t)(walk_id_base + a), alias, n_alias,
+                                  c, tgt, lane, dp, dn);
+        else
+            dump_empty_position(S, K, lane, dp, dn);
+        if (pairs == 0) {
+            for (int x = lane; x < SL; x += 32) { kp[x] = invalid; gp[x] = 0.f; }
+        } else {
+            const Row<FPL> u = row_load<FPL>(w_in, c, lane);
+            int kk = 0;
+            for (int base = 0; base < SL; base += TCH) {
+                int32_t ids[TCH];
+#pragma unroll
+                for (int k = 0; k < TCH; ++k) ids[k] = base + k < SL ? tgt[base + k] : -1;
+                Row<FPL> rows[TCH];
+                float f[TCH];
+#pragma unroll
+                for (int k = 0; k < TCH; ++k)
+                    if (ids[k] >= 0) rows[k] = row_load<FPL>(w_out, ids[k], lane);
+#pragma unroll
+                for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
+#pragma unroll
+                for (int k = 0; k < TCH; ++k) f[k] = warp_sum(f[k]);
+#pragma unroll
+                for (int k = 0; k < TCH; ++k) {
+                    int kt = kk + k;
+                    while (kt >= T1) kt -= T1;
+                    float g = 0.f;
+                    if (ids[k] >= 0) {
+                        const bool is_ctx = kt == 0;
+                        g = sigmoidf_exact(f[k]) - (is_ctx ? 1.f : 0.f);
+                        loss += softplusf(is_ctx ? -f[k] : f[k]);
+#pragma unroll
+                        for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g, rows[k].v[j], acc.v[j]);
+                    }
+                    if (lane == k && base + k < SL) {
+                        kp[base + k] = ids[k] >= 0 ? (uint32_t)ids[k] : invalid;
+                        gp[base + k] = g;
+                    }
+                }
+                kk += TCH;
+                while (kk >= T1) kk -= T1;
+            }
+        }
+        row_store<FPL>(GU, pos, lane, acc);
+        if (lane == 0) {
+            keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
+            loss_pos[pos] = (double)loss;
+            pairs_pos[pos] = pairs;
+        }
+    }
+}
+
+// Pass 3: one warp per run of equal keys below n_nodes: v_row -= lr * sum_j g_j * u_center(j),
+// contributions taken in sorted (= index) order.
+template <int FPL>
+__global__ void __launch_bounds__(256)
+sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
+                      const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
+                      const uint32_t *__restrict__ vals, const float *__restrict__ gbuf,
+                      uint32_t n_keys, uint32_t n_nodes, int32_t SL, float lr)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t x = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); x < n_keys;
+         x += n_warps) {
+        const uint32_t key = keys[x];
+        if (key >= n_nodes) continue;
+        if (x > 0 && keys[x - 1] == key) continue;
+        Row<FPL> acc;
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+        for (int64_t y = x; y < n_keys; y += 4) {
+            float g[4];
+            int32_t c[4];
+            bool more = true;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const bool in = more && (y + q < n_keys) && (keys[y + q] == key);
+                more = in;
+                g[q] = 0.f;
+                c[q] = -1;
+                if (in) {
+                    const uint32_t idx = vals[y + q];
+                    g[q] = gbuf[idx];
+                    c[q] = walks[idx / (uint32_t)SL];
+                }
+            }
+            Row<FPL> r[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (c[q] >= 0) r[q] = row_load<FPL>(w_in, c[q], lane);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (c[q] >= 0) {
+#pragma unroll
+                    for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g[q], r[q].v[j], acc.v[j]);
+                }
+            if (!more) break;
+        }
+        Row<FPL> row = row_load<FPL>(w_out, key, lane);
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) row.v[j] = fmaf(-lr, acc.v[j], row.v[j]);
+        row_store<FPL>(w_out, key, lane, row);
+    }
+}
+
+// Pass 4: runs of keys in [n_nodes, 2 n_nodes): u_row -= lr * sum of the positions' GU rows.
+template <int FPL>
+__global__ void __launch_bounds__(256)
+sgns_apply_in_kernel(float *__restrict__ w_in, const float *__restrict__ GU,
+                     const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals,
+                     uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, float lr)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t x = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); x < n_keys;
+         x += n_warps) {
+        const uint32_t key = keys[x];
+        if (key < n_nodes || key >= 2u * n_nodes) continue;
+        if (x > 0 && keys[x - 1] == key) continue;
+        Row<FPL> acc;
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+        for (int64_t y = x; y < n_keys && keys[y] == key; ++y) {
+            const Row<FPL> r = row_load<FPL>(GU, (int64_t)(vals[y] - n_slots), lane);
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) acc.v[j] += r.v[j];
+        }
+        const int64_t c = (int64_t)(key - n_nodes);
+        Row<FPL> row = row_load<FPL>(w_in, c, lane);
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) row.v[j] = fmaf(-lr, acc.v[j], row.v[j]);
+        row_store<FPL>(w_in, c, lane, row);
+    }
+}
+
+// Fixed-order reduction of the per-position losses and pair counts (one block).
+__global__ void __launch_bounds__(1024)
+sgns_reduce_kernel(const double *__restrict__ loss_pos, const int32_t *__restrict__ pairs_pos,
+                   int64_t n_pos, double *loss_out, long long *pairs_out)
+{
+    __shared__ double sl[1024];
+    __shared__ long long sp[1024];
+    double l = 0.0;
+    long long p = 0;
+    for (int64_t x = threadIdx.x; x < n_pos; x += 1024) { l += loss_pos[x]; p += pairs_pos[x]; }
+    sl[threadIdx.x] = l;
+    sp[threadIdx.x] = p;
+    __syncthreads();
+    for (int o = 512; o > 0; o >>= 1) {
+        if (threadIdx.x < o) { sl[threadIdx.x] += sl[threadIdx.x + o]; sp[threadIdx.x] += sp[threadIdx.x + o]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        if (loss_out) *loss_out += sl[0];
+        if (pairs_out) *pairs_out += sp[0];
+    }
+}
+
+// ---------------------------------------------------------------- host side
+struct SgnsArgs {
+    float *w_in, *w_out;
+    int64_t n_nodes;
+    int32_t dim;
+    const int32_t *walks;
+    int64_t n_walks, walk_id_base;
+    int32_t L, w, K;
+    const uint64_t *alias;
+    float lr;
+    uint64_t seed;
+    double *loss;
+    int64_t *pairs;
+    int32_t *dump_pairs, *dump_negs;
+};
+
+static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
+
+template <int FPL, bool RED>
+static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
+{
+    const int SL = 2 * a.w * (1 + a.K);
+    const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(a.L + SL);
+    auto kern = sgns_hogwild_kernel<FPL, RED>;
+    if (smem > 48 * 1024)
+        GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    GS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SGNS_WARPS * 32, smem));
+    if (per_sm < 1) per_sm = 1;
+    int64_t blocks = (a.n_walks + SGNS_WARPS - 1) / SGNS_WARPS;
+    const int64_t cap = (int64_t)sm_count() * per_sm;
+    if (blocks > cap) blocks = cap;
+    kern<<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+        a.w_in, a.w_out, a.walks, a.n_walks, a.walk_id_base, a.L, a.w, a.K, a.alias,
+        (uint32_t)a.n_nodes, a.lr, a.seed, a.loss, (unsigned long long *)a.pairs, a.dump_pairs,
+        a.dump_negs);
+    GS_CUDA_TRY(cudaGetLastError());
+    return GS_OK;
+}
+
+static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+template <int FPL>
+static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
+{
+    const int SL = 2 * a.w * (1 + a.K);
+    const int64_t n_pos = a.n_walks * a.L;
+    const int64_t n_slots = n_pos * SL;
+    const int64_t n_keys = n_slots + n_pos;
+    if (n_keys > ((int64_t)1 << 30)) {
+        set_error("deterministic step: %lld slots exceed 2^30; use smaller batches",
+                  (long long)n_keys);
+        return GS_ERR_UNSUPPORTED;
+    }
+    // scratch carve-up
+    const size_t b_keys = align_up(sizeof(uint32_t) * (size_t)n_keys);
+    const size_t b_g = align_up(sizeof(float) * (size_t)n_slots);
+    const size_t b_gu = align_up(sizeof(float) * (size_t)n_pos * a.dim);
+    const size_t b_loss = align_up(sizeof(double) * (size_t)n_pos);
+    const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)n_pos);
+    const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)n_keys));
+    void *ws = nullptr;
+    gs_status s = workspace_get(WS_SGNS, 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt, &ws);
+    if (s != GS_OK) return s;
+    char *p = (char *)ws;
+    uint32_t *keysA = (uint32_t *)p; p += b_keys;
+    uint32_t *keysB = (uint32_t *)p; p += b_keys;
+    uint32_t *valsA = (uint32_t *)p; p += b_keys;
+    uint32_t *valsB = (uint32_t *)p; p += b_keys;
+    float *gbuf = (float *)p; p += b_g;
+    float *GU = (float *)p; p += b_gu;
+    double *loss_pos = (double *)p; p += b_loss;
+    int32_t *pairs_pos = (int32_t *)p; p += b_pairs;
+    uint32_t *counts = (uint32_t *)p;
+
+    {
+        const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
+        int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
+        const int64_t cap = (int64_t)sm_count() * 16;
+        if (blocks > cap) blocks = cap;
+        sgns_coef_kernel<FPL><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+            a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
+            (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
+            a.dump_pairs, a.dump_negs);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    uint32_t *ks = nullptr, *vs = nullptr;
+    radix_sort_pairs(keysA, valsA, keysB, valsB, (uint32_t)n_keys,
+                     bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
+    GS_CUDA_TRY(cudaGetLastError());
+    {
+        int64_t blocks = (n_keys + 7) / 8;
+        const int64_t cap = (int64_t)sm_count() * 8 * 8;
+        if (blocks > cap) blocks = cap;
+        sgns_apply_out_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
+            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr);
+        GS_CUDA_TRY(cudaGetLastError());
+        sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
+            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    if (a.loss || a.pairs) {
+        sgns_reduce_kernel<<<1, 1024, 0, st>>>(loss_pos, pairs_pos, n_pos, a.loss,
+                                               (long long *)a.pairs);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    return GS_OK;
+}
+
+template <int FPL>
+static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
+{
+    if (mode == GS_DETERMINISTIC) return run_deterministic<FPL>(a, st);
+    if (mode == GS_HOGWILD) return run_hogwild<FPL, false>(a, st);
+    return run_hogwild<FPL, true>(a, st);
+}
+
+gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                    int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                    const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
+                    int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st)
+{
+    if (n_walks == 0) return GS_OK;
+    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                   seed, loss, pairs, dump_pairs, dump_negs };
+    switch (dim) {
+        case 32: return run_mode<1>(a, mode, st);
+        case 64: return run_mode<2>(a, mode, st);
+        case 128: return run_mode<4>(a, mode, st);
+        case 256: return run_mode<8>(a, mode, st);
+        default:
+            set_error("dim %d not supported (32, 64, 128, 256)", dim);
+            return GS_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace gs

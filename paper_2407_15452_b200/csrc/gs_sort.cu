@@ -1,0 +1,152 @@
+// Stable least-significant-digit radix sort of (key, value) pairs, 8 bits per
+// pass.  It groups the gradient contributions of a synchronous SGNS step by
+// destination row while keeping contributions of one row in index order, which
+// is what makes the summation order (and so the result bits) fixed.
+//
+// Per pass: (1) per-tile digit histograms, (2) one exclusive scan over the
+// digit-major (digit, tile) counts, (3) a scatter in which each warp ranks its
+// items round by round with match_any, so that equal digits keep their order.
+#include "gs_common.cuh"
+
+namespace gs {
+
+constexpr int SORT_THREADS = 256;
+constexpr int SORT_ITEMS = 8;
+constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 2048 keys per block
+constexpr int RADIX = 256;
+
+__global__ void __launch_bounds__(SORT_THREADS)
+sort_hist_kernel(const uint32_t *__restrict__ keys, uint32_t n, int shift, uint32_t n_tiles,
+                 uint32_t *__restrict__ counts)
+{
+    __shared__ uint32_t h[RADIX];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t base = blockIdx.x * SORT_TILE;
+#pragma unroll
+    for (int r = 0; r < SORT_ITEMS; ++r) {
+        const uint32_t i = base + r * SORT_THREADS + threadIdx.x;
+        if (i < n) atomicAdd(&h[(keys[i] >> shift) & (RADIX - 1)], 1u);
+    }
+    __syncthreads();
+    counts[threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
+}
+
+// Exclusive scan of m counters by one block: each thread owns a contiguous chunk.
+__global__ void __launch_bounds__(1024) sort_scan_kernel(uint32_t *__restrict__ counts, uint32_t m)
+{
+    __shared__ uint32_t part[1024];
+    const uint32_t chunk = (m + 1023u) / 1024u;
+    const uint32_t lo = threadIdx.x * chunk;
+    const uint32_t hi = lo + chunk < m ? lo + chunk : m;
+    uint32_t s = 0;
+    for (uint32_t i = lo; i < hi; ++i) s += counts[i];
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {               // Hillis-Steele inclusive scan
+        const uint32_t add = threadIdx.x >= (unsigned)o ? part[threadIdx.x - o] : 0u;
+        __syncthreads();
+        part[threadIdx.x] += add;
+        __syncthreads();
+    }
+    uint32_t run = part[threadIdx.x] - s;
+    for (uint32_t i = lo; i < hi; ++i) {
+        const uint32_t c = counts[i];
+        counts[i] = run;
+        run += c;
+    }
+}
+
+template <bool IOTA>
+__global__ void __launch_bounds__(SORT_THREADS)
+sort_scatter_kernel(const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in,
+                    uint32_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out, uint32_t n,
+                    int shift, uint32_t n_tiles, const uint32_t *__restrict__ offsets)
+{
+    constexpr int WARPS = SORT_THREADS / 32;
+    __shared__ uint32_t cnt[WARPS][RADIX];
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    for (int x = threadIdx.x; x < WARPS * RADIX; x += SORT_THREADS) (&cnt[0][0])[x] = 0;
+    __syncthreads();
+
+    // warp wi owns the contiguous run [base, base + 32 * SORT_ITEMS), visited in index order
+    const uint32_t base = blockIdx.x * SORT_TILE + wi * (32 * SORT_ITEMS);
+    uint32_t key[SORT_ITEMS], val[SORT_ITEMS], loc[SORT_ITEMS];
+#pragma unroll
+    for (int r = 0; r < SORT_ITEMS; ++r) {
+        const uint32_t i = base + r * 32 + lane;
+        const bool ok = i < n;
+        key[r] = ok ? keys_in[i] : 0u;
+        val[r] = ok ? (IOTA ? i : vals_in[i]) : 0u;
+        const uint32_t d = ok ? ((key[r] >> shift) & (RADIX - 1)) : RADIX;   // RADIX = absent
+        const unsigned peers = __match_any_sync(0xffffffffu, d);
+        const int leader = __ffs(peers) - 1;
+        uint32_t before = 0;
+        if (ok && lane == leader) {
+            before = cnt[wi][d];
+            cnt[wi][d] = before + __popc(peers);
+        }
+        before = __shfl_sync(0xffffffffu, before, leader);
+        loc[r] = before + __popc(peers & ((1u << lane) - 1u));
+        __syncwarp();
+    }
+    __syncthreads();
+    {   // digit threadIdx.x: turn per-warp counts into start positions in the output
+        const int d = threadIdx.x;
+        uint32_t run = offsets[d * n_tiles + blockIdx.x];
+#pragma unroll
+        for (int k = 0; k < WARPS; ++k) {
+            const uint32_t c = cnt[k][d];
+            cnt[k][d] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < SORT_ITEMS; ++r) {
+        const uint32_t i = base + r * 32 + lane;
+        if (i < n) {
+            const uint32_t dst = cnt[wi][(key[r] >> shift) & (RADIX - 1)] + loc[r];
+            keys_out[dst] = key[r];
+            vals_out[dst] = val[r];
+        }
+    }
+}
+
+size_t sort_counts_bytes(uint32_t n)
+{
+    const uint32_t n_tiles = (n + SORT_TILE - 1) / SORT_TILE;
+    return sizeof(uint32_t) * (size_t)RADIX * (n_tiles ? n_tiles : 1);
+}
+
+// Sorts n pairs by the low `bits` bits of the key.  The first pass takes value i for
+// item i (no input value array).  Buffers A hold the input; on return *keys_sorted /
+// *vals_sorted point at whichever of A / B holds the result.  Returns launches made.
+int radix_sort_pairs(uint32_t *keysA, uint32_t *valsA, uint32_t *keysB, uint32_t *valsB,
+                     uint32_t n, int bits, uint32_t *counts, cudaStream_t st,
+                     uint32_t **keys_sorted, uint32_t **vals_sorted)
+{
+    const uint32_t n_tiles = (n + SORT_TILE - 1) / SORT_TILE;
+    uint32_t *kin = keysA, *vin = valsA, *kout = keysB, *vout = valsB;
+    int launches = 0;
+    bool first = true;
+    for (int shift = 0; shift < bits && n > 0; shift += 8) {
+        sort_hist_kernel<<<n_tiles, SORT_THREADS, 0, st>>>(kin, n, shift, n_tiles, counts);
+        sort_scan_kernel<<<1, 1024, 0, st>>>(counts, RADIX * n_tiles);
+        if (first)
+            sort_scatter_kernel<true><<<n_tiles, SORT_THREADS, 0, st>>>(kin, vin, kout, vout, n,
+                                                                        shift, n_tiles, counts);
+        else
+            sort_scatter_kernel<false><<<n_tiles, SORT_THREADS, 0, st>>>(kin, vin, kout, vout, n,
+                                                                         shift, n_tiles, counts);
+        launches += 3;
+        first = false;
+        uint32_t *t = kin; kin = kout; kout = t;
+        t = vin; vin = vout; vout = t;
+    }
+    *keys_sorted = kin;
+    *vals_sorted = vin;
+    return launches;
+}
+
+}  // namespace gs

@@ -1,0 +1,332 @@
+// Graph validation, table initialisation and the two walk samplers.
+//
+// Walks are chains of dependent random reads (offset pair, then one column), so
+// throughput comes from the number of walks in flight, not from per-walk
+// parallelism: the uniform sampler runs one walk per THREAD; the node2vec
+// sampler runs one walk per group of G lanes that evaluate G rejection rounds
+// speculatively and keep the first accepted one, which is exactly the outcome
+// of running the rounds one after another.
+#include "gs_common.cuh"
+
+namespace gs {
+
+// ------------------------------------------------------------------ validation
+struct CsrReport {
+    unsigned long long bad_row;        // first row with broken offsets / column range
+    unsigned long long unsorted_row;   // first row that is not strictly increasing
+    unsigned long long max_degree;
+    unsigned long long ends_bad;       // offsets[0] != 0 or offsets[n] != n_edges
+};
+
+template <typename OffT>
+__global__ void __launch_bounds__(256)
+validate_csr_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
+                    int64_t n_nodes, int64_t n_edges, int check_sorted, CsrReport *rep)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    unsigned long long local_max = 0;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < n_nodes; v += stride) {
+        const int64_t o0 = (int64_t)off[v], o1 = (int64_t)off[v + 1];
+        if (v == 0 && o0 != 0) atomicExch(&rep->ends_bad, 1ull);
+        if (v == n_nodes - 1 && o1 != n_edges) atomicExch(&rep->ends_bad, 1ull);
+        if (o0 < 0 || o1 < o0 || o1 > n_edges) {
+            atomicMin(&rep->bad_row, (unsigned long long)v);
+            continue;                                   // never index cols with a broken range
+        }
+        const unsigned long long deg = (unsigned long long)(o1 - o0);
+        local_max = deg > local_max ? deg : local_max;
+        int32_t last = -1;
+        bool range_ok = true, sorted_ok = true;
+        for (int64_t e = o0; e < o1; ++e) {
+            const int32_t c = col[e];
+            range_ok &= (c >= 0) && ((int64_t)c < n_nodes);
+            sorted_ok &= c > last;
+            last = c;
+        }
+        if (!range_ok) atomicMin(&rep->bad_row, (unsigned long long)v);
+        if (check_sorted && !sorted_ok) atomicMin(&rep->unsorted_row, (unsigned long long)v);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, local_max, o);
+        local_max = other > local_max ? other : local_max;
+    }
+    if ((threadIdx.x & 31) == 0 && local_max) atomicMax(&rep->max_degree, local_max);
+}
+
+gs_status validate_csr(const gs_graph *g, bool check_sorted, cudaStream_t st,
+                       int64_t *bad_row, int64_t *unsorted_row, int64_t *max_degree, bool *ends_bad)
+{
+    void *ws = nullptr;
+    gs_status s = workspace_get(WS_COUNTERS, 256, &ws);
+    if (s != GS_OK) return s;
+    CsrReport *rep = (CsrReport *)ws;
+    CsrReport init = { ~0ull, ~0ull, 0ull, 0ull };
+    GS_CUDA_TRY(cudaMemcpyAsync(rep, &init, sizeof(init), cudaMemcpyHostToDevice, st));
+    if (g->n_nodes > 0) {
+        const int threads = 256;
+        int64_t blocks = (g->n_nodes + threads - 1) / threads;
+        const int64_t cap = (int64_t)sm_count() * 64;
+        if (blocks > cap) blocks = cap;
+        if (g->offsets64)
+            validate_csr_kernel<int64_t><<<(unsigned)blocks, threads, 0, st>>>(
+                (const int64_t *)g->d_offsets, g->d_cols, g->n_nodes, g->n_edges, check_sorted, rep);
+        else
+            validate_csr_kernel<int32_t><<<(unsigned)blocks, threads, 0, st>>>(
+                (const int32_t *)g->d_offsets, g->d_cols, g->n_nodes, g->n_edges, check_sorted, rep);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    CsrReport h;
+    GS_CUDA_TRY(cudaMemcpyAsync(&h, rep, sizeof(h), cudaMemcpyDeviceToHost, st));
+    GS_CUDA_TRY(cudaStreamSynchronize(st));
+    *bad_row = h.bad_row == ~0ull ? -1 : (int64_t)h.bad_row;
+    *unsorted_row = h.unsorted_row == ~0ull ? -1 : (int64_t)h.unsorted_row;
+    *max_degree = (int64_t)h.max_degree;
+    *ends_bad = h.ends_bad != 0;
+    return GS_OK;
+}
+
+// ------------------------------------------------------------------ table init
+__global__ void __launch_bounds__(256)
+init_rows_kernel(float *__restrict__ w, int64_t n_rows, int32_t dim, uint64_t seed)
+{
+    const int32_t quads = dim >> 2;
+    const int64_t total = n_rows * quads;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const float inv_d = 1.0f / (float)dim;             // dim is a power of two here: exact
+    for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < total; x += stride) {
+        const int64_t row = x / quads;
+        const uint32_t qd = (uint32_t)(x - row * quads);
+        const uint4 r = draw(seed, (uint64_t)row, qd, TAG_INIT, 0);
+        float4 v;
+        v.x = ((float)(r.x >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        v.y = ((float)(r.y >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        v.z = ((float)(r.z >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        v.w = ((float)(r.w >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        reinterpret_cast<float4 *>(w)[x] = v;
+    }
+}
+
+gs_status init_embeddings(float *w_in, float *w_out, int64_t n, int32_t dim, uint64_t seed,
+                          cudaStream_t st)
+{
+    if (w_in && n > 0) {
+        const int64_t total = n * (dim >> 2);
+        int64_t blocks = (total + 255) / 256;
+        const int64_t cap = (int64_t)sm_count() * 32;
+        if (blocks > cap) blocks = cap;
+        init_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(w_in, n, dim, seed);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    if (w_out && n > 0)
+        GS_CUDA_TRY(cudaMemsetAsync(w_out, 0, sizeof(float) * (size_t)n * (size_t)dim, st));
+    return GS_OK;
+}
+
+// ------------------------------------------------------------------ uniform walks
+// One walk per thread.  Per transition: two adjacent offsets, one Philox block,
+// one column read, one 4-byte store into the walk-major output.
+template <typename OffT>
+__global__ void __launch_bounds__(256)
+uniform_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
+                    const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
+                    int64_t walk_id_base, int32_t L, uint64_t seed,
+                    int32_t *__restrict__ walks, unsigned long long *steps_out)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    unsigned int my_steps = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
+        const uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
+        int32_t *W = walks + i * (int64_t)L;
+        W[0] = cur;
+        int32_t t = 0;
+        for (; t + 1 < L; ++t) {
+            const int64_t o0 = load_off(off, cur), o1 = load_off(off, (int64_t)cur + 1);
+            const uint32_t deg = (uint32_t)(o1 - o0);
+            if (deg == 0) break;
+            const uint4 r = draw(seed, id, (uint32_t)t, TAG_UNIFORM, 0);
+            cur = __ldg(col + o0 + (int64_t)__umulhi(r.x, deg));
+            W[t + 1] = cur;
+            ++my_steps;
+        }
+        for (int32_t s = t + 1; s < L; ++s) W[s] = -1;
+    }
+    if (steps_out) {
+        for (int o = 16; o > 0; o >>= 1) my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
+        if ((threadIdx.x & 31) == 0 && my_steps) atomicAdd(steps_out, (unsigned long long)my_steps);
+    }
+}
+
+gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
+                               int64_t base, int32_t L, uint64_t seed, int32_t *walks,
+                               unsigned long long *steps, cudaStream_t st)
+{
+    if (n_walks == 0) return GS_OK;
+    const int threads = 256;
+    int64_t blocks = (n_walks + threads - 1) / threads;
+    const int64_t cap = (int64_t)sm_count() * 8 * 16;
+    if (blocks > cap) blocks = cap;
+    if (g->offsets64)
+        uniform_walk_kernel<int64_t><<<(unsigned)blocks, threads, 0, st>>>(
+            (const int64_t *)g->d_offsets, g->d_cols, starts, g->n_nodes, n_walks, base, L, seed,
+            walks, steps);
+    else
+        uniform_walk_kernel<int32_t><<<(unsigned)blocks, threads, 0, st>>>(
+            (const int32_t *)g->d_offsets, g->d_cols, starts, g->n_nodes, n_walks, base, L, seed,
+            walks, steps);
+    GS_CUDA_TRY(cudaGetLastError());
+    return GS_OK;
+}
+
+// ------------------------------------------------------------------ node2vec walks
+struct N2VThresholds {
+    unsigned long long t_prev, t_near, t_far;   // floor(weight / max weight * 2^32), <= 2^32
+};
+
+// x in cols[lo, hi) ?  (strictly increasing row, at most 32 halvings of a < 2^32 range)
+__device__ __forceinline__ bool row_contains(const int32_t *__restrict__ col, int64_t lo,
+                                             int64_t hi, int32_t x)
+{
+    const int64_t end = hi;
+    while (lo < hi) {
+        const int64_t mid = lo + ((hi - lo) >> 1);
+        if (__ldg(col + mid) < x) lo = mid + 1; else hi = mid;
+    }
+    return lo < end && __ldg(col + lo) == x;
+}
+
+// G lanes per walk; lane k of a group evaluates rejection round base + k.
+template <typename OffT, int G>
+__global__ void __launch_bounds__(256)
+node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
+                     const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
+                     int64_t walk_id_base, int32_t L, uint64_t seed, N2VThresholds T,
+                     int32_t max_rounds, int32_t *__restrict__ walks,
+                     unsigned long long *steps_out, unsigned long long *caps_out)
+{
+    const int lane = threadIdx.x & 31;
+    const int sub = lane % G;                       // round offset inside the group
+    const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane - sub));
+    const int64_t groups_per_grid = (int64_t)gridDim.x * (blockDim.x / G);
+    const unsigned long long t_lo = T.t_near < T.t_far ? T.t_near : T.t_far;
+    const unsigned long long t_hi = T.t_near < T.t_far ? T.t_far : T.t_near;
+    unsigned int my_steps = 0, my_caps = 0;
+
+    // n_walks is rounded up per warp so that every lane of a warp runs the same number of
+    // outer iterations (the group ballots below need their whole group present).
+    for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G; i < n_walks;
+         i += groups_per_grid) {
+        const uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
+        int32_t prev = -1;
+        int64_t p0 = 0, p1 = 0;                     // adjacency range of prev
+        int32_t *W = walks + i * (int64_t)L;
+        if (sub == 0) W[0] = cur;
+        int32_t t = 0;
+        for (; t + 1 < L; ++t) {
+            const int64_t o0 = load_off(off, cur), o1 = load_off(off, (int64_t)cur + 1);
+            const uint32_t deg = (uint32_t)(o1 - o0);
+            if (deg == 0) break;
+            int32_t nxt;
+            if (t == 0) {
+                const uint4 r = draw(seed, id, 0u, TAG_NODE2VEC, 0);
+                nxt = __ldg(col + o0 + (int64_t)__umulhi(r.x, deg));
+            } else {
+                nxt = -1;
+                for (int32_t rbase = 0;; rbase += G) {
+                    const int32_t s = rbase + sub;
+                    const bool live = s < max_rounds;
+                    int32_t x = -1;
+                    bool acc = false;
+                    if (live) {
+                        const uint4 r = draw(seed, id, (uint32_t)t, TAG_NODE2VEC, (uint32_t)s);
+                        x = __ldg(col + o0 + (int64_t)__umulhi(r.x, deg));
+                        const unsigned long long r1 = r.y;
+                        if (x == prev) acc = r1 < T.t_prev;
+                        else if (r1 < t_lo) acc = true;          // accepted in either class
+                        else if (r1 >= t_hi) acc = false;        // rejected in either class
+                        else acc = r1 < (row_contains(col, p0, p1, x) ? T.t_near : T.t_far);
+                    }
+                    const unsigned votes = __ballot_sync(gmask, acc) & gmask;
+                    if (votes) {
+                        nxt = __shfl_sync(gmask, x, __ffs(votes) - 1);
+                        break;
+                    }
+                    if (rbase + G >= max_rounds) {               // cap: keep the last proposal
+                        const int last_lane = (lane - sub) + (max_rounds - 1 - rbase);
+                        nxt = __shfl_sync(gmask, x, last_lane);
+                        if (sub == 0) ++my_caps;
+                        break;
+                    }
+                }
+            }
+            prev = cur; p0 = o0; p1 = o1;
+            cur = nxt;
+            if (sub == 0) { W[t + 1] = cur; ++my_steps; }
+        }
+        if (sub == 0)
+            for (int32_t s = t + 1; s < L; ++s) W[s] = -1;
+    }
+    if (steps_out && my_steps) atomicAdd(steps_out, (unsigned long long)my_steps);
+    if (caps_out && my_caps) atomicAdd(caps_out, (unsigned long long)my_caps);
+}
+
+void node2vec_thresholds(double p, double q, N2VThresholds *T)
+{
+    const double a[3] = { 1.0 / p, 1.0, 1.0 / q };
+    double m = a[0];
+    for (int c = 1; c < 3; ++c) m = a[c] > m ? a[c] : m;
+    unsigned long long out[3];
+    for (int c = 0; c < 3; ++c) {
+        double v = floor(a[c] / m * 4294967296.0);
+        if (v > 4294967296.0) v = 4294967296.0;
+        out[c] = (unsigned long long)v;
+    }
+    T->t_prev = out[0]; T->t_near = out[1]; T->t_far = out[2];
+}
+
+template <typename OffT, int G>
+static void launch_n2v(const gs_graph *g, const int32_t *starts, int64_t n_walks, int64_t base,
+                       int32_t L, uint64_t seed, const N2VThresholds &T, int32_t max_rounds,
+                       int32_t *walks, unsigned long long *steps, unsigned long long *caps,
+                       cudaStream_t st)
+{
+    const int threads = 256;
+    const int64_t per_block = threads / G;
+    int64_t blocks = (n_walks + per_block - 1) / per_block;
+    const int64_t cap = (int64_t)sm_count() * 8 * 16;
+    if (blocks > cap) blocks = cap;
+    node2vec_walk_kernel<OffT, G><<<(unsigned)blocks, threads, 0, st>>>(
+        (const OffT *)g->d_offsets, g->d_cols, starts, g->n_nodes, n_walks, base, L, seed, T,
+        max_rounds, walks, steps, caps);
+}
+
+gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
+                                int64_t base, int32_t L, uint64_t seed, double p, double q,
+                                int32_t max_rounds, int group, int32_t *walks,
+                                unsigned long long *steps, unsigned long long *caps,
+                                cudaStream_t st)
+{
+    if (n_walks == 0) return GS_OK;
+    N2VThresholds T;
+    node2vec_thresholds(p, q, &T);
+#define GS_N2V(GG)                                                                              \
+    do {                                                                                        \
+        if (g->offsets64) launch_n2v<int64_t, GG>(g, starts, n_walks, base, L, seed, T,         \
+                                                  max_rounds, walks, steps, caps, st);          \
+        else launch_n2v<int32_t, GG>(g, starts, n_walks, base, L, seed, T, max_rounds, walks,   \
+                                     steps, caps, st);                                          \
+    } while (0)
+    switch (group) {
+        case 1: GS_N2V(1); break;
+        case 2: GS_N2V(2); break;
+        case 8: GS_N2V(8); break;
+        case 32: GS_N2V(32); break;
+        default: GS_N2V(4); break;
+    }
+#undef GS_N2V
+    GS_CUDA_TRY(cudaGetLastError());
+    return GS_OK;
+}
+
+}  // namespace gs

@@ -1,0 +1,375 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle on the same
+seeded inputs.  Integer outputs (walks, pairs, negative draws, counts) must be bit-exact;
+embeddings after one synchronous step within 1e-4 absolute of the fp64 oracle; epoch loss
+within 1e-3 relative."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gs_oracle as O
+from paper_2407_15452_b200 import binding as B
+from paper_2407_15452_b200 import workloads as WL
+from tests.helpers import alias_to_device, compact_problem, degree_alias, np_graph
+
+pytestmark = pytest.mark.gpu
+
+EMB_TOL = 1e-4        # max |delta| after one synchronous step (fp32 kernels vs fp64 oracle)
+LOSS_RTOL = 1e-3      # mean epoch loss
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    wl = WL.WORKLOADS["tiny_deepwalk"]
+    g = wl.make_graph()
+    off, col = np_graph(g)
+    thr, alias = degree_alias(off)
+    return wl, g, off, col, thr, alias
+
+
+def load(g, offsets64=False, flags=B.GS_VALIDATE | B.GS_REQUIRE_SORTED):
+    off = g.offsets.to(torch.int64 if offsets64 else torch.int32).to(DEV)
+    return B.gs_graph_load_csr(off, g.cols.to(DEV), flags)
+
+
+# ---------------------------------------------------------------- graph loading
+def test_graph_validation_reports_errors(tiny):
+    _, g, off, col, _, _ = tiny
+    G = load(g)
+    info = G.info()
+    assert info["n_nodes"] == g.n_nodes and info["n_edges"] == g.n_edges
+    assert info["max_degree"] == int((off[1:] - off[:-1]).max()) and info["rows_sorted"]
+    # unsorted row
+    bad = g.cols.clone()
+    v = int(np.flatnonzero((off[1:] - off[:-1]) >= 2)[5])
+    a = int(off[v])
+    bad[a], bad[a + 1] = g.cols[a + 1].item(), g.cols[a].item()
+    with pytest.raises(B.GsError) as e:
+        B.gs_graph_load_csr(g.offsets.to(DEV), bad.to(DEV), B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    assert e.value.status == -3 and f"row {v} " in str(e.value)
+    B.gs_graph_load_csr(g.offsets.to(DEV), bad.to(DEV), B.GS_VALIDATE).close()   # fine unsorted
+    # column out of range
+    bad = g.cols.clone()
+    bad[a] = g.n_nodes
+    with pytest.raises(B.GsError) as e:
+        B.gs_graph_load_csr(g.offsets.to(DEV), bad.to(DEV), B.GS_VALIDATE)
+    assert e.value.status == -2 and f"row {v} " in str(e.value)
+    # decreasing offsets, wrong end
+    boff = g.offsets.clone()
+    boff[v + 1] = boff[v] - 1
+    with pytest.raises(B.GsError) as e:
+        B.gs_graph_load_csr(boff.to(DEV), g.cols.to(DEV), B.GS_VALIDATE)
+    assert e.value.status == -2
+    boff = g.offsets.clone()
+    boff[-1] -= 1
+    with pytest.raises(B.GsError) as e:
+        B.gs_graph_load_csr(boff.to(DEV), g.cols.to(DEV), B.GS_VALIDATE)
+    assert e.value.status == -2
+    # node2vec refuses a graph whose rows were not verified
+    G2 = load(g, flags=B.GS_VALIDATE)
+    with pytest.raises(B.GsError) as e:
+        B.gs_node2vec_walks(G2, None, 4, 0, 5, 0, 0.5, 2.0)
+    assert e.value.status == -3
+
+
+# ---------------------------------------------------------------- walks
+@pytest.mark.parametrize("offsets64", [False, True])
+def test_uniform_walks_bit_exact(tiny, offsets64):
+    wl, g, off, col, _, _ = tiny
+    G = load(g, offsets64)
+    n = g.n_nodes
+    steps = torch.zeros(1, dtype=torch.int64, device=DEV)
+    # ragged count (not a multiple of the block size), ids continue past one repetition
+    got = B.gs_random_walks(G, None, 2 * n + 77, 123, wl.walk_len, 0, steps=steps)
+    want, st = O.uniform_walks(off, col, None, 2 * n + 77, 123, wl.walk_len, 0)
+    assert np.array_equal(got.cpu().numpy(), want)
+    assert int(steps.item()) == st
+    # explicit start nodes, another seed, long walks
+    rng = np.random.default_rng(1)
+    starts = rng.integers(0, n, size=3001).astype(np.int32)
+    got = B.gs_random_walks(G, torch.from_numpy(starts).to(DEV), 3001, 5_000_000_000, 80,
+                            0xDEADBEEFCAFEF00D)
+    want, _ = O.uniform_walks(off, col, starts, 3001, 5_000_000_000, 80, 0xDEADBEEFCAFEF00D)
+    assert np.array_equal(got.cpu().numpy(), want)
+
+
+def test_uniform_walks_dead_ends_and_degenerate_sizes():
+    g = WL.rmat_graph(3000, 9000, seed=5)           # directed: dead ends
+    off, col = np_graph(g)
+    G = load(g, offsets64=True, flags=B.GS_VALIDATE)
+    got = B.gs_random_walks(G, None, 6000, 0, 20, 9)
+    want, _ = O.uniform_walks(off, col, None, 6000, 0, 20, 9)
+    assert (want == -1).any() and np.array_equal(got.cpu().numpy(), want)
+    assert B.gs_random_walks(G, None, 0, 0, 20, 9).shape == (0, 20)
+    got = B.gs_random_walks(G, None, 10, 0, 1, 9)                      # length 1: just the start
+    assert np.array_equal(got.cpu().numpy()[:, 0], np.arange(10))
+
+
+@pytest.mark.parametrize("p,q,max_rounds", [(0.5, 2.0, 1024), (4.0, 0.25, 1024), (1.0, 1.0, 1024),
+                                             (0.5, 2.0, 3), (100.0, 100.0, 1), (0.5, 2.0, 37)])
+def test_node2vec_walks_bit_exact_for_every_group_width(tiny, p, q, max_rounds):
+    _, g, off, col, _, _ = tiny
+    G = load(g)
+    n_walks, L = 5003, 24
+    want, st, caps = O.node2vec_walks(off, col, None, n_walks, 77, L, 5, p, q, max_rounds)
+    try:
+        for lanes in (1, 2, 4, 8, 32):
+            B.gs_tune_node2vec_group(lanes)
+            steps = torch.zeros(1, dtype=torch.int64, device=DEV)
+            hits = torch.zeros(1, dtype=torch.int64, device=DEV)
+            got = B.gs_node2vec_walks(G, None, n_walks, 77, L, 5, p, q, max_rounds, steps=steps,
+                                      cap_hits=hits)
+            assert np.array_equal(got.cpu().numpy(), want), lanes
+            assert int(steps.item()) == st and int(hits.item()) == caps, lanes
+    finally:
+        B.gs_tune_node2vec_group(4)
+    if max_rounds <= 3:
+        assert caps > 0
+
+
+def test_node2vec_on_directed_graph_with_dead_ends_and_int64_offsets():
+    g = WL.rmat_graph(3000, 12000, seed=6)
+    off, col = np_graph(g)
+    G = load(g, offsets64=True)
+    rng = np.random.default_rng(2)
+    starts = rng.integers(0, 3000, size=4000).astype(np.int32)
+    want, _, _ = O.node2vec_walks(off, col, starts, 4000, 0, 30, 11, 0.25, 4.0)
+    got = B.gs_node2vec_walks(G, torch.from_numpy(starts).to(DEV), 4000, 0, 30, 11, 0.25, 4.0)
+    assert np.array_equal(got.cpu().numpy(), want)
+
+
+# ---------------------------------------------------------------- initialisation
+@pytest.mark.parametrize("dim", [32, 64, 128, 256])
+def test_initial_tables_equal_oracle_exactly(dim):
+    n = 5000
+    w_in = torch.empty((n, dim), dtype=torch.float32, device=DEV)
+    w_out = torch.full((n, dim), 7.0, dtype=torch.float32, device=DEV)
+    B.gs_init_embeddings(w_in, w_out, seed=42)
+    want = O.init_rows(np.arange(n), dim, 42)
+    assert np.array_equal(w_in.cpu().numpy().astype(np.float64), want)
+    assert not w_out.any()
+
+
+# ---------------------------------------------------------------- SGNS step
+def run_step(w_in, w_out, walks, base, w, K, alias_dev, lr, seed, mode, dump=True):
+    n_walks, L = walks.shape
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    pd = nd = None
+    if dump:
+        pd = torch.full((n_walks, L, 2 * w, 2), -7, dtype=torch.int32, device=DEV)
+        nd = torch.full((n_walks, L, 2 * w, max(K, 1)), -7, dtype=torch.int32, device=DEV)[..., :K].contiguous()
+    B.gs_sgns_step(w_in, w_out, walks, base, w, K, alias_dev, lr, seed, mode, loss, cnt, pd, nd)
+    torch.cuda.synchronize()
+    return loss.item(), cnt.item(), pd, nd
+
+
+def oracle_step(U0, V0, walks, base, w, K, thr, alias, lr, seed):
+    c, o, ng, n_pairs = O.expand_lists(walks, base, w, K, thr, alias, seed)
+    U, V = U0.astype(np.float64), V0.astype(np.float64)
+    loss, cnt = O.sgns_det_from_lists(U, V, c, o, ng, lr)
+    return U, V, loss, cnt, c, o, ng
+
+
+def random_tables(n, dim, seed, scale=0.3):
+    gen = torch.Generator().manual_seed(seed)
+    w_in = (torch.rand((n, dim), generator=gen) - 0.5) * scale
+    w_out = (torch.rand((n, dim), generator=gen) - 0.5) * scale
+    return w_in, w_out
+
+
+@pytest.mark.parametrize("dim,L,w,K", [(64, 10, 5, 5), (128, 40, 10, 5), (32, 7, 3, 4),
+                                        (256, 12, 2, 1), (128, 6, 8, 10), (64, 9, 4, 0)])
+def test_deterministic_step_matches_oracle(tiny, dim, L, w, K):
+    _, g, off, col, thr, alias = tiny
+    n = g.n_nodes
+    n_walks = 301                                      # several blocks and a ragged tail
+    walks, _ = O.uniform_walks(off, col, None, n_walks, 50, L, 3)
+    walks[5, L // 2:] = -1                             # a walk that stopped early
+    walks[6, :] = -1
+    w_in0, w_out0 = random_tables(n, dim, 1)
+    U, V, loss_o, cnt_o, c, o, ng = oracle_step(w_in0.numpy(), w_out0.numpy(), walks, 50, w, K,
+                                                thr, alias, 0.025, 3)
+    a_dev = alias_to_device(thr, alias)
+    w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+    loss, cnt, pd, nd = run_step(w_in, w_out, torch.from_numpy(walks).to(DEV), 50, w, K, a_dev,
+                                 0.025, 3, B.GS_DETERMINISTIC)
+    # integer work: pairs and negative draws bit-exact
+    pd = pd.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+    if K > 0:
+        assert np.array_equal(nd.cpu().numpy().reshape(-1, K), ng)
+    assert cnt == cnt_o
+    assert abs(loss - loss_o) <= 2e-6 * abs(loss_o)
+    assert np.abs(w_in.cpu().numpy() - U).max() <= EMB_TOL
+    assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL
+    # and the step really moved the tables by much more than the tolerance
+    assert np.abs(V - w_out0.numpy()).max() > 20 * EMB_TOL
+    # bitwise reproducible
+    w_in2, w_out2 = w_in0.to(DEV), w_out0.to(DEV)
+    loss2, _, _, _ = run_step(w_in2, w_out2, torch.from_numpy(walks).to(DEV), 50, w, K, a_dev,
+                              0.025, 3, B.GS_DETERMINISTIC, dump=False)
+    assert torch.equal(w_in, w_in2) and torch.equal(w_out, w_out2) and loss == loss2
+
+
+def test_deterministic_step_hub_rows_with_thousands_of_contributions():
+    # a star: every walk alternates hub / leaf, so one output row collects most contributions
+    n = 400
+    leaves = torch.arange(1, n, dtype=torch.int64)
+    hub = torch.zeros(n - 1, dtype=torch.int64)
+    g = WL._csr_from_directed(torch.cat([hub, leaves]), torch.cat([leaves, hub]), n, False)
+    off, col = np_graph(g)
+    thr, alias = degree_alias(off)
+    walks, _ = O.uniform_walks(off, col, None, 512, 0, 40, 8)
+    w_in0, w_out0 = random_tables(n, 128, 2, scale=0.1)
+    U, V, loss_o, cnt_o, *_ = oracle_step(w_in0.numpy(), w_out0.numpy(), walks, 0, 5, 5, thr,
+                                          alias, 0.001, 8)
+    w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+    loss, cnt, _, _ = run_step(w_in, w_out, torch.from_numpy(walks).to(DEV), 0, 5, 5,
+                               alias_to_device(thr, alias), 0.001, 8, B.GS_DETERMINISTIC, dump=False)
+    assert cnt == cnt_o and abs(loss - loss_o) <= 2e-6 * abs(loss_o)
+    assert np.abs(w_in.cpu().numpy() - U).max() <= EMB_TOL
+    assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL
+
+
+@pytest.mark.parametrize("mode", [B.GS_HOGWILD, B.GS_HOGWILD_RED])
+def test_lock_free_modes_draw_the_same_pairs_and_negatives(tiny, mode):
+    _, g, off, col, thr, alias = tiny
+    L, w, K, dim = 10, 5, 5, 64
+    walks, _ = O.uniform_walks(off, col, None, 700, 0, L, 3)
+    walks[9, 4:] = -1
+    c, o, ng, n_pairs = O.expand_lists(walks, 0, w, K, thr, alias, 3)
+    w_in = torch.empty((g.n_nodes, dim), dtype=torch.float32, device=DEV)
+    w_out = torch.empty_like(w_in)
+    B.gs_init_embeddings(w_in, w_out, 0)
+    loss, cnt, pd, nd = run_step(w_in, w_out, torch.from_numpy(walks).to(DEV), 0, w, K,
+                                 alias_to_device(thr, alias), 0.025, 3, mode)
+    pd = pd.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+    assert np.array_equal(nd.cpu().numpy().reshape(-1, K), ng)
+    assert cnt == n_pairs
+    assert torch.isfinite(w_in).all() and torch.isfinite(w_out).all()
+    # from zero output vectors the first terms are ln 2 each; later ones are already smaller
+    unmasked = (ng[c >= 0] != o[c >= 0][:, None]).sum()
+    assert 0.9 * (cnt + unmasked) * np.log(2) < loss <= (cnt + unmasked) * np.log(2) * (1 + 1e-6)
+
+
+def test_lock_free_single_walk_equals_sequential_oracle():
+    # One walk = one warp running its positions in order: no races between warps.  Rows that
+    # repeat inside one chunk of targets are the only difference to strictly sequential SGD,
+    # so use a walk and negatives without repeats.
+    n, dim, L, w, K = 4000, 128, 12, 2, 3
+    rng = np.random.default_rng(4)
+    walk = rng.permutation(n)[:L].astype(np.int32)[None, :]
+    thr, alias = O.build_alias(np.ones(n), 1.0)
+    c, o, ng, _ = O.expand_lists(walk, 0, w, K, thr, alias, 12)
+    w_in0, w_out0 = random_tables(n, dim, 5)
+    U, V = w_in0.numpy().astype(np.float64), w_out0.numpy().astype(np.float64)
+    loss_o, cnt_o = O.sgns_seq_from_lists(U, V, c, o, ng, 2 * w, 0.05)
+    for mode in (B.GS_HOGWILD, B.GS_HOGWILD_RED):
+        w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+        loss, cnt, _, _ = run_step(w_in, w_out, torch.from_numpy(walk).to(DEV), 0, w, K,
+                                   alias_to_device(thr, alias), 0.05, 12, mode, dump=False)
+        assert cnt == cnt_o and abs(loss - loss_o) < 1e-5 * abs(loss_o)
+        # negatives may repeat across the chunk of one position; allow those few rows to differ
+        diff_in = np.abs(w_in.cpu().numpy() - U).max(axis=1)
+        diff_out = np.abs(w_out.cpu().numpy() - V).max(axis=1)
+        assert (diff_in > 1e-5).sum() <= 2 and (diff_out > 1e-5).sum() <= 4
+        assert np.abs(V - w_out0.numpy()).max() > 1e-3
+
+
+def test_sgns_step_edge_cases(tiny):
+    _, g, off, col, thr, alias = tiny
+    a_dev = alias_to_device(thr, alias)
+    w_in0, w_out0 = random_tables(g.n_nodes, 64, 3)
+    for mode in (B.GS_DETERMINISTIC, B.GS_HOGWILD):
+        w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+        # no walks at all
+        loss, cnt, _, _ = run_step(w_in, w_out, torch.empty((0, 10), dtype=torch.int32, device=DEV),
+                                   0, 5, 5, a_dev, 0.1, 0, mode, dump=False)
+        assert loss == 0.0 and cnt == 0
+        # walks made only of dead entries / single nodes: no pairs, tables untouched
+        walks = torch.full((33, 10), -1, dtype=torch.int32, device=DEV)
+        walks[:, 0] = torch.arange(33, dtype=torch.int32)
+        loss, cnt, pd, nd = run_step(w_in, w_out, walks, 0, 5, 5, a_dev, 0.1, 0, mode)
+        assert loss == 0.0 and cnt == 0 and (pd == -1).all() and (nd == -1).all()
+        assert torch.equal(w_in.cpu(), w_in0) and torch.equal(w_out.cpu(), w_out0)
+    with pytest.raises(B.GsError) as e:
+        B.gs_sgns_step(w_in, w_out, walks, 0, 33, 5, a_dev, 0.1, 0, 0)
+    assert e.value.status == -6
+
+
+# ---------------------------------------------------------------- epoch
+def test_epoch_tiny_deepwalk_deterministic_matches_oracle(tiny):
+    wl, g, off, col, thr, alias = tiny
+    n = g.n_nodes
+    U = O.init_rows(np.arange(n), wl.dim, 0)
+    V = np.zeros_like(U)
+    want = O.sgns_epoch(off, col, thr, alias, U, V, walks_per_node=1, L=wl.walk_len, w=wl.window,
+                        K=wl.n_neg, lr0=wl.lr0, schedule="linear", batch_walks=512, seed=0)
+    G = load(g)
+    w_in = torch.empty((n, wl.dim), dtype=torch.float32, device=DEV)
+    w_out = torch.empty_like(w_in)
+    B.gs_init_embeddings(w_in, w_out, 0)
+    res = B.gs_sgns_epoch(G, alias_to_device(thr, alias), w_in, w_out, walks_per_node=1,
+                          walk_len=wl.walk_len, window=wl.window, n_neg=wl.n_neg, lr0=wl.lr0,
+                          batch_walks=512, seed=0, mode=B.GS_DETERMINISTIC,
+                          lr_schedule=B.GS_LR_LINEAR)
+    assert res.pairs == want["pairs"] and res.steps == want["steps"]
+    assert res.batches == (n + 511) // 512
+    assert abs(res.loss_sum / res.pairs - want["loss_sum"] / want["pairs"]) <= LOSS_RTOL * want["loss_sum"] / want["pairs"]
+    assert np.abs(w_in.cpu().numpy() - U).max() <= EMB_TOL
+    assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL
+    # resume: two halves equal one run, bit for bit
+    w_in2 = torch.empty_like(w_in)
+    w_out2 = torch.empty_like(w_in)
+    B.gs_init_embeddings(w_in2, w_out2, 0)
+    kw = dict(walks_per_node=1, walk_len=wl.walk_len, window=wl.window, n_neg=wl.n_neg,
+              lr0=wl.lr0, batch_walks=512, seed=0, mode=B.GS_DETERMINISTIC,
+              lr_schedule=B.GS_LR_LINEAR)
+    r1 = B.gs_sgns_epoch(G, alias_to_device(thr, alias), w_in2, w_out2, first_batch=0, num_batches=7, **kw)
+    r2 = B.gs_sgns_epoch(G, alias_to_device(thr, alias), w_in2, w_out2, first_batch=7, **kw)
+    assert torch.equal(w_in, w_in2) and torch.equal(w_out, w_out2)
+    assert r1.pairs + r2.pairs == res.pairs
+
+
+def test_epoch_lock_free_loss_within_one_percent_of_deterministic(tiny):
+    wl, g, off, col, thr, alias = tiny
+    G = load(g)
+    a_dev = alias_to_device(thr, alias)
+    losses = {}
+    for mode in (B.GS_DETERMINISTIC, B.GS_HOGWILD, B.GS_HOGWILD_RED):
+        w_in = torch.empty((g.n_nodes, wl.dim), dtype=torch.float32, device=DEV)
+        w_out = torch.empty_like(w_in)
+        B.gs_init_embeddings(w_in, w_out, 0)
+        # several passes so that the tables move away from their start and the modes can differ
+        for ep in range(3):
+            res = B.gs_sgns_epoch(G, a_dev, w_in, w_out, walks_per_node=4, walk_len=wl.walk_len,
+                                  window=wl.window, n_neg=wl.n_neg, lr0=wl.lr0, batch_walks=512,
+                                  seed=ep, mode=mode)
+        losses[mode] = res.loss_sum / res.pairs
+    det = losses[B.GS_DETERMINISTIC]
+    assert det < 0.95 * (1 + wl.n_neg) * np.log(2)          # training did reduce the loss
+    for mode in (B.GS_HOGWILD, B.GS_HOGWILD_RED):
+        assert abs(losses[mode] - det) <= 0.01 * det, losses
+
+
+def test_epoch_node2vec_runs_and_counts_match_oracle(tiny):
+    wl, g, off, col, thr, alias = tiny
+    n = g.n_nodes
+    U = O.init_rows(np.arange(n), 64, 1)
+    V = np.zeros_like(U)
+    want = O.sgns_epoch(off, col, thr, alias, U, V, walks_per_node=1, L=12, w=3, K=3, lr0=0.025,
+                        schedule="constant", batch_walks=1000, seed=1, kind="node2vec", p=0.5,
+                        q=2.0, num_batches=4)
+    G = load(g)
+    w_in = torch.empty((n, 64), dtype=torch.float32, device=DEV)
+    w_out = torch.empty_like(w_in)
+    B.gs_init_embeddings(w_in, w_out, 1)
+    res = B.gs_sgns_epoch(G, alias_to_device(thr, alias), w_in, w_out, walks_per_node=1,
+                          walk_len=12, window=3, n_neg=3, lr0=0.025, batch_walks=1000, seed=1,
+                          mode=B.GS_DETERMINISTIC, walk_kind=B.GS_WALK_NODE2VEC, p=0.5, q=2.0,
+                          num_batches=4)
+    assert res.pairs == want["pairs"] and res.steps == want["steps"] and res.batches == 4
+    assert abs(res.loss_sum - want["loss_sum"]) <= LOSS_RTOL * want["loss_sum"]
+    assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL

@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the walk + SGNS hot path on synthetic power-law graphs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one mini-batch of the whole path: generate `batch_walks` random walks from the
+CSR graph, expand them to (center, context) pairs with negative draws, and apply the SGNS
+update to the embedding tables (lock-free mode for the large workloads).  The default
+workload is the 50M-node DeepWalk configuration.  Prints ONE JSON line.
+
+`value` is pair-updates/s with every input resident in HBM; `e2e` is the same metric with
+the step's host inputs (start nodes, pinned memory) copied in and its result (loss, pair
+count) copied out inside the timed region, through the same C-ABI calls.  `roofline` is
+for the SGNS kernel (the dominant one); `walk` gives the walk sampler's own figures.
+With --gpus N every rank runs an independent replica of the same workload on its own GPU
+(the path has no exchange step); the value is the sum over ranks divided by the slowest
+rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "sgns_pair_updates_per_s"
+UNIT = "pair-updates/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="deepwalk_large")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the node count (testing)")
+    ap.add_argument("--batch-walks", type=int, default=1 << 20)
+    ap.add_argument("--mode", default="hogwild", choices=["hogwild", "hogwild_red", "deterministic"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-sample-walks", type=int, default=8192)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiling runs)")
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------- helpers
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200", "-i", str(self.index)], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [l.split(",") for l in open(self.path).read().strip().splitlines() if l.strip()]
+            os.unlink(self.path)
+            sm = [float(r[0]) for r in rows]
+            out["sm_mhz"] = statistics.median(sm) if sm else None
+            out["sm_max_mhz"] = float(rows[0][1]) if rows else None
+            out["power_w_max"] = max(float(r[2]) for r in rows) if rows else None
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            out["reasons"] = [n for k, n in enumerate(names)
+                              if any("Active" in r[3 + k] and "Not" not in r[3 + k] for r in rows)]
+            out["samples"] = len(rows)
+        except Exception as e:          # clock sampling must never break the benchmark
+            out["error"] = str(e)
+        return out
+
+
+def measured_peak_gbs():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def algorithmic_bytes(pairs, positions, dim, n_neg):
+    """Row traffic the update must move: per pair 1+K output rows read and written plus K
+    alias entries; per center position one input row read and written plus its walk entry."""
+    return pairs * ((1 + n_neg) * 2 * 4 * dim + 8 * n_neg) + positions * (2 * 4 * dim + 4)
+
+
+def walk_bytes(steps, offsets64):
+    """Payload of a walk transition: two offsets, one column, one stored entry."""
+    return steps * ((16 if offsets64 else 8) + 4 + 4)
+
+
+def build_inputs(wl, scale, device):
+    from paper_2407_15452_b200 import binding as B
+    t0 = time.time()
+    g = wl.make_graph(device=device, scale=scale)
+    deg = g.degrees()
+    info = {"n_nodes": g.n_nodes, "n_edges": g.n_edges, "max_degree": int(deg.max()),
+            "frac_isolated": float((deg == 0).double().mean()), "graph_s": round(time.time() - t0, 1)}
+    t0 = time.time()
+    table = B.gs_build_alias(deg.cpu().numpy().astype(np.float64), 0.75)
+    info["alias_s"] = round(time.time() - t0, 1)
+    return g, table, info
+
+
+# ---------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(wl, off, col, table, n_walks, base, seed):
+    """Times the CPU oracle on `n_walks` walks of the workload: walks, pair/negative expansion,
+    sequential SGNS on the touched rows.  Returns (pairs, steps, seconds by stage)."""
+    from oracle import gs_oracle as O
+    thr = (table & np.uint64(0xFFFFFFFF)).astype(np.uint32)
+    alias = (table >> np.uint64(32)).astype(np.int32)
+    t0 = time.perf_counter()
+    if wl.walk_kind == "uniform":
+        walks, steps = O.uniform_walks(off, col, None, n_walks, base, wl.walk_len, seed)
+    else:
+        walks, steps, _ = O.node2vec_walks(off, col, None, n_walks, base, wl.walk_len, seed, wl.p, wl.q)
+    t1 = time.perf_counter()
+    c, o, ng, pairs = O.expand_lists(walks, base, wl.window, wl.n_neg, thr, alias, seed)
+    t2 = time.perf_counter()
+    # input data handling (not timed): renumber touched rows, materialise their start values
+    allv = np.concatenate([c, o, ng.ravel()])
+    ids = np.unique(allv[allv >= 0])
+    remap = lambda a: np.where(a >= 0, np.searchsorted(ids, np.maximum(a, 0)), -1).astype(np.int32)
+    cc, oo, nn = remap(c), remap(o), remap(ng)
+    U = O.init_rows(ids, wl.dim, seed)
+    V = np.zeros_like(U)
+    t3 = time.perf_counter()
+    O.sgns_seq_from_lists(U, V, cc, oo, nn, 2 * wl.window, wl.lr0)
+    t4 = time.perf_counter()
+    return pairs, steps, {"walk_s": t1 - t0, "expand_s": t2 - t1, "sgns_s": t4 - t3}
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle, as it stands, on the host cores."""
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    device = "cuda" if torch.cuda.is_available() else "cpu"
+    scale = args.scale if device == "cuda" else min(args.scale, 0.02)
+    g, table, info = build_inputs(wl, scale, device)
+    off = g.offsets.cpu().numpy().astype(np.int64)
+    col = g.cols.cpu().numpy()
+    del g
+    n = min(max(args.cpu_sample_walks // 8, 1), 1024)
+    for s in range(args.warmup):
+        oracle_sample(wl, off, col, table, n, s * n, wl.graph_seed)
+    pairs = steps = 0
+    secs = 0.0
+    for s in range(args.steps):
+        p, st, t = oracle_sample(wl, off, col, table, n, (args.warmup + s) * n, wl.graph_seed)
+        pairs += p
+        steps += st
+        secs += t["walk_s"] + t["expand_s"] + t["sgns_s"]
+    value = pairs / secs
+    sample = f"{n} walks per step (walks + pair/negative expansion + sequential SGNS on touched rows)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "gpu_launches": 0,
+        "config": {"workload": wl.name, "scale": scale, **info},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------- our arm
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_15452_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()                                            # fail loudly if the library is missing
+
+    g, table, info = build_inputs(wl, args.scale, dev)
+    n = g.n_nodes
+    G = B.gs_graph_load_csr(g.offsets, g.cols, B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    alias = torch.from_numpy(table.view(np.int64)).to(dev)
+    w_in = torch.empty((n, wl.dim), dtype=torch.float32, device=dev)
+    w_out = torch.empty_like(w_in)
+    seed = wl.graph_seed
+    B.gs_init_embeddings(w_in, w_out, seed)
+    mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,
+            "deterministic": B.GS_DETERMINISTIC}[args.mode]
+    kind = B.GS_WALK_UNIFORM if wl.walk_kind == "uniform" else B.GS_WALK_NODE2VEC
+    total_walks = n * wl.walks_per_node
+    bw = min(args.batch_walks, total_walks)
+    if mode == B.GS_DETERMINISTIC:
+        bw = min(bw, 512)
+    nb_total = (total_walks + bw - 1) // bw
+    ekw = dict(walks_per_node=wl.walks_per_node, walk_len=wl.walk_len, window=wl.window,
+               n_neg=wl.n_neg, lr0=wl.lr0, batch_walks=bw, seed=seed, mode=mode, walk_kind=kind,
+               p=wl.p, q=wl.q)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def batch_of(step):                                # replicas walk disjoint parts of the epoch
+        return (step * world + rank) % nb_total
+
+    # ---- device-resident timing -------------------------------------------------------
+    for s in range(args.warmup):
+        B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=batch_of(s), num_batches=1, **ekw)
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pairs = steps = walks_done = 0
+    loss = 0.0
+    ms_walk = ms_sgns = 0.0
+    ev0.record()
+    for s in range(args.steps):
+        b = batch_of(args.warmup + s)
+        r = B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=b, num_batches=1, **ekw)
+        pairs += r.pairs
+        steps += r.steps
+        loss += r.loss_sum
+        ms_walk += r.ms_walk
+        ms_sgns += r.ms_sgns
+        walks_done += min(bw, total_walks - b * bw)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms = ev0.elapsed_time(ev1)
+
+    # ---- end to end: host inputs in, result out, same C-ABI calls ---------------------------
+    e2e_pairs, e2e_s = 0, float("nan")
+    if not args.no_e2e:
+        h_starts = torch.empty(bw, dtype=torch.int32).pin_memory()
+        d_starts = torch.empty(bw, dtype=torch.int32, device=dev)
+        d_walks = torch.empty((bw, wl.walk_len), dtype=torch.int32, device=dev)
+        d_res = torch.zeros(2, dtype=torch.float64, device=dev)   # [loss, pair count as int64 bits]
+        d_loss = d_res[0:1]
+        d_cnt = d_res[1:2].view(torch.int64)
+        h_res = torch.zeros(2, dtype=torch.float64).pin_memory()
+
+        def e2e_step(step):
+            b = batch_of(step)
+            base = b * bw
+            cnt = min(bw, total_walks - base)
+            h_starts[:cnt] = (torch.arange(base, base + cnt, dtype=torch.int64) % n).to(torch.int32)
+            d_starts[:cnt].copy_(h_starts[:cnt], non_blocking=True)
+            d_res.zero_()
+            if kind == B.GS_WALK_UNIFORM:
+                B.gs_random_walks(G, d_starts, cnt, base, wl.walk_len, seed, out=d_walks)
+            else:
+                B.gs_node2vec_walks(G, d_starts, cnt, base, wl.walk_len, seed, wl.p, wl.q, out=d_walks)
+            B.gs_sgns_step(w_in, w_out, d_walks[:cnt], base, wl.window, wl.n_neg, alias, wl.lr0,
+                           seed, mode, d_loss, d_cnt)
+            h_res.copy_(d_res, non_blocking=True)
+            torch.cuda.synchronize()
+            return int(h_res[1:2].view(torch.int64).item())
+
+        for s in range(min(args.warmup, 2)):
+            e2e_step(args.warmup + args.steps + s)
+        barrier()
+        t0 = time.perf_counter()
+        for s in range(args.steps):
+            e2e_pairs += e2e_step(args.warmup + args.steps + 2 + s)
+        barrier()
+        e2e_s = time.perf_counter() - t0
+
+    # ---- max over ranks, sums over ranks ------------------------------------------------------
+    if world > 1:
+        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_s = t.tolist()
+        c = torch.tensor([pairs, steps, e2e_pairs], dtype=torch.int64, device=dev)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        pairs_all, steps_all, e2e_pairs_all = c.tolist()
+    else:
+        pairs_all, steps_all, e2e_pairs_all = pairs, steps, e2e_pairs
+
+    if rank == 0:
+        peak, peak_kind = measured_peak_gbs()
+        launches = args.steps                                     # SGNS launches on this rank
+        positions = steps + walks_done                            # walk entries = center positions
+        sgns_bytes = algorithmic_bytes(pairs, positions, wl.dim, wl.n_neg) / launches
+        sgns_ms = ms_sgns / launches
+        achieved = sgns_bytes / (sgns_ms * 1e-3) / 1e9
+        wbytes = walk_bytes(steps, wl.offsets64) / launches
+        walk_ms = ms_walk / launches
+        out = {
+            "metric": METRIC, "value": pairs_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": wl.name, "mode": args.mode, "batch_walks": bw,
+                       "walk_kind": wl.walk_kind, "walk_len": wl.walk_len, "window": wl.window,
+                       "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale,
+                       "l2": "tables (2 x n x dim x 4 B) and CSR far exceed the 126 MB L2; no flush",
+                       "multi_gpu": "replicas only", **info},
+            "gpu_launches": 2 * args.steps,
+            "mean_loss": loss / max(pairs, 1),
+            "walk_steps_per_s": steps_all / (ms * 1e-3),
+            "clocks": clocks,
+            "e2e": {"value": e2e_pairs_all / e2e_s, "unit": UNIT,
+                    "h2d_bytes_per_step": 4 * bw, "d2h_bytes_per_step": 16},
+            "roofline": {"bound": "hbm",
+                         "kernel": "sgns_hogwild_kernel" if mode else "sgns (coef+sort+apply)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (ms_sgns * 1e-3)},
+            "walk": {"kernel": "uniform_walk_kernel" if kind == B.GS_WALK_UNIFORM else "node2vec_walk_kernel",
+                     "walk_steps_per_s_kernel": steps / (ms_walk * 1e-3), "ms_per_launch": walk_ms,
+                     "payload_gbs": wbytes / (walk_ms * 1e-3) / 1e9,
+                     "payload_frac": wbytes / (walk_ms * 1e-3) / 1e9 / peak,
+                     "sector_gbs": (steps / launches) * 68 / (walk_ms * 1e-3) / 1e9},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            off = g.offsets.cpu().numpy().astype(np.int64)
+            col = g.cols.cpu().numpy()
+            p, st, t = oracle_sample(wl, off, col, table, args.cpu_sample_walks, 0, seed)
+            tot = t["walk_s"] + t["expand_s"] + t["sgns_s"]
+            out["cpu_baseline"] = {
+                "value": p / tot, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": f"first {args.cpu_sample_walks} walks of the workload: walks, pair/negative "
+                          f"expansion, sequential SGNS on the touched rows ({tot:.1f} s)",
+                "walk_steps_per_s": st / t["walk_s"], "sgns_pair_updates_per_s": p / t["sgns_s"]}
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    from paper_2407_15452_b200.workloads import WORKLOADS
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -381,9 +381,9 @@ sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
         const uint32_t key = keys[x];
         if (key >= n_nodes) continue;
         if (x > 0 && keys[x - 1] == key) continue;
-        Row<FPL> acc;
+        double acc[FPL];                 // a hub row can collect 10^5 terms: sum them in fp64
 #pragma unroll
-        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+        for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
         for (int64_t y = x; y < n_keys; y += 4) {
             float g[4];
             int32_t c[4];
@@ -408,13 +408,13 @@ sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
             for (int q = 0; q < 4; ++q)
                 if (c[q] >= 0) {
 #pragma unroll
-                    for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g[q], r[q].v[j], acc.v[j]);
+                    for (int j = 0; j < FPL; ++j) acc[j] += (double)(g[q] * r[q].v[j]);
                 }
             if (!more) break;
         }
         Row<FPL> row = row_load<FPL>(w_out, key, lane);
 #pragma unroll
-        for (int j = 0; j < FPL; ++j) row.v[j] = fmaf(-lr, acc.v[j], row.v[j]);
+        for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
         row_store<FPL>(w_out, key, lane, row);
     }
 }
@@ -433,18 +433,18 @@ sgns_apply_in_kernel(float *__restrict__ w_in, const float *__restrict__ GU,
         const uint32_t key = keys[x];
         if (key < n_nodes || key >= 2u * n_nodes) continue;
         if (x > 0 && keys[x - 1] == key) continue;
-        Row<FPL> acc;
+        double acc[FPL];
 #pragma unroll
-        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+        for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
         for (int64_t y = x; y < n_keys && keys[y] == key; ++y) {
             const Row<FPL> r = row_load<FPL>(GU, (int64_t)(vals[y] - n_slots), lane);
 #pragma unroll
-            for (int j = 0; j < FPL; ++j) acc.v[j] += r.v[j];
+            for (int j = 0; j < FPL; ++j) acc[j] += (double)r.v[j];
         }
         const int64_t c = (int64_t)(key - n_nodes);
         Row<FPL> row = row_load<FPL>(w_in, c, lane);
 #pragma unroll
-        for (int j = 0; j < FPL; ++j) row.v[j] = fmaf(-lr, acc.v[j], row.v[j]);
+        for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
         row_store<FPL>(w_in, c, lane, row);
     }
 }

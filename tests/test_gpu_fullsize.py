@@ -1,0 +1,126 @@
+"""GPU parity at the full sizes of the named workloads, in the launch shape bench.py times
+(one mini-batch of up to 2^20 walks from the middle of the epoch).
+
+The oracle cannot run a whole batch at these sizes in seconds, so: walks are compared on
+sampled ranges of walk ids computed one range at a time; counters are checked against
+properties that hold at any size; the synchronous SGNS step is compared on 512 walks with the
+oracle working on the touched rows only (ids renumbered one-to-one, row values read from the
+device before the step as input data)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gs_oracle as O
+from paper_2407_15452_b200 import binding as B
+from paper_2407_15452_b200 import workloads as WL
+from tests.helpers import compact_problem, unpack_alias
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+EMB_TOL = 1e-4
+
+
+def count_pairs(walks, w):
+    """Pairs formed by a batch of walks (pure counting on the device)."""
+    ok = walks >= 0
+    total = 0
+    for k in range(1, w + 1):
+        if k < walks.shape[1]:
+            total += 2 * int((ok[:, k:] & ok[:, :-k]).sum())
+    return total
+
+
+@pytest.mark.parametrize("name", ["deepwalk_medium", "node2vec_4m", "deepwalk_large", "rmat_billion"])
+def test_fullsize_workload(name):
+    wl = WL.WORKLOADS[name]
+    torch.cuda.empty_cache()
+    g = wl.make_graph(device=DEV)
+    n = g.n_nodes
+    assert n == wl.n_nodes
+    G = B.gs_graph_load_csr(g.offsets, g.cols, B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    deg = g.degrees()
+    assert G.info()["max_degree"] == int(deg.max())
+    off = g.offsets.cpu().numpy().astype(np.int64)
+    col = g.cols.cpu().numpy()
+    seed = wl.graph_seed
+
+    # ---- alias table: product builder == oracle builder, bit for bit, at full size
+    degf = deg.cpu().numpy().astype(np.float64)
+    table = B.gs_build_alias(degf, 0.75)
+    thr, alias = O.build_alias(degf, 0.75)
+    t2, a2 = unpack_alias(table)
+    assert np.array_equal(t2, thr) and np.array_equal(a2, alias)
+    del t2, a2, degf
+    a_dev = torch.from_numpy(table.view(np.int64)).to(DEV)
+
+    # ---- walks of one bench-sized batch from the middle of the epoch
+    total = n * wl.walks_per_node
+    bw = min(1 << 20, total)
+    base = ((total // bw) // 2) * bw
+    steps = torch.zeros(1, dtype=torch.int64, device=DEV)
+    caps = torch.zeros(1, dtype=torch.int64, device=DEV)
+    if wl.walk_kind == "uniform":
+        walks = B.gs_random_walks(G, None, bw, base, wl.walk_len, seed, steps=steps)
+    else:
+        walks = B.gs_node2vec_walks(G, None, bw, base, wl.walk_len, seed, wl.p, wl.q,
+                                    steps=steps, cap_hits=caps)
+    torch.cuda.synchronize()
+    assert int(steps.item()) == int((walks[:, 1:] >= 0).sum())
+    assert int(caps.item()) == 0
+    assert torch.equal(walks[:, 0].to(torch.int64),
+                       (torch.arange(base, base + bw, device=DEV) % n))
+    for lo in (0, bw // 2 - 333, bw - 1024):
+        if wl.walk_kind == "uniform":
+            want, _ = O.uniform_walks(off, col, None, 1024, base + lo, wl.walk_len, seed)
+        else:
+            want, _, _ = O.node2vec_walks(off, col, None, 1024, base + lo, wl.walk_len, seed, wl.p, wl.q)
+        assert np.array_equal(walks[lo:lo + 1024].cpu().numpy(), want), lo
+
+    # ---- tables; one lock-free step on the whole batch (makes the output rows non-zero)
+    w_in = torch.empty((n, wl.dim), dtype=torch.float32, device=DEV)
+    w_out = torch.empty_like(w_in)
+    B.gs_init_embeddings(w_in, w_out, seed)
+    probe = torch.from_numpy(np.random.default_rng(0).integers(0, n, 64)).to(DEV)
+    assert np.array_equal(w_in[probe].cpu().numpy().astype(np.float64),
+                          O.init_rows(probe.cpu().numpy(), wl.dim, seed))
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    B.gs_sgns_step(w_in, w_out, walks, base, wl.window, wl.n_neg, a_dev, wl.lr0, seed,
+                   B.GS_HOGWILD, loss, cnt)
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == count_pairs(walks, wl.window)
+    per_pair = loss.item() / cnt.item()
+    assert 0.3 < per_pair <= (1 + wl.n_neg) * np.log(2) * (1 + 1e-6)
+
+    # ---- synchronous step on 512 walks against the oracle on the touched rows
+    sub = walks[4096:4096 + 512].contiguous()
+    sub_h = sub.cpu().numpy()
+    c, o, ng, n_pairs = O.expand_lists(sub_h, base + 4096, wl.window, wl.n_neg, thr, alias, seed)
+    ids, cc, oo, nn = compact_problem(c, o, ng)
+    ids_dev = torch.from_numpy(ids).to(DEV)
+    U = w_in[ids_dev].cpu().numpy().astype(np.float64)
+    V = w_out[ids_dev].cpu().numpy().astype(np.float64)
+    assert np.abs(V).max() > 0
+    untouched = torch.from_numpy(np.setdiff1d(np.random.default_rng(1).integers(0, n, 4096), ids)).to(DEV)
+    before_in, before_out = w_in[untouched].clone(), w_out[untouched].clone()
+    loss_o, cnt_o = O.sgns_det_from_lists(U, V, cc, oo, nn, wl.lr0)
+    loss.zero_()
+    cnt.zero_()
+    pd = torch.empty((512, wl.walk_len, 2 * wl.window, 2), dtype=torch.int32, device=DEV)
+    nd = torch.empty((512, wl.walk_len, 2 * wl.window, wl.n_neg), dtype=torch.int32, device=DEV)
+    B.gs_sgns_step(w_in, w_out, sub, base + 4096, wl.window, wl.n_neg, a_dev, wl.lr0, seed,
+                   B.GS_DETERMINISTIC, loss, cnt, pd, nd)
+    torch.cuda.synchronize()
+    pd = pd.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+    assert np.array_equal(nd.cpu().numpy().reshape(-1, wl.n_neg), ng)
+    assert int(cnt.item()) == cnt_o == n_pairs
+    assert abs(loss.item() - loss_o) <= 2e-6 * abs(loss_o)
+    assert np.abs(w_in[ids_dev].cpu().numpy() - U).max() <= EMB_TOL
+    assert np.abs(w_out[ids_dev].cpu().numpy() - V).max() <= EMB_TOL
+    assert torch.equal(w_in[untouched], before_in) and torch.equal(w_out[untouched], before_out)
+
+    G.close()
+    del w_in, w_out, walks, g, a_dev
+    B.gs_release_workspace()
+    torch.cuda.empty_cache()

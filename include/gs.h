@@ -195,6 +195,42 @@ GS_API gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, in
                        double *d_loss_sum, int64_t *d_pair_count,
                        int32_t *d_pairs_dump, int32_t *d_negs_dump, void *stream);
 
+/*
+ * gs_sgns_step with GS_DETERMINISTIC for callers that must not allocate device
+ * memory: code running where cudaMalloc is forbidden or unsafe - inside a
+ * region whose memory budget is already fully handed out, in a real-time loop
+ * that cannot take the implicit device synchronisation of an allocation, or
+ * under a host framework that owns the allocator and forbids foreign calls to
+ * it.  (The paper has no counterpart; this is a convenience of this library.)
+ *
+ * Same arguments, arithmetic, launch order and result bits as gs_sgns_step in
+ * deterministic mode (without the dump arrays), but the grouping scratch comes
+ * from a fixed 32 MiB array that is part of the library image: every GPU that
+ * loads the library carries those 32 MiB until the process ends.  The call
+ * performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * Limit: the batch must need at most 32 MiB of scratch,
+ *   slots = n_walks * walk_len * (2*window*(1+n_neg) + 1)
+ *   bytes ~ 20 * slots + n_walks * walk_len * (4*dim + 12)  (+ < 1 % for the sort)
+ * e.g. up to about 380 walks of length 40 with window 5, 5 negatives, dim 128.
+ * Larger batches are rejected with GS_ERR_UNSUPPORTED and a message that
+ * states the bytes needed; nothing is launched in that case.
+ *
+ * The first call on each device looks up the array's device address (one
+ * cudaGetSymbolAddress with that device current); make that first call
+ * outside any stream capture.  All calls on a device share the one array and
+ * it keeps whatever the previous call left: every pass overwrites what it
+ * later reads, so stale contents are harmless, but two calls whose kernels
+ * overlap on the GPU (different streams, no ordering between them) race on
+ * the array and corrupt each other - order them.
+ */
+GS_API gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t dim,
+                                     const int32_t *d_walks, int64_t n_walks,
+                                     int64_t walk_id_base, int32_t walk_len, int32_t window,
+                                     int32_t n_neg, const uint64_t *d_alias, float lr,
+                                     uint64_t seed, double *d_loss_sum, int64_t *d_pair_count,
+                                     void *stream);
+
 #define GS_WALK_UNIFORM   0
 #define GS_WALK_NODE2VEC  1
 #define GS_LR_CONSTANT    0

@@ -26,7 +26,7 @@ GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
 EXPORTS = [
     "gs_last_error", "gs_graph_load_csr", "gs_graph_free", "gs_graph_info", "gs_build_alias",
     "gs_init_embeddings", "gs_random_walks", "gs_node2vec_walks", "gs_sgns_step",
-    "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group",
+    "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static",
 ]
 
 
@@ -193,6 +193,22 @@ def gs_sgns_step(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int,
         ctypes.c_float(lr), ctypes.c_uint64(seed), ctypes.c_int32(mode),
         _dev(loss_sum, torch.float64, "loss_sum", True), _dev(pair_count, torch.int64, "pair_count", True),
         _dev(pairs_dump, torch.int32, "pairs_dump", True), _dev(negs_dump, torch.int32, "negs_dump", True),
+        _stream()))
+
+
+def gs_sgns_step_static(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int, alias,
+                        lr: float, seed: int, loss_sum=None, pair_count=None):
+    """Deterministic SGNS step that allocates nothing on the device (fixed 32 MiB scratch inside
+    the library).  For callers that may not call cudaMalloc; small batches only - see gs.h."""
+    n_nodes, dim = w_in.shape
+    n_walks, walk_len = walks.shape
+    _check(lib().gs_sgns_step_static(
+        _dev(w_in, torch.float32, "w_in"), _dev(w_out, torch.float32, "w_out"),
+        ctypes.c_int64(n_nodes), ctypes.c_int32(dim), _dev(walks, torch.int32, "walks", n_walks == 0),
+        ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base), ctypes.c_int32(walk_len),
+        ctypes.c_int32(window), ctypes.c_int32(n_neg), _dev(alias, torch.int64, "alias", n_neg == 0),
+        ctypes.c_float(lr), ctypes.c_uint64(seed),
+        _dev(loss_sum, torch.float64, "loss_sum", True), _dev(pair_count, torch.int64, "pair_count", True),
         _stream()))
 
 

@@ -16,6 +16,8 @@
 // contribution index) key per target; the keys are radix-sorted, and one warp
 // per distinct row sums that row's contributions in index order and writes the
 // row once.  No floating-point atomics anywhere on this path.
+#include <mutex>
+
 #include "gs_common.cuh"
 
 namespace gs {
@@ -609,3 +611,139 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
 }
 
 }  // namespace gs
+
+
+// ---------------------------------------------------------------- fixed-scratch variant
+// Scratch of gs_sgns_step_static: part of the library image, so every GPU that loads the
+// library holds these bytes until the process exits.  Host code must not hand the symbol
+// itself to a kernel (on the host it is only a stand-in); it asks the runtime for the device
+// address once per device and passes that.
+#define GS_STATIC_SCRATCH_BYTES (32u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[GS_STATIC_SCRATCH_BYTES];
+
+namespace gs {
+
+static std::mutex g_static_mu;
+static unsigned char *g_static_ptr[64] = { nullptr };
+
+static gs_status static_scratch_address(unsigned char **out)
+{
+    int dev = 0;
+    GS_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) { set_error("device index %d not supported", dev); return GS_ERR_UNSUPPORTED; }
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void *p = nullptr;
+        GS_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_ptr[dev] = (unsigned char *)p;
+    }
+    *out = g_static_ptr[dev];
+    return GS_OK;
+}
+
+// Same kernels and the same order of launches as run_deterministic, with the scratch
+// carved out of the fixed array instead of the growing per-device cache.
+template <int FPL>
+static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scratch, cudaStream_t st)
+{
+    const int SL = 2 * a.w * (1 + a.K);
+    const int64_t n_pos = a.n_walks * a.L;
+    const int64_t n_slots = n_pos * SL;
+    const int64_t n_keys = n_slots + n_pos;
+    const size_t b_keys = align_up(sizeof(uint32_t) * (size_t)n_keys);
+    const size_t b_g = align_up(sizeof(float) * (size_t)n_slots);
+    const size_t b_gu = align_up(sizeof(float) * (size_t)n_pos * a.dim);
+    const size_t b_loss = align_up(sizeof(double) * (size_t)n_pos);
+    const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)n_pos);
+    const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)n_keys));
+    const size_t need = 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt;
+    if (n_keys > ((int64_t)1 << 30) || need > (size_t)GS_STATIC_SCRATCH_BYTES) {
+        set_error("gs_sgns_step_static: this batch needs %zu bytes of scratch, the fixed array has %u; "
+                  "pass fewer walks per call or use gs_sgns_step", need, GS_STATIC_SCRATCH_BYTES);
+        return GS_ERR_UNSUPPORTED;
+    }
+    // Every byte that is read below is written first by the pass before it (keys, g, GU, loss
+    // and pair counts by the coefficient pass for all slots; digit counts by the histogram
+    // pass for all tiles), so nothing left over from an earlier call can leak in.
+    char *p = (char *)scratch;
+    uint32_t *keysA = (uint32_t *)p; p += b_keys;
+    uint32_t *keysB = (uint32_t *)p; p += b_keys;
+    uint32_t *valsA = (uint32_t *)p; p += b_keys;
+    uint32_t *valsB = (uint32_t *)p; p += b_keys;
+    float *gbuf = (float *)p; p += b_g;
+    float *GU = (float *)p; p += b_gu;
+    double *loss_pos = (double *)p; p += b_loss;
+    int32_t *pairs_pos = (int32_t *)p; p += b_pairs;
+    uint32_t *counts = (uint32_t *)p;
+    {
+        const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
+        int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
+        const int64_t cap = (int64_t)sm_count() * 16;
+        if (blocks > cap) blocks = cap;
+        sgns_coef_kernel<FPL><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+            a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
+            (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
+            a.dump_pairs, a.dump_negs);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    uint32_t *ks = nullptr, *vs = nullptr;
+    radix_sort_pairs(keysA, valsA, keysB, valsB, (uint32_t)n_keys,
+                     bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
+    GS_CUDA_TRY(cudaGetLastError());
+    {
+        int64_t blocks = (n_keys + 7) / 8;
+        const int64_t cap = (int64_t)sm_count() * 8 * 8;
+        if (blocks > cap) blocks = cap;
+        sgns_apply_out_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
+            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr);
+        GS_CUDA_TRY(cudaGetLastError());
+        sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
+            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    if (a.loss || a.pairs) {
+        sgns_reduce_kernel<<<1, 1024, 0, st>>>(loss_pos, pairs_pos, n_pos, a.loss,
+                                               (long long *)a.pairs);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    return GS_OK;
+}
+
+}  // namespace gs
+
+extern "C" gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t dim,
+                                         const int32_t *d_walks, int64_t n_walks,
+                                         int64_t walk_id_base, int32_t walk_len, int32_t window,
+                                         int32_t n_neg, const uint64_t *d_alias, float lr,
+                                         uint64_t seed, double *d_loss_sum, int64_t *d_pair_count,
+                                         void *stream)
+{
+    using namespace gs;
+    if (!d_w_in || !d_w_out) { set_error("invalid argument: table pointer is NULL"); return GS_ERR_INVALID_ARG; }
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) { set_error("invalid argument: n_nodes must be in [1, 2^31)"); return GS_ERR_INVALID_ARG; }
+    if (n_walks < 0 || walk_id_base < 0) { set_error("invalid argument: negative n_walks or walk_id_base"); return GS_ERR_INVALID_ARG; }
+    if (n_walks > 0 && !d_walks) { set_error("invalid argument: d_walks is NULL"); return GS_ERR_INVALID_ARG; }
+    if (n_neg > 0 && !d_alias) { set_error("invalid argument: d_alias is NULL"); return GS_ERR_INVALID_ARG; }
+    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out) & 15) { set_error("invalid argument: tables must be 16-byte aligned"); return GS_ERR_INVALID_ARG; }
+    if (walk_len < 1 || walk_len > 1024 || window < 1 || window > 32 || n_neg < 0 || n_neg > 32 ||
+        2 * window * (1 + n_neg) > 512) {
+        set_error("gs_sgns_step_static: walk_len/window/n_neg outside the range gs_sgns_step accepts");
+        return GS_ERR_UNSUPPORTED;
+    }
+    if (n_walks == 0) return GS_OK;
+    unsigned char *scratch = nullptr;
+    gs_status s = static_scratch_address(&scratch);
+    if (s != GS_OK) return s;
+    SgnsArgs a = { d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len, window,
+                   n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr };
+    cudaStream_t st = (cudaStream_t)stream;
+    switch (dim) {
+        case 32: return run_deterministic_static<1>(a, scratch, st);
+        case 64: return run_deterministic_static<2>(a, scratch, st);
+        case 128: return run_deterministic_static<4>(a, scratch, st);
+        case 256: return run_deterministic_static<8>(a, scratch, st);
+        default:
+            set_error("dim %d not supported (32, 64, 128, 256)", dim);
+            return GS_ERR_UNSUPPORTED;
+    }
+}

@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--cpu-sample-walks", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiling runs)")
+    ap.add_argument("--stage", default="all", choices=["all", "walks"],
+                    help="'walks' times the walk sampler alone (no tables are allocated)")
     return ap.parse_args()
 
 
@@ -197,6 +199,59 @@ def run_reference(args, wl):
     }))
 
 
+# ---------------------------------------------------------------------------- walk sampler alone
+def run_walks_only(args, wl, g, G, info, dev):
+    """Times gs_random_walks / gs_node2vec_walks alone on batches of the workload (1 GPU)."""
+    import torch
+    from paper_2407_15452_b200 import binding as B
+    n = g.n_nodes
+    total_walks = n * wl.walks_per_node
+    bw = min(args.batch_walks, total_walks)
+    nb_total = (total_walks + bw - 1) // bw
+    out = torch.empty((bw, wl.walk_len), dtype=torch.int32, device=dev)
+    steps = torch.zeros(1, dtype=torch.int64, device=dev)
+
+    def run(b):
+        base = (b % nb_total) * bw
+        cnt = min(bw, total_walks - base)
+        if wl.walk_kind == "uniform":
+            B.gs_random_walks(G, None, cnt, base, wl.walk_len, wl.graph_seed, out=out, steps=steps)
+        else:
+            B.gs_node2vec_walks(G, None, cnt, base, wl.walk_len, wl.graph_seed, wl.p, wl.q, out=out,
+                                steps=steps)
+
+    for s in range(args.warmup):
+        run(s)
+    torch.cuda.synchronize()
+    steps.zero_()
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for s in range(args.steps):
+        run(args.warmup + s)
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    st = int(steps.item())
+    peak, peak_kind = measured_peak_gbs()
+    payload = walk_bytes(st, wl.offsets64) / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "walk_steps_per_s", "value": st / (ms * 1e-3), "unit": "walk-steps/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "data": "synthetic", "gpu_launches": args.steps, "clocks": clocks,
+        "config": {"workload": wl.name, "stage": "walks", "batch_walks": bw, "walk_kind": wl.walk_kind,
+                   "walk_len": wl.walk_len, "scale": args.scale, **info},
+        "roofline": {"bound": "hbm", "kernel": "uniform_walk_vec_kernel" if wl.walk_kind == "uniform" else "node2vec_walk_kernel",
+                     "achieved": payload, "peak": peak, "unit": "GB/s", "frac": payload / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "sector_gbs": st * 68 / (ms * 1e-3) / 1e9,
+                     "sector_frac": st * 68 / (ms * 1e-3) / 1e9 / peak},
+    }))
+
+
 # ---------------------------------------------------------------------------- our arm
 def run_ours(args, wl):
     import torch
@@ -215,6 +270,8 @@ def run_ours(args, wl):
     g, table, info = build_inputs(wl, args.scale, dev)
     n = g.n_nodes
     G = B.gs_graph_load_csr(g.offsets, g.cols, B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    if args.stage == "walks":
+        return run_walks_only(args, wl, g, G, info, dev)
     alias = torch.from_numpy(table.view(np.int64)).to(dev)
     w_in = torch.empty((n, wl.dim), dtype=torch.float32, device=dev)
     w_out = torch.empty_like(w_in)

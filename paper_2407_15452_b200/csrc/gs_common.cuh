@@ -70,11 +70,27 @@ __device__ __forceinline__ uint4 draw(uint64_t seed, uint64_t id, uint32_t step,
                          make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)));
 }
 
-// CSR offset of node v for either offset width
-template <typename OffT>
-__device__ __forceinline__ int64_t load_off(const OffT *off, int64_t v)
+// Read-only loads for isolated random accesses (a CSR offset, a column, an alias cell).
+// By default a miss pulls a whole 128-byte line out of DRAM; the 64-byte prefetch-size hint
+// halves that for data whose neighbours will not be used.  The line still allocates in L1, so
+// the second offset of a pair hits there.
+__device__ __forceinline__ int32_t ld_random(const int32_t *p)
 {
-    return (int64_t)__ldg(off + v);
+    int32_t v;
+    asm("ld.global.nc.L2::64B.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ int64_t ld_random(const int64_t *p)
+{
+    long long v;
+    asm("ld.global.nc.L2::64B.s64 %0, [%1];" : "=l"(v) : "l"(p));
+    return (int64_t)v;
+}
+__device__ __forceinline__ uint64_t ld_random(const uint64_t *p)
+{
+    unsigned long long v;
+    asm("ld.global.nc.L2::64B.u64 %0, [%1];" : "=l"(v) : "l"(p));
+    return (uint64_t)v;
 }
 
 }  // namespace gs

@@ -104,10 +104,42 @@ __device__ __forceinline__ float warp_sum(float s)
     return s;                       // identical bits on every lane (commutative pairs)
 }
 
-__device__ __forceinline__ float sigmoidf_exact(float x) { return 1.0f / (1.0f + expf(-x)); }
-__device__ __forceinline__ float softplusf(float x)
+// sigmoid(z) and softplus(z) = log(1 + e^z) from one exponential, stable for either sign
+__device__ __forceinline__ void sigmoid_softplus(float z, float &sig, float &sp)
 {
-    return fmaxf(x, 0.f) + log1pf(expf(-fabsf(x)));
+    const float e = expf(-fabsf(z));
+    const float r = 1.0f / (1.0f + e);
+    sig = z >= 0.f ? r : e * r;
+    sp = fmaxf(z, 0.f) + log1pf(e);
+}
+
+// The dot products f[0..TCH) of a chunk are known to every lane.  Lane k < TCH evaluates the
+// transcendentals of target k only (the other lanes idle through those few instructions):
+// for a context (label 1) the term is softplus(-f) and g = sigmoid(f) - 1 = -sigmoid(-f); for a
+// negative softplus(f) and g = sigmoid(f).  Returns this lane's g (0 for an absent target) and
+// adds its loss term to `loss`.
+template <int N>
+__device__ __forceinline__ float lane_coefficient(const float (&f)[N], int lane, int32_t my_id,
+                                                  bool my_is_ctx, float &loss)
+{
+    float mf = f[0];
+#pragma unroll
+    for (int k = 1; k < N; ++k) mf = lane == k ? f[k] : mf;
+    float g = 0.f;
+    if (lane < N && my_id >= 0) {
+        float sig, sp;
+        sigmoid_softplus(my_is_ctx ? -mf : mf, sig, sp);
+        g = my_is_ctx ? -sig : sig;
+        loss += sp;
+    }
+    return g;
+}
+
+__device__ __forceinline__ double warp_sum_double(double s)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return s;
 }
 
 // ---------------------------------------------------------------- target list of one position
@@ -146,11 +178,11 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
                 if (valid) {
                     const uint4 r = draw(seed, id, (uint32_t)(i * S + s), TAG_NEGATIVE, (uint32_t)m);
                     const uint32_t j0 = __umulhi(r.x, n_alias);
-                    const uint64_t e0 = __ldg(alias + j0);
+                    const uint64_t e0 = ld_random(alias + j0);
                     n0 = r.y < (uint32_t)e0 ? (int32_t)j0 : (int32_t)(e0 >> 32);
                     if (two) {
                         const uint32_t j1 = __umulhi(r.z, n_alias);
-                        const uint64_t e1 = __ldg(alias + j1);
+                        const uint64_t e1 = ld_random(alias + j1);
                         n1 = r.w < (uint32_t)e1 ? (int32_t)j1 : (int32_t)(e1 >> 32);
                     }
                 }
@@ -177,8 +209,8 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
 }
 
 // ---------------------------------------------------------------- lock-free kernel
-template <int FPL, bool RED>
-__global__ void __launch_bounds__(SGNS_WARPS * 32)
+template <int FPL, bool RED, int MINB>
+__global__ void __launch_bounds__(SGNS_WARPS * 32, MINB)
 sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
                     const int32_t *__restrict__ walks, int64_t n_walks, int64_t walk_id_base,
                     int32_t L, int32_t w, int32_t K, const uint64_t *__restrict__ alias,
@@ -212,8 +244,8 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
             Row<FPL> acc;
 #pragma unroll
             for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
-            float loss = 0.f;
-            int kk = 0;                                  // (base + k) mod T1, tracked incrementally
+            float loss = 0.f;                            // this lane's share of the position's loss
+            int kk = 0;                                  // base mod T1, tracked incrementally
             for (int base = 0; base < SL; base += TCH) {
                 int32_t ids[TCH];
                 bool any = false;
@@ -232,14 +264,14 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
                     for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
 #pragma unroll
                     for (int k = 0; k < TCH; ++k) f[k] = warp_sum(f[k]);
+                    int my_kt = kk + (lane < TCH ? lane : 0);
+                    while (my_kt >= T1) my_kt -= T1;
+                    const int32_t my_id = (lane < TCH && base + lane < SL) ? tgt[base + lane] : -1;
+                    const float my_g = lane_coefficient<TCH>(f, lane, my_id, my_kt == 0, loss);
 #pragma unroll
                     for (int k = 0; k < TCH; ++k) {
-                        int kt = kk + k;
-                        while (kt >= T1) kt -= T1;
+                        const float g = __shfl_sync(0xffffffffu, my_g, k);
                         if (ids[k] >= 0) {
-                            const bool is_ctx = kt == 0;
-                            const float g = sigmoidf_exact(f[k]) - (is_ctx ? 1.f : 0.f);
-                            loss += softplusf(is_ctx ? -f[k] : f[k]);
                             const float step = -lr * g;
                             Row<FPL> delta;
 #pragma unroll
@@ -271,6 +303,7 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
             loss_acc += (double)loss;
         }
     }
+    loss_acc = warp_sum_double(loss_acc);
     if (lane == 0) {
         if (loss_out && pair_acc) atomicAdd(loss_out, loss_acc);
         if (pairs_out && pair_acc) atomicAdd(pairs_out, pair_acc);
@@ -337,27 +370,28 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
                 for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
 #pragma unroll
                 for (int k = 0; k < TCH; ++k) f[k] = warp_sum(f[k]);
+                int my_kt = kk + (lane < TCH ? lane : 0);
+                while (my_kt >= T1) my_kt -= T1;
+                const bool mine = lane < TCH && base + lane < SL;
+                const int32_t my_id = mine ? tgt[base + lane] : -1;
+                const float my_g = lane_coefficient<TCH>(f, lane, my_id, my_kt == 0, loss);
+                if (mine) {
+                    kp[base + lane] = my_id >= 0 ? (uint32_t)my_id : invalid;
+                    gp[base + lane] = my_g;
+                }
 #pragma unroll
                 for (int k = 0; k < TCH; ++k) {
-                    int kt = kk + k;
-                    while (kt >= T1) kt -= T1;
-                    float g = 0.f;
+                    const float g = __shfl_sync(0xffffffffu, my_g, k);
                     if (ids[k] >= 0) {
-                        const bool is_ctx = kt == 0;
-                        g = sigmoidf_exact(f[k]) - (is_ctx ? 1.f : 0.f);
-                        loss += softplusf(is_ctx ? -f[k] : f[k]);
 #pragma unroll
                         for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g, rows[k].v[j], acc.v[j]);
-                    }
-                    if (lane == k && base + k < SL) {
-                        kp[base + k] = ids[k] >= 0 ? (uint32_t)ids[k] : invalid;
-                        gp[base + k] = g;
                     }
                 }
                 kk += TCH;
                 while (kk >= T1) kk -= T1;
             }
         }
+        loss = warp_sum(loss);                     // lane-local shares, fixed butterfly order
         row_store<FPL>(GU, pos, lane, acc);
         if (lane == 0) {
             keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
@@ -492,12 +526,12 @@ struct SgnsArgs {
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
-template <int FPL, bool RED>
-static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
+template <int FPL, bool RED, int MINB>
+static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
     const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(a.L + SL);
-    auto kern = sgns_hogwild_kernel<FPL, RED>;
+    auto kern = sgns_hogwild_kernel<FPL, RED, MINB>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -512,6 +546,14 @@ static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
         a.dump_negs);
     GS_CUDA_TRY(cudaGetLastError());
     return GS_OK;
+}
+
+// Resident blocks per SM asked of the compiler: 5 blocks of 4 warps (96 registers per thread)
+// measured best for rows of up to 128 floats; wider rows need the registers.
+template <int FPL, bool RED>
+static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
+{
+    return run_hogwild_b<FPL, RED, (FPL <= 4 ? 5 : 4)>(a, st);
 }
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }

@@ -141,15 +141,65 @@ uniform_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ co
         W[0] = cur;
         int32_t t = 0;
         for (; t + 1 < L; ++t) {
-            const int64_t o0 = load_off(off, cur), o1 = load_off(off, (int64_t)cur + 1);
+            const int64_t o0 = ld_random(off + cur), o1 = ld_random(off + cur + 1);
             const uint32_t deg = (uint32_t)(o1 - o0);
             if (deg == 0) break;
             const uint4 r = draw(seed, id, (uint32_t)t, TAG_UNIFORM, 0);
-            cur = __ldg(col + o0 + (int64_t)__umulhi(r.x, deg));
+            cur = ld_random(col + o0 + (int64_t)__umulhi(r.x, deg));
             W[t + 1] = cur;
             ++my_steps;
         }
         for (int32_t s = t + 1; s < L; ++s) W[s] = -1;
+    }
+    if (steps_out) {
+        for (int o = 16; o > 0; o >>= 1) my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
+        if ((threadIdx.x & 31) == 0 && my_steps) atomicAdd(steps_out, (unsigned long long)my_steps);
+    }
+}
+
+// Same walks, stored 32 bytes at a time: entries are collected four per int4 and two int4
+// leave together, so the output reaches L2 as whole sectors instead of 4-byte fragments
+// (fragments that are evicted before their sector is complete cost a DRAM read to fill and a
+// second write).  Needs L % 4 == 0 and a 16-byte aligned output.
+template <typename OffT>
+__global__ void __launch_bounds__(256, 6)
+uniform_walk_vec_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
+                        const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
+                        int64_t walk_id_base, int32_t L, uint64_t seed,
+                        int32_t *__restrict__ walks, unsigned long long *steps_out)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int quads = L >> 2;
+    unsigned int my_steps = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
+        const uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
+        bool alive = true;
+        int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
+        int4 pend = make_int4(0, 0, 0, 0);
+        for (int q = 0; q < quads; ++q) {
+            int32_t v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int e = 4 * q + k;                 // entry index; entry 0 is the start node
+                if (e > 0 && alive) {
+                    const int64_t o0 = ld_random(off + cur), o1 = ld_random(off + cur + 1);
+                    const uint32_t deg = (uint32_t)(o1 - o0);
+                    if (deg == 0) {
+                        alive = false;
+                    } else {
+                        const uint4 r = draw(seed, id, (uint32_t)(e - 1), TAG_UNIFORM, 0);
+                        cur = ld_random(col + o0 + (int64_t)__umulhi(r.x, deg));
+                        ++my_steps;
+                    }
+                }
+                v[k] = alive ? cur : -1;
+            }
+            const int4 now = make_int4(v[0], v[1], v[2], v[3]);
+            if (q & 1) { W4[q - 1] = pend; W4[q] = now; }
+            else if (q == quads - 1) W4[q] = now;
+            else pend = now;
+        }
     }
     if (steps_out) {
         for (int o = 16; o > 0; o >>= 1) my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
@@ -166,14 +216,13 @@ gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t
     int64_t blocks = (n_walks + threads - 1) / threads;
     const int64_t cap = (int64_t)sm_count() * 8 * 16;
     if (blocks > cap) blocks = cap;
-    if (g->offsets64)
-        uniform_walk_kernel<int64_t><<<(unsigned)blocks, threads, 0, st>>>(
-            (const int64_t *)g->d_offsets, g->d_cols, starts, g->n_nodes, n_walks, base, L, seed,
-            walks, steps);
-    else
-        uniform_walk_kernel<int32_t><<<(unsigned)blocks, threads, 0, st>>>(
-            (const int32_t *)g->d_offsets, g->d_cols, starts, g->n_nodes, n_walks, base, L, seed,
-            walks, steps);
+    const bool vec = (L % 4 == 0) && (((uintptr_t)walks & 15) == 0);
+#define GS_UW(KERNEL, T)                                                                        \
+    KERNEL<T><<<(unsigned)blocks, threads, 0, st>>>((const T *)g->d_offsets, g->d_cols, starts, \
+                                                    g->n_nodes, n_walks, base, L, seed, walks, steps)
+    if (g->offsets64) { if (vec) GS_UW(uniform_walk_vec_kernel, int64_t); else GS_UW(uniform_walk_kernel, int64_t); }
+    else { if (vec) GS_UW(uniform_walk_vec_kernel, int32_t); else GS_UW(uniform_walk_kernel, int32_t); }
+#undef GS_UW
     GS_CUDA_TRY(cudaGetLastError());
     return GS_OK;
 }
@@ -190,9 +239,9 @@ __device__ __forceinline__ bool row_contains(const int32_t *__restrict__ col, in
     const int64_t end = hi;
     while (lo < hi) {
         const int64_t mid = lo + ((hi - lo) >> 1);
-        if (__ldg(col + mid) < x) lo = mid + 1; else hi = mid;
+        if (ld_random(col + mid) < x) lo = mid + 1; else hi = mid;
     }
-    return lo < end && __ldg(col + lo) == x;
+    return lo < end && ld_random(col + lo) == x;
 }
 
 // G lanes per walk; lane k of a group evaluates rejection round base + k.
@@ -224,13 +273,13 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
         if (sub == 0) W[0] = cur;
         int32_t t = 0;
         for (; t + 1 < L; ++t) {
-            const int64_t o0 = load_off(off, cur), o1 = load_off(off, (int64_t)cur + 1);
+            const int64_t o0 = ld_random(off + cur), o1 = ld_random(off + cur + 1);
             const uint32_t deg = (uint32_t)(o1 - o0);
             if (deg == 0) break;
             int32_t nxt;
             if (t == 0) {
                 const uint4 r = draw(seed, id, 0u, TAG_NODE2VEC, 0);
-                nxt = __ldg(col + o0 + (int64_t)__umulhi(r.x, deg));
+                nxt = ld_random(col + o0 + (int64_t)__umulhi(r.x, deg));
             } else {
                 nxt = -1;
                 for (int32_t rbase = 0;; rbase += G) {
@@ -240,7 +289,7 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
                     bool acc = false;
                     if (live) {
                         const uint4 r = draw(seed, id, (uint32_t)t, TAG_NODE2VEC, (uint32_t)s);
-                        x = __ldg(col + o0 + (int64_t)__umulhi(r.x, deg));
+                        x = ld_random(col + o0 + (int64_t)__umulhi(r.x, deg));
                         const unsigned long long r1 = r.y;
                         if (x == prev) acc = r1 < T.t_prev;
                         else if (r1 < t_lo) acc = true;          // accepted in either class

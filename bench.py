@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--cpu-sample-walks", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiling runs)")
+    ap.add_argument("--no-walk-index", action="store_true",
+                    help="walk over the plain CSR (two random reads per transition)")
     ap.add_argument("--stage", default="all", choices=["all", "walks"],
                     help="'walks' times the walk sampler alone (no tables are allocated)")
     return ap.parse_args()
@@ -118,9 +120,17 @@ def algorithmic_bytes(pairs, positions, dim, n_neg):
     return pairs * ((1 + n_neg) * 2 * 4 * dim + 8 * n_neg) + positions * (2 * 4 * dim + 4)
 
 
-def walk_bytes(steps, offsets64):
-    """Payload of a walk transition: two offsets, one column, one stored entry."""
-    return steps * ((16 if offsets64 else 8) + 4 + 4)
+def walk_bytes(steps, offsets64, indexed=False):
+    """Payload of a walk transition: two offsets and one column (or one 16-byte index record),
+    plus the stored entry."""
+    return steps * ((16 if indexed else (16 if offsets64 else 8) + 4) + 4)
+
+
+def walk_granule_bytes(steps, indexed=False):
+    """DRAM cannot move less than a 64-byte granule per isolated random read (measured: the
+    64-byte fetch hint is the smallest the L2 honours): one granule per record, or one for the
+    offset pair and one for the column, plus the 4 bytes stored."""
+    return steps * ((64 if indexed else 128) + 4)
 
 
 def build_inputs(wl, scale, device):
@@ -199,6 +209,12 @@ def run_reference(args, wl):
     }))
 
 
+def walk_kernel_name(wl, indexed):
+    if wl.walk_kind != "uniform":
+        return "node2vec_walk_kernel"
+    return "uniform_walk_index_kernel" if indexed else "uniform_walk_vec_kernel"
+
+
 # ---------------------------------------------------------------------------- walk sampler alone
 def run_walks_only(args, wl, g, G, info, dev):
     """Times gs_random_walks / gs_node2vec_walks alone on batches of the workload (1 GPU)."""
@@ -236,7 +252,9 @@ def run_walks_only(args, wl, g, G, info, dev):
     ms = ev0.elapsed_time(ev1)
     st = int(steps.item())
     peak, peak_kind = measured_peak_gbs()
-    payload = walk_bytes(st, wl.offsets64) / (ms * 1e-3) / 1e9
+    indexed = "walk_index_bytes" in info
+    payload = walk_bytes(st, wl.offsets64, indexed) / (ms * 1e-3) / 1e9
+    granule = walk_granule_bytes(st, indexed) / (ms * 1e-3) / 1e9
     print(json.dumps({
         "metric": "walk_steps_per_s", "value": st / (ms * 1e-3), "unit": "walk-steps/s", "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
@@ -244,11 +262,10 @@ def run_walks_only(args, wl, g, G, info, dev):
         "data": "synthetic", "gpu_launches": args.steps, "clocks": clocks,
         "config": {"workload": wl.name, "stage": "walks", "batch_walks": bw, "walk_kind": wl.walk_kind,
                    "walk_len": wl.walk_len, "scale": args.scale, **info},
-        "roofline": {"bound": "hbm", "kernel": "uniform_walk_vec_kernel" if wl.walk_kind == "uniform" else "node2vec_walk_kernel",
+        "roofline": {"bound": "hbm", "kernel": walk_kernel_name(wl, indexed),
                      "achieved": payload, "peak": peak, "unit": "GB/s", "frac": payload / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": None,
-                     "sector_gbs": st * 68 / (ms * 1e-3) / 1e9,
-                     "sector_frac": st * 68 / (ms * 1e-3) / 1e9 / peak},
+                     "granule_gbs": granule, "granule_frac": granule / peak},
     }))
 
 
@@ -257,6 +274,7 @@ def run_ours(args, wl):
     import torch
     import torch.distributed as dist
     from paper_2407_15452_b200 import binding as B
+    from paper_2407_15452_b200 import replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -269,7 +287,11 @@ def run_ours(args, wl):
 
     g, table, info = build_inputs(wl, args.scale, dev)
     n = g.n_nodes
-    G = B.gs_graph_load_csr(g.offsets, g.cols, B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    flags = B.GS_VALIDATE | B.GS_REQUIRE_SORTED
+    if wl.walk_kind == "uniform" and not args.no_walk_index:
+        flags |= B.GS_BUILD_WALK_INDEX                  # 16 B per CSR entry, one read per transition
+        info["walk_index_bytes"] = 16 * g.n_edges
+    G = B.gs_graph_load_csr(g.offsets, g.cols, flags)
     if args.stage == "walks":
         return run_walks_only(args, wl, g, G, info, dev)
     alias = torch.from_numpy(table.view(np.int64)).to(dev)
@@ -296,7 +318,7 @@ def run_ours(args, wl):
             torch.cuda.synchronize()
 
     def batch_of(step):                                # replicas walk disjoint parts of the epoch
-        return (step * world + rank) % nb_total
+        return replicas.batch_of(step, rank, world, nb_total)
 
     # ---- device-resident timing -------------------------------------------------------
     for s in range(args.warmup):
@@ -362,15 +384,8 @@ def run_ours(args, wl):
         e2e_s = time.perf_counter() - t0
 
     # ---- max over ranks, sums over ranks ------------------------------------------------------
-    if world > 1:
-        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_s = t.tolist()
-        c = torch.tensor([pairs, steps, e2e_pairs], dtype=torch.int64, device=dev)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        pairs_all, steps_all, e2e_pairs_all = c.tolist()
-    else:
-        pairs_all, steps_all, e2e_pairs_all = pairs, steps, e2e_pairs
+    (ms, e2e_s), (pairs_all, steps_all, e2e_pairs_all) = replicas.reduce_timing(
+        [ms, e2e_s], [pairs, steps, e2e_pairs], device=dev)
 
     if rank == 0:
         peak, peak_kind = measured_peak_gbs()
@@ -379,7 +394,9 @@ def run_ours(args, wl):
         sgns_bytes = algorithmic_bytes(pairs, positions, wl.dim, wl.n_neg) / launches
         sgns_ms = ms_sgns / launches
         achieved = sgns_bytes / (sgns_ms * 1e-3) / 1e9
-        wbytes = walk_bytes(steps, wl.offsets64) / launches
+        indexed = "walk_index_bytes" in info
+        wbytes = walk_bytes(steps, wl.offsets64, indexed) / launches
+        gbytes = walk_granule_bytes(steps, indexed) / launches
         walk_ms = ms_walk / launches
         out = {
             "metric": METRIC, "value": pairs_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -402,11 +419,12 @@ def run_ours(args, wl):
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}", "traffic": None,
                          "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (ms_sgns * 1e-3)},
-            "walk": {"kernel": "uniform_walk_kernel" if kind == B.GS_WALK_UNIFORM else "node2vec_walk_kernel",
+            "walk": {"kernel": walk_kernel_name(wl, indexed),
                      "walk_steps_per_s_kernel": steps / (ms_walk * 1e-3), "ms_per_launch": walk_ms,
                      "payload_gbs": wbytes / (walk_ms * 1e-3) / 1e9,
                      "payload_frac": wbytes / (walk_ms * 1e-3) / 1e9 / peak,
-                     "sector_gbs": (steps / launches) * 68 / (walk_ms * 1e-3) / 1e9},
+                     "granule_gbs": gbytes / (walk_ms * 1e-3) / 1e9,
+                     "granule_frac": gbytes / (walk_ms * 1e-3) / 1e9 / peak},
         }
         if not args.no_cpu_baseline and world == 1:
             off = g.offsets.cpu().numpy().astype(np.int64)

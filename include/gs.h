@@ -62,6 +62,7 @@ typedef struct gs_graph gs_graph;
 
 #define GS_VALIDATE        1u   /* check offsets and column range on the device    */
 #define GS_REQUIRE_SORTED  2u   /* additionally require strictly increasing rows   */
+#define GS_BUILD_WALK_INDEX 4u  /* build the per-entry walk index (implies GS_VALIDATE) */
 
 /*
  * Wraps a CSR graph that already lives in device memory (the whole topology
@@ -73,13 +74,19 @@ typedef struct gs_graph gs_graph;
  * WAITS for the result (one small device-to-host read).  node2vec needs
  * GS_REQUIRE_SORTED rows.  On error *out is NULL; GS_ERR_BAD_CSR /
  * GS_ERR_UNSORTED_ADJ name the first offending row in gs_last_error().
+ * With GS_BUILD_WALK_INDEX the handle also owns 16 bytes of device memory per
+ * CSR entry (allocated here, freed by gs_graph_free; GS_ERR_OOM if it does not
+ * fit): entry e records cols[e] with that node's degree and offset, so that a
+ * uniform-walk transition needs one random read instead of two.  Walks are
+ * identical with or without the index.
  */
 GS_API gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges,
                             const void *d_offsets, int32_t offsets_are_64bit,
                             const int32_t *d_cols, uint32_t flags,
                             void *stream, gs_graph **out);
 
-/* Frees the handle only; the CSR arrays stay the caller's. NULL is allowed. */
+/* Frees the handle (and its walk index, waiting for the device if there is one); the CSR
+ * arrays stay the caller's. NULL is allowed. */
 GS_API void gs_graph_free(gs_graph *g);
 
 /* max_degree is -1 if the graph was loaded without GS_VALIDATE. */

@@ -5,4 +5,4 @@
 inputs.  Importing the package loads nothing native; the binding loads the
 shared library on first use and raises if it has not been built.
 """
-__all__ = ["binding", "workloads", "build"]
+__all__ = ["binding", "workloads", "build", "replicas"]

@@ -18,7 +18,7 @@ import torch
 _LIB_PATH = Path(__file__).resolve().parent / "libgs_b200.so"
 _lib = None
 
-GS_VALIDATE, GS_REQUIRE_SORTED = 1, 2
+GS_VALIDATE, GS_REQUIRE_SORTED, GS_BUILD_WALK_INDEX = 1, 2, 4
 GS_DETERMINISTIC, GS_HOGWILD, GS_HOGWILD_RED = 0, 1, 2
 GS_WALK_UNIFORM, GS_WALK_NODE2VEC = 0, 1
 GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1

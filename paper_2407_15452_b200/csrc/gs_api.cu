@@ -17,6 +17,7 @@ namespace gs {
 // ---- implemented in the kernel files ------------------------------------------
 gs_status validate_csr(const gs_graph *g, bool check_sorted, cudaStream_t st, int64_t *bad_row,
                        int64_t *unsorted_row, int64_t *max_degree, bool *ends_bad);
+gs_status build_walk_index(const gs_graph *g, int4 *rec, cudaStream_t st);
 gs_status init_embeddings(float *w_in, float *w_out, int64_t n, int32_t dim, uint64_t seed,
                           cudaStream_t st);
 gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
@@ -153,7 +154,8 @@ gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offs
     if (n_edges > 0 && !d_cols) return invalid("d_cols is NULL");
     if (!offsets_are_64bit && n_edges >= ((int64_t)1 << 31))
         return invalid("int32 offsets cannot address 2^31 or more edges");
-    if (flags & ~(GS_VALIDATE | GS_REQUIRE_SORTED)) return invalid("unknown flag");
+    if (flags & ~(GS_VALIDATE | GS_REQUIRE_SORTED | GS_BUILD_WALK_INDEX)) return invalid("unknown flag");
+    if (flags & GS_BUILD_WALK_INDEX) flags |= GS_VALIDATE;     // the index is built from checked data
     gs_graph *g = new (std::nothrow) gs_graph;
     if (!g) { set_error("out of host memory"); return GS_ERR_OOM; }
     g->n_nodes = n_nodes;
@@ -164,6 +166,7 @@ gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offs
     g->sorted = 0;
     g->max_degree = -1;
     g->device = 0;
+    g->d_edge_rec = nullptr;
     cudaGetDevice(&g->device);
     if (flags & (GS_VALIDATE | GS_REQUIRE_SORTED)) {
         int64_t bad = -1, unsorted = -1, maxdeg = 0;
@@ -191,11 +194,30 @@ gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offs
         g->max_degree = maxdeg;
         g->sorted = want_sorted ? 1 : 0;
     }
+    if ((flags & GS_BUILD_WALK_INDEX) && n_edges > 0) {
+        void *rec = nullptr;
+        cudaError_t e = cudaMalloc(&rec, sizeof(int4) * (size_t)n_edges);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            delete g;
+            set_error("walk index of %lld x 16 bytes could not be allocated: %s", (long long)n_edges,
+                      cudaGetErrorString(e));
+            return GS_ERR_OOM;
+        }
+        g->d_edge_rec = (int4 *)rec;
+        gs_status s = build_walk_index(g, g->d_edge_rec, (cudaStream_t)stream);
+        if (s != GS_OK) { cudaFree(rec); delete g; return s; }
+    }
     *out = g;
     return GS_OK;
 }
 
-void gs_graph_free(gs_graph *g) { delete g; }
+void gs_graph_free(gs_graph *g)
+{
+    if (!g) return;
+    if (g->d_edge_rec) cudaFree(g->d_edge_rec);          // waits for kernels that may still read it
+    delete g;
+}
 
 gs_status gs_graph_info(const gs_graph *g, int64_t *n_nodes, int64_t *n_edges, int64_t *max_degree,
                         int32_t *rows_sorted)

@@ -40,6 +40,7 @@ struct gs_graph {
     int32_t sorted;       // rows verified strictly increasing
     int64_t max_degree;   // -1 when not validated
     int device;
+    int4 *d_edge_rec;     // optional walk index, library-owned: {neighbour, its degree, its offset}
 };
 
 namespace gs {
@@ -85,6 +86,13 @@ __device__ __forceinline__ int64_t ld_random(const int64_t *p)
     long long v;
     asm("ld.global.nc.L2::64B.s64 %0, [%1];" : "=l"(v) : "l"(p));
     return (int64_t)v;
+}
+__device__ __forceinline__ int4 ld_random(const int4 *p)
+{
+    int4 v;
+    asm("ld.global.nc.L2::64B.v4.s32 {%0, %1, %2, %3}, [%4];"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
 }
 __device__ __forceinline__ uint64_t ld_random(const uint64_t *p)
 {

@@ -207,6 +207,91 @@ uniform_walk_vec_kernel(const OffT *__restrict__ off, const int32_t *__restrict_
     }
 }
 
+// ------------------------------------------------------------------ walk index
+// Record of CSR entry e: the neighbour c = cols[e] together with c's own degree and offset.
+// With it a transition reads ONE random 16-byte record (pick a record in the current node's
+// range; it already says where the next node's range is) instead of an offset pair and then a
+// column: half the random DRAM accesses per transition, paid for with 16 bytes per entry.
+template <typename OffT>
+__global__ void __launch_bounds__(256)
+build_walk_index_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
+                        int64_t n_edges, int4 *__restrict__ rec)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_edges; e += stride) {
+        const int32_t c = col[e];
+        const int64_t o0 = ld_random(off + c), o1 = ld_random(off + c + 1);
+        rec[e] = make_int4(c, (int32_t)(uint32_t)(o1 - o0), (int32_t)(uint32_t)o0,
+                           (int32_t)(uint32_t)((uint64_t)o0 >> 32));
+    }
+}
+
+gs_status build_walk_index(const gs_graph *g, int4 *rec, cudaStream_t st)
+{
+    if (g->n_edges == 0) return GS_OK;
+    int64_t blocks = (g->n_edges + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 64;
+    if (blocks > cap) blocks = cap;
+    if (g->offsets64)
+        build_walk_index_kernel<int64_t><<<(unsigned)blocks, 256, 0, st>>>(
+            (const int64_t *)g->d_offsets, g->d_cols, g->n_edges, rec);
+    else
+        build_walk_index_kernel<int32_t><<<(unsigned)blocks, 256, 0, st>>>(
+            (const int32_t *)g->d_offsets, g->d_cols, g->n_edges, rec);
+    GS_CUDA_TRY(cudaGetLastError());
+    return GS_OK;
+}
+
+// Uniform walks over the index: one record read per transition, sector-wide stores.
+template <typename OffT>
+__global__ void __launch_bounds__(256, 6)
+uniform_walk_index_kernel(const OffT *__restrict__ off, const int4 *__restrict__ rec,
+                          const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
+                          int64_t walk_id_base, int32_t L, uint64_t seed,
+                          int32_t *__restrict__ walks, unsigned long long *steps_out)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int quads = L >> 2;
+    unsigned int my_steps = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
+        const uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
+        int64_t o0 = ld_random(off + cur);
+        uint32_t deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
+        bool alive = true;
+        int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
+        int4 pend = make_int4(0, 0, 0, 0);
+        for (int q = 0; q < quads; ++q) {
+            int32_t v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int e = 4 * q + k;
+                if (e > 0 && alive) {
+                    if (deg == 0) {
+                        alive = false;
+                    } else {
+                        const uint4 r = draw(seed, id, (uint32_t)(e - 1), TAG_UNIFORM, 0);
+                        const int4 x = ld_random(rec + o0 + (int64_t)__umulhi(r.x, deg));
+                        cur = x.x;
+                        deg = (uint32_t)x.y;
+                        o0 = (int64_t)(((uint64_t)(uint32_t)x.w << 32) | (uint32_t)x.z);
+                        ++my_steps;
+                    }
+                }
+                v[k] = alive ? cur : -1;
+            }
+            const int4 now = make_int4(v[0], v[1], v[2], v[3]);
+            if (q & 1) { W4[q - 1] = pend; W4[q] = now; }
+            else if (q == quads - 1) W4[q] = now;
+            else pend = now;
+        }
+    }
+    if (steps_out) {
+        for (int o = 16; o > 0; o >>= 1) my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
+        if ((threadIdx.x & 31) == 0 && my_steps) atomicAdd(steps_out, (unsigned long long)my_steps);
+    }
+}
+
 gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
                                int64_t base, int32_t L, uint64_t seed, int32_t *walks,
                                unsigned long long *steps, cudaStream_t st)
@@ -220,7 +305,16 @@ gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t
 #define GS_UW(KERNEL, T)                                                                        \
     KERNEL<T><<<(unsigned)blocks, threads, 0, st>>>((const T *)g->d_offsets, g->d_cols, starts, \
                                                     g->n_nodes, n_walks, base, L, seed, walks, steps)
-    if (g->offsets64) { if (vec) GS_UW(uniform_walk_vec_kernel, int64_t); else GS_UW(uniform_walk_kernel, int64_t); }
+    if (vec && g->d_edge_rec) {
+        if (g->offsets64)
+            uniform_walk_index_kernel<int64_t><<<(unsigned)blocks, threads, 0, st>>>(
+                (const int64_t *)g->d_offsets, g->d_edge_rec, starts, g->n_nodes, n_walks, base, L,
+                seed, walks, steps);
+        else
+            uniform_walk_index_kernel<int32_t><<<(unsigned)blocks, threads, 0, st>>>(
+                (const int32_t *)g->d_offsets, g->d_edge_rec, starts, g->n_nodes, n_walks, base, L,
+                seed, walks, steps);
+    } else if (g->offsets64) { if (vec) GS_UW(uniform_walk_vec_kernel, int64_t); else GS_UW(uniform_walk_kernel, int64_t); }
     else { if (vec) GS_UW(uniform_walk_vec_kernel, int32_t); else GS_UW(uniform_walk_kernel, int32_t); }
 #undef GS_UW
     GS_CUDA_TRY(cudaGetLastError());

@@ -93,6 +93,29 @@ def test_uniform_walks_bit_exact(tiny, offsets64):
     assert np.array_equal(got.cpu().numpy(), want)
 
 
+@pytest.mark.parametrize("offsets64", [False, True])
+def test_uniform_walks_over_the_walk_index_are_the_same_walks(tiny, offsets64):
+    wl, g, off, col, _, _ = tiny
+    G = load(g, offsets64, flags=B.GS_BUILD_WALK_INDEX)
+    steps = torch.zeros(1, dtype=torch.int64, device=DEV)
+    got = B.gs_random_walks(G, None, 20011, 999, 40, 17, steps=steps)
+    want, st = O.uniform_walks(off, col, None, 20011, 999, 40, 17)
+    assert np.array_equal(got.cpu().numpy(), want) and int(steps.item()) == st
+    # odd walk length: falls back to the scalar path, same result
+    got = B.gs_random_walks(G, None, 777, 5, 13, 17)
+    want, _ = O.uniform_walks(off, col, None, 777, 5, 13, 17)
+    assert np.array_equal(got.cpu().numpy(), want)
+    G.close()
+    # directed graph with dead ends
+    g2 = WL.rmat_graph(3000, 9000, seed=5)
+    off2, col2 = np_graph(g2)
+    G2 = load(g2, offsets64, flags=B.GS_BUILD_WALK_INDEX)
+    starts = np.random.default_rng(3).integers(0, 3000, 5000).astype(np.int32)
+    got = B.gs_random_walks(G2, torch.from_numpy(starts).to(DEV), 5000, 0, 24, 9)
+    want, _ = O.uniform_walks(off2, col2, starts, 5000, 0, 24, 9)
+    assert (want == -1).any() and np.array_equal(got.cpu().numpy(), want)
+
+
 def test_uniform_walks_dead_ends_and_degenerate_sizes():
     g = WL.rmat_graph(3000, 9000, seed=5)           # directed: dead ends
     off, col = np_graph(g)

@@ -175,7 +175,7 @@ GS_API gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts,
  * increments are grouped by destination row, summed in a fixed order without
  * atomics and applied once: U -= lr * GU, V -= lr * GV (sum over pairs, not
  * mean).  Two runs give identical bits.  Scratch grows with
- * n_walks * walk_len * 2 * window * (1 + n_neg) (20 bytes per slot);
+ * n_walks * walk_len * 2 * window * (1 + n_neg) (about 20 + dim/16 bytes per slot);
  * GS_ERR_UNSUPPORTED beyond 2^30 slots.
  * GS_HOGWILD / GS_HOGWILD_RED: one warp per walk runs positions in order;
  * per position the center row is read once, every target row is read,
@@ -218,8 +218,8 @@ GS_API gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, in
  *
  * Limit: the batch must need at most 32 MiB of scratch,
  *   slots = n_walks * walk_len * (2*window*(1+n_neg) + 1)
- *   bytes ~ 20 * slots + n_walks * walk_len * (4*dim + 12)  (+ < 1 % for the sort)
- * e.g. up to about 380 walks of length 40 with window 5, 5 negatives, dim 128.
+ *   bytes ~ (20 + dim/16) * slots + n_walks * walk_len * (4*dim + 12)  (+ < 1 % for the sort)
+ * e.g. up to about 300 walks of length 40 with window 5, 5 negatives, dim 128.
  * Larger batches are rejected with GS_ERR_UNSUPPORTED and a message that
  * states the bytes needed; nothing is launched in that case.
  *

@@ -401,52 +401,141 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
     }
 }
 
-// Pass 3: one warp per run of equal keys below n_nodes: v_row -= lr * sum_j g_j * u_center(j),
-// contributions taken in sorted (= index) order.
+// Passes 3 and 4 walk the sorted keys in chunks of 32: lane l looks at key 32*chunk + l and
+// flags it if it starts a run of equal keys; the warp then sums each flagged run in index order
+// (fp64 accumulators: a hub row can collect 10^5 terms) and writes the row once.  The metadata
+// of 32 contributions is fetched by the 32 lanes at once and the rows 8 (or 4) at a time.
+//
+// Pass 3, keys below n_nodes: v_row -= lr * sum_j g_j * u_center(j).
+// Runs are cut at every multiple of RUN_CUT sorted positions so that no warp sums more than
+// RUN_CUT rows in a chain (a hub row of a 512-walk batch collects thousands).  A run that lies
+// inside one block of RUN_CUT positions is finished here.  Otherwise its first piece leaves a
+// partial sum in tail_part[block], each later piece in lead_part[block], and
+// sgns_apply_out_fixup_kernel adds the pieces in block order and writes the row.
+constexpr int RUN_CUT = 256;
+
 template <int FPL>
 __global__ void __launch_bounds__(256)
 sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
                       const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
                       const uint32_t *__restrict__ vals, const float *__restrict__ gbuf,
-                      uint32_t n_keys, uint32_t n_nodes, int32_t SL, float lr)
+                      uint32_t n_keys, uint32_t n_nodes, int32_t SL, float lr,
+                      double *__restrict__ lead_part, double *__restrict__ tail_part)
+{
+    // One warp per block of RUN_CUT sorted positions.  The 32 lanes fetch the metadata of 32
+    // contributions at once; rows are then fetched G at a time - the center row of every
+    // contribution and, where a run starts, the output row it will update - so that a block
+    // full of one-element runs costs a few memory round trips, not one per run.
+    constexpr int G = FPL <= 4 ? 8 : 4;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t n_blocks = ((int64_t)n_keys + RUN_CUT - 1) / RUN_CUT;
+    for (int64_t b = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); b < n_blocks;
+         b += n_warps) {
+        const int64_t base = b * RUN_CUT;
+        const int64_t end = base + RUN_CUT < (int64_t)n_keys ? base + RUN_CUT : (int64_t)n_keys;
+        uint32_t carry_key = base > 0 ? keys[base - 1] : 0xFFFFFFFFu;     // key before the block
+        bool have = false, lead = false;         // a run is open / it started before this block
+        uint32_t cur_key = 0;
+        Row<FPL> cur_v;
+        double acc[FPL];
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) { acc[j] = 0.0; cur_v.v[j] = 0.f; }
+        if (carry_key < n_nodes && keys[base] == carry_key) { have = true; lead = true; cur_key = carry_key; }
+
+        auto close_run = [&](bool goes_on) {
+            double *part = nullptr;
+            if (lead) part = lead_part;
+            else if (goes_on) part = tail_part;
+            if (part) {
+                double *dst = part + b * (int64_t)(FPL * 32);
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) dst[j * 32 + lane] = acc[j];
+            } else {
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) cur_v.v[j] = (float)((double)cur_v.v[j] - (double)lr * acc[j]);
+                row_store<FPL>(w_out, cur_key, lane, cur_v);
+            }
+        };
+
+        for (int64_t s0 = base; s0 < end; s0 += 32) {
+            const int64_t i = s0 + lane;
+            const uint32_t my_key = i < end ? keys[i] : 0xFFFFFFFFu;
+            const bool usable = my_key < n_nodes;                     // sorted: usable lanes are a prefix
+            float g = 0.f;
+            int32_t c = 0;
+            if (usable) {
+                const uint32_t idx = vals[i];
+                g = gbuf[idx];
+                c = walks[idx / (uint32_t)SL];
+            }
+            uint32_t before = __shfl_up_sync(0xffffffffu, my_key, 1);
+            if (lane == 0) before = carry_key;
+            carry_key = __shfl_sync(0xffffffffu, my_key, 31);
+            const unsigned hmask = __ballot_sync(0xffffffffu, usable && my_key != before);
+            const int n = __popc(__ballot_sync(0xffffffffu, usable));
+            for (int q0 = 0; q0 < n; q0 += G) {
+                Row<FPL> ru[G], rv[G];
+#pragma unroll
+                for (int q = 0; q < G; ++q) {
+                    const int32_t cq = __shfl_sync(0xffffffffu, c, (q0 + q) & 31);
+                    const uint32_t kq = __shfl_sync(0xffffffffu, my_key, (q0 + q) & 31);
+                    if (q0 + q < n) {
+                        ru[q] = row_load<FPL>(w_in, cq, lane);
+                        if ((hmask >> (q0 + q)) & 1u) rv[q] = row_load<FPL>(w_out, kq, lane);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < G; ++q) {
+                    const float gq = __shfl_sync(0xffffffffu, g, (q0 + q) & 31);
+                    const uint32_t kq = __shfl_sync(0xffffffffu, my_key, (q0 + q) & 31);
+                    if (q0 + q < n) {
+                        if ((hmask >> (q0 + q)) & 1u) {               // a run starts here
+                            if (have) close_run(false);
+                            have = true;
+                            lead = false;
+                            cur_key = kq;
+                            cur_v = rv[q];
+#pragma unroll
+                            for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
+                        }
+#pragma unroll
+                        for (int j = 0; j < FPL; ++j) acc[j] += (double)(gq * ru[q].v[j]);
+                    }
+                }
+            }
+            if (n < 32) break;                                        // the rest is not ours
+        }
+        if (have) close_run(end < (int64_t)n_keys && keys[end] == cur_key);
+    }
+}
+
+// One warp per block of RUN_CUT sorted positions: if a run starts in the block and continues
+// past its end, add its pieces (tail of this block, then the leading pieces of the following
+// blocks while they carry the same key) and write the row.
+template <int FPL>
+__global__ void __launch_bounds__(256)
+sgns_apply_out_fixup_kernel(float *__restrict__ w_out, const uint32_t *__restrict__ keys,
+                            uint32_t n_keys, uint32_t n_nodes, float lr,
+                            const double *__restrict__ lead_part, const double *__restrict__ tail_part)
 {
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t x = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); x < n_keys;
-         x += n_warps) {
-        const uint32_t key = keys[x];
-        if (key >= n_nodes) continue;
-        if (x > 0 && keys[x - 1] == key) continue;
-        double acc[FPL];                 // a hub row can collect 10^5 terms: sum them in fp64
+    const int64_t n_blocks = ((int64_t)n_keys + RUN_CUT - 1) / RUN_CUT;
+    for (int64_t b = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); b + 1 < n_blocks;
+         b += n_warps) {
+        const int64_t last = (b + 1) * RUN_CUT - 1;                  // last position of block b
+        const uint32_t key = keys[last];
+        if (key >= n_nodes || keys[last + 1] != key) continue;       // nothing crosses this boundary
+        if (keys[b * RUN_CUT] == key && b > 0 && keys[b * RUN_CUT - 1] == key) continue;   // run started earlier
+        double acc[FPL];
+        const double *t = tail_part + b * (int64_t)(FPL * 32);
 #pragma unroll
-        for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
-        for (int64_t y = x; y < n_keys; y += 4) {
-            float g[4];
-            int32_t c[4];
-            bool more = true;
+        for (int j = 0; j < FPL; ++j) acc[j] = t[j * 32 + lane];
+        for (int64_t nb = b + 1; nb < n_blocks && keys[nb * RUN_CUT] == key; ++nb) {
+            const double *l = lead_part + nb * (int64_t)(FPL * 32);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const bool in = more && (y + q < n_keys) && (keys[y + q] == key);
-                more = in;
-                g[q] = 0.f;
-                c[q] = -1;
-                if (in) {
-                    const uint32_t idx = vals[y + q];
-                    g[q] = gbuf[idx];
-                    c[q] = walks[idx / (uint32_t)SL];
-                }
-            }
-            Row<FPL> r[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (c[q] >= 0) r[q] = row_load<FPL>(w_in, c[q], lane);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (c[q] >= 0) {
-#pragma unroll
-                    for (int j = 0; j < FPL; ++j) acc[j] += (double)(g[q] * r[q].v[j]);
-                }
-            if (!more) break;
+            for (int j = 0; j < FPL; ++j) acc[j] += l[j * 32 + lane];
         }
         Row<FPL> row = row_load<FPL>(w_out, key, lane);
 #pragma unroll
@@ -455,33 +544,58 @@ sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
     }
 }
 
-// Pass 4: runs of keys in [n_nodes, 2 n_nodes): u_row -= lr * sum of the positions' GU rows.
+// Pass 4, keys in [n_nodes, 2 n_nodes): u_row -= lr * sum of the positions' GU rows.
 template <int FPL>
 __global__ void __launch_bounds__(256)
 sgns_apply_in_kernel(float *__restrict__ w_in, const float *__restrict__ GU,
                      const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals,
                      uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, float lr)
 {
+    constexpr int U = FPL <= 4 ? 8 : 4;
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t x = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); x < n_keys;
-         x += n_warps) {
-        const uint32_t key = keys[x];
-        if (key < n_nodes || key >= 2u * n_nodes) continue;
-        if (x > 0 && keys[x - 1] == key) continue;
-        double acc[FPL];
+    const int64_t n_chunks = ((int64_t)n_keys + 31) >> 5;
+    for (int64_t ch = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); ch < n_chunks;
+         ch += n_warps) {
+        const int64_t i = ch * 32 + lane;
+        const uint32_t my_key = i < n_keys ? keys[i] : 0xFFFFFFFFu;
+        const bool head = i < n_keys && my_key >= n_nodes && my_key < 2u * n_nodes &&
+                          (i == 0 || keys[i - 1] != my_key);
+        unsigned heads = __ballot_sync(0xffffffffu, head);
+        while (heads) {
+            const int hl = __ffs(heads) - 1;
+            heads &= heads - 1;
+            const uint32_t key = __shfl_sync(0xffffffffu, my_key, hl);
+            double acc[FPL];
 #pragma unroll
-        for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
-        for (int64_t y = x; y < n_keys && keys[y] == key; ++y) {
-            const Row<FPL> r = row_load<FPL>(GU, (int64_t)(vals[y] - n_slots), lane);
+            for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
+            for (int64_t y0 = ch * 32 + hl;; y0 += 32) {
+                const int64_t y = y0 + lane;
+                const bool in = y < n_keys && keys[y] == key;
+                const int cnt = __popc(__ballot_sync(0xffffffffu, in));
+                const uint32_t pos = in ? vals[y] - n_slots : 0u;
+                for (int q0 = 0; q0 < cnt; q0 += U) {
+                    Row<FPL> r[U];
 #pragma unroll
-            for (int j = 0; j < FPL; ++j) acc[j] += (double)r.v[j];
+                    for (int q = 0; q < U; ++q) {
+                        const uint32_t pq = __shfl_sync(0xffffffffu, pos, (q0 + q) & 31);
+                        if (q0 + q < cnt) r[q] = row_load<FPL>(GU, (int64_t)pq, lane);
+                    }
+#pragma unroll
+                    for (int q = 0; q < U; ++q)
+                        if (q0 + q < cnt) {
+#pragma unroll
+                            for (int j = 0; j < FPL; ++j) acc[j] += (double)r[q].v[j];
+                        }
+                }
+                if (cnt < 32) break;
+            }
+            const int64_t c = (int64_t)(key - n_nodes);
+            Row<FPL> row = row_load<FPL>(w_in, c, lane);
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
+            row_store<FPL>(w_in, c, lane, row);
         }
-        const int64_t c = (int64_t)(key - n_nodes);
-        Row<FPL> row = row_load<FPL>(w_in, c, lane);
-#pragma unroll
-        for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
-        row_store<FPL>(w_in, c, lane, row);
     }
 }
 
@@ -577,8 +691,10 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
     const size_t b_loss = align_up(sizeof(double) * (size_t)n_pos);
     const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)n_pos);
     const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)n_keys));
+    const int64_t n_cut = (n_keys + RUN_CUT - 1) / RUN_CUT;
+    const size_t b_part = align_up(sizeof(double) * (size_t)n_cut * a.dim);
     void *ws = nullptr;
-    gs_status s = workspace_get(WS_SGNS, 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt, &ws);
+    gs_status s = workspace_get(WS_SGNS, 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt + 2 * b_part, &ws);
     if (s != GS_OK) return s;
     char *p = (char *)ws;
     uint32_t *keysA = (uint32_t *)p; p += b_keys;
@@ -589,7 +705,9 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
     float *GU = (float *)p; p += b_gu;
     double *loss_pos = (double *)p; p += b_loss;
     int32_t *pairs_pos = (int32_t *)p; p += b_pairs;
-    uint32_t *counts = (uint32_t *)p;
+    uint32_t *counts = (uint32_t *)p; p += b_cnt;
+    double *lead_part = (double *)p; p += b_part;
+    double *tail_part = (double *)p;
 
     {
         const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
@@ -607,12 +725,18 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
                      bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
     GS_CUDA_TRY(cudaGetLastError());
     {
-        int64_t blocks = (n_keys + 7) / 8;
+        int64_t blocks = (n_keys + 255) / 256;                  // 8 warps x 32 keys per block
         const int64_t cap = (int64_t)sm_count() * 8 * 8;
         if (blocks > cap) blocks = cap;
-        sgns_apply_out_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
-            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr);
+        sgns_apply_out_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
+            lead_part, tail_part);
         GS_CUDA_TRY(cudaGetLastError());
+        if (n_cut > 1) {
+            sgns_apply_out_fixup_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part);
+            GS_CUDA_TRY(cudaGetLastError());
+        }
         sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
             a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr);
         GS_CUDA_TRY(cudaGetLastError());
@@ -698,7 +822,9 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
     const size_t b_loss = align_up(sizeof(double) * (size_t)n_pos);
     const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)n_pos);
     const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)n_keys));
-    const size_t need = 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt;
+    const int64_t n_cut = (n_keys + RUN_CUT - 1) / RUN_CUT;
+    const size_t b_part = align_up(sizeof(double) * (size_t)n_cut * a.dim);
+    const size_t need = 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt + 2 * b_part;
     if (n_keys > ((int64_t)1 << 30) || need > (size_t)GS_STATIC_SCRATCH_BYTES) {
         set_error("gs_sgns_step_static: this batch needs %zu bytes of scratch, the fixed array has %u; "
                   "pass fewer walks per call or use gs_sgns_step", need, GS_STATIC_SCRATCH_BYTES);
@@ -706,7 +832,8 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
     }
     // Every byte that is read below is written first by the pass before it (keys, g, GU, loss
     // and pair counts by the coefficient pass for all slots; digit counts by the histogram
-    // pass for all tiles), so nothing left over from an earlier call can leak in.
+    // pass for all tiles; the partial sums of cut runs by the apply pass before the fix-up
+    // pass reads exactly those), so nothing left over from an earlier call can leak in.
     char *p = (char *)scratch;
     uint32_t *keysA = (uint32_t *)p; p += b_keys;
     uint32_t *keysB = (uint32_t *)p; p += b_keys;
@@ -716,7 +843,9 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
     float *GU = (float *)p; p += b_gu;
     double *loss_pos = (double *)p; p += b_loss;
     int32_t *pairs_pos = (int32_t *)p; p += b_pairs;
-    uint32_t *counts = (uint32_t *)p;
+    uint32_t *counts = (uint32_t *)p; p += b_cnt;
+    double *lead_part = (double *)p; p += b_part;
+    double *tail_part = (double *)p;
     {
         const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
         int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
@@ -733,12 +862,18 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
                      bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
     GS_CUDA_TRY(cudaGetLastError());
     {
-        int64_t blocks = (n_keys + 7) / 8;
+        int64_t blocks = (n_keys + 255) / 256;                  // 8 warps x 32 keys per block
         const int64_t cap = (int64_t)sm_count() * 8 * 8;
         if (blocks > cap) blocks = cap;
-        sgns_apply_out_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
-            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr);
+        sgns_apply_out_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
+            lead_part, tail_part);
         GS_CUDA_TRY(cudaGetLastError());
+        if (n_cut > 1) {
+            sgns_apply_out_fixup_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part);
+            GS_CUDA_TRY(cudaGetLastError());
+        }
         sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
             a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr);
         GS_CUDA_TRY(cudaGetLastError());

@@ -3,8 +3,8 @@
 // destination row while keeping contributions of one row in index order, which
 // is what makes the summation order (and so the result bits) fixed.
 //
-// Per pass: (1) per-tile digit histograms, (2) one exclusive scan over the
-// digit-major (digit, tile) counts, (3) a scatter in which each warp ranks its
+// Per pass: (1) per-tile digit histograms, (2) per digit an exclusive scan over
+// the tiles (256 blocks) plus the digit totals, (3) a scatter in which each warp ranks its
 // items round by round with match_any, so that equal digits keep their order.
 #include "gs_common.cuh"
 
@@ -32,39 +32,66 @@ sort_hist_kernel(const uint32_t *__restrict__ keys, uint32_t n, int shift, uint3
     counts[threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
 }
 
-// Exclusive scan of m counters by one block: each thread owns a contiguous chunk.
-__global__ void __launch_bounds__(1024) sort_scan_kernel(uint32_t *__restrict__ counts, uint32_t m)
+// Block d turns the per-tile counts of digit d into exclusive prefixes over the tiles and
+// leaves the digit's total in totals[d].  (The prefix over digits is taken by the scatter
+// kernel itself, from the 256 totals.)
+__global__ void __launch_bounds__(256)
+sort_scan_kernel(uint32_t *__restrict__ counts, uint32_t n_tiles, uint32_t *__restrict__ totals)
 {
-    __shared__ uint32_t part[1024];
-    const uint32_t chunk = (m + 1023u) / 1024u;
-    const uint32_t lo = threadIdx.x * chunk;
-    const uint32_t hi = lo + chunk < m ? lo + chunk : m;
-    uint32_t s = 0;
-    for (uint32_t i = lo; i < hi; ++i) s += counts[i];
-    part[threadIdx.x] = s;
+    __shared__ uint32_t warp_sum[8];
+    __shared__ uint32_t carry_s;
+    uint32_t *c = counts + (size_t)blockIdx.x * n_tiles;
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry_s = 0;
     __syncthreads();
-    for (int o = 1; o < 1024; o <<= 1) {               // Hillis-Steele inclusive scan
-        const uint32_t add = threadIdx.x >= (unsigned)o ? part[threadIdx.x - o] : 0u;
+    for (uint32_t base = 0; base < n_tiles; base += 256) {
+        const uint32_t i = base + threadIdx.x;
+        const uint32_t v = i < n_tiles ? c[i] : 0u;
+        uint32_t incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) warp_sum[wi] = incl;
         __syncthreads();
-        part[threadIdx.x] += add;
+        uint32_t before = carry_s;
+        for (int k = 0; k < wi; ++k) before += warp_sum[k];
+        if (i < n_tiles) c[i] = before + incl - v;
+        __syncthreads();
+        if (threadIdx.x == 255) carry_s = before + incl;
         __syncthreads();
     }
-    uint32_t run = part[threadIdx.x] - s;
-    for (uint32_t i = lo; i < hi; ++i) {
-        const uint32_t c = counts[i];
-        counts[i] = run;
-        run += c;
-    }
+    if (threadIdx.x == 0) totals[blockIdx.x] = carry_s;
 }
 
 template <bool IOTA>
 __global__ void __launch_bounds__(SORT_THREADS)
 sort_scatter_kernel(const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in,
                     uint32_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out, uint32_t n,
-                    int shift, uint32_t n_tiles, const uint32_t *__restrict__ offsets)
+                    int shift, uint32_t n_tiles, const uint32_t *__restrict__ offsets,
+                    const uint32_t *__restrict__ totals)
 {
     constexpr int WARPS = SORT_THREADS / 32;
     __shared__ uint32_t cnt[WARPS][RADIX];
+    __shared__ uint32_t digit_base[RADIX];
+    {   // exclusive prefix of the 256 digit totals (thread d owns digit d)
+        const uint32_t t = totals[threadIdx.x];
+        uint32_t incl = t;
+        const int ln = threadIdx.x & 31;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_up_sync(0xffffffffu, incl, o);
+            if (ln >= o) incl += u;
+        }
+        digit_base[threadIdx.x] = incl - t;                // prefix inside the warp's 32 digits
+        if (ln == 31) cnt[0][threadIdx.x >> 5] = incl;     // warp totals, parked in cnt for a moment
+        __syncthreads();
+        uint32_t before = 0;
+        for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) before += cnt[0][k];
+        __syncthreads();
+        digit_base[threadIdx.x] += before;
+    }
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     for (int x = threadIdx.x; x < WARPS * RADIX; x += SORT_THREADS) (&cnt[0][0])[x] = 0;
     __syncthreads();
@@ -93,7 +120,7 @@ sort_scatter_kernel(const uint32_t *__restrict__ keys_in, const uint32_t *__rest
     __syncthreads();
     {   // digit threadIdx.x: turn per-warp counts into start positions in the output
         const int d = threadIdx.x;
-        uint32_t run = offsets[d * n_tiles + blockIdx.x];
+        uint32_t run = digit_base[d] + offsets[d * n_tiles + blockIdx.x];
 #pragma unroll
         for (int k = 0; k < WARPS; ++k) {
             const uint32_t c = cnt[k][d];
@@ -116,7 +143,7 @@ sort_scatter_kernel(const uint32_t *__restrict__ keys_in, const uint32_t *__rest
 size_t sort_counts_bytes(uint32_t n)
 {
     const uint32_t n_tiles = (n + SORT_TILE - 1) / SORT_TILE;
-    return sizeof(uint32_t) * (size_t)RADIX * (n_tiles ? n_tiles : 1);
+    return sizeof(uint32_t) * ((size_t)RADIX * (n_tiles ? n_tiles : 1) + RADIX);   // + digit totals
 }
 
 // Sorts n pairs by the low `bits` bits of the key.  The first pass takes value i for
@@ -128,17 +155,18 @@ int radix_sort_pairs(uint32_t *keysA, uint32_t *valsA, uint32_t *keysB, uint32_t
 {
     const uint32_t n_tiles = (n + SORT_TILE - 1) / SORT_TILE;
     uint32_t *kin = keysA, *vin = valsA, *kout = keysB, *vout = valsB;
+    uint32_t *totals = counts + (size_t)RADIX * (n_tiles ? n_tiles : 1);
     int launches = 0;
     bool first = true;
     for (int shift = 0; shift < bits && n > 0; shift += 8) {
         sort_hist_kernel<<<n_tiles, SORT_THREADS, 0, st>>>(kin, n, shift, n_tiles, counts);
-        sort_scan_kernel<<<1, 1024, 0, st>>>(counts, RADIX * n_tiles);
+        sort_scan_kernel<<<RADIX, 256, 0, st>>>(counts, n_tiles, totals);
         if (first)
             sort_scatter_kernel<true><<<n_tiles, SORT_THREADS, 0, st>>>(kin, vin, kout, vout, n,
-                                                                        shift, n_tiles, counts);
+                                                                        shift, n_tiles, counts, totals);
         else
             sort_scatter_kernel<false><<<n_tiles, SORT_THREADS, 0, st>>>(kin, vin, kout, vout, n,
-                                                                         shift, n_tiles, counts);
+                                                                         shift, n_tiles, counts, totals);
         launches += 3;
         first = false;
         uint32_t *t = kin; kin = kout; kout = t;

@@ -288,7 +288,7 @@ def run_ours(args, wl):
     g, table, info = build_inputs(wl, args.scale, dev)
     n = g.n_nodes
     flags = B.GS_VALIDATE | B.GS_REQUIRE_SORTED
-    if wl.walk_kind == "uniform" and not args.no_walk_index:
+    if not args.no_walk_index:
         flags |= B.GS_BUILD_WALK_INDEX                  # 16 B per CSR entry, one read per transition
         info["walk_index_bytes"] = 16 * g.n_edges
     G = B.gs_graph_load_csr(g.offsets, g.cols, flags)

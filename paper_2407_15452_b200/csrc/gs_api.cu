@@ -303,7 +303,7 @@ gs_status gs_random_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_
                                 (unsigned long long *)d_steps, (cudaStream_t)stream);
 }
 
-static int g_n2v_group = 4;   // lanes per walk in the node2vec sampler
+static int g_n2v_group = 1;   // lanes per walk in the node2vec sampler (1 measured fastest)
 
 gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_walks,
                             int64_t walk_id_base, int32_t walk_len, uint64_t seed, double p,

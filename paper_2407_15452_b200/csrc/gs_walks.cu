@@ -414,6 +414,95 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
     if (caps_out && my_caps) atomicAdd(caps_out, (unsigned long long)my_caps);
 }
 
+// One walk per thread (the fastest mapping measured: walks in flight matter more than lanes
+// per walk).  Rejection rounds run one after another; the state carries the adjacency range of
+// the current and of the previous node, so a round costs one random read (the proposal) plus,
+// when the draw falls between the two class thresholds, a binary search in adj(prev).  With the
+// walk index the proposal's record already holds the next node's range; without it the range
+// is read from the offsets at the start of the next transition.  Entries leave 32 bytes at a
+// time.  Needs L % 4 == 0 and a 16-byte aligned output.
+template <typename OffT, bool INDEX>
+__global__ void __launch_bounds__(256, 4)
+node2vec_thread_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
+                       const int4 *__restrict__ rec, const int32_t *__restrict__ starts,
+                       int64_t n_nodes, int64_t n_walks, int64_t walk_id_base, int32_t L,
+                       uint64_t seed, N2VThresholds T, int32_t max_rounds,
+                       int32_t *__restrict__ walks, unsigned long long *steps_out,
+                       unsigned long long *caps_out)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int quads = L >> 2;
+    const unsigned long long t_lo = T.t_near < T.t_far ? T.t_near : T.t_far;
+    const unsigned long long t_hi = T.t_near < T.t_far ? T.t_far : T.t_near;
+    unsigned int my_steps = 0, my_caps = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
+        const uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
+        int64_t o0 = ld_random(off + cur);
+        uint32_t deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
+        int32_t prev = -1;
+        int64_t p0 = 0, p1 = 0;
+        bool alive = true;
+        int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
+        int4 pend = make_int4(0, 0, 0, 0);
+        for (int q = 0; q < quads; ++q) {
+            int32_t v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int e = 4 * q + k;                       // entry index, transition t = e - 1
+                if (e > 0 && alive) {
+                    if (deg == 0) {
+                        alive = false;
+                    } else {
+                        int32_t x = -1;
+                        uint32_t xdeg = 0;
+                        int64_t xoff = 0;
+                        const int32_t rounds = e == 1 ? 1 : max_rounds;
+                        bool acc = false;
+                        for (int32_t sr = 0; sr < rounds && !acc; ++sr) {
+                            const uint4 r = draw(seed, id, (uint32_t)(e - 1), TAG_NODE2VEC, (uint32_t)sr);
+                            const int64_t at = o0 + (int64_t)__umulhi(r.x, deg);
+                            if (INDEX) {
+                                const int4 rc = ld_random(rec + at);
+                                x = rc.x;
+                                xdeg = (uint32_t)rc.y;
+                                xoff = (int64_t)(((uint64_t)(uint32_t)rc.w << 32) | (uint32_t)rc.z);
+                            } else {
+                                x = ld_random(col + at);
+                            }
+                            const unsigned long long r1 = r.y;
+                            if (e == 1) acc = true;            // first transition: uniform
+                            else if (x == prev) acc = r1 < T.t_prev;
+                            else if (r1 < t_lo) acc = true;
+                            else if (r1 >= t_hi) acc = false;
+                            else acc = r1 < (row_contains(col, p0, p1, x) ? T.t_near : T.t_far);
+                        }
+                        if (!acc) ++my_caps;                   // cap reached: keep the last proposal
+                        prev = cur; p0 = o0; p1 = o0 + deg;
+                        cur = x;
+                        if (INDEX) { o0 = xoff; deg = xdeg; }
+                        else { o0 = ld_random(off + cur); deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0); }
+                        ++my_steps;
+                    }
+                }
+                v[k] = alive ? cur : -1;
+            }
+            const int4 now = make_int4(v[0], v[1], v[2], v[3]);
+            if (q & 1) { W4[q - 1] = pend; W4[q] = now; }
+            else if (q == quads - 1) W4[q] = now;
+            else pend = now;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
+        my_caps += __shfl_xor_sync(0xffffffffu, my_caps, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (steps_out && my_steps) atomicAdd(steps_out, (unsigned long long)my_steps);
+        if (caps_out && my_caps) atomicAdd(caps_out, (unsigned long long)my_caps);
+    }
+}
+
 void node2vec_thresholds(double p, double q, N2VThresholds *T)
 {
     const double a[3] = { 1.0 / p, 1.0, 1.0 / q };
@@ -453,6 +542,21 @@ gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_
     if (n_walks == 0) return GS_OK;
     N2VThresholds T;
     node2vec_thresholds(p, q, &T);
+    if (group == 1 && L % 4 == 0 && (((uintptr_t)walks & 15) == 0)) {
+        const int threads = 256;
+        int64_t blocks = (n_walks + threads - 1) / threads;
+        const int64_t cap = (int64_t)sm_count() * 8 * 16;
+        if (blocks > cap) blocks = cap;
+#define GS_N2T(T_, IDX)                                                                           \
+        node2vec_thread_kernel<T_, IDX><<<(unsigned)blocks, threads, 0, st>>>(                      \
+            (const T_ *)g->d_offsets, g->d_cols, g->d_edge_rec, starts, g->n_nodes, n_walks, base, L, \
+            seed, T, max_rounds, walks, steps, caps)
+        if (g->offsets64) { if (g->d_edge_rec) GS_N2T(int64_t, true); else GS_N2T(int64_t, false); }
+        else { if (g->d_edge_rec) GS_N2T(int32_t, true); else GS_N2T(int32_t, false); }
+#undef GS_N2T
+        GS_CUDA_TRY(cudaGetLastError());
+        return GS_OK;
+    }
 #define GS_N2V(GG)                                                                              \
     do {                                                                                        \
         if (g->offsets64) launch_n2v<int64_t, GG>(g, starts, n_walks, base, L, seed, T,         \

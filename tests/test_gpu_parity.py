@@ -132,7 +132,8 @@ def test_uniform_walks_dead_ends_and_degenerate_sizes():
                                              (0.5, 2.0, 3), (100.0, 100.0, 1), (0.5, 2.0, 37)])
 def test_node2vec_walks_bit_exact_for_every_group_width(tiny, p, q, max_rounds):
     _, g, off, col, _, _ = tiny
-    G = load(g)
+    # with the walk index when the cap is the default, without it otherwise: both paths covered
+    G = load(g, flags=B.GS_VALIDATE | B.GS_REQUIRE_SORTED | (B.GS_BUILD_WALK_INDEX if max_rounds == 1024 else 0))
     n_walks, L = 5003, 24
     want, st, caps = O.node2vec_walks(off, col, None, n_walks, 77, L, 5, p, q, max_rounds)
     try:
@@ -145,7 +146,7 @@ def test_node2vec_walks_bit_exact_for_every_group_width(tiny, p, q, max_rounds):
             assert np.array_equal(got.cpu().numpy(), want), lanes
             assert int(steps.item()) == st and int(hits.item()) == caps, lanes
     finally:
-        B.gs_tune_node2vec_group(4)
+        B.gs_tune_node2vec_group(1)
     if max_rounds <= 3:
         assert caps > 0
 
@@ -159,6 +160,12 @@ def test_node2vec_on_directed_graph_with_dead_ends_and_int64_offsets():
     want, _, _ = O.node2vec_walks(off, col, starts, 4000, 0, 30, 11, 0.25, 4.0)
     got = B.gs_node2vec_walks(G, torch.from_numpy(starts).to(DEV), 4000, 0, 30, 11, 0.25, 4.0)
     assert np.array_equal(got.cpu().numpy(), want)
+    # one walk per thread, over the walk index and without it, walk length a multiple of 4
+    want, _, _ = O.node2vec_walks(off, col, starts, 4000, 9, 32, 12, 0.25, 4.0)
+    for flags in (3, 7):
+        G2 = load(g, offsets64=True, flags=flags)
+        got = B.gs_node2vec_walks(G2, torch.from_numpy(starts).to(DEV), 4000, 9, 32, 12, 0.25, 4.0)
+        assert np.array_equal(got.cpu().numpy(), want), flags
 
 
 # ---------------------------------------------------------------- initialisation

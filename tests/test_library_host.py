@@ -78,5 +78,5 @@ def test_argument_errors_are_status_codes_without_touching_a_gpu(lib):
                              ctypes.c_uint64(0), None, None, None)
     assert st == -1
     assert lib.gs_tune_node2vec_group(3) == -1
-    assert lib.gs_tune_node2vec_group(4) == 0
+    assert lib.gs_tune_node2vec_group(1) == 0
     lib.gs_graph_free(None)

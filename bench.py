@@ -114,6 +114,26 @@ def measured_peak_gbs():
     return 6650.0, "fallback"
 
 
+def recorded_traffic(kernel, workload):
+    """DRAM bytes per pair (or per transition) of `kernel` taken from the ncu summary under
+    profiles/, or None when there is none or the kernel's source has changed since the capture
+    (the summary records the sha256 of the source file)."""
+    import hashlib
+    import re
+    f = ROOT / "profiles" / f"{kernel}__{workload}.md"
+    if not f.exists():
+        return None
+    text = f.read_text()
+    m = re.search(r"dram_bytes_per_unit\s*=\s*([0-9.eE+-]+)", text)
+    h = re.search(r"source\s*=\s*(\S+)\s+sha256\s*=\s*([0-9a-f]{64})", text)
+    if not m or not h:
+        return None
+    src = ROOT / h.group(1)
+    if not src.exists() or hashlib.sha256(src.read_bytes()).hexdigest() != h.group(2):
+        return None
+    return float(m.group(1))
+
+
 def algorithmic_bytes(pairs, positions, dim, n_neg):
     """Row traffic the update must move: per pair 1+K output rows read and written plus K
     alias entries; per center position one input row read and written plus its walk entry."""
@@ -398,6 +418,8 @@ def run_ours(args, wl):
         wbytes = walk_bytes(steps, wl.offsets64, indexed) / launches
         gbytes = walk_granule_bytes(steps, indexed) / launches
         walk_ms = ms_walk / launches
+        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if mode else None
+        traffic = per_pair * pairs / launches if per_pair else None
         out = {
             "metric": METRIC, "value": pairs_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
@@ -417,7 +439,7 @@ def run_ours(args, wl):
             "roofline": {"bound": "hbm",
                          "kernel": "sgns_hogwild_kernel" if mode else "sgns (coef+sort+apply)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "peak_kind": f"of {peak_kind}", "traffic": traffic,
                          "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (ms_sgns * 1e-3)},
             "walk": {"kernel": walk_kernel_name(wl, indexed),
                      "walk_steps_per_s_kernel": steps / (ms_walk * 1e-3), "ms_per_launch": walk_ms,

@@ -1,7 +1,8 @@
 // Skip-gram-with-negative-sampling update kernels.
 //
-// A row of an embedding table is dim fp32 values; a warp holds one row as
-// FPL = dim/32 values per lane (16-byte vector accesses for dim >= 128), so a
+// A row of an embedding table is dim fp32 values, always moved with 16-byte
+// accesses: a whole warp holds one row for dim >= 128, half a warp for dim 64,
+// a quarter for dim 32 (so one warp-wide access moves 1, 2 or 4 rows), and a
 // row read or write is one fully coalesced request.  Dot products are
 // butterfly shuffles.  The path is bound by row traffic in HBM/L2, not by
 // arithmetic, so there is no tensor-core work here.
@@ -142,6 +143,73 @@ __device__ __forceinline__ double warp_sum_double(double s)
     return s;
 }
 
+// ---------------------------------------------------------------- rows held by part of a warp
+// For dim < 128 a full warp per row would move only 128 or 256 bytes per instruction, and the
+// per-row instruction cost - not bytes - would set the pace.  There a row is held by LPR = 16
+// or 8 lanes (16 bytes per lane) and one warp-wide access moves NG = 2 or 4 different rows.
+template <int DIM> struct RowGeom {
+    static constexpr int FPL = DIM >= 128 ? DIM / 32 : 4;   // floats per lane
+    static constexpr int LPR = DIM / FPL;                   // lanes per row: 32, 32, 16, 8
+    static constexpr int NG = 32 / LPR;                     // rows per warp-wide access
+};
+
+template <int DIM>
+__device__ __forceinline__ Row<RowGeom<DIM>::FPL> grow_load(const float *__restrict__ tab, int64_t r, int sub)
+{
+    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR;
+    Row<FPL> out;
+    const float4 *p = reinterpret_cast<const float4 *>(tab + r * (int64_t)DIM);
+#pragma unroll
+    for (int q = 0; q < FPL / 4; ++q) {
+        const float4 t = p[q * LPR + sub];
+        out.v[4 * q] = t.x; out.v[4 * q + 1] = t.y; out.v[4 * q + 2] = t.z; out.v[4 * q + 3] = t.w;
+    }
+    return out;
+}
+
+template <int DIM>
+__device__ __forceinline__ void grow_store(float *__restrict__ tab, int64_t r, int sub,
+                                           const Row<RowGeom<DIM>::FPL> &x)
+{
+    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR;
+    float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
+#pragma unroll
+    for (int q = 0; q < FPL / 4; ++q)
+        p[q * LPR + sub] = make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]);
+}
+
+template <int DIM>
+__device__ __forceinline__ void grow_red_add(float *__restrict__ tab, int64_t r, int sub,
+                                             const Row<RowGeom<DIM>::FPL> &x)
+{
+    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR;
+    float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
+#pragma unroll
+    for (int q = 0; q < FPL / 4; ++q)
+        atomicAdd(p + q * LPR + sub,
+                  make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
+}
+
+// sum over the LPR lanes that hold one row (identical bits on each of them)
+template <int LPR>
+__device__ __forceinline__ float group_sum(float s)
+{
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return s;
+}
+
+// add up the per-group copies of a row held by the NG groups of a warp
+template <int DIM>
+__device__ __forceinline__ void sum_over_groups(Row<RowGeom<DIM>::FPL> &x)
+{
+#pragma unroll
+    for (int o = RowGeom<DIM>::LPR; o < 32; o <<= 1) {
+#pragma unroll
+        for (int j = 0; j < RowGeom<DIM>::FPL; ++j) x.v[j] += __shfl_xor_sync(0xffffffffu, x.v[j], o);
+    }
+}
+
 // ---------------------------------------------------------------- target list of one position
 // Slot layout: tgt[s * (1 + K) + 0] = context of slot s, tgt[s * (1 + K) + 1 + k] = negative k;
 // -1 where the pair does not exist or the negative equals the context (masked).
@@ -209,24 +277,33 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
 }
 
 // ---------------------------------------------------------------- lock-free kernel
-template <int FPL, bool RED, int MINB>
+template <int DIM, bool RED, int MINB>
 __global__ void __launch_bounds__(SGNS_WARPS * 32, MINB)
 sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
                     const int32_t *__restrict__ walks, int64_t n_walks, int64_t walk_id_base,
                     int32_t L, int32_t w, int32_t K, const uint64_t *__restrict__ alias,
                     uint32_t n_alias, float lr, uint64_t seed, double *loss_out,
-                    unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs)
+                    unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs,
+                    unsigned long long *ticket)
 {
+    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR, NG = RowGeom<DIM>::NG;
+    constexpr int CH = TCH * NG;                         // targets per chunk
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    const int grp = lane / LPR, sub = lane % LPR;
     const int S = 2 * w, T1 = 1 + K, SL = S * T1;
     int32_t *W = smem + wi * (L + SL);
     int32_t *tgt = W + L;
-    const int64_t n_warps = (int64_t)gridDim.x * SGNS_WARPS;
     double loss_acc = 0.0;
     unsigned long long pair_acc = 0;
 
-    for (int64_t a = (int64_t)blockIdx.x * SGNS_WARPS + wi; a < n_walks; a += n_warps) {
+    // Walks differ in length (dead ends), so warps draw the next walk from a shared ticket
+    // counter instead of taking a fixed share.
+    for (;;) {
+        unsigned long long tk = 0;
+        if (lane == 0) tk = atomicAdd(ticket, 1ull);
+        const int64_t a = (int64_t)__shfl_sync(0xffffffffu, tk, 0);
+        if (a >= n_walks) break;
         const uint64_t id = (uint64_t)(walk_id_base + a);
         __syncwarp();
         for (int x = lane; x < L; x += 32) W[x] = walks[a * L + x];
@@ -240,37 +317,42 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
                                             dp, dn);
             if (pairs == 0) continue;
             pair_acc += (unsigned long long)pairs;
-            const Row<FPL> u = row_load<FPL>(w_in, c, lane);
-            Row<FPL> acc;
+            const Row<FPL> u = grow_load<DIM>(w_in, c, sub);     // every group holds the center row
+            Row<FPL> acc;                                        // this group's share of its gradient
 #pragma unroll
             for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
             float loss = 0.f;                            // this lane's share of the position's loss
             int kk = 0;                                  // base mod T1, tracked incrementally
-            for (int base = 0; base < SL; base += TCH) {
+            for (int base = 0; base < SL; base += CH) {
+                // target k of group grp is list entry base + k * NG + grp
                 int32_t ids[TCH];
                 bool any = false;
 #pragma unroll
                 for (int k = 0; k < TCH; ++k) {
-                    ids[k] = base + k < SL ? tgt[base + k] : -1;
+                    const int t = base + k * NG + grp;
+                    ids[k] = t < SL ? tgt[t] : -1;
                     any |= ids[k] >= 0;
                 }
-                if (any) {
+                if (__any_sync(0xffffffffu, any)) {
                     Row<FPL> rows[TCH];
                     float f[TCH];
 #pragma unroll
                     for (int k = 0; k < TCH; ++k)
-                        if (ids[k] >= 0) rows[k] = row_load<FPL>(w_out, ids[k], lane);
+                        if (ids[k] >= 0) rows[k] = grow_load<DIM>(w_out, ids[k], sub);
 #pragma unroll
                     for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
 #pragma unroll
-                    for (int k = 0; k < TCH; ++k) f[k] = warp_sum(f[k]);
-                    int my_kt = kk + (lane < TCH ? lane : 0);
+                    for (int k = 0; k < TCH; ++k) f[k] = group_sum<LPR>(f[k]);
+                    // lane `sub` of a group evaluates the group's target `sub`
+                    const int my_t = base + sub * NG + grp;
+                    const bool mine = sub < TCH && my_t < SL;
+                    int my_kt = kk + (sub < TCH ? sub * NG + grp : 0);
                     while (my_kt >= T1) my_kt -= T1;
-                    const int32_t my_id = (lane < TCH && base + lane < SL) ? tgt[base + lane] : -1;
-                    const float my_g = lane_coefficient<TCH>(f, lane, my_id, my_kt == 0, loss);
+                    const int32_t my_id = mine ? tgt[my_t] : -1;
+                    const float my_g = lane_coefficient<TCH>(f, sub, my_id, my_kt == 0, loss);
 #pragma unroll
                     for (int k = 0; k < TCH; ++k) {
-                        const float g = __shfl_sync(0xffffffffu, my_g, k);
+                        const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + k);
                         if (ids[k] >= 0) {
                             const float step = -lr * g;
                             Row<FPL> delta;
@@ -280,25 +362,26 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
                                 delta.v[j] = step * u.v[j];
                                 rows[k].v[j] += delta.v[j];
                             }
-                            if (RED) row_red_add<FPL>(w_out, ids[k], lane, delta);
-                            else row_store<FPL>(w_out, ids[k], lane, rows[k]);
+                            if (RED) grow_red_add<DIM>(w_out, ids[k], sub, delta);
+                            else grow_store<DIM>(w_out, ids[k], sub, rows[k]);
                         }
                     }
                 }
-                kk += TCH;
+                kk += CH;
                 while (kk >= T1) kk -= T1;
             }
             // center row: add the accumulated increment to the row as it is now
+            sum_over_groups<DIM>(acc);
             Row<FPL> delta;
 #pragma unroll
             for (int j = 0; j < FPL; ++j) delta.v[j] = -lr * acc.v[j];
             if (RED) {
-                row_red_add<FPL>(w_in, c, lane, delta);
+                if (grp == 0) grow_red_add<DIM>(w_in, c, sub, delta);
             } else {
-                Row<FPL> now = row_load<FPL>(w_in, c, lane);
+                Row<FPL> now = grow_load<DIM>(w_in, c, sub);
 #pragma unroll
                 for (int j = 0; j < FPL; ++j) now.v[j] += delta.v[j];
-                row_store<FPL>(w_in, c, lane, now);
+                if (grp == 0) grow_store<DIM>(w_in, c, sub, now);
             }
             loss_acc += (double)loss;
         }
@@ -315,7 +398,7 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
 //   keys[x] = destination row of w_out (or `invalid`), gbuf[x] = coefficient g,
 // and per position: keys[n_slots + pos] = n_nodes + center (or `invalid`),
 // GU[pos] = sum g * v (gradient of the center row), loss_pos, pairs_pos.
-template <int FPL>
+template <int DIM>
 __global__ void __launch_bounds__(SGNS_WARPS * 32)
 sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out,
                  const int32_t *__restrict__ walks, int64_t n_pos, int64_t walk_id_base, int32_t L,
@@ -324,8 +407,11 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
                  float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos,
                  int32_t *__restrict__ pairs_pos, int32_t *dump_pairs, int32_t *dump_negs)
 {
+    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR, NG = RowGeom<DIM>::NG;
+    constexpr int CH = TCH * NG;
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    const int grp = lane / LPR, sub = lane % LPR;
     const int S = 2 * w, T1 = 1 + K, SL = S * T1;
     int32_t *tgt = smem + wi * SL;
     const uint32_t invalid = 2u * n_nodes;
@@ -355,44 +441,49 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
         if (pairs == 0) {
             for (int x = lane; x < SL; x += 32) { kp[x] = invalid; gp[x] = 0.f; }
         } else {
-            const Row<FPL> u = row_load<FPL>(w_in, c, lane);
+            const Row<FPL> u = grow_load<DIM>(w_in, c, sub);
             int kk = 0;
-            for (int base = 0; base < SL; base += TCH) {
+            for (int base = 0; base < SL; base += CH) {
                 int32_t ids[TCH];
 #pragma unroll
-                for (int k = 0; k < TCH; ++k) ids[k] = base + k < SL ? tgt[base + k] : -1;
+                for (int k = 0; k < TCH; ++k) {
+                    const int t = base + k * NG + grp;
+                    ids[k] = t < SL ? tgt[t] : -1;
+                }
                 Row<FPL> rows[TCH];
                 float f[TCH];
 #pragma unroll
                 for (int k = 0; k < TCH; ++k)
-                    if (ids[k] >= 0) rows[k] = row_load<FPL>(w_out, ids[k], lane);
+                    if (ids[k] >= 0) rows[k] = grow_load<DIM>(w_out, ids[k], sub);
 #pragma unroll
                 for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
 #pragma unroll
-                for (int k = 0; k < TCH; ++k) f[k] = warp_sum(f[k]);
-                int my_kt = kk + (lane < TCH ? lane : 0);
+                for (int k = 0; k < TCH; ++k) f[k] = group_sum<LPR>(f[k]);
+                const int my_t = base + sub * NG + grp;
+                const bool mine = sub < TCH && my_t < SL;
+                int my_kt = kk + (sub < TCH ? sub * NG + grp : 0);
                 while (my_kt >= T1) my_kt -= T1;
-                const bool mine = lane < TCH && base + lane < SL;
-                const int32_t my_id = mine ? tgt[base + lane] : -1;
-                const float my_g = lane_coefficient<TCH>(f, lane, my_id, my_kt == 0, loss);
+                const int32_t my_id = mine ? tgt[my_t] : -1;
+                const float my_g = lane_coefficient<TCH>(f, sub, my_id, my_kt == 0, loss);
                 if (mine) {
-                    kp[base + lane] = my_id >= 0 ? (uint32_t)my_id : invalid;
-                    gp[base + lane] = my_g;
+                    kp[my_t] = my_id >= 0 ? (uint32_t)my_id : invalid;
+                    gp[my_t] = my_g;
                 }
 #pragma unroll
                 for (int k = 0; k < TCH; ++k) {
-                    const float g = __shfl_sync(0xffffffffu, my_g, k);
+                    const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + k);
                     if (ids[k] >= 0) {
 #pragma unroll
                         for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g, rows[k].v[j], acc.v[j]);
                     }
                 }
-                kk += TCH;
+                kk += CH;
                 while (kk >= T1) kk -= T1;
             }
         }
         loss = warp_sum(loss);                     // lane-local shares, fixed butterfly order
-        row_store<FPL>(GU, pos, lane, acc);
+        sum_over_groups<DIM>(acc);                 // fixed order as well
+        if (grp == 0) grow_store<DIM>(GU, pos, sub, acc);
         if (lane == 0) {
             keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
             loss_pos[pos] = (double)loss;
@@ -640,12 +731,12 @@ struct SgnsArgs {
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
-template <int FPL, bool RED, int MINB>
+template <int DIM, bool RED, int MINB>
 static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
     const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(a.L + SL);
-    auto kern = sgns_hogwild_kernel<FPL, RED, MINB>;
+    auto kern = sgns_hogwild_kernel<DIM, RED, MINB>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -654,27 +745,33 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
     int64_t blocks = (a.n_walks + SGNS_WARPS - 1) / SGNS_WARPS;
     const int64_t cap = (int64_t)sm_count() * per_sm;
     if (blocks > cap) blocks = cap;
+    void *ws = nullptr;
+    gs_status ws_s = workspace_get(WS_COUNTERS, 256, &ws);
+    if (ws_s != GS_OK) return ws_s;
+    unsigned long long *ticket = (unsigned long long *)((char *)ws + 128);   // bytes 0..127: other counters
+    GS_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned long long), st));
     kern<<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
         a.w_in, a.w_out, a.walks, a.n_walks, a.walk_id_base, a.L, a.w, a.K, a.alias,
         (uint32_t)a.n_nodes, a.lr, a.seed, a.loss, (unsigned long long *)a.pairs, a.dump_pairs,
-        a.dump_negs);
+        a.dump_negs, ticket);
     GS_CUDA_TRY(cudaGetLastError());
     return GS_OK;
 }
 
 // Resident blocks per SM asked of the compiler: 5 blocks of 4 warps (96 registers per thread)
 // measured best for rows of up to 128 floats; wider rows need the registers.
-template <int FPL, bool RED>
+template <int DIM, bool RED>
 static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
-    return run_hogwild_b<FPL, RED, (FPL <= 4 ? 5 : 4)>(a, st);
+    return run_hogwild_b<DIM, RED, (DIM <= 128 ? 5 : 4)>(a, st);
 }
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
-template <int FPL>
+template <int DIM>
 static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
 {
+    constexpr int FPL = DIM / 32;                        // the apply passes use a whole warp per row
     const int SL = 2 * a.w * (1 + a.K);
     const int64_t n_pos = a.n_walks * a.L;
     const int64_t n_slots = n_pos * SL;
@@ -714,7 +811,7 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
         int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
         const int64_t cap = (int64_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
-        sgns_coef_kernel<FPL><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+        sgns_coef_kernel<DIM><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
             a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
             (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
             a.dump_pairs, a.dump_negs);
@@ -749,12 +846,12 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
     return GS_OK;
 }
 
-template <int FPL>
+template <int DIM>
 static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
 {
-    if (mode == GS_DETERMINISTIC) return run_deterministic<FPL>(a, st);
-    if (mode == GS_HOGWILD) return run_hogwild<FPL, false>(a, st);
-    return run_hogwild<FPL, true>(a, st);
+    if (mode == GS_DETERMINISTIC) return run_deterministic<DIM>(a, st);
+    if (mode == GS_HOGWILD) return run_hogwild<DIM, false>(a, st);
+    return run_hogwild<DIM, true>(a, st);
 }
 
 gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
@@ -766,10 +863,10 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
                    seed, loss, pairs, dump_pairs, dump_negs };
     switch (dim) {
-        case 32: return run_mode<1>(a, mode, st);
-        case 64: return run_mode<2>(a, mode, st);
-        case 128: return run_mode<4>(a, mode, st);
-        case 256: return run_mode<8>(a, mode, st);
+        case 32: return run_mode<32>(a, mode, st);
+        case 64: return run_mode<64>(a, mode, st);
+        case 128: return run_mode<128>(a, mode, st);
+        case 256: return run_mode<256>(a, mode, st);
         default:
             set_error("dim %d not supported (32, 64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;
@@ -809,9 +906,10 @@ static gs_status static_scratch_address(unsigned char **out)
 
 // Same kernels and the same order of launches as run_deterministic, with the scratch
 // carved out of the fixed array instead of the growing per-device cache.
-template <int FPL>
+template <int DIM>
 static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scratch, cudaStream_t st)
 {
+    constexpr int FPL = DIM / 32;
     const int SL = 2 * a.w * (1 + a.K);
     const int64_t n_pos = a.n_walks * a.L;
     const int64_t n_slots = n_pos * SL;
@@ -851,7 +949,7 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
         int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
         const int64_t cap = (int64_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
-        sgns_coef_kernel<FPL><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+        sgns_coef_kernel<DIM><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
             a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
             (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
             a.dump_pairs, a.dump_negs);
@@ -915,10 +1013,10 @@ extern "C" gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t 
                    n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr };
     cudaStream_t st = (cudaStream_t)stream;
     switch (dim) {
-        case 32: return run_deterministic_static<1>(a, scratch, st);
-        case 64: return run_deterministic_static<2>(a, scratch, st);
-        case 128: return run_deterministic_static<4>(a, scratch, st);
-        case 256: return run_deterministic_static<8>(a, scratch, st);
+        case 32: return run_deterministic_static<32>(a, scratch, st);
+        case 64: return run_deterministic_static<64>(a, scratch, st);
+        case 128: return run_deterministic_static<128>(a, scratch, st);
+        case 256: return run_deterministic_static<256>(a, scratch, st);
         default:
             set_error("dim %d not supported (32, 64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;

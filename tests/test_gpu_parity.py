@@ -284,11 +284,12 @@ def test_lock_free_modes_draw_the_same_pairs_and_negatives(tiny, mode):
     assert 0.9 * (cnt + unmasked) * np.log(2) < loss <= (cnt + unmasked) * np.log(2) * (1 + 1e-6)
 
 
-def test_lock_free_single_walk_equals_sequential_oracle():
+@pytest.mark.parametrize("dim", [32, 64, 128, 256])
+def test_lock_free_single_walk_equals_sequential_oracle(dim):
     # One walk = one warp running its positions in order: no races between warps.  Rows that
     # repeat inside one chunk of targets are the only difference to strictly sequential SGD,
     # so use a walk and negatives without repeats.
-    n, dim, L, w, K = 4000, 128, 12, 2, 3
+    n, L, w, K = 4000, 12, 2, 3
     rng = np.random.default_rng(4)
     walk = rng.permutation(n)[:L].astype(np.int32)[None, :]
     thr, alias = O.build_alias(np.ones(n), 1.0)

@@ -409,6 +409,60 @@ int gso_sgns_det_from_lists(double *U, double *V, int64_t n_rows, int32_t d,
 }
 
 /* ------------------------------------------------------------------------
+ * Summed gradients of a mini-batch at fixed tables: the GU, GV of the
+ * synchronous step above, returned instead of applied (both arrays are
+ * n_rows x d and are overwritten).  Used by the momentum update below.
+ * ---------------------------------------------------------------------- */
+int gso_sgns_grad_from_lists(const double *U, const double *V, int64_t n_rows, int32_t d,
+                             int64_t n_slots, int32_t K,
+                             const int32_t *centers, const int32_t *contexts,
+                             const int32_t *negs, double *GU, double *GV,
+                             double *loss_sum, int64_t *pair_count)
+{
+    memset(GU, 0, sizeof(double) * (size_t)(n_rows * d));
+    memset(GV, 0, sizeof(double) * (size_t)(n_rows * d));
+    double loss = 0.0;
+    int64_t pairs = 0;
+    for (int64_t e = 0; e < n_slots; ++e) {
+        if (centers[e] < 0) continue;
+        int64_t c = centers[e], o = contexts[e];
+        const double *u = U + c * d;
+        ++pairs;
+        for (int32_t k = -1; k < K; ++k) {
+            int64_t t = (k < 0) ? o : negs[e * K + k];
+            if (k >= 0 && (t < 0 || t == o)) continue;
+            const double *v = V + t * d;
+            double f = dot(u, v, d);
+            double g = (k < 0) ? sigmoid(f) - 1.0 : sigmoid(f);
+            loss += (k < 0) ? softplus(-f) : softplus(f);
+            for (int32_t j = 0; j < d; ++j) {
+                GU[c * d + j] += g * v[j];
+                GV[t * d + j] += g * u[j];
+            }
+        }
+    }
+    if (loss_sum) *loss_sum = loss;
+    if (pair_count) *pair_count = pairs;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * SGD with momentum as the paper's storage applies it (Section 3.2, the
+ * description of the momentum update): per iteration, over the WHOLE table,
+ *   momentum <- mu * momentum            (mult)
+ *   momentum[rows of the batch] += grad  (put)
+ *   model    <- model - lr * momentum    (mult_add)
+ * x, m, g are arrays of n values (a table flattened); g is zero outside the
+ * batch's rows.
+ * ---------------------------------------------------------------------- */
+void gso_momentum_update(double *x, double *m, const double *g, int64_t n, double lr, double mu)
+{
+    for (int64_t i = 0; i < n; ++i) m[i] = mu * m[i];
+    for (int64_t i = 0; i < n; ++i) m[i] += g[i];
+    for (int64_t i = 0; i < n; ++i) x[i] -= lr * m[i];
+}
+
+/* ------------------------------------------------------------------------
  * Sequential per-pair SGD (each pair sees all earlier updates): the
  * race-free limit of the lock-free mode of Section 3.2 "Synchronization".
  * For each center position the center row is held fixed while its pairs

@@ -186,6 +186,37 @@ def sgns_det_from_lists(U, V, centers, contexts, negs, lr, order=None):
     return float(loss.value), int(cnt.value)
 
 
+def sgns_grad_from_lists(U, V, centers, contexts, negs):
+    """Summed mini-batch gradients at fixed tables.  Returns (GU, GV, loss_sum, pair_count)."""
+    n_rows, d = U.shape
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    K = negs.shape[1]
+    GU, GV = np.empty_like(U), np.empty_like(V)
+    loss = ctypes.c_double(0.0)
+    cnt = ctypes.c_int64(0)
+    lib().gso_sgns_grad_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int64(n_rows), ctypes.c_int32(d),
+        ctypes.c_int64(len(centers)), ctypes.c_int32(K), _p(centers, ctypes.c_int32),
+        _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32), _p(GU, ctypes.c_double),
+        _p(GV, ctypes.c_double), ctypes.byref(loss), ctypes.byref(cnt))
+    return GU, GV, float(loss.value), int(cnt.value)
+
+
+def momentum_update(x, m, g, lr, mu):
+    """In place: m <- mu m; m += g; x <- x - lr m, over whole tables (Section 3.2)."""
+    assert x.flags.c_contiguous and m.flags.c_contiguous and g.flags.c_contiguous
+    lib().gso_momentum_update(_p(x, ctypes.c_double), _p(m, ctypes.c_double), _p(g, ctypes.c_double),
+                              ctypes.c_int64(x.size), ctypes.c_double(lr), ctypes.c_double(mu))
+
+
+def sgns_momentum_step_from_lists(U, V, MU, MV, centers, contexts, negs, lr, mu):
+    """Synchronous mini-batch step with momentum on dense float64 tables, in place."""
+    GU, GV, loss, cnt = sgns_grad_from_lists(U, V, centers, contexts, negs)
+    momentum_update(U, MU, GU, lr, mu)
+    momentum_update(V, MV, GV, lr, mu)
+    return loss, cnt
+
+
 def sgns_seq_from_lists(U, V, centers, contexts, negs, S, lr):
     """Sequential per-pair SGD in place (race-free limit of the lock-free mode)."""
     assert U.dtype == np.float64 and V.dtype == np.float64

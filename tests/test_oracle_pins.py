@@ -423,6 +423,53 @@ def test_sequential_mode_sees_earlier_updates():
     assert np.allclose(Vb[2], v2, atol=1e-14)
 
 
+# ---------------------------------------------------------------- momentum
+def test_gradient_function_agrees_with_the_synchronous_step():
+    U, V, c, o, ng, n_pairs = small_problem(8)
+    GU, GV, loss, cnt = O.sgns_grad_from_lists(U, V, c, o, ng)
+    U1, V1 = U.copy(), V.copy()
+    l1, c1 = O.sgns_det_from_lists(U1, V1, c, o, ng, 0.5)
+    assert cnt == c1 == n_pairs and abs(loss - l1) < 1e-12 * abs(l1)
+    assert np.allclose((U - U1) / 0.5, GU, atol=1e-13) and np.allclose((V - V1) / 0.5, GV, atol=1e-13)
+
+
+def test_momentum_update_matches_library_sgd_and_closed_forms():
+    rng = np.random.default_rng(9)
+    x0 = rng.normal(size=(7, 5))
+    grads = [rng.normal(size=(7, 5)) * (rng.random((7, 1)) < 0.5) for _ in range(6)]   # sparse rows
+    lr, mu = 0.05, 0.9
+    # library routine: torch.optim.SGD(momentum) is buf <- mu buf + g ; p <- p - lr buf
+    p = torch.tensor(x0.copy(), requires_grad=True)
+    opt = torch.optim.SGD([p], lr=lr, momentum=mu)
+    x, m = x0.copy(), np.zeros_like(x0)
+    for g in grads:
+        p.grad = torch.tensor(g)
+        opt.step()
+        O.momentum_update(x, m, np.ascontiguousarray(g), lr, mu)
+        assert np.allclose(x, p.detach().numpy(), atol=1e-14)
+    # mu = 0 is plain SGD
+    x, m = x0.copy(), np.zeros_like(x0)
+    O.momentum_update(x, m, grads[0], lr, 0.0)
+    assert np.allclose(x, x0 - lr * grads[0], atol=1e-15)
+    # one impulse, then k iterations without gradient: geometric series
+    x, m = x0.copy(), np.zeros_like(x0)
+    O.momentum_update(x, m, grads[1], lr, mu)
+    zero = np.zeros_like(x0)
+    for _ in range(4):
+        O.momentum_update(x, m, zero, lr, mu)
+    assert np.allclose(x, x0 - lr * grads[1] * (1 - mu ** 5) / (1 - mu), atol=1e-13)
+    assert np.allclose(m, grads[1] * mu ** 4, atol=1e-14)
+
+
+def test_momentum_step_with_zero_momentum_is_the_synchronous_step():
+    U, V, c, o, ng, _ = small_problem(10)
+    Ua, Va, Ub, Vb = U.copy(), V.copy(), U.copy(), V.copy()
+    la, ca = O.sgns_det_from_lists(Ua, Va, c, o, ng, 0.1)
+    lb, cb = O.sgns_momentum_step_from_lists(Ub, Vb, np.zeros_like(U), np.zeros_like(V), c, o, ng, 0.1, 0.0)
+    assert ca == cb and abs(la - lb) < 1e-12
+    assert np.allclose(Ua, Ub, atol=1e-14) and np.allclose(Va, Vb, atol=1e-14)
+
+
 # ---------------------------------------------------------------- initialisation
 def test_initial_rows_are_uniform_and_exact_in_single_precision():
     rows = np.arange(0, 4000, dtype=np.int64) * 12345

@@ -238,6 +238,44 @@ GS_API gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t n_no
                                      uint64_t seed, double *d_loss_sum, int64_t *d_pair_count,
                                      void *stream);
 
+/*
+ * Synchronous mini-batch step with SGD momentum (Section 3.2, the momentum
+ * update carried out inside the storage: multiply the momentum matrix by the
+ * momentum value, add the batch's gradients to its rows, subtract lr times
+ * the momentum from the model).  Defined densely, for EVERY row per iteration,
+ *   m <- momentum * m ;  m[rows of the batch] += grad ;  w <- w - lr * m
+ * but applied sparsely: a row that a batch does not touch is brought up to
+ * date only when a later batch reads it (k missed iterations:
+ * w -= lr m (mu + ... + mu^k), m *= mu^k), which is the same arithmetic up to
+ * rounding as long as lr and momentum are THE SAME IN EVERY CALL of a run.
+ *   d_m_in, d_m_out       : momentum tables, same shape as the embedding tables,
+ *                           zero before the first iteration
+ *   d_last_in, d_last_out : int32[n_nodes], iteration up to which each row is
+ *                           current; zero before the first iteration
+ *   iteration             : 0, 1, 2, ... one per call; gradients as in
+ *                           gs_sgns_step(GS_DETERMINISTIC) (same pairs, draws,
+ *                           summation order, no floating-point atomics)
+ * Between calls only rows with d_last == iteration are current; call
+ * gs_momentum_flush on each table before reading the tables elsewhere.
+ * 0 <= momentum < 1.  Scratch as for the deterministic step.
+ */
+GS_API gs_status gs_sgns_step_momentum(float *d_w_in, float *d_w_out, float *d_m_in, float *d_m_out,
+                                       int32_t *d_last_in, int32_t *d_last_out, int64_t n_nodes,
+                                       int32_t dim, const int32_t *d_walks, int64_t n_walks,
+                                       int64_t walk_id_base, int32_t walk_len, int32_t window,
+                                       int32_t n_neg, const uint64_t *d_alias, float lr,
+                                       float momentum, int32_t iteration, uint64_t seed,
+                                       double *d_loss_sum, int64_t *d_pair_count, void *stream);
+
+/*
+ * Brings every row of one table (and its momentum) up to `iteration`, i.e. to
+ * the state the dense definition above has after `iteration` iterations, and
+ * stamps d_last.  One pass over the table.
+ */
+GS_API gs_status gs_momentum_flush(float *d_w, float *d_m, int32_t *d_last, int64_t n_rows,
+                                   int32_t dim, float lr, float momentum, int32_t iteration,
+                                   void *stream);
+
 #define GS_WALK_UNIFORM   0
 #define GS_WALK_NODE2VEC  1
 #define GS_LR_CONSTANT    0

@@ -26,7 +26,7 @@ GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
 EXPORTS = [
     "gs_last_error", "gs_graph_load_csr", "gs_graph_free", "gs_graph_info", "gs_build_alias",
     "gs_init_embeddings", "gs_random_walks", "gs_node2vec_walks", "gs_sgns_step",
-    "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static",
+    "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static", "gs_sgns_step_momentum", "gs_momentum_flush",
 ]
 
 
@@ -210,6 +210,32 @@ def gs_sgns_step_static(w_in, w_out, walks, walk_id_base: int, window: int, n_ne
         ctypes.c_float(lr), ctypes.c_uint64(seed),
         _dev(loss_sum, torch.float64, "loss_sum", True), _dev(pair_count, torch.int64, "pair_count", True),
         _stream()))
+
+
+def gs_sgns_step_momentum(w_in, w_out, m_in, m_out, last_in, last_out, walks, walk_id_base: int,
+                          window: int, n_neg: int, alias, lr: float, momentum: float, iteration: int,
+                          seed: int, loss_sum=None, pair_count=None):
+    """Synchronous step with SGD momentum, rows updated lazily (see gs.h)."""
+    n_nodes, dim = w_in.shape
+    n_walks, walk_len = walks.shape
+    _check(lib().gs_sgns_step_momentum(
+        _dev(w_in, torch.float32, "w_in"), _dev(w_out, torch.float32, "w_out"),
+        _dev(m_in, torch.float32, "m_in"), _dev(m_out, torch.float32, "m_out"),
+        _dev(last_in, torch.int32, "last_in"), _dev(last_out, torch.int32, "last_out"),
+        ctypes.c_int64(n_nodes), ctypes.c_int32(dim), _dev(walks, torch.int32, "walks", n_walks == 0),
+        ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base), ctypes.c_int32(walk_len),
+        ctypes.c_int32(window), ctypes.c_int32(n_neg), _dev(alias, torch.int64, "alias", n_neg == 0),
+        ctypes.c_float(lr), ctypes.c_float(momentum), ctypes.c_int32(iteration), ctypes.c_uint64(seed),
+        _dev(loss_sum, torch.float64, "loss_sum", True), _dev(pair_count, torch.int64, "pair_count", True),
+        _stream()))
+
+
+def gs_momentum_flush(w, m, last, lr: float, momentum: float, iteration: int):
+    n_rows, dim = w.shape
+    _check(lib().gs_momentum_flush(
+        _dev(w, torch.float32, "w"), _dev(m, torch.float32, "m"), _dev(last, torch.int32, "last"),
+        ctypes.c_int64(n_rows), ctypes.c_int32(dim), ctypes.c_float(lr), ctypes.c_float(momentum),
+        ctypes.c_int32(iteration), _stream()))
 
 
 @dataclass

@@ -33,6 +33,14 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
                     const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                     int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st);
 
+gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_out, int32_t *last_in,
+                             int32_t *last_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                             int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                             const uint64_t *alias, float lr, float mu, int32_t iter, uint64_t seed,
+                             double *loss, int64_t *pairs, cudaStream_t st);
+gs_status momentum_flush(float *w, float *m, int32_t *last, int64_t n_rows, int32_t dim, float lr,
+                         float mu, int32_t iter, cudaStream_t st);
+
 // ---- errors ----------------------------------------------------------------------
 static thread_local char g_err[512] = "";
 
@@ -364,6 +372,42 @@ gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t d
     return sgns_step(d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len,
                      window, n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count,
                      d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------ momentum
+gs_status gs_sgns_step_momentum(float *d_w_in, float *d_w_out, float *d_m_in, float *d_m_out,
+                                int32_t *d_last_in, int32_t *d_last_out, int64_t n_nodes,
+                                int32_t dim, const int32_t *d_walks, int64_t n_walks,
+                                int64_t walk_id_base, int32_t walk_len, int32_t window, int32_t n_neg,
+                                const uint64_t *d_alias, float lr, float momentum, int32_t iteration,
+                                uint64_t seed, double *d_loss_sum, int64_t *d_pair_count, void *stream)
+{
+    if (!d_w_in || !d_w_out || !d_m_in || !d_m_out || !d_last_in || !d_last_out)
+        return invalid("table, momentum or stamp pointer is NULL");
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
+    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
+    if (n_walks > 0 && !d_walks) return invalid("d_walks is NULL");
+    if (!(momentum >= 0.f) || !(momentum < 1.f)) return invalid("momentum must be in [0, 1)");
+    if (iteration < 0 || iteration == 0x7FFFFFFF) return invalid("iteration must be in [0, 2^31 - 1)");
+    gs_status s = check_sgns_shape(dim, walk_len, window, n_neg, GS_DETERMINISTIC);
+    if (s != GS_OK) return s;
+    if (n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
+    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out | (uintptr_t)d_m_in | (uintptr_t)d_m_out) & 15)
+        return invalid("tables must be 16-byte aligned");
+    return sgns_step_momentum(d_w_in, d_w_out, d_m_in, d_m_out, d_last_in, d_last_out, n_nodes, dim,
+                              d_walks, n_walks, walk_id_base, walk_len, window, n_neg, d_alias, lr,
+                              momentum, iteration, seed, d_loss_sum, d_pair_count, (cudaStream_t)stream);
+}
+
+gs_status gs_momentum_flush(float *d_w, float *d_m, int32_t *d_last, int64_t n_rows, int32_t dim,
+                            float lr, float momentum, int32_t iteration, void *stream)
+{
+    if (!d_w || !d_m || !d_last) return invalid("null pointer");
+    if (n_rows < 0) return invalid("n_rows < 0");
+    if (!dim_ok(dim)) { set_error("dim %d not supported (32, 64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
+    if (!(momentum >= 0.f) || !(momentum < 1.f)) return invalid("momentum must be in [0, 1)");
+    if (iteration < 0) return invalid("iteration < 0");
+    return momentum_flush(d_w, d_m, d_last, n_rows, dim, lr, momentum, iteration, (cudaStream_t)stream);
 }
 
 // ------------------------------------------------------------------ epoch driver

@@ -398,7 +398,9 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
 //   keys[x] = destination row of w_out (or `invalid`), gbuf[x] = coefficient g,
 // and per position: keys[n_slots + pos] = n_nodes + center (or `invalid`),
 // GU[pos] = sum g * v (gradient of the center row), loss_pos, pairs_pos.
-template <int DIM>
+// MODE 0: everything.  MODE 1: keys only (no table is read; used by the momentum step to learn
+// which rows the batch will touch before it reads them).  MODE 2: everything but the keys.
+template <int DIM, int MODE>
 __global__ void __launch_bounds__(SGNS_WARPS * 32)
 sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out,
                  const int32_t *__restrict__ walks, int64_t n_pos, int64_t walk_id_base, int32_t L,
@@ -439,7 +441,12 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
         else
             dump_empty_position(S, K, lane, dp, dn);
         if (pairs == 0) {
-            for (int x = lane; x < SL; x += 32) { kp[x] = invalid; gp[x] = 0.f; }
+            for (int x = lane; x < SL; x += 32) {
+                if (MODE != 2) kp[x] = invalid;
+                if (MODE != 1) gp[x] = 0.f;
+            }
+        } else if (MODE == 1) {
+            for (int x = lane; x < SL; x += 32) kp[x] = tgt[x] >= 0 ? (uint32_t)tgt[x] : invalid;
         } else {
             const Row<FPL> u = grow_load<DIM>(w_in, c, sub);
             int kk = 0;
@@ -466,7 +473,7 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
                 const int32_t my_id = mine ? tgt[my_t] : -1;
                 const float my_g = lane_coefficient<TCH>(f, sub, my_id, my_kt == 0, loss);
                 if (mine) {
-                    kp[my_t] = my_id >= 0 ? (uint32_t)my_id : invalid;
+                    if (MODE != 2) kp[my_t] = my_id >= 0 ? (uint32_t)my_id : invalid;
                     gp[my_t] = my_g;
                 }
 #pragma unroll
@@ -483,13 +490,132 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
         }
         loss = warp_sum(loss);                     // lane-local shares, fixed butterfly order
         sum_over_groups<DIM>(acc);                 // fixed order as well
-        if (grp == 0) grow_store<DIM>(GU, pos, sub, acc);
+        if (MODE != 1 && grp == 0) grow_store<DIM>(GU, pos, sub, acc);
         if (lane == 0) {
-            keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
-            loss_pos[pos] = (double)loss;
-            pairs_pos[pos] = pairs;
+            if (MODE != 2) keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
+            if (MODE != 1) { loss_pos[pos] = (double)loss; pairs_pos[pos] = pairs; }
         }
     }
+}
+
+// Optional momentum state of a table (m == nullptr: plain SGD).  With momentum the write of a
+// row is  m <- mu m + grad ; row <- row - lr m ; last[row] <- next_iter  (Section 3.2: mult, put,
+// mult_add, restricted to the rows of the batch; the other rows are brought up to date lazily by
+// momentum_catchup before they are read again).
+struct MomState {
+    float *m;
+    int32_t *last;
+    float mu;
+    int32_t next_iter;
+};
+
+template <int FPL>
+__device__ __forceinline__ void write_updated_row(float *__restrict__ tab, int64_t r, int lane,
+                                                  Row<FPL> &row, const double (&acc)[FPL], float lr,
+                                                  const MomState &ms)
+{
+    if (ms.m) {
+        Row<FPL> m = row_load<FPL>(ms.m, r, lane);
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) {
+            const double mm = (double)ms.mu * (double)m.v[j] + acc[j];
+            m.v[j] = (float)mm;
+            row.v[j] = (float)((double)row.v[j] - (double)lr * mm);
+        }
+        row_store<FPL>(ms.m, r, lane, m);
+        if (lane == 0) ms.last[r] = ms.next_iter;
+    } else {
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
+    }
+    row_store<FPL>(tab, r, lane, row);
+}
+
+// A row last written at iteration `last` and read at iteration `iter` missed k = iter - last
+// dense updates without gradient:  row -= lr m (mu + ... + mu^k),  m *= mu^k.
+__device__ __forceinline__ void catchup_factors(float mu, int k, double &f_row, double &f_m)
+{
+    f_m = pow((double)mu, (double)k);
+    f_row = (double)mu * (1.0 - f_m) / (1.0 - (double)mu);
+}
+
+// One warp per 32 sorted keys: every run head is a distinct row the batch is about to read.
+template <int FPL>
+__global__ void __launch_bounds__(256)
+momentum_catchup_kernel(float *__restrict__ w_in, float *__restrict__ w_out, MomState ms_in,
+                        MomState ms_out, const uint32_t *__restrict__ keys, uint32_t n_keys,
+                        uint32_t n_nodes, float lr, int32_t iter)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t n_chunks = ((int64_t)n_keys + 31) >> 5;
+    for (int64_t ch = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); ch < n_chunks;
+         ch += n_warps) {
+        const int64_t i = ch * 32 + lane;
+        const uint32_t key = i < n_keys ? keys[i] : 0xFFFFFFFFu;
+        const bool head = i < n_keys && key < 2u * n_nodes && (i == 0 || keys[i - 1] != key);
+        const bool is_out = key < n_nodes;
+        const uint32_t r = is_out ? key : key - n_nodes;
+        int k = 0;
+        if (head) {
+            int32_t *lp = (is_out ? ms_out.last : ms_in.last) + r;
+            k = iter - *lp;
+            if (k > 0) *lp = iter;
+        }
+        unsigned todo = __ballot_sync(0xffffffffu, head && k > 0);
+        while (todo) {
+            const int l = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const uint32_t rr = __shfl_sync(0xffffffffu, r, l);
+            const int kk = __shfl_sync(0xffffffffu, k, l);
+            const bool out = __shfl_sync(0xffffffffu, (int)is_out, l) != 0;
+            float *tab = out ? w_out : w_in;
+            float *mt = out ? ms_out.m : ms_in.m;
+            double f_row, f_m;
+            catchup_factors(ms_out.mu, kk, f_row, f_m);
+            Row<FPL> row = row_load<FPL>(tab, rr, lane);
+            Row<FPL> m = row_load<FPL>(mt, rr, lane);
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) {
+                row.v[j] = (float)((double)row.v[j] - (double)lr * f_row * (double)m.v[j]);
+                m.v[j] = (float)(f_m * (double)m.v[j]);
+            }
+            row_store<FPL>(tab, rr, lane, row);
+            row_store<FPL>(mt, rr, lane, m);
+        }
+    }
+}
+
+// Dense catch-up of a whole table (end of training, or before the table is read elsewhere).
+__global__ void __launch_bounds__(256)
+momentum_flush_kernel(float *__restrict__ w, float *__restrict__ m, int32_t *__restrict__ last,
+                      int64_t n_rows, int32_t dim, float lr, float mu, int32_t iter)
+{
+    const int32_t quads = dim >> 2;
+    const int64_t total = n_rows * quads;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < total; x += stride) {
+        const int64_t row = x / quads;
+        const int k = iter - last[row];
+        if (k <= 0) continue;
+        double f_row, f_m;
+        catchup_factors(mu, k, f_row, f_m);
+        float4 a = reinterpret_cast<float4 *>(w)[x], b = reinterpret_cast<float4 *>(m)[x];
+        a.x = (float)((double)a.x - (double)lr * f_row * (double)b.x); b.x = (float)(f_m * (double)b.x);
+        a.y = (float)((double)a.y - (double)lr * f_row * (double)b.y); b.y = (float)(f_m * (double)b.y);
+        a.z = (float)((double)a.z - (double)lr * f_row * (double)b.z); b.z = (float)(f_m * (double)b.z);
+        a.w = (float)((double)a.w - (double)lr * f_row * (double)b.w); b.w = (float)(f_m * (double)b.w);
+        reinterpret_cast<float4 *>(w)[x] = a;
+        reinterpret_cast<float4 *>(m)[x] = b;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+momentum_stamp_kernel(int32_t *__restrict__ last, int64_t n_rows, int32_t iter)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < n_rows; x += stride)
+        if (last[x] < iter) last[x] = iter;
 }
 
 // Passes 3 and 4 walk the sorted keys in chunks of 32: lane l looks at key 32*chunk + l and
@@ -511,7 +637,7 @@ sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
                       const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
                       const uint32_t *__restrict__ vals, const float *__restrict__ gbuf,
                       uint32_t n_keys, uint32_t n_nodes, int32_t SL, float lr,
-                      double *__restrict__ lead_part, double *__restrict__ tail_part)
+                      double *__restrict__ lead_part, double *__restrict__ tail_part, MomState ms)
 {
     // One warp per block of RUN_CUT sorted positions.  The 32 lanes fetch the metadata of 32
     // contributions at once; rows are then fetched G at a time - the center row of every
@@ -543,9 +669,7 @@ sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
 #pragma unroll
                 for (int j = 0; j < FPL; ++j) dst[j * 32 + lane] = acc[j];
             } else {
-#pragma unroll
-                for (int j = 0; j < FPL; ++j) cur_v.v[j] = (float)((double)cur_v.v[j] - (double)lr * acc[j]);
-                row_store<FPL>(w_out, cur_key, lane, cur_v);
+                write_updated_row<FPL>(w_out, cur_key, lane, cur_v, acc, lr, ms);
             }
         };
 
@@ -608,7 +732,8 @@ template <int FPL>
 __global__ void __launch_bounds__(256)
 sgns_apply_out_fixup_kernel(float *__restrict__ w_out, const uint32_t *__restrict__ keys,
                             uint32_t n_keys, uint32_t n_nodes, float lr,
-                            const double *__restrict__ lead_part, const double *__restrict__ tail_part)
+                            const double *__restrict__ lead_part, const double *__restrict__ tail_part,
+                            MomState ms)
 {
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -629,9 +754,7 @@ sgns_apply_out_fixup_kernel(float *__restrict__ w_out, const uint32_t *__restric
             for (int j = 0; j < FPL; ++j) acc[j] += l[j * 32 + lane];
         }
         Row<FPL> row = row_load<FPL>(w_out, key, lane);
-#pragma unroll
-        for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
-        row_store<FPL>(w_out, key, lane, row);
+        write_updated_row<FPL>(w_out, key, lane, row, acc, lr, ms);
     }
 }
 
@@ -640,7 +763,7 @@ template <int FPL>
 __global__ void __launch_bounds__(256)
 sgns_apply_in_kernel(float *__restrict__ w_in, const float *__restrict__ GU,
                      const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals,
-                     uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, float lr)
+                     uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, float lr, MomState ms)
 {
     constexpr int U = FPL <= 4 ? 8 : 4;
     const int lane = threadIdx.x & 31;
@@ -683,9 +806,7 @@ sgns_apply_in_kernel(float *__restrict__ w_in, const float *__restrict__ GU,
             }
             const int64_t c = (int64_t)(key - n_nodes);
             Row<FPL> row = row_load<FPL>(w_in, c, lane);
-#pragma unroll
-            for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
-            row_store<FPL>(w_in, c, lane, row);
+            write_updated_row<FPL>(w_in, c, lane, row, acc, lr, ms);
         }
     }
 }
@@ -768,10 +889,23 @@ static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// Momentum state handed in by gs_sgns_step_momentum (nullptr for the plain step).
+struct MomHost {
+    float *m_in, *m_out;
+    int32_t *last_in, *last_out;
+    float mu;
+    int32_t iter;
+};
+
 template <int DIM>
-static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
+static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const MomHost *mom = nullptr)
 {
     constexpr int FPL = DIM / 32;                        // the apply passes use a whole warp per row
+    MomState ms_in = { nullptr, nullptr, 0.f, 0 }, ms_out = { nullptr, nullptr, 0.f, 0 };
+    if (mom) {
+        ms_in = MomState{ mom->m_in, mom->last_in, mom->mu, mom->iter + 1 };
+        ms_out = MomState{ mom->m_out, mom->last_out, mom->mu, mom->iter + 1 };
+    }
     const int SL = 2 * a.w * (1 + a.K);
     const int64_t n_pos = a.n_walks * a.L;
     const int64_t n_slots = n_pos * SL;
@@ -806,36 +940,45 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st)
     double *lead_part = (double *)p; p += b_part;
     double *tail_part = (double *)p;
 
-    {
-        const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
-        int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
-        const int64_t cap = (int64_t)sm_count() * 16;
-        if (blocks > cap) blocks = cap;
-        sgns_coef_kernel<DIM><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
-            a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
-            (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
-            a.dump_pairs, a.dump_negs);
-        GS_CUDA_TRY(cudaGetLastError());
-    }
+    const size_t coef_smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
+    int64_t coef_blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
+    if (coef_blocks > (int64_t)sm_count() * 16) coef_blocks = (int64_t)sm_count() * 16;
+#define GS_COEF(MODE)                                                                              \
+    sgns_coef_kernel<DIM, MODE><<<(unsigned)coef_blocks, SGNS_WARPS * 32, coef_smem, st>>>(         \
+        a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias, (uint32_t)a.n_nodes, \
+        (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos, a.dump_pairs, a.dump_negs)
+    if (mom) GS_COEF(1); else GS_COEF(0);            // with momentum: the keys first, no table reads
+    GS_CUDA_TRY(cudaGetLastError());
     uint32_t *ks = nullptr, *vs = nullptr;
     radix_sort_pairs(keysA, valsA, keysB, valsB, (uint32_t)n_keys,
                      bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
     GS_CUDA_TRY(cudaGetLastError());
+    if (mom) {
+        // bring every row the batch touches up to iteration `iter`, then compute the coefficients
+        int64_t cb = (n_keys + 255) / 256;
+        if (cb > (int64_t)sm_count() * 64) cb = (int64_t)sm_count() * 64;
+        momentum_catchup_kernel<FPL><<<(unsigned)cb, 256, 0, st>>>(
+            a.w_in, a.w_out, ms_in, ms_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, mom->iter);
+        GS_CUDA_TRY(cudaGetLastError());
+        GS_COEF(2);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+#undef GS_COEF
     {
         int64_t blocks = (n_keys + 255) / 256;                  // 8 warps x 32 keys per block
         const int64_t cap = (int64_t)sm_count() * 8 * 8;
         if (blocks > cap) blocks = cap;
         sgns_apply_out_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
             a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
-            lead_part, tail_part);
+            lead_part, tail_part, ms_out);
         GS_CUDA_TRY(cudaGetLastError());
         if (n_cut > 1) {
             sgns_apply_out_fixup_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part);
+                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part, ms_out);
             GS_CUDA_TRY(cudaGetLastError());
         }
         sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
-            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr);
+            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr, ms_in);
         GS_CUDA_TRY(cudaGetLastError());
     }
     if (a.loss || a.pairs) {
@@ -871,6 +1014,44 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
             set_error("dim %d not supported (32, 64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;
     }
+}
+
+gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_out, int32_t *last_in,
+                             int32_t *last_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                             int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                             const uint64_t *alias, float lr, float mu, int32_t iter, uint64_t seed,
+                             double *loss, int64_t *pairs, cudaStream_t st)
+{
+    if (n_walks == 0) return GS_OK;
+    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                   seed, loss, pairs, nullptr, nullptr };
+    MomHost mom = { m_in, m_out, last_in, last_out, mu, iter };
+    switch (dim) {
+        case 32: return run_deterministic<32>(a, st, &mom);
+        case 64: return run_deterministic<64>(a, st, &mom);
+        case 128: return run_deterministic<128>(a, st, &mom);
+        case 256: return run_deterministic<256>(a, st, &mom);
+        default:
+            set_error("dim %d not supported (32, 64, 128, 256)", dim);
+            return GS_ERR_UNSUPPORTED;
+    }
+}
+
+gs_status momentum_flush(float *w, float *m, int32_t *last, int64_t n_rows, int32_t dim, float lr,
+                         float mu, int32_t iter, cudaStream_t st)
+{
+    if (n_rows == 0) return GS_OK;
+    const int64_t total = n_rows * (dim >> 2);
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 32;
+    if (blocks > cap) blocks = cap;
+    momentum_flush_kernel<<<(unsigned)blocks, 256, 0, st>>>(w, m, last, n_rows, dim, lr, mu, iter);
+    GS_CUDA_TRY(cudaGetLastError());
+    int64_t b2 = (n_rows + 255) / 256;
+    if (b2 > cap) b2 = cap;
+    momentum_stamp_kernel<<<(unsigned)b2, 256, 0, st>>>(last, n_rows, iter);   // once every value is done
+    GS_CUDA_TRY(cudaGetLastError());
+    return GS_OK;
 }
 
 }  // namespace gs
@@ -949,7 +1130,7 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
         int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
         const int64_t cap = (int64_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
-        sgns_coef_kernel<DIM><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+        sgns_coef_kernel<DIM, 0><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
             a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
             (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
             a.dump_pairs, a.dump_negs);
@@ -965,15 +1146,17 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
         if (blocks > cap) blocks = cap;
         sgns_apply_out_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
             a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
-            lead_part, tail_part);
+            lead_part, tail_part, MomState{ nullptr, nullptr, 0.f, 0 });
         GS_CUDA_TRY(cudaGetLastError());
         if (n_cut > 1) {
             sgns_apply_out_fixup_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part);
+                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part,
+                MomState{ nullptr, nullptr, 0.f, 0 });
             GS_CUDA_TRY(cudaGetLastError());
         }
         sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
-            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr);
+            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr,
+            MomState{ nullptr, nullptr, 0.f, 0 });
         GS_CUDA_TRY(cudaGetLastError());
     }
     if (a.loss || a.pairs) {

@@ -45,7 +45,7 @@ def parse_args():
     ap.add_argument("--workload", default="deepwalk_large")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the node count (testing)")
     ap.add_argument("--batch-walks", type=int, default=1 << 20)
-    ap.add_argument("--mode", default="hogwild", choices=["hogwild", "hogwild_red", "deterministic"])
+    ap.add_argument("--mode", default="hogwild", choices=["hogwild", "hogwild_red", "deterministic", "momentum"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample-walks", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -289,6 +289,70 @@ def run_walks_only(args, wl, g, G, info, dev):
     }))
 
 
+# ---------------------------------------------------------------------------- momentum step
+def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
+    """Times walks + gs_sgns_step_momentum on batches of 512 walks (synchronous, momentum 0.9 as
+    in the paper's production run).  1 GPU."""
+    import torch
+    from paper_2407_15452_b200 import binding as B
+    n = g.n_nodes
+    bw = min(args.batch_walks, 512)
+    total_walks = n * wl.walks_per_node
+    nb_total = (total_walks + bw - 1) // bw
+    m_in, m_out = torch.zeros_like(w_in), torch.zeros_like(w_out)
+    last_in = torch.zeros(n, dtype=torch.int32, device=dev)
+    last_out = torch.zeros_like(last_in)
+    walks = torch.empty((bw, wl.walk_len), dtype=torch.int32, device=dev)
+    loss = torch.zeros(1, dtype=torch.float64, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+    mu = 0.9
+    seed, lr = wl.graph_seed, wl.lr0 * (1.0 - mu)      # same effective step lr / (1 - mu) as the plain runs
+
+    def step(it):
+        base = (it % nb_total) * bw
+        k = min(bw, total_walks - base)
+        if wl.walk_kind == "uniform":
+            B.gs_random_walks(G, None, k, base, wl.walk_len, seed, out=walks)
+        else:
+            B.gs_node2vec_walks(G, None, k, base, wl.walk_len, seed, wl.p, wl.q, out=walks)
+        B.gs_sgns_step_momentum(w_in, w_out, m_in, m_out, last_in, last_out, walks[:k], base,
+                                wl.window, wl.n_neg, alias, lr, mu, it, seed, loss, cnt)
+
+    for it in range(args.warmup):
+        step(it)
+    torch.cuda.synchronize()
+    loss.zero_()
+    cnt.zero_()
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for it in range(args.warmup, args.warmup + args.steps):
+        step(it)
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    pairs = int(cnt.item())
+    peak, peak_kind = measured_peak_gbs()
+    # per pair and target: the embedding row and its momentum row, each read and written once
+    model = pairs * (1 + wl.n_neg) * 4 * wl.dim * 4
+    gbs = model / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "gpu_launches": None, "clocks": clocks, "mean_loss": loss.item() / max(pairs, 1),
+        "config": {"workload": wl.name, "mode": "momentum", "momentum": mu, "lr": lr, "batch_walks": bw,
+                   "walk_len": wl.walk_len, "window": wl.window, "n_neg": wl.n_neg, "dim": wl.dim,
+                   "scale": args.scale, **info},
+        "roofline": {"bound": "hbm", "kernel": "momentum step (keys, sort, catch-up, coefficients, apply)",
+                     "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "bytes_model": "per pair and target: row and momentum row, read + written"},
+    }))
+
+
 # ---------------------------------------------------------------------------- our arm
 def run_ours(args, wl):
     import torch
@@ -319,6 +383,8 @@ def run_ours(args, wl):
     w_out = torch.empty_like(w_in)
     seed = wl.graph_seed
     B.gs_init_embeddings(w_in, w_out, seed)
+    if args.mode == "momentum":
+        return run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev)
     mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,
             "deterministic": B.GS_DETERMINISTIC}[args.mode]
     kind = B.GS_WALK_UNIFORM if wl.walk_kind == "uniform" else B.GS_WALK_NODE2VEC

@@ -179,7 +179,8 @@ def oracle_sample(wl, off, col, table, n_walks, base, seed):
     else:
         walks, steps, _ = O.node2vec_walks(off, col, None, n_walks, base, wl.walk_len, seed, wl.p, wl.q)
     t1 = time.perf_counter()
-    c, o, ng, pairs = O.expand_lists(walks, base, wl.window, wl.n_neg, thr, alias, seed)
+    c, o, ng, pairs = O.expand_lists(walks, base, wl.window, wl.n_neg, thr, alias, seed,
+                                     forward_only=wl.forward_only)
     t2 = time.perf_counter()
     # input data handling (not timed): renumber touched rows, materialise their start values
     allv = np.concatenate([c, o, ng.ravel()])
@@ -387,10 +388,12 @@ def run_ours(args, wl):
         return run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev)
     mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,
             "deterministic": B.GS_DETERMINISTIC}[args.mode]
+    if wl.forward_only:
+        mode |= B.GS_PAIRS_FORWARD_ONLY
     kind = B.GS_WALK_UNIFORM if wl.walk_kind == "uniform" else B.GS_WALK_NODE2VEC
     total_walks = n * wl.walks_per_node
     bw = min(args.batch_walks, total_walks)
-    if mode == B.GS_DETERMINISTIC:
+    if (mode & 0xFF) == B.GS_DETERMINISTIC:
         bw = min(bw, 512)
     nb_total = (total_walks + bw - 1) // bw
     ekw = dict(walks_per_node=wl.walks_per_node, walk_len=wl.walk_len, window=wl.window,
@@ -484,7 +487,7 @@ def run_ours(args, wl):
         wbytes = walk_bytes(steps, wl.offsets64, indexed) / launches
         gbytes = walk_granule_bytes(steps, indexed) / launches
         walk_ms = ms_walk / launches
-        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if mode else None
+        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if (mode & 0xFF) else None
         traffic = per_pair * pairs / launches if per_pair else None
         out = {
             "metric": METRIC, "value": pairs_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -503,7 +506,7 @@ def run_ours(args, wl):
             "e2e": {"value": e2e_pairs_all / e2e_s, "unit": UNIT,
                     "h2d_bytes_per_step": 4 * bw, "d2h_bytes_per_step": 16},
             "roofline": {"bound": "hbm",
-                         "kernel": "sgns_hogwild_kernel" if mode else "sgns (coef+sort+apply)",
+                         "kernel": "sgns_hogwild_kernel" if (mode & 0xFF) else "sgns (coef+sort+apply)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}", "traffic": traffic,
                          "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (ms_sgns * 1e-3)},

@@ -158,6 +158,11 @@ GS_API gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts,
 #define GS_HOGWILD        1   /* lock-free: plain loads and stores, rows may race   */
 #define GS_HOGWILD_RED    2   /* lock-free: increments sent as reductions (no lost  */
                               /* updates, gradients may still be stale)             */
+#define GS_PAIRS_FORWARD_ONLY 0x100  /* OR into `mode`: keep only pairs whose context comes  */
+                                     /* LATER in the walk.  Walks of two nodes with window 1 */
+                                     /* then give one (source, neighbour) pair per source    */
+                                     /* with n_neg negatives: the batch shape of LINE        */
+                                     /* (Section 3.2: B x (2 + num_neg) nodes).              */
 
 /*
  * One SGNS update over a batch of walks.

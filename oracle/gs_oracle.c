@@ -200,6 +200,7 @@ int64_t gso_node2vec_walks(int64_t n_nodes, const int64_t *off, const int32_t *c
  * b < thr[jj] else alias[jj].  Negatives 2m and 2m+1 use words (0,1) and
  * (2,3) of the Philox block with step = i*2w + sigma, sub = m.
  *
+ * forward_only != 0 keeps only the pairs with j > i.
  * Output lists are laid out by slot: entry e = (walk*L + i)*2w + sigma;
  * centers[e] = contexts[e] = -1 and negs[e*K..] = -1 where no pair exists.
  * Returns the number of pairs.
@@ -207,7 +208,7 @@ int64_t gso_node2vec_walks(int64_t n_nodes, const int64_t *off, const int32_t *c
 int64_t gso_expand_lists(const int32_t *walks, int64_t n_walks, int64_t walk_id_base,
                          int32_t L, int32_t w, int32_t K,
                          const uint32_t *thr, const int32_t *alias, int64_t n_alias,
-                         uint64_t seed,
+                         uint64_t seed, int32_t forward_only,
                          int32_t *centers, int32_t *contexts, int32_t *negs)
 {
     int64_t n_pairs = 0;
@@ -221,6 +222,10 @@ int64_t gso_expand_lists(const int32_t *walks, int64_t n_walks, int64_t walk_id_
                 /* invert sigma = j - i + w - (j > i) */
                 int32_t j = (sg < w) ? (i - w + sg) : (i - w + sg + 1);
                 int ok = (W[i] >= 0) && (j >= 0) && (j < L) && (W[j] >= 0);
+                /* forward_only: only contexts that come later in the walk.  With walks of two
+                 * nodes and w = 1 this is the edge sampling of LINE (Section 3.2: a source, one
+                 * positive and num_neg negatives per source node). */
+                if (forward_only && j < i) ok = 0;
                 centers[e] = ok ? W[i] : -1;
                 contexts[e] = ok ? W[j] : -1;
                 for (int32_t k = 0; k < K; ++k) negs[e * K + k] = -1;

@@ -107,7 +107,7 @@ def node2vec_walks(off, col, starts, n_walks, walk_id_base, L, seed, p, q, max_r
     return walks, int(steps), int(caps.value)
 
 
-def expand_lists(walks, walk_id_base, w, K, thr, alias, seed):
+def expand_lists(walks, walk_id_base, w, K, thr, alias, seed, forward_only=False):
     """Window pairs and negative draws, slot layout [(walk, i, sigma)].
 
     Returns (centers[n_slots], contexts[n_slots], negs[n_slots, K], n_pairs).
@@ -124,7 +124,7 @@ def expand_lists(walks, walk_id_base, w, K, thr, alias, seed):
         _p(walks, ctypes.c_int32), ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base),
         ctypes.c_int32(L), ctypes.c_int32(w), ctypes.c_int32(K),
         _p(thr, ctypes.c_uint32), _p(alias, ctypes.c_int32), ctypes.c_int64(len(thr)),
-        ctypes.c_uint64(seed),
+        ctypes.c_uint64(seed), ctypes.c_int32(1 if forward_only else 0),
         _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32))
     return centers, contexts, negs, int(n_pairs)
 

@@ -20,6 +20,7 @@ _lib = None
 
 GS_VALIDATE, GS_REQUIRE_SORTED, GS_BUILD_WALK_INDEX = 1, 2, 4
 GS_DETERMINISTIC, GS_HOGWILD, GS_HOGWILD_RED = 0, 1, 2
+GS_PAIRS_FORWARD_ONLY = 0x100
 GS_WALK_UNIFORM, GS_WALK_NODE2VEC = 0, 1
 GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
 

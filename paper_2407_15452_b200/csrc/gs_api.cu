@@ -350,7 +350,9 @@ static gs_status check_sgns_shape(int32_t dim, int32_t L, int32_t w, int32_t K, 
     if (w < 1 || w > 32) { set_error("window %d outside [1, 32]", w); return GS_ERR_UNSUPPORTED; }
     if (K < 0 || K > 32) { set_error("n_neg %d outside [0, 32]", K); return GS_ERR_UNSUPPORTED; }
     if (2 * w * (1 + K) > 512) { set_error("2*window*(1+n_neg) = %d exceeds 512", 2 * w * (1 + K)); return GS_ERR_UNSUPPORTED; }
-    if (mode != GS_DETERMINISTIC && mode != GS_HOGWILD && mode != GS_HOGWILD_RED) return invalid("unknown mode");
+    const int32_t base_mode = mode & ~GS_PAIRS_FORWARD_ONLY;
+    if (base_mode != GS_DETERMINISTIC && base_mode != GS_HOGWILD && base_mode != GS_HOGWILD_RED)
+        return invalid("unknown mode");
     return GS_OK;
 }
 

@@ -215,11 +215,12 @@ __device__ __forceinline__ void sum_over_groups(Row<RowGeom<DIM>::FPL> &x)
 // -1 where the pair does not exist or the negative equals the context (masked).
 // W points at the walk (global or shared), c = W[i] >= 0.  Returns the number of pairs
 // (identical on every lane).  dump_* (nullable) are this position's rows of the dump arrays.
+// fwd != 0 keeps only contexts that come later in the walk (edge sampling of LINE).
 __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_t i, int32_t w,
                                              int32_t K, uint64_t seed, uint64_t id,
                                              const uint64_t *__restrict__ alias, uint32_t n_alias,
                                              int32_t c, int32_t *tgt, int lane,
-                                             int32_t *dump_pairs, int32_t *dump_negs)
+                                             int32_t *dump_pairs, int32_t *dump_negs, int fwd)
 {
     const int S = 2 * w, T1 = 1 + K;
     const int hp = K > 0 ? (K + 1) / 2 : 1;          // Philox blocks per slot (>= 1 work item)
@@ -231,7 +232,7 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
         if (it < S * hp) {
             const int s = it / hp, m = it - s * hp;
             const int j = i - w + s + (s >= w ? 1 : 0);
-            const int32_t ctx = (j >= 0 && j < L) ? W[j] : -1;
+            const int32_t ctx = (j >= 0 && j < L && !(fwd && s < w)) ? W[j] : -1;   // fwd: only j > i
             valid = ctx >= 0;
             if (m == 0) {
                 tgt[s * T1] = ctx;
@@ -284,7 +285,7 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
                     int32_t L, int32_t w, int32_t K, const uint64_t *__restrict__ alias,
                     uint32_t n_alias, float lr, uint64_t seed, double *loss_out,
                     unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs,
-                    unsigned long long *ticket)
+                    unsigned long long *ticket, int fwd)
 {
     constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR, NG = RowGeom<DIM>::NG;
     constexpr int CH = TCH * NG;                         // targets per chunk
@@ -314,7 +315,7 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
             int32_t *dn = dump_negs ? dump_negs + ((a * L + i) * S) * (int64_t)K : nullptr;
             if (c < 0) { dump_empty_position(S, K, lane, dp, dn); continue; }
             const int pairs = build_targets(W, L, i, w, K, seed, id, alias, n_alias, c, tgt, lane,
-                                            dp, dn);
+                                            dp, dn, fwd);
             if (pairs == 0) continue;
             pair_acc += (unsigned long long)pairs;
             const Row<FPL> u = grow_load<DIM>(w_in, c, sub);     // every group holds the center row
@@ -407,7 +408,7 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
                  int32_t w, int32_t K, const uint64_t *__restrict__ alias, uint32_t n_alias,
                  uint32_t n_nodes, uint64_t seed, uint32_t *__restrict__ keys,
                  float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos,
-                 int32_t *__restrict__ pairs_pos, int32_t *dump_pairs, int32_t *dump_negs)
+                 int32_t *__restrict__ pairs_pos, int32_t *dump_pairs, int32_t *dump_negs, int fwd)
 {
     constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR, NG = RowGeom<DIM>::NG;
     constexpr int CH = TCH * NG;
@@ -437,7 +438,7 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
         __syncwarp();
         if (c >= 0)
             pairs = build_targets(W, L, i, w, K, seed, (uint64_t)(walk_id_base + a), alias, n_alias,
-                                  c, tgt, lane, dp, dn);
+                                  c, tgt, lane, dp, dn, fwd);
         else
             dump_empty_position(S, K, lane, dp, dn);
         if (pairs == 0) {
@@ -848,6 +849,7 @@ struct SgnsArgs {
     double *loss;
     int64_t *pairs;
     int32_t *dump_pairs, *dump_negs;
+    int fwd;                      // forward-only pairs
 };
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
@@ -874,7 +876,7 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
     kern<<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
         a.w_in, a.w_out, a.walks, a.n_walks, a.walk_id_base, a.L, a.w, a.K, a.alias,
         (uint32_t)a.n_nodes, a.lr, a.seed, a.loss, (unsigned long long *)a.pairs, a.dump_pairs,
-        a.dump_negs, ticket);
+        a.dump_negs, ticket, a.fwd);
     GS_CUDA_TRY(cudaGetLastError());
     return GS_OK;
 }
@@ -946,7 +948,7 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
 #define GS_COEF(MODE)                                                                              \
     sgns_coef_kernel<DIM, MODE><<<(unsigned)coef_blocks, SGNS_WARPS * 32, coef_smem, st>>>(         \
         a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias, (uint32_t)a.n_nodes, \
-        (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos, a.dump_pairs, a.dump_negs)
+        (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos, a.dump_pairs, a.dump_negs, a.fwd)
     if (mom) GS_COEF(1); else GS_COEF(0);            // with momentum: the keys first, no table reads
     GS_CUDA_TRY(cudaGetLastError());
     uint32_t *ks = nullptr, *vs = nullptr;
@@ -1004,7 +1006,8 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs };
+                   seed, loss, pairs, dump_pairs, dump_negs, (mode & GS_PAIRS_FORWARD_ONLY) ? 1 : 0 };
+    mode &= ~GS_PAIRS_FORWARD_ONLY;
     switch (dim) {
         case 32: return run_mode<32>(a, mode, st);
         case 64: return run_mode<64>(a, mode, st);
@@ -1024,7 +1027,7 @@ gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_ou
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, nullptr, nullptr };
+                   seed, loss, pairs, nullptr, nullptr, 0 };
     MomHost mom = { m_in, m_out, last_in, last_out, mu, iter };
     switch (dim) {
         case 32: return run_deterministic<32>(a, st, &mom);
@@ -1133,7 +1136,7 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
         sgns_coef_kernel<DIM, 0><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
             a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
             (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
-            a.dump_pairs, a.dump_negs);
+            a.dump_pairs, a.dump_negs, a.fwd);
         GS_CUDA_TRY(cudaGetLastError());
     }
     uint32_t *ks = nullptr, *vs = nullptr;
@@ -1193,7 +1196,7 @@ extern "C" gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t 
     gs_status s = static_scratch_address(&scratch);
     if (s != GS_OK) return s;
     SgnsArgs a = { d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len, window,
-                   n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr };
+                   n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr, 0 };
     cudaStream_t st = (cudaStream_t)stream;
     switch (dim) {
         case 32: return run_deterministic_static<32>(a, scratch, st);

@@ -227,6 +227,7 @@ class Workload:
     p: float = 1.0
     q: float = 1.0
     n_edges_target: int = 0
+    forward_only: bool = False   # pairs (i, j) with j > i only: LINE's (source, neighbour) edges
 
     def make_graph(self, device="cpu", scale: float = 1.0) -> CSRGraph:
         """Generate the graph; scale < 1 shrinks the node count (same recipe)."""
@@ -245,6 +246,11 @@ WORKLOADS = {
                                 "uniform", 10, 40, 10, 5, 128, 0.025, "constant"),
     "node2vec_4m": Workload("node2vec_4m", "chung_lu", 4_000_000, 16, 2.3, 2, False,
                             "node2vec", 10, 80, 10, 5, 128, 0.025, "constant", p=0.5, q=2.0),
+    # LINE (Section 3.2 / Section 4: a source, one positive and 5 negatives per source node): each
+    # "walk" is one sampled edge; the paper's lr 1.0 belongs to its mean-reduced loss, the summed
+    # per-pair update here keeps the word2vec-scale 0.025
+    "line_medium": Workload("line_medium", "chung_lu", 1_000_000, 20, 2.1, 1, False,
+                            "uniform", 20, 2, 1, 5, 128, 0.025, "constant", forward_only=True),
     "deepwalk_large": Workload("deepwalk_large", "chung_lu", 50_000_000, 16, 2.1, 3, True,
                                "uniform", 4, 40, 5, 5, 128, 0.025, "constant"),
     "rmat_billion": Workload("rmat_billion", "rmat", 100_000_000, 10, 0.0, 4, True,

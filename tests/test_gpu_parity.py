@@ -242,6 +242,34 @@ def test_deterministic_step_matches_oracle(tiny, dim, L, w, K):
     assert torch.equal(w_in, w_in2) and torch.equal(w_out, w_out2) and loss == loss2
 
 
+@pytest.mark.parametrize("L,w,K,dim", [(2, 1, 5, 128), (9, 3, 2, 64)])
+def test_forward_only_pairs_line_shape(tiny, L, w, K, dim):
+    # LINE: walks of two nodes, window 1, forward pairs only -> one (source, neighbour) pair per walk
+    _, g, off, col, thr, alias = tiny
+    n = g.n_nodes
+    walks, _ = O.uniform_walks(off, col, None, 1500, 0, L, 4)
+    c, o, ng, n_pairs = O.expand_lists(walks, 0, w, K, thr, alias, 4, forward_only=True)
+    if L == 2:
+        assert n_pairs == int((walks[:, 1] >= 0).sum())
+    w_in0, w_out0 = random_tables(n, dim, 7)
+    U, V = w_in0.numpy().astype(np.float64), w_out0.numpy().astype(np.float64)
+    loss_o, cnt_o = O.sgns_det_from_lists(U, V, c, o, ng, 0.025)
+    a_dev = alias_to_device(thr, alias)
+    wd = torch.from_numpy(walks).to(DEV)
+    for mode in (B.GS_DETERMINISTIC, B.GS_HOGWILD):
+        w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+        loss, cnt, pd, nd = run_step(w_in, w_out, wd, 0, w, K, a_dev, 0.025, 4,
+                                     mode | B.GS_PAIRS_FORWARD_ONLY)
+        pd = pd.cpu().numpy().reshape(-1, 2)
+        assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+        assert np.array_equal(nd.cpu().numpy().reshape(-1, K), ng)
+        assert cnt == cnt_o == n_pairs
+        if mode == B.GS_DETERMINISTIC:
+            assert abs(loss - loss_o) <= 2e-6 * abs(loss_o)
+            assert np.abs(w_in.cpu().numpy() - U).max() <= EMB_TOL
+            assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL
+
+
 def test_deterministic_step_hub_rows_with_thousands_of_contributions():
     # a star: every walk alternates hub / leaf, so one output row collects most contributions
     n = 400

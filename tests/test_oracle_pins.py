@@ -241,6 +241,35 @@ def test_pair_expansion_count_identity_and_brute_force(L, w):
     assert (ng.reshape(6, L, 2 * w, 2)[c < 0] == -1).all()
 
 
+def test_forward_only_pairs_are_the_later_half_and_line_edges():
+    rng = np.random.default_rng(3)
+    walks = rng.integers(0, 50, size=(5, 9)).astype(np.int32)
+    walks[4, 5:] = -1
+    thr = np.full(50, 0xFFFFFFFF, dtype=np.uint32)
+    alias = np.arange(50, dtype=np.int32)
+    w = 3
+    c, o, ng, n_all = O.expand_lists(walks, 0, w, 2, thr, alias, 1)
+    cf, of, ngf, n_fwd = O.expand_lists(walks, 0, w, 2, thr, alias, 1, forward_only=True)
+    for a in range(5):
+        want = [(i, j, x, y) for (i, j, x, y) in brute_pairs(walks[a], w) if j > i]
+        got = []
+        for i in range(9):
+            for sg in range(2 * w):
+                e = (a * 9 + i) * 2 * w + sg
+                if cf[e] >= 0:
+                    j = i - w + sg + (1 if sg >= w else 0)
+                    got.append((i, j, int(cf[e]), int(of[e])))
+                    assert np.array_equal(ngf[e], ng[e])      # same draws as in the two-sided list
+        assert got == want
+    assert 2 * n_fwd == n_all                                  # pairs are symmetric: half are forward
+    # LINE: walks of two nodes, window 1 -> exactly one pair (source, neighbour) per source
+    edges = rng.integers(0, 50, size=(40, 2)).astype(np.int32)
+    cl, ol, _, n_line = O.expand_lists(edges, 0, 1, 3, thr, alias, 1, forward_only=True)
+    assert n_line == 40
+    sel = cl >= 0
+    assert np.array_equal(cl[sel], edges[:, 0]) and np.array_equal(ol[sel], edges[:, 1])
+
+
 # ---------------------------------------------------------------- alias table, negatives
 def implied_mass(thr, alias):
     n = len(thr)

@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the node count (testing)")
     ap.add_argument("--batch-walks", type=int, default=1 << 20)
     ap.add_argument("--mode", default="hogwild", choices=["hogwild", "hogwild_red", "deterministic", "momentum"])
+    ap.add_argument("--table-dtype", default="f32", choices=["f32", "f16"],
+                    help="storage type of the embedding tables (arithmetic is fp32 either way)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample-walks", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -134,10 +136,11 @@ def recorded_traffic(kernel, workload):
     return float(m.group(1))
 
 
-def algorithmic_bytes(pairs, positions, dim, n_neg):
+def algorithmic_bytes(pairs, positions, dim, n_neg, elem=4):
     """Row traffic the update must move: per pair 1+K output rows read and written plus K
-    alias entries; per center position one input row read and written plus its walk entry."""
-    return pairs * ((1 + n_neg) * 2 * 4 * dim + 8 * n_neg) + positions * (2 * 4 * dim + 4)
+    alias entries; per center position one input row read and written plus its walk entry.
+    elem = bytes per stored table value."""
+    return pairs * ((1 + n_neg) * 2 * elem * dim + 8 * n_neg) + positions * (2 * elem * dim + 4)
 
 
 def walk_bytes(steps, offsets64, indexed=False):
@@ -380,10 +383,12 @@ def run_ours(args, wl):
     if args.stage == "walks":
         return run_walks_only(args, wl, g, G, info, dev)
     alias = torch.from_numpy(table.view(np.int64)).to(dev)
-    w_in = torch.empty((n, wl.dim), dtype=torch.float32, device=dev)
+    f16 = args.table_dtype == "f16"
+    w_in = torch.empty((n, wl.dim), dtype=torch.float16 if f16 else torch.float32, device=dev)
     w_out = torch.empty_like(w_in)
     seed = wl.graph_seed
-    B.gs_init_embeddings(w_in, w_out, seed)
+    (B.gs_init_embeddings_f16 if f16 else B.gs_init_embeddings)(w_in, w_out, seed)
+    step_fn = B.gs_sgns_step_f16 if f16 else B.gs_sgns_step
     if args.mode == "momentum":
         return run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev)
     mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,
@@ -457,8 +462,8 @@ def run_ours(args, wl):
                 B.gs_random_walks(G, d_starts, cnt, base, wl.walk_len, seed, out=d_walks)
             else:
                 B.gs_node2vec_walks(G, d_starts, cnt, base, wl.walk_len, seed, wl.p, wl.q, out=d_walks)
-            B.gs_sgns_step(w_in, w_out, d_walks[:cnt], base, wl.window, wl.n_neg, alias, wl.lr0,
-                           seed, mode, d_loss, d_cnt)
+            step_fn(w_in, w_out, d_walks[:cnt], base, wl.window, wl.n_neg, alias, wl.lr0,
+                    seed, mode, d_loss, d_cnt)
             h_res.copy_(d_res, non_blocking=True)
             torch.cuda.synchronize()
             return int(h_res[1:2].view(torch.int64).item())
@@ -480,21 +485,22 @@ def run_ours(args, wl):
         peak, peak_kind = measured_peak_gbs()
         launches = args.steps                                     # SGNS launches on this rank
         positions = steps + walks_done                            # walk entries = center positions
-        sgns_bytes = algorithmic_bytes(pairs, positions, wl.dim, wl.n_neg) / launches
+        sgns_bytes = algorithmic_bytes(pairs, positions, wl.dim, wl.n_neg, 2 if f16 else 4) / launches
         sgns_ms = ms_sgns / launches
         achieved = sgns_bytes / (sgns_ms * 1e-3) / 1e9
         indexed = "walk_index_bytes" in info
         wbytes = walk_bytes(steps, wl.offsets64, indexed) / launches
         gbytes = walk_granule_bytes(steps, indexed) / launches
         walk_ms = ms_walk / launches
-        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if (mode & 0xFF) else None
+        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if (mode & 0xFF) and not f16 else None
         traffic = per_pair * pairs / launches if per_pair else None
         out = {
             "metric": METRIC, "value": pairs_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": wl.name, "mode": args.mode, "batch_walks": bw,
+            "config": {"workload": wl.name, "mode": args.mode, "table_dtype": args.table_dtype,
+                       "batch_walks": bw,
                        "walk_kind": wl.walk_kind, "walk_len": wl.walk_len, "window": wl.window,
                        "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale,
                        "l2": "tables (2 x n x dim x 4 B) and CSR far exceed the 126 MB L2; no flush",

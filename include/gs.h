@@ -281,8 +281,31 @@ GS_API gs_status gs_momentum_flush(float *d_w, float *d_m, int32_t *d_last, int6
                                    int32_t dim, float lr, float momentum, int32_t iteration,
                                    void *stream);
 
+/*
+ * Half-precision table storage (the paper's production tables are fp16: 1e9 x
+ * 128 values in 256 GB, Section 4.2).  d_w_in / d_w_out hold IEEE half values,
+ * [n_nodes][dim] row-major, dim in {64, 128, 256}.  Every row is widened to
+ * fp32 when read, all arithmetic is as in gs_sgns_step, and a written row is
+ * rounded to nearest-even half.  Row traffic halves; increments far below half
+ * an ulp of the stored value are lost (no stochastic rounding).
+ * Modes: GS_DETERMINISTIC (bitwise reproducible) and GS_HOGWILD;
+ * GS_HOGWILD_RED returns GS_ERR_UNSUPPORTED.  Other arguments as gs_sgns_step.
+ * gs_init_embeddings_f16 writes the start values of gs_init_embeddings rounded
+ * to half.
+ */
+GS_API gs_status gs_init_embeddings_f16(void *d_w_in, void *d_w_out, int64_t n_nodes,
+                                        int32_t dim, uint64_t seed, void *stream);
+GS_API gs_status gs_sgns_step_f16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
+                                  const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                                  int32_t walk_len, int32_t window, int32_t n_neg,
+                                  const uint64_t *d_alias, float lr, uint64_t seed, int32_t mode,
+                                  double *d_loss_sum, int64_t *d_pair_count,
+                                  int32_t *d_pairs_dump, int32_t *d_negs_dump, void *stream);
+
 #define GS_WALK_UNIFORM   0
 #define GS_WALK_NODE2VEC  1
+#define GS_TABLE_F32      0
+#define GS_TABLE_F16      1   /* tables of IEEE half, see gs_sgns_step_f16      */
 #define GS_LR_CONSTANT    0
 #define GS_LR_LINEAR      1   /* lr_b = lr0 * max(1 - b / total_batches, 1e-4) */
 
@@ -296,7 +319,7 @@ typedef struct gs_sgns_config {
     int32_t lr_schedule;      /* GS_LR_*                                         */
     int32_t mode;             /* GS_DETERMINISTIC | GS_HOGWILD | GS_HOGWILD_RED  */
     int32_t max_rounds;       /* node2vec rejection cap                          */
-    int32_t reserved;
+    int32_t table_dtype;      /* GS_TABLE_F32 (0) or GS_TABLE_F16                */
     double  p, q;             /* node2vec parameters                             */
     double  lr0;
     int64_t batch_walks;      /* walks per mini-batch (512 in the paper's runs)  */
@@ -325,7 +348,7 @@ typedef struct gs_epoch_stats {
  * fills *h_out (host struct).  Epoch defaults of the paper: batch 512.
  */
 GS_API gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias,
-                        float *d_w_in, float *d_w_out, const gs_sgns_config *cfg,
+                        void *d_w_in, void *d_w_out, const gs_sgns_config *cfg,
                         gs_epoch_stats *h_out, void *stream);
 
 /* Frees the cached scratch memory of the current device (waits for the device). */

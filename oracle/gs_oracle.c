@@ -517,3 +517,63 @@ int gso_sgns_seq_from_lists(double *U, double *V, int32_t d,
     if (pair_count) *pair_count = pairs;
     return 0;
 }
+
+/* ------------------------------------------------------------------------
+ * Half-precision table storage (the paper's production tables are fp16,
+ * Section 4.2): values are stored as IEEE binary16, read back exactly, all
+ * arithmetic is done in full precision, and every written value is rounded
+ * to the nearest binary16 (ties to even).
+ * ---------------------------------------------------------------------- */
+static double rn16(double x)
+{
+    return (double)(_Float16)x;
+}
+
+void gso_round_f16(double *x, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) x[i] = rn16(x[i]);
+}
+
+/* Sequential per-pair SGD as gso_sgns_seq_from_lists, on binary16-valued tables:
+ * each updated output row and each updated center row is rounded when written. */
+int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
+                                int64_t n_slots, int32_t S, int32_t K,
+                                const int32_t *centers, const int32_t *contexts,
+                                const int32_t *negs, double lr,
+                                double *loss_sum, int64_t *pair_count)
+{
+    double *acc = (double *)malloc(sizeof(double) * (size_t)d);
+    if (!acc) return -1;
+    double loss = 0.0;
+    int64_t pairs = 0;
+    for (int64_t base = 0; base < n_slots; base += S) {
+        int64_t c = -1;
+        for (int32_t j = 0; j < d; ++j) acc[j] = 0.0;
+        for (int32_t sg = 0; sg < S && base + sg < n_slots; ++sg) {
+            int64_t e = base + sg;
+            if (centers[e] < 0) continue;
+            c = centers[e];
+            const double *u = U + c * d;
+            int64_t o = contexts[e];
+            ++pairs;
+            for (int32_t k = -1; k < K; ++k) {
+                int64_t t = (k < 0) ? o : negs[e * K + k];
+                if (k >= 0 && (t < 0 || t == o)) continue;
+                double *v = V + t * d;
+                double f = dot(u, v, d);
+                double g = (k < 0) ? sigmoid(f) - 1.0 : sigmoid(f);
+                loss += (k < 0) ? softplus(-f) : softplus(f);
+                for (int32_t j = 0; j < d; ++j) {
+                    acc[j] += g * v[j];
+                    v[j] = rn16(v[j] - lr * g * u[j]);
+                }
+            }
+        }
+        if (c >= 0)
+            for (int32_t j = 0; j < d; ++j) U[c * d + j] = rn16(U[c * d + j] - lr * acc[j]);
+    }
+    free(acc);
+    if (loss_sum) *loss_sum = loss;
+    if (pair_count) *pair_count = pairs;
+    return 0;
+}

@@ -235,6 +235,39 @@ def sgns_seq_from_lists(U, V, centers, contexts, negs, S, lr):
     return float(loss.value), int(cnt.value)
 
 
+def round_f16(x):
+    """In place: every value to the nearest IEEE binary16 (ties to even)."""
+    assert x.dtype == np.float64 and x.flags.c_contiguous
+    lib().gso_round_f16(_p(x, ctypes.c_double), ctypes.c_int64(x.size))
+    return x
+
+
+def sgns_det_f16_from_lists(U, V, centers, contexts, negs, lr):
+    """Synchronous step on binary16-valued tables: full-precision step, written rows rounded
+    (rows that are not written hold binary16 values already, so rounding them changes nothing)."""
+    out = sgns_det_from_lists(U, V, centers, contexts, negs, lr)
+    round_f16(U)
+    round_f16(V)
+    return out
+
+
+def sgns_seq_f16_from_lists(U, V, centers, contexts, negs, S, lr):
+    """Sequential per-pair SGD on binary16-valued tables, in place."""
+    d = U.shape[1]
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    K = negs.shape[1]
+    loss = ctypes.c_double(0.0)
+    cnt = ctypes.c_int64(0)
+    rc = lib().gso_sgns_seq_f16_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int32(d),
+        ctypes.c_int64(len(centers)), ctypes.c_int32(S), ctypes.c_int32(K),
+        _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32),
+        ctypes.c_double(lr), ctypes.byref(loss), ctypes.byref(cnt))
+    if rc != 0:
+        raise MemoryError("oracle accumulator")
+    return float(loss.value), int(cnt.value)
+
+
 def lr_at(schedule, lr0, b, num_batches):
     """Learning rate of mini-batch b: 'constant', or 'linear' decay floored at 1e-4 lr0."""
     if schedule == "constant":

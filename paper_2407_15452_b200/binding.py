@@ -23,11 +23,13 @@ GS_DETERMINISTIC, GS_HOGWILD, GS_HOGWILD_RED = 0, 1, 2
 GS_PAIRS_FORWARD_ONLY = 0x100
 GS_WALK_UNIFORM, GS_WALK_NODE2VEC = 0, 1
 GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
+GS_TABLE_F32, GS_TABLE_F16 = 0, 1
 
 EXPORTS = [
     "gs_last_error", "gs_graph_load_csr", "gs_graph_free", "gs_graph_info", "gs_build_alias",
     "gs_init_embeddings", "gs_random_walks", "gs_node2vec_walks", "gs_sgns_step",
     "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static", "gs_sgns_step_momentum", "gs_momentum_flush",
+    "gs_init_embeddings_f16", "gs_sgns_step_f16",
 ]
 
 
@@ -42,7 +44,7 @@ class SgnsConfig(ctypes.Structure):
         ("dim", ctypes.c_int32), ("walks_per_node", ctypes.c_int32), ("walk_len", ctypes.c_int32),
         ("window", ctypes.c_int32), ("n_neg", ctypes.c_int32), ("walk_kind", ctypes.c_int32),
         ("lr_schedule", ctypes.c_int32), ("mode", ctypes.c_int32), ("max_rounds", ctypes.c_int32),
-        ("reserved", ctypes.c_int32), ("p", ctypes.c_double), ("q", ctypes.c_double),
+        ("table_dtype", ctypes.c_int32), ("p", ctypes.c_double), ("q", ctypes.c_double),
         ("lr0", ctypes.c_double), ("batch_walks", ctypes.c_int64), ("first_batch", ctypes.c_int64),
         ("num_batches", ctypes.c_int64), ("seed", ctypes.c_uint64),
     ]
@@ -197,6 +199,33 @@ def gs_sgns_step(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int,
         _stream()))
 
 
+def gs_init_embeddings_f16(w_in, w_out, seed: int):
+    """Start values of gs_init_embeddings rounded to half; tables are torch.float16."""
+    ref = w_in if w_in is not None else w_out
+    n, d = ref.shape
+    _check(lib().gs_init_embeddings_f16(_dev(w_in, torch.float16, "w_in", True),
+                                        _dev(w_out, torch.float16, "w_out", True),
+                                        ctypes.c_int64(n), ctypes.c_int32(d), ctypes.c_uint64(seed),
+                                        _stream()))
+
+
+def gs_sgns_step_f16(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int, alias,
+                     lr: float, seed: int, mode: int, loss_sum=None, pair_count=None,
+                     pairs_dump=None, negs_dump=None):
+    """gs_sgns_step on torch.float16 tables (fp32 arithmetic, round-to-nearest write-back)."""
+    n_nodes, dim = w_in.shape
+    n_walks, walk_len = walks.shape
+    _check(lib().gs_sgns_step_f16(
+        _dev(w_in, torch.float16, "w_in"), _dev(w_out, torch.float16, "w_out"),
+        ctypes.c_int64(n_nodes), ctypes.c_int32(dim), _dev(walks, torch.int32, "walks", n_walks == 0),
+        ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base), ctypes.c_int32(walk_len),
+        ctypes.c_int32(window), ctypes.c_int32(n_neg), _dev(alias, torch.int64, "alias", n_neg == 0),
+        ctypes.c_float(lr), ctypes.c_uint64(seed), ctypes.c_int32(mode),
+        _dev(loss_sum, torch.float64, "loss_sum", True), _dev(pair_count, torch.int64, "pair_count", True),
+        _dev(pairs_dump, torch.int32, "pairs_dump", True), _dev(negs_dump, torch.int32, "negs_dump", True),
+        _stream()))
+
+
 def gs_sgns_step_static(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int, alias,
                         lr: float, seed: int, loss_sum=None, pair_count=None):
     """Deterministic SGNS step that allocates nothing on the device (fixed 32 MiB scratch inside
@@ -255,14 +284,18 @@ def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len,
                   lr0, batch_walks, seed, mode, walk_kind=GS_WALK_UNIFORM,
                   lr_schedule=GS_LR_CONSTANT, p=1.0, q=1.0, max_rounds=1024, first_batch=0,
                   num_batches=0) -> EpochResult:
+    if w_in.dtype not in (torch.float32, torch.float16) or w_out.dtype != w_in.dtype:
+        raise TypeError("tables must both be float32 or both float16")
+    tdt = w_in.dtype
     cfg = SgnsConfig(dim=w_in.shape[1], walks_per_node=walks_per_node, walk_len=walk_len,
                      window=window, n_neg=n_neg, walk_kind=walk_kind, lr_schedule=lr_schedule,
-                     mode=mode, max_rounds=max_rounds, reserved=0, p=p, q=q, lr0=lr0,
+                     mode=mode, max_rounds=max_rounds,
+                     table_dtype=GS_TABLE_F16 if tdt == torch.float16 else GS_TABLE_F32, p=p, q=q, lr0=lr0,
                      batch_walks=batch_walks, first_batch=first_batch, num_batches=num_batches,
                      seed=seed)
     st = EpochStats()
     _check(lib().gs_sgns_epoch(graph._h, _dev(alias, torch.int64, "alias", n_neg == 0),
-                               _dev(w_in, torch.float32, "w_in"), _dev(w_out, torch.float32, "w_out"),
+                               _dev(w_in, tdt, "w_in"), _dev(w_out, tdt, "w_out"),
                                ctypes.byref(cfg), ctypes.byref(st), _stream()))
     return EpochResult(st.loss_sum, st.pairs, st.steps, st.cap_hits, st.batches, st.ms_walk,
                        st.ms_sgns, st.ms_total)

@@ -19,6 +19,8 @@
 // row once.  No floating-point atomics anywhere on this path.
 #include <mutex>
 
+#include <cuda_fp16.h>
+
 #include "gs_common.cuh"
 
 namespace gs {
@@ -68,6 +70,48 @@ __device__ __forceinline__ void row_store(float *__restrict__ tab, int64_t r, in
         for (int q = 0; q < FPL / 4; ++q)
             reinterpret_cast<float4 *>(p)[q * 32 + lane] =
                 make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]);
+    }
+}
+
+// The same whole-warp row access for tables stored as IEEE half (arithmetic stays fp32).  A lane
+// holds the same COLUMNS as in the fp32 layout above (4 consecutive columns per access q, at
+// (q * 32 + lane) * 4), so fp32 scratch rows and half table rows can be combined lane by lane.
+template <int FPL>
+__device__ __forceinline__ Row<FPL> row_load(const __half *__restrict__ tab, int64_t r, int lane)
+{
+    Row<FPL> out;
+    const __half *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 2) {
+        const float2 f = __half22float2(reinterpret_cast<const __half2 *>(p)[lane]);
+        out.v[0] = f.x; out.v[1] = f.y;
+    } else {
+        static_assert(FPL % 4 == 0, "half tables need dim 64, 128 or 256");
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q) {
+            const uint2 t = reinterpret_cast<const uint2 *>(p)[q * 32 + lane];
+            const __half2 *h = reinterpret_cast<const __half2 *>(&t);
+            const float2 a = __half22float2(h[0]), b = __half22float2(h[1]);
+            out.v[4 * q] = a.x; out.v[4 * q + 1] = a.y; out.v[4 * q + 2] = b.x; out.v[4 * q + 3] = b.y;
+        }
+    }
+    return out;
+}
+
+template <int FPL>
+__device__ __forceinline__ void row_store(__half *__restrict__ tab, int64_t r, int lane, const Row<FPL> &x)
+{
+    __half *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 2) {
+        reinterpret_cast<__half2 *>(p)[lane] = __floats2half2_rn(x.v[0], x.v[1]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q) {
+            uint2 t;
+            __half2 *h = reinterpret_cast<__half2 *>(&t);
+            h[0] = __floats2half2_rn(x.v[4 * q], x.v[4 * q + 1]);
+            h[1] = __floats2half2_rn(x.v[4 * q + 2], x.v[4 * q + 3]);
+            reinterpret_cast<uint2 *>(p)[q * 32 + lane] = t;
+        }
     }
 }
 
@@ -147,48 +191,100 @@ __device__ __forceinline__ double warp_sum_double(double s)
 // For dim < 128 a full warp per row would move only 128 or 256 bytes per instruction, and the
 // per-row instruction cost - not bytes - would set the pace.  There a row is held by LPR = 16
 // or 8 lanes (16 bytes per lane) and one warp-wide access moves NG = 2 or 4 different rows.
-template <int DIM> struct RowGeom {
-    static constexpr int FPL = DIM >= 128 ? DIM / 32 : 4;   // floats per lane
-    static constexpr int LPR = DIM / FPL;                   // lanes per row: 32, 32, 16, 8
+// T is the storage type of the table (float, or IEEE half with fp32 arithmetic): a lane always
+// moves 16 bytes per access, i.e. 4 floats or 8 halves.
+template <int DIM, typename T = float> struct RowGeom {
+    static constexpr int PER16 = 16 / (int)sizeof(T);       // values per 16-byte access
+    static constexpr int BYTES = DIM * (int)sizeof(T);
+    static constexpr int LPR = BYTES / 16 >= 32 ? 32 : BYTES / 16;   // lanes per row
+    static constexpr int FPL = DIM / LPR;                   // values per lane
     static constexpr int NG = 32 / LPR;                     // rows per warp-wide access
 };
 
-template <int DIM>
-__device__ __forceinline__ Row<RowGeom<DIM>::FPL> grow_load(const float *__restrict__ tab, int64_t r, int sub)
+__device__ __forceinline__ void unpack16(const uint4 &t, float *v)
 {
-    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR;
-    Row<FPL> out;
-    const float4 *p = reinterpret_cast<const float4 *>(tab + r * (int64_t)DIM);
+    v[0] = __uint_as_float(t.x); v[1] = __uint_as_float(t.y);
+    v[2] = __uint_as_float(t.z); v[3] = __uint_as_float(t.w);
+}
+__device__ __forceinline__ uint4 pack16(const float *v, const float *)
+{
+    return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]),
+                      __float_as_uint(v[3]));
+}
+__device__ __forceinline__ void unpack16h(const uint4 &t, float *v)
+{
+    const __half2 *h = reinterpret_cast<const __half2 *>(&t);
 #pragma unroll
-    for (int q = 0; q < FPL / 4; ++q) {
-        const float4 t = p[q * LPR + sub];
-        out.v[4 * q] = t.x; out.v[4 * q + 1] = t.y; out.v[4 * q + 2] = t.z; out.v[4 * q + 3] = t.w;
+    for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(h[j]); v[2 * j] = f.x; v[2 * j + 1] = f.y; }
+}
+__device__ __forceinline__ uint4 pack16(const float *v, const __half *)
+{
+    uint4 t;
+    __half2 *h = reinterpret_cast<__half2 *>(&t);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) h[j] = __floats2half2_rn(v[2 * j], v[2 * j + 1]);   // round to nearest even
+    return t;
+}
+
+// Lane `sub` of a row group holds, for access q, the PER16 columns starting at
+// (q * LPR + sub) * PER16.
+template <int DIM, typename T>
+__device__ __forceinline__ Row<RowGeom<DIM, T>::FPL> grow_load(const T *__restrict__ tab, int64_t r, int sub)
+{
+    using G = RowGeom<DIM, T>;
+    Row<G::FPL> out;
+    const uint4 *p = reinterpret_cast<const uint4 *>(tab + r * (int64_t)DIM);
+#pragma unroll
+    for (int q = 0; q < G::FPL / G::PER16; ++q) {
+        const uint4 t = p[q * G::LPR + sub];
+        if constexpr (sizeof(T) == 4) unpack16(t, out.v + G::PER16 * q);
+        else unpack16h(t, out.v + G::PER16 * q);
     }
     return out;
 }
 
-template <int DIM>
-__device__ __forceinline__ void grow_store(float *__restrict__ tab, int64_t r, int sub,
-                                           const Row<RowGeom<DIM>::FPL> &x)
+template <int DIM, typename T>
+__device__ __forceinline__ void grow_store(T *__restrict__ tab, int64_t r, int sub,
+                                           const Row<RowGeom<DIM, T>::FPL> &x)
 {
-    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR;
-    float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
+    using G = RowGeom<DIM, T>;
+    uint4 *p = reinterpret_cast<uint4 *>(tab + r * (int64_t)DIM);
 #pragma unroll
-    for (int q = 0; q < FPL / 4; ++q)
-        p[q * LPR + sub] = make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]);
+    for (int q = 0; q < G::FPL / G::PER16; ++q)
+        p[q * G::LPR + sub] = pack16(x.v + G::PER16 * q, (const T *)nullptr);
 }
 
+// Stores a row held in the geometry of a T table into an fp32 scratch row (natural column order).
+template <int DIM, typename T>
+__device__ __forceinline__ void grow_store_f32(float *__restrict__ tab, int64_t r, int sub,
+                                               const Row<RowGeom<DIM, T>::FPL> &x)
+{
+    using G = RowGeom<DIM, T>;
+    float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
+#pragma unroll
+    for (int q = 0; q < G::FPL / G::PER16; ++q) {
+#pragma unroll
+        for (int e = 0; e < G::PER16 / 4; ++e) {
+            const float *v = x.v + G::PER16 * q + 4 * e;
+            p[(q * G::LPR + sub) * (G::PER16 / 4) + e] = make_float4(v[0], v[1], v[2], v[3]);
+        }
+    }
+}
+
+// row += x as reductions (fp32 tables only)
 template <int DIM>
 __device__ __forceinline__ void grow_red_add(float *__restrict__ tab, int64_t r, int sub,
-                                             const Row<RowGeom<DIM>::FPL> &x)
+                                             const Row<RowGeom<DIM, float>::FPL> &x)
 {
-    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR;
+    constexpr int FPL = RowGeom<DIM, float>::FPL, LPR = RowGeom<DIM, float>::LPR;
     float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
 #pragma unroll
     for (int q = 0; q < FPL / 4; ++q)
         atomicAdd(p + q * LPR + sub,
                   make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
 }
+template <int DIM>
+__device__ __forceinline__ void grow_red_add(__half *, int64_t, int, const Row<RowGeom<DIM, __half>::FPL> &) {}
 
 // sum over the LPR lanes that hold one row (identical bits on each of them)
 template <int LPR>
@@ -199,14 +295,14 @@ __device__ __forceinline__ float group_sum(float s)
     return s;
 }
 
-// add up the per-group copies of a row held by the NG groups of a warp
-template <int DIM>
-__device__ __forceinline__ void sum_over_groups(Row<RowGeom<DIM>::FPL> &x)
+// add up the per-group copies of a row held by the NG = 32 / LPR groups of a warp
+template <int LPR, int FPL>
+__device__ __forceinline__ void sum_over_groups(Row<FPL> &x)
 {
 #pragma unroll
-    for (int o = RowGeom<DIM>::LPR; o < 32; o <<= 1) {
+    for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
-        for (int j = 0; j < RowGeom<DIM>::FPL; ++j) x.v[j] += __shfl_xor_sync(0xffffffffu, x.v[j], o);
+        for (int j = 0; j < FPL; ++j) x.v[j] += __shfl_xor_sync(0xffffffffu, x.v[j], o);
     }
 }
 
@@ -278,16 +374,16 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
 }
 
 // ---------------------------------------------------------------- lock-free kernel
-template <int DIM, bool RED, int MINB>
+template <int DIM, typename T, bool RED, int MINB>
 __global__ void __launch_bounds__(SGNS_WARPS * 32, MINB)
-sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
+sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     const int32_t *__restrict__ walks, int64_t n_walks, int64_t walk_id_base,
                     int32_t L, int32_t w, int32_t K, const uint64_t *__restrict__ alias,
                     uint32_t n_alias, float lr, uint64_t seed, double *loss_out,
                     unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs,
                     unsigned long long *ticket, int fwd)
 {
-    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR, NG = RowGeom<DIM>::NG;
+    constexpr int FPL = RowGeom<DIM, T>::FPL, LPR = RowGeom<DIM, T>::LPR, NG = RowGeom<DIM, T>::NG;
     constexpr int CH = TCH * NG;                         // targets per chunk
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
@@ -372,7 +468,7 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
                 while (kk >= T1) kk -= T1;
             }
             // center row: add the accumulated increment to the row as it is now
-            sum_over_groups<DIM>(acc);
+            sum_over_groups<LPR, FPL>(acc);
             Row<FPL> delta;
 #pragma unroll
             for (int j = 0; j < FPL; ++j) delta.v[j] = -lr * acc.v[j];
@@ -401,16 +497,16 @@ sgns_hogwild_kernel(float *__restrict__ w_in, float *__restrict__ w_out,
 // GU[pos] = sum g * v (gradient of the center row), loss_pos, pairs_pos.
 // MODE 0: everything.  MODE 1: keys only (no table is read; used by the momentum step to learn
 // which rows the batch will touch before it reads them).  MODE 2: everything but the keys.
-template <int DIM, int MODE>
+template <int DIM, typename T, int MODE>
 __global__ void __launch_bounds__(SGNS_WARPS * 32)
-sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out,
+sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out,
                  const int32_t *__restrict__ walks, int64_t n_pos, int64_t walk_id_base, int32_t L,
                  int32_t w, int32_t K, const uint64_t *__restrict__ alias, uint32_t n_alias,
                  uint32_t n_nodes, uint64_t seed, uint32_t *__restrict__ keys,
                  float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos,
                  int32_t *__restrict__ pairs_pos, int32_t *dump_pairs, int32_t *dump_negs, int fwd)
 {
-    constexpr int FPL = RowGeom<DIM>::FPL, LPR = RowGeom<DIM>::LPR, NG = RowGeom<DIM>::NG;
+    constexpr int FPL = RowGeom<DIM, T>::FPL, LPR = RowGeom<DIM, T>::LPR, NG = RowGeom<DIM, T>::NG;
     constexpr int CH = TCH * NG;
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
@@ -490,8 +586,8 @@ sgns_coef_kernel(const float *__restrict__ w_in, const float *__restrict__ w_out
             }
         }
         loss = warp_sum(loss);                     // lane-local shares, fixed butterfly order
-        sum_over_groups<DIM>(acc);                 // fixed order as well
-        if (MODE != 1 && grp == 0) grow_store<DIM>(GU, pos, sub, acc);
+        sum_over_groups<LPR, FPL>(acc);                 // fixed order as well
+        if (MODE != 1 && grp == 0) grow_store_f32<DIM, T>(GU, pos, sub, acc);
         if (lane == 0) {
             if (MODE != 2) keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
             if (MODE != 1) { loss_pos[pos] = (double)loss; pairs_pos[pos] = pairs; }
@@ -510,8 +606,8 @@ struct MomState {
     int32_t next_iter;
 };
 
-template <int FPL>
-__device__ __forceinline__ void write_updated_row(float *__restrict__ tab, int64_t r, int lane,
+template <int FPL, typename T>
+__device__ __forceinline__ void write_updated_row(T *__restrict__ tab, int64_t r, int lane,
                                                   Row<FPL> &row, const double (&acc)[FPL], float lr,
                                                   const MomState &ms)
 {
@@ -632,9 +728,9 @@ momentum_stamp_kernel(int32_t *__restrict__ last, int64_t n_rows, int32_t iter)
 // sgns_apply_out_fixup_kernel adds the pieces in block order and writes the row.
 constexpr int RUN_CUT = 256;
 
-template <int FPL>
+template <int FPL, typename T>
 __global__ void __launch_bounds__(256)
-sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
+sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
                       const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
                       const uint32_t *__restrict__ vals, const float *__restrict__ gbuf,
                       uint32_t n_keys, uint32_t n_nodes, int32_t SL, float lr,
@@ -670,7 +766,7 @@ sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
 #pragma unroll
                 for (int j = 0; j < FPL; ++j) dst[j * 32 + lane] = acc[j];
             } else {
-                write_updated_row<FPL>(w_out, cur_key, lane, cur_v, acc, lr, ms);
+                write_updated_row<FPL, T>(w_out, cur_key, lane, cur_v, acc, lr, ms);
             }
         };
 
@@ -729,9 +825,9 @@ sgns_apply_out_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
 // One warp per block of RUN_CUT sorted positions: if a run starts in the block and continues
 // past its end, add its pieces (tail of this block, then the leading pieces of the following
 // blocks while they carry the same key) and write the row.
-template <int FPL>
+template <int FPL, typename T>
 __global__ void __launch_bounds__(256)
-sgns_apply_out_fixup_kernel(float *__restrict__ w_out, const uint32_t *__restrict__ keys,
+sgns_apply_out_fixup_kernel(T *__restrict__ w_out, const uint32_t *__restrict__ keys,
                             uint32_t n_keys, uint32_t n_nodes, float lr,
                             const double *__restrict__ lead_part, const double *__restrict__ tail_part,
                             MomState ms)
@@ -755,14 +851,14 @@ sgns_apply_out_fixup_kernel(float *__restrict__ w_out, const uint32_t *__restric
             for (int j = 0; j < FPL; ++j) acc[j] += l[j * 32 + lane];
         }
         Row<FPL> row = row_load<FPL>(w_out, key, lane);
-        write_updated_row<FPL>(w_out, key, lane, row, acc, lr, ms);
+        write_updated_row<FPL, T>(w_out, key, lane, row, acc, lr, ms);
     }
 }
 
 // Pass 4, keys in [n_nodes, 2 n_nodes): u_row -= lr * sum of the positions' GU rows.
-template <int FPL>
+template <int FPL, typename T>
 __global__ void __launch_bounds__(256)
-sgns_apply_in_kernel(float *__restrict__ w_in, const float *__restrict__ GU,
+sgns_apply_in_kernel(T *__restrict__ w_in, const float *__restrict__ GU,
                      const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals,
                      uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, float lr, MomState ms)
 {
@@ -807,7 +903,7 @@ sgns_apply_in_kernel(float *__restrict__ w_in, const float *__restrict__ GU,
             }
             const int64_t c = (int64_t)(key - n_nodes);
             Row<FPL> row = row_load<FPL>(w_in, c, lane);
-            write_updated_row<FPL>(w_in, c, lane, row, acc, lr, ms);
+            write_updated_row<FPL, T>(w_in, c, lane, row, acc, lr, ms);
         }
     }
 }
@@ -837,7 +933,7 @@ sgns_reduce_kernel(const double *__restrict__ loss_pos, const int32_t *__restric
 
 // ---------------------------------------------------------------- host side
 struct SgnsArgs {
-    float *w_in, *w_out;
+    void *w_in, *w_out;           // tables of float or __half, as the caller of run_* says
     int64_t n_nodes;
     int32_t dim;
     const int32_t *walks;
@@ -854,12 +950,12 @@ struct SgnsArgs {
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
-template <int DIM, bool RED, int MINB>
+template <int DIM, typename T, bool RED, int MINB>
 static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
     const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(a.L + SL);
-    auto kern = sgns_hogwild_kernel<DIM, RED, MINB>;
+    auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -874,7 +970,7 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
     unsigned long long *ticket = (unsigned long long *)((char *)ws + 128);   // bytes 0..127: other counters
     GS_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned long long), st));
     kern<<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
-        a.w_in, a.w_out, a.walks, a.n_walks, a.walk_id_base, a.L, a.w, a.K, a.alias,
+        (T *)a.w_in, (T *)a.w_out, a.walks, a.n_walks, a.walk_id_base, a.L, a.w, a.K, a.alias,
         (uint32_t)a.n_nodes, a.lr, a.seed, a.loss, (unsigned long long *)a.pairs, a.dump_pairs,
         a.dump_negs, ticket, a.fwd);
     GS_CUDA_TRY(cudaGetLastError());
@@ -882,11 +978,11 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 }
 
 // Resident blocks per SM asked of the compiler: 5 blocks of 4 warps (96 registers per thread)
-// measured best for rows of up to 128 floats; wider rows need the registers.
-template <int DIM, bool RED>
+// measured best when a lane holds 4 values of a row; 8 values per lane need the registers.
+template <int DIM, typename T, bool RED>
 static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
-    return run_hogwild_b<DIM, RED, (DIM <= 128 ? 5 : 4)>(a, st);
+    return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL <= 4 ? 5 : 4)>(a, st);
 }
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -899,9 +995,10 @@ struct MomHost {
     int32_t iter;
 };
 
-template <int DIM>
+template <int DIM, typename T>
 static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const MomHost *mom = nullptr)
 {
+    T *w_in = (T *)a.w_in, *w_out = (T *)a.w_out;
     constexpr int FPL = DIM / 32;                        // the apply passes use a whole warp per row
     MomState ms_in = { nullptr, nullptr, 0.f, 0 }, ms_out = { nullptr, nullptr, 0.f, 0 };
     if (mom) {
@@ -946,8 +1043,8 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
     int64_t coef_blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
     if (coef_blocks > (int64_t)sm_count() * 16) coef_blocks = (int64_t)sm_count() * 16;
 #define GS_COEF(MODE)                                                                              \
-    sgns_coef_kernel<DIM, MODE><<<(unsigned)coef_blocks, SGNS_WARPS * 32, coef_smem, st>>>(         \
-        a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias, (uint32_t)a.n_nodes, \
+    sgns_coef_kernel<DIM, T, MODE><<<(unsigned)coef_blocks, SGNS_WARPS * 32, coef_smem, st>>>(         \
+        w_in, w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias, (uint32_t)a.n_nodes, \
         (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos, a.dump_pairs, a.dump_negs, a.fwd)
     if (mom) GS_COEF(1); else GS_COEF(0);            // with momentum: the keys first, no table reads
     GS_CUDA_TRY(cudaGetLastError());
@@ -959,8 +1056,9 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
         // bring every row the batch touches up to iteration `iter`, then compute the coefficients
         int64_t cb = (n_keys + 255) / 256;
         if (cb > (int64_t)sm_count() * 64) cb = (int64_t)sm_count() * 64;
-        momentum_catchup_kernel<FPL><<<(unsigned)cb, 256, 0, st>>>(
-            a.w_in, a.w_out, ms_in, ms_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, mom->iter);
+        if constexpr (sizeof(T) == 4)
+            momentum_catchup_kernel<FPL><<<(unsigned)cb, 256, 0, st>>>(
+                w_in, w_out, ms_in, ms_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, mom->iter);
         GS_CUDA_TRY(cudaGetLastError());
         GS_COEF(2);
         GS_CUDA_TRY(cudaGetLastError());
@@ -970,17 +1068,17 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
         int64_t blocks = (n_keys + 255) / 256;                  // 8 warps x 32 keys per block
         const int64_t cap = (int64_t)sm_count() * 8 * 8;
         if (blocks > cap) blocks = cap;
-        sgns_apply_out_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
+        sgns_apply_out_kernel<FPL, T><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+            w_in, w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
             lead_part, tail_part, ms_out);
         GS_CUDA_TRY(cudaGetLastError());
         if (n_cut > 1) {
-            sgns_apply_out_fixup_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part, ms_out);
+            sgns_apply_out_fixup_kernel<FPL, T><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+                w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part, ms_out);
             GS_CUDA_TRY(cudaGetLastError());
         }
-        sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
-            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr, ms_in);
+        sgns_apply_in_kernel<FPL, T><<<(unsigned)blocks, 256, 0, st>>>(
+            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr, ms_in);
         GS_CUDA_TRY(cudaGetLastError());
     }
     if (a.loss || a.pairs) {
@@ -991,12 +1089,14 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
     return GS_OK;
 }
 
-template <int DIM>
+template <int DIM, typename T>
 static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
 {
-    if (mode == GS_DETERMINISTIC) return run_deterministic<DIM>(a, st);
-    if (mode == GS_HOGWILD) return run_hogwild<DIM, false>(a, st);
-    return run_hogwild<DIM, true>(a, st);
+    if (mode == GS_DETERMINISTIC) return run_deterministic<DIM, T>(a, st);
+    if (mode == GS_HOGWILD) return run_hogwild<DIM, T, false>(a, st);
+    if constexpr (sizeof(T) == 4) return run_hogwild<DIM, T, true>(a, st);
+    set_error("GS_HOGWILD_RED is not available for half-precision tables");
+    return GS_ERR_UNSUPPORTED;
 }
 
 gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
@@ -1009,12 +1109,32 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
                    seed, loss, pairs, dump_pairs, dump_negs, (mode & GS_PAIRS_FORWARD_ONLY) ? 1 : 0 };
     mode &= ~GS_PAIRS_FORWARD_ONLY;
     switch (dim) {
-        case 32: return run_mode<32>(a, mode, st);
-        case 64: return run_mode<64>(a, mode, st);
-        case 128: return run_mode<128>(a, mode, st);
-        case 256: return run_mode<256>(a, mode, st);
+        case 32: return run_mode<32, float>(a, mode, st);
+        case 64: return run_mode<64, float>(a, mode, st);
+        case 128: return run_mode<128, float>(a, mode, st);
+        case 256: return run_mode<256, float>(a, mode, st);
         default:
             set_error("dim %d not supported (32, 64, 128, 256)", dim);
+            return GS_ERR_UNSUPPORTED;
+    }
+}
+
+// Tables stored as IEEE half, arithmetic in fp32, write-back rounded to nearest even.
+gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                        int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                        const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
+                        int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st)
+{
+    if (n_walks == 0) return GS_OK;
+    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                   seed, loss, pairs, dump_pairs, dump_negs, (mode & GS_PAIRS_FORWARD_ONLY) ? 1 : 0 };
+    mode &= ~GS_PAIRS_FORWARD_ONLY;
+    switch (dim) {
+        case 64: return run_mode<64, __half>(a, mode, st);
+        case 128: return run_mode<128, __half>(a, mode, st);
+        case 256: return run_mode<256, __half>(a, mode, st);
+        default:
+            set_error("dim %d not supported with half-precision tables (64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;
     }
 }
@@ -1030,10 +1150,10 @@ gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_ou
                    seed, loss, pairs, nullptr, nullptr, 0 };
     MomHost mom = { m_in, m_out, last_in, last_out, mu, iter };
     switch (dim) {
-        case 32: return run_deterministic<32>(a, st, &mom);
-        case 64: return run_deterministic<64>(a, st, &mom);
-        case 128: return run_deterministic<128>(a, st, &mom);
-        case 256: return run_deterministic<256>(a, st, &mom);
+        case 32: return run_deterministic<32, float>(a, st, &mom);
+        case 64: return run_deterministic<64, float>(a, st, &mom);
+        case 128: return run_deterministic<128, float>(a, st, &mom);
+        case 256: return run_deterministic<256, float>(a, st, &mom);
         default:
             set_error("dim %d not supported (32, 64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;
@@ -1094,6 +1214,7 @@ template <int DIM>
 static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scratch, cudaStream_t st)
 {
     constexpr int FPL = DIM / 32;
+    float *w_in = (float *)a.w_in, *w_out = (float *)a.w_out;
     const int SL = 2 * a.w * (1 + a.K);
     const int64_t n_pos = a.n_walks * a.L;
     const int64_t n_slots = n_pos * SL;
@@ -1133,8 +1254,8 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
         int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
         const int64_t cap = (int64_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
-        sgns_coef_kernel<DIM, 0><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
-            a.w_in, a.w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
+        sgns_coef_kernel<DIM, float, 0><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+            w_in, w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
             (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
             a.dump_pairs, a.dump_negs, a.fwd);
         GS_CUDA_TRY(cudaGetLastError());
@@ -1147,18 +1268,18 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
         int64_t blocks = (n_keys + 255) / 256;                  // 8 warps x 32 keys per block
         const int64_t cap = (int64_t)sm_count() * 8 * 8;
         if (blocks > cap) blocks = cap;
-        sgns_apply_out_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-            a.w_in, a.w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
+        sgns_apply_out_kernel<FPL, float><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+            w_in, w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
             lead_part, tail_part, MomState{ nullptr, nullptr, 0.f, 0 });
         GS_CUDA_TRY(cudaGetLastError());
         if (n_cut > 1) {
-            sgns_apply_out_fixup_kernel<FPL><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-                a.w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part,
+            sgns_apply_out_fixup_kernel<FPL, float><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
+                w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part,
                 MomState{ nullptr, nullptr, 0.f, 0 });
             GS_CUDA_TRY(cudaGetLastError());
         }
-        sgns_apply_in_kernel<FPL><<<(unsigned)blocks, 256, 0, st>>>(
-            a.w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr,
+        sgns_apply_in_kernel<FPL, float><<<(unsigned)blocks, 256, 0, st>>>(
+            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr,
             MomState{ nullptr, nullptr, 0.f, 0 });
         GS_CUDA_TRY(cudaGetLastError());
     }

@@ -1,0 +1,154 @@
+"""GPU parity with tables stored as IEEE half (fp32 arithmetic, round-to-nearest write-back).
+
+The oracle computes in fp64 and rounds a written value once to binary16; the kernels compute
+in fp32 (fp64 accumulators in the synchronous apply pass) and round the fp32 result.  The two
+can differ by one binary16 ulp where the value lies next to a rounding boundary, so the bar is:
+no element differs by more than one ulp of binary16 at its magnitude, and all but a small
+fraction are bit-equal."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gs_oracle as O
+from paper_2407_15452_b200 import binding as B
+from paper_2407_15452_b200 import workloads as WL
+from tests.helpers import alias_to_device, degree_alias, np_graph
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def ulp16(x):
+    """Spacing of binary16 at |x| (normal range; 2^-24 below 2^-14)."""
+    a = np.maximum(np.abs(x), 2.0 ** -14)
+    return 2.0 ** (np.floor(np.log2(a)) - 10)
+
+
+def check_close_f16(got, want, max_mismatch_frac):
+    got = got.astype(np.float64)
+    diff = np.abs(got - want)
+    assert (diff <= ulp16(want) * 1.0001).all(), float((diff / ulp16(want)).max())
+    assert np.mean(diff > 0) <= max_mismatch_frac, float(np.mean(diff > 0))
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    wl = WL.WORKLOADS["tiny_deepwalk"]
+    g = wl.make_graph()
+    off, col = np_graph(g)
+    thr, alias = degree_alias(off)
+    return g, off, col, thr, alias
+
+
+def half_tables(n, dim, seed, scale=0.5):
+    gen = torch.Generator().manual_seed(seed)
+    a = ((torch.rand((n, dim), generator=gen) - 0.5) * scale).to(torch.float16)
+    b = ((torch.rand((n, dim), generator=gen) - 0.5) * scale).to(torch.float16)
+    return a, b
+
+
+@pytest.mark.parametrize("dim", [64, 128, 256])
+def test_initial_tables_are_the_rounded_start_values(dim):
+    n = 3000
+    w_in = torch.empty((n, dim), dtype=torch.float16, device=DEV)
+    w_out = torch.ones((n, dim), dtype=torch.float16, device=DEV)
+    B.gs_init_embeddings_f16(w_in, w_out, 9)
+    want = O.round_f16(O.init_rows(np.arange(n), dim, 9))
+    assert np.array_equal(w_in.cpu().numpy().astype(np.float64), want)
+    assert not w_out.any()
+
+
+@pytest.mark.parametrize("dim,L,w,K", [(128, 20, 5, 5), (64, 10, 3, 10), (256, 8, 2, 3)])
+def test_deterministic_step_on_half_tables(tiny, dim, L, w, K):
+    g, off, col, thr, alias = tiny
+    n = g.n_nodes
+    walks, _ = O.uniform_walks(off, col, None, 400, 10, L, 2)
+    walks[7, L // 2:] = -1
+    c, o, ng, n_pairs = O.expand_lists(walks, 10, w, K, thr, alias, 2)
+    h_in, h_out = half_tables(n, dim, 1)
+    U, V = h_in.numpy().astype(np.float64), h_out.numpy().astype(np.float64)
+    U0, V0 = U.copy(), V.copy()
+    lr = 0.05
+    loss_o, cnt_o = O.sgns_det_f16_from_lists(U, V, c, o, ng, lr)
+    a_dev = alias_to_device(thr, alias)
+    wd = torch.from_numpy(walks).to(DEV)
+    w_in, w_out = h_in.to(DEV), h_out.to(DEV)
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    pd = torch.empty((400, L, 2 * w, 2), dtype=torch.int32, device=DEV)
+    nd = torch.empty((400, L, 2 * w, K), dtype=torch.int32, device=DEV)
+    B.gs_sgns_step_f16(w_in, w_out, wd, 10, w, K, a_dev, lr, 2, B.GS_DETERMINISTIC, loss, cnt, pd, nd)
+    torch.cuda.synchronize()
+    pd = pd.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+    assert np.array_equal(nd.cpu().numpy().reshape(-1, K), ng)
+    assert cnt.item() == cnt_o == n_pairs
+    assert abs(loss.item() - loss_o) <= 2e-6 * abs(loss_o)
+    check_close_f16(w_in.cpu().numpy(), U, 0.01)
+    check_close_f16(w_out.cpu().numpy(), V, 0.01)
+    # the step changed many stored values (it is not lost in the rounding)
+    assert np.mean(V != V0) > 0.02 and np.mean(U != U0) > 0.02
+    # bitwise reproducible
+    w_in2, w_out2 = h_in.to(DEV), h_out.to(DEV)
+    B.gs_sgns_step_f16(w_in2, w_out2, wd, 10, w, K, a_dev, lr, 2, B.GS_DETERMINISTIC)
+    torch.cuda.synchronize()
+    assert torch.equal(w_in, w_in2) and torch.equal(w_out, w_out2)
+
+
+@pytest.mark.parametrize("dim", [64, 128, 256])
+def test_lock_free_single_walk_on_half_tables_equals_sequential_oracle(dim):
+    n, L, w, K = 4000, 12, 2, 3
+    rng = np.random.default_rng(4)
+    walk = rng.permutation(n)[:L].astype(np.int32)[None, :]
+    thr, alias = O.build_alias(np.ones(n), 1.0)
+    c, o, ng, _ = O.expand_lists(walk, 0, w, K, thr, alias, 12)
+    h_in, h_out = half_tables(n, dim, 5, scale=0.6)
+    U, V = h_in.numpy().astype(np.float64), h_out.numpy().astype(np.float64)
+    loss_o, cnt_o = O.sgns_seq_f16_from_lists(U, V, c, o, ng, 2 * w, 0.05)
+    w_in, w_out = h_in.to(DEV), h_out.to(DEV)
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    B.gs_sgns_step_f16(w_in, w_out, torch.from_numpy(walk).to(DEV), 0, w, K,
+                       alias_to_device(thr, alias), 0.05, 12, B.GS_HOGWILD, loss, cnt)
+    torch.cuda.synchronize()
+    assert cnt.item() == cnt_o and abs(loss.item() - loss_o) < 1e-4 * abs(loss_o)
+    # rows repeated inside one chunk of targets (rare) may differ; everything else within one ulp
+    gi, go = w_in.cpu().numpy().astype(np.float64), w_out.cpu().numpy().astype(np.float64)
+    bad_in = (np.abs(gi - U) > 4 * ulp16(U)).any(axis=1).sum()
+    bad_out = (np.abs(go - V) > 4 * ulp16(V)).any(axis=1).sum()
+    assert bad_in <= 2 and bad_out <= 4
+    assert np.mean(go != h_out.numpy().astype(np.float64)) > 0.001
+
+
+def test_half_tables_reject_what_they_do_not_support(tiny):
+    g, off, col, thr, alias = tiny
+    a_dev = alias_to_device(thr, alias)
+    walks = torch.zeros((4, 8), dtype=torch.int32, device=DEV)
+    w32 = torch.zeros((g.n_nodes, 32), dtype=torch.float16, device=DEV)
+    with pytest.raises(B.GsError) as e:
+        B.gs_sgns_step_f16(w32, w32.clone(), walks, 0, 2, 2, a_dev, 0.1, 0, B.GS_HOGWILD)
+    assert e.value.status == -6
+    w = torch.zeros((g.n_nodes, 64), dtype=torch.float16, device=DEV)
+    with pytest.raises(B.GsError) as e:
+        B.gs_sgns_step_f16(w, w.clone(), walks, 0, 2, 2, a_dev, 0.1, 0, B.GS_HOGWILD_RED)
+    assert e.value.status == -6
+
+
+def test_epoch_on_half_tables_trains(tiny):
+    g, off, col, thr, alias = tiny
+    G = B.gs_graph_load_csr(g.offsets.to(DEV), g.cols.to(DEV), B.GS_VALIDATE | B.GS_BUILD_WALK_INDEX)
+    a_dev = alias_to_device(thr, alias)
+    losses = {}
+    for dt in (torch.float32, torch.float16):
+        w_in = torch.empty((g.n_nodes, 64), dtype=dt, device=DEV)
+        w_out = torch.empty_like(w_in)
+        (B.gs_init_embeddings if dt == torch.float32 else B.gs_init_embeddings_f16)(w_in, w_out, 0)
+        for ep in range(3):
+            res = B.gs_sgns_epoch(G, a_dev, w_in, w_out, walks_per_node=4, walk_len=12, window=4,
+                                  n_neg=5, lr0=0.025, batch_walks=4096, seed=ep, mode=B.GS_HOGWILD)
+        losses[dt] = res.loss_sum / res.pairs
+    # round-to-nearest write-back drops increments far below half an ulp of the stored value, so
+    # late in training the half tables lag a little (6-7 % here after three passes over a 10^4-node
+    # graph; on the 1M-node workload the two track each other within 1 % over half an epoch)
+    assert losses[torch.float16] < 0.9 * 6 * np.log(2)
+    assert abs(losses[torch.float16] - losses[torch.float32]) <= 0.10 * losses[torch.float32], losses

@@ -499,6 +499,34 @@ def test_momentum_step_with_zero_momentum_is_the_synchronous_step():
     assert np.allclose(Ua, Ub, atol=1e-14) and np.allclose(Va, Vb, atol=1e-14)
 
 
+# ---------------------------------------------------------------- half-precision storage
+def test_binary16_rounding_matches_library_conversion_and_ties_to_even():
+    rng = np.random.default_rng(11)
+    x = np.concatenate([rng.normal(size=5000), rng.normal(size=5000) * 1e-3, [0.0, 65504.0, -65504.0]])
+    # exact ties: midpoints between neighbouring binary16 values
+    h = np.float16(0.3).astype(np.float64)
+    nxt = np.nextafter(np.float16(0.3), np.float16(1.0)).astype(np.float64)
+    x = np.concatenate([x, [(h + nxt) / 2, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11]])
+    got = O.round_f16(x.copy())
+    assert np.array_equal(got, x.astype(np.float16).astype(np.float64))     # numpy: IEEE RN-even
+    assert got[-2] == 1.0 and got[-1] == 1.0 + 2.0 ** -9                      # ties go to even
+
+
+def test_half_precision_sequential_step_reduces_to_full_precision_plus_rounding():
+    # one pair, rows touched once: the f16 result is the rounded full-precision result
+    rng = np.random.default_rng(12)
+    U = O.round_f16(rng.normal(size=(8, 4)))
+    V = O.round_f16(rng.normal(size=(8, 4)))
+    c = np.array([1], dtype=np.int32)
+    o = np.array([2], dtype=np.int32)
+    ng = np.array([[3, 4]], dtype=np.int32)
+    Ua, Va, Ub, Vb = U.copy(), V.copy(), U.copy(), V.copy()
+    O.sgns_seq_from_lists(Ua, Va, c, o, ng, 1, 0.3)
+    O.sgns_seq_f16_from_lists(Ub, Vb, c, o, ng, 1, 0.3)
+    assert np.array_equal(Ub, O.round_f16(Ua)) and np.array_equal(Vb, O.round_f16(Va))
+    assert not np.array_equal(Vb, V)
+
+
 # ---------------------------------------------------------------- initialisation
 def test_initial_rows_are_uniform_and_exact_in_single_precision():
     rows = np.arange(0, 4000, dtype=np.int64) * 12345

@@ -115,24 +115,6 @@ __device__ __forceinline__ void row_store(__half *__restrict__ tab, int64_t r, i
     }
 }
 
-// row += x, sent as reductions (no value returned)
-template <int FPL>
-__device__ __forceinline__ void row_red_add(float *__restrict__ tab, int64_t r, int lane,
-                                            const Row<FPL> &x)
-{
-    float *p = tab + r * (int64_t)(FPL * 32);
-    if constexpr (FPL == 1) {
-        atomicAdd(p + lane, x.v[0]);
-    } else if constexpr (FPL == 2) {
-        atomicAdd(reinterpret_cast<float2 *>(p) + lane, make_float2(x.v[0], x.v[1]));
-    } else {
-#pragma unroll
-        for (int q = 0; q < FPL / 4; ++q)
-            atomicAdd(reinterpret_cast<float4 *>(p) + q * 32 + lane,
-                      make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
-    }
-}
-
 template <int FPL>
 __device__ __forceinline__ float row_dot(const Row<FPL> &a, const Row<FPL> &b)
 {

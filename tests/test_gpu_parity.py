@@ -270,6 +270,45 @@ def test_forward_only_pairs_line_shape(tiny, L, w, K, dim):
             assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL
 
 
+@pytest.mark.parametrize("dim,L,w,K,n_walks", [(128, 1024, 32, 7, 3),     # longest walk, 512 targets per position
+                                                 (64, 40, 7, 32, 9),        # most negatives
+                                                 (32, 5, 32, 0, 70),        # window wider than the walk, no negatives
+                                                 (256, 1, 1, 3, 50)])       # walks of one node: no pairs at all
+def test_limits_of_the_supported_shapes(tiny, dim, L, w, K, n_walks):
+    _, g, off, col, thr, alias = tiny
+    n = g.n_nodes
+    walks, _ = O.uniform_walks(off, col, None, n_walks, 0, L, 6)
+    c, o, ng, n_pairs = O.expand_lists(walks, 0, w, K, thr, alias, 6)
+    w_in0, w_out0 = random_tables(n, dim, 11, scale=0.2)
+    U, V = w_in0.numpy().astype(np.float64), w_out0.numpy().astype(np.float64)
+    loss_o, cnt_o = O.sgns_det_from_lists(U, V, c, o, ng, 0.01)
+    a_dev = alias_to_device(thr, alias)
+    wd = torch.from_numpy(walks).to(DEV)
+    for mode in (B.GS_DETERMINISTIC, B.GS_HOGWILD, B.GS_HOGWILD_RED):
+        w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+        loss, cnt, pd, nd = run_step(w_in, w_out, wd, 0, w, K, a_dev, 0.01, 6, mode)
+        pd = pd.cpu().numpy().reshape(-1, 2)
+        assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+        if K > 0:
+            assert np.array_equal(nd.cpu().numpy().reshape(-1, K), ng)
+        assert cnt == cnt_o == n_pairs
+        if mode == B.GS_DETERMINISTIC:
+            assert abs(loss - loss_o) <= 2e-6 * max(abs(loss_o), 1e-30)
+            assert np.abs(w_in.cpu().numpy() - U).max() <= EMB_TOL
+            assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL
+        else:
+            assert torch.isfinite(w_in).all() and torch.isfinite(w_out).all()
+    if L == 1:
+        assert n_pairs == 0
+    # one past each limit is refused
+    for bad in (dict(window=33), dict(n_neg=33), dict(window=32, n_neg=8)):
+        kw = dict(window=2, n_neg=2)
+        kw.update(bad)
+        with pytest.raises(B.GsError) as e:
+            B.gs_sgns_step(w_in, w_out, wd, 0, kw["window"], kw["n_neg"], a_dev, 0.01, 6, B.GS_HOGWILD)
+        assert e.value.status == -6
+
+
 def test_deterministic_step_hub_rows_with_thousands_of_contributions():
     # a star: every walk alternates hub / leaf, so one output row collects most contributions
     n = 400

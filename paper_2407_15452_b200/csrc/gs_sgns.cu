@@ -30,7 +30,7 @@ int radix_sort_pairs(uint32_t *keysA, uint32_t *valsA, uint32_t *keysB, uint32_t
                      uint32_t **keys_sorted, uint32_t **vals_sorted);
 size_t sort_counts_bytes(uint32_t n);
 
-constexpr int TCH = 6;            // target rows in flight per warp
+constexpr int TCH = 6;            // target rows in flight per row group (3 for half rows, see run_hogwild)
 constexpr int SGNS_WARPS = 4;     // warps per block
 
 // ---------------------------------------------------------------- row vectors
@@ -356,7 +356,7 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
 }
 
 // ---------------------------------------------------------------- lock-free kernel
-template <int DIM, typename T, bool RED, int MINB>
+template <int DIM, typename T, bool RED, int MINB, int TC>
 __global__ void __launch_bounds__(SGNS_WARPS * 32, MINB)
 sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     const int32_t *__restrict__ walks, int64_t n_walks, int64_t walk_id_base,
@@ -366,7 +366,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     unsigned long long *ticket, int fwd)
 {
     constexpr int FPL = RowGeom<DIM, T>::FPL, LPR = RowGeom<DIM, T>::LPR, NG = RowGeom<DIM, T>::NG;
-    constexpr int CH = TCH * NG;                         // targets per chunk
+    constexpr int CH = TC * NG;                          // targets per chunk
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int grp = lane / LPR, sub = lane % LPR;
@@ -404,33 +404,33 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             int kk = 0;                                  // base mod T1, tracked incrementally
             for (int base = 0; base < SL; base += CH) {
                 // target k of group grp is list entry base + k * NG + grp
-                int32_t ids[TCH];
+                int32_t ids[TC];
                 bool any = false;
 #pragma unroll
-                for (int k = 0; k < TCH; ++k) {
+                for (int k = 0; k < TC; ++k) {
                     const int t = base + k * NG + grp;
                     ids[k] = t < SL ? tgt[t] : -1;
                     any |= ids[k] >= 0;
                 }
                 if (__any_sync(0xffffffffu, any)) {
-                    Row<FPL> rows[TCH];
-                    float f[TCH];
+                    Row<FPL> rows[TC];
+                    float f[TC];
 #pragma unroll
-                    for (int k = 0; k < TCH; ++k)
+                    for (int k = 0; k < TC; ++k)
                         if (ids[k] >= 0) rows[k] = grow_load<DIM>(w_out, ids[k], sub);
 #pragma unroll
-                    for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
+                    for (int k = 0; k < TC; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
 #pragma unroll
-                    for (int k = 0; k < TCH; ++k) f[k] = group_sum<LPR>(f[k]);
+                    for (int k = 0; k < TC; ++k) f[k] = group_sum<LPR>(f[k]);
                     // lane `sub` of a group evaluates the group's target `sub`
                     const int my_t = base + sub * NG + grp;
-                    const bool mine = sub < TCH && my_t < SL;
-                    int my_kt = kk + (sub < TCH ? sub * NG + grp : 0);
+                    const bool mine = sub < TC && my_t < SL;
+                    int my_kt = kk + (sub < TC ? sub * NG + grp : 0);
                     while (my_kt >= T1) my_kt -= T1;
                     const int32_t my_id = mine ? tgt[my_t] : -1;
-                    const float my_g = lane_coefficient<TCH>(f, sub, my_id, my_kt == 0, loss);
+                    const float my_g = lane_coefficient<TC>(f, sub, my_id, my_kt == 0, loss);
 #pragma unroll
-                    for (int k = 0; k < TCH; ++k) {
+                    for (int k = 0; k < TC; ++k) {
                         const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + k);
                         if (ids[k] >= 0) {
                             const float step = -lr * g;
@@ -932,12 +932,12 @@ struct SgnsArgs {
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
-template <int DIM, typename T, bool RED, int MINB>
+template <int DIM, typename T, bool RED, int MINB, int TC = TCH>
 static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
     const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(a.L + SL);
-    auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB>;
+    auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB, TC>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -964,7 +964,10 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 template <int DIM, typename T, bool RED>
 static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
-    return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL <= 4 ? 5 : 4)>(a, st);
+    if constexpr (sizeof(T) == 2)            // half rows: 3 rows per group in flight, 6 blocks (measured)
+        return run_hogwild_b<DIM, T, RED, 6, 3>(a, st);
+    else
+        return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL <= 4 ? 5 : 4), TCH>(a, st);
 }
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }

@@ -16,7 +16,10 @@
  *    buffer is allocated and freed by the caller; the library borrows it for
  *    the duration of the call (a graph handle borrows the CSR arrays until
  *    gs_graph_free).  The library allocates only its own scratch memory
- *    (cached per device, released by gs_release_workspace).
+ *    (cached per device, released by gs_release_workspace).  That scratch is
+ *    per DEVICE, not per stream: SGNS calls on one device must be ordered
+ *    after one another (same stream, or events between streams); two that
+ *    overlap on the GPU would share grouping buffers and the walk ticket.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *    Calls enqueue work on it and return without waiting unless stated.
  *  - Every function returns a gs_status; nothing throws, aborts or traps.

@@ -25,7 +25,11 @@
  * edges; degree-proportional stationarity; node2vec closed-form transition
  * weights; pair-count identity; alias-table mass identity; finite-difference
  * gradients; closed form of the first step from zero output vectors;
- * pair-order independence of the synchronous step.
+ * pair-order independence of the synchronous step; for the variants (window
+ * shrinking, sub-sampling, start shuffle, Adam): window range, symmetry and
+ * uniformity, exact keep thresholds at f = 4t and 16t with binomial retention
+ * counts, bijectivity and uniformity of the shuffle, torch's Adam and
+ * SparseAdam.
  * gso_sgns_seq_from_lists (sequential per-pair SGD, the reference point for
  * the racy Hogwild mode) has no exact counterpart on the GPU: parity unpinned.
  */
@@ -59,7 +63,8 @@ void gso_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
 }
 
 /* Stream tags: which consumer of random words a counter belongs to. */
-enum { TAG_UNIFORM_WALK = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4 };
+enum { TAG_UNIFORM_WALK = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4,
+       TAG_WINDOW = 5, TAG_SUBSAMPLE = 6, TAG_SHUFFLE = 7 };
 
 /* Keying shared (as a published convention, not as code) with the GPU path:
  * key = 64-bit seed; counter = (id low, id high, step, tag<<24 | sub). */
@@ -201,6 +206,12 @@ int64_t gso_node2vec_walks(int64_t n_nodes, const int64_t *off, const int32_t *c
  * (2,3) of the Philox block with step = i*2w + sigma, sub = m.
  *
  * forward_only != 0 keeps only the pairs with j > i.
+ * shrink != 0 draws a window per center position, as word2vec does (Mikolov
+ * et al. 2013 describe the effect as giving nearer words more weight): position
+ * i of walk `id` uses w_i = 1 + mulhi(word 0 of the block with step = i,
+ * TAG_WINDOW, sub 0; w), uniform on 1..w, and keeps the pairs with
+ * |i-j| <= w_i.  Slots and the keying of the negatives are those of the full
+ * window, so a kept pair has the same negatives with or without shrinking.
  * Output lists are laid out by slot: entry e = (walk*L + i)*2w + sigma;
  * centers[e] = contexts[e] = -1 and negs[e*K..] = -1 where no pair exists.
  * Returns the number of pairs.
@@ -208,7 +219,7 @@ int64_t gso_node2vec_walks(int64_t n_nodes, const int64_t *off, const int32_t *c
 int64_t gso_expand_lists(const int32_t *walks, int64_t n_walks, int64_t walk_id_base,
                          int32_t L, int32_t w, int32_t K,
                          const uint32_t *thr, const int32_t *alias, int64_t n_alias,
-                         uint64_t seed, int32_t forward_only,
+                         uint64_t seed, int32_t forward_only, int32_t shrink,
                          int32_t *centers, int32_t *contexts, int32_t *negs)
 {
     int64_t n_pairs = 0;
@@ -217,6 +228,12 @@ int64_t gso_expand_lists(const int32_t *walks, int64_t n_walks, int64_t walk_id_
         const int32_t *W = walks + a * (int64_t)L;
         uint64_t id = (uint64_t)(walk_id_base + a);
         for (int32_t i = 0; i < L; ++i) {
+            int32_t w_i = w;
+            if (shrink) {
+                uint32_t r[4];
+                draw4(seed, id, (uint32_t)i, TAG_WINDOW, 0, r);
+                w_i = 1 + (int32_t)scale32(r[0], (uint64_t)w);
+            }
             for (int32_t sg = 0; sg < S; ++sg) {
                 int64_t e = (a * (int64_t)L + i) * S + sg;
                 /* invert sigma = j - i + w - (j > i) */
@@ -226,6 +243,7 @@ int64_t gso_expand_lists(const int32_t *walks, int64_t n_walks, int64_t walk_id_
                  * nodes and w = 1 this is the edge sampling of LINE (Section 3.2: a source, one
                  * positive and num_neg negatives per source node). */
                 if (forward_only && j < i) ok = 0;
+                if (j - i > w_i || i - j > w_i) ok = 0;
                 centers[e] = ok ? W[i] : -1;
                 contexts[e] = ok ? W[j] : -1;
                 for (int32_t k = 0; k < K; ++k) negs[e * K + k] = -1;
@@ -576,4 +594,131 @@ int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
     if (loss_sum) *loss_sum = loss;
     if (pair_count) *pair_count = pairs;
     return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Sub-sampling of frequent nodes (Mikolov et al. 2013, "Distributed
+ * representations of words and phrases", Section 2.3): an occurrence of a
+ * node whose relative frequency f exceeds t is discarded with probability
+ * 1 - sqrt(t / f).  keep(v) = min(1, sqrt(t / f(v))), f(v) = weight(v) / sum.
+ * thr[v] = floor(keep * 2^32), or 0xFFFFFFFF when keep >= 1 ("always").
+ * Returns 0, or -1 when no weight is positive.
+ * ---------------------------------------------------------------------- */
+int gso_keep_thresholds(const double *weights, int64_t n, double t, uint32_t *thr)
+{
+    double total = 0.0;
+    for (int64_t v = 0; v < n; ++v) total += weights[v] > 0.0 ? weights[v] : 0.0;
+    if (!(total > 0.0)) return -1;
+    for (int64_t v = 0; v < n; ++v) {
+        thr[v] = 0xFFFFFFFFu;
+        if (!(weights[v] > 0.0)) continue;
+        double f = weights[v] / total;
+        double keep = sqrt(t / f);
+        if (keep < 1.0) {
+            double x = floor(keep * 4294967296.0);
+            thr[v] = x >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)x;
+        }
+    }
+    return 0;
+}
+
+/* Entry t of walk `id` (node v = W[t] >= 0) is kept iff thr[v] == 0xFFFFFFFF or
+ * word 0 of the block (id, step = t, TAG_SUBSAMPLE, sub 0) is below thr[v].  The
+ * kept entries are moved to the front in their order (the window then spans
+ * the discarded occurrences, as in word2vec) and the rest of the row is -1.
+ * Returns the number of kept entries. */
+int64_t gso_subsample_walks(const int32_t *walks, int64_t n_walks, int64_t walk_id_base,
+                            int32_t L, const uint32_t *thr, uint64_t seed, int32_t *out)
+{
+    int64_t kept = 0;
+    for (int64_t a = 0; a < n_walks; ++a) {
+        const int32_t *W = walks + a * (int64_t)L;
+        int32_t *O = out + a * (int64_t)L;
+        uint64_t id = (uint64_t)(walk_id_base + a);
+        int32_t n = 0;
+        for (int32_t t = 0; t < L; ++t) {
+            int32_t v = W[t];
+            if (v < 0) continue;
+            int keep = 1;
+            if (thr[v] != 0xFFFFFFFFu) {
+                uint32_t r[4];
+                draw4(seed, id, (uint32_t)t, TAG_SUBSAMPLE, 0, r);
+                keep = r[0] < thr[v];
+            }
+            if (keep) O[n++] = v;
+        }
+        kept += n;
+        for (; n < L; ++n) O[n] = -1;
+    }
+    return kept;
+}
+
+/* ------------------------------------------------------------------------
+ * Start-node shuffle: a keyed bijection of [0, n) per (seed, epoch), so that
+ * the walks of an epoch start from the nodes in a different order each time.
+ * Balanced Feistel network of four rounds on 2k bits (4^k >= n, k minimal,
+ * k >= 1) whose round function is word 0 of the Philox block
+ * (id = right half | epoch << 32, step = round, TAG_SHUFFLE, sub 0) masked to
+ * k bits; values that land outside [0, n) are fed through the network again
+ * (cycle walking; a Feistel network is a bijection of its domain, so this
+ * restricts it to a bijection of [0, n)).
+ * ---------------------------------------------------------------------- */
+static uint64_t feistel_once(uint64_t x, int k, uint64_t seed, uint32_t epoch)
+{
+    uint64_t mask = ((uint64_t)1 << k) - 1;
+    uint64_t left = x >> k, right = x & mask;
+    for (uint32_t round = 0; round < 4; ++round) {
+        uint32_t r[4];
+        draw4(seed, right | ((uint64_t)epoch << 32), round, TAG_SHUFFLE, 0, r);
+        uint64_t f = (uint64_t)r[0] & mask;
+        uint64_t nl = right, nr = left ^ f;
+        left = nl; right = nr;
+    }
+    return (left << k) | right;
+}
+
+int64_t gso_shuffle_node(int64_t v, int64_t n, uint64_t seed, uint32_t epoch)
+{
+    int k = 1;
+    while (((uint64_t)1 << (2 * k)) < (uint64_t)n) ++k;
+    uint64_t y = (uint64_t)v;
+    do { y = feistel_once(y, k, seed, epoch); } while (y >= (uint64_t)n);
+    return (int64_t)y;
+}
+
+/* starts[i] = shuffle(node (walk_id_first + i) mod n) */
+void gso_shuffled_starts(int64_t n, uint64_t seed, uint32_t epoch, int64_t walk_id_first,
+                         int64_t count, int32_t *starts)
+{
+    for (int64_t i = 0; i < count; ++i)
+        starts[i] = (int32_t)gso_shuffle_node((walk_id_first + i) % n, n, seed, epoch);
+}
+
+/* ------------------------------------------------------------------------
+ * Adam (Kingma & Ba 2015, Algorithm 1), which the paper names beside SGD with
+ * momentum as an optimizer kept inside the storage (Section 3.2).  Applied to
+ * the rows of the mini-batch only (rows outside it keep their values and
+ * their moments, as a sparse-gradient Adam does); `step` counts iterations
+ * from 1 and is the same for every row:
+ *   m <- b1 m + (1-b1) g ;  v <- b2 v + (1-b2) g^2
+ *   x <- x - lr * (m / (1-b1^step)) / (sqrt(v / (1-b2^step)) + eps)
+ * rows[0..n_rows) are the distinct touched rows of a table of width d; g is
+ * the dense gradient table (only the touched rows are read).
+ * ---------------------------------------------------------------------- */
+void gso_adam_rows(double *x, double *m, double *v, const double *g, int32_t d,
+                   const int64_t *rows, int64_t n_rows, double lr, double b1, double b2,
+                   double eps, int64_t step)
+{
+    double c1 = 1.0 - pow(b1, (double)step);
+    double c2 = 1.0 - pow(b2, (double)step);
+    for (int64_t a = 0; a < n_rows; ++a) {
+        for (int32_t j = 0; j < d; ++j) {
+            int64_t e = rows[a] * d + j;
+            m[e] = b1 * m[e] + (1.0 - b1) * g[e];
+            v[e] = b2 * v[e] + (1.0 - b2) * g[e] * g[e];
+            double mhat = m[e] / c1;
+            double vhat = v[e] / c2;
+            x[e] -= lr * mhat / (sqrt(vhat) + eps);
+        }
+    }
 }

@@ -50,6 +50,8 @@ def lib():
         L.gso_node2vec_walks.restype = ctypes.c_int64
         L.gso_expand_lists.restype = ctypes.c_int64
         L.gso_sgns_loss_from_lists.restype = ctypes.c_double
+        L.gso_subsample_walks.restype = ctypes.c_int64
+        L.gso_shuffle_node.restype = ctypes.c_int64
         _lib = L
     return _lib
 
@@ -107,7 +109,7 @@ def node2vec_walks(off, col, starts, n_walks, walk_id_base, L, seed, p, q, max_r
     return walks, int(steps), int(caps.value)
 
 
-def expand_lists(walks, walk_id_base, w, K, thr, alias, seed, forward_only=False):
+def expand_lists(walks, walk_id_base, w, K, thr, alias, seed, forward_only=False, shrink=False):
     """Window pairs and negative draws, slot layout [(walk, i, sigma)].
 
     Returns (centers[n_slots], contexts[n_slots], negs[n_slots, K], n_pairs).
@@ -125,6 +127,7 @@ def expand_lists(walks, walk_id_base, w, K, thr, alias, seed, forward_only=False
         ctypes.c_int32(L), ctypes.c_int32(w), ctypes.c_int32(K),
         _p(thr, ctypes.c_uint32), _p(alias, ctypes.c_int32), ctypes.c_int64(len(thr)),
         ctypes.c_uint64(seed), ctypes.c_int32(1 if forward_only else 0),
+        ctypes.c_int32(1 if shrink else 0),
         _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32))
     return centers, contexts, negs, int(n_pairs)
 
@@ -268,6 +271,77 @@ def sgns_seq_f16_from_lists(U, V, centers, contexts, negs, S, lr):
     return float(loss.value), int(cnt.value)
 
 
+def keep_thresholds(weights, t):
+    """Sub-sampling thresholds: keep(v) = min(1, sqrt(t / f(v))) as uint32 (0xFFFFFFFF = always)."""
+    wgt = np.ascontiguousarray(weights, dtype=np.float64)
+    thr = np.empty(len(wgt), dtype=np.uint32)
+    rc = lib().gso_keep_thresholds(_p(wgt, ctypes.c_double), ctypes.c_int64(len(wgt)),
+                                   ctypes.c_double(t), _p(thr, ctypes.c_uint32))
+    if rc != 0:
+        raise ValueError("sub-sampling needs at least one positive weight")
+    return thr
+
+
+def subsample_walks(walks, walk_id_base, keep_thr, seed):
+    """Drops walk entries by the keep thresholds and compacts each walk.  Returns (walks, kept)."""
+    walks = _i32(walks)
+    n_walks, L = walks.shape
+    keep_thr = np.ascontiguousarray(keep_thr, dtype=np.uint32)
+    out = np.empty_like(walks)
+    kept = lib().gso_subsample_walks(_p(walks, ctypes.c_int32), ctypes.c_int64(n_walks),
+                                     ctypes.c_int64(walk_id_base), ctypes.c_int32(L),
+                                     _p(keep_thr, ctypes.c_uint32), ctypes.c_uint64(seed),
+                                     _p(out, ctypes.c_int32))
+    return out, int(kept)
+
+
+def shuffle_node(v, n, seed, epoch):
+    return int(lib().gso_shuffle_node(ctypes.c_int64(v), ctypes.c_int64(n), ctypes.c_uint64(seed),
+                                      ctypes.c_uint32(epoch)))
+
+
+def shuffled_starts(n, seed, epoch, walk_id_first, count):
+    """Start nodes of walk ids [first, first + count): the keyed bijection of (id mod n)."""
+    out = np.empty(count, dtype=np.int32)
+    lib().gso_shuffled_starts(ctypes.c_int64(n), ctypes.c_uint64(seed), ctypes.c_uint32(epoch),
+                              ctypes.c_int64(walk_id_first), ctypes.c_int64(count),
+                              _p(out, ctypes.c_int32))
+    return out
+
+
+def adam_rows(x, m, v, g, rows, lr, b1, b2, eps, step):
+    """In place Adam update of the given distinct rows of table x with moments m, v."""
+    for a in (x, m, v, g):
+        assert a.dtype == np.float64 and a.flags.c_contiguous
+    rows = _i64(rows)
+    lib().gso_adam_rows(_p(x, ctypes.c_double), _p(m, ctypes.c_double), _p(v, ctypes.c_double),
+                        _p(g, ctypes.c_double), ctypes.c_int32(x.shape[1]), _p(rows, ctypes.c_int64),
+                        ctypes.c_int64(len(rows)), ctypes.c_double(lr), ctypes.c_double(b1),
+                        ctypes.c_double(b2), ctypes.c_double(eps), ctypes.c_int64(step))
+
+
+def touched_rows(centers, contexts, negs):
+    """Distinct rows a mini-batch reads and writes: (rows of the input table, rows of the output
+    table).  A masked negative (equal to its pair's context) is not a touched row by itself."""
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    ok = centers >= 0
+    rows_in = np.unique(centers[ok])
+    ng = negs[ok]
+    unmasked = ng[(ng >= 0) & (ng != contexts[ok][:, None])]
+    rows_out = np.unique(np.concatenate([contexts[ok], unmasked]))
+    return rows_in.astype(np.int64), rows_out.astype(np.int64)
+
+
+def sgns_adam_step_from_lists(U, V, MU, VU, MV, VV, centers, contexts, negs, lr, b1, b2, eps, step):
+    """Synchronous mini-batch step with Adam on the batch's rows, dense float64 tables, in place.
+    (MU, VU) and (MV, VV) are the first and second moments of U and V."""
+    GU, GV, loss, cnt = sgns_grad_from_lists(U, V, centers, contexts, negs)
+    rows_in, rows_out = touched_rows(centers, contexts, negs)
+    adam_rows(U, MU, VU, GU, rows_in, lr, b1, b2, eps, step)
+    adam_rows(V, MV, VV, GV, rows_out, lr, b1, b2, eps, step)
+    return loss, cnt
+
+
 def lr_at(schedule, lr0, b, num_batches):
     """Learning rate of mini-batch b: 'constant', or 'linear' decay floored at 1e-4 lr0."""
     if schedule == "constant":
@@ -279,10 +353,13 @@ def lr_at(schedule, lr0, b, num_batches):
 
 def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, schedule,
                batch_walks, seed, mode="det", kind="uniform", p=1.0, q=1.0,
-               first_batch=0, num_batches=None):
+               first_batch=0, num_batches=None, shrink=False, keep_thr=None, shuffle_epoch=None):
     """One pass over walk ids rep*N + v in order, batch by batch (dense tables).
 
     Each batch: generate its walks, expand pairs and negatives, apply one step.
+    shuffle_epoch (int or None): walk id a starts at the keyed bijection of a mod N for that
+    epoch instead of at a mod N.  keep_thr (uint32[N] or None): frequent-node sub-sampling of
+    the generated walks before the windows are formed.  shrink: per-position window draw.
     Returns dict(loss_sum, pairs, steps).  Tables are updated in place.
     """
     n_nodes = len(off) - 1
@@ -294,11 +371,14 @@ def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, sche
     for b in range(first_batch, first_batch + num_batches):
         base = b * batch_walks
         n = min(batch_walks, total - base)
+        starts = None if shuffle_epoch is None else shuffled_starts(n_nodes, seed, shuffle_epoch, base, n)
         if kind == "uniform":
-            walks, st = uniform_walks(off, col, None, n, base, L, seed)
+            walks, st = uniform_walks(off, col, starts, n, base, L, seed)
         else:
-            walks, st, _ = node2vec_walks(off, col, None, n, base, L, seed, p, q)
-        c, o, ng, _ = expand_lists(walks, base, w, K, thr, alias, seed)
+            walks, st, _ = node2vec_walks(off, col, starts, n, base, L, seed, p, q)
+        if keep_thr is not None:
+            walks, _ = subsample_walks(walks, base, keep_thr, seed)
+        c, o, ng, _ = expand_lists(walks, base, w, K, thr, alias, seed, shrink=shrink)
         lr = lr_at(schedule, lr0, b, nb_total)
         if mode == "det":
             ls, pc = sgns_det_from_lists(U, V, c, o, ng, lr)

@@ -1,0 +1,245 @@
+"""Pins of the oracle's walk/pair variants and of its Adam update (CPU only).
+
+Window shrinking, sub-sampling of frequent nodes and the start-node shuffle each draw their
+own random words, so each is pinned by what its definition fixes: value ranges and
+distributions, exact special cases, invariants that a slip (off-by-one window, inverted
+comparison, a round function that is not undone) breaks.  Adam is pinned against torch's
+optimizers.
+"""
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+from oracle import gs_oracle as O
+from paper_2407_15452_b200 import workloads as WL
+
+CHI2_P = 1e-4
+
+
+def np_graph(g):
+    return g.offsets.cpu().numpy().astype(np.int64), g.cols.cpu().numpy()
+
+
+def chi2_uniform_ok(counts):
+    counts = np.asarray(counts, dtype=np.float64)
+    exp = counts.sum() / len(counts)
+    stat = ((counts - exp) ** 2 / exp).sum()
+    return stat < stats.chi2.ppf(1 - CHI2_P, len(counts) - 1)
+
+
+def tiny_setup(n=300, L=30, n_walks=600, seed=5):
+    g = WL.chung_lu_graph(n, 8, 2.3, seed=21)
+    off, col = np_graph(g)
+    thr, alias = O.build_alias((off[1:] - off[:-1]).astype(np.float64), 0.75)
+    walks, _ = O.uniform_walks(off, col, None, n_walks, 40, L, seed)
+    return off, col, thr, alias, walks
+
+
+# ---------------------------------------------------------------- window shrinking
+@pytest.mark.parametrize("w", [1, 3, 5, 8])
+def test_shrunk_windows_are_symmetric_uniform_on_1_to_w_and_keep_the_negatives(w):
+    off, col, thr, alias, walks = tiny_setup()
+    n_walks, L = walks.shape
+    K, S = 3, 2 * w
+    c0, o0, n0, p0 = O.expand_lists(walks, 40, w, K, thr, alias, 9)
+    c1, o1, n1, p1 = O.expand_lists(walks, 40, w, K, thr, alias, 9, shrink=True)
+    full = c0.reshape(n_walks, L, S) >= 0
+    kept = c1.reshape(n_walks, L, S) >= 0
+    assert not (kept & ~full).any()                       # nothing new appears
+    # a kept pair is the pair of the full window, negatives included
+    m = c1 >= 0
+    assert np.array_equal(c1[m], c0[m]) and np.array_equal(o1[m], o0[m])
+    assert np.array_equal(n1[m], n0[m]) and (n1[~m] == -1).all()
+    assert p1 == int(m.sum()) and (p1 < p0 or w == 1)
+    # distance of slot sigma from the center: w - sigma for sigma < w, sigma - w + 1 otherwise
+    dist = np.array([w - s if s < w else s - w + 1 for s in range(S)])
+    counts = np.zeros(w + 1, dtype=np.int64)
+    for a in range(n_walks):
+        for i in range(L):
+            if not full[a, i].any():
+                continue
+            present = full[a, i]
+            # the window the position used: every available slot within it is kept, none beyond
+            ks = kept[a, i]
+            if not ks.any():
+                # only possible when the available slots are all farther than the drawn window
+                assert dist[present].min() > 1
+                continue
+            b = dist[ks].max()
+            assert 1 <= b <= w
+            assert np.array_equal(ks, present & (dist <= b))       # symmetric, contiguous
+            # with the full window available the drawn width is exactly b
+            if present.all():
+                counts[b] += 1
+    assert counts[0] == 0
+    if w > 1:
+        assert counts[1:].min() > 50 and chi2_uniform_ok(counts[1:])   # uniform on 1..w
+
+
+def test_shrunk_window_mean_pair_count_is_w_plus_one():
+    # interior positions of full walks: 2 * E[w_i] = w + 1 pairs on average
+    w, L = 6, 40
+    walks = np.tile(np.arange(L, dtype=np.int32), (4000, 1))
+    thr, alias = O.build_alias(np.ones(L), 0.75)
+    c, _, _, _ = O.expand_lists(walks, 0, w, 1, thr, alias, 2, shrink=True)
+    per_pos = (c.reshape(4000, L, 2 * w) >= 0).sum(axis=2)[:, w:L - w]
+    mean = per_pos.mean()
+    sd = np.sqrt(4 * (w * w - 1) / 12.0 / per_pos.size)            # 2 * uniform{1..w}
+    assert abs(mean - (w + 1)) < 5 * sd
+
+
+# ---------------------------------------------------------------- sub-sampling
+def test_keep_thresholds_exact_special_cases():
+    # relative frequencies 1/2, 1/4, 1/8, 1/8 and t = 1/32: sqrt(t/f) = 1/4, sqrt(1/8), 1/2, 1/2
+    wgt = np.array([4.0, 2.0, 1.0, 1.0])
+    thr = O.keep_thresholds(wgt, 1.0 / 32)
+    assert thr[0] == 2 ** 30 and thr[2] == 2 ** 31 and thr[3] == 2 ** 31
+    assert abs(int(thr[1]) - 2 ** 32 / np.sqrt(8.0)) <= 1
+    # f <= t: always kept
+    assert (O.keep_thresholds(wgt, 0.5) == 0xFFFFFFFF).all()
+    # zero weight never occurs in a walk; it is marked "always"
+    assert O.keep_thresholds(np.array([0.0, 1.0]), 0.1)[0] == 0xFFFFFFFF
+    with pytest.raises(ValueError):
+        O.keep_thresholds(np.zeros(3), 0.1)
+
+
+def test_subsampled_walks_are_ordered_subsequences_with_the_stated_retention():
+    off, col, thr_a, alias, walks = tiny_setup(n=200, L=40, n_walks=3000)
+    n = len(off) - 1
+    deg = (off[1:] - off[:-1]).astype(np.float64)
+    t = 1.0 / (4 * n)                                            # most nodes are above t
+    keep_thr = O.keep_thresholds(deg, t)
+    out, kept = O.subsample_walks(walks, 40, keep_thr, 13)
+    assert kept == int((out >= 0).sum())
+    seen = np.zeros(n)
+    stay = np.zeros(n)
+    for W, Z in zip(walks, out):
+        z = Z[Z >= 0]
+        assert (Z[len(z):] == -1).all()                           # -1 only as a suffix
+        # z is a subsequence of W: greedy match
+        k = 0
+        for v in W[W >= 0]:
+            if k < len(z) and z[k] == v:
+                k += 1
+        assert k == len(z)
+        np.add.at(seen, W[W >= 0], 1)
+        np.add.at(stay, z, 1)
+    f = deg / deg.sum()
+    p_keep = np.minimum(1.0, np.sqrt(t / np.maximum(f, 1e-300)))
+    for v in np.argsort(-seen)[:40]:                              # the most visited nodes
+        sd = np.sqrt(seen[v] * p_keep[v] * (1 - p_keep[v])) + 1e-9
+        assert abs(stay[v] - seen[v] * p_keep[v]) < 5 * sd + 1, (v, stay[v], seen[v], p_keep[v])
+    # with every threshold at "always" the walks come back unchanged
+    same, kept_all = O.subsample_walks(walks, 40, np.full(n, 0xFFFFFFFF, dtype=np.uint32), 13)
+    assert np.array_equal(same, walks) and kept_all == int((walks >= 0).sum())
+    # a threshold of zero drops every occurrence of that node
+    z = np.full(n, 0xFFFFFFFF, dtype=np.uint32)
+    hub = int(np.argmax(seen))
+    z[hub] = 0
+    dropped, _ = O.subsample_walks(walks, 40, z, 13)
+    assert not (dropped == hub).any()
+    assert (dropped >= 0).sum() == (walks >= 0).sum() - seen[hub]
+
+
+def test_subsampling_decisions_depend_on_walk_id_and_position_only():
+    off, col, thr_a, alias, walks = tiny_setup(n=200, L=20, n_walks=64)
+    keep_thr = O.keep_thresholds((off[1:] - off[:-1]).astype(np.float64), 1e-3)
+    whole, _ = O.subsample_walks(walks, 40, keep_thr, 13)
+    part, _ = O.subsample_walks(walks[10:30], 50, keep_thr, 13)
+    assert np.array_equal(whole[10:30], part)
+    other, _ = O.subsample_walks(walks, 41, keep_thr, 13)
+    assert not np.array_equal(whole, other)
+
+
+# ---------------------------------------------------------------- start-node shuffle
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 16, 17, 1000, 1024, 1025, 65537])
+def test_shuffle_is_a_bijection_of_the_node_range(n):
+    for epoch in (0, 1, 7):
+        st = O.shuffled_starts(n, 99, epoch, 0, n)
+        assert np.array_equal(np.sort(st), np.arange(n, dtype=np.int32))
+
+
+def test_shuffle_depends_on_seed_and_epoch_and_wraps_over_walk_ids():
+    n = 5000
+    a = O.shuffled_starts(n, 1, 0, 0, n)
+    assert not np.array_equal(a, O.shuffled_starts(n, 1, 1, 0, n))
+    assert not np.array_equal(a, O.shuffled_starts(n, 2, 0, 0, n))
+    assert (a != np.arange(n)).mean() > 0.99                    # about one fixed point expected
+    # walk id a starts at shuffle(a mod n): the second repetition repeats the first
+    b = O.shuffled_starts(n, 1, 0, n - 10, 30)
+    assert np.array_equal(b[:10], a[-10:]) and np.array_equal(b[10:], a[:20])
+    assert O.shuffle_node(17, n, 1, 0) == a[17]
+
+
+def test_shuffle_images_are_uniform_over_epochs():
+    n = 12
+    counts = np.zeros((n, n))
+    for epoch in range(6000):
+        st = O.shuffled_starts(n, 3, epoch, 0, n)
+        counts[np.arange(n), st] += 1
+    for v in range(n):
+        assert chi2_uniform_ok(counts[v])                        # image of node v
+        assert chi2_uniform_ok(counts[:, v])                     # preimage of node v
+
+
+# ---------------------------------------------------------------- Adam
+def test_adam_rows_match_library_adam_dense_and_sparse():
+    rng = np.random.default_rng(0)
+    n, d, lr, b1, b2, eps = 7, 5, 0.01, 0.9, 0.999, 1e-8
+    x0 = rng.normal(size=(n, d))
+    # dense: every row touched in every step = torch.optim.Adam
+    x, m, v = x0.copy(), np.zeros((n, d)), np.zeros((n, d))
+    p = torch.tensor(x0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([p], lr=lr, betas=(b1, b2), eps=eps)
+    for step in range(1, 6):
+        g = rng.normal(size=(n, d))
+        O.adam_rows(x, m, v, g, np.arange(n), lr, b1, b2, eps, step)
+        p.grad = torch.tensor(g)
+        opt.step()
+    assert np.abs(x - p.detach().numpy()).max() < 1e-12
+    # sparse: only some rows per step = torch.optim.SparseAdam (moments of the other rows rest,
+    # one step counter for all rows).  That routine adds eps before the bias correction of the
+    # second moment, Algorithm 1 after it (pinned by the dense case above); with a vanishing
+    # eps the two agree, which isolates the row selection.
+    eps = 1e-300
+    x, m, v = x0.copy(), np.zeros((n, d)), np.zeros((n, d))
+    p = torch.nn.Parameter(torch.tensor(x0, dtype=torch.float64))
+    opt = torch.optim.SparseAdam([p], lr=lr, betas=(b1, b2), eps=eps)
+    for step in range(1, 8):
+        rows = np.sort(rng.choice(n, size=3, replace=False))
+        g = np.zeros((n, d))
+        g[rows] = rng.normal(size=(3, d))
+        O.adam_rows(x, m, v, g, rows, lr, b1, b2, eps, step)
+        p.grad = torch.sparse_coo_tensor(torch.tensor(rows[None, :]), torch.tensor(g[rows]), (n, d))
+        opt.step()
+    assert np.abs(x - p.detach().numpy()).max() < 1e-12
+    # first step of Adam moves every touched value by lr * sign(g) (up to eps)
+    x, m, v = np.zeros((2, 3)), np.zeros((2, 3)), np.zeros((2, 3))
+    g = np.array([[1.0, -2.0, 0.5], [3.0, 3.0, 3.0]])
+    O.adam_rows(x, m, v, g, np.array([0]), lr, b1, b2, 1e-8, 1)
+    assert np.allclose(x[0], -lr * np.sign(g[0]), atol=1e-9) and (x[1] == 0).all()
+
+
+def test_touched_rows_and_adam_step_on_lists():
+    off, col, thr, alias, walks = tiny_setup(n=120, L=12, n_walks=40)
+    n = len(off) - 1
+    c, o, ng, pairs = O.expand_lists(walks, 40, 3, 4, thr, alias, 9)
+    rows_in, rows_out = O.touched_rows(c, o, ng)
+    ok = c >= 0
+    assert set(rows_in) == set(c[ok])
+    want_out = set(o[ok])
+    for e in np.nonzero(ok)[0]:
+        want_out |= {x for x in ng[e] if x >= 0 and x != o[e]}
+    assert set(rows_out) == want_out
+    rng = np.random.default_rng(1)
+    U, V = rng.normal(size=(n, 8)) * 0.1, rng.normal(size=(n, 8)) * 0.1
+    U0, V0 = U.copy(), V.copy()
+    MU, VU, MV, VV = (np.zeros_like(U) for _ in range(4))
+    loss, cnt = O.sgns_adam_step_from_lists(U, V, MU, VU, MV, VV, c, o, ng, 0.01, 0.9, 0.999, 1e-8, 1)
+    assert cnt == pairs and loss > 0
+    untouched_in = np.setdiff1d(np.arange(n), rows_in)
+    assert np.array_equal(U[untouched_in], U0[untouched_in]) and (MU[untouched_in] == 0).all()
+    GU, GV, _, _ = O.sgns_grad_from_lists(U0, V0, c, o, ng)
+    moved = np.abs(GV) > 1e-6                                     # step 1: lr * sign(g)
+    assert np.allclose((V - V0)[moved], -0.01 * np.sign(GV[moved]), atol=1e-6)

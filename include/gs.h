@@ -31,6 +31,9 @@
  *      tag 2 node2vec     : id = walk id, step = t, sub = rejection round
  *      tag 3 negatives    : id = walk id, step = i * 2w + slot, sub = m
  *      tag 4 table init   : id = row, step = column / 4
+ *      tag 5 window draw  : id = walk id, step = position i
+ *      tag 6 sub-sampling : id = walk id, step = position t
+ *      tag 7 start shuffle: id = right half | epoch << 32, step = Feistel round
  *  - A 32-bit word r is mapped to [0, n) as (r * n) >> 32.
  */
 #ifndef GS_H
@@ -166,6 +169,13 @@ GS_API gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts,
                                      /* then give one (source, neighbour) pair per source    */
                                      /* with n_neg negatives: the batch shape of LINE        */
                                      /* (Section 3.2: B x (2 + num_neg) nodes).              */
+#define GS_WINDOW_SHRINK      0x200   /* OR into `mode`: position i of a walk uses the window   */
+                                     /* w_i = 1 + ((word0 * window) >> 32), uniform on        */
+                                     /* 1..window (tag 5), and keeps the pairs with           */
+                                     /* |i-j| <= w_i: word2vec's shrinking window, which      */
+                                     /* weights near contexts more.  Slots and the keying of  */
+                                     /* the negatives stay those of the full window.  (The    */
+                                     /* paper's runs use a fixed window, Section 4.)          */
 
 /*
  * One SGNS update over a batch of walks.
@@ -305,6 +315,65 @@ GS_API gs_status gs_sgns_step_f16(void *d_w_in, void *d_w_out, int64_t n_nodes, 
                                   double *d_loss_sum, int64_t *d_pair_count,
                                   int32_t *d_pairs_dump, int32_t *d_negs_dump, void *stream);
 
+/*
+ * Synchronous mini-batch step with Adam (Kingma & Ba 2015, Algorithm 1), the second optimizer
+ * the paper keeps inside its storage (Section 3.2).  Gradients as in
+ * gs_sgns_step(GS_DETERMINISTIC); only the rows of the batch move (the rows that occur as a
+ * center, a context or an unmasked negative), as a sparse-gradient Adam does: a row outside the
+ * batch keeps its value and its moments.  For every value of a touched row with summed
+ * gradient g:
+ *   m <- beta1 m + (1-beta1) g ;  v <- beta2 v + (1-beta2) g^2
+ *   x <- x - lr * (m / (1-beta1^step)) / (sqrt(v / (1-beta2^step)) + eps)
+ *   d_m_*, d_v_* : first and second moments, shape of the tables, zero before step 1
+ *   step         : 1, 2, 3, ... one per call, the same for every row
+ *   pair_mode    : 0, or GS_PAIRS_FORWARD_ONLY / GS_WINDOW_SHRINK OR-ed together
+ * 0 <= beta1, beta2 < 1, eps > 0.  Bitwise reproducible; scratch as for the deterministic step.
+ */
+GS_API gs_status gs_sgns_step_adam(float *d_w_in, float *d_w_out, float *d_m_in, float *d_v_in,
+                                   float *d_m_out, float *d_v_out, int64_t n_nodes, int32_t dim,
+                                   const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                                   int32_t walk_len, int32_t window, int32_t n_neg,
+                                   const uint64_t *d_alias, float lr, float beta1, float beta2,
+                                   float eps, int64_t step, uint64_t seed, int32_t pair_mode,
+                                   double *d_loss_sum, int64_t *d_pair_count, void *stream);
+
+/* ---------------------------------------------------------------- corpus variants */
+/*
+ * Sub-sampling of frequent nodes, as word2vec thins frequent words (Mikolov et al. 2013,
+ * Section 2.3; the paper's pipeline has no such step): an occurrence of node v is kept with
+ * probability min(1, sqrt(t / f(v))), f(v) = h_weights[v] / sum of weights.
+ * HOST function: h_thr_out[v] = floor(keep * 2^32), or 0xFFFFFFFF for "always" (keep >= 1 or
+ * zero weight).  Errors: GS_ERR_INVALID_ARG (null, n <= 0, t <= 0, negative or non-finite
+ * weight, no positive weight).  The caller uploads the thresholds.
+ */
+GS_API gs_status gs_build_keep_thresholds(const double *h_weights, int64_t n, double t,
+                                          uint32_t *h_thr_out);
+
+/*
+ * Applies the thresholds to walks: entry t of walk id (node v >= 0) stays iff
+ * d_keep_thr[v] == 0xFFFFFFFF or word 0 of the block (tag 6, step t) is below d_keep_thr[v].
+ * Kept entries move to the front of the walk in their order, the rest of the row becomes -1,
+ * so the windows of gs_sgns_step then span the dropped occurrences.  d_walks_out may be
+ * d_walks (in place).  d_kept (nullable): the number of kept entries is ADDED.
+ * Node ids in d_walks must be below the length of d_keep_thr (not checked).
+ */
+GS_API gs_status gs_subsample_walks(const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                                    int32_t walk_len, const uint32_t *d_keep_thr, uint64_t seed,
+                                    int32_t *d_walks_out, uint64_t *d_kept, void *stream);
+
+/*
+ * Start nodes in shuffled order: d_starts_out[i] = P((walk_id_first + i) mod n_nodes), where P
+ * is a bijection of [0, n_nodes) chosen by (seed, epoch), so that consecutive walk ids (and
+ * with them the mini-batches) start from nodes spread over the graph and every epoch uses a
+ * different order.  P is a four-round balanced Feistel network on 2k bits, 4^k >= n_nodes with
+ * k minimal, round function = word 0 of the Philox block (tag 7) masked to k bits; results
+ * outside [0, n_nodes) are passed through the network again.  Pass the result as d_starts to
+ * the walk calls.  (The paper does not say in which order the sources are visited.)
+ */
+GS_API gs_status gs_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epoch,
+                                    int64_t walk_id_first, int64_t count, int32_t *d_starts_out,
+                                    void *stream);
+
 #define GS_WALK_UNIFORM   0
 #define GS_WALK_NODE2VEC  1
 #define GS_TABLE_F32      0
@@ -320,7 +389,9 @@ typedef struct gs_sgns_config {
     int32_t n_neg;
     int32_t walk_kind;        /* GS_WALK_*                                       */
     int32_t lr_schedule;      /* GS_LR_*                                         */
-    int32_t mode;             /* GS_DETERMINISTIC | GS_HOGWILD | GS_HOGWILD_RED  */
+    int32_t mode;             /* GS_DETERMINISTIC | GS_HOGWILD | GS_HOGWILD_RED, */
+                              /* optionally OR-ed with GS_PAIRS_FORWARD_ONLY,    */
+                              /* GS_WINDOW_SHRINK                                */
     int32_t max_rounds;       /* node2vec rejection cap                          */
     int32_t table_dtype;      /* GS_TABLE_F32 (0) or GS_TABLE_F16                */
     double  p, q;             /* node2vec parameters                             */
@@ -329,6 +400,10 @@ typedef struct gs_sgns_config {
     int64_t first_batch;      /* resume point; batches are numbered over the     */
     int64_t num_batches;      /* whole epoch; <= 0 means "to the end"            */
     uint64_t seed;
+    const uint32_t *d_keep_thr; /* device, n_nodes thresholds of gs_build_keep_thresholds: */
+                              /* walks are sub-sampled before the update; NULL = off      */
+    int32_t shuffle_starts;   /* != 0: walk id a starts at the gs_shuffled_starts image  */
+    uint32_t epoch;           /* of a mod n_nodes for this epoch instead of at a mod n   */
 } gs_sgns_config;
 
 typedef struct gs_epoch_stats {

@@ -21,6 +21,7 @@ _lib = None
 GS_VALIDATE, GS_REQUIRE_SORTED, GS_BUILD_WALK_INDEX = 1, 2, 4
 GS_DETERMINISTIC, GS_HOGWILD, GS_HOGWILD_RED = 0, 1, 2
 GS_PAIRS_FORWARD_ONLY = 0x100
+GS_WINDOW_SHRINK = 0x200
 GS_WALK_UNIFORM, GS_WALK_NODE2VEC = 0, 1
 GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
 GS_TABLE_F32, GS_TABLE_F16 = 0, 1
@@ -29,7 +30,8 @@ EXPORTS = [
     "gs_last_error", "gs_graph_load_csr", "gs_graph_free", "gs_graph_info", "gs_build_alias",
     "gs_init_embeddings", "gs_random_walks", "gs_node2vec_walks", "gs_sgns_step",
     "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static", "gs_sgns_step_momentum", "gs_momentum_flush",
-    "gs_init_embeddings_f16", "gs_sgns_step_f16",
+    "gs_init_embeddings_f16", "gs_sgns_step_f16", "gs_sgns_step_adam", "gs_build_keep_thresholds",
+    "gs_subsample_walks", "gs_shuffled_starts",
 ]
 
 
@@ -47,6 +49,7 @@ class SgnsConfig(ctypes.Structure):
         ("table_dtype", ctypes.c_int32), ("p", ctypes.c_double), ("q", ctypes.c_double),
         ("lr0", ctypes.c_double), ("batch_walks", ctypes.c_int64), ("first_batch", ctypes.c_int64),
         ("num_batches", ctypes.c_int64), ("seed", ctypes.c_uint64),
+        ("d_keep_thr", ctypes.c_void_p), ("shuffle_starts", ctypes.c_int32), ("epoch", ctypes.c_uint32),
     ]
 
 
@@ -268,6 +271,60 @@ def gs_momentum_flush(w, m, last, lr: float, momentum: float, iteration: int):
         ctypes.c_int32(iteration), _stream()))
 
 
+def gs_sgns_step_adam(w_in, w_out, m_in, v_in, m_out, v_out, walks, walk_id_base: int, window: int,
+                      n_neg: int, alias, lr: float, beta1: float, beta2: float, eps: float, step: int,
+                      seed: int, pair_mode: int = 0, loss_sum=None, pair_count=None):
+    """Synchronous step with Adam on the rows of the batch (see gs.h); step counts from 1."""
+    n_nodes, dim = w_in.shape
+    n_walks, walk_len = walks.shape
+    _check(lib().gs_sgns_step_adam(
+        _dev(w_in, torch.float32, "w_in"), _dev(w_out, torch.float32, "w_out"),
+        _dev(m_in, torch.float32, "m_in"), _dev(v_in, torch.float32, "v_in"),
+        _dev(m_out, torch.float32, "m_out"), _dev(v_out, torch.float32, "v_out"),
+        ctypes.c_int64(n_nodes), ctypes.c_int32(dim), _dev(walks, torch.int32, "walks", n_walks == 0),
+        ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base), ctypes.c_int32(walk_len),
+        ctypes.c_int32(window), ctypes.c_int32(n_neg), _dev(alias, torch.int64, "alias", n_neg == 0),
+        ctypes.c_float(lr), ctypes.c_float(beta1), ctypes.c_float(beta2), ctypes.c_float(eps),
+        ctypes.c_int64(step), ctypes.c_uint64(seed), ctypes.c_int32(pair_mode),
+        _dev(loss_sum, torch.float64, "loss_sum", True), _dev(pair_count, torch.int64, "pair_count", True),
+        _stream()))
+
+
+def gs_build_keep_thresholds(weights: np.ndarray, t: float) -> np.ndarray:
+    """Host call.  Sub-sampling thresholds (uint32, 0xFFFFFFFF = always kept)."""
+    w = np.ascontiguousarray(weights, dtype=np.float64)
+    out = np.empty(len(w), dtype=np.uint32)
+    _check(lib().gs_build_keep_thresholds(w.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(len(w)),
+                                          ctypes.c_double(t), out.ctypes.data_as(ctypes.c_void_p)))
+    return out
+
+
+def gs_subsample_walks(walks, walk_id_base: int, keep_thr, seed: int, out=None, kept=None):
+    """Drops walk entries by the thresholds (int32 CUDA tensor holding the uint32 bit patterns)
+    and compacts each walk; out may be walks itself."""
+    n_walks, walk_len = walks.shape
+    if out is None:
+        out = torch.empty_like(walks)
+    _check(lib().gs_subsample_walks(
+        _dev(walks, torch.int32, "walks", n_walks == 0), ctypes.c_int64(n_walks),
+        ctypes.c_int64(walk_id_base), ctypes.c_int32(walk_len),
+        _dev(keep_thr, torch.int32, "keep_thr", n_walks == 0), ctypes.c_uint64(seed),
+        _dev(out, torch.int32, "out", n_walks == 0), _dev(kept, torch.int64, "kept", True), _stream()))
+    return out
+
+
+def gs_shuffled_starts(n_nodes: int, seed: int, epoch: int, walk_id_first: int, count: int, device,
+                       out=None):
+    """Start nodes of walk ids [first, first + count) under the keyed bijection of the epoch."""
+    if out is None:
+        out = torch.empty(count, dtype=torch.int32, device=device)
+    _check(lib().gs_shuffled_starts(ctypes.c_int64(n_nodes), ctypes.c_uint64(seed),
+                                    ctypes.c_uint32(epoch), ctypes.c_int64(walk_id_first),
+                                    ctypes.c_int64(count), _dev(out, torch.int32, "out", count == 0),
+                                    _stream()))
+    return out
+
+
 @dataclass
 class EpochResult:
     loss_sum: float
@@ -283,7 +340,7 @@ class EpochResult:
 def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len, window, n_neg,
                   lr0, batch_walks, seed, mode, walk_kind=GS_WALK_UNIFORM,
                   lr_schedule=GS_LR_CONSTANT, p=1.0, q=1.0, max_rounds=1024, first_batch=0,
-                  num_batches=0) -> EpochResult:
+                  num_batches=0, keep_thr=None, shuffle_epoch=None) -> EpochResult:
     if w_in.dtype not in (torch.float32, torch.float16) or w_out.dtype != w_in.dtype:
         raise TypeError("tables must both be float32 or both float16")
     tdt = w_in.dtype
@@ -292,7 +349,9 @@ def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len,
                      mode=mode, max_rounds=max_rounds,
                      table_dtype=GS_TABLE_F16 if tdt == torch.float16 else GS_TABLE_F32, p=p, q=q, lr0=lr0,
                      batch_walks=batch_walks, first_batch=first_batch, num_batches=num_batches,
-                     seed=seed)
+                     seed=seed, d_keep_thr=_dev(keep_thr, torch.int32, "keep_thr", True).value,
+                     shuffle_starts=0 if shuffle_epoch is None else 1,
+                     epoch=0 if shuffle_epoch is None else shuffle_epoch)
     st = EpochStats()
     _check(lib().gs_sgns_epoch(graph._h, _dev(alias, torch.int64, "alias", n_neg == 0),
                                _dev(w_in, tdt, "w_in"), _dev(w_out, tdt, "w_out"),

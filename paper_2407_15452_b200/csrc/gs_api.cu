@@ -46,6 +46,16 @@ gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_ou
                              double *loss, int64_t *pairs, cudaStream_t st);
 gs_status momentum_flush(float *w, float *m, int32_t *last, int64_t n_rows, int32_t dim, float lr,
                          float mu, int32_t iter, cudaStream_t st);
+gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, float *m_out,
+                         float *v_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                         const uint64_t *alias, float lr, float b1, float b2, float eps, int64_t step,
+                         uint64_t seed, int32_t pair_mode, double *loss, int64_t *pairs, cudaStream_t st);
+gs_status launch_subsample_walks(const int32_t *walks, int64_t n_walks, int64_t base, int32_t L,
+                                 const uint32_t *keep_thr, uint64_t seed, int32_t *out,
+                                 unsigned long long *kept, cudaStream_t st);
+gs_status launch_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epoch, int64_t first,
+                                 int64_t count, int32_t *starts, cudaStream_t st);
 
 // ---- errors ----------------------------------------------------------------------
 static thread_local char g_err[512] = "";
@@ -72,8 +82,8 @@ static gs_status invalid(const char *msg)
 
 // ---- per-device state ----------------------------------------------------------------
 struct DeviceState {
-    void *ws[WS_SLOTS] = { nullptr, nullptr, nullptr, nullptr };
-    size_t ws_bytes[WS_SLOTS] = { 0, 0, 0, 0 };
+    void *ws[WS_SLOTS] = {};
+    size_t ws_bytes[WS_SLOTS] = {};
     int sms = 0;
 };
 static std::mutex g_mu;
@@ -356,7 +366,7 @@ static gs_status check_sgns_shape(int32_t dim, int32_t L, int32_t w, int32_t K, 
     if (w < 1 || w > 32) { set_error("window %d outside [1, 32]", w); return GS_ERR_UNSUPPORTED; }
     if (K < 0 || K > 32) { set_error("n_neg %d outside [0, 32]", K); return GS_ERR_UNSUPPORTED; }
     if (2 * w * (1 + K) > 512) { set_error("2*window*(1+n_neg) = %d exceeds 512", 2 * w * (1 + K)); return GS_ERR_UNSUPPORTED; }
-    const int32_t base_mode = mode & ~GS_PAIRS_FORWARD_ONLY;
+    const int32_t base_mode = mode & ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     if (base_mode != GS_DETERMINISTIC && base_mode != GS_HOGWILD && base_mode != GS_HOGWILD_RED)
         return invalid("unknown mode");
     return GS_OK;
@@ -450,6 +460,84 @@ gs_status gs_momentum_flush(float *d_w, float *d_m, int32_t *d_last, int64_t n_r
     return momentum_flush(d_w, d_m, d_last, n_rows, dim, lr, momentum, iteration, (cudaStream_t)stream);
 }
 
+// ------------------------------------------------------------------ Adam
+gs_status gs_sgns_step_adam(float *d_w_in, float *d_w_out, float *d_m_in, float *d_v_in,
+                            float *d_m_out, float *d_v_out, int64_t n_nodes, int32_t dim,
+                            const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                            int32_t walk_len, int32_t window, int32_t n_neg, const uint64_t *d_alias,
+                            float lr, float beta1, float beta2, float eps, int64_t step, uint64_t seed,
+                            int32_t pair_mode, double *d_loss_sum, int64_t *d_pair_count, void *stream)
+{
+    if (!d_w_in || !d_w_out || !d_m_in || !d_v_in || !d_m_out || !d_v_out)
+        return invalid("table or moment pointer is NULL");
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
+    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
+    if (n_walks > 0 && !d_walks) return invalid("d_walks is NULL");
+    if (!(beta1 >= 0.f) || !(beta1 < 1.f) || !(beta2 >= 0.f) || !(beta2 < 1.f))
+        return invalid("beta1 and beta2 must be in [0, 1)");
+    if (!(eps > 0.f)) return invalid("eps must be positive");
+    if (step < 1) return invalid("step counts from 1");
+    if (pair_mode & ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK)) return invalid("unknown pair_mode flag");
+    gs_status s = check_sgns_shape(dim, walk_len, window, n_neg, GS_DETERMINISTIC);
+    if (s != GS_OK) return s;
+    if (n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
+    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out | (uintptr_t)d_m_in | (uintptr_t)d_m_out |
+         (uintptr_t)d_v_in | (uintptr_t)d_v_out) & 15)
+        return invalid("tables must be 16-byte aligned");
+    return sgns_step_adam(d_w_in, d_w_out, d_m_in, d_v_in, d_m_out, d_v_out, n_nodes, dim, d_walks,
+                          n_walks, walk_id_base, walk_len, window, n_neg, d_alias, lr, beta1, beta2,
+                          eps, step, seed, pair_mode, d_loss_sum, d_pair_count, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------ corpus variants
+gs_status gs_build_keep_thresholds(const double *h_weights, int64_t n, double t, uint32_t *h_thr_out)
+{
+    if (!h_weights || !h_thr_out) return invalid("null pointer");
+    if (n <= 0) return invalid("n must be positive");
+    if (!(t > 0.0) || !isfinite(t)) return invalid("t must be positive");
+    double sum = 0.0;
+    for (int64_t v = 0; v < n; ++v) {
+        const double x = h_weights[v];
+        if (!(x >= 0.0) || !isfinite(x)) return invalid("weights must be finite and >= 0");
+        sum += x;
+    }
+    if (!(sum > 0.0)) return invalid("no positive weight");
+    for (int64_t v = 0; v < n; ++v) {
+        uint32_t thr = 0xFFFFFFFFu;                       // always kept
+        if (h_weights[v] > 0.0) {
+            const double freq = h_weights[v] / sum;
+            const double keep = sqrt(t / freq);
+            if (keep < 1.0) {
+                const double scaled = floor(keep * 4294967296.0);
+                if (scaled < 4294967295.0) thr = (uint32_t)scaled;
+            }
+        }
+        h_thr_out[v] = thr;
+    }
+    return GS_OK;
+}
+
+gs_status gs_subsample_walks(const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                             int32_t walk_len, const uint32_t *d_keep_thr, uint64_t seed,
+                             int32_t *d_walks_out, uint64_t *d_kept, void *stream)
+{
+    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
+    if (walk_len < 1 || walk_len > 1024) { set_error("walk_len %d outside [1, 1024]", walk_len); return GS_ERR_UNSUPPORTED; }
+    if (n_walks > 0 && (!d_walks || !d_walks_out || !d_keep_thr)) return invalid("null pointer");
+    return launch_subsample_walks(d_walks, n_walks, walk_id_base, walk_len, d_keep_thr, seed,
+                                  d_walks_out, (unsigned long long *)d_kept, (cudaStream_t)stream);
+}
+
+gs_status gs_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epoch, int64_t walk_id_first,
+                             int64_t count, int32_t *d_starts_out, void *stream)
+{
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
+    if (walk_id_first < 0 || count < 0) return invalid("negative walk_id_first or count");
+    if (count > 0 && !d_starts_out) return invalid("d_starts_out is NULL");
+    return launch_shuffled_starts(n_nodes, seed, epoch, walk_id_first, count, d_starts_out,
+                                  (cudaStream_t)stream);
+}
+
 // ------------------------------------------------------------------ epoch driver
 struct EpochCounters {
     double loss;
@@ -538,6 +626,7 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
     TimerRing t_walk, t_sgns;
     gs_status rc = GS_OK;
     int32_t *wbuf[2] = { nullptr, nullptr };
+    int32_t *sbuf[2] = { nullptr, nullptr };
     EpochCounters *ctr = nullptr;
     EpochCounters host_ctr;
     memset(&host_ctr, 0, sizeof(host_ctr));
@@ -556,6 +645,11 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
         EP_CALL(workspace_get(WS_WALKS0, wbytes, &p)); wbuf[0] = (int32_t *)p;
         EP_CALL(workspace_get(WS_WALKS1, wbytes, &p)); wbuf[1] = (int32_t *)p;
         EP_CALL(workspace_get(WS_COUNTERS, 256, &p)); ctr = (EpochCounters *)p;
+        if (cfg->shuffle_starts) {                       // start nodes of the two batches in flight
+            EP_CALL(workspace_get(WS_STARTS, 2 * sizeof(int32_t) * (size_t)cfg->batch_walks, &p));
+            sbuf[0] = (int32_t *)p;
+            sbuf[1] = sbuf[0] + cfg->batch_walks;
+        }
     }
     EP_TRY(cudaStreamCreateWithFlags(&s_walk, cudaStreamNonBlocking));
     for (int i = 0; i < 2; ++i) {
@@ -578,13 +672,21 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
         if (b - cfg->first_batch >= 2) EP_TRY(cudaStreamWaitEvent(s_walk, ev_sgns[buf], 0));
         {
             const int tk = t_walk.start(s_walk);
+            const int32_t *starts = nullptr;
+            if (cfg->shuffle_starts) {
+                EP_CALL(launch_shuffled_starts(g->n_nodes, cfg->seed, cfg->epoch, base, n, sbuf[buf], s_walk));
+                starts = sbuf[buf];
+            }
             if (cfg->walk_kind == GS_WALK_UNIFORM)
-                EP_CALL(launch_uniform_walks(g, nullptr, n, base, cfg->walk_len, cfg->seed, wbuf[buf],
+                EP_CALL(launch_uniform_walks(g, starts, n, base, cfg->walk_len, cfg->seed, wbuf[buf],
                                              &ctr->steps, s_walk));
             else
-                EP_CALL(launch_node2vec_walks(g, nullptr, n, base, cfg->walk_len, cfg->seed, cfg->p,
+                EP_CALL(launch_node2vec_walks(g, starts, n, base, cfg->walk_len, cfg->seed, cfg->p,
                                               cfg->q, cfg->max_rounds, g_n2v_group, wbuf[buf],
                                               &ctr->steps, &ctr->caps, s_walk));
+            if (cfg->d_keep_thr)
+                EP_CALL(launch_subsample_walks(wbuf[buf], n, base, cfg->walk_len, cfg->d_keep_thr,
+                                               cfg->seed, wbuf[buf], nullptr, s_walk));
             t_walk.stop(tk, s_walk);
         }
         EP_TRY(cudaEventRecord(ev_walk[buf], s_walk));

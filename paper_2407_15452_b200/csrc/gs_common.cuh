@@ -24,7 +24,7 @@ gs_status cuda_fail(cudaError_t e, const char *what);
 // Returns a 256-byte aligned scratch block of at least `bytes` for slot `slot`
 // (independent blocks so that kernels on different streams do not share one).
 gs_status workspace_get(int slot, size_t bytes, void **out);
-enum { WS_WALKS0 = 0, WS_WALKS1 = 1, WS_SGNS = 2, WS_COUNTERS = 3, WS_SLOTS = 4 };
+enum { WS_WALKS0 = 0, WS_WALKS1 = 1, WS_SGNS = 2, WS_COUNTERS = 3, WS_STARTS = 4, WS_SLOTS = 5 };
 
 int sm_count();
 
@@ -46,7 +46,8 @@ struct gs_graph {
 namespace gs {
 
 // ---- Philox4x32-10 ---------------------------------------------------------------
-enum : uint32_t { TAG_UNIFORM = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4 };
+enum : uint32_t { TAG_UNIFORM = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4,
+                  TAG_WINDOW = 5, TAG_SUBSAMPLE = 6, TAG_SHUFFLE = 7 };
 
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k)
 {

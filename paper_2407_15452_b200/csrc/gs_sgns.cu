@@ -293,14 +293,22 @@ __device__ __forceinline__ void sum_over_groups(Row<FPL> &x)
 // -1 where the pair does not exist or the negative equals the context (masked).
 // W points at the walk (global or shared), c = W[i] >= 0.  Returns the number of pairs
 // (identical on every lane).  dump_* (nullable) are this position's rows of the dump arrays.
-// fwd != 0 keeps only contexts that come later in the walk (edge sampling of LINE).
+// flags & PAIR_FWD keeps only contexts that come later in the walk (edge sampling of LINE);
+// flags & PAIR_SHRINK draws the window of this position, w_i = 1 + mulhi(word, w) uniform on
+// 1..w (word2vec's shrinking window), and keeps the contexts within w_i.  Slots and the keying
+// of the negatives stay those of the full window.
+enum { PAIR_FWD = 1, PAIR_SHRINK = 2 };
+
 __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_t i, int32_t w,
                                              int32_t K, uint64_t seed, uint64_t id,
                                              const uint64_t *__restrict__ alias, uint32_t n_alias,
                                              int32_t c, int32_t *tgt, int lane,
-                                             int32_t *dump_pairs, int32_t *dump_negs, int fwd)
+                                             int32_t *dump_pairs, int32_t *dump_negs, int flags)
 {
     const int S = 2 * w, T1 = 1 + K;
+    const bool fwd = (flags & PAIR_FWD) != 0;
+    int w_i = w;
+    if (flags & PAIR_SHRINK) w_i = 1 + (int)__umulhi(draw(seed, id, (uint32_t)i, TAG_WINDOW, 0).x, (uint32_t)w);
     const int hp = K > 0 ? (K + 1) / 2 : 1;          // Philox blocks per slot (>= 1 work item)
     int pairs = 0;
     __syncwarp();                                    // earlier readers of tgt are done
@@ -310,7 +318,8 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
         if (it < S * hp) {
             const int s = it / hp, m = it - s * hp;
             const int j = i - w + s + (s >= w ? 1 : 0);
-            const int32_t ctx = (j >= 0 && j < L && !(fwd && s < w)) ? W[j] : -1;   // fwd: only j > i
+            const bool in_window = j - i <= w_i && i - j <= w_i && !(fwd && s < w);   // fwd: only j > i
+            const int32_t ctx = (j >= 0 && j < L && in_window) ? W[j] : -1;
             valid = ctx >= 0;
             if (m == 0) {
                 tgt[s * T1] = ctx;
@@ -581,11 +590,20 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out,
 // row is  m <- mu m + grad ; row <- row - lr m ; last[row] <- next_iter  (Section 3.2: mult, put,
 // mult_add, restricted to the rows of the batch; the other rows are brought up to date lazily by
 // momentum_catchup before they are read again).
+//
+// With v != nullptr the state is Adam's instead (Kingma & Ba 2015, Algorithm 1; Section 3.2 names
+// Adam next to SGD with momentum): m and v are the first and second moments, mu is beta1, and
+// only the rows of the batch move (no catch-up: a row outside the batch keeps row, m and v):
+//   m <- b1 m + (1-b1) g ; v <- b2 v + (1-b2) g^2 ; row <- row - lr (m/c1) / (sqrt(v/c2) + eps)
+// with c1 = 1 - b1^step, c2 = 1 - b2^step computed on the host.
 struct MomState {
     float *m;
     int32_t *last;
     float mu;
     int32_t next_iter;
+    float *v;
+    float b2, eps;
+    double c1, c2;
 };
 
 template <int FPL, typename T>
@@ -593,7 +611,22 @@ __device__ __forceinline__ void write_updated_row(T *__restrict__ tab, int64_t r
                                                   Row<FPL> &row, const double (&acc)[FPL], float lr,
                                                   const MomState &ms)
 {
-    if (ms.m) {
+    if (ms.v) {
+        Row<FPL> m = row_load<FPL>(ms.m, r, lane);
+        Row<FPL> v = row_load<FPL>(ms.v, r, lane);
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) {
+            const double g = acc[j];
+            const double mm = (double)ms.mu * (double)m.v[j] + (1.0 - (double)ms.mu) * g;
+            const double vv = (double)ms.b2 * (double)v.v[j] + (1.0 - (double)ms.b2) * g * g;
+            m.v[j] = (float)mm;
+            v.v[j] = (float)vv;
+            row.v[j] = (float)((double)row.v[j] -
+                               (double)lr * (mm / ms.c1) / (sqrt(vv / ms.c2) + (double)ms.eps));
+        }
+        row_store<FPL>(ms.m, r, lane, m);
+        row_store<FPL>(ms.v, r, lane, v);
+    } else if (ms.m) {
         Row<FPL> m = row_load<FPL>(ms.m, r, lane);
 #pragma unroll
         for (int j = 0; j < FPL; ++j) {
@@ -927,7 +960,7 @@ struct SgnsArgs {
     double *loss;
     int64_t *pairs;
     int32_t *dump_pairs, *dump_negs;
-    int fwd;                      // forward-only pairs
+    int fwd;                      // PAIR_* flags of build_targets
 };
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
@@ -978,6 +1011,10 @@ struct MomHost {
     int32_t *last_in, *last_out;
     float mu;
     int32_t iter;
+    // Adam (gs_sgns_step_adam): second moments, beta2, eps and the 1-based step; mu is beta1
+    float *v_in, *v_out;
+    float b2, eps;
+    int64_t step;
 };
 
 template <int DIM, typename T>
@@ -986,7 +1023,14 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
     T *w_in = (T *)a.w_in, *w_out = (T *)a.w_out;
     constexpr int FPL = DIM / 32;                        // the apply passes use a whole warp per row
     MomState ms_in = { nullptr, nullptr, 0.f, 0 }, ms_out = { nullptr, nullptr, 0.f, 0 };
-    if (mom) {
+    const bool adam = mom && mom->v_in;
+    if (adam) {
+        const double c1 = 1.0 - pow((double)mom->mu, (double)mom->step);
+        const double c2 = 1.0 - pow((double)mom->b2, (double)mom->step);
+        ms_in = MomState{ mom->m_in, nullptr, mom->mu, 0, mom->v_in, mom->b2, mom->eps, c1, c2 };
+        ms_out = MomState{ mom->m_out, nullptr, mom->mu, 0, mom->v_out, mom->b2, mom->eps, c1, c2 };
+        mom = nullptr;                                   // no lazy catch-up: the plain order of passes
+    } else if (mom) {
         ms_in = MomState{ mom->m_in, mom->last_in, mom->mu, mom->iter + 1 };
         ms_out = MomState{ mom->m_out, mom->last_out, mom->mu, mom->iter + 1 };
     }
@@ -1074,6 +1118,11 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
     return GS_OK;
 }
 
+static int pair_flags_of(int32_t mode)
+{
+    return ((mode & GS_PAIRS_FORWARD_ONLY) ? PAIR_FWD : 0) | ((mode & GS_WINDOW_SHRINK) ? PAIR_SHRINK : 0);
+}
+
 template <int DIM, typename T>
 static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
 {
@@ -1091,8 +1140,8 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, (mode & GS_PAIRS_FORWARD_ONLY) ? 1 : 0 };
-    mode &= ~GS_PAIRS_FORWARD_ONLY;
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode) };
+    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     switch (dim) {
         case 32: return run_mode<32, float>(a, mode, st);
         case 64: return run_mode<64, float>(a, mode, st);
@@ -1112,8 +1161,8 @@ gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, c
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, (mode & GS_PAIRS_FORWARD_ONLY) ? 1 : 0 };
-    mode &= ~GS_PAIRS_FORWARD_ONLY;
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode) };
+    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     switch (dim) {
         case 64: return run_mode<64, __half>(a, mode, st);
         case 128: return run_mode<128, __half>(a, mode, st);
@@ -1133,7 +1182,28 @@ gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_ou
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
                    seed, loss, pairs, nullptr, nullptr, 0 };
-    MomHost mom = { m_in, m_out, last_in, last_out, mu, iter };
+    MomHost mom = { m_in, m_out, last_in, last_out, mu, iter, nullptr, nullptr, 0.f, 0.f, 0 };
+    switch (dim) {
+        case 32: return run_deterministic<32, float>(a, st, &mom);
+        case 64: return run_deterministic<64, float>(a, st, &mom);
+        case 128: return run_deterministic<128, float>(a, st, &mom);
+        case 256: return run_deterministic<256, float>(a, st, &mom);
+        default:
+            set_error("dim %d not supported (32, 64, 128, 256)", dim);
+            return GS_ERR_UNSUPPORTED;
+    }
+}
+
+gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, float *m_out,
+                         float *v_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                         const uint64_t *alias, float lr, float b1, float b2, float eps, int64_t step,
+                         uint64_t seed, int32_t pair_mode, double *loss, int64_t *pairs, cudaStream_t st)
+{
+    if (n_walks == 0) return GS_OK;
+    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                   seed, loss, pairs, nullptr, nullptr, pair_flags_of(pair_mode) };
+    MomHost mom = { m_in, m_out, nullptr, nullptr, b1, 0, v_in, v_out, b2, eps, step };
     switch (dim) {
         case 32: return run_deterministic<32, float>(a, st, &mom);
         case 64: return run_deterministic<64, float>(a, st, &mom);

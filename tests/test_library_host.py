@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 
 def test_struct_layouts_match_header():
-    assert ctypes.sizeof(B.SgnsConfig) == 10 * 4 + 3 * 8 + 3 * 8 + 8
+    assert ctypes.sizeof(B.SgnsConfig) == 10 * 4 + 3 * 8 + 3 * 8 + 8 + 8 + 2 * 4
     assert ctypes.sizeof(B.EpochStats) == 8 + 4 * 8 + 3 * 4 + 4
 
 
@@ -57,6 +57,21 @@ def test_host_alias_builder_rejects_bad_input(lib):
         B.gs_build_alias(np.array([1.0, np.nan]), 0.75)
 
 
+def test_host_keep_thresholds_match_oracle_bit_for_bit(lib):
+    rng = np.random.default_rng(5)
+    w = rng.pareto(1.1, size=30000) + 0.01
+    w[rng.integers(0, 30000, 300)] = 0.0
+    for t in (1e-3, 1e-5, 1e-7):
+        got = B.gs_build_keep_thresholds(w, t)
+        want = O.keep_thresholds(w, t)
+        assert np.array_equal(got, want)
+        assert (got == 0xFFFFFFFF).any() and (got != 0xFFFFFFFF).any()
+    with pytest.raises(B.GsError):
+        B.gs_build_keep_thresholds(np.zeros(4), 1e-3)
+    with pytest.raises(B.GsError):
+        B.gs_build_keep_thresholds(np.ones(4), 0.0)
+
+
 def test_argument_errors_are_status_codes_without_touching_a_gpu(lib):
     h = ctypes.c_void_p(0)
     st = lib.gs_graph_load_csr(ctypes.c_int64(0), ctypes.c_int64(0), None, 0, None, 0, None,
@@ -77,6 +92,18 @@ def test_argument_errors_are_status_codes_without_touching_a_gpu(lib):
     st = lib.gs_random_walks(None, None, ctypes.c_int64(1), ctypes.c_int64(0), 4,
                              ctypes.c_uint64(0), None, None, None)
     assert st == -1
+    st = lib.gs_shuffled_starts(ctypes.c_int64(0), ctypes.c_uint64(1), ctypes.c_uint32(0),
+                                ctypes.c_int64(0), ctypes.c_int64(4), ctypes.c_void_p(16), None)
+    assert st == -1 and b"n_nodes" in lib.gs_last_error()
+    st = lib.gs_subsample_walks(ctypes.c_void_p(16), ctypes.c_int64(2), ctypes.c_int64(0), 2000,
+                                ctypes.c_void_p(16), ctypes.c_uint64(0), ctypes.c_void_p(16), None, None)
+    assert st == -6 and b"walk_len" in lib.gs_last_error()
+    p16 = ctypes.c_void_p(256)
+    st = lib.gs_sgns_step_adam(p16, p16, p16, p16, p16, p16, ctypes.c_int64(10), 128, p16,
+                               ctypes.c_int64(1), ctypes.c_int64(0), 4, 2, 1, p16, ctypes.c_float(0.1),
+                               ctypes.c_float(0.9), ctypes.c_float(0.999), ctypes.c_float(1e-8),
+                               ctypes.c_int64(0), ctypes.c_uint64(0), 0, None, None, None)
+    assert st == -1 and b"step" in lib.gs_last_error()
     assert lib.gs_tune_node2vec_group(3) == -1
     assert lib.gs_tune_node2vec_group(1) == 0
     lib.gs_graph_free(None)

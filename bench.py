@@ -45,7 +45,11 @@ def parse_args():
     ap.add_argument("--workload", default="deepwalk_large")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the node count (testing)")
     ap.add_argument("--batch-walks", type=int, default=1 << 20)
-    ap.add_argument("--mode", default="hogwild", choices=["hogwild", "hogwild_red", "deterministic", "momentum"])
+    ap.add_argument("--mode", default="hogwild",
+                    choices=["hogwild", "hogwild_red", "deterministic", "momentum", "adam"])
+    ap.add_argument("--variants", default="",
+                    help="comma list of shrink (per-position window draw), subsample (frequent-node "
+                         "sub-sampling, t = 1e-5), shuffle (keyed start-node order)")
     ap.add_argument("--table-dtype", default="f32", choices=["f32", "f16"],
                     help="storage type of the embedding tables (arithmetic is fp32 either way)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -239,6 +243,22 @@ def walk_kernel_name(wl, indexed):
     return "uniform_walk_index_kernel" if indexed else "uniform_walk_vec_kernel"
 
 
+def parse_variants(args):
+    v = {x for x in args.variants.split(",") if x}
+    bad = v - {"shrink", "subsample", "shuffle"}
+    if bad:
+        raise SystemExit(f"unknown variant(s): {sorted(bad)}")
+    return v
+
+
+def keep_thresholds_device(g, dev, t=1e-5):
+    """Sub-sampling thresholds from the degrees (host call of the library), uploaded."""
+    import torch
+    from paper_2407_15452_b200 import binding as B
+    thr = B.gs_build_keep_thresholds(g.degrees().cpu().numpy().astype(np.float64), t)
+    return torch.from_numpy(thr.view(np.int32)).to(dev)
+
+
 # ---------------------------------------------------------------------------- walk sampler alone
 def run_walks_only(args, wl, g, G, info, dev):
     """Times gs_random_walks / gs_node2vec_walks alone on batches of the workload (1 GPU)."""
@@ -250,20 +270,29 @@ def run_walks_only(args, wl, g, G, info, dev):
     nb_total = (total_walks + bw - 1) // bw
     out = torch.empty((bw, wl.walk_len), dtype=torch.int32, device=dev)
     steps = torch.zeros(1, dtype=torch.int64, device=dev)
+    variants = parse_variants(args)
+    starts = torch.empty(bw, dtype=torch.int32, device=dev) if "shuffle" in variants else None
+    keep_thr = keep_thresholds_device(g, dev) if "subsample" in variants else None
+    kept = torch.zeros(1, dtype=torch.int64, device=dev)
 
     def run(b):
         base = (b % nb_total) * bw
         cnt = min(bw, total_walks - base)
+        if starts is not None:
+            B.gs_shuffled_starts(n, wl.graph_seed, 0, base, cnt, dev, out=starts)
         if wl.walk_kind == "uniform":
-            B.gs_random_walks(G, None, cnt, base, wl.walk_len, wl.graph_seed, out=out, steps=steps)
+            B.gs_random_walks(G, starts, cnt, base, wl.walk_len, wl.graph_seed, out=out, steps=steps)
         else:
-            B.gs_node2vec_walks(G, None, cnt, base, wl.walk_len, wl.graph_seed, wl.p, wl.q, out=out,
+            B.gs_node2vec_walks(G, starts, cnt, base, wl.walk_len, wl.graph_seed, wl.p, wl.q, out=out,
                                 steps=steps)
+        if keep_thr is not None:
+            B.gs_subsample_walks(out[:cnt], base, keep_thr, wl.graph_seed, out=out[:cnt], kept=kept)
 
     for s in range(args.warmup):
         run(s)
     torch.cuda.synchronize()
     steps.zero_()
+    kept.zero_()
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -283,9 +312,11 @@ def run_walks_only(args, wl, g, G, info, dev):
         "metric": "walk_steps_per_s", "value": st / (ms * 1e-3), "unit": "walk-steps/s", "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
-        "data": "synthetic", "gpu_launches": args.steps, "clocks": clocks,
+        "data": "synthetic", "gpu_launches": args.steps * (1 + len(variants & {"shuffle", "subsample"})),
+        "clocks": clocks,
         "config": {"workload": wl.name, "stage": "walks", "batch_walks": bw, "walk_kind": wl.walk_kind,
-                   "walk_len": wl.walk_len, "scale": args.scale, **info},
+                   "walk_len": wl.walk_len, "scale": args.scale, "variants": sorted(variants),
+                   "kept_entries": int(kept.item()) if keep_thr is not None else None, **info},
         "roofline": {"bound": "hbm", "kernel": walk_kernel_name(wl, indexed),
                      "achieved": payload, "peak": peak, "unit": "GB/s", "frac": payload / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": None,
@@ -295,22 +326,28 @@ def run_walks_only(args, wl, g, G, info, dev):
 
 # ---------------------------------------------------------------------------- momentum step
 def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
-    """Times walks + gs_sgns_step_momentum on batches of 512 walks (synchronous, momentum 0.9 as
-    in the paper's production run).  1 GPU."""
+    """Times walks + gs_sgns_step_momentum (or gs_sgns_step_adam with --mode adam) on batches of
+    512 walks (synchronous; momentum 0.9 as in the paper's production run).  1 GPU."""
     import torch
     from paper_2407_15452_b200 import binding as B
     n = g.n_nodes
     bw = min(args.batch_walks, 512)
     total_walks = n * wl.walks_per_node
     nb_total = (total_walks + bw - 1) // bw
+    adam = args.mode == "adam"
     m_in, m_out = torch.zeros_like(w_in), torch.zeros_like(w_out)
-    last_in = torch.zeros(n, dtype=torch.int32, device=dev)
-    last_out = torch.zeros_like(last_in)
+    if adam:
+        v_in, v_out = torch.zeros_like(w_in), torch.zeros_like(w_out)
+    else:
+        last_in = torch.zeros(n, dtype=torch.int32, device=dev)
+        last_out = torch.zeros_like(last_in)
     walks = torch.empty((bw, wl.walk_len), dtype=torch.int32, device=dev)
     loss = torch.zeros(1, dtype=torch.float64, device=dev)
     cnt = torch.zeros(1, dtype=torch.int64, device=dev)
     mu = 0.9
     seed, lr = wl.graph_seed, wl.lr0 * (1.0 - mu)      # same effective step lr / (1 - mu) as the plain runs
+    if adam:
+        lr = 0.001                                     # Adam's usual step size
 
     def step(it):
         base = (it % nb_total) * bw
@@ -319,8 +356,12 @@ def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
             B.gs_random_walks(G, None, k, base, wl.walk_len, seed, out=walks)
         else:
             B.gs_node2vec_walks(G, None, k, base, wl.walk_len, seed, wl.p, wl.q, out=walks)
-        B.gs_sgns_step_momentum(w_in, w_out, m_in, m_out, last_in, last_out, walks[:k], base,
-                                wl.window, wl.n_neg, alias, lr, mu, it, seed, loss, cnt)
+        if adam:
+            B.gs_sgns_step_adam(w_in, w_out, m_in, v_in, m_out, v_out, walks[:k], base, wl.window,
+                                wl.n_neg, alias, lr, 0.9, 0.999, 1e-8, it + 1, seed, 0, loss, cnt)
+        else:
+            B.gs_sgns_step_momentum(w_in, w_out, m_in, m_out, last_in, last_out, walks[:k], base,
+                                    wl.window, wl.n_neg, alias, lr, mu, it, seed, loss, cnt)
 
     for it in range(args.warmup):
         step(it)
@@ -339,21 +380,23 @@ def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
     ms = ev0.elapsed_time(ev1)
     pairs = int(cnt.item())
     peak, peak_kind = measured_peak_gbs()
-    # per pair and target: the embedding row and its momentum row, each read and written once
-    model = pairs * (1 + wl.n_neg) * 4 * wl.dim * 4
+    # per pair and target: the embedding row and its momentum row (Adam: both moment rows), each
+    # read and written once
+    model = pairs * (1 + wl.n_neg) * (6 if adam else 4) * wl.dim * 4
     gbs = model / (ms * 1e-3) / 1e9
     print(json.dumps({
         "metric": METRIC, "value": pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "gpu_launches": None, "clocks": clocks, "mean_loss": loss.item() / max(pairs, 1),
-        "config": {"workload": wl.name, "mode": "momentum", "momentum": mu, "lr": lr, "batch_walks": bw,
+        "config": {"workload": wl.name, "mode": args.mode, "momentum": mu, "lr": lr, "batch_walks": bw,
                    "walk_len": wl.walk_len, "window": wl.window, "n_neg": wl.n_neg, "dim": wl.dim,
                    "scale": args.scale, **info},
-        "roofline": {"bound": "hbm", "kernel": "momentum step (keys, sort, catch-up, coefficients, apply)",
+        "roofline": {"bound": "hbm", "kernel": "adam step (coefficients, sort, apply)" if adam else
+                     "momentum step (keys, sort, catch-up, coefficients, apply)",
                      "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": None,
-                     "bytes_model": "per pair and target: row and momentum row, read + written"},
+                     "bytes_model": "per pair and target: row and moment row(s), read + written"},
     }))
 
 
@@ -389,12 +432,16 @@ def run_ours(args, wl):
     seed = wl.graph_seed
     (B.gs_init_embeddings_f16 if f16 else B.gs_init_embeddings)(w_in, w_out, seed)
     step_fn = B.gs_sgns_step_f16 if f16 else B.gs_sgns_step
-    if args.mode == "momentum":
+    if args.mode in ("momentum", "adam"):
         return run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev)
     mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,
             "deterministic": B.GS_DETERMINISTIC}[args.mode]
     if wl.forward_only:
         mode |= B.GS_PAIRS_FORWARD_ONLY
+    variants = parse_variants(args)
+    if "shrink" in variants:
+        mode |= B.GS_WINDOW_SHRINK
+    keep_thr = keep_thresholds_device(g, dev) if "subsample" in variants else None
     kind = B.GS_WALK_UNIFORM if wl.walk_kind == "uniform" else B.GS_WALK_NODE2VEC
     total_walks = n * wl.walks_per_node
     bw = min(args.batch_walks, total_walks)
@@ -403,7 +450,7 @@ def run_ours(args, wl):
     nb_total = (total_walks + bw - 1) // bw
     ekw = dict(walks_per_node=wl.walks_per_node, walk_len=wl.walk_len, window=wl.window,
                n_neg=wl.n_neg, lr0=wl.lr0, batch_walks=bw, seed=seed, mode=mode, walk_kind=kind,
-               p=wl.p, q=wl.q)
+               p=wl.p, q=wl.q, keep_thr=keep_thr, shuffle_epoch=0 if "shuffle" in variants else None)
 
     def barrier():
         torch.cuda.synchronize()
@@ -462,6 +509,8 @@ def run_ours(args, wl):
                 B.gs_random_walks(G, d_starts, cnt, base, wl.walk_len, seed, out=d_walks)
             else:
                 B.gs_node2vec_walks(G, d_starts, cnt, base, wl.walk_len, seed, wl.p, wl.q, out=d_walks)
+            if keep_thr is not None:
+                B.gs_subsample_walks(d_walks[:cnt], base, keep_thr, seed, out=d_walks[:cnt])
             step_fn(w_in, w_out, d_walks[:cnt], base, wl.window, wl.n_neg, alias, wl.lr0,
                     seed, mode, d_loss, d_cnt)
             h_res.copy_(d_res, non_blocking=True)
@@ -502,7 +551,7 @@ def run_ours(args, wl):
             "config": {"workload": wl.name, "mode": args.mode, "table_dtype": args.table_dtype,
                        "batch_walks": bw,
                        "walk_kind": wl.walk_kind, "walk_len": wl.walk_len, "window": wl.window,
-                       "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale,
+                       "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale, "variants": sorted(variants),
                        "l2": "tables (2 x n x dim x 4 B) and CSR far exceed the 126 MB L2; no flush",
                        "multi_gpu": "replicas only", **info},
             "gpu_launches": 2 * args.steps,

@@ -612,17 +612,17 @@ __device__ __forceinline__ void write_updated_row(T *__restrict__ tab, int64_t r
                                                   const MomState &ms)
 {
     if (ms.v) {
+        // fp32 arithmetic on the fp64 gradient sum rounded once: the moments are stored in fp32
+        // anyway, and double-precision square roots and divisions would cost more than the rows.
         Row<FPL> m = row_load<FPL>(ms.m, r, lane);
         Row<FPL> v = row_load<FPL>(ms.v, r, lane);
+        const float b1 = ms.mu, b2 = ms.b2, inv_c1 = (float)(1.0 / ms.c1), inv_c2 = (float)(1.0 / ms.c2);
 #pragma unroll
         for (int j = 0; j < FPL; ++j) {
-            const double g = acc[j];
-            const double mm = (double)ms.mu * (double)m.v[j] + (1.0 - (double)ms.mu) * g;
-            const double vv = (double)ms.b2 * (double)v.v[j] + (1.0 - (double)ms.b2) * g * g;
-            m.v[j] = (float)mm;
-            v.v[j] = (float)vv;
-            row.v[j] = (float)((double)row.v[j] -
-                               (double)lr * (mm / ms.c1) / (sqrt(vv / ms.c2) + (double)ms.eps));
+            const float g = (float)acc[j];
+            m.v[j] = fmaf(b1, m.v[j], (1.0f - b1) * g);
+            v.v[j] = fmaf(b2, v.v[j], (1.0f - b2) * (g * g));
+            row.v[j] -= lr * (m.v[j] * inv_c1) / (sqrtf(v.v[j] * inv_c2) + ms.eps);
         }
         row_store<FPL>(ms.m, r, lane, m);
         row_store<FPL>(ms.v, r, lane, v);

@@ -308,6 +308,8 @@ def run_walks_only(args, wl, g, G, info, dev):
     indexed = "walk_index_bytes" in info
     payload = walk_bytes(st, wl.offsets64, indexed) / (ms * 1e-3) / 1e9
     granule = walk_granule_bytes(st, indexed) / (ms * 1e-3) / 1e9
+    # ceiling of one isolated random read per transition, measured on the same index in this run
+    read_rate = B.gs_probe_random_reads(G, 1 << 28) if indexed else None
     print(json.dumps({
         "metric": "walk_steps_per_s", "value": st / (ms * 1e-3), "unit": "walk-steps/s", "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
@@ -320,7 +322,9 @@ def run_walks_only(args, wl, g, G, info, dev):
         "roofline": {"bound": "hbm", "kernel": walk_kernel_name(wl, indexed),
                      "achieved": payload, "peak": peak, "unit": "GB/s", "frac": payload / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": None,
-                     "granule_gbs": granule, "granule_frac": granule / peak},
+                     "granule_gbs": granule, "granule_frac": granule / peak,
+                     "random_reads_per_s": read_rate,
+                     "frac_of_random_read_rate": st / (ms * 1e-3) / read_rate if read_rate else None},
     }))
 
 

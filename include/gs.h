@@ -159,6 +159,17 @@ GS_API gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts,
                             int32_t *d_walks_out, uint64_t *d_steps,
                             uint64_t *d_cap_hits, void *stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): times independent random 16-byte reads of the
+ * graph's walk index (GS_BUILD_WALK_INDEX required), issued with the load instruction the walk
+ * kernels use.  A walk transition is one such read that depends on the one before it, so the
+ * rate found here is the ceiling for walk transitions per second on this device and graph.
+ * n_reads is rounded up to a multiple of 65,536 (*h_reads_done); the kernel runs twice and the
+ * second run is timed with events on `stream` (*h_ms_out).  WAITS for completion.
+ */
+GS_API gs_status gs_probe_random_reads(const gs_graph *g, int64_t n_reads, int64_t *h_reads_done,
+                                       float *h_ms_out, void *stream);
+
 /* ---------------------------------------------------------------- SGNS */
 #define GS_DETERMINISTIC  0   /* synchronous mini-batch step, bitwise reproducible */
 #define GS_HOGWILD        1   /* lock-free: plain loads and stores, rows may race   */

@@ -31,7 +31,7 @@ EXPORTS = [
     "gs_init_embeddings", "gs_random_walks", "gs_node2vec_walks", "gs_sgns_step",
     "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static", "gs_sgns_step_momentum", "gs_momentum_flush",
     "gs_init_embeddings_f16", "gs_sgns_step_f16", "gs_sgns_step_adam", "gs_build_keep_thresholds",
-    "gs_subsample_walks", "gs_shuffled_starts",
+    "gs_subsample_walks", "gs_shuffled_starts", "gs_probe_random_reads",
 ]
 
 
@@ -182,6 +182,14 @@ def gs_node2vec_walks(graph: Graph, starts, n_walks: int, walk_id_base: int, wal
         _dev(out, torch.int32, "out"), _dev(steps, torch.int64, "steps", True),
         _dev(cap_hits, torch.int64, "cap_hits", True), _stream()))
     return out
+
+
+def gs_probe_random_reads(graph: Graph, n_reads: int):
+    """Random 16-byte reads per second over the graph's walk index (measurement aid)."""
+    done, ms = ctypes.c_int64(0), ctypes.c_float(0.0)
+    _check(lib().gs_probe_random_reads(graph._h, ctypes.c_int64(n_reads), ctypes.byref(done),
+                                       ctypes.byref(ms), _stream()))
+    return done.value / (ms.value * 1e-3)
 
 
 def gs_sgns_step(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int, alias,

@@ -54,6 +54,7 @@ gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, fl
 gs_status launch_subsample_walks(const int32_t *walks, int64_t n_walks, int64_t base, int32_t L,
                                  const uint32_t *keep_thr, uint64_t seed, int32_t *out,
                                  unsigned long long *kept, cudaStream_t st);
+gs_status random_read_probe(const gs_graph *g, int64_t n_reads, float *ms_out, cudaStream_t st);
 gs_status launch_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epoch, int64_t first,
                                  int64_t count, int32_t *starts, cudaStream_t st);
 
@@ -356,6 +357,17 @@ gs_status gs_tune_node2vec_group(int32_t lanes)
         return invalid("lanes per walk must be 1, 2, 4, 8 or 32");
     g_n2v_group = lanes;
     return GS_OK;
+}
+
+gs_status gs_probe_random_reads(const gs_graph *g, int64_t n_reads, int64_t *h_reads_done,
+                                float *h_ms_out, void *stream)
+{
+    if (!g || !h_reads_done || !h_ms_out) return invalid("null pointer");
+    if (!g->d_edge_rec) return invalid("the graph was loaded without GS_BUILD_WALK_INDEX");
+    if (n_reads < 1 || n_reads > ((int64_t)1 << 36)) return invalid("n_reads outside [1, 2^36]");
+    const int64_t per_block = 256 * 256;
+    *h_reads_done = (n_reads + per_block - 1) / per_block * per_block;
+    return random_read_probe(g, n_reads, h_ms_out, (cudaStream_t)stream);
 }
 
 // ------------------------------------------------------------------ SGNS

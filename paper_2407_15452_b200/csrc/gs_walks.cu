@@ -616,4 +616,54 @@ gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_
     return GS_OK;
 }
 
+// ---------------------------------------------------------------- measurement aid
+// Independent random 16-byte reads of the walk index with the same load instruction the walk
+// kernels use.  A walk transition is one such read that depends on the previous one; this kernel
+// gives the rate the memory system sustains when nothing but the reads is done, i.e. the ceiling
+// of any sampler that needs one isolated DRAM access per transition.
+__device__ __forceinline__ uint64_t probe_mix(uint64_t x)
+{
+    x ^= x >> 33; x *= 0xff51afd7ed558ccdull; x ^= x >> 33; x *= 0xc4ceb9fe1a85ec53ull; x ^= x >> 33;
+    return x;
+}
+
+__global__ void __launch_bounds__(256)
+random_read_probe_kernel(const int4 *__restrict__ rec, uint64_t n_rec, int iters, unsigned long long *sink)
+{
+    uint64_t s = probe_mix((uint64_t)blockIdx.x * blockDim.x + threadIdx.x + 1);
+    int acc = 0;
+    for (int it = 0; it < iters; it += 4) {
+        int4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { s = probe_mix(s + u + 1); v[u] = ld_random(rec + (s % n_rec)); }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc += v[u].x;
+    }
+    if (acc == 0x7fffffff) atomicAdd(sink, 1ull);           // keeps the loads alive
+}
+
+gs_status random_read_probe(const gs_graph *g, int64_t n_reads, float *ms_out, cudaStream_t st)
+{
+    const int iters = 256;
+    int64_t blocks = (n_reads + 256 * iters - 1) / (256 * iters);
+    if (blocks < 1) blocks = 1;
+    void *ws = nullptr;
+    gs_status s = workspace_get(WS_COUNTERS, 256, &ws);
+    if (s != GS_OK) return s;
+    unsigned long long *sink = (unsigned long long *)((char *)ws + 192);
+    cudaEvent_t e0, e1;
+    GS_CUDA_TRY(cudaEventCreate(&e0));
+    GS_CUDA_TRY(cudaEventCreate(&e1));
+    random_read_probe_kernel<<<(unsigned)blocks, 256, 0, st>>>(g->d_edge_rec, (uint64_t)g->n_edges, iters, sink);
+    cudaEventRecord(e0, st);
+    random_read_probe_kernel<<<(unsigned)blocks, 256, 0, st>>>(g->d_edge_rec, (uint64_t)g->n_edges, iters, sink);
+    cudaEventRecord(e1, st);
+    cudaError_t e = cudaEventSynchronize(e1);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(ms_out, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (e != cudaSuccess) return cuda_fail(e, "random read probe");
+    return GS_OK;
+}
+
 }  // namespace gs

@@ -1,8 +1,8 @@
 // Skip-gram-with-negative-sampling update kernels.
 //
 // A row of an embedding table is dim fp32 values, always moved with 16-byte
-// accesses: a whole warp holds one row for dim >= 128, half a warp for dim 64,
-// a quarter for dim 32 (so one warp-wide access moves 1, 2 or 4 rows), and a
+// accesses: a whole warp holds one row for dim >= 128, a quarter of a warp for
+// dim 64 and 32 (so one warp-wide access moves 1 or 4 rows), and a
 // row read or write is one fully coalesced request.  Dot products are
 // butterfly shuffles.  The path is bound by row traffic in HBM/L2, not by
 // arithmetic, so there is no tensor-core work here.
@@ -172,13 +172,16 @@ __device__ __forceinline__ double warp_sum_double(double s)
 // ---------------------------------------------------------------- rows held by part of a warp
 // For dim < 128 a full warp per row would move only 128 or 256 bytes per instruction, and the
 // per-row instruction cost - not bytes - would set the pace.  There a row is held by LPR = 16
-// or 8 lanes (16 bytes per lane) and one warp-wide access moves NG = 2 or 4 different rows.
+// or 8 lanes and one warp-wide access moves NG = 2 or 4 different rows.
 // T is the storage type of the table (float, or IEEE half with fp32 arithmetic): a lane always
 // moves 16 bytes per access, i.e. 4 floats or 8 halves.
 template <int DIM, typename T = float> struct RowGeom {
     static constexpr int PER16 = 16 / (int)sizeof(T);       // values per 16-byte access
     static constexpr int BYTES = DIM * (int)sizeof(T);
-    static constexpr int LPR = BYTES / 16 >= 32 ? 32 : BYTES / 16;   // lanes per row
+    // lanes per row: 16 bytes per lane, except that a 256-byte fp32 row is held by 8 lanes (32
+    // bytes each, four rows per warp-wide access): measured +5 % on the dim-64 workload, while
+    // half rows of 256 bytes run 13 % slower that way (16 values per lane cost a resident block)
+    static constexpr int LPR = BYTES / 16 >= 32 ? 32 : (BYTES == 256 && sizeof(T) == 4 ? 8 : BYTES / 16);
     static constexpr int FPL = DIM / LPR;                   // values per lane
     static constexpr int NG = 32 / LPR;                     // rows per warp-wide access
 };
@@ -998,7 +1001,7 @@ template <int DIM, typename T, bool RED>
 static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
     if constexpr (sizeof(T) == 2)            // half rows: 3 rows per group in flight, 6 blocks (measured)
-        return run_hogwild_b<DIM, T, RED, 6, 3>(a, st);
+        return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL > 8 ? 4 : 6), 3>(a, st);
     else
         return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL <= 4 ? 5 : 4), TCH>(a, st);
 }

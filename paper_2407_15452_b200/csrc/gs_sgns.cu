@@ -1,9 +1,9 @@
 // Skip-gram-with-negative-sampling update kernels.
 //
 // A row of an embedding table is dim fp32 values, always moved with 16-byte
-// accesses: a whole warp holds one row for dim >= 128, a quarter of a warp for
-// dim 64 and 32 (so one warp-wide access moves 1 or 4 rows), and a
-// row read or write is one fully coalesced request.  Dot products are
+// accesses: a whole warp holds one row of dim 256, half a warp one of dim 128,
+// a quarter one of dim 64 or 32 (so one warp-wide access moves 1, 2 or 4 rows),
+// and the lanes of a row read or write it as contiguous 16-byte pieces.  Dot products are
 // butterfly shuffles.  The path is bound by row traffic in HBM/L2, not by
 // arithmetic, so there is no tensor-core work here.
 //
@@ -175,13 +175,18 @@ __device__ __forceinline__ double warp_sum_double(double s)
 // or 8 lanes and one warp-wide access moves NG = 2 or 4 different rows.
 // T is the storage type of the table (float, or IEEE half with fp32 arithmetic): a lane always
 // moves 16 bytes per access, i.e. 4 floats or 8 halves.
-template <int DIM, typename T = float> struct RowGeom {
+template <int DIM, typename T = float, bool NARROW = false> struct RowGeom {
     static constexpr int PER16 = 16 / (int)sizeof(T);       // values per 16-byte access
     static constexpr int BYTES = DIM * (int)sizeof(T);
-    // lanes per row: 16 bytes per lane, except that a 256-byte fp32 row is held by 8 lanes (32
-    // bytes each, four rows per warp-wide access): measured +5 % on the dim-64 workload, while
-    // half rows of 256 bytes run 13 % slower that way (16 values per lane cost a resident block)
-    static constexpr int LPR = BYTES / 16 >= 32 ? 32 : (BYTES == 256 && sizeof(T) == 4 ? 8 : BYTES / 16);
+    // lanes per row: 16 bytes per lane for half tables and for fp32 rows of 128 bytes; fp32 rows
+    // of 256 and 512 bytes give a lane 32 bytes (8 and 16 lanes per row, 4 and 2 rows per
+    // warp-wide access), which halves the per-row instruction overhead: measured +5 % on the
+    // dim-64 workload and +4 % / +10 % on the 50M-node / 1M-node dim-128 workloads.  Half rows
+    // of 256 bytes run 13 % slower that way (16 values per lane cost a resident block).
+    // NARROW keeps 16 bytes per lane for those rows too: with few targets per position (LINE: one
+    // pair per walk) wide chunks stay half empty and the narrow layout is 20 % faster.
+    static constexpr int LPR = !NARROW && sizeof(T) == 4 && (BYTES == 256 || BYTES == 512)
+                                   ? BYTES / 32 : (BYTES / 16 >= 32 ? 32 : BYTES / 16);
     static constexpr int FPL = DIM / LPR;                   // values per lane
     static constexpr int NG = 32 / LPR;                     // rows per warp-wide access
 };
@@ -213,10 +218,10 @@ __device__ __forceinline__ uint4 pack16(const float *v, const __half *)
 
 // Lane `sub` of a row group holds, for access q, the PER16 columns starting at
 // (q * LPR + sub) * PER16.
-template <int DIM, typename T>
-__device__ __forceinline__ Row<RowGeom<DIM, T>::FPL> grow_load(const T *__restrict__ tab, int64_t r, int sub)
+template <int DIM, typename T, bool NARROW = false>
+__device__ __forceinline__ Row<RowGeom<DIM, T, NARROW>::FPL> grow_load(const T *__restrict__ tab, int64_t r, int sub)
 {
-    using G = RowGeom<DIM, T>;
+    using G = RowGeom<DIM, T, NARROW>;
     Row<G::FPL> out;
     const uint4 *p = reinterpret_cast<const uint4 *>(tab + r * (int64_t)DIM);
 #pragma unroll
@@ -228,11 +233,11 @@ __device__ __forceinline__ Row<RowGeom<DIM, T>::FPL> grow_load(const T *__restri
     return out;
 }
 
-template <int DIM, typename T>
+template <int DIM, typename T, bool NARROW = false>
 __device__ __forceinline__ void grow_store(T *__restrict__ tab, int64_t r, int sub,
-                                           const Row<RowGeom<DIM, T>::FPL> &x)
+                                           const Row<RowGeom<DIM, T, NARROW>::FPL> &x)
 {
-    using G = RowGeom<DIM, T>;
+    using G = RowGeom<DIM, T, NARROW>;
     uint4 *p = reinterpret_cast<uint4 *>(tab + r * (int64_t)DIM);
 #pragma unroll
     for (int q = 0; q < G::FPL / G::PER16; ++q)
@@ -257,19 +262,19 @@ __device__ __forceinline__ void grow_store_f32(float *__restrict__ tab, int64_t 
 }
 
 // row += x as reductions (fp32 tables only)
-template <int DIM>
+template <int DIM, bool NARROW>
 __device__ __forceinline__ void grow_red_add(float *__restrict__ tab, int64_t r, int sub,
-                                             const Row<RowGeom<DIM, float>::FPL> &x)
+                                             const Row<RowGeom<DIM, float, NARROW>::FPL> &x)
 {
-    constexpr int FPL = RowGeom<DIM, float>::FPL, LPR = RowGeom<DIM, float>::LPR;
+    constexpr int FPL = RowGeom<DIM, float, NARROW>::FPL, LPR = RowGeom<DIM, float, NARROW>::LPR;
     float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
 #pragma unroll
     for (int q = 0; q < FPL / 4; ++q)
         atomicAdd(p + q * LPR + sub,
                   make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
 }
-template <int DIM>
-__device__ __forceinline__ void grow_red_add(__half *, int64_t, int, const Row<RowGeom<DIM, __half>::FPL> &) {}
+template <int DIM, bool NARROW>
+__device__ __forceinline__ void grow_red_add(__half *, int64_t, int, const Row<RowGeom<DIM, __half, NARROW>::FPL> &) {}
 
 // sum over the LPR lanes that hold one row (identical bits on each of them)
 template <int LPR>
@@ -368,7 +373,7 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
 }
 
 // ---------------------------------------------------------------- lock-free kernel
-template <int DIM, typename T, bool RED, int MINB, int TC>
+template <int DIM, typename T, bool RED, int MINB, int TC, bool NARROW>
 __global__ void __launch_bounds__(SGNS_WARPS * 32, MINB)
 sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     const int32_t *__restrict__ walks, int64_t n_walks, int64_t walk_id_base,
@@ -377,7 +382,8 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs,
                     unsigned long long *ticket, int fwd)
 {
-    constexpr int FPL = RowGeom<DIM, T>::FPL, LPR = RowGeom<DIM, T>::LPR, NG = RowGeom<DIM, T>::NG;
+    using G = RowGeom<DIM, T, NARROW>;
+    constexpr int FPL = G::FPL, LPR = G::LPR, NG = G::NG;
     constexpr int CH = TC * NG;                          // targets per chunk
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
@@ -408,7 +414,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                                             dp, dn, fwd);
             if (pairs == 0) continue;
             pair_acc += (unsigned long long)pairs;
-            const Row<FPL> u = grow_load<DIM>(w_in, c, sub);     // every group holds the center row
+            const Row<FPL> u = grow_load<DIM, T, NARROW>(w_in, c, sub);     // every group holds the center row
             Row<FPL> acc;                                        // this group's share of its gradient
 #pragma unroll
             for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
@@ -429,7 +435,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     float f[TC];
 #pragma unroll
                     for (int k = 0; k < TC; ++k)
-                        if (ids[k] >= 0) rows[k] = grow_load<DIM>(w_out, ids[k], sub);
+                        if (ids[k] >= 0) rows[k] = grow_load<DIM, T, NARROW>(w_out, ids[k], sub);
 #pragma unroll
                     for (int k = 0; k < TC; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
 #pragma unroll
@@ -453,8 +459,8 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                                 delta.v[j] = step * u.v[j];
                                 rows[k].v[j] += delta.v[j];
                             }
-                            if (RED) grow_red_add<DIM>(w_out, ids[k], sub, delta);
-                            else grow_store<DIM>(w_out, ids[k], sub, rows[k]);
+                            if (RED) grow_red_add<DIM, NARROW>(w_out, ids[k], sub, delta);
+                            else grow_store<DIM, T, NARROW>(w_out, ids[k], sub, rows[k]);
                         }
                     }
                 }
@@ -467,12 +473,12 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
 #pragma unroll
             for (int j = 0; j < FPL; ++j) delta.v[j] = -lr * acc.v[j];
             if (RED) {
-                if (grp == 0) grow_red_add<DIM>(w_in, c, sub, delta);
+                if (grp == 0) grow_red_add<DIM, NARROW>(w_in, c, sub, delta);
             } else {
-                Row<FPL> now = grow_load<DIM>(w_in, c, sub);
+                Row<FPL> now = grow_load<DIM, T, NARROW>(w_in, c, sub);
 #pragma unroll
                 for (int j = 0; j < FPL; ++j) now.v[j] += delta.v[j];
-                if (grp == 0) grow_store<DIM>(w_in, c, sub, now);
+                if (grp == 0) grow_store<DIM, T, NARROW>(w_in, c, sub, now);
             }
             loss_acc += (double)loss;
         }
@@ -968,12 +974,12 @@ struct SgnsArgs {
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
-template <int DIM, typename T, bool RED, int MINB, int TC = TCH>
+template <int DIM, typename T, bool RED, int MINB, int TC = TCH, bool NARROW = false>
 static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
     const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(a.L + SL);
-    auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB, TC>;
+    auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB, TC, NARROW>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -1002,8 +1008,15 @@ static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
     if constexpr (sizeof(T) == 2)            // half rows: 3 rows per group in flight, 6 blocks (measured)
         return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL > 8 ? 4 : 6), 3>(a, st);
-    else
-        return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL <= 4 ? 5 : 4), TCH>(a, st);
+    else {
+        // few targets per position (fewer than two wide chunks): 16 bytes per lane, one chunk
+        // of TCH rows per row group, so that chunks are full
+        using W = RowGeom<DIM, T, false>;
+        using N = RowGeom<DIM, T, true>;
+        if (W::LPR != N::LPR && 2 * a.w * (1 + a.K) < 2 * TCH * W::NG)
+            return run_hogwild_b<DIM, T, RED, (N::FPL <= 4 ? 5 : 4), TCH, true>(a, st);
+        return run_hogwild_b<DIM, T, RED, (W::FPL <= 4 ? 5 : 4), TCH>(a, st);
+    }
 }
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }

@@ -103,7 +103,7 @@ GS_API gs_status gs_graph_info(const gs_graph *g, int64_t *n_nodes, int64_t *n_e
 /*
  * HOST function.  Builds the alias table of p(v) ~ h_weights[v]^power (the
  * word2vec unigram^0.75 negative distribution when weights are node
- * frequencies or degrees; the paper only says nodes are "negatively sampled",
+ * frequencies or degrees; the paper only says that negatives are sampled,
  * Section 3.2).  Zero weights get probability zero.  Entry v of h_table_out
  * packs thr (low 32 bits) and alias (high 32 bits): a draw with words (a, b)
  * picks cell j = (a * n) >> 32 and returns j if b < thr[j], else alias[j].
@@ -126,7 +126,7 @@ GS_API gs_status gs_init_embeddings(float *d_w_in, float *d_w_out, int64_t n_nod
 
 /* ---------------------------------------------------------------- walks */
 /*
- * DeepWalk walks (Section 2.2: "random walks from each node").
+ * DeepWalk walks (Section 2.2: every node is the source of random walks).
  *   d_starts     : n_walks start nodes, or NULL for start = walk id mod n_nodes
  *   walk id      : walk_id_base + index; selects the random stream
  *   walk_len     : number of NODES per walk (Section 3.2 counts a batch as
@@ -142,8 +142,8 @@ GS_API gs_status gs_random_walks(const gs_graph *g, const int32_t *d_starts,
                           uint64_t *d_steps, void *stream);
 
 /*
- * node2vec walks (Section 2.2: "biased random walk to balance between
- * breadth-first and depth-first traversals"; Grover & Leskovec 2016).  After
+ * node2vec walks (Section 2.2: a biased walk that trades breadth-first
+ * against depth-first exploration; Grover & Leskovec 2016).  After
  * the move prev -> cur, neighbour x of cur has weight 1/p if x = prev, 1 if x
  * is a neighbour of prev, 1/q otherwise.  Sampled by rejection with tag 2:
  * round s proposes x = cols[off[cur] + ((word0 * deg) >> 32)] and accepts iff

@@ -18,8 +18,8 @@
  *   - updates of a mini-batch are written as increments, and trainers may race
  *     on the same rows, Hogwild style (Section 3.2 "Synchronization").
  * Everything the paper leaves open (RNG, index mapping, negative distribution,
- * masking, gradient scaling) follows the readings listed in the design notes
- * of this repository; each function below states the reading it implements.
+ * masking, gradient scaling) is a reading; each function below states the
+ * reading it implements.
  *
  * Parity pins (see tests, "not gpu"): Philox known answers; walks follow
  * edges; degree-proportional stationarity; node2vec closed-form transition
@@ -83,7 +83,7 @@ static uint64_t scale32(uint32_t r, uint64_t n)
 }
 
 /* ------------------------------------------------------------------------
- * Uniform (DeepWalk) walks.  Section 2.2: "random walks from each node".
+ * Uniform (DeepWalk) walks.  Section 2.2: every node is the source of walks.
  * walk[0] = start; each transition picks a uniformly random out-neighbour.
  * A node without out-neighbours ends the walk; the remaining entries are -1.
  * starts == NULL means start node = walk id mod n_nodes.
@@ -327,7 +327,7 @@ void gso_init_rows(const int64_t *rows, int64_t n_rows, int32_t d, uint64_t seed
 /* ------------------------------------------------------------------------
  * SGNS objective for one pair (c, o) with negatives n_1..n_K:
  *   loss = softplus(-<U_c,V_o>) + sum_k softplus(<U_c,V_nk>)
- * (Mikolov et al. 2013, the "skip-gram and negative sampling" of Section
+ * (Mikolov et al. 2013, the skip-gram objective with negative sampling named in Section
  * 2.2).  A negative equal to the pair's context is masked: no loss term and
  * no gradient.
  * ---------------------------------------------------------------------- */

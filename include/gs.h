@@ -423,6 +423,7 @@ typedef struct gs_epoch_stats {
     int64_t steps;            /* walk transitions taken                          */
     int64_t cap_hits;         /* node2vec rejection cap hits                     */
     int64_t batches;
+    int64_t masked_negs;      /* negatives dropped because they equal their context */
     float   ms_walk;          /* device time of the walk kernels                 */
     float   ms_sgns;          /* device time of the SGNS kernels                 */
     float   ms_total;

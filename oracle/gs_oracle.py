@@ -367,7 +367,7 @@ def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, sche
     nb_total = (total + batch_walks - 1) // batch_walks
     if num_batches is None:
         num_batches = nb_total - first_batch
-    loss_sum, pairs, steps = 0.0, 0, 0
+    loss_sum, pairs, steps, masked = 0.0, 0, 0, 0
     for b in range(first_batch, first_batch + num_batches):
         base = b * batch_walks
         n = min(batch_walks, total - base)
@@ -387,4 +387,5 @@ def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, sche
         loss_sum += ls
         pairs += pc
         steps += st
-    return {"loss_sum": loss_sum, "pairs": pairs, "steps": steps}
+        masked += int(((ng == o[:, None]) & (c >= 0)[:, None]).sum())   # negatives equal to their context
+    return {"loss_sum": loss_sum, "pairs": pairs, "steps": steps, "masked_negs": masked}

@@ -56,7 +56,8 @@ class SgnsConfig(ctypes.Structure):
 class EpochStats(ctypes.Structure):
     _fields_ = [
         ("loss_sum", ctypes.c_double), ("pairs", ctypes.c_int64), ("steps", ctypes.c_int64),
-        ("cap_hits", ctypes.c_int64), ("batches", ctypes.c_int64), ("ms_walk", ctypes.c_float),
+        ("cap_hits", ctypes.c_int64), ("batches", ctypes.c_int64), ("masked_negs", ctypes.c_int64),
+        ("ms_walk", ctypes.c_float),
         ("ms_sgns", ctypes.c_float), ("ms_total", ctypes.c_float),
     ]
 
@@ -340,6 +341,7 @@ class EpochResult:
     steps: int
     cap_hits: int
     batches: int
+    masked_negs: int
     ms_walk: float
     ms_sgns: float
     ms_total: float
@@ -364,7 +366,7 @@ def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len,
     _check(lib().gs_sgns_epoch(graph._h, _dev(alias, torch.int64, "alias", n_neg == 0),
                                _dev(w_in, tdt, "w_in"), _dev(w_out, tdt, "w_out"),
                                ctypes.byref(cfg), ctypes.byref(st), _stream()))
-    return EpochResult(st.loss_sum, st.pairs, st.steps, st.cap_hits, st.batches, st.ms_walk,
+    return EpochResult(st.loss_sum, st.pairs, st.steps, st.cap_hits, st.batches, st.masked_negs, st.ms_walk,
                        st.ms_sgns, st.ms_total)
 
 

@@ -31,12 +31,14 @@ gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_
 gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                     int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                     const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
-                    int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st);
+                    int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
+                    unsigned long long *masked = nullptr);
 
 gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                         const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
-                        int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st);
+                        int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
+                        unsigned long long *masked = nullptr);
 gs_status init_embeddings_f16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
                               cudaStream_t st);
 gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_out, int32_t *last_in,
@@ -556,6 +558,7 @@ struct EpochCounters {
     long long pairs;
     unsigned long long steps;
     unsigned long long caps;
+    unsigned long long masked;
 };
 
 namespace {
@@ -714,12 +717,12 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
                 EP_CALL(sgns_step_f16(d_w_in, d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
                                       cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
                                       cfg->seed, cfg->mode, &ctr->loss, (int64_t *)&ctr->pairs, nullptr,
-                                      nullptr, s_sgns));
+                                      nullptr, s_sgns, &ctr->masked));
             else
                 EP_CALL(sgns_step((float *)d_w_in, (float *)d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n,
                                   base, cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
                                   cfg->seed, cfg->mode, &ctr->loss, (int64_t *)&ctr->pairs, nullptr,
-                                  nullptr, s_sgns));
+                                  nullptr, s_sgns, &ctr->masked));
             t_sgns.stop(tk, s_sgns);
         }
         EP_TRY(cudaEventRecord(ev_sgns[buf], s_sgns));
@@ -735,6 +738,7 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
     h_out->pairs = (int64_t)host_ctr.pairs;
     h_out->steps = (int64_t)host_ctr.steps;
     h_out->cap_hits = (int64_t)host_ctr.caps;
+    h_out->masked_negs = (int64_t)host_ctr.masked;
     h_out->ms_walk = (float)t_walk.total_ms;
     h_out->ms_sgns = (float)t_sgns.total_ms;
     EP_TRY(cudaEventElapsedTime(&h_out->ms_total, ev_begin, ev_end));

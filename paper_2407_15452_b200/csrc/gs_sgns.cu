@@ -299,8 +299,8 @@ __device__ __forceinline__ void sum_over_groups(Row<FPL> &x)
 // ---------------------------------------------------------------- target list of one position
 // Slot layout: tgt[s * (1 + K) + 0] = context of slot s, tgt[s * (1 + K) + 1 + k] = negative k;
 // -1 where the pair does not exist or the negative equals the context (masked).
-// W points at the walk (global or shared), c = W[i] >= 0.  Returns the number of pairs
-// (identical on every lane).  dump_* (nullable) are this position's rows of the dump arrays.
+// W points at the walk (global or shared), c = W[i] >= 0.  Returns the number of pairs in the low
+// 8 bits and the number of masked negatives above them (identical on every lane).  dump_* (nullable) are this position's rows of the dump arrays.
 // flags & PAIR_FWD keeps only contexts that come later in the walk (edge sampling of LINE);
 // flags & PAIR_SHRINK draws the window of this position, w_i = 1 + mulhi(word, w) uniform on
 // 1..w (word2vec's shrinking window), and keeps the contexts within w_i.  Slots and the keying
@@ -318,11 +318,11 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
     int w_i = w;
     if (flags & PAIR_SHRINK) w_i = 1 + (int)__umulhi(draw(seed, id, (uint32_t)i, TAG_WINDOW, 0).x, (uint32_t)w);
     const int hp = K > 0 ? (K + 1) / 2 : 1;          // Philox blocks per slot (>= 1 work item)
-    int pairs = 0;
+    int pairs = 0, masked = 0;
     __syncwarp();                                    // earlier readers of tgt are done
     for (int it0 = 0; it0 < S * hp; it0 += 32) {
         const int it = it0 + lane;
-        bool valid = false;
+        bool valid = false, hid0 = false, hid1 = false;
         if (it < S * hp) {
             const int s = it / hp, m = it - s * hp;
             const int j = i - w + s + (s >= w ? 1 : 0);
@@ -354,15 +354,18 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
                     dump_negs[s * K + 2 * m] = n0;
                     if (two) dump_negs[s * K + 2 * m + 1] = n1;
                 }
+                hid0 = valid && n0 == ctx;
+                hid1 = valid && two && n1 == ctx;
                 tgt[s * T1 + 1 + 2 * m] = (n0 == ctx) ? -1 : n0;
                 if (two) tgt[s * T1 + 2 + 2 * m] = (n1 == ctx) ? -1 : n1;
             }
             valid = valid && m == 0;
         }
         pairs += __popc(__ballot_sync(0xffffffffu, valid));
+        masked += __popc(__ballot_sync(0xffffffffu, hid0)) + __popc(__ballot_sync(0xffffffffu, hid1));
     }
     __syncwarp();
-    return pairs;
+    return pairs | (masked << 8);
 }
 
 __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int lane,
@@ -380,7 +383,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     int32_t L, int32_t w, int32_t K, const uint64_t *__restrict__ alias,
                     uint32_t n_alias, float lr, uint64_t seed, double *loss_out,
                     unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs,
-                    unsigned long long *ticket, int fwd)
+                    unsigned long long *ticket, int fwd, unsigned long long *masked_out)
 {
     using G = RowGeom<DIM, T, NARROW>;
     constexpr int FPL = G::FPL, LPR = G::LPR, NG = G::NG;
@@ -392,7 +395,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     int32_t *W = smem + wi * (L + SL);
     int32_t *tgt = W + L;
     double loss_acc = 0.0;
-    unsigned long long pair_acc = 0;
+    unsigned long long pair_acc = 0, masked_acc = 0;
 
     // Walks differ in length (dead ends), so warps draw the next walk from a shared ticket
     // counter instead of taking a fixed share.
@@ -410,8 +413,10 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             int32_t *dp = dump_pairs ? dump_pairs + ((a * L + i) * S) * 2 : nullptr;
             int32_t *dn = dump_negs ? dump_negs + ((a * L + i) * S) * (int64_t)K : nullptr;
             if (c < 0) { dump_empty_position(S, K, lane, dp, dn); continue; }
-            const int pairs = build_targets(W, L, i, w, K, seed, id, alias, n_alias, c, tgt, lane,
-                                            dp, dn, fwd);
+            const int packed = build_targets(W, L, i, w, K, seed, id, alias, n_alias, c, tgt, lane,
+                                             dp, dn, fwd);
+            const int pairs = packed & 0xFF;
+            masked_acc += (unsigned long long)(packed >> 8);
             if (pairs == 0) continue;
             pair_acc += (unsigned long long)pairs;
             const Row<FPL> u = grow_load<DIM, T, NARROW>(w_in, c, sub);     // every group holds the center row
@@ -487,6 +492,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     if (lane == 0) {
         if (loss_out && pair_acc) atomicAdd(loss_out, loss_acc);
         if (pairs_out && pair_acc) atomicAdd(pairs_out, pair_acc);
+        if (masked_out && masked_acc) atomicAdd(masked_out, masked_acc);
     }
 }
 
@@ -532,10 +538,12 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out,
         float loss = 0.f;
         int pairs = 0;
         __syncwarp();
-        if (c >= 0)
-            pairs = build_targets(W, L, i, w, K, seed, (uint64_t)(walk_id_base + a), alias, n_alias,
-                                  c, tgt, lane, dp, dn, fwd);
-        else
+        int packed = 0;
+        if (c >= 0) {
+            packed = build_targets(W, L, i, w, K, seed, (uint64_t)(walk_id_base + a), alias, n_alias,
+                                   c, tgt, lane, dp, dn, fwd);
+            pairs = packed & 0xFF;
+        } else
             dump_empty_position(S, K, lane, dp, dn);
         if (pairs == 0) {
             for (int x = lane; x < SL; x += 32) {
@@ -590,7 +598,7 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out,
         if (MODE != 1 && grp == 0) grow_store_f32<DIM, T>(GU, pos, sub, acc);
         if (lane == 0) {
             if (MODE != 2) keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
-            if (MODE != 1) { loss_pos[pos] = (double)loss; pairs_pos[pos] = pairs; }
+            if (MODE != 1) { loss_pos[pos] = (double)loss; pairs_pos[pos] = packed; }   // pairs | masked << 8
         }
     }
 }
@@ -935,23 +943,33 @@ sgns_apply_in_kernel(T *__restrict__ w_in, const float *__restrict__ GU,
 // Fixed-order reduction of the per-position losses and pair counts (one block).
 __global__ void __launch_bounds__(1024)
 sgns_reduce_kernel(const double *__restrict__ loss_pos, const int32_t *__restrict__ pairs_pos,
-                   int64_t n_pos, double *loss_out, long long *pairs_out)
+                   int64_t n_pos, double *loss_out, long long *pairs_out, unsigned long long *masked_out)
 {
     __shared__ double sl[1024];
-    __shared__ long long sp[1024];
+    __shared__ long long sp[1024], sm[1024];
     double l = 0.0;
-    long long p = 0;
-    for (int64_t x = threadIdx.x; x < n_pos; x += 1024) { l += loss_pos[x]; p += pairs_pos[x]; }
+    long long p = 0, m = 0;
+    for (int64_t x = threadIdx.x; x < n_pos; x += 1024) {
+        l += loss_pos[x];
+        p += pairs_pos[x] & 0xFF;                        // pairs | masked negatives << 8
+        m += pairs_pos[x] >> 8;
+    }
     sl[threadIdx.x] = l;
     sp[threadIdx.x] = p;
+    sm[threadIdx.x] = m;
     __syncthreads();
     for (int o = 512; o > 0; o >>= 1) {
-        if (threadIdx.x < o) { sl[threadIdx.x] += sl[threadIdx.x + o]; sp[threadIdx.x] += sp[threadIdx.x + o]; }
+        if (threadIdx.x < o) {
+            sl[threadIdx.x] += sl[threadIdx.x + o];
+            sp[threadIdx.x] += sp[threadIdx.x + o];
+            sm[threadIdx.x] += sm[threadIdx.x + o];
+        }
         __syncthreads();
     }
     if (threadIdx.x == 0) {
         if (loss_out) *loss_out += sl[0];
         if (pairs_out) *pairs_out += sp[0];
+        if (masked_out) *masked_out += (unsigned long long)sm[0];
     }
 }
 
@@ -970,6 +988,7 @@ struct SgnsArgs {
     int64_t *pairs;
     int32_t *dump_pairs, *dump_negs;
     int fwd;                      // PAIR_* flags of build_targets
+    unsigned long long *masked;   // nullable: masked negatives are ADDED
 };
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
@@ -996,7 +1015,7 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
     kern<<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
         (T *)a.w_in, (T *)a.w_out, a.walks, a.n_walks, a.walk_id_base, a.L, a.w, a.K, a.alias,
         (uint32_t)a.n_nodes, a.lr, a.seed, a.loss, (unsigned long long *)a.pairs, a.dump_pairs,
-        a.dump_negs, ticket, a.fwd);
+        a.dump_negs, ticket, a.fwd, a.masked);
     GS_CUDA_TRY(cudaGetLastError());
     return GS_OK;
 }
@@ -1126,9 +1145,9 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
             w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr, ms_in);
         GS_CUDA_TRY(cudaGetLastError());
     }
-    if (a.loss || a.pairs) {
+    if (a.loss || a.pairs || a.masked) {
         sgns_reduce_kernel<<<1, 1024, 0, st>>>(loss_pos, pairs_pos, n_pos, a.loss,
-                                               (long long *)a.pairs);
+                                               (long long *)a.pairs, a.masked);
         GS_CUDA_TRY(cudaGetLastError());
     }
     return GS_OK;
@@ -1152,11 +1171,12 @@ static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
 gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                     int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                     const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
-                    int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st)
+                    int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
+                    unsigned long long *masked)
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode) };
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked };
     mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     switch (dim) {
         case 32: return run_mode<32, float>(a, mode, st);
@@ -1173,11 +1193,12 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
 gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                         const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
-                        int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st)
+                        int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
+                        unsigned long long *masked)
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode) };
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked };
     mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     switch (dim) {
         case 64: return run_mode<64, __half>(a, mode, st);
@@ -1197,7 +1218,7 @@ gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_ou
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, nullptr, nullptr, 0 };
+                   seed, loss, pairs, nullptr, nullptr, 0, nullptr };
     MomHost mom = { m_in, m_out, last_in, last_out, mu, iter, nullptr, nullptr, 0.f, 0.f, 0 };
     switch (dim) {
         case 32: return run_deterministic<32, float>(a, st, &mom);
@@ -1218,7 +1239,7 @@ gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, fl
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, nullptr, nullptr, pair_flags_of(pair_mode) };
+                   seed, loss, pairs, nullptr, nullptr, pair_flags_of(pair_mode), nullptr };
     MomHost mom = { m_in, m_out, nullptr, nullptr, b1, 0, v_in, v_out, b2, eps, step };
     switch (dim) {
         case 32: return run_deterministic<32, float>(a, st, &mom);
@@ -1354,9 +1375,9 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
             MomState{ nullptr, nullptr, 0.f, 0 });
         GS_CUDA_TRY(cudaGetLastError());
     }
-    if (a.loss || a.pairs) {
+    if (a.loss || a.pairs || a.masked) {
         sgns_reduce_kernel<<<1, 1024, 0, st>>>(loss_pos, pairs_pos, n_pos, a.loss,
-                                               (long long *)a.pairs);
+                                               (long long *)a.pairs, a.masked);
         GS_CUDA_TRY(cudaGetLastError());
     }
     return GS_OK;
@@ -1388,7 +1409,7 @@ extern "C" gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t 
     gs_status s = static_scratch_address(&scratch);
     if (s != GS_OK) return s;
     SgnsArgs a = { d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len, window,
-                   n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr, 0 };
+                   n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr, 0, nullptr };
     cudaStream_t st = (cudaStream_t)stream;
     switch (dim) {
         case 32: return run_deterministic_static<32>(a, scratch, st);

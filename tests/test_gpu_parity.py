@@ -414,6 +414,7 @@ def test_epoch_tiny_deepwalk_deterministic_matches_oracle(tiny):
                           batch_walks=512, seed=0, mode=B.GS_DETERMINISTIC,
                           lr_schedule=B.GS_LR_LINEAR)
     assert res.pairs == want["pairs"] and res.steps == want["steps"]
+    assert res.masked_negs == want["masked_negs"] > 0
     assert res.batches == (n + 511) // 512
     assert abs(res.loss_sum / res.pairs - want["loss_sum"] / want["pairs"]) <= LOSS_RTOL * want["loss_sum"] / want["pairs"]
     assert np.abs(w_in.cpu().numpy() - U).max() <= EMB_TOL
@@ -501,5 +502,12 @@ def test_epoch_node2vec_runs_and_counts_match_oracle(tiny):
                           mode=B.GS_DETERMINISTIC, walk_kind=B.GS_WALK_NODE2VEC, p=0.5, q=2.0,
                           num_batches=4)
     assert res.pairs == want["pairs"] and res.steps == want["steps"] and res.batches == 4
+    assert res.masked_negs == want["masked_negs"]
     assert abs(res.loss_sum - want["loss_sum"]) <= LOSS_RTOL * want["loss_sum"]
     assert np.abs(w_out.cpu().numpy() - V).max() <= EMB_TOL
+    # the integer statistics do not depend on the update mode
+    res2 = B.gs_sgns_epoch(G, alias_to_device(thr, alias), w_in, w_out, walks_per_node=1,
+                           walk_len=12, window=3, n_neg=3, lr0=0.025, batch_walks=1000, seed=1,
+                           mode=B.GS_HOGWILD, walk_kind=B.GS_WALK_NODE2VEC, p=0.5, q=2.0,
+                           num_batches=4)
+    assert (res2.pairs, res2.steps, res2.masked_negs) == (res.pairs, res.steps, res.masked_negs)

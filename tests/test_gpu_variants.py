@@ -125,6 +125,7 @@ def test_epoch_with_shuffle_subsampling_and_shrinking_matches_oracle(tiny):
                           batch_walks=512, seed=3, mode=B.GS_DETERMINISTIC | B.GS_WINDOW_SHRINK,
                           lr_schedule=B.GS_LR_LINEAR, keep_thr=thr_to_device(keep_thr), shuffle_epoch=4)
     assert res.pairs == want["pairs"] and res.steps == want["steps"]
+    assert res.masked_negs == want["masked_negs"]
     mean_o = want["loss_sum"] / want["pairs"]
     assert abs(res.loss_sum / res.pairs - mean_o) <= 1e-3 * mean_o
     assert np.abs(w_in.cpu().numpy() - U).max() <= EMB_TOL

@@ -53,7 +53,7 @@ def parse_args():
     ap.add_argument("--table-dtype", default="f32", choices=["f32", "f16"],
                     help="storage type of the embedding tables (arithmetic is fp32 either way)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cpu-sample-walks", type=int, default=8192)
+    ap.add_argument("--cpu-sample-walks", type=int, default=16384)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiling runs)")
     ap.add_argument("--no-walk-index", action="store_true",
@@ -239,8 +239,15 @@ def run_reference(args, wl):
 
 def walk_kernel_name(wl, indexed):
     if wl.walk_kind != "uniform":
-        return "node2vec_walk_kernel"
+        return "node2vec_thread_kernel"
     return "uniform_walk_index_kernel" if indexed else "uniform_walk_vec_kernel"
+
+
+def sync_step_launches(n_nodes, extra=0):
+    """Kernels of one synchronous batch: walks, coefficients, three per radix pass of 8 bits over
+    keys below 2 n_nodes, apply (output rows, fix-up, input rows), loss reduction."""
+    passes = ((2 * n_nodes).bit_length() + 7) // 8
+    return 1 + 1 + 3 * passes + 3 + 1 + extra
 
 
 def parse_variants(args):
@@ -392,7 +399,8 @@ def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
         "metric": METRIC, "value": pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "gpu_launches": None, "clocks": clocks, "mean_loss": loss.item() / max(pairs, 1),
+        "gpu_launches": sync_step_launches(n, 0 if adam else 2) * args.steps,   # momentum: keys pass + catch-up
+        "clocks": clocks, "mean_loss": loss.item() / max(pairs, 1),
         "config": {"workload": wl.name, "mode": args.mode, "momentum": mu, "lr": lr, "batch_walks": bw,
                    "walk_len": wl.walk_len, "window": wl.window, "n_neg": wl.n_neg, "dim": wl.dim,
                    "scale": args.scale, **info},
@@ -466,8 +474,11 @@ def run_ours(args, wl):
         return replicas.batch_of(step, rank, world, nb_total)
 
     # ---- device-resident timing -------------------------------------------------------
-    for s in range(args.warmup):
-        B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=batch_of(s), num_batches=1, **ekw)
+    # warm-up: one call per batch, so the walk kernel runs alone here (inside a multi-batch call it
+    # shares the GPU with the update of the previous batch); its own figures are taken from these
+    warm = [B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=batch_of(s), num_batches=1, **ekw)
+            for s in range(args.warmup)]
+    warm = warm[1:] if len(warm) > 1 else warm
     sampler = ClockSampler(local)
     barrier()
     if rank == 0:
@@ -477,15 +488,20 @@ def run_ours(args, wl):
     loss = 0.0
     ms_walk = ms_sgns = 0.0
     ev0.record()
-    for s in range(args.steps):
-        b = batch_of(args.warmup + s)
-        r = B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=b, num_batches=1, **ekw)
+    # One replica takes consecutive mini-batches: the K timed steps are ONE call of the epoch
+    # driver over K batches, as a user runs it (walk generation of batch b+1 then overlaps the
+    # update of batch b).  Several replicas interleave their batches, so they call per step.
+    one_call = world == 1 and args.warmup + args.steps <= nb_total
+    calls = [(args.warmup, args.steps)] if one_call else \
+            [(batch_of(args.warmup + s), 1) for s in range(args.steps)]
+    for b, nb in calls:
+        r = B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=b, num_batches=nb, **ekw)
         pairs += r.pairs
         steps += r.steps
         loss += r.loss_sum
         ms_walk += r.ms_walk
         ms_sgns += r.ms_sgns
-        walks_done += min(bw, total_walks - b * bw)
+        walks_done += sum(min(bw, total_walks - x * bw) for x in range(b, b + nb))
     ev1.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
@@ -542,9 +558,13 @@ def run_ours(args, wl):
         sgns_ms = ms_sgns / launches
         achieved = sgns_bytes / (sgns_ms * 1e-3) / 1e9
         indexed = "walk_index_bytes" in info
-        wbytes = walk_bytes(steps, wl.offsets64, indexed) / launches
-        gbytes = walk_granule_bytes(steps, indexed) / launches
-        walk_ms = ms_walk / launches
+        if one_call and warm:                          # walk kernel alone: the warm-up calls
+            w_steps, w_ms, w_n = sum(r.steps for r in warm), sum(r.ms_walk for r in warm), len(warm)
+        else:
+            w_steps, w_ms, w_n = steps, ms_walk, launches
+        wbytes = walk_bytes(w_steps, wl.offsets64, indexed) / w_n
+        gbytes = walk_granule_bytes(w_steps, indexed) / w_n
+        walk_ms = w_ms / w_n
         per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if (mode & 0xFF) and not f16 else None
         traffic = per_pair * pairs / launches if per_pair else None
         out = {
@@ -557,8 +577,11 @@ def run_ours(args, wl):
                        "walk_kind": wl.walk_kind, "walk_len": wl.walk_len, "window": wl.window,
                        "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale, "variants": sorted(variants),
                        "l2": "tables (2 x n x dim x 4 B) and CSR far exceed the 126 MB L2; no flush",
+                       "timed_region": "one gs_sgns_epoch call over the K batches" if one_call else
+                                       "one gs_sgns_epoch call per batch",
                        "multi_gpu": "replicas only", **info},
-            "gpu_launches": 2 * args.steps,
+            "gpu_launches": ((2 if (mode & 0xFF) else sync_step_launches(n))
+                             + len(variants & {"shuffle", "subsample"})) * args.steps,
             "mean_loss": loss / max(pairs, 1),
             "walk_steps_per_s": steps_all / (ms * 1e-3),
             "clocks": clocks,
@@ -570,7 +593,7 @@ def run_ours(args, wl):
                          "peak_kind": f"of {peak_kind}", "traffic": traffic,
                          "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (ms_sgns * 1e-3)},
             "walk": {"kernel": walk_kernel_name(wl, indexed),
-                     "walk_steps_per_s_kernel": steps / (ms_walk * 1e-3), "ms_per_launch": walk_ms,
+                     "walk_steps_per_s_kernel": w_steps / (w_ms * 1e-3), "ms_per_launch": walk_ms,
                      "payload_gbs": wbytes / (walk_ms * 1e-3) / 1e9,
                      "payload_frac": wbytes / (walk_ms * 1e-3) / 1e9 / peak,
                      "granule_gbs": gbytes / (walk_ms * 1e-3) / 1e9,

@@ -127,7 +127,8 @@ GS_API gs_status gs_init_embeddings(float *d_w_in, float *d_w_out, int64_t n_nod
 /* ---------------------------------------------------------------- walks */
 /*
  * DeepWalk walks (Section 2.2: every node is the source of random walks).
- *   d_starts     : n_walks start nodes, or NULL for start = walk id mod n_nodes
+ *   d_starts     : n_walks start nodes, or NULL for start = walk id mod n_nodes;
+ *                  a start outside [0, n_nodes) gives a walk of -1 entries
  *   walk id      : walk_id_base + index; selects the random stream
  *   walk_len     : number of NODES per walk (Section 3.2 counts a batch as
  *                  B x walk_len nodes, sources included); >= 1
@@ -214,7 +215,8 @@ GS_API gs_status gs_probe_random_reads(const gs_graph *g, int64_t n_reads, int64
  *
  *   d_w_in, d_w_out : [n_nodes][dim] fp32 row-major, 16-byte aligned,
  *                     dim in {32, 64, 128, 256}
- *   d_walks         : [n_walks][walk_len] int32 (as written by the walk calls)
+ *   d_walks         : [n_walks][walk_len] int32 (as written by the walk calls); an
+ *                     entry outside [0, n_nodes) counts as absent, like -1
  *   d_loss_sum      : the batch's summed loss is ADDED (nullable)
  *   d_pair_count    : the number of pairs is ADDED (nullable)
  *   d_pairs_dump    : nullable; [n_walks][walk_len][2*window][2] int32
@@ -366,11 +368,12 @@ GS_API gs_status gs_build_keep_thresholds(const double *h_weights, int64_t n, do
  * Kept entries move to the front of the walk in their order, the rest of the row becomes -1,
  * so the windows of gs_sgns_step then span the dropped occurrences.  d_walks_out may be
  * d_walks (in place).  d_kept (nullable): the number of kept entries is ADDED.
- * Node ids in d_walks must be below the length of d_keep_thr (not checked).
+ * d_keep_thr has n_nodes entries; an entry of d_walks outside [0, n_nodes) is dropped.
  */
 GS_API gs_status gs_subsample_walks(const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
-                                    int32_t walk_len, const uint32_t *d_keep_thr, uint64_t seed,
-                                    int32_t *d_walks_out, uint64_t *d_kept, void *stream);
+                                    int32_t walk_len, const uint32_t *d_keep_thr, int64_t n_nodes,
+                                    uint64_t seed, int32_t *d_walks_out, uint64_t *d_kept,
+                                    void *stream);
 
 /*
  * Start nodes in shuffled order: d_starts_out[i] = P((walk_id_first + i) mod n_nodes), where P

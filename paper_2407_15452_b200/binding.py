@@ -317,7 +317,8 @@ def gs_subsample_walks(walks, walk_id_base: int, keep_thr, seed: int, out=None, 
     _check(lib().gs_subsample_walks(
         _dev(walks, torch.int32, "walks", n_walks == 0), ctypes.c_int64(n_walks),
         ctypes.c_int64(walk_id_base), ctypes.c_int32(walk_len),
-        _dev(keep_thr, torch.int32, "keep_thr", n_walks == 0), ctypes.c_uint64(seed),
+        _dev(keep_thr, torch.int32, "keep_thr", n_walks == 0),
+        ctypes.c_int64(keep_thr.numel() if keep_thr is not None else 1), ctypes.c_uint64(seed),
         _dev(out, torch.int32, "out", n_walks == 0), _dev(kept, torch.int64, "kept", True), _stream()))
     return out
 

@@ -54,7 +54,7 @@ gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, fl
                          const uint64_t *alias, float lr, float b1, float b2, float eps, int64_t step,
                          uint64_t seed, int32_t pair_mode, double *loss, int64_t *pairs, cudaStream_t st);
 gs_status launch_subsample_walks(const int32_t *walks, int64_t n_walks, int64_t base, int32_t L,
-                                 const uint32_t *keep_thr, uint64_t seed, int32_t *out,
+                                 const uint32_t *keep_thr, int64_t n_nodes, uint64_t seed, int32_t *out,
                                  unsigned long long *kept, cudaStream_t st);
 gs_status random_read_probe(const gs_graph *g, int64_t n_reads, float *ms_out, cudaStream_t st);
 gs_status launch_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epoch, int64_t first,
@@ -532,13 +532,14 @@ gs_status gs_build_keep_thresholds(const double *h_weights, int64_t n, double t,
 }
 
 gs_status gs_subsample_walks(const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
-                             int32_t walk_len, const uint32_t *d_keep_thr, uint64_t seed,
-                             int32_t *d_walks_out, uint64_t *d_kept, void *stream)
+                             int32_t walk_len, const uint32_t *d_keep_thr, int64_t n_nodes,
+                             uint64_t seed, int32_t *d_walks_out, uint64_t *d_kept, void *stream)
 {
     if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
     if (walk_len < 1 || walk_len > 1024) { set_error("walk_len %d outside [1, 1024]", walk_len); return GS_ERR_UNSUPPORTED; }
     if (n_walks > 0 && (!d_walks || !d_walks_out || !d_keep_thr)) return invalid("null pointer");
-    return launch_subsample_walks(d_walks, n_walks, walk_id_base, walk_len, d_keep_thr, seed,
+    return launch_subsample_walks(d_walks, n_walks, walk_id_base, walk_len, d_keep_thr, n_nodes, seed,
                                   d_walks_out, (unsigned long long *)d_kept, (cudaStream_t)stream);
 }
 
@@ -701,7 +702,7 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
                                               &ctr->steps, &ctr->caps, s_walk));
             if (cfg->d_keep_thr)
                 EP_CALL(launch_subsample_walks(wbuf[buf], n, base, cfg->walk_len, cfg->d_keep_thr,
-                                               cfg->seed, wbuf[buf], nullptr, s_walk));
+                                               g->n_nodes, cfg->seed, wbuf[buf], nullptr, s_walk));
             t_walk.stop(tk, s_walk);
         }
         EP_TRY(cudaEventRecord(ev_walk[buf], s_walk));

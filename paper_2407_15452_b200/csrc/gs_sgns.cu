@@ -327,7 +327,8 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
             const int s = it / hp, m = it - s * hp;
             const int j = i - w + s + (s >= w ? 1 : 0);
             const bool in_window = j - i <= w_i && i - j <= w_i && !(fwd && s < w);   // fwd: only j > i
-            const int32_t ctx = (j >= 0 && j < L && in_window) ? W[j] : -1;
+            int32_t ctx = (j >= 0 && j < L && in_window) ? W[j] : -1;
+            if ((uint32_t)ctx >= n_alias) ctx = -1;        // absent, or not a node of the tables
             valid = ctx >= 0;
             if (m == 0) {
                 tgt[s * T1] = ctx;
@@ -344,10 +345,12 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
                     const uint32_t j0 = __umulhi(r.x, n_alias);
                     const uint64_t e0 = ld_random(alias + j0);
                     n0 = r.y < (uint32_t)e0 ? (int32_t)j0 : (int32_t)(e0 >> 32);
+                    if ((uint32_t)n0 >= n_alias) n0 = -1;      // a table entry that names no node
                     if (two) {
                         const uint32_t j1 = __umulhi(r.z, n_alias);
                         const uint64_t e1 = ld_random(alias + j1);
                         n1 = r.w < (uint32_t)e1 ? (int32_t)j1 : (int32_t)(e1 >> 32);
+                        if ((uint32_t)n1 >= n_alias) n1 = -1;
                     }
                 }
                 if (dump_negs) {
@@ -412,7 +415,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             const int32_t c = W[i];
             int32_t *dp = dump_pairs ? dump_pairs + ((a * L + i) * S) * 2 : nullptr;
             int32_t *dn = dump_negs ? dump_negs + ((a * L + i) * S) * (int64_t)K : nullptr;
-            if (c < 0) { dump_empty_position(S, K, lane, dp, dn); continue; }
+            if ((uint32_t)c >= n_alias) { dump_empty_position(S, K, lane, dp, dn); continue; }   // -1 or no such row
             const int packed = build_targets(W, L, i, w, K, seed, id, alias, n_alias, c, tgt, lane,
                                              dp, dn, fwd);
             const int pairs = packed & 0xFF;
@@ -539,7 +542,7 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out,
         int pairs = 0;
         __syncwarp();
         int packed = 0;
-        if (c >= 0) {
+        if ((uint32_t)c < n_nodes) {                   // -1, or an id outside the tables: no pairs
             packed = build_targets(W, L, i, w, K, seed, (uint64_t)(walk_id_base + a), alias, n_alias,
                                    c, tgt, lane, dp, dn, fwd);
             pairs = packed & 0xFF;

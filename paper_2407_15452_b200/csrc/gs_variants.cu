@@ -12,8 +12,8 @@ namespace gs {
 // before it is written, so `out` may be the same buffer as `walks`.
 __global__ void __launch_bounds__(256)
 subsample_walks_kernel(const int32_t *walks, int64_t n_walks, int64_t walk_id_base, int32_t L,
-                       const uint32_t *__restrict__ keep_thr, uint64_t seed, int32_t *out,
-                       unsigned long long *kept_out)
+                       const uint32_t *__restrict__ keep_thr, uint32_t n_nodes, uint64_t seed,
+                       int32_t *out, unsigned long long *kept_out)
 {
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -27,7 +27,7 @@ subsample_walks_kernel(const int32_t *walks, int64_t n_walks, int64_t walk_id_ba
         for (int t0 = 0; t0 < L; t0 += 32) {
             const int t = t0 + lane;
             const int32_t v = t < L ? W[t] : -1;
-            bool keep = v >= 0;
+            bool keep = (uint32_t)v < n_nodes;              // -1 and ids without a threshold are dropped
             if (keep) {
                 const uint32_t thr = ld_random(reinterpret_cast<const int32_t *>(keep_thr) + v);
                 if (thr != 0xFFFFFFFFu)
@@ -47,15 +47,15 @@ subsample_walks_kernel(const int32_t *walks, int64_t n_walks, int64_t walk_id_ba
 }
 
 gs_status launch_subsample_walks(const int32_t *walks, int64_t n_walks, int64_t base, int32_t L,
-                                 const uint32_t *keep_thr, uint64_t seed, int32_t *out,
+                                 const uint32_t *keep_thr, int64_t n_nodes, uint64_t seed, int32_t *out,
                                  unsigned long long *kept, cudaStream_t st)
 {
     if (n_walks == 0) return GS_OK;
     int64_t blocks = (n_walks + 7) / 8;
     const int64_t cap = (int64_t)sm_count() * 8 * 4;
     if (blocks > cap) blocks = cap;
-    subsample_walks_kernel<<<(unsigned)blocks, 256, 0, st>>>(walks, n_walks, base, L, keep_thr, seed,
-                                                           out, kept);
+    subsample_walks_kernel<<<(unsigned)blocks, 256, 0, st>>>(walks, n_walks, base, L, keep_thr,
+                                                           (uint32_t)n_nodes, seed, out, kept);
     GS_CUDA_TRY(cudaGetLastError());
     return GS_OK;
 }

@@ -177,10 +177,11 @@ uniform_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ co
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
+        const bool bad = (uint64_t)(uint32_t)cur >= (uint64_t)n_nodes;   // start outside the graph: empty walk
         int32_t *W = walks + i * (int64_t)L;
-        W[0] = cur;
+        W[0] = bad ? -1 : cur;
         int32_t t = 0;
-        for (; t + 1 < L; ++t) {
+        for (; !bad && t + 1 < L; ++t) {
             const int64_t o0 = ld_random(off + cur), o1 = ld_random(off + cur + 1);
             const uint32_t deg = (uint32_t)(o1 - o0);
             if (deg == 0) break;
@@ -214,7 +215,7 @@ uniform_walk_vec_kernel(const OffT *__restrict__ off, const int32_t *__restrict_
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
-        bool alive = true;
+        bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
         int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
         int4 pend = make_int4(0, 0, 0, 0);
         for (int q = 0; q < quads; ++q) {
@@ -296,9 +297,13 @@ uniform_walk_index_kernel(const OffT *__restrict__ off, const int4 *__restrict__
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
-        int64_t o0 = ld_random(off + cur);
-        uint32_t deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
-        bool alive = true;
+        bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
+        int64_t o0 = 0;
+        uint32_t deg = 0;
+        if (alive) {
+            o0 = ld_random(off + cur);
+            deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
+        }
         int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
         int4 pend = make_int4(0, 0, 0, 0);
         for (int q = 0; q < quads; ++q) {
@@ -404,9 +409,10 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
         int32_t prev = -1;
         int64_t p0 = 0, p1 = 0;                     // adjacency range of prev
         int32_t *W = walks + i * (int64_t)L;
-        if (sub == 0) W[0] = cur;
+        const bool bad = (uint64_t)(uint32_t)cur >= (uint64_t)n_nodes;   // same for the whole group
+        if (sub == 0) W[0] = bad ? -1 : cur;
         int32_t t = 0;
-        for (; t + 1 < L; ++t) {
+        for (; !bad && t + 1 < L; ++t) {
             const int64_t o0 = ld_random(off + cur), o1 = ld_random(off + cur + 1);
             const uint32_t deg = (uint32_t)(o1 - o0);
             if (deg == 0) break;
@@ -478,11 +484,15 @@ node2vec_thread_kernel(const OffT *__restrict__ off, const int32_t *__restrict__
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
-        int64_t o0 = ld_random(off + cur);
-        uint32_t deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
+        bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
+        int64_t o0 = 0;
+        uint32_t deg = 0;
+        if (alive) {
+            o0 = ld_random(off + cur);
+            deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
+        }
         int32_t prev = -1;
         int64_t p0 = 0, p1 = 0;
-        bool alive = true;
         int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
         int4 pend = make_int4(0, 0, 0, 0);
         for (int q = 0; q < quads; ++q) {

@@ -511,3 +511,59 @@ def test_epoch_node2vec_runs_and_counts_match_oracle(tiny):
                            mode=B.GS_HOGWILD, walk_kind=B.GS_WALK_NODE2VEC, p=0.5, q=2.0,
                            num_batches=4)
     assert (res2.pairs, res2.steps, res2.masked_negs) == (res.pairs, res.steps, res.masked_negs)
+
+
+# ---------------------------------------------------------------- ids outside the graph
+def test_out_of_range_ids_count_as_absent_instead_of_faulting(tiny):
+    # The library never dereferences an id it has not range-checked: a start node, a walk entry or
+    # an alias-table cell outside [0, n_nodes) is treated like -1.
+    wl, g, off, col, thr, alias = tiny
+    n = g.n_nodes
+    starts = np.array([3, -5, n, 2**31 - 1, 7, n + 1000, 0, n - 1] * 40, dtype=np.int32)
+    ok = (starts >= 0) & (starts < n)
+    want, _ = O.uniform_walks(off, col, np.where(ok, starts, 0).astype(np.int32), len(starts), 9, 16, 2)
+    want[~ok] = -1
+    sd = torch.from_numpy(starts).to(DEV)
+    for flags in (B.GS_VALIDATE | B.GS_REQUIRE_SORTED, B.GS_BUILD_WALK_INDEX | B.GS_REQUIRE_SORTED):
+        G = load(g, flags=flags)
+        assert np.array_equal(B.gs_random_walks(G, sd, len(starts), 9, 16, 2).cpu().numpy(), want)
+        assert np.array_equal(B.gs_random_walks(G, sd, len(starts), 9, 13, 2).cpu().numpy()[~ok],
+                              np.full((int((~ok).sum()), 13), -1))
+        want2, _, _ = O.node2vec_walks(off, col, np.where(ok, starts, 0).astype(np.int32), len(starts), 9, 16,
+                                       2, 0.5, 2.0)
+        want2[~ok] = -1
+        for lanes in (1, 4, 32):
+            B.gs_tune_node2vec_group(lanes)
+            got = B.gs_node2vec_walks(G, sd, len(starts), 9, 16, 2, 0.5, 2.0)
+            assert np.array_equal(got.cpu().numpy(), want2)
+        B.gs_tune_node2vec_group(1)
+    # walk entries outside the tables behave like -1 in the update
+    walks, _ = O.uniform_walks(off, col, None, 200, 0, 12, 5)
+    dirty = walks.copy()
+    rng = np.random.default_rng(0)
+    hit = rng.random(walks.shape) < 0.1
+    dirty[hit] = rng.choice([n, n + 7, 2**31 - 1, -9], size=int(hit.sum()))
+    clean = np.where(hit, -1, walks).astype(np.int32)
+    a_dev = alias_to_device(thr, alias)
+    w_in0, w_out0 = random_tables(n, 64, 4)
+    res = []
+    for wk in (clean, dirty):
+        w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+        loss, cnt, pd, nd = run_step(w_in, w_out, torch.from_numpy(wk).to(DEV), 0, 3, 4, a_dev, 0.025, 5,
+                                     B.GS_DETERMINISTIC)
+        res.append((loss, cnt, pd, nd, w_in, w_out))
+    assert res[0][0] == res[1][0] and res[0][1] == res[1][1] > 0
+    for x, y in zip(res[0][2:], res[1][2:]):
+        assert torch.equal(x, y)
+    w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+    loss, cnt, _, _ = run_step(w_in, w_out, torch.from_numpy(dirty).to(DEV), 0, 3, 4, a_dev, 0.025, 5,
+                               B.GS_HOGWILD, dump=False)
+    assert cnt == res[0][1] and np.isfinite(loss) and torch.isfinite(w_out).all()
+    # an alias table whose cells point outside the graph yields no such negative
+    bad_alias = alias.copy()
+    bad_alias[::3] = n + 5
+    w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+    loss, cnt, pd, nd = run_step(w_in, w_out, torch.from_numpy(clean).to(DEV), 0, 3, 4,
+                                 alias_to_device(thr, bad_alias), 0.025, 5, B.GS_DETERMINISTIC)
+    ndn = nd.cpu().numpy()
+    assert ndn.max() < n and cnt == res[0][1] and torch.isfinite(w_out).all()

@@ -217,3 +217,16 @@ def test_random_read_probe_reports_a_rate_and_needs_the_walk_index(tiny):
     with pytest.raises(B.GsError) as e:
         B.gs_probe_random_reads(G2, 1 << 20)
     assert e.value.status == -1
+
+
+def test_subsampling_drops_entries_outside_the_threshold_table(tiny):
+    _, g, off, col, _, _ = tiny
+    n = g.n_nodes
+    keep_thr = np.full(n, 0xFFFFFFFF, dtype=np.uint32)
+    walks, _ = O.uniform_walks(off, col, None, 300, 0, 20, 1)
+    dirty = walks.copy()
+    hit = np.random.default_rng(2).random(walks.shape) < 0.15
+    dirty[hit] = n + 3
+    want, _ = O.subsample_walks(np.where(hit, -1, walks).astype(np.int32), 0, keep_thr, 1)
+    got = B.gs_subsample_walks(torch.from_numpy(dirty).to(DEV), 0, thr_to_device(keep_thr), 1)
+    assert np.array_equal(got.cpu().numpy(), want)

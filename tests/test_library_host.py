@@ -96,7 +96,8 @@ def test_argument_errors_are_status_codes_without_touching_a_gpu(lib):
                                 ctypes.c_int64(0), ctypes.c_int64(4), ctypes.c_void_p(16), None)
     assert st == -1 and b"n_nodes" in lib.gs_last_error()
     st = lib.gs_subsample_walks(ctypes.c_void_p(16), ctypes.c_int64(2), ctypes.c_int64(0), 2000,
-                                ctypes.c_void_p(16), ctypes.c_uint64(0), ctypes.c_void_p(16), None, None)
+                                ctypes.c_void_p(16), ctypes.c_int64(5), ctypes.c_uint64(0),
+                                ctypes.c_void_p(16), None, None)
     assert st == -6 and b"walk_len" in lib.gs_last_error()
     p16 = ctypes.c_void_p(256)
     st = lib.gs_sgns_step_adam(p16, p16, p16, p16, p16, p16, ctypes.c_int64(10), 128, p16,

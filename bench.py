@@ -58,6 +58,10 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiling runs)")
     ap.add_argument("--no-walk-index", action="store_true",
                     help="walk over the plain CSR (two random reads per transition)")
+    ap.add_argument("--no-edge-set", action="store_true",
+                    help="node2vec: membership in adj(prev) by binary search instead of the hashed edge set")
+    ap.add_argument("--n2v-lanes", type=int, default=None,
+                    help="node2vec kernel: 0 flattened loop, 1 nested loops, 2..32 lanes per walk")
     ap.add_argument("--stage", default="all", choices=["all", "walks"],
                     help="'walks' times the walk sampler alone (no tables are allocated)")
     return ap.parse_args()
@@ -434,7 +438,12 @@ def run_ours(args, wl):
     if not args.no_walk_index:
         flags |= B.GS_BUILD_WALK_INDEX                  # 16 B per CSR entry, one read per transition
         info["walk_index_bytes"] = 16 * g.n_edges
+    if wl.walk_kind != "uniform" and not args.no_edge_set:
+        info["edge_set"] = True
+        flags |= B.GS_BUILD_EDGE_SET                    # hashed "is x a neighbour of prev" for node2vec
     G = B.gs_graph_load_csr(g.offsets, g.cols, flags)
+    if args.n2v_lanes is not None:
+        B.gs_tune_node2vec_group(args.n2v_lanes)
     if args.stage == "walks":
         return run_walks_only(args, wl, g, G, info, dev)
     alias = torch.from_numpy(table.view(np.int64)).to(dev)

@@ -69,6 +69,7 @@ typedef struct gs_graph gs_graph;
 #define GS_VALIDATE        1u   /* check offsets and column range on the device    */
 #define GS_REQUIRE_SORTED  2u   /* additionally require strictly increasing rows   */
 #define GS_BUILD_WALK_INDEX 4u  /* build the per-entry walk index (implies GS_VALIDATE) */
+#define GS_BUILD_EDGE_SET  8u   /* build the hashed edge set for node2vec (implies GS_VALIDATE) */
 
 /*
  * Wraps a CSR graph that already lives in device memory (the whole topology
@@ -85,6 +86,10 @@ typedef struct gs_graph gs_graph;
  * fit): entry e records cols[e] with that node's degree and offset, so that a
  * uniform-walk transition needs one random read instead of two.  Walks are
  * identical with or without the index.
+ * With GS_BUILD_EDGE_SET the handle also owns a hash table of all CSR entries
+ * (8 bytes per slot, 2 to 4 slots per entry; GS_ERR_OOM if it does not fit):
+ * node2vec then decides "is x a neighbour of prev" with one or two reads instead
+ * of a binary search over the row of prev.  Walks are identical with or without it.
  */
 GS_API gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges,
                             const void *d_offsets, int32_t offsets_are_64bit,
@@ -448,11 +453,12 @@ GS_API gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias,
 GS_API gs_status gs_release_workspace(void);
 
 /*
- * Tuning knob: lanes that cooperate on one node2vec walk (1, 2, 4, 8 or 32;
- * default 1, the fastest measured: 4.9e9 transitions/s against 1.9e9 with a
- * whole warp per walk on the 4M-node workload).  With more than one lane, lane
- * k of a group evaluates rejection round base + k and the first accepted round
- * wins, so walks do not depend on this setting.
+ * Tuning knob: which node2vec kernel runs.  0 (default): one lane per walk, rejection rounds and
+ * transitions flattened into one loop, so a lane that has accepted starts its next transition
+ * without waiting for its warp (1.0e10 transitions/s on the 4M-node workload with the edge set).
+ * 1: one lane per walk, nested loops (7.2e9).  2, 4, 8, 32: that many lanes cooperate on a walk,
+ * lane k of a group evaluates rejection round base + k and the first accepted round wins
+ * (4.3e9 ... 1.9e9 without the edge set).  Walks do not depend on this setting.
  */
 GS_API gs_status gs_tune_node2vec_group(int32_t lanes);
 

@@ -18,7 +18,7 @@ import torch
 _LIB_PATH = Path(__file__).resolve().parent / "libgs_b200.so"
 _lib = None
 
-GS_VALIDATE, GS_REQUIRE_SORTED, GS_BUILD_WALK_INDEX = 1, 2, 4
+GS_VALIDATE, GS_REQUIRE_SORTED, GS_BUILD_WALK_INDEX, GS_BUILD_EDGE_SET = 1, 2, 4, 8
 GS_DETERMINISTIC, GS_HOGWILD, GS_HOGWILD_RED = 0, 1, 2
 GS_PAIRS_FORWARD_ONLY = 0x100
 GS_WINDOW_SHRINK = 0x200

@@ -18,6 +18,8 @@ namespace gs {
 gs_status validate_csr(const gs_graph *g, bool check_sorted, cudaStream_t st, int64_t *bad_row,
                        int64_t *unsorted_row, int64_t *max_degree, bool *ends_bad);
 gs_status build_walk_index(const gs_graph *g, int4 *rec, cudaStream_t st);
+gs_status build_edge_hash(const gs_graph *g, unsigned long long *table, unsigned long long mask,
+                          cudaStream_t st);
 gs_status init_embeddings(float *w_in, float *w_out, int64_t n, int32_t dim, uint64_t seed,
                           cudaStream_t st);
 gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
@@ -181,8 +183,8 @@ gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offs
     if (n_edges > 0 && !d_cols) return invalid("d_cols is NULL");
     if (!offsets_are_64bit && n_edges >= ((int64_t)1 << 31))
         return invalid("int32 offsets cannot address 2^31 or more edges");
-    if (flags & ~(GS_VALIDATE | GS_REQUIRE_SORTED | GS_BUILD_WALK_INDEX)) return invalid("unknown flag");
-    if (flags & GS_BUILD_WALK_INDEX) flags |= GS_VALIDATE;     // the index is built from checked data
+    if (flags & ~(GS_VALIDATE | GS_REQUIRE_SORTED | GS_BUILD_WALK_INDEX | GS_BUILD_EDGE_SET)) return invalid("unknown flag");
+    if (flags & (GS_BUILD_WALK_INDEX | GS_BUILD_EDGE_SET)) flags |= GS_VALIDATE;   // built from checked data
     gs_graph *g = new (std::nothrow) gs_graph;
     if (!g) { set_error("out of host memory"); return GS_ERR_OOM; }
     g->n_nodes = n_nodes;
@@ -194,6 +196,8 @@ gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offs
     g->max_degree = -1;
     g->device = 0;
     g->d_edge_rec = nullptr;
+    g->d_edge_hash = nullptr;
+    g->hash_mask = 0;
     cudaGetDevice(&g->device);
     if (flags & (GS_VALIDATE | GS_REQUIRE_SORTED)) {
         int64_t bad = -1, unsorted = -1, maxdeg = 0;
@@ -235,6 +239,23 @@ gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offs
         gs_status s = build_walk_index(g, g->d_edge_rec, (cudaStream_t)stream);
         if (s != GS_OK) { cudaFree(rec); delete g; return s; }
     }
+    if ((flags & GS_BUILD_EDGE_SET) && n_edges > 0) {
+        unsigned long long cap = 1024;
+        while (cap < 2ull * (unsigned long long)n_edges) cap <<= 1;      // at most half full
+        void *tab = nullptr;
+        cudaError_t e = cudaMalloc(&tab, sizeof(unsigned long long) * (size_t)cap);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            if (g->d_edge_rec) cudaFree(g->d_edge_rec);
+            delete g;
+            set_error("edge set of %llu x 8 bytes could not be allocated: %s", cap, cudaGetErrorString(e));
+            return GS_ERR_OOM;
+        }
+        g->d_edge_hash = (unsigned long long *)tab;
+        g->hash_mask = cap - 1;
+        gs_status s = build_edge_hash(g, g->d_edge_hash, g->hash_mask, (cudaStream_t)stream);
+        if (s != GS_OK) { cudaFree(tab); if (g->d_edge_rec) cudaFree(g->d_edge_rec); delete g; return s; }
+    }
     *out = g;
     return GS_OK;
 }
@@ -242,6 +263,7 @@ gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges, const void *d_offs
 void gs_graph_free(gs_graph *g)
 {
     if (!g) return;
+    if (g->d_edge_hash) cudaFree(g->d_edge_hash);
     if (g->d_edge_rec) cudaFree(g->d_edge_rec);          // waits for kernels that may still read it
     delete g;
 }
@@ -330,7 +352,7 @@ gs_status gs_random_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_
                                 (unsigned long long *)d_steps, (cudaStream_t)stream);
 }
 
-static int g_n2v_group = 1;   // lanes per walk in the node2vec sampler (1 measured fastest)
+static int g_n2v_group = 0;   // node2vec kernel: 0 = one lane per walk, flattened loop (measured fastest)
 
 gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_walks,
                             int64_t walk_id_base, int32_t walk_len, uint64_t seed, double p,
@@ -351,12 +373,12 @@ gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts, int64_t 
                                  (cudaStream_t)stream);
 }
 
-// Tuning knob used by the benchmarks: lanes per walk (1, 2, 4, 8, 32) of the node2vec sampler.
+// Tuning knob used by the benchmarks: kernel / lanes per walk (0, 1, 2, 4, 8, 32) of the node2vec sampler.
 // Results do not depend on it.
 gs_status gs_tune_node2vec_group(int32_t lanes)
 {
-    if (lanes != 1 && lanes != 2 && lanes != 4 && lanes != 8 && lanes != 32)
-        return invalid("lanes per walk must be 1, 2, 4, 8 or 32");
+    if (lanes != 0 && lanes != 1 && lanes != 2 && lanes != 4 && lanes != 8 && lanes != 32)
+        return invalid("lanes per walk must be 0 (one lane, flattened loop), 1, 2, 4, 8 or 32");
     g_n2v_group = lanes;
     return GS_OK;
 }

@@ -41,6 +41,8 @@ struct gs_graph {
     int64_t max_degree;   // -1 when not validated
     int device;
     int4 *d_edge_rec;     // optional walk index, library-owned: {neighbour, its degree, its offset}
+    unsigned long long *d_edge_hash;   // optional edge set, library-owned: open-addressing table of
+    unsigned long long hash_mask;      // keys (row << 32 | column), capacity hash_mask + 1 (power of two)
 };
 
 namespace gs {

@@ -383,6 +383,73 @@ __device__ __forceinline__ bool row_contains(const int32_t *__restrict__ col, in
     return lo < end && ld_random(col + lo) == x;
 }
 
+// ------------------------------------------------------------------ edge set
+// "Is x a neighbour of prev" by binary search costs about log2(deg(prev)) dependent random reads,
+// and the walk sampler is bound by the number of such reads.  The optional edge set answers it
+// with one or two: every CSR entry (u, v) is stored as the key u << 32 | v in an open-addressing
+// table (linear probing, at most half full, 8 bytes per slot, so the probes of one lookup fall in
+// one 64-byte granule most of the time).  Built once per graph, read-only afterwards.
+constexpr unsigned long long EDGE_EMPTY = 0xFFFFFFFFFFFFFFFFull;
+
+__device__ __forceinline__ unsigned long long edge_mix(unsigned long long x)
+{
+    x ^= x >> 33; x *= 0xff51afd7ed558ccdull; x ^= x >> 33; x *= 0xc4ceb9fe1a85ec53ull; x ^= x >> 33;
+    return x;
+}
+
+// One warp per row; lanes take the row's entries 32 at a time.
+template <typename OffT>
+__global__ void __launch_bounds__(256)
+build_edge_hash_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col, int64_t n_nodes,
+                       unsigned long long *table, unsigned long long mask)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t u = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); u < n_nodes; u += n_warps) {
+        const int64_t b = (int64_t)off[u], e = (int64_t)off[u + 1];
+        for (int64_t x = b + lane; x < e; x += 32) {
+            const unsigned long long key = ((unsigned long long)u << 32) | (unsigned int)col[x];
+            unsigned long long slot = edge_mix(key) & mask;
+            for (unsigned long long n = 0; n <= mask; ++n) {          // the table is at most half full
+                const unsigned long long old = atomicCAS(table + slot, EDGE_EMPTY, key);
+                if (old == EDGE_EMPTY || old == key) break;
+                slot = (slot + 1) & mask;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ bool edge_set_contains(const unsigned long long *__restrict__ table,
+                                                  unsigned long long mask, int32_t u, int32_t v)
+{
+    const unsigned long long key = ((unsigned long long)(unsigned int)u << 32) | (unsigned int)v;
+    unsigned long long slot = edge_mix(key) & mask;
+    for (unsigned long long n = 0; n <= mask; ++n) {
+        const unsigned long long k = ld_random(reinterpret_cast<const uint64_t *>(table) + slot);
+        if (k == key) return true;
+        if (k == EDGE_EMPTY) return false;
+        slot = (slot + 1) & mask;
+    }
+    return false;
+}
+
+gs_status build_edge_hash(const gs_graph *g, unsigned long long *table, unsigned long long mask,
+                          cudaStream_t st)
+{
+    GS_CUDA_TRY(cudaMemsetAsync(table, 0xFF, sizeof(unsigned long long) * (size_t)(mask + 1), st));
+    int64_t blocks = (g->n_nodes + 7) / 8;
+    const int64_t cap = (int64_t)sm_count() * 64;
+    if (blocks > cap) blocks = cap;
+    if (g->offsets64)
+        build_edge_hash_kernel<int64_t><<<(unsigned)blocks, 256, 0, st>>>(
+            (const int64_t *)g->d_offsets, g->d_cols, g->n_nodes, table, mask);
+    else
+        build_edge_hash_kernel<int32_t><<<(unsigned)blocks, 256, 0, st>>>(
+            (const int32_t *)g->d_offsets, g->d_cols, g->n_nodes, table, mask);
+    GS_CUDA_TRY(cudaGetLastError());
+    return GS_OK;
+}
+
 // G lanes per walk; lane k of a group evaluates rejection round base + k.
 template <typename OffT, int G>
 __global__ void __launch_bounds__(256)
@@ -467,10 +534,11 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
 // walk index the proposal's record already holds the next node's range; without it the range
 // is read from the offsets at the start of the next transition.  Entries leave 32 bytes at a
 // time.  Needs L % 4 == 0 and a 16-byte aligned output.
-template <typename OffT, bool INDEX>
+template <typename OffT, bool INDEX, bool HASH>
 __global__ void __launch_bounds__(256, 4)
 node2vec_thread_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
-                       const int4 *__restrict__ rec, const int32_t *__restrict__ starts,
+                       const int4 *__restrict__ rec, const unsigned long long *__restrict__ edge_set,
+                       unsigned long long edge_mask, const int32_t *__restrict__ starts,
                        int64_t n_nodes, int64_t n_walks, int64_t walk_id_base, int32_t L,
                        uint64_t seed, N2VThresholds T, int32_t max_rounds,
                        int32_t *__restrict__ walks, unsigned long long *steps_out,
@@ -525,7 +593,11 @@ node2vec_thread_kernel(const OffT *__restrict__ off, const int32_t *__restrict__
                             else if (x == prev) acc = r1 < T.t_prev;
                             else if (r1 < t_lo) acc = true;
                             else if (r1 >= t_hi) acc = false;
-                            else acc = r1 < (row_contains(col, p0, p1, x) ? T.t_near : T.t_far);
+                            else {
+                                const bool near = HASH ? edge_set_contains(edge_set, edge_mask, prev, x)
+                                                       : row_contains(col, p0, p1, x);
+                                acc = r1 < (near ? T.t_near : T.t_far);
+                            }
                         }
                         if (!acc) ++my_caps;                   // cap reached: keep the last proposal
                         prev = cur; p0 = o0; p1 = o0 + deg;
@@ -542,6 +614,111 @@ node2vec_thread_kernel(const OffT *__restrict__ off, const int32_t *__restrict__
             else if (q == quads - 1) W4[q] = now;
             else pend = now;
         }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
+        my_caps += __shfl_xor_sync(0xffffffffu, my_caps, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (steps_out && my_steps) atomicAdd(steps_out, (unsigned long long)my_steps);
+        if (caps_out && my_caps) atomicAdd(caps_out, (unsigned long long)my_caps);
+    }
+}
+
+// One walk per thread again, but with the rejection rounds and the transitions of a walk flattened
+// into ONE loop: every trip of the loop is one round of whatever transition the lane is at.  In the
+// kernel above a lane that has accepted waits until the slowest lane of its warp has (the number of
+// rounds is geometric, so the slowest of 32 needs about three times the mean); here it starts its
+// next transition at once, and the memory system sees a request from every lane on every trip.
+// Finished entries collect in shared memory, eight per thread, and leave as two 16-byte stores.
+template <typename OffT, bool INDEX, bool HASH>
+__global__ void __launch_bounds__(256, 4)
+node2vec_flat_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
+                     const int4 *__restrict__ rec, const unsigned long long *__restrict__ edge_set,
+                     unsigned long long edge_mask, const int32_t *__restrict__ starts,
+                     int64_t n_nodes, int64_t n_walks, int64_t walk_id_base, int32_t L,
+                     uint64_t seed, N2VThresholds T, int32_t max_rounds,
+                     int32_t *__restrict__ walks, unsigned long long *steps_out,
+                     unsigned long long *caps_out)
+{
+    __shared__ int32_t buf[8][256];                        // buf[j][thread]: conflict-free
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const unsigned long long t_lo = T.t_near < T.t_far ? T.t_near : T.t_far;
+    const unsigned long long t_hi = T.t_near < T.t_far ? T.t_far : T.t_near;
+    const int tx = threadIdx.x;
+    unsigned int my_steps = 0, my_caps = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
+        const uint64_t id = (uint64_t)(walk_id_base + i);
+        int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
+        bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
+        int64_t o0 = 0;
+        uint32_t deg = 0;
+        if (alive) {
+            o0 = ld_random(off + cur);
+            deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
+        }
+        int32_t prev = -1;
+        int64_t p0 = 0, p1 = 0;
+        int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
+        buf[0][tx] = alive ? cur : -1;
+        int32_t e = 1;                                     // next entry to produce
+        int32_t sr = 0;                                    // rejection round of the transition into entry e
+        while (e < L) {
+            int32_t out = -1;                              // entry e once it is decided
+            bool done = !alive || deg == 0;                // dead end: the rest of the walk is -1
+            if (done) {
+                alive = false;
+            } else {
+                const uint4 r = draw(seed, id, (uint32_t)(e - 1), TAG_NODE2VEC, (uint32_t)sr);
+                const int64_t at = o0 + (int64_t)__umulhi(r.x, deg);
+                int32_t x;
+                uint32_t xdeg = 0;
+                int64_t xoff = 0;
+                if (INDEX) {
+                    const int4 rc = ld_random(rec + at);
+                    x = rc.x;
+                    xdeg = (uint32_t)rc.y;
+                    xoff = (int64_t)(((uint64_t)(uint32_t)rc.w << 32) | (uint32_t)rc.z);
+                } else {
+                    x = ld_random(col + at);
+                }
+                const unsigned long long r1 = r.y;
+                bool acc;
+                if (e == 1) acc = true;                    // first transition: uniform
+                else if (x == prev) acc = r1 < T.t_prev;
+                else if (r1 < t_lo) acc = true;
+                else if (r1 >= t_hi) acc = false;
+                else {
+                    const bool near = HASH ? edge_set_contains(edge_set, edge_mask, prev, x)
+                                           : row_contains(col, p0, p1, x);
+                    acc = r1 < (near ? T.t_near : T.t_far);
+                }
+                const bool last = sr + 1 >= (e == 1 ? 1 : max_rounds);
+                if (acc || last) {
+                    if (!acc) ++my_caps;                   // cap reached: keep the last proposal
+                    prev = cur; p0 = o0; p1 = o0 + deg;
+                    cur = x;
+                    if (INDEX) { o0 = xoff; deg = xdeg; }
+                    else { o0 = ld_random(off + cur); deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0); }
+                    ++my_steps;
+                    out = cur;
+                    done = true;
+                    sr = 0;
+                } else {
+                    ++sr;
+                }
+            }
+            if (done) {
+                buf[e & 7][tx] = out;
+                ++e;
+                if ((e & 7) == 0) {                        // entries [e - 8, e) are complete
+                    W4[(e >> 2) - 2] = make_int4(buf[0][tx], buf[1][tx], buf[2][tx], buf[3][tx]);
+                    W4[(e >> 2) - 1] = make_int4(buf[4][tx], buf[5][tx], buf[6][tx], buf[7][tx]);
+                }
+            }
+        }
+        if (L & 4)                                         // L = 8m + 4: the last four entries
+            W4[(L >> 2) - 1] = make_int4(buf[0][tx], buf[1][tx], buf[2][tx], buf[3][tx]);
     }
     for (int o = 16; o > 0; o >>= 1) {
         my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
@@ -592,21 +769,31 @@ gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_
     if (n_walks == 0) return GS_OK;
     N2VThresholds T;
     node2vec_thresholds(p, q, &T);
-    if (group == 1 && L % 4 == 0 && (((uintptr_t)walks & 15) == 0)) {
+    if (group <= 1 && L % 4 == 0 && (((uintptr_t)walks & 15) == 0)) {
         const int threads = 256;
         int64_t blocks = (n_walks + threads - 1) / threads;
         const int64_t cap = (int64_t)sm_count() * 8 * 16;
         if (blocks > cap) blocks = cap;
-#define GS_N2T(T_, IDX)                                                                           \
-        node2vec_thread_kernel<T_, IDX><<<(unsigned)blocks, threads, 0, st>>>(                      \
-            (const T_ *)g->d_offsets, g->d_cols, g->d_edge_rec, starts, g->n_nodes, n_walks, base, L, \
-            seed, T, max_rounds, walks, steps, caps)
-        if (g->offsets64) { if (g->d_edge_rec) GS_N2T(int64_t, true); else GS_N2T(int64_t, false); }
-        else { if (g->d_edge_rec) GS_N2T(int32_t, true); else GS_N2T(int32_t, false); }
+#define GS_N2T(T_, IDX, HSH)                                                                      \
+        do {                                                                                      \
+            if (group == 0)                                                                       \
+                node2vec_flat_kernel<T_, IDX, HSH><<<(unsigned)blocks, threads, 0, st>>>(           \
+                    (const T_ *)g->d_offsets, g->d_cols, g->d_edge_rec, g->d_edge_hash, g->hash_mask, \
+                    starts, g->n_nodes, n_walks, base, L, seed, T, max_rounds, walks, steps, caps); \
+            else                                                                                  \
+                node2vec_thread_kernel<T_, IDX, HSH><<<(unsigned)blocks, threads, 0, st>>>(         \
+                    (const T_ *)g->d_offsets, g->d_cols, g->d_edge_rec, g->d_edge_hash, g->hash_mask, \
+                    starts, g->n_nodes, n_walks, base, L, seed, T, max_rounds, walks, steps, caps); \
+        } while (0)
+#define GS_N2T_H(T_, IDX) do { if (g->d_edge_hash) GS_N2T(T_, IDX, true); else GS_N2T(T_, IDX, false); } while (0)
+        if (g->offsets64) { if (g->d_edge_rec) GS_N2T_H(int64_t, true); else GS_N2T_H(int64_t, false); }
+        else { if (g->d_edge_rec) GS_N2T_H(int32_t, true); else GS_N2T_H(int32_t, false); }
+#undef GS_N2T_H
 #undef GS_N2T
         GS_CUDA_TRY(cudaGetLastError());
         return GS_OK;
     }
+    if (group == 0) group = 1;                 // odd walk length or unaligned output: generic kernel
 #define GS_N2V(GG)                                                                              \
     do {                                                                                        \
         if (g->offsets64) launch_n2v<int64_t, GG>(g, starts, n_walks, base, L, seed, T,         \

@@ -137,7 +137,7 @@ def test_node2vec_walks_bit_exact_for_every_group_width(tiny, p, q, max_rounds):
     n_walks, L = 5003, 24
     want, st, caps = O.node2vec_walks(off, col, None, n_walks, 77, L, 5, p, q, max_rounds)
     try:
-        for lanes in (1, 2, 4, 8, 32):
+        for lanes in (0, 1, 2, 4, 8, 32):
             B.gs_tune_node2vec_group(lanes)
             steps = torch.zeros(1, dtype=torch.int64, device=DEV)
             hits = torch.zeros(1, dtype=torch.int64, device=DEV)
@@ -146,7 +146,7 @@ def test_node2vec_walks_bit_exact_for_every_group_width(tiny, p, q, max_rounds):
             assert np.array_equal(got.cpu().numpy(), want), lanes
             assert int(steps.item()) == st and int(hits.item()) == caps, lanes
     finally:
-        B.gs_tune_node2vec_group(1)
+        B.gs_tune_node2vec_group(0)
     if max_rounds <= 3:
         assert caps > 0
 
@@ -162,10 +162,33 @@ def test_node2vec_on_directed_graph_with_dead_ends_and_int64_offsets():
     assert np.array_equal(got.cpu().numpy(), want)
     # one walk per thread, over the walk index and without it, walk length a multiple of 4
     want, _, _ = O.node2vec_walks(off, col, starts, 4000, 9, 32, 12, 0.25, 4.0)
-    for flags in (3, 7):
-        G2 = load(g, offsets64=True, flags=flags)
-        got = B.gs_node2vec_walks(G2, torch.from_numpy(starts).to(DEV), 4000, 9, 32, 12, 0.25, 4.0)
-        assert np.array_equal(got.cpu().numpy(), want), flags
+    for flags in (3, 7, 3 | B.GS_BUILD_EDGE_SET, 7 | B.GS_BUILD_EDGE_SET):      # edge set: hashed membership test
+        for o64 in (True, False):
+            G2 = load(g, offsets64=o64, flags=flags)
+            for lanes in (0, 1):                       # flattened loop, nested loops
+                B.gs_tune_node2vec_group(lanes)
+                got = B.gs_node2vec_walks(G2, torch.from_numpy(starts).to(DEV), 4000, 9, 32, 12, 0.25, 4.0)
+                assert np.array_equal(got.cpu().numpy(), want), (flags, o64, lanes)
+                for L in (4, 12, 36):                  # 8m + 4 entries: the tail store of the flat kernel
+                    w2, _, _ = O.node2vec_walks(off, col, starts[:500], 500, 3, L, 12, 0.25, 4.0)
+                    g2 = B.gs_node2vec_walks(G2, torch.from_numpy(starts[:500].copy()).to(DEV), 500, 3, L, 12,
+                                             0.25, 4.0)
+                    assert np.array_equal(g2.cpu().numpy(), w2), (flags, o64, lanes, L)
+    B.gs_tune_node2vec_group(0)
+
+
+@pytest.mark.parametrize("p,q", [(0.5, 2.0), (4.0, 0.25), (2.0, 0.5)])
+def test_node2vec_with_the_edge_set_is_bit_exact_on_the_power_law_graph(tiny, p, q):
+    # hubs with thousands of neighbours and many triangles: every class of candidate occurs
+    _, g, off, col, _, _ = tiny
+    G = load(g, flags=B.GS_REQUIRE_SORTED | B.GS_BUILD_WALK_INDEX | B.GS_BUILD_EDGE_SET)
+    want, st, caps = O.node2vec_walks(off, col, None, 20000, 5, 40, 21, p, q)
+    for lanes in (0, 1):
+        B.gs_tune_node2vec_group(lanes)
+        steps = torch.zeros(1, dtype=torch.int64, device=DEV)
+        got = B.gs_node2vec_walks(G, None, 20000, 5, 40, 21, p, q, steps=steps)
+        assert np.array_equal(got.cpu().numpy(), want) and int(steps.item()) == st
+    B.gs_tune_node2vec_group(0)
 
 
 # ---------------------------------------------------------------- initialisation
@@ -532,11 +555,11 @@ def test_out_of_range_ids_count_as_absent_instead_of_faulting(tiny):
         want2, _, _ = O.node2vec_walks(off, col, np.where(ok, starts, 0).astype(np.int32), len(starts), 9, 16,
                                        2, 0.5, 2.0)
         want2[~ok] = -1
-        for lanes in (1, 4, 32):
+        for lanes in (0, 1, 4, 32):
             B.gs_tune_node2vec_group(lanes)
             got = B.gs_node2vec_walks(G, sd, len(starts), 9, 16, 2, 0.5, 2.0)
             assert np.array_equal(got.cpu().numpy(), want2)
-        B.gs_tune_node2vec_group(1)
+        B.gs_tune_node2vec_group(0)
     # walk entries outside the tables behave like -1 in the update
     walks, _ = O.uniform_walks(off, col, None, 200, 0, 12, 5)
     dirty = walks.copy()

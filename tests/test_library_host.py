@@ -107,4 +107,5 @@ def test_argument_errors_are_status_codes_without_touching_a_gpu(lib):
     assert st == -1 and b"step" in lib.gs_last_error()
     assert lib.gs_tune_node2vec_group(3) == -1
     assert lib.gs_tune_node2vec_group(1) == 0
+    assert lib.gs_tune_node2vec_group(0) == 0
     lib.gs_graph_free(None)

@@ -37,7 +37,11 @@ def test_fullsize_workload(name):
     g = wl.make_graph(device=DEV)
     n = g.n_nodes
     assert n == wl.n_nodes
-    G = B.gs_graph_load_csr(g.offsets, g.cols, B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    # the graph handle bench.py uses: walk index, and the hashed edge set for node2vec
+    flags = B.GS_VALIDATE | B.GS_REQUIRE_SORTED | B.GS_BUILD_WALK_INDEX
+    if wl.walk_kind != "uniform":
+        flags |= B.GS_BUILD_EDGE_SET
+    G = B.gs_graph_load_csr(g.offsets, g.cols, flags)
     deg = g.degrees()
     assert G.info()["max_degree"] == int(deg.max())
     off = g.offsets.cpu().numpy().astype(np.int64)

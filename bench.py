@@ -243,7 +243,7 @@ def run_reference(args, wl):
 
 def walk_kernel_name(wl, indexed):
     if wl.walk_kind != "uniform":
-        return "node2vec_thread_kernel"
+        return "node2vec_flat_kernel"
     return "uniform_walk_index_kernel" if indexed else "uniform_walk_vec_kernel"
 
 

@@ -120,6 +120,40 @@ def test_lock_free_single_walk_on_half_tables_equals_sequential_oracle(dim):
     assert np.mean(go != h_out.numpy().astype(np.float64)) > 0.001
 
 
+@pytest.mark.parametrize("dim,L,w", [(128, 40, 5), (64, 20, 5), (256, 24, 3)])
+def test_lock_free_many_walks_without_shared_rows_on_half_tables(dim, L, w):
+    # No two walks share a row, no walk visits a node twice, no negatives: nothing can race, so
+    # the concurrent run must follow the sequential oracle (rounded at every write) to within the
+    # few binary16 ulps that fp32-vs-fp64 rounding of the up to 2w updates of a row can differ by.
+    n_walks, span = 500, 64
+    n = n_walks * span
+    rng = np.random.default_rng(dim)
+    walks = np.empty((n_walks, L), dtype=np.int32)
+    for k in range(n_walks):
+        walks[k] = k * span + rng.permutation(span)[:L]
+    thr, alias = O.build_alias(np.ones(n), 1.0)
+    c, o, ng, n_pairs = O.expand_lists(walks, 0, w, 0, thr, alias, 3)
+    h_in, h_out = half_tables(n, dim, 6, scale=0.6)
+    U, V = h_in.numpy().astype(np.float64), h_out.numpy().astype(np.float64)
+    loss_o, cnt_o = O.sgns_seq_f16_from_lists(U, V, c, o, ng, 2 * w, 0.05)
+    w_in, w_out = h_in.to(DEV), h_out.to(DEV)
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    B.gs_sgns_step_f16(w_in, w_out, torch.from_numpy(walks).to(DEV), 0, w, 0, None, 0.05, 3,
+                       B.GS_HOGWILD, loss, cnt)
+    torch.cuda.synchronize()
+    assert cnt.item() == cnt_o == n_pairs and abs(loss.item() - loss_o) < 1e-4 * abs(loss_o)
+    gi, go = w_in.cpu().numpy().astype(np.float64), w_out.cpu().numpy().astype(np.float64)
+    # a rounding is made at the magnitude the value has WHEN it is written: between its start and
+    # its end value, and not below the size of one update (about lr * |g| * |u| <= 5e-3)
+    U0, V0 = h_in.numpy().astype(np.float64), h_out.numpy().astype(np.float64)
+    for got, want, start in ((gi, U, U0), (go, V, V0)):
+        scale = np.maximum(np.maximum(np.abs(want), np.abs(start)), 5e-3)
+        assert (np.abs(got - want) <= 4 * ulp16(scale)).all()
+        assert np.mean(got == want) > 0.9
+    assert np.mean(go != h_out.numpy().astype(np.float64)) > 0.3        # the step did move the rows
+
+
 def test_half_tables_reject_what_they_do_not_support(tiny):
     g, off, col, thr, alias = tiny
     a_dev = alias_to_device(thr, alias)

@@ -399,6 +399,35 @@ def test_lock_free_single_walk_equals_sequential_oracle(dim):
         assert np.abs(V - w_out0.numpy()).max() > 1e-3
 
 
+@pytest.mark.parametrize("dim,L,w", [(128, 40, 5), (64, 20, 5), (256, 24, 3), (32, 16, 2), (128, 2, 1)])
+def test_lock_free_many_walks_without_shared_rows_equal_sequential_oracle(dim, L, w):
+    # Hundreds of walks run concurrently (ticket counter, several row groups per warp, every launch
+    # shape of the kernel), but no two walks share a row and no walk visits a node twice: walk k
+    # runs along its own stretch of distinct nodes, and K = 0 leaves no negative draws.  Without
+    # shared rows nothing can race, so the concurrent result must equal strictly sequential SGD.
+    n_walks, span = 700, 64
+    n = n_walks * span
+    rng = np.random.default_rng(dim + L)
+    walks = np.empty((n_walks, L), dtype=np.int32)
+    for k in range(n_walks):
+        walks[k] = k * span + rng.permutation(span)[:L]
+    walks[5, L // 2:] = -1                                # a walk that ended early
+    thr, alias = O.build_alias(np.ones(n), 1.0)
+    c, o, ng, n_pairs = O.expand_lists(walks, 9, w, 0, thr, alias, 3)
+    w_in0, w_out0 = random_tables(n, dim, 8)
+    U, V = w_in0.numpy().astype(np.float64), w_out0.numpy().astype(np.float64)
+    loss_o, cnt_o = O.sgns_seq_from_lists(U, V, c, o, ng, 2 * w, 0.05)
+    assert cnt_o == n_pairs > 0
+    for mode in (B.GS_HOGWILD, B.GS_HOGWILD_RED):
+        w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+        loss, cnt, _, _ = run_step(w_in, w_out, torch.from_numpy(walks).to(DEV), 9, w, 0, None, 0.05, 3,
+                                   mode, dump=False)
+        assert cnt == cnt_o and abs(loss - loss_o) < 2e-6 * abs(loss_o)
+        assert np.abs(w_in.cpu().numpy() - U).max() <= 1e-5
+        assert np.abs(w_out.cpu().numpy() - V).max() <= 1e-5
+    assert np.abs(V - w_out0.numpy()).max() > 1e-3
+
+
 def test_sgns_step_edge_cases(tiny):
     _, g, off, col, thr, alias = tiny
     a_dev = alias_to_device(thr, alias)

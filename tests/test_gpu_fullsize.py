@@ -80,6 +80,25 @@ def test_fullsize_workload(name):
             want, _, _ = O.node2vec_walks(off, col, None, 1024, base + lo, wl.walk_len, seed, wl.p, wl.q)
         assert np.array_equal(walks[lo:lo + 1024].cpu().numpy(), want), lo
 
+    # ---- corpus variants at full size: shuffled start order is a bijection of all nodes and
+    # matches the oracle on sampled ranges; sub-sampled walks match the oracle on sampled ranges
+    starts_all = B.gs_shuffled_starts(n, seed, 3, 0, n, DEV)
+    assert int(torch.bincount(starts_all.to(torch.int64), minlength=n).max()) == 1
+    for lo in (0, n // 2 - 77, n - 4096):
+        assert np.array_equal(starts_all[lo:lo + 4096].cpu().numpy(), O.shuffled_starts(n, seed, 3, lo, 4096))
+    del starts_all
+    degf = deg.cpu().numpy().astype(np.float64)
+    keep_thr = B.gs_build_keep_thresholds(degf, 1e-6)
+    assert np.array_equal(keep_thr, O.keep_thresholds(degf, 1e-6))
+    del degf
+    kept = torch.zeros(1, dtype=torch.int64, device=DEV)
+    thinned = B.gs_subsample_walks(walks, base, torch.from_numpy(keep_thr.view(np.int32)).to(DEV), seed, kept=kept)
+    assert int(kept.item()) == int((thinned >= 0).sum()) < int((walks >= 0).sum())
+    for lo in (0, bw // 2 - 333, bw - 1024):
+        want, _ = O.subsample_walks(walks[lo:lo + 1024].cpu().numpy(), base + lo, keep_thr, seed)
+        assert np.array_equal(thinned[lo:lo + 1024].cpu().numpy(), want), lo
+    del thinned, keep_thr
+
     # ---- tables; one lock-free step on the whole batch (makes the output rows non-zero)
     w_in = torch.empty((n, wl.dim), dtype=torch.float32, device=DEV)
     w_out = torch.empty_like(w_in)

@@ -891,55 +891,71 @@ sgns_apply_out_fixup_kernel(T *__restrict__ w_out, const uint32_t *__restrict__ 
 }
 
 // Pass 4, keys in [n_nodes, 2 n_nodes): u_row -= lr * sum of the positions' GU rows.
+// The center keys sort behind every output-row key and before the invalid ones, so they form one
+// stretch of at most n_pos sorted positions.  Every warp finds where that stretch starts (a
+// search over keys that stay in L2) and then takes ONE position of it: if a run of equal keys
+// starts there, the warp sums the run's GU rows in index order and writes the row.  (A warp per 32
+// sorted positions left the whole pass to the few hundred warps whose chunk held center keys.)
 template <int FPL, typename T>
 __global__ void __launch_bounds__(256)
 sgns_apply_in_kernel(T *__restrict__ w_in, const float *__restrict__ GU,
                      const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals,
-                     uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, float lr, MomState ms)
+                     uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, uint32_t n_pos, float lr,
+                     MomState ms)
 {
     constexpr int U = FPL <= 4 ? 8 : 4;
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int64_t n_chunks = ((int64_t)n_keys + 31) >> 5;
-    for (int64_t ch = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); ch < n_chunks;
-         ch += n_warps) {
-        const int64_t i = ch * 32 + lane;
-        const uint32_t my_key = i < n_keys ? keys[i] : 0xFFFFFFFFu;
-        const bool head = i < n_keys && my_key >= n_nodes && my_key < 2u * n_nodes &&
-                          (i == 0 || keys[i - 1] != my_key);
-        unsigned heads = __ballot_sync(0xffffffffu, head);
-        while (heads) {
-            const int hl = __ffs(heads) - 1;
-            heads &= heads - 1;
-            const uint32_t key = __shfl_sync(0xffffffffu, my_key, hl);
-            double acc[FPL];
-#pragma unroll
-            for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
-            for (int64_t y0 = ch * 32 + hl;; y0 += 32) {
-                const int64_t y = y0 + lane;
-                const bool in = y < n_keys && keys[y] == key;
-                const int cnt = __popc(__ballot_sync(0xffffffffu, in));
-                const uint32_t pos = in ? vals[y] - n_slots : 0u;
-                for (int q0 = 0; q0 < cnt; q0 += U) {
-                    Row<FPL> r[U];
-#pragma unroll
-                    for (int q = 0; q < U; ++q) {
-                        const uint32_t pq = __shfl_sync(0xffffffffu, pos, (q0 + q) & 31);
-                        if (q0 + q < cnt) r[q] = row_load<FPL>(GU, (int64_t)pq, lane);
-                    }
-#pragma unroll
-                    for (int q = 0; q < U; ++q)
-                        if (q0 + q < cnt) {
-#pragma unroll
-                            for (int j = 0; j < FPL; ++j) acc[j] += (double)r[q].v[j];
-                        }
-                }
-                if (cnt < 32) break;
-            }
-            const int64_t c = (int64_t)(key - n_nodes);
-            Row<FPL> row = row_load<FPL>(w_in, c, lane);
-            write_updated_row<FPL, T>(w_in, c, lane, row, acc, lr, ms);
+    // first sorted position whose key is not an output row: 32-way search, the lanes probe 32
+    // evenly spaced positions per step (5 round trips for 2^25 keys instead of 25)
+    int64_t first = 0;
+    {
+        int64_t lo = 0, hi = n_keys;                               // answer in [lo, hi]
+        while (hi - lo > 32) {
+            const int64_t step = (hi - lo + 31) / 32;
+            const int64_t p = lo + (int64_t)(lane + 1) * step - 1;  // last position of slice `lane`
+            const bool below = p < hi && keys[p] < n_nodes;         // the whole slice is below
+            const int full = __popc(__ballot_sync(0xffffffffu, below));   // sorted: a prefix of lanes
+            lo += (int64_t)full * step;
+            if (lo + step < hi) hi = lo + step;
         }
+        const bool below = lo + lane < hi && keys[lo + lane] < n_nodes;
+        first = lo + __popc(__ballot_sync(0xffffffffu, below));
+    }
+    for (int64_t wi = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); wi < (int64_t)n_pos;
+         wi += n_warps) {
+        const int64_t i = first + wi;
+        if (i >= (int64_t)n_keys) break;
+        const uint32_t key = keys[i];
+        if (key >= 2u * n_nodes) break;                              // the invalid keys come last
+        if (wi > 0 && keys[i - 1] == key) continue;                  // inside a run: its head does the work
+        double acc[FPL];
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) acc[j] = 0.0;
+        for (int64_t y0 = i;; y0 += 32) {
+            const int64_t y = y0 + lane;
+            const bool in = y < n_keys && keys[y] == key;
+            const int cnt = __popc(__ballot_sync(0xffffffffu, in));
+            const uint32_t pos = in ? vals[y] - n_slots : 0u;
+            for (int q0 = 0; q0 < cnt; q0 += U) {
+                Row<FPL> r[U];
+#pragma unroll
+                for (int q = 0; q < U; ++q) {
+                    const uint32_t pq = __shfl_sync(0xffffffffu, pos, (q0 + q) & 31);
+                    if (q0 + q < cnt) r[q] = row_load<FPL>(GU, (int64_t)pq, lane);
+                }
+#pragma unroll
+                for (int q = 0; q < U; ++q)
+                    if (q0 + q < cnt) {
+#pragma unroll
+                        for (int j = 0; j < FPL; ++j) acc[j] += (double)r[q].v[j];
+                    }
+            }
+            if (cnt < 32) break;
+        }
+        const int64_t c = (int64_t)(key - n_nodes);
+        Row<FPL> row = row_load<FPL>(w_in, c, lane);
+        write_updated_row<FPL, T>(w_in, c, lane, row, acc, lr, ms);
     }
 }
 
@@ -1144,8 +1160,11 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
                 w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part, ms_out);
             GS_CUDA_TRY(cudaGetLastError());
         }
-        sgns_apply_in_kernel<FPL, T><<<(unsigned)blocks, 256, 0, st>>>(
-            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr, ms_in);
+        int64_t in_blocks = (n_pos + 7) / 8;                    // one warp per center position
+        if (in_blocks > cap) in_blocks = cap;
+        sgns_apply_in_kernel<FPL, T><<<(unsigned)in_blocks, 256, 0, st>>>(
+            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, (uint32_t)n_pos,
+            a.lr, ms_in);
         GS_CUDA_TRY(cudaGetLastError());
     }
     if (a.loss || a.pairs || a.masked) {
@@ -1373,9 +1392,11 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
                 MomState{ nullptr, nullptr, 0.f, 0 });
             GS_CUDA_TRY(cudaGetLastError());
         }
-        sgns_apply_in_kernel<FPL, float><<<(unsigned)blocks, 256, 0, st>>>(
-            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, a.lr,
-            MomState{ nullptr, nullptr, 0.f, 0 });
+        int64_t in_blocks = (n_pos + 7) / 8;                    // one warp per center position
+        if (in_blocks > cap) in_blocks = cap;
+        sgns_apply_in_kernel<FPL, float><<<(unsigned)in_blocks, 256, 0, st>>>(
+            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, (uint32_t)n_pos,
+            a.lr, MomState{ nullptr, nullptr, 0.f, 0 });
         GS_CUDA_TRY(cudaGetLastError());
     }
     if (a.loss || a.pairs || a.masked) {

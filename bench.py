@@ -341,8 +341,8 @@ def run_walks_only(args, wl, g, G, info, dev):
 
 # ---------------------------------------------------------------------------- momentum step
 def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
-    """Times walks + gs_sgns_step_momentum (or gs_sgns_step_adam with --mode adam) on batches of
-    512 walks (synchronous; momentum 0.9 as in the paper's production run).  1 GPU."""
+    """Times the epoch driver with the momentum (or, --mode adam, Adam) step on batches of 512 walks
+    (synchronous; momentum 0.9 as in the paper's production run).  1 GPU."""
     import torch
     from paper_2407_15452_b200 import binding as B
     n = g.n_nodes
@@ -356,44 +356,32 @@ def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
     else:
         last_in = torch.zeros(n, dtype=torch.int32, device=dev)
         last_out = torch.zeros_like(last_in)
-    walks = torch.empty((bw, wl.walk_len), dtype=torch.int32, device=dev)
-    loss = torch.zeros(1, dtype=torch.float64, device=dev)
-    cnt = torch.zeros(1, dtype=torch.int64, device=dev)
     mu = 0.9
     seed, lr = wl.graph_seed, wl.lr0 * (1.0 - mu)      # same effective step lr / (1 - mu) as the plain runs
     if adam:
         lr = 0.001                                     # Adam's usual step size
-
-    def step(it):
-        base = (it % nb_total) * bw
-        k = min(bw, total_walks - base)
-        if wl.walk_kind == "uniform":
-            B.gs_random_walks(G, None, k, base, wl.walk_len, seed, out=walks)
-        else:
-            B.gs_node2vec_walks(G, None, k, base, wl.walk_len, seed, wl.p, wl.q, out=walks)
-        if adam:
-            B.gs_sgns_step_adam(w_in, w_out, m_in, v_in, m_out, v_out, walks[:k], base, wl.window,
-                                wl.n_neg, alias, lr, 0.9, 0.999, 1e-8, it + 1, seed, 0, loss, cnt)
-        else:
-            B.gs_sgns_step_momentum(w_in, w_out, m_in, m_out, last_in, last_out, walks[:k], base,
-                                    wl.window, wl.n_neg, alias, lr, mu, it, seed, loss, cnt)
-
-    for it in range(args.warmup):
-        step(it)
-    torch.cuda.synchronize()
-    loss.zero_()
-    cnt.zero_()
+    kind = B.GS_WALK_UNIFORM if wl.walk_kind == "uniform" else B.GS_WALK_NODE2VEC
+    kw = dict(walks_per_node=wl.walks_per_node, walk_len=wl.walk_len, window=wl.window, n_neg=wl.n_neg,
+              lr0=lr, batch_walks=bw, seed=seed, mode=B.GS_DETERMINISTIC, walk_kind=kind, p=wl.p, q=wl.q,
+              momentum=mu, m_in=m_in, m_out=m_out)
+    if adam:
+        kw.update(optimizer=B.GS_OPT_ADAM, beta2=0.999, eps=1e-8, v_in=v_in, v_out=v_out)
+    else:
+        kw.update(optimizer=B.GS_OPT_MOMENTUM, last_in=last_in, last_out=last_out)
+    # the epoch driver runs the optimizer step per batch; one call covers the K timed batches
+    assert args.warmup + args.steps <= nb_total
+    B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=0, num_batches=args.warmup, **kw)
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    for it in range(args.warmup, args.warmup + args.steps):
-        step(it)
+    r = B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=args.warmup, num_batches=args.steps, **kw)
     ev1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
     ms = ev0.elapsed_time(ev1)
-    pairs = int(cnt.item())
+    pairs = r.pairs
+    loss = torch.tensor([r.loss_sum])
     peak, peak_kind = measured_peak_gbs()
     # per pair and target: the embedding row and its momentum row (Adam: both moment rows), each
     # read and written once

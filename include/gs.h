@@ -399,6 +399,9 @@ GS_API gs_status gs_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epo
 #define GS_TABLE_F16      1   /* tables of IEEE half, see gs_sgns_step_f16      */
 #define GS_LR_CONSTANT    0
 #define GS_LR_LINEAR      1   /* lr_b = lr0 * max(1 - b / total_batches, 1e-4) */
+#define GS_OPT_SGD        0
+#define GS_OPT_MOMENTUM   1
+#define GS_OPT_ADAM       2
 
 typedef struct gs_sgns_config {
     int32_t dim;
@@ -423,6 +426,20 @@ typedef struct gs_sgns_config {
                               /* walks are sub-sampled before the update; NULL = off      */
     int32_t shuffle_starts;   /* != 0: walk id a starts at the gs_shuffled_starts image  */
     uint32_t epoch;           /* of a mod n_nodes for this epoch instead of at a mod n   */
+    /* Optimizer of the synchronous mode (Section 3.2 keeps SGD with momentum and Adam inside the
+     * storage; its large run uses momentum 0.9).  GS_OPT_SGD: plain steps, the fields below are
+     * ignored.  GS_OPT_MOMENTUM: every batch is one gs_sgns_step_momentum with iteration =
+     * iteration_base + batch index; needs GS_LR_CONSTANT, fp32 tables, no pair flags; rows are
+     * brought up to date lazily, so call gs_momentum_flush(iteration = iteration_base + index of
+     * the last batch + 1) before reading the tables elsewhere.  GS_OPT_ADAM: every batch is one
+     * gs_sgns_step_adam with step = iteration_base + batch index + 1; fp32 tables. */
+    int32_t optimizer;        /* GS_OPT_*                                                */
+    float   momentum;         /* GS_OPT_MOMENTUM: momentum value; GS_OPT_ADAM: beta1     */
+    float   beta2, eps;       /* GS_OPT_ADAM                                             */
+    int64_t iteration_base;   /* iterations done before batch 0 of this epoch            */
+    float  *d_m_in, *d_m_out; /* momentum tables / first moments, shape of the tables    */
+    float  *d_v_in, *d_v_out; /* GS_OPT_ADAM: second moments                             */
+    int32_t *d_last_in, *d_last_out;   /* GS_OPT_MOMENTUM: per-row iteration stamps      */
 } gs_sgns_config;
 
 typedef struct gs_epoch_stats {
@@ -432,6 +449,7 @@ typedef struct gs_epoch_stats {
     int64_t cap_hits;         /* node2vec rejection cap hits                     */
     int64_t batches;
     int64_t masked_negs;      /* negatives dropped because they equal their context */
+                              /* (counted with GS_OPT_SGD only)                      */
     float   ms_walk;          /* device time of the walk kernels                 */
     float   ms_sgns;          /* device time of the SGNS kernels                 */
     float   ms_total;

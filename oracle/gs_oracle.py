@@ -353,13 +353,17 @@ def lr_at(schedule, lr0, b, num_batches):
 
 def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, schedule,
                batch_walks, seed, mode="det", kind="uniform", p=1.0, q=1.0,
-               first_batch=0, num_batches=None, shrink=False, keep_thr=None, shuffle_epoch=None):
+               first_batch=0, num_batches=None, shrink=False, keep_thr=None, shuffle_epoch=None,
+               optimizer="sgd", state=None, momentum=0.9, beta2=0.999, eps=1e-8, iteration_base=0):
     """One pass over walk ids rep*N + v in order, batch by batch (dense tables).
 
     Each batch: generate its walks, expand pairs and negatives, apply one step.
     shuffle_epoch (int or None): walk id a starts at the keyed bijection of a mod N for that
     epoch instead of at a mod N.  keep_thr (uint32[N] or None): frequent-node sub-sampling of
     the generated walks before the windows are formed.  shrink: per-position window draw.
+    optimizer: "sgd"; "momentum" (dense update of both tables per batch, Section 3.2; state =
+    dict(MU, MV) of zero-initialised tables); "adam" (rows of the batch only; state = dict(MU, VU,
+    MV, VV); step = iteration_base + batch index + 1).  Both need mode "det".
     Returns dict(loss_sum, pairs, steps).  Tables are updated in place.
     """
     n_nodes = len(off) - 1
@@ -380,7 +384,12 @@ def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, sche
             walks, _ = subsample_walks(walks, base, keep_thr, seed)
         c, o, ng, _ = expand_lists(walks, base, w, K, thr, alias, seed, shrink=shrink)
         lr = lr_at(schedule, lr0, b, nb_total)
-        if mode == "det":
+        if optimizer == "momentum":
+            ls, pc = sgns_momentum_step_from_lists(U, V, state["MU"], state["MV"], c, o, ng, lr, momentum)
+        elif optimizer == "adam":
+            ls, pc = sgns_adam_step_from_lists(U, V, state["MU"], state["VU"], state["MV"], state["VV"],
+                                               c, o, ng, lr, momentum, beta2, eps, iteration_base + b + 1)
+        elif mode == "det":
             ls, pc = sgns_det_from_lists(U, V, c, o, ng, lr)
         else:
             ls, pc = sgns_seq_from_lists(U, V, c, o, ng, 2 * w, lr)

@@ -25,6 +25,7 @@ GS_WINDOW_SHRINK = 0x200
 GS_WALK_UNIFORM, GS_WALK_NODE2VEC = 0, 1
 GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
 GS_TABLE_F32, GS_TABLE_F16 = 0, 1
+GS_OPT_SGD, GS_OPT_MOMENTUM, GS_OPT_ADAM = 0, 1, 2
 
 EXPORTS = [
     "gs_last_error", "gs_graph_load_csr", "gs_graph_free", "gs_graph_info", "gs_build_alias",
@@ -50,6 +51,10 @@ class SgnsConfig(ctypes.Structure):
         ("lr0", ctypes.c_double), ("batch_walks", ctypes.c_int64), ("first_batch", ctypes.c_int64),
         ("num_batches", ctypes.c_int64), ("seed", ctypes.c_uint64),
         ("d_keep_thr", ctypes.c_void_p), ("shuffle_starts", ctypes.c_int32), ("epoch", ctypes.c_uint32),
+        ("optimizer", ctypes.c_int32), ("momentum", ctypes.c_float), ("beta2", ctypes.c_float),
+        ("eps", ctypes.c_float), ("iteration_base", ctypes.c_int64),
+        ("d_m_in", ctypes.c_void_p), ("d_m_out", ctypes.c_void_p), ("d_v_in", ctypes.c_void_p),
+        ("d_v_out", ctypes.c_void_p), ("d_last_in", ctypes.c_void_p), ("d_last_out", ctypes.c_void_p),
     ]
 
 
@@ -351,7 +356,9 @@ class EpochResult:
 def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len, window, n_neg,
                   lr0, batch_walks, seed, mode, walk_kind=GS_WALK_UNIFORM,
                   lr_schedule=GS_LR_CONSTANT, p=1.0, q=1.0, max_rounds=1024, first_batch=0,
-                  num_batches=0, keep_thr=None, shuffle_epoch=None) -> EpochResult:
+                  num_batches=0, keep_thr=None, shuffle_epoch=None, optimizer=GS_OPT_SGD, momentum=0.0,
+                  beta2=0.999, eps=1e-8, iteration_base=0, m_in=None, m_out=None, v_in=None, v_out=None,
+                  last_in=None, last_out=None) -> EpochResult:
     if w_in.dtype not in (torch.float32, torch.float16) or w_out.dtype != w_in.dtype:
         raise TypeError("tables must both be float32 or both float16")
     tdt = w_in.dtype
@@ -362,7 +369,15 @@ def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len,
                      batch_walks=batch_walks, first_batch=first_batch, num_batches=num_batches,
                      seed=seed, d_keep_thr=_dev(keep_thr, torch.int32, "keep_thr", True).value,
                      shuffle_starts=0 if shuffle_epoch is None else 1,
-                     epoch=0 if shuffle_epoch is None else shuffle_epoch)
+                     epoch=0 if shuffle_epoch is None else shuffle_epoch,
+                     optimizer=optimizer, momentum=momentum, beta2=beta2, eps=eps,
+                     iteration_base=iteration_base,
+                     d_m_in=_dev(m_in, torch.float32, "m_in", True).value,
+                     d_m_out=_dev(m_out, torch.float32, "m_out", True).value,
+                     d_v_in=_dev(v_in, torch.float32, "v_in", True).value,
+                     d_v_out=_dev(v_out, torch.float32, "v_out", True).value,
+                     d_last_in=_dev(last_in, torch.int32, "last_in", True).value,
+                     d_last_out=_dev(last_out, torch.int32, "last_out", True).value)
     st = EpochStats()
     _check(lib().gs_sgns_epoch(graph._h, _dev(alias, torch.int64, "alias", n_neg == 0),
                                _dev(w_in, tdt, "w_in"), _dev(w_out, tdt, "w_out"),

@@ -650,6 +650,24 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
         if (!(cfg->p > 0.0) || !(cfg->q > 0.0)) return invalid("p and q must be positive");
         if (cfg->max_rounds < 1 || cfg->max_rounds > 65536) return invalid("max_rounds outside [1, 65536]");
     }
+    if (cfg->optimizer != GS_OPT_SGD) {
+        if (cfg->optimizer != GS_OPT_MOMENTUM && cfg->optimizer != GS_OPT_ADAM) return invalid("unknown optimizer");
+        if (f16) { set_error("momentum and Adam need fp32 tables"); return GS_ERR_UNSUPPORTED; }
+        if ((cfg->mode & 0xFF) != GS_DETERMINISTIC) return invalid("momentum and Adam run in the synchronous mode only");
+        if (cfg->iteration_base < 0 || cfg->iteration_base > 0x7FFFFFF0) return invalid("iteration_base outside [0, 2^31 - 16)");
+        if (!cfg->d_m_in || !cfg->d_m_out) return invalid("moment tables are NULL");
+        if (cfg->optimizer == GS_OPT_MOMENTUM) {
+            if (cfg->lr_schedule != GS_LR_CONSTANT) return invalid("momentum needs a constant learning rate");
+            if (cfg->mode != GS_DETERMINISTIC) return invalid("momentum takes no pair flags");
+            if (!cfg->d_last_in || !cfg->d_last_out) return invalid("iteration stamps are NULL");
+            if (!(cfg->momentum >= 0.f) || !(cfg->momentum < 1.f)) return invalid("momentum must be in [0, 1)");
+        } else {
+            if (!cfg->d_v_in || !cfg->d_v_out) return invalid("second-moment tables are NULL");
+            if (!(cfg->momentum >= 0.f) || !(cfg->momentum < 1.f) || !(cfg->beta2 >= 0.f) || !(cfg->beta2 < 1.f))
+                return invalid("beta1 and beta2 must be in [0, 1)");
+            if (!(cfg->eps > 0.f)) return invalid("eps must be positive");
+        }
+    }
     memset(h_out, 0, sizeof(*h_out));
     const int64_t total_walks = g->n_nodes * (int64_t)cfg->walks_per_node;
     const int64_t nb_total = (total_walks + cfg->batch_walks - 1) / cfg->batch_walks;
@@ -736,7 +754,20 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
                 lr = cfg->lr0 * (f > 1e-4 ? f : 1e-4);
             }
             const int tk = t_sgns.start(s_sgns);
-            if (f16)
+            if (cfg->optimizer == GS_OPT_MOMENTUM)
+                EP_CALL(sgns_step_momentum((float *)d_w_in, (float *)d_w_out, cfg->d_m_in, cfg->d_m_out,
+                                           cfg->d_last_in, cfg->d_last_out, g->n_nodes, cfg->dim, wbuf[buf],
+                                           n, base, cfg->walk_len, cfg->window, cfg->n_neg, d_alias,
+                                           (float)lr, cfg->momentum, (int32_t)(cfg->iteration_base + b),
+                                           cfg->seed, &ctr->loss, (int64_t *)&ctr->pairs, s_sgns));
+            else if (cfg->optimizer == GS_OPT_ADAM)
+                EP_CALL(sgns_step_adam((float *)d_w_in, (float *)d_w_out, cfg->d_m_in, cfg->d_v_in,
+                                       cfg->d_m_out, cfg->d_v_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
+                                       cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
+                                       cfg->momentum, cfg->beta2, cfg->eps, cfg->iteration_base + b + 1,
+                                       cfg->seed, cfg->mode & ~0xFF, &ctr->loss, (int64_t *)&ctr->pairs,
+                                       s_sgns));
+            else if (f16)
                 EP_CALL(sgns_step_f16(d_w_in, d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
                                       cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
                                       cfg->seed, cfg->mode, &ctr->loss, (int64_t *)&ctr->pairs, nullptr,

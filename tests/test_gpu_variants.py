@@ -230,3 +230,80 @@ def test_subsampling_drops_entries_outside_the_threshold_table(tiny):
     want, _ = O.subsample_walks(np.where(hit, -1, walks).astype(np.int32), 0, keep_thr, 1)
     got = B.gs_subsample_walks(torch.from_numpy(dirty).to(DEV), 0, thr_to_device(keep_thr), 1)
     assert np.array_equal(got.cpu().numpy(), want)
+
+
+# ---------------------------------------------------------------- optimizers inside the epoch driver
+def test_epoch_with_momentum_matches_the_dense_oracle(tiny):
+    wl, g, off, col, thr, alias = tiny
+    n, dim, mu, lr = g.n_nodes, wl.dim, 0.9, 0.0025
+    U = O.init_rows(np.arange(n), dim, 0)
+    V = np.zeros_like(U)
+    state = {"MU": np.zeros_like(U), "MV": np.zeros_like(U)}
+    nb = 8                                               # eight batches of 512 walks, then two halves
+    want = O.sgns_epoch(off, col, thr, alias, U, V, walks_per_node=1, L=wl.walk_len, w=wl.window,
+                        K=wl.n_neg, lr0=lr, schedule="constant", batch_walks=512, seed=0, num_batches=nb,
+                        optimizer="momentum", state=state, momentum=mu)
+    G = B.gs_graph_load_csr(g.offsets.to(DEV), g.cols.to(DEV), B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    w_in = torch.empty((n, dim), dtype=torch.float32, device=DEV)
+    w_out = torch.empty_like(w_in)
+    B.gs_init_embeddings(w_in, w_out, 0)
+    m_in, m_out = torch.zeros_like(w_in), torch.zeros_like(w_in)
+    last_in = torch.zeros(n, dtype=torch.int32, device=DEV)
+    last_out = torch.zeros_like(last_in)
+    kw = dict(walks_per_node=1, walk_len=wl.walk_len, window=wl.window, n_neg=wl.n_neg, lr0=lr,
+              batch_walks=512, seed=0, mode=B.GS_DETERMINISTIC, optimizer=B.GS_OPT_MOMENTUM, momentum=mu,
+              m_in=m_in, m_out=m_out, last_in=last_in, last_out=last_out)
+    a_dev = alias_to_device(thr, alias)
+    r1 = B.gs_sgns_epoch(G, a_dev, w_in, w_out, first_batch=0, num_batches=3, **kw)
+    r2 = B.gs_sgns_epoch(G, a_dev, w_in, w_out, first_batch=3, num_batches=nb - 3, **kw)
+    B.gs_momentum_flush(w_in, m_in, last_in, lr, mu, nb)
+    B.gs_momentum_flush(w_out, m_out, last_out, lr, mu, nb)
+    torch.cuda.synchronize()
+    assert r1.pairs + r2.pairs == want["pairs"] and r1.batches + r2.batches == nb
+    assert abs(r1.loss_sum + r2.loss_sum - want["loss_sum"]) <= 1e-3 * want["loss_sum"]
+    for got, ref in ((w_in, U), (w_out, V), (m_in, state["MU"]), (m_out, state["MV"])):
+        assert np.abs(got.cpu().numpy() - ref).max() <= EMB_TOL
+    assert np.abs(state["MV"]).max() > 50 * EMB_TOL
+    with pytest.raises(B.GsError):                        # momentum needs a constant learning rate
+        B.gs_sgns_epoch(G, a_dev, w_in, w_out, num_batches=1, lr_schedule=B.GS_LR_LINEAR, **kw)
+    with pytest.raises(B.GsError):                        # and the synchronous mode
+        B.gs_sgns_epoch(G, a_dev, w_in, w_out, num_batches=1, **{**kw, "mode": B.GS_HOGWILD})
+
+
+def test_epoch_with_adam_matches_the_oracle(tiny):
+    wl, g, off, col, thr, alias = tiny
+    n, dim, lr = g.n_nodes, wl.dim, 0.001
+    rng = np.random.default_rng(3)
+    U0 = ((rng.random((n, dim)) - 0.5) * 0.4).astype(np.float32).astype(np.float64)
+    V0 = ((rng.random((n, dim)) - 0.5) * 0.4).astype(np.float32).astype(np.float64)
+    U, V = U0.copy(), V0.copy()
+    MU, VU, MV, VV = (np.zeros_like(U) for _ in range(4))
+    nb, base_it = 5, 7
+    near_zero_U, near_zero_V = np.zeros(U.shape, bool), np.zeros(V.shape, bool)
+    pairs, loss_o = 0, 0.0
+    for b in range(nb):                                   # the oracle's epoch, batch by batch, so that the
+        walks, _ = O.uniform_walks(off, col, None, 512, b * 512, wl.walk_len, 0)   # sign-sensitive values are known
+        c, o, ng, _ = O.expand_lists(walks, b * 512, wl.window, wl.n_neg, thr, alias, 0, shrink=True)
+        GU, GV, _, _ = O.sgns_grad_from_lists(U, V, c, o, ng)
+        rows_in, rows_out = O.touched_rows(c, o, ng)
+        near_zero_U[rows_in] |= np.abs(GU[rows_in]) < 1e-6
+        near_zero_V[rows_out] |= np.abs(GV[rows_out]) < 1e-6
+        ls, pc = O.sgns_adam_step_from_lists(U, V, MU, VU, MV, VV, c, o, ng, lr, 0.9, 0.999, 1e-8,
+                                             base_it + b + 1)
+        pairs += pc
+        loss_o += ls
+    G = B.gs_graph_load_csr(g.offsets.to(DEV), g.cols.to(DEV), B.GS_VALIDATE | B.GS_REQUIRE_SORTED)
+    w_in = torch.from_numpy(U0.astype(np.float32)).to(DEV)
+    w_out = torch.from_numpy(V0.astype(np.float32)).to(DEV)
+    m_in, v_in, m_out, v_out = (torch.zeros_like(w_in) for _ in range(4))
+    res = B.gs_sgns_epoch(G, alias_to_device(thr, alias), w_in, w_out, walks_per_node=1,
+                          walk_len=wl.walk_len, window=wl.window, n_neg=wl.n_neg, lr0=lr, batch_walks=512,
+                          seed=0, mode=B.GS_DETERMINISTIC | B.GS_WINDOW_SHRINK, num_batches=nb,
+                          optimizer=B.GS_OPT_ADAM, momentum=0.9, beta2=0.999, eps=1e-8,
+                          iteration_base=base_it, m_in=m_in, m_out=m_out, v_in=v_in, v_out=v_out)
+    assert res.pairs == pairs and abs(res.loss_sum - loss_o) <= 1e-3 * loss_o
+    for got, ref, near_zero in ((w_in, U, near_zero_U), (w_out, V, near_zero_V)):
+        delta = np.abs(got.cpu().numpy() - ref)
+        assert delta[~near_zero].max() <= EMB_TOL and delta.max() <= 4 * lr * nb
+    for got, ref in ((m_in, MU), (v_in, VU), (m_out, MV), (v_out, VV)):
+        assert np.abs(got.cpu().numpy() - ref).max() <= 1e-4 * np.abs(ref).max()

@@ -391,6 +391,8 @@ def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, sche
                                                c, o, ng, lr, momentum, beta2, eps, iteration_base + b + 1)
         elif mode == "det":
             ls, pc = sgns_det_from_lists(U, V, c, o, ng, lr)
+        elif mode == "det_f16":                        # binary16-valued tables, written rows rounded
+            ls, pc = sgns_det_f16_from_lists(U, V, c, o, ng, lr)
         else:
             ls, pc = sgns_seq_from_lists(U, V, c, o, ng, 2 * w, lr)
         loss_sum += ls

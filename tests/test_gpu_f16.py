@@ -168,6 +168,36 @@ def test_half_tables_reject_what_they_do_not_support(tiny):
     assert e.value.status == -6
 
 
+def test_synchronous_epoch_on_half_tables_matches_the_rounded_oracle(tiny):
+    g, off, col, thr, alias = tiny
+    n, dim = g.n_nodes, 64
+    U = O.init_rows(np.arange(n), dim, 2)
+    O.round_f16(U)
+    V = np.zeros_like(U)
+    U0 = U.copy()
+    want = O.sgns_epoch(off, col, thr, alias, U, V, walks_per_node=1, L=10, w=5, K=5, lr0=0.025,
+                        schedule="linear", batch_walks=512, seed=2, mode="det_f16")
+    G = B.gs_graph_load_csr(g.offsets.to(DEV), g.cols.to(DEV), B.GS_VALIDATE)
+    w_in = torch.empty((n, dim), dtype=torch.float16, device=DEV)
+    w_out = torch.empty_like(w_in)
+    B.gs_init_embeddings_f16(w_in, w_out, 2)
+    assert np.array_equal(w_in.cpu().numpy().astype(np.float64), U0)
+    res = B.gs_sgns_epoch(G, alias_to_device(thr, alias), w_in, w_out, walks_per_node=1, walk_len=10,
+                          window=5, n_neg=5, lr0=0.025, batch_walks=512, seed=2, mode=B.GS_DETERMINISTIC,
+                          lr_schedule=B.GS_LR_LINEAR)
+    assert res.pairs == want["pairs"] and res.steps == want["steps"]
+    assert abs(res.loss_sum - want["loss_sum"]) <= 1e-3 * want["loss_sum"]
+    # a row is rewritten once per batch that touches it; a one-ulp difference of one write feeds the
+    # later gradients, so allow a few ulps at the magnitude the value had, and ask that nearly all
+    # values are bit-equal
+    for got, ref, start in ((w_in, U, U0), (w_out, V, np.zeros_like(V))):
+        got = got.cpu().numpy().astype(np.float64)
+        scale = np.maximum(np.maximum(np.abs(ref), np.abs(start)), 1e-3)
+        assert (np.abs(got - ref) <= 4 * ulp16(scale)).all()
+        assert np.mean(got == ref) > 0.97
+    assert np.abs(V).max() > 0.01
+
+
 def test_epoch_on_half_tables_trains(tiny):
     g, off, col, thr, alias = tiny
     G = B.gs_graph_load_csr(g.offsets.to(DEV), g.cols.to(DEV), B.GS_VALIDATE | B.GS_BUILD_WALK_INDEX)

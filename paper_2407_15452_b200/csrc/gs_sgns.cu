@@ -379,6 +379,9 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
 }
 
 // ---------------------------------------------------------------- lock-free kernel
+// walks covered by one ticket of the lock-free kernel (host and device agree on the buffer size)
+__host__ __device__ __forceinline__ int hogwild_walks_per_ticket(int L) { return L <= 16 ? 32 / L : 1; }
+
 template <int DIM, typename T, bool RED, int MINB, int TC, bool NARROW>
 __global__ void __launch_bounds__(SGNS_WARPS * 32, MINB)
 sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
@@ -395,22 +398,29 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int grp = lane / LPR, sub = lane % LPR;
     const int S = 2 * w, T1 = 1 + K, SL = S * T1;
-    int32_t *W = smem + wi * (L + SL);
-    int32_t *tgt = W + L;
+    // Walks differ in length (dead ends), so warps draw walks from a shared ticket counter
+    // instead of taking a fixed share.  A ticket covers `wpt` consecutive walks: one for ordinary
+    // walks, up to 16 when walks are short (LINE: two nodes), so that the round trips of the
+    // ticket and of the walk entries are paid once per 32 entries and not once per pair.
+    const int wpt = hogwild_walks_per_ticket(L);
+    int32_t *Wbuf = smem + wi * (wpt * L + SL);
+    int32_t *tgt = Wbuf + wpt * L;
     double loss_acc = 0.0;
     unsigned long long pair_acc = 0, masked_acc = 0;
 
-    // Walks differ in length (dead ends), so warps draw the next walk from a shared ticket
-    // counter instead of taking a fixed share.
     for (;;) {
         unsigned long long tk = 0;
-        if (lane == 0) tk = atomicAdd(ticket, 1ull);
-        const int64_t a = (int64_t)__shfl_sync(0xffffffffu, tk, 0);
-        if (a >= n_walks) break;
+        if (lane == 0) tk = atomicAdd(ticket, (unsigned long long)wpt);
+        const int64_t a0 = (int64_t)__shfl_sync(0xffffffffu, tk, 0);
+        if (a0 >= n_walks) break;
+        const int nw = n_walks - a0 < wpt ? (int)(n_walks - a0) : wpt;
+        __syncwarp();
+        for (int x = lane; x < nw * L; x += 32) Wbuf[x] = walks[a0 * L + x];
+        __syncwarp();
+      for (int wq = 0; wq < nw; ++wq) {
+        const int64_t a = a0 + wq;
+        const int32_t *W = Wbuf + wq * L;
         const uint64_t id = (uint64_t)(walk_id_base + a);
-        __syncwarp();
-        for (int x = lane; x < L; x += 32) W[x] = walks[a * L + x];
-        __syncwarp();
         for (int32_t i = 0; i < L; ++i) {
             const int32_t c = W[i];
             int32_t *dp = dump_pairs ? dump_pairs + ((a * L + i) * S) * 2 : nullptr;
@@ -490,6 +500,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             }
             loss_acc += (double)loss;
         }
+      }
     }
     loss_acc = warp_sum_double(loss_acc);
     if (lane == 0) {
@@ -1016,7 +1027,7 @@ template <int DIM, typename T, bool RED, int MINB, int TC = TCH, bool NARROW = f
 static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
-    const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(a.L + SL);
+    const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(hogwild_walks_per_ticket(a.L) * a.L + SL);
     auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB, TC, NARROW>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -1148,9 +1159,7 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
     }
 #undef GS_COEF
     {
-        int64_t blocks = (n_keys + 255) / 256;                  // 8 warps x 32 keys per block
         const int64_t cap = (int64_t)sm_count() * 8 * 8;
-        if (blocks > cap) blocks = cap;
         sgns_apply_out_kernel<FPL, T><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
             w_in, w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
             lead_part, tail_part, ms_out);
@@ -1379,9 +1388,7 @@ static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scra
                      bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
     GS_CUDA_TRY(cudaGetLastError());
     {
-        int64_t blocks = (n_keys + 255) / 256;                  // 8 warps x 32 keys per block
         const int64_t cap = (int64_t)sm_count() * 8 * 8;
-        if (blocks > cap) blocks = cap;
         sgns_apply_out_kernel<FPL, float><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
             w_in, w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
             lead_part, tail_part, MomState{ nullptr, nullptr, 0.f, 0 });

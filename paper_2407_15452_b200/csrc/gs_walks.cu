@@ -1,11 +1,11 @@
-// Graph validation, table initialisation and the two walk samplers.
+// Graph validation, table initialisation, the two walk samplers and their optional indexes.
 //
-// Walks are chains of dependent random reads (offset pair, then one column), so
-// throughput comes from the number of walks in flight, not from per-walk
-// parallelism: the uniform sampler runs one walk per THREAD; the node2vec
-// sampler runs one walk per group of G lanes that evaluate G rejection rounds
-// speculatively and keep the first accepted one, which is exactly the outcome
-// of running the rounds one after another.
+// Walks are chains of dependent random reads, so throughput comes from the number of walks in
+// flight, not from per-walk parallelism: both samplers run one walk per THREAD.  The walk index
+// makes a uniform transition one random 16-byte read; the node2vec sampler flattens rejection
+// rounds and transitions into one loop and answers its neighbour test from a hashed edge set.
+// The kernels that give G lanes to a walk (speculative rejection rounds, first accepted round
+// wins) and the nested-loop kernel are kept for comparison behind gs_tune_node2vec_group.
 #include <cuda_fp16.h>
 
 #include "gs_common.cuh"
@@ -527,7 +527,7 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
     if (caps_out && my_caps) atomicAdd(caps_out, (unsigned long long)my_caps);
 }
 
-// One walk per thread (the fastest mapping measured: walks in flight matter more than lanes
+// One walk per thread, nested loops (walks in flight matter more than lanes
 // per walk).  Rejection rounds run one after another; the state carries the adjacency range of
 // the current and of the previous node, so a round costs one random read (the proposal) plus,
 // when the draw falls between the two class thresholds, a binary search in adj(prev).  With the

@@ -552,13 +552,56 @@ void gso_round_f16(double *x, int64_t n)
     for (int64_t i = 0; i < n; ++i) x[i] = rn16(x[i]);
 }
 
-/* Sequential per-pair SGD as gso_sgns_seq_from_lists, on binary16-valued tables:
- * each updated output row and each updated center row is rounded when written. */
+/* bfloat16: sign, 8 exponent bits (those of binary32), 7 fraction bits, i.e. 8 significant
+ * bits.  One rounding of the fp64 value to the nearest such number, ties to even: the value is
+ * scaled so that its 8 significant bits are the integer part, rounded with the current
+ * (to-nearest-even) mode and scaled back.  Below 2^-126 the spacing stays 2^-133 (subnormals);
+ * values beyond the largest finite bfloat16 round to infinity. */
+static double rnb16(double x)
+{
+    if (x == 0.0 || isnan(x) || isinf(x)) return x;
+    int e;
+    frexp(x, &e);                        /* |x| = m * 2^e, 0.5 <= m < 1 */
+    int q = e - 8;                       /* spacing 2^q keeps 8 significant bits */
+    if (q < -133) q = -133;
+    double r = ldexp(nearbyint(ldexp(x, -q)), q);
+    if (fabs(r) > 3.3895313892515355e38) r = (r > 0.0) ? INFINITY : -INFINITY;   /* (2 - 2^-7) * 2^127 */
+    return r;
+}
+
+void gso_round_bf16(double *x, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) x[i] = rnb16(x[i]);
+}
+
+/* Sequential per-pair SGD as gso_sgns_seq_from_lists, on tables whose values are kept in a
+ * 16-bit format (fmt 0: binary16, 1: bfloat16): each updated output row and each updated center
+ * row is rounded when written. */
+static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
+                            const int32_t *centers, const int32_t *contexts, const int32_t *negs,
+                            double lr, int fmt, double *loss_sum, int64_t *pair_count);
+
 int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
                                 int64_t n_slots, int32_t S, int32_t K,
                                 const int32_t *centers, const int32_t *contexts,
                                 const int32_t *negs, double lr,
                                 double *loss_sum, int64_t *pair_count)
+{
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 0, loss_sum, pair_count);
+}
+
+int gso_sgns_seq_bf16_from_lists(double *U, double *V, int32_t d,
+                                 int64_t n_slots, int32_t S, int32_t K,
+                                 const int32_t *centers, const int32_t *contexts,
+                                 const int32_t *negs, double lr,
+                                 double *loss_sum, int64_t *pair_count)
+{
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 1, loss_sum, pair_count);
+}
+
+static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
+                            const int32_t *centers, const int32_t *contexts, const int32_t *negs,
+                            double lr, int fmt, double *loss_sum, int64_t *pair_count)
 {
     double *acc = (double *)malloc(sizeof(double) * (size_t)d);
     if (!acc) return -1;
@@ -583,12 +626,15 @@ int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
                 loss += (k < 0) ? softplus(-f) : softplus(f);
                 for (int32_t j = 0; j < d; ++j) {
                     acc[j] += g * v[j];
-                    v[j] = rn16(v[j] - lr * g * u[j]);
+                    v[j] = fmt ? rnb16(v[j] - lr * g * u[j]) : rn16(v[j] - lr * g * u[j]);
                 }
             }
         }
         if (c >= 0)
-            for (int32_t j = 0; j < d; ++j) U[c * d + j] = rn16(U[c * d + j] - lr * acc[j]);
+            for (int32_t j = 0; j < d; ++j) {
+                double nv = U[c * d + j] - lr * acc[j];
+                U[c * d + j] = fmt ? rnb16(nv) : rn16(nv);
+            }
     }
     free(acc);
     if (loss_sum) *loss_sum = loss;

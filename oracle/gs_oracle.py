@@ -245,6 +245,38 @@ def round_f16(x):
     return x
 
 
+def round_bf16(x):
+    """In place: every value to the nearest bfloat16 (8 significant bits, ties to even)."""
+    assert x.dtype == np.float64 and x.flags.c_contiguous
+    lib().gso_round_bf16(_p(x, ctypes.c_double), ctypes.c_int64(x.size))
+    return x
+
+
+def sgns_det_bf16_from_lists(U, V, centers, contexts, negs, lr):
+    """Synchronous step on bfloat16-valued tables: full-precision step, written rows rounded."""
+    out = sgns_det_from_lists(U, V, centers, contexts, negs, lr)
+    round_bf16(U)
+    round_bf16(V)
+    return out
+
+
+def sgns_seq_bf16_from_lists(U, V, centers, contexts, negs, S, lr):
+    """Sequential per-pair SGD on bfloat16-valued tables, in place."""
+    d = U.shape[1]
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    K = negs.shape[1]
+    loss = ctypes.c_double(0.0)
+    cnt = ctypes.c_int64(0)
+    rc = lib().gso_sgns_seq_bf16_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int32(d),
+        ctypes.c_int64(len(centers)), ctypes.c_int32(S), ctypes.c_int32(K),
+        _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32),
+        ctypes.c_double(lr), ctypes.byref(loss), ctypes.byref(cnt))
+    if rc != 0:
+        raise MemoryError("oracle accumulator")
+    return float(loss.value), int(cnt.value)
+
+
 def sgns_det_f16_from_lists(U, V, centers, contexts, negs, lr):
     """Synchronous step on binary16-valued tables: full-precision step, written rows rounded
     (rows that are not written hold binary16 values already, so rounding them changes nothing)."""
@@ -393,6 +425,8 @@ def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, sche
             ls, pc = sgns_det_from_lists(U, V, c, o, ng, lr)
         elif mode == "det_f16":                        # binary16-valued tables, written rows rounded
             ls, pc = sgns_det_f16_from_lists(U, V, c, o, ng, lr)
+        elif mode == "det_bf16":
+            ls, pc = sgns_det_bf16_from_lists(U, V, c, o, ng, lr)
         else:
             ls, pc = sgns_seq_from_lists(U, V, c, o, ng, 2 * w, lr)
         loss_sum += ls

@@ -512,6 +512,41 @@ def test_binary16_rounding_matches_library_conversion_and_ties_to_even():
     assert got[-2] == 1.0 and got[-1] == 1.0 + 2.0 ** -9                      # ties go to even
 
 
+def test_bfloat16_rounding_matches_library_conversion_and_ties_to_even():
+    rng = np.random.default_rng(13)
+    # fp32-representable inputs, so that the library's float -> bfloat16 conversion is ONE rounding
+    x = np.concatenate([rng.normal(size=5000), rng.normal(size=5000) * 1e-3, rng.normal(size=2000) * 1e30,
+                        rng.normal(size=2000) * 1e-39, [0.0, -0.0, 3.3895313892515355e38, 1e-45]])
+    x = x.astype(np.float32).astype(np.float64)
+    got = O.round_bf16(x.copy())
+    want = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(got, want)
+    # ties: 1 + 2^-8 lies midway between 1 and 1 + 2^-7 and goes to the even neighbour; 1 + 3*2^-8
+    # lies midway between 1 + 2^-7 and 1 + 2^-6 and goes up to the even one
+    t = O.round_bf16(np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -40]))
+    assert t[0] == 1.0 and t[1] == 1.0 + 2.0 ** -6 and t[2] == 1.0 + 2.0 ** -7
+    # a value that a detour over fp32 would round twice: just above a bfloat16 midpoint by less than
+    # half an fp32 ulp
+    v = 1.0 + 2.0 ** -8 + 2.0 ** -30
+    assert O.round_bf16(np.array([v]))[0] == 1.0 + 2.0 ** -7
+    assert np.float64(np.float32(v)) == 1.0 + 2.0 ** -8            # fp32 first would land on the tie
+    assert np.isinf(O.round_bf16(np.array([3.4e38]))[0])
+
+
+def test_bfloat16_sequential_step_reduces_to_full_precision_plus_rounding():
+    rng = np.random.default_rng(14)
+    U = O.round_bf16(rng.normal(size=(8, 4)))
+    V = O.round_bf16(rng.normal(size=(8, 4)))
+    c = np.array([1], dtype=np.int32)
+    o = np.array([2], dtype=np.int32)
+    ng = np.array([[3, 4]], dtype=np.int32)
+    Ua, Va, Ub, Vb = U.copy(), V.copy(), U.copy(), V.copy()
+    O.sgns_seq_from_lists(Ua, Va, c, o, ng, 1, 0.3)
+    O.sgns_seq_bf16_from_lists(Ub, Vb, c, o, ng, 1, 0.3)
+    assert np.array_equal(Ub, O.round_bf16(Ua)) and np.array_equal(Vb, O.round_bf16(Va))
+    assert not np.array_equal(Vb, V)
+
+
 def test_half_precision_sequential_step_reduces_to_full_precision_plus_rounding():
     # one pair, rows touched once: the f16 result is the rounded full-precision result
     rng = np.random.default_rng(12)

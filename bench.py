@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--variants", default="",
                     help="comma list of shrink (per-position window draw), subsample (frequent-node "
                          "sub-sampling, t = 1e-5), shuffle (keyed start-node order)")
-    ap.add_argument("--table-dtype", default="f32", choices=["f32", "f16"],
+    ap.add_argument("--table-dtype", default="f32", choices=["f32", "f16", "bf16"],
                     help="storage type of the embedding tables (arithmetic is fp32 either way)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample-walks", type=int, default=16384)
@@ -435,12 +435,14 @@ def run_ours(args, wl):
     if args.stage == "walks":
         return run_walks_only(args, wl, g, G, info, dev)
     alias = torch.from_numpy(table.view(np.int64)).to(dev)
-    f16 = args.table_dtype == "f16"
-    w_in = torch.empty((n, wl.dim), dtype=torch.float16 if f16 else torch.float32, device=dev)
+    f16 = args.table_dtype != "f32"                    # a 16-bit storage format
+    tdt = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[args.table_dtype]
+    w_in = torch.empty((n, wl.dim), dtype=tdt, device=dev)
     w_out = torch.empty_like(w_in)
     seed = wl.graph_seed
-    (B.gs_init_embeddings_f16 if f16 else B.gs_init_embeddings)(w_in, w_out, seed)
-    step_fn = B.gs_sgns_step_f16 if f16 else B.gs_sgns_step
+    {"f32": B.gs_init_embeddings, "f16": B.gs_init_embeddings_f16,
+     "bf16": B.gs_init_embeddings_bf16}[args.table_dtype](w_in, w_out, seed)
+    step_fn = {"f32": B.gs_sgns_step, "f16": B.gs_sgns_step_f16, "bf16": B.gs_sgns_step_bf16}[args.table_dtype]
     if args.mode in ("momentum", "adam"):
         return run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev)
     mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,

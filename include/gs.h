@@ -334,6 +334,24 @@ GS_API gs_status gs_sgns_step_f16(void *d_w_in, void *d_w_out, int64_t n_nodes, 
                                   int32_t *d_pairs_dump, int32_t *d_negs_dump, void *stream);
 
 /*
+ * The same with bfloat16 storage (sign, the 8 exponent bits of fp32, 7 fraction bits): the other
+ * 16-bit format in use for embedding tables; the range of fp32 at 8 significant bits, where IEEE
+ * half has 11 bits and a narrow range.  The paper's tables are fp16 (Section 4.2); this variant is
+ * offered beside it.  d_w_in / d_w_out hold bfloat16 values, dim in {64, 128, 256}; rows are
+ * widened to fp32 when read, arithmetic as in gs_sgns_step, written rows rounded to nearest even.
+ * With 8 significant bits an increment below 2^-9 of the stored value is lost, so plain SGD stalls
+ * earlier than with half tables.  Modes as gs_sgns_step_f16.
+ */
+GS_API gs_status gs_init_embeddings_bf16(void *d_w_in, void *d_w_out, int64_t n_nodes,
+                                         int32_t dim, uint64_t seed, void *stream);
+GS_API gs_status gs_sgns_step_bf16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
+                                   const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                                   int32_t walk_len, int32_t window, int32_t n_neg,
+                                   const uint64_t *d_alias, float lr, uint64_t seed, int32_t mode,
+                                   double *d_loss_sum, int64_t *d_pair_count,
+                                   int32_t *d_pairs_dump, int32_t *d_negs_dump, void *stream);
+
+/*
  * Synchronous mini-batch step with Adam (Kingma & Ba 2015, Algorithm 1), the second optimizer
  * the paper keeps inside its storage (Section 3.2).  Gradients as in
  * gs_sgns_step(GS_DETERMINISTIC); only the rows of the batch move (the rows that occur as a
@@ -397,6 +415,7 @@ GS_API gs_status gs_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epo
 #define GS_WALK_NODE2VEC  1
 #define GS_TABLE_F32      0
 #define GS_TABLE_F16      1   /* tables of IEEE half, see gs_sgns_step_f16      */
+#define GS_TABLE_BF16     2   /* tables of bfloat16, see gs_sgns_step_bf16      */
 #define GS_LR_CONSTANT    0
 #define GS_LR_LINEAR      1   /* lr_b = lr0 * max(1 - b / total_batches, 1e-4) */
 #define GS_OPT_SGD        0
@@ -415,7 +434,7 @@ typedef struct gs_sgns_config {
                               /* optionally OR-ed with GS_PAIRS_FORWARD_ONLY,    */
                               /* GS_WINDOW_SHRINK                                */
     int32_t max_rounds;       /* node2vec rejection cap                          */
-    int32_t table_dtype;      /* GS_TABLE_F32 (0) or GS_TABLE_F16                */
+    int32_t table_dtype;      /* GS_TABLE_F32 (0), GS_TABLE_F16 or GS_TABLE_BF16 */
     double  p, q;             /* node2vec parameters                             */
     double  lr0;
     int64_t batch_walks;      /* walks per mini-batch (512 in the paper's runs)  */

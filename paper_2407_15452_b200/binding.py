@@ -24,7 +24,7 @@ GS_PAIRS_FORWARD_ONLY = 0x100
 GS_WINDOW_SHRINK = 0x200
 GS_WALK_UNIFORM, GS_WALK_NODE2VEC = 0, 1
 GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
-GS_TABLE_F32, GS_TABLE_F16 = 0, 1
+GS_TABLE_F32, GS_TABLE_F16, GS_TABLE_BF16 = 0, 1, 2
 GS_OPT_SGD, GS_OPT_MOMENTUM, GS_OPT_ADAM = 0, 1, 2
 
 EXPORTS = [
@@ -33,6 +33,7 @@ EXPORTS = [
     "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static", "gs_sgns_step_momentum", "gs_momentum_flush",
     "gs_init_embeddings_f16", "gs_sgns_step_f16", "gs_sgns_step_adam", "gs_build_keep_thresholds",
     "gs_subsample_walks", "gs_shuffled_starts", "gs_probe_random_reads",
+    "gs_init_embeddings_bf16", "gs_sgns_step_bf16",
 ]
 
 
@@ -243,6 +244,33 @@ def gs_sgns_step_f16(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: 
         _stream()))
 
 
+def gs_init_embeddings_bf16(w_in, w_out, seed: int):
+    """Start values of gs_init_embeddings rounded to bfloat16; tables are torch.bfloat16."""
+    ref = w_in if w_in is not None else w_out
+    n, d = ref.shape
+    _check(lib().gs_init_embeddings_bf16(_dev(w_in, torch.bfloat16, "w_in", True),
+                                        _dev(w_out, torch.bfloat16, "w_out", True),
+                                        ctypes.c_int64(n), ctypes.c_int32(d), ctypes.c_uint64(seed),
+                                        _stream()))
+
+
+def gs_sgns_step_bf16(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int, alias,
+                     lr: float, seed: int, mode: int, loss_sum=None, pair_count=None,
+                     pairs_dump=None, negs_dump=None):
+    """gs_sgns_step on torch.bfloat16 tables (fp32 arithmetic, round-to-nearest write-back)."""
+    n_nodes, dim = w_in.shape
+    n_walks, walk_len = walks.shape
+    _check(lib().gs_sgns_step_bf16(
+        _dev(w_in, torch.bfloat16, "w_in"), _dev(w_out, torch.bfloat16, "w_out"),
+        ctypes.c_int64(n_nodes), ctypes.c_int32(dim), _dev(walks, torch.int32, "walks", n_walks == 0),
+        ctypes.c_int64(n_walks), ctypes.c_int64(walk_id_base), ctypes.c_int32(walk_len),
+        ctypes.c_int32(window), ctypes.c_int32(n_neg), _dev(alias, torch.int64, "alias", n_neg == 0),
+        ctypes.c_float(lr), ctypes.c_uint64(seed), ctypes.c_int32(mode),
+        _dev(loss_sum, torch.float64, "loss_sum", True), _dev(pair_count, torch.int64, "pair_count", True),
+        _dev(pairs_dump, torch.int32, "pairs_dump", True), _dev(negs_dump, torch.int32, "negs_dump", True),
+        _stream()))
+
+
 def gs_sgns_step_static(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int, alias,
                         lr: float, seed: int, loss_sum=None, pair_count=None):
     """Deterministic SGNS step that allocates nothing on the device (fixed 32 MiB scratch inside
@@ -359,13 +387,14 @@ def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len,
                   num_batches=0, keep_thr=None, shuffle_epoch=None, optimizer=GS_OPT_SGD, momentum=0.0,
                   beta2=0.999, eps=1e-8, iteration_base=0, m_in=None, m_out=None, v_in=None, v_out=None,
                   last_in=None, last_out=None) -> EpochResult:
-    if w_in.dtype not in (torch.float32, torch.float16) or w_out.dtype != w_in.dtype:
-        raise TypeError("tables must both be float32 or both float16")
+    if w_in.dtype not in (torch.float32, torch.float16, torch.bfloat16) or w_out.dtype != w_in.dtype:
+        raise TypeError("tables must both be float32, both float16 or both bfloat16")
     tdt = w_in.dtype
     cfg = SgnsConfig(dim=w_in.shape[1], walks_per_node=walks_per_node, walk_len=walk_len,
                      window=window, n_neg=n_neg, walk_kind=walk_kind, lr_schedule=lr_schedule,
                      mode=mode, max_rounds=max_rounds,
-                     table_dtype=GS_TABLE_F16 if tdt == torch.float16 else GS_TABLE_F32, p=p, q=q, lr0=lr0,
+                     table_dtype={torch.float16: GS_TABLE_F16, torch.bfloat16: GS_TABLE_BF16}.get(tdt, GS_TABLE_F32),
+                     p=p, q=q, lr0=lr0,
                      batch_walks=batch_walks, first_batch=first_batch, num_batches=num_batches,
                      seed=seed, d_keep_thr=_dev(keep_thr, torch.int32, "keep_thr", True).value,
                      shuffle_starts=0 if shuffle_epoch is None else 1,

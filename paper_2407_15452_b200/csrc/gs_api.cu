@@ -43,6 +43,13 @@ gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, c
                         unsigned long long *masked = nullptr);
 gs_status init_embeddings_f16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
                               cudaStream_t st);
+gs_status init_embeddings_bf16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
+                               cudaStream_t st);
+gs_status sgns_step_bf16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                         const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
+                         int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
+                         unsigned long long *masked = nullptr);
 gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_out, int32_t *last_in,
                              int32_t *last_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                              int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
@@ -460,6 +467,36 @@ gs_status gs_sgns_step_f16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t
                          d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
 }
 
+// ------------------------------------------------------------------ bfloat16 tables
+gs_status gs_init_embeddings_bf16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
+                                 uint64_t seed, void *stream)
+{
+    if (n_nodes < 0) return invalid("n_nodes < 0");
+    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
+    return init_embeddings_bf16(d_w_in, d_w_out, n_nodes, dim, seed, (cudaStream_t)stream);
+}
+
+gs_status gs_sgns_step_bf16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
+                           const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                           int32_t walk_len, int32_t window, int32_t n_neg, const uint64_t *d_alias,
+                           float lr, uint64_t seed, int32_t mode, double *d_loss_sum,
+                           int64_t *d_pair_count, int32_t *d_pairs_dump, int32_t *d_negs_dump,
+                           void *stream)
+{
+    if (!d_w_in || !d_w_out) return invalid("table pointer is NULL");
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
+    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
+    if (n_walks > 0 && !d_walks) return invalid("d_walks is NULL");
+    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
+    gs_status s = check_sgns_shape(128, walk_len, window, n_neg, mode);
+    if (s != GS_OK) return s;
+    if (n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
+    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out) & 15) return invalid("tables must be 16-byte aligned");
+    return sgns_step_bf16(d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len,
+                         window, n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count,
+                         d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
+}
+
 // ------------------------------------------------------------------ momentum
 gs_status gs_sgns_step_momentum(float *d_w_in, float *d_w_out, float *d_m_in, float *d_m_out,
                                 int32_t *d_last_in, int32_t *d_last_out, int64_t n_nodes,
@@ -635,8 +672,11 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
 {
     if (!g || !cfg || !h_out) return invalid("null pointer");
     if (!d_w_in || !d_w_out) return invalid("table pointer is NULL");
-    if (cfg->table_dtype != GS_TABLE_F32 && cfg->table_dtype != GS_TABLE_F16) return invalid("unknown table_dtype");
-    const bool f16 = cfg->table_dtype == GS_TABLE_F16;
+    if (cfg->table_dtype != GS_TABLE_F32 && cfg->table_dtype != GS_TABLE_F16 &&
+        cfg->table_dtype != GS_TABLE_BF16)
+        return invalid("unknown table_dtype");
+    const bool f16 = cfg->table_dtype != GS_TABLE_F32;         // a 16-bit storage format
+    const bool bf16 = cfg->table_dtype == GS_TABLE_BF16;
     if (f16 && !dim_ok_f16(cfg->dim)) { set_error("dim %d not supported with half-precision tables (64, 128, 256)", cfg->dim); return GS_ERR_UNSUPPORTED; }
     gs_status s = check_sgns_shape(f16 ? 128 : cfg->dim, cfg->walk_len, cfg->window, cfg->n_neg, cfg->mode);
     if (s != GS_OK) return s;
@@ -767,6 +807,11 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
                                        cfg->momentum, cfg->beta2, cfg->eps, cfg->iteration_base + b + 1,
                                        cfg->seed, cfg->mode & ~0xFF, &ctr->loss, (int64_t *)&ctr->pairs,
                                        s_sgns));
+            else if (bf16)
+                EP_CALL(sgns_step_bf16(d_w_in, d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
+                                       cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
+                                       cfg->seed, cfg->mode, &ctr->loss, (int64_t *)&ctr->pairs, nullptr,
+                                       nullptr, s_sgns, &ctr->masked));
             else if (f16)
                 EP_CALL(sgns_step_f16(d_w_in, d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
                                       cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,

@@ -18,7 +18,9 @@
 // per distinct row sums that row's contributions in index order and writes the
 // row once.  No floating-point atomics anywhere on this path.
 #include <mutex>
+#include <type_traits>
 
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "gs_common.cuh"
@@ -110,6 +112,46 @@ __device__ __forceinline__ void row_store(__half *__restrict__ tab, int64_t r, i
             __half2 *h = reinterpret_cast<__half2 *>(&t);
             h[0] = __floats2half2_rn(x.v[4 * q], x.v[4 * q + 1]);
             h[1] = __floats2half2_rn(x.v[4 * q + 2], x.v[4 * q + 3]);
+            reinterpret_cast<uint2 *>(p)[q * 32 + lane] = t;
+        }
+    }
+}
+
+// ... and for tables stored as bfloat16.
+template <int FPL>
+__device__ __forceinline__ Row<FPL> row_load(const __nv_bfloat16 *__restrict__ tab, int64_t r, int lane)
+{
+    Row<FPL> out;
+    const __nv_bfloat16 *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 2) {
+        const float2 f = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162 *>(p)[lane]);
+        out.v[0] = f.x; out.v[1] = f.y;
+    } else {
+        static_assert(FPL % 4 == 0, "bfloat16 tables need dim 64, 128 or 256");
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q) {
+            const uint2 t = reinterpret_cast<const uint2 *>(p)[q * 32 + lane];
+            const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&t);
+            const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+            out.v[4 * q] = a.x; out.v[4 * q + 1] = a.y; out.v[4 * q + 2] = b.x; out.v[4 * q + 3] = b.y;
+        }
+    }
+    return out;
+}
+
+template <int FPL>
+__device__ __forceinline__ void row_store(__nv_bfloat16 *__restrict__ tab, int64_t r, int lane, const Row<FPL> &x)
+{
+    __nv_bfloat16 *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 2) {
+        reinterpret_cast<__nv_bfloat162 *>(p)[lane] = __floats2bfloat162_rn(x.v[0], x.v[1]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q) {
+            uint2 t;
+            __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&t);
+            h[0] = __floats2bfloat162_rn(x.v[4 * q], x.v[4 * q + 1]);
+            h[1] = __floats2bfloat162_rn(x.v[4 * q + 2], x.v[4 * q + 3]);
             reinterpret_cast<uint2 *>(p)[q * 32 + lane] = t;
         }
     }
@@ -207,6 +249,20 @@ __device__ __forceinline__ void unpack16h(const uint4 &t, float *v)
 #pragma unroll
     for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(h[j]); v[2 * j] = f.x; v[2 * j + 1] = f.y; }
 }
+__device__ __forceinline__ void unpack16b(const uint4 &t, float *v)
+{
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&t);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { const float2 f = __bfloat1622float2(h[j]); v[2 * j] = f.x; v[2 * j + 1] = f.y; }
+}
+__device__ __forceinline__ uint4 pack16(const float *v, const __nv_bfloat16 *)
+{
+    uint4 t;
+    __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&t);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) h[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);   // round to nearest even
+    return t;
+}
 __device__ __forceinline__ uint4 pack16(const float *v, const __half *)
 {
     uint4 t;
@@ -228,7 +284,8 @@ __device__ __forceinline__ Row<RowGeom<DIM, T, NARROW>::FPL> grow_load(const T *
     for (int q = 0; q < G::FPL / G::PER16; ++q) {
         const uint4 t = p[q * G::LPR + sub];
         if constexpr (sizeof(T) == 4) unpack16(t, out.v + G::PER16 * q);
-        else unpack16h(t, out.v + G::PER16 * q);
+        else if constexpr (std::is_same<T, __half>::value) unpack16h(t, out.v + G::PER16 * q);
+        else unpack16b(t, out.v + G::PER16 * q);
     }
     return out;
 }
@@ -275,6 +332,9 @@ __device__ __forceinline__ void grow_red_add(float *__restrict__ tab, int64_t r,
 }
 template <int DIM, bool NARROW>
 __device__ __forceinline__ void grow_red_add(__half *, int64_t, int, const Row<RowGeom<DIM, __half, NARROW>::FPL> &) {}
+template <int DIM, bool NARROW>
+__device__ __forceinline__ void grow_red_add(__nv_bfloat16 *, int64_t, int,
+                                             const Row<RowGeom<DIM, __nv_bfloat16, NARROW>::FPL> &) {}
 
 // sum over the LPR lanes that hold one row (identical bits on each of them)
 template <int LPR>
@@ -1055,7 +1115,9 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 template <int DIM, typename T, bool RED>
 static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
-    if constexpr (sizeof(T) == 2)            // half rows: 3 rows per group in flight, 6 blocks (measured)
+    if constexpr (std::is_same<T, __nv_bfloat16>::value)   // 6 blocks would spill; 5 blocks of 96 registers
+        return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL > 8 ? 4 : 5), 3>(a, st);
+    else if constexpr (sizeof(T) == 2)       // half rows: 3 rows per group in flight, 6 blocks (measured)
         return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL > 8 ? 4 : 6), 3>(a, st);
     else {
         // few targets per position (fewer than two wide chunks): 16 bytes per lane, one chunk
@@ -1195,7 +1257,7 @@ static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
     if (mode == GS_DETERMINISTIC) return run_deterministic<DIM, T>(a, st);
     if (mode == GS_HOGWILD) return run_hogwild<DIM, T, false>(a, st);
     if constexpr (sizeof(T) == 4) return run_hogwild<DIM, T, true>(a, st);
-    set_error("GS_HOGWILD_RED is not available for half-precision tables");
+    set_error("GS_HOGWILD_RED is not available for 16-bit tables");
     return GS_ERR_UNSUPPORTED;
 }
 
@@ -1237,6 +1299,27 @@ gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, c
         case 256: return run_mode<256, __half>(a, mode, st);
         default:
             set_error("dim %d not supported with half-precision tables (64, 128, 256)", dim);
+            return GS_ERR_UNSUPPORTED;
+    }
+}
+
+// Tables stored as bfloat16: as above with the other 16-bit format.
+gs_status sgns_step_bf16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                         const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
+                         int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
+                         unsigned long long *masked)
+{
+    if (n_walks == 0) return GS_OK;
+    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked };
+    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
+    switch (dim) {
+        case 64: return run_mode<64, __nv_bfloat16>(a, mode, st);
+        case 128: return run_mode<128, __nv_bfloat16>(a, mode, st);
+        case 256: return run_mode<256, __nv_bfloat16>(a, mode, st);
+        default:
+            set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;
     }
 }

@@ -6,6 +6,7 @@
 // rounds and transitions into one loop and answers its neighbour test from a hashed edge set.
 // The kernels that give G lanes to a walk (speculative rejection rounds, first accepted round
 // wins) and the nested-loop kernel are kept for comparison behind gs_tune_node2vec_group.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "gs_common.cuh"
@@ -128,6 +129,44 @@ init_rows_f16_kernel(__half *__restrict__ w, int64_t n_rows, int32_t dim, uint64
         p[0] = __floats2half2_rn(a, b);
         p[1] = __floats2half2_rn(c, d);
     }
+}
+
+// ... and rounded to bfloat16 (round to nearest even).
+__global__ void __launch_bounds__(256)
+init_rows_bf16_kernel(__nv_bfloat16 *__restrict__ w, int64_t n_rows, int32_t dim, uint64_t seed)
+{
+    const int32_t quads = dim >> 2;
+    const int64_t total = n_rows * quads;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const float inv_d = 1.0f / (float)dim;
+    for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < total; x += stride) {
+        const int64_t row = x / quads;
+        const uint32_t qd = (uint32_t)(x - row * quads);
+        const uint4 r = draw(seed, (uint64_t)row, qd, TAG_INIT, 0);
+        const float a = ((float)(r.x >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        const float b = ((float)(r.y >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        const float c = ((float)(r.z >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        const float d = ((float)(r.w >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
+        __nv_bfloat162 *p = reinterpret_cast<__nv_bfloat162 *>(w) + 2 * x;
+        p[0] = __floats2bfloat162_rn(a, b);
+        p[1] = __floats2bfloat162_rn(c, d);
+    }
+}
+
+gs_status init_embeddings_bf16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
+                               cudaStream_t st)
+{
+    if (w_in && n > 0) {
+        const int64_t total = n * (dim >> 2);
+        int64_t blocks = (total + 255) / 256;
+        const int64_t cap = (int64_t)sm_count() * 32;
+        if (blocks > cap) blocks = cap;
+        init_rows_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((__nv_bfloat16 *)w_in, n, dim, seed);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    if (w_out && n > 0)
+        GS_CUDA_TRY(cudaMemsetAsync(w_out, 0, sizeof(__nv_bfloat16) * (size_t)n * (size_t)dim, st));
+    return GS_OK;
 }
 
 gs_status init_embeddings_f16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,

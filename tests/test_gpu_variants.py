@@ -101,6 +101,15 @@ def test_shuffled_starts_bit_exact_and_bijective(n):
     assert B.gs_shuffled_starts(n, 1, 0, 5, 0, DEV).numel() == 0
 
 
+def test_shuffled_starts_at_the_largest_node_count():
+    # 2^31 - 1 nodes: 32-bit halves in the network, ids beyond 2^31 as walk ids; sampled ranges only
+    n = 2**31 - 1
+    for first in (0, n - 500, 5 * n + 12345):
+        got = B.gs_shuffled_starts(n, 77, 3, first, 4096, DEV).cpu().numpy()
+        assert np.array_equal(got, O.shuffled_starts(n, 77, 3, first, 4096))
+        assert got.min() >= 0 and len(np.unique(got)) == 4096
+
+
 # ---------------------------------------------------------------- epoch with every variant on
 def test_epoch_with_shuffle_subsampling_and_shrinking_matches_oracle(tiny):
     wl, g, off, col, thr, alias = tiny

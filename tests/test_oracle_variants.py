@@ -160,6 +160,14 @@ def test_shuffle_is_a_bijection_of_the_node_range(n):
         assert np.array_equal(np.sort(st), np.arange(n, dtype=np.int32))
 
 
+def test_shuffle_stays_injective_at_the_largest_node_count():
+    n = 2**31 - 1
+    st = O.shuffled_starts(n, 5, 1, 0, 200_000).astype(np.int64)
+    assert st.min() >= 0 and st.max() < n and len(np.unique(st)) == len(st)
+    # images are spread over the whole range
+    assert chi2_uniform_ok(np.bincount(st * 16 // n, minlength=16))
+
+
 def test_shuffle_depends_on_seed_and_epoch_and_wraps_over_walk_ids():
     n = 5000
     a = O.shuffled_starts(n, 1, 0, 0, n)

@@ -835,7 +835,7 @@ momentum_stamp_kernel(int32_t *__restrict__ last, int64_t n_rows, int32_t iter)
 constexpr int RUN_CUT = 256;
 
 template <int FPL, typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
                       const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
                       const uint32_t *__restrict__ vals, const float *__restrict__ gbuf,
@@ -876,17 +876,35 @@ sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
             }
         };
 
-        for (int64_t s0 = base; s0 < end; s0 += 32) {
-            const int64_t i = s0 + lane;
-            const uint32_t my_key = i < end ? keys[i] : 0xFFFFFFFFu;
-            const bool usable = my_key < n_nodes;                     // sorted: usable lanes are a prefix
-            float g = 0.f;
-            int32_t c = 0;
-            if (usable) {
-                const uint32_t idx = vals[i];
+        // The metadata of a chunk of 32 contributions is a chain of two dependent reads (sorted key
+        // and contribution index, then coefficient and center node).  It is fetched two chunks
+        // ahead (first link) and one chunk ahead (second link), so that the rows of the current
+        // chunk never wait for it.
+        auto link1 = [&](int64_t i, uint32_t &key, uint32_t &idx) {
+            key = i < end ? keys[i] : 0xFFFFFFFFu;
+            idx = i < end ? vals[i] : 0u;
+        };
+        auto link2 = [&](uint32_t key, uint32_t idx, float &g, int32_t &c) {
+            g = 0.f;
+            c = 0;
+            if (key < n_nodes) {
                 g = gbuf[idx];
                 c = walks[idx / (uint32_t)SL];
             }
+        };
+        uint32_t my_key, key1, idx0, idx1;
+        float g;
+        int32_t c;
+        link1(base + lane, my_key, idx0);
+        link1(base + 32 + lane, key1, idx1);
+        link2(my_key, idx0, g, c);
+        for (int64_t s0 = base; s0 < end; s0 += 32) {
+            uint32_t key2, idx2;
+            link1(s0 + 64 + lane, key2, idx2);                        // two chunks ahead
+            float g1;
+            int32_t c1;
+            link2(key1, idx1, g1, c1);                                // one chunk ahead
+            const bool usable = my_key < n_nodes;                     // sorted: usable lanes are a prefix
             uint32_t before = __shfl_up_sync(0xffffffffu, my_key, 1);
             if (lane == 0) before = carry_key;
             carry_key = __shfl_sync(0xffffffffu, my_key, 31);
@@ -923,6 +941,8 @@ sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
                 }
             }
             if (n < 32) break;                                        // the rest is not ours
+            my_key = key1; g = g1; c = c1;
+            key1 = key2; idx1 = idx2;
         }
         if (have) close_run(end < (int64_t)n_keys && keys[end] == cur_key);
     }

@@ -15,6 +15,10 @@ for the SGNS kernel (the dominant one); `walk` gives the walk sampler's own figu
 With --gpus N every rank runs an independent replica of the same workload on its own GPU
 (the path has no exchange step); the value is the sum over ranks divided by the slowest
 rank's time.
+
+The default single-GPU run also carries `per_config`: short legs over the other named
+workloads and the synchronous mode (device-resident timing only), each with its own roofline
+block; --no-per-config leaves them out.
 """
 from __future__ import annotations
 
@@ -64,6 +68,10 @@ def parse_args():
                     help="node2vec kernel: 0 flattened loop, 1 nested loops, 2..32 lanes per walk")
     ap.add_argument("--stage", default="all", choices=["all", "walks"],
                     help="'walks' times the walk sampler alone (no tables are allocated)")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="skip the short legs over the other workloads that the default run adds")
+    ap.add_argument("--cpu-workers", type=int, default=0,
+                    help="processes of the all-cores oracle leg (0: one per usable core, at most 64)")
     return ap.parse_args()
 
 
@@ -122,6 +130,9 @@ def measured_peak_gbs():
         except Exception:
             pass
     return 6650.0, "fallback"
+
+
+NOMINAL_HBM_GBS = 8000.0      # the device's nominal HBM3e bandwidth, for context
 
 
 def recorded_traffic(kernel, workload):
@@ -206,18 +217,78 @@ def oracle_sample(wl, off, col, table, n_walks, base, seed):
     return pairs, steps, {"walk_s": t1 - t0, "expand_s": t2 - t1, "sgns_s": t4 - t3}
 
 
+def _oracle_worker(job):
+    """One process of the all-cores oracle leg: maps the shared inputs and runs the oracle, as it
+    stands, on its own range of walk ids (its own copy of the touched rows).  Returns
+    (pairs, steps, seconds of oracle work)."""
+    folder, wl_name, n_walks, base, seed, start_at = job
+    from paper_2407_15452_b200.workloads import WORKLOADS
+    wl = WORKLOADS[wl_name]
+    off = np.load(os.path.join(folder, "off.npy"), mmap_mode="r")
+    col = np.load(os.path.join(folder, "col.npy"), mmap_mode="r")
+    table = np.load(os.path.join(folder, "alias.npy"), mmap_mode="r")
+    n_nodes = len(off) - 1
+    # the sample's own part of the alias table is small next to the CSR: read it whole
+    table = np.ascontiguousarray(table)
+    oracle_sample(wl, off, col, table, 8, base, seed)            # loads the library, touches pages
+    while time.time() < start_at:                                 # all processes start together
+        time.sleep(0.005)
+    p, st, t = oracle_sample(wl, off, col, table, n_walks, base, seed)
+    return p, st, t["walk_s"] + t["expand_s"] + t["sgns_s"], n_nodes
+
+
+def oracle_all_cores(wl, off, col, table, seed, workers, walks_each):
+    """The oracle on all host cores: `workers` processes (spawned, so that none inherits a CUDA
+    context), each running the single-threaded oracle on a disjoint range of walk ids with its own
+    copy of the rows it touches.  Rate = pairs of all processes / slowest process."""
+    import multiprocessing as mp
+    import shutil
+    usable = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    if workers <= 0:
+        workers = min(usable, 64)
+    root = "/dev/shm" if os.path.isdir("/dev/shm") and os.access("/dev/shm", os.W_OK) else None
+    folder = tempfile.mkdtemp(prefix="gs_oracle_", dir=root)
+    try:
+        np.save(os.path.join(folder, "off.npy"), off)
+        np.save(os.path.join(folder, "col.npy"), col)
+        np.save(os.path.join(folder, "alias.npy"), table)
+        start_at = time.time() + 3.0 + 0.1 * workers
+        jobs = [(folder, wl.name, walks_each, (1 << 20) + k * walks_each, seed, start_at) for k in range(workers)]
+        with mp.get_context("spawn").Pool(workers) as pool:
+            res = pool.map(_oracle_worker, jobs, chunksize=1)
+    finally:
+        shutil.rmtree(folder, ignore_errors=True)
+    pairs = sum(r[0] for r in res)
+    steps = sum(r[1] for r in res)
+    slowest = max(r[2] for r in res)
+    return {"value": pairs / slowest, "unit": UNIT, "cores": workers, "host_cores": usable,
+            "kind": "oracle, one single-threaded process per core on disjoint walk-id ranges",
+            "sample": f"{workers} x {walks_each} walks ({slowest:.1f} s for the slowest process)",
+            "walk_steps": steps}
+
+
 def run_reference(args, wl):
-    """--impl reference: the CPU oracle, as it stands, on the host cores."""
+    """--impl reference: the CPU oracle, as it stands, on the host cores.  Nothing of the CUDA
+    library is loaded: the alias table comes from the oracle's own builder."""
     import torch
+    from oracle import gs_oracle as O
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     device = "cuda" if torch.cuda.is_available() else "cpu"
     scale = args.scale if device == "cuda" else min(args.scale, 0.02)
-    g, table, info = build_inputs(wl, scale, device)
+    t0 = time.time()
+    g = wl.make_graph(device=device, scale=scale)
+    deg = g.degrees()
+    info = {"n_nodes": g.n_nodes, "n_edges": g.n_edges, "max_degree": int(deg.max()),
+            "frac_isolated": float((deg == 0).double().mean()), "graph_s": round(time.time() - t0, 1)}
+    t0 = time.time()
+    thr, alias = O.build_alias(deg.cpu().numpy().astype(np.float64), 0.75)
+    table = (alias.astype(np.uint64) << np.uint64(32)) | thr.astype(np.uint64)
+    info["alias_s"] = round(time.time() - t0, 1)
     off = g.offsets.cpu().numpy().astype(np.int64)
     col = g.cols.cpu().numpy()
-    del g
+    del g, deg, thr, alias
     n = min(max(args.cpu_sample_walks // 8, 1), 1024)
     for s in range(args.warmup):
         oracle_sample(wl, off, col, table, n, s * n, wl.graph_seed)
@@ -248,10 +319,11 @@ def walk_kernel_name(wl, indexed):
 
 
 def sync_step_launches(n_nodes, extra=0):
-    """Kernels of one synchronous batch: walks, coefficients, three per radix pass of 8 bits over
-    keys below 2 n_nodes, apply (output rows, fix-up, input rows), loss reduction."""
+    """Kernels of one synchronous batch: walks; targets and three per radix pass of at most 8 bits
+    over keys below 2 n_nodes (the table-independent part); coefficients, apply (output rows,
+    fix-up, input rows), loss reduction."""
     passes = ((2 * n_nodes).bit_length() + 7) // 8
-    return 1 + 1 + 3 * passes + 3 + 1 + extra
+    return 1 + 1 + 3 * passes + 1 + 3 + 1 + extra
 
 
 def parse_variants(args):
@@ -268,6 +340,26 @@ def keep_thresholds_device(g, dev, t=1e-5):
     from paper_2407_15452_b200 import binding as B
     thr = B.gs_build_keep_thresholds(g.degrees().cpu().numpy().astype(np.float64), t)
     return torch.from_numpy(thr.view(np.int32)).to(dev)
+
+
+def probe_random_reads(n_records, n_reads, dev):
+    """Independent random 16-byte reads per second over a buffer of n_records records, measured by
+    the benchmark's own probe library (libbench_probe.so, built from bench_probe.cu)."""
+    import ctypes
+    import torch
+    so = ROOT / "libbench_probe.so"
+    if not so.exists():
+        return None
+    lib = ctypes.CDLL(str(so))
+    buf = torch.zeros(n_records * 4, dtype=torch.int32, device=dev)
+    done, ms = ctypes.c_int64(0), ctypes.c_float(0.0)
+    rc = lib.bench_probe_random_reads(ctypes.c_void_p(buf.data_ptr()), ctypes.c_int64(n_records),
+                                      ctypes.c_int64(n_reads), ctypes.byref(done), ctypes.byref(ms),
+                                      ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    del buf
+    if rc != 0 or ms.value <= 0:
+        return None
+    return done.value / (ms.value * 1e-3)
 
 
 # ---------------------------------------------------------------------------- walk sampler alone
@@ -319,8 +411,9 @@ def run_walks_only(args, wl, g, G, info, dev):
     indexed = "walk_index_bytes" in info
     payload = walk_bytes(st, wl.offsets64, indexed) / (ms * 1e-3) / 1e9
     granule = walk_granule_bytes(st, indexed) / (ms * 1e-3) / 1e9
-    # ceiling of one isolated random read per transition, measured on the same index in this run
-    read_rate = B.gs_probe_random_reads(G, 1 << 28) if indexed else None
+    # ceiling of one isolated random read per transition, measured in this run on a buffer of the
+    # walk index's size (16 bytes per CSR entry)
+    read_rate = probe_random_reads(g.n_edges, 1 << 28, dev) if indexed else None
     print(json.dumps({
         "metric": "walk_steps_per_s", "value": st / (ms * 1e-3), "unit": "walk-steps/s", "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
@@ -391,7 +484,7 @@ def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
         "metric": METRIC, "value": pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "gpu_launches": sync_step_launches(n, 0 if adam else 2) * args.steps,   # momentum: keys pass + catch-up
+        "gpu_launches": sync_step_launches(n, 0 if adam else 1) * args.steps,   # momentum: + catch-up
         "clocks": clocks, "mean_loss": loss.item() / max(pairs, 1),
         "config": {"workload": wl.name, "mode": args.mode, "momentum": mu, "lr": lr, "batch_walks": bw,
                    "walk_len": wl.walk_len, "window": wl.window, "n_neg": wl.n_neg, "dim": wl.dim,
@@ -405,20 +498,18 @@ def run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev):
 
 
 # ---------------------------------------------------------------------------- our arm
-def run_ours(args, wl):
+def fractions(gbs, peak):
+    """The same rate against the measured copy bandwidth and against the nominal figure."""
+    return {"frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+
+
+def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
+    """Builds the inputs of `wl`, times the path as `args` says and returns the result line as a
+    dict (rank 0; None elsewhere).  Frees everything it allocated on the device."""
     import torch
     import torch.distributed as dist
     from paper_2407_15452_b200 import binding as B
     from paper_2407_15452_b200 import replicas
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    B.lib()                                            # fail loudly if the library is missing
 
     g, table, info = build_inputs(wl, args.scale, dev)
     n = g.n_nodes
@@ -459,9 +550,12 @@ def run_ours(args, wl):
     if (mode & 0xFF) == B.GS_DETERMINISTIC:
         bw = min(bw, 512)
     nb_total = (total_walks + bw - 1) // bw
+    lr_schedule = B.GS_LR_LINEAR if wl.lr_schedule == "linear" else B.GS_LR_CONSTANT
     ekw = dict(walks_per_node=wl.walks_per_node, walk_len=wl.walk_len, window=wl.window,
                n_neg=wl.n_neg, lr0=wl.lr0, batch_walks=bw, seed=seed, mode=mode, walk_kind=kind,
-               p=wl.p, q=wl.q, keep_thr=keep_thr, shuffle_epoch=0 if "shuffle" in variants else None)
+               p=wl.p, q=wl.q, keep_thr=keep_thr, shuffle_epoch=0 if "shuffle" in variants else None,
+               lr_schedule=lr_schedule)
+    n_steps = min(args.steps, max(nb_total - args.warmup, 1))   # a small workload has fewer batches
 
     def barrier():
         torch.cuda.synchronize()
@@ -490,9 +584,9 @@ def run_ours(args, wl):
     # One replica takes consecutive mini-batches: the K timed steps are ONE call of the epoch
     # driver over K batches, as a user runs it (walk generation of batch b+1 then overlaps the
     # update of batch b).  Several replicas interleave their batches, so they call per step.
-    one_call = world == 1 and args.warmup + args.steps <= nb_total
-    calls = [(args.warmup, args.steps)] if one_call else \
-            [(batch_of(args.warmup + s), 1) for s in range(args.steps)]
+    one_call = world == 1 and args.warmup + n_steps <= nb_total
+    calls = [(args.warmup, n_steps)] if one_call else \
+            [(batch_of(args.warmup + s), 1) for s in range(n_steps)]
     for b, nb in calls:
         r = B.gs_sgns_epoch(G, alias, w_in, w_out, first_batch=b, num_batches=nb, **ekw)
         pairs += r.pairs
@@ -508,7 +602,7 @@ def run_ours(args, wl):
 
     # ---- end to end: host inputs in, result out, same C-ABI calls ---------------------------
     e2e_pairs, e2e_s = 0, float("nan")
-    if not args.no_e2e:
+    if with_e2e:
         h_starts = torch.empty(bw, dtype=torch.int32).pin_memory()
         d_starts = torch.empty(bw, dtype=torch.int32, device=dev)
         d_walks = torch.empty((bw, wl.walk_len), dtype=torch.int32, device=dev)
@@ -537,11 +631,11 @@ def run_ours(args, wl):
             return int(h_res[1:2].view(torch.int64).item())
 
         for s in range(min(args.warmup, 2)):
-            e2e_step(args.warmup + args.steps + s)
+            e2e_step(args.warmup + n_steps + s)
         barrier()
         t0 = time.perf_counter()
-        for s in range(args.steps):
-            e2e_pairs += e2e_step(args.warmup + args.steps + 2 + s)
+        for s in range(n_steps):
+            e2e_pairs += e2e_step(args.warmup + n_steps + 2 + s)
         barrier()
         e2e_s = time.perf_counter() - t0
 
@@ -549,9 +643,10 @@ def run_ours(args, wl):
     (ms, e2e_s), (pairs_all, steps_all, e2e_pairs_all) = replicas.reduce_timing(
         [ms, e2e_s], [pairs, steps, e2e_pairs], device=dev)
 
+    out = None
     if rank == 0:
         peak, peak_kind = measured_peak_gbs()
-        launches = args.steps                                     # SGNS launches on this rank
+        launches = n_steps                                        # SGNS launches on this rank
         positions = steps + walks_done                            # walk entries = center positions
         sgns_bytes = algorithmic_bytes(pairs, positions, wl.dim, wl.n_neg, 2 if f16 else 4) / launches
         sgns_ms = ms_sgns / launches
@@ -564,41 +659,50 @@ def run_ours(args, wl):
         wbytes = walk_bytes(w_steps, wl.offsets64, indexed) / w_n
         gbytes = walk_granule_bytes(w_steps, indexed) / w_n
         walk_ms = w_ms / w_n
-        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if (mode & 0xFF) and not f16 else None
+        lock_free = (mode & 0xFF) != B.GS_DETERMINISTIC
+        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if lock_free and not f16 else None
         traffic = per_pair * pairs / launches if per_pair else None
+        payload_gbs = wbytes / (walk_ms * 1e-3) / 1e9
+        granule_gbs = gbytes / (walk_ms * 1e-3) / 1e9
         out = {
             "metric": METRIC, "value": pairs_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "steps": n_steps, "warmup": args.warmup, "ms_per_step": ms / n_steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": wl.name, "mode": args.mode, "table_dtype": args.table_dtype,
                        "batch_walks": bw,
                        "walk_kind": wl.walk_kind, "walk_len": wl.walk_len, "window": wl.window,
                        "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale, "variants": sorted(variants),
-                       "l2": "tables (2 x n x dim x 4 B) and CSR far exceed the 126 MB L2; no flush",
+                       "l2": "tables (2 x n x dim x 4 B) and CSR far exceed the 126 MB L2; no flush"
+                             if 2 * n * wl.dim * (2 if f16 else 4) > (1 << 30) else
+                             "every step takes a new batch of walks; tables of this workload are "
+                             "smaller than 1 GB, rows may stay in the 126 MB L2 between steps",
                        "timed_region": "one gs_sgns_epoch call over the K batches" if one_call else
                                        "one gs_sgns_epoch call per batch",
                        "multi_gpu": "replicas only", **info},
-            "gpu_launches": ((2 if (mode & 0xFF) else sync_step_launches(n))
-                             + len(variants & {"shuffle", "subsample"})) * args.steps,
+            "gpu_launches": ((2 if lock_free else sync_step_launches(n))
+                             + len(variants & {"shuffle", "subsample"})) * n_steps,
             "mean_loss": loss / max(pairs, 1),
             "walk_steps_per_s": steps_all / (ms * 1e-3),
             "clocks": clocks,
-            "e2e": {"value": e2e_pairs_all / e2e_s, "unit": UNIT,
-                    "h2d_bytes_per_step": 4 * bw, "d2h_bytes_per_step": 16},
             "roofline": {"bound": "hbm",
-                         "kernel": "sgns_hogwild_kernel" if (mode & 0xFF) else "sgns (coef+sort+apply)",
-                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "kernel": "sgns_hogwild_kernel" if lock_free else "synchronous step (coefficients, sort, apply)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", **fractions(achieved, peak),
                          "peak_kind": f"of {peak_kind}", "traffic": traffic,
                          "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (ms_sgns * 1e-3)},
             "walk": {"kernel": walk_kernel_name(wl, indexed),
                      "walk_steps_per_s_kernel": w_steps / (w_ms * 1e-3), "ms_per_launch": walk_ms,
-                     "payload_gbs": wbytes / (walk_ms * 1e-3) / 1e9,
-                     "payload_frac": wbytes / (walk_ms * 1e-3) / 1e9 / peak,
-                     "granule_gbs": gbytes / (walk_ms * 1e-3) / 1e9,
-                     "granule_frac": gbytes / (walk_ms * 1e-3) / 1e9 / peak},
+                     "payload_gbs": payload_gbs, "payload_frac": payload_gbs / peak,
+                     "payload_frac_of_nominal_8TBs": payload_gbs / NOMINAL_HBM_GBS,
+                     "granule_gbs": granule_gbs, "granule_frac": granule_gbs / peak,
+                     "granule_frac_of_nominal_8TBs": granule_gbs / NOMINAL_HBM_GBS,
+                     "note": "payload = CSR bytes read + entries stored (the stated metric); granule "
+                             "counts the 64 bytes DRAM moves per isolated read (supplementary)"},
         }
-        if not args.no_cpu_baseline and world == 1:
+        if with_e2e:
+            out["e2e"] = {"value": e2e_pairs_all / e2e_s, "unit": UNIT,
+                          "h2d_bytes_per_step": 4 * bw, "d2h_bytes_per_step": 16}
+        if with_cpu and world == 1:
             off = g.offsets.cpu().numpy().astype(np.int64)
             col = g.cols.cpu().numpy()
             p, st, t = oracle_sample(wl, off, col, table, args.cpu_sample_walks, 0, seed)
@@ -608,6 +712,66 @@ def run_ours(args, wl):
                 "sample": f"first {args.cpu_sample_walks} walks of the workload: walks, pair/negative "
                           f"expansion, sequential SGNS on the touched rows ({tot:.1f} s)",
                 "walk_steps_per_s": st / t["walk_s"], "sgns_pair_updates_per_s": p / t["sgns_s"]}
+            try:
+                out["cpu_baseline"]["all_cores"] = oracle_all_cores(wl, off, col, table, seed,
+                                                                    args.cpu_workers, 1024)
+            except Exception as e:                       # the single-core figure stands on its own
+                out["cpu_baseline"]["all_cores"] = {"unavailable": f"{type(e).__name__}: {e}"}
+    G.close()
+    del w_in, w_out, alias, g, G
+    B.gs_release_workspace()
+    torch.cuda.empty_cache()
+    return out
+
+
+# The default run's short legs: (workload, mode, steps, warm-up).  The synchronous mode takes
+# batches of 512 walks, so its legs run a few hundred steps inside one call of the epoch driver;
+# the tiny workload is its whole epoch (20 batches).
+PER_CONFIG_LEGS = [
+    ("tiny_deepwalk", "deterministic", 17, 3),
+    ("deepwalk_medium", "deterministic", 300, 5),
+    ("deepwalk_medium", "hogwild", 8, 3),
+    ("node2vec_4m", "hogwild", 6, 3),
+    ("rmat_billion", "hogwild", 10, 3),
+]
+
+
+def run_ours(args, wl):
+    import argparse
+    import torch
+    import torch.distributed as dist
+    from paper_2407_15452_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()                                            # fail loudly if the library is missing
+
+    plain = (args.workload == "deepwalk_large" and args.mode == "hogwild" and args.stage == "all"
+             and args.table_dtype == "f32" and not args.variants and args.scale == 1.0)
+    out = run_leg(args, wl, dev, rank, world, local, with_e2e=not args.no_e2e,
+                  with_cpu=not args.no_cpu_baseline)
+    if out is not None and plain and world == 1 and not args.no_per_config:
+        legs = {}
+        for name, mode, steps, warmup in PER_CONFIG_LEGS:
+            from paper_2407_15452_b200.workloads import WORKLOADS
+            largs = argparse.Namespace(**{**vars(args), "workload": name, "mode": mode, "steps": steps,
+                                          "warmup": warmup, "batch_walks": 1 << 20})
+            t0 = time.time()
+            r = run_leg(largs, WORKLOADS[name], dev, rank, world, local, with_e2e=False, with_cpu=False)
+            legs[f"{name}/{mode}"] = {
+                "pair_updates_per_s": r["value"], "walk_steps_per_s": r["walk_steps_per_s"],
+                "ms_per_step": r["ms_per_step"], "steps": r["steps"], "warmup": r["warmup"],
+                "batch_walks": r["config"]["batch_walks"], "mean_loss": r["mean_loss"],
+                "gpu_launches": r["gpu_launches"], "n_nodes": r["config"]["n_nodes"],
+                "n_edges": r["config"]["n_edges"], "roofline": r["roofline"], "walk": r["walk"],
+                "clocks": r["clocks"], "leg_s": round(time.time() - t0, 1)}
+        out["per_config"] = legs
+    if out is not None:
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -96,11 +96,14 @@ GS_API gs_status gs_graph_load_csr(int64_t n_nodes, int64_t n_edges,
                             const int32_t *d_cols, uint32_t flags,
                             void *stream, gs_graph **out);
 
-/* Frees the handle (and its walk index, waiting for the device if there is one); the CSR
- * arrays stay the caller's. NULL is allowed. */
+/* Releases the resident topology of gs_graph_load_csr (Section 3.1 keeps it for the lifetime
+ * of a trainer): frees the handle and the walk index and edge set it owns, waiting for the
+ * device if there are any; the CSR arrays stay the caller's.  NULL is allowed. */
 GS_API void gs_graph_free(gs_graph *g);
 
-/* max_degree is -1 if the graph was loaded without GS_VALIDATE. */
+/* Sizes of the resident graph G = (V, E) of Section 2.2: |V|, the number of CSR entries, the
+ * largest out-degree (-1 if the graph was loaded without GS_VALIDATE) and whether the rows
+ * were verified strictly increasing.  Output pointers may be NULL. */
 GS_API gs_status gs_graph_info(const gs_graph *g, int64_t *n_nodes, int64_t *n_edges,
                         int64_t *max_degree, int32_t *rows_sorted);
 
@@ -165,17 +168,6 @@ GS_API gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts,
                             int32_t *d_walks_out, uint64_t *d_steps,
                             uint64_t *d_cap_hits, void *stream);
 
-/*
- * Measurement aid (no counterpart in the paper): times independent random 16-byte reads of the
- * graph's walk index (GS_BUILD_WALK_INDEX required), issued with the load instruction the walk
- * kernels use.  A walk transition is one such read that depends on the one before it, so the
- * rate found here is the ceiling for walk transitions per second on this device and graph.
- * n_reads is rounded up to a multiple of 65,536 (*h_reads_done); the kernel runs twice and the
- * second run is timed with events on `stream` (*h_ms_out).  WAITS for completion.
- */
-GS_API gs_status gs_probe_random_reads(const gs_graph *g, int64_t n_reads, int64_t *h_reads_done,
-                                       float *h_ms_out, void *stream);
-
 /* ---------------------------------------------------------------- SGNS */
 #define GS_DETERMINISTIC  0   /* synchronous mini-batch step, bitwise reproducible */
 #define GS_HOGWILD        1   /* lock-free: plain loads and stores, rows may race   */
@@ -195,7 +187,11 @@ GS_API gs_status gs_probe_random_reads(const gs_graph *g, int64_t n_reads, int64
                                      /* paper's runs use a fixed window, Section 4.)          */
 
 /*
- * One SGNS update over a batch of walks.
+ * One SGNS update over a batch of walks: skip-gram with negative sampling on
+ * the nodes of random walks (Section 2.2), run as the paper's training
+ * iteration - fetch the rows of the batch, compute the loss and its gradients,
+ * write the increments back (Section 3.2 "Node Embedding Training"; the two
+ * update disciplines are those of Section 3.2 "Synchronization").
  *
  * Pairs: for position i of a walk and j with 0 < |i-j| <= window inside the
  * walk, both entries >= 0: center = walk[i], context = walk[j], slot
@@ -216,7 +212,12 @@ GS_API gs_status gs_probe_random_reads(const gs_graph *g, int64_t n_reads, int64
  * per position the center row is read once, every target row is read,
  * updated from the current center row and written back at once, and the
  * center row receives its accumulated increment after the last pair.
- * Results depend on scheduling.
+ * Results depend on scheduling.  Target rows are handled a chunk at a time
+ * (6 to 24 rows, all loaded before any is stored): with GS_HOGWILD a row that
+ * occurs more than once in a chunk keeps the increment of its last occurrence
+ * only, like a row that two warps update at the same moment (adding the
+ * occurrences up instead was measured and lowers the loss no further);
+ * GS_HOGWILD_RED adds every increment.
  *
  *   d_w_in, d_w_out : [n_nodes][dim] fp32 row-major, 16-byte aligned,
  *                     dim in {32, 64, 128, 256}
@@ -253,15 +254,19 @@ GS_API gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, in
  * performs no cudaMalloc / cudaFree and calls no allocating routine.
  *
  * Limit: the batch must need at most 32 MiB of scratch,
- *   slots = n_walks * walk_len * (2*window*(1+n_neg) + 1)
- *   bytes ~ (20 + dim/16) * slots + n_walks * walk_len * (4*dim + 12)  (+ < 1 % for the sort)
+ *   slots = n_walks * walk_len * (P + 1), P = 2*window*(1+n_neg) rounded up to a power of two
+ *   bytes ~ (24 + dim/16) * slots + n_walks * walk_len * (4*dim + 16)  (+ < 1 % for the sort)
  * e.g. up to about 300 walks of length 40 with window 5, 5 negatives, dim 128.
  * Larger batches are rejected with GS_ERR_UNSUPPORTED and a message that
  * states the bytes needed; nothing is launched in that case.
  *
  * The first call on each device looks up the array's device address (one
- * cudaGetSymbolAddress with that device current); make that first call
- * outside any stream capture.  All calls on a device share the one array and
+ * cudaGetSymbolAddress with that device current).  With lazy module loading
+ * that lookup, and the first launch of each kernel, is also what makes the
+ * driver load this library's device code and set aside the 32 MiB, which may
+ * allocate and synchronise inside the driver: make one call per device during
+ * set-up, outside any stream capture, before entering the region that must
+ * not allocate.  All calls on a device share the one array and
  * it keeps whatever the previous call left: every pass overwrites what it
  * later reads, so stale contents are harmless, but two calls whose kernels
  * overlap on the GPU (different streams, no ordering between them) race on
@@ -450,7 +455,9 @@ typedef struct gs_sgns_config {
      * ignored.  GS_OPT_MOMENTUM: every batch is one gs_sgns_step_momentum with iteration =
      * iteration_base + batch index; needs GS_LR_CONSTANT, fp32 tables, no pair flags; rows are
      * brought up to date lazily, so call gs_momentum_flush(iteration = iteration_base + index of
-     * the last batch + 1) before reading the tables elsewhere.  GS_OPT_ADAM: every batch is one
+     * the last batch + 1) before reading the tables elsewhere; iteration_base + the index after
+     * the last batch of the call must stay below 2^31 - 1 (GS_ERR_INVALID_ARG otherwise: the
+     * per-row stamps are 32-bit).  GS_OPT_ADAM: every batch is one
      * gs_sgns_step_adam with step = iteration_base + batch index + 1; fp32 tables. */
     int32_t optimizer;        /* GS_OPT_*                                                */
     float   momentum;         /* GS_OPT_MOMENTUM: momentum value; GS_OPT_ADAM: beta1     */
@@ -470,8 +477,11 @@ typedef struct gs_epoch_stats {
     int64_t masked_negs;      /* negatives dropped because they equal their context */
                               /* (counted with GS_OPT_SGD only)                      */
     float   ms_walk;          /* device time of the walk kernels                 */
-    float   ms_sgns;          /* device time of the SGNS kernels                 */
+    float   ms_sgns;          /* device time of the SGNS kernels on the caller's stream */
     float   ms_total;
+    float   ms_prepare;       /* synchronous mode: device time of the table-independent */
+                              /* part of the step (targets, sort) on the walk stream    */
+    int64_t refused_ids;      /* see gs_refused_ids: what this call added to the counter */
 } gs_epoch_stats;
 
 /*
@@ -479,23 +489,40 @@ typedef struct gs_epoch_stats {
  * b = walk ids [b*batch_walks, (b+1)*batch_walks): generate the walks, then
  * one gs_sgns_step with lr_b (the paper's loop: sample, fetch rows, compute,
  * write back, barrier - Section 3.2).  Walk generation of batch b+1 overlaps
- * the SGNS step of batch b on a second stream.  WAITS for completion and
- * fills *h_out (host struct).  Epoch defaults of the paper: batch 512.
+ * the SGNS step of batch b on a second stream; in the synchronous mode that
+ * stream also lists and sorts the contributions of batch b+1, which needs no
+ * table (results are the same as with one gs_sgns_step per batch).  WAITS for
+ * completion and fills *h_out (host struct).  Epoch defaults of the paper: batch 512.
  */
 GS_API gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias,
                         void *d_w_in, void *d_w_out, const gs_sgns_config *cfg,
                         gs_epoch_stats *h_out, void *stream);
 
+/*
+ * Sticky per-device count of ids that the kernels refused (the paper has no counterpart: its
+ * storage is addressed with node ids that the partitioner made, Section 3.1).  The library never
+ * dereferences an id it has not range-checked; a start node passed in d_starts, a walk entry other
+ * than -1, or an alias-table cell that lies outside [0, n_nodes) is treated as absent - and
+ * counted here, so that a corrupt input does not pass unnoticed as "fewer pairs".  Counted by
+ * gs_random_walks / gs_node2vec_walks (explicit start nodes), by every gs_sgns_step* call except
+ * gs_sgns_step_static, and by gs_sgns_epoch (which also reports its own share in
+ * gs_epoch_stats.refused_ids).  Reads the counter of the current device into *h_count after the
+ * work queued on `stream` so far, clears it if clear != 0, and WAITS.  gs_release_workspace
+ * also clears it.
+ */
+GS_API gs_status gs_refused_ids(uint64_t *h_count, int32_t clear, void *stream);
+
 /* Frees the cached scratch memory of the current device (waits for the device). */
 GS_API gs_status gs_release_workspace(void);
 
 /*
- * Tuning knob: which node2vec kernel runs.  0 (default): one lane per walk, rejection rounds and
- * transitions flattened into one loop, so a lane that has accepted starts its next transition
- * without waiting for its warp (1.0e10 transitions/s on the 4M-node workload with the edge set).
- * 1: one lane per walk, nested loops (7.2e9).  2, 4, 8, 32: that many lanes cooperate on a walk,
- * lane k of a group evaluates rejection round base + k and the first accepted round wins
- * (4.3e9 ... 1.9e9 without the edge set).  Walks do not depend on this setting.
+ * Which node2vec kernel runs (Section 2.2 names node2vec; the sampler is this library's).
+ * 0 (default): one lane per walk, rejection rounds and transitions flattened into one loop, so
+ * a lane that has accepted starts its next transition without waiting for its warp.  1, 2, 4,
+ * 8, 32: the generic kernel with that many lanes cooperating on a walk - lane k of a group
+ * evaluates rejection round base + k and the first accepted round wins; it also serves walk
+ * lengths that are not a multiple of 4 and unaligned outputs whatever the setting.  Walks do
+ * not depend on this setting.  Other values: GS_ERR_INVALID_ARG.
  */
 GS_API gs_status gs_tune_node2vec_group(int32_t lanes);
 

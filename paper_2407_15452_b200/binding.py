@@ -32,7 +32,7 @@ EXPORTS = [
     "gs_init_embeddings", "gs_random_walks", "gs_node2vec_walks", "gs_sgns_step",
     "gs_sgns_epoch", "gs_release_workspace", "gs_tune_node2vec_group", "gs_sgns_step_static", "gs_sgns_step_momentum", "gs_momentum_flush",
     "gs_init_embeddings_f16", "gs_sgns_step_f16", "gs_sgns_step_adam", "gs_build_keep_thresholds",
-    "gs_subsample_walks", "gs_shuffled_starts", "gs_probe_random_reads",
+    "gs_subsample_walks", "gs_shuffled_starts", "gs_refused_ids",
     "gs_init_embeddings_bf16", "gs_sgns_step_bf16",
 ]
 
@@ -64,7 +64,8 @@ class EpochStats(ctypes.Structure):
         ("loss_sum", ctypes.c_double), ("pairs", ctypes.c_int64), ("steps", ctypes.c_int64),
         ("cap_hits", ctypes.c_int64), ("batches", ctypes.c_int64), ("masked_negs", ctypes.c_int64),
         ("ms_walk", ctypes.c_float),
-        ("ms_sgns", ctypes.c_float), ("ms_total", ctypes.c_float),
+        ("ms_sgns", ctypes.c_float), ("ms_total", ctypes.c_float), ("ms_prepare", ctypes.c_float),
+        ("refused_ids", ctypes.c_int64),
     ]
 
 
@@ -189,14 +190,6 @@ def gs_node2vec_walks(graph: Graph, starts, n_walks: int, walk_id_base: int, wal
         _dev(out, torch.int32, "out"), _dev(steps, torch.int64, "steps", True),
         _dev(cap_hits, torch.int64, "cap_hits", True), _stream()))
     return out
-
-
-def gs_probe_random_reads(graph: Graph, n_reads: int):
-    """Random 16-byte reads per second over the graph's walk index (measurement aid)."""
-    done, ms = ctypes.c_int64(0), ctypes.c_float(0.0)
-    _check(lib().gs_probe_random_reads(graph._h, ctypes.c_int64(n_reads), ctypes.byref(done),
-                                       ctypes.byref(ms), _stream()))
-    return done.value / (ms.value * 1e-3)
 
 
 def gs_sgns_step(w_in, w_out, walks, walk_id_base: int, window: int, n_neg: int, alias,
@@ -379,6 +372,8 @@ class EpochResult:
     ms_walk: float
     ms_sgns: float
     ms_total: float
+    ms_prepare: float = 0.0
+    refused_ids: int = 0
 
 
 def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len, window, n_neg,
@@ -412,7 +407,14 @@ def gs_sgns_epoch(graph: Graph, alias, w_in, w_out, *, walks_per_node, walk_len,
                                _dev(w_in, tdt, "w_in"), _dev(w_out, tdt, "w_out"),
                                ctypes.byref(cfg), ctypes.byref(st), _stream()))
     return EpochResult(st.loss_sum, st.pairs, st.steps, st.cap_hits, st.batches, st.masked_negs, st.ms_walk,
-                       st.ms_sgns, st.ms_total)
+                       st.ms_sgns, st.ms_total, st.ms_prepare, st.refused_ids)
+
+
+def gs_refused_ids(clear: bool = False) -> int:
+    """Ids refused by the kernels of the current device so far (waits for the current stream)."""
+    out = ctypes.c_uint64(0)
+    _check(lib().gs_refused_ids(ctypes.byref(out), ctypes.c_int32(1 if clear else 0), _stream()))
+    return out.value
 
 
 def gs_release_workspace():

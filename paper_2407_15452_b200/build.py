@@ -4,6 +4,8 @@
 
 Sources: csrc/*.cu; public header: include/gs.h at the repository root.
 Output: paper_2407_15452_b200/libgs_b200.so (objects under _build/).
+Also builds the benchmark's own measurement aid, bench_probe.cu at the repository root, into
+libbench_probe.so beside it (not part of the library).
 """
 from __future__ import annotations
 
@@ -58,5 +60,20 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
+PROBE_SRC = ROOT / "bench_probe.cu"
+PROBE_LIB = ROOT / "libbench_probe.so"
+
+
+def build_probe(force: bool = False) -> Path:
+    """The random-read probe that bench.py --stage walks loads (one file, no dependencies)."""
+    if force or _stale(PROBE_LIB, [PROBE_SRC]):
+        cmd = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
+               "-std=c++17", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
+               "-o", str(PROBE_LIB), str(PROBE_SRC)]
+        subprocess.run(cmd, check=True)
+    return PROBE_LIB
+
+
 if __name__ == "__main__":
+    print(build_probe(force="--force" in sys.argv))
     print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv))

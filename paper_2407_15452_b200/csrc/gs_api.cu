@@ -24,23 +24,23 @@ gs_status init_embeddings(float *w_in, float *w_out, int64_t n, int32_t dim, uin
                           cudaStream_t st);
 gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
                                int64_t base, int32_t L, uint64_t seed, int32_t *walks,
-                               unsigned long long *steps, cudaStream_t st);
+                               unsigned long long *steps, unsigned long long *refused, cudaStream_t st);
 gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
                                 int64_t base, int32_t L, uint64_t seed, double p, double q,
                                 int32_t max_rounds, int group, int32_t *walks,
                                 unsigned long long *steps, unsigned long long *caps,
-                                cudaStream_t st);
+                                unsigned long long *refused, cudaStream_t st);
 gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                     int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                     const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                     int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
-                    unsigned long long *masked = nullptr);
+                    unsigned long long *masked = nullptr, int prepared = -1);
 
 gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                         const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                         int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
-                        unsigned long long *masked = nullptr);
+                        unsigned long long *masked = nullptr, int prepared = -1);
 gs_status init_embeddings_f16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
                               cudaStream_t st);
 gs_status init_embeddings_bf16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
@@ -49,23 +49,26 @@ gs_status sgns_step_bf16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, 
                          int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                          const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                          int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
-                         unsigned long long *masked = nullptr);
+                         unsigned long long *masked = nullptr, int prepared = -1);
 gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_out, int32_t *last_in,
                              int32_t *last_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                              int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                              const uint64_t *alias, float lr, float mu, int32_t iter, uint64_t seed,
-                             double *loss, int64_t *pairs, cudaStream_t st);
+                             double *loss, int64_t *pairs, cudaStream_t st, int prepared = -1);
+gs_status sgns_prepare_sync(int64_t n_nodes, int32_t dim, const int32_t *walks, int64_t n_walks,
+                            int64_t walk_id_base, int32_t L, int32_t w, int32_t K, const uint64_t *alias,
+                            uint64_t seed, int32_t pair_mode, int set, cudaStream_t st);
 gs_status momentum_flush(float *w, float *m, int32_t *last, int64_t n_rows, int32_t dim, float lr,
                          float mu, int32_t iter, cudaStream_t st);
 gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, float *m_out,
                          float *v_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                          int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                          const uint64_t *alias, float lr, float b1, float b2, float eps, int64_t step,
-                         uint64_t seed, int32_t pair_mode, double *loss, int64_t *pairs, cudaStream_t st);
+                         uint64_t seed, int32_t pair_mode, double *loss, int64_t *pairs, cudaStream_t st,
+                         int prepared = -1);
 gs_status launch_subsample_walks(const int32_t *walks, int64_t n_walks, int64_t base, int32_t L,
                                  const uint32_t *keep_thr, int64_t n_nodes, uint64_t seed, int32_t *out,
                                  unsigned long long *kept, cudaStream_t st);
-gs_status random_read_probe(const gs_graph *g, int64_t n_reads, float *ms_out, cudaStream_t st);
 gs_status launch_shuffled_starts(int64_t n_nodes, uint64_t seed, uint32_t epoch, int64_t first,
                                  int64_t count, int32_t *starts, cudaStream_t st);
 
@@ -144,11 +147,22 @@ gs_status workspace_get(int slot, size_t bytes, void **out)
             set_error("scratch allocation of %zu bytes failed: %s", want, cudaGetErrorString(e));
             return GS_ERR_OOM;
         }
+        if (slot == WS_COUNTERS && (e = cudaMemset(p, 0, want)) != cudaSuccess) {   // counters start at zero
+            cudaFree(p);
+            return cuda_fail(e, "cudaMemset(counters)");
+        }
         d->ws[slot] = p;
         d->ws_bytes[slot] = want;
     }
     *out = d->ws[slot];
     return GS_OK;
+}
+
+unsigned long long *refused_counter()
+{
+    void *ws = nullptr;
+    if (workspace_get(WS_COUNTERS, 256, &ws) != GS_OK) return nullptr;
+    return (unsigned long long *)((char *)ws + 160);
 }
 
 static bool dim_ok(int32_t dim) { return dim == 32 || dim == 64 || dim == 128 || dim == 256; }
@@ -160,6 +174,20 @@ using namespace gs;
 extern "C" {
 
 const char *gs_last_error(void) { return g_err; }
+
+gs_status gs_refused_ids(uint64_t *h_count, int32_t clear, void *stream)
+{
+    if (!h_count) return invalid("h_count is NULL");
+    unsigned long long *ctr = refused_counter();
+    if (!ctr) return GS_ERR_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long v = 0;
+    GS_CUDA_TRY(cudaMemcpyAsync(&v, ctr, sizeof(v), cudaMemcpyDeviceToHost, st));
+    if (clear) GS_CUDA_TRY(cudaMemsetAsync(ctr, 0, sizeof(v), st));
+    GS_CUDA_TRY(cudaStreamSynchronize(st));
+    *h_count = (uint64_t)v;
+    return GS_OK;
+}
 
 gs_status gs_release_workspace(void)
 {
@@ -356,10 +384,11 @@ gs_status gs_random_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_
     gs_status s = check_walk_args(g, n_walks, walk_id_base, walk_len, d_walks_out);
     if (s != GS_OK) return s;
     return launch_uniform_walks(g, d_starts, n_walks, walk_id_base, walk_len, seed, d_walks_out,
-                                (unsigned long long *)d_steps, (cudaStream_t)stream);
+                                (unsigned long long *)d_steps, d_starts ? refused_counter() : nullptr,
+                                (cudaStream_t)stream);
 }
 
-static int g_n2v_group = 0;   // node2vec kernel: 0 = one lane per walk, flattened loop (measured fastest)
+static int g_n2v_group = 0;   // node2vec kernel: 0 = one lane per walk, flattened loop (the default)
 
 gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts, int64_t n_walks,
                             int64_t walk_id_base, int32_t walk_len, uint64_t seed, double p,
@@ -377,28 +406,17 @@ gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts, int64_t 
     return launch_node2vec_walks(g, d_starts, n_walks, walk_id_base, walk_len, seed, p, q,
                                  max_rounds, g_n2v_group, d_walks_out,
                                  (unsigned long long *)d_steps, (unsigned long long *)d_cap_hits,
-                                 (cudaStream_t)stream);
+                                 d_starts ? refused_counter() : nullptr, (cudaStream_t)stream);
 }
 
-// Tuning knob used by the benchmarks: kernel / lanes per walk (0, 1, 2, 4, 8, 32) of the node2vec sampler.
-// Results do not depend on it.
+// Which node2vec kernel runs: 0 the flattened one-lane kernel, 1..32 the generic kernel with that
+// many lanes per walk.  Results do not depend on it.
 gs_status gs_tune_node2vec_group(int32_t lanes)
 {
     if (lanes != 0 && lanes != 1 && lanes != 2 && lanes != 4 && lanes != 8 && lanes != 32)
         return invalid("lanes per walk must be 0 (one lane, flattened loop), 1, 2, 4, 8 or 32");
     g_n2v_group = lanes;
     return GS_OK;
-}
-
-gs_status gs_probe_random_reads(const gs_graph *g, int64_t n_reads, int64_t *h_reads_done,
-                                float *h_ms_out, void *stream)
-{
-    if (!g || !h_reads_done || !h_ms_out) return invalid("null pointer");
-    if (!g->d_edge_rec) return invalid("the graph was loaded without GS_BUILD_WALK_INDEX");
-    if (n_reads < 1 || n_reads > ((int64_t)1 << 36)) return invalid("n_reads outside [1, 2^36]");
-    const int64_t per_block = 256 * 256;
-    *h_reads_done = (n_reads + per_block - 1) / per_block * per_block;
-    return random_read_probe(g, n_reads, h_ms_out, (cudaStream_t)stream);
 }
 
 // ------------------------------------------------------------------ SGNS
@@ -714,18 +732,33 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
     int64_t b_end = cfg->num_batches > 0 ? cfg->first_batch + cfg->num_batches : nb_total;
     if (b_end > nb_total) b_end = nb_total;
     if (cfg->first_batch >= b_end) return GS_OK;
+    // momentum stamps and the iteration argument are 32-bit: the last batch's iteration + 1 must fit
+    if (cfg->optimizer == GS_OPT_MOMENTUM && cfg->iteration_base + b_end > (int64_t)0x7FFFFFFE) {
+        set_error("invalid argument: iteration_base + last batch = %lld exceeds 2^31 - 2; start a new "
+                  "run of iterations (flush the momentum first)", (long long)(cfg->iteration_base + b_end));
+        return GS_ERR_INVALID_ARG;
+    }
 
-    cudaStream_t s_sgns = (cudaStream_t)stream;
+    // The updates run on a stream of the highest priority and the walk sampler (with the
+    // table-independent part of the synchronous step) on one of the lowest, both owned by this
+    // call: where blocks of both are waiting for an SM, those of the update, which every batch
+    // waits for, go first.  The caller's stream is joined at both ends.
+    cudaStream_t s_user = (cudaStream_t)stream;
+    cudaStream_t s_sgns = nullptr;
     cudaStream_t s_walk = nullptr;
+    cudaEvent_t ev_join = nullptr;
     cudaEvent_t ev_walk[2] = { nullptr, nullptr }, ev_sgns[2] = { nullptr, nullptr };
     cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
-    TimerRing t_walk, t_sgns;
+    TimerRing t_walk, t_sgns, t_prep;
+    const bool sync_mode = (cfg->mode & 0xFF) == GS_DETERMINISTIC;
     gs_status rc = GS_OK;
     int32_t *wbuf[2] = { nullptr, nullptr };
     int32_t *sbuf[2] = { nullptr, nullptr };
     EpochCounters *ctr = nullptr;
     EpochCounters host_ctr;
     memset(&host_ctr, 0, sizeof(host_ctr));
+    unsigned long long refused_before = 0, refused_after = 0;
+    unsigned long long *refused_ctr = nullptr;
 
 #define EP_TRY(expr)                                                   \
     do {                                                               \
@@ -747,16 +780,27 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
             sbuf[1] = sbuf[0] + cfg->batch_walks;
         }
     }
-    EP_TRY(cudaStreamCreateWithFlags(&s_walk, cudaStreamNonBlocking));
+    {
+        int least = 0, greatest = 0;
+        EP_TRY(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+        EP_TRY(cudaStreamCreateWithPriority(&s_sgns, cudaStreamNonBlocking, greatest));
+        EP_TRY(cudaStreamCreateWithPriority(&s_walk, cudaStreamNonBlocking, least));
+        EP_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
+        EP_TRY(cudaEventRecord(ev_join, s_user));
+        EP_TRY(cudaStreamWaitEvent(s_sgns, ev_join, 0));         // after the caller's earlier work
+    }
     for (int i = 0; i < 2; ++i) {
         EP_TRY(cudaEventCreateWithFlags(&ev_walk[i], cudaEventDisableTiming));
         EP_TRY(cudaEventCreateWithFlags(&ev_sgns[i], cudaEventDisableTiming));
     }
     EP_TRY(cudaEventCreate(&ev_begin));
     EP_TRY(cudaEventCreate(&ev_end));
-    if (!t_walk.init() || !t_sgns.init()) { rc = cuda_fail(cudaGetLastError(), "cudaEventCreate"); goto done; }
+    if (!t_walk.init() || !t_sgns.init() || !t_prep.init()) { rc = cuda_fail(cudaGetLastError(), "cudaEventCreate"); goto done; }
 
     EP_TRY(cudaMemsetAsync(ctr, 0, sizeof(EpochCounters), s_sgns));
+    refused_ctr = refused_counter();
+    if (refused_ctr)
+        EP_TRY(cudaMemcpyAsync(&refused_before, refused_ctr, sizeof(refused_before), cudaMemcpyDeviceToHost, s_sgns));
     EP_TRY(cudaEventRecord(ev_begin, s_sgns));
     EP_TRY(cudaStreamWaitEvent(s_walk, ev_begin, 0));        // the walk stream starts after prior work
 
@@ -775,15 +819,25 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
             }
             if (cfg->walk_kind == GS_WALK_UNIFORM)
                 EP_CALL(launch_uniform_walks(g, starts, n, base, cfg->walk_len, cfg->seed, wbuf[buf],
-                                             &ctr->steps, s_walk));
+                                             &ctr->steps, nullptr, s_walk));
             else
                 EP_CALL(launch_node2vec_walks(g, starts, n, base, cfg->walk_len, cfg->seed, cfg->p,
                                               cfg->q, cfg->max_rounds, g_n2v_group, wbuf[buf],
-                                              &ctr->steps, &ctr->caps, s_walk));
+                                              &ctr->steps, &ctr->caps, nullptr, s_walk));
             if (cfg->d_keep_thr)
                 EP_CALL(launch_subsample_walks(wbuf[buf], n, base, cfg->walk_len, cfg->d_keep_thr,
                                                g->n_nodes, cfg->seed, wbuf[buf], nullptr, s_walk));
             t_walk.stop(tk, s_walk);
+        }
+        // Synchronous mode: the targets of the batch and their sorted keys do not depend on the
+        // tables, so they are produced here, on the walk stream, into scratch set `buf`, while the
+        // update of the batch before this one still runs on the other stream.
+        const int prepared = sync_mode ? buf : -1;
+        if (sync_mode) {
+            const int tk = t_prep.start(s_walk);
+            EP_CALL(sgns_prepare_sync(g->n_nodes, cfg->dim, wbuf[buf], n, base, cfg->walk_len, cfg->window,
+                                      cfg->n_neg, d_alias, cfg->seed, cfg->mode & ~0xFF, buf, s_walk));
+            t_prep.stop(tk, s_walk);
         }
         EP_TRY(cudaEventRecord(ev_walk[buf], s_walk));
         EP_TRY(cudaStreamWaitEvent(s_sgns, ev_walk[buf], 0));
@@ -799,40 +853,44 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
                                            cfg->d_last_in, cfg->d_last_out, g->n_nodes, cfg->dim, wbuf[buf],
                                            n, base, cfg->walk_len, cfg->window, cfg->n_neg, d_alias,
                                            (float)lr, cfg->momentum, (int32_t)(cfg->iteration_base + b),
-                                           cfg->seed, &ctr->loss, (int64_t *)&ctr->pairs, s_sgns));
+                                           cfg->seed, &ctr->loss, (int64_t *)&ctr->pairs, s_sgns, prepared));
             else if (cfg->optimizer == GS_OPT_ADAM)
                 EP_CALL(sgns_step_adam((float *)d_w_in, (float *)d_w_out, cfg->d_m_in, cfg->d_v_in,
                                        cfg->d_m_out, cfg->d_v_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
                                        cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
                                        cfg->momentum, cfg->beta2, cfg->eps, cfg->iteration_base + b + 1,
                                        cfg->seed, cfg->mode & ~0xFF, &ctr->loss, (int64_t *)&ctr->pairs,
-                                       s_sgns));
+                                       s_sgns, prepared));
             else if (bf16)
                 EP_CALL(sgns_step_bf16(d_w_in, d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
                                        cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
                                        cfg->seed, cfg->mode, &ctr->loss, (int64_t *)&ctr->pairs, nullptr,
-                                       nullptr, s_sgns, &ctr->masked));
+                                       nullptr, s_sgns, &ctr->masked, prepared));
             else if (f16)
                 EP_CALL(sgns_step_f16(d_w_in, d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n, base,
                                       cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
                                       cfg->seed, cfg->mode, &ctr->loss, (int64_t *)&ctr->pairs, nullptr,
-                                      nullptr, s_sgns, &ctr->masked));
+                                      nullptr, s_sgns, &ctr->masked, prepared));
             else
                 EP_CALL(sgns_step((float *)d_w_in, (float *)d_w_out, g->n_nodes, cfg->dim, wbuf[buf], n,
                                   base, cfg->walk_len, cfg->window, cfg->n_neg, d_alias, (float)lr,
                                   cfg->seed, cfg->mode, &ctr->loss, (int64_t *)&ctr->pairs, nullptr,
-                                  nullptr, s_sgns, &ctr->masked));
+                                  nullptr, s_sgns, &ctr->masked, prepared));
             t_sgns.stop(tk, s_sgns);
         }
         EP_TRY(cudaEventRecord(ev_sgns[buf], s_sgns));
         ++h_out->batches;
     }
     EP_TRY(cudaEventRecord(ev_end, s_sgns));
+    EP_TRY(cudaStreamWaitEvent(s_user, ev_end, 0));              // the caller's later work comes after
     EP_TRY(cudaMemcpyAsync(&host_ctr, ctr, sizeof(host_ctr), cudaMemcpyDeviceToHost, s_sgns));
+    if (refused_ctr)
+        EP_TRY(cudaMemcpyAsync(&refused_after, refused_ctr, sizeof(refused_after), cudaMemcpyDeviceToHost, s_sgns));
     EP_TRY(cudaStreamSynchronize(s_sgns));
     EP_TRY(cudaStreamSynchronize(s_walk));
     t_walk.finish();
     t_sgns.finish();
+    t_prep.finish();
     h_out->loss_sum = host_ctr.loss;
     h_out->pairs = (int64_t)host_ctr.pairs;
     h_out->steps = (int64_t)host_ctr.steps;
@@ -840,22 +898,27 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
     h_out->masked_negs = (int64_t)host_ctr.masked;
     h_out->ms_walk = (float)t_walk.total_ms;
     h_out->ms_sgns = (float)t_sgns.total_ms;
+    h_out->ms_prepare = (float)t_prep.total_ms;
+    h_out->refused_ids = (int64_t)(refused_after - refused_before);
     EP_TRY(cudaEventElapsedTime(&h_out->ms_total, ev_begin, ev_end));
 
 done:
     if (rc != GS_OK) {                       // let queued work drain before buffers are reused
         if (s_walk) cudaStreamSynchronize(s_walk);
-        cudaStreamSynchronize(s_sgns);
+        if (s_sgns) cudaStreamSynchronize(s_sgns);
     }
     t_walk.destroy();
     t_sgns.destroy();
+    t_prep.destroy();
     for (int i = 0; i < 2; ++i) {
         if (ev_walk[i]) cudaEventDestroy(ev_walk[i]);
         if (ev_sgns[i]) cudaEventDestroy(ev_sgns[i]);
     }
     if (ev_begin) cudaEventDestroy(ev_begin);
     if (ev_end) cudaEventDestroy(ev_end);
+    if (ev_join) cudaEventDestroy(ev_join);
     if (s_walk) cudaStreamDestroy(s_walk);
+    if (s_sgns) cudaStreamDestroy(s_sgns);
 #undef EP_TRY
 #undef EP_CALL
     return rc;

@@ -24,9 +24,14 @@ gs_status cuda_fail(cudaError_t e, const char *what);
 // Returns a 256-byte aligned scratch block of at least `bytes` for slot `slot`
 // (independent blocks so that kernels on different streams do not share one).
 gs_status workspace_get(int slot, size_t bytes, void **out);
-enum { WS_WALKS0 = 0, WS_WALKS1 = 1, WS_SGNS = 2, WS_COUNTERS = 3, WS_STARTS = 4, WS_SLOTS = 5 };
+enum { WS_WALKS0 = 0, WS_WALKS1 = 1, WS_SGNS = 2, WS_COUNTERS = 3, WS_STARTS = 4, WS_SGNS1 = 5, WS_SLOTS = 6 };
 
 int sm_count();
+
+// Device counter of the current device to which kernels add the ids they refused (start nodes,
+// walk entries, alias cells outside [0, n_nodes)); nullptr if it cannot be had.  Lives in the
+// WS_COUNTERS block (bytes 0..127: epoch counters, 128: walk ticket, 160: this counter).
+unsigned long long *refused_counter();
 
 // ---- graph handle --------------------------------------------------------------
 }  // namespace gs

@@ -12,11 +12,15 @@
 // negatives, slot by slot) are listed in shared memory, and the list is
 // consumed in chunks of TCH rows whose loads are all in flight together.
 //
-// Synchronous mode: one warp per position computes the coefficients g and the
-// center-row gradient from the entry tables and emits one (destination row,
-// contribution index) key per target; the keys are radix-sorted, and one warp
-// per distinct row sums that row's contributions in index order and writes the
-// row once.  No floating-point atomics anywhere on this path.
+// Synchronous mode, in two parts.  Part A needs no table: one warp per position lists
+// the targets of its pairs and emits one (destination row, contribution index) key per
+// target, and the keys are radix-sorted.  Part B reads the entry tables: one warp per
+// position computes the coefficients g and the center-row gradient; then the sorted
+// contributions are walked run by run, each run summed in index order and its row
+// written once.  No result depends on the order in which anything executes: a sum is
+// formed by one warp in a fixed order, and every value of a table receives exactly one
+// addition per step.  Because part A does not touch the tables, the epoch driver runs
+// it for batch b+1 on a second stream while batch b is in part B.
 #include <mutex>
 #include <type_traits>
 
@@ -27,8 +31,8 @@
 
 namespace gs {
 
-int radix_sort_pairs(uint32_t *keysA, uint32_t *valsA, uint32_t *keysB, uint32_t *valsB,
-                     uint32_t n, int bits, uint32_t *counts, cudaStream_t st,
+int radix_sort_pairs(const uint32_t *keys_src, uint32_t *keysB, uint32_t *valsB, uint32_t *keysC,
+                     uint32_t *valsC, uint32_t n, int bits, uint32_t *counts, cudaStream_t st,
                      uint32_t **keys_sorted, uint32_t **vals_sorted);
 size_t sort_counts_bytes(uint32_t n);
 
@@ -359,8 +363,11 @@ __device__ __forceinline__ void sum_over_groups(Row<FPL> &x)
 // ---------------------------------------------------------------- target list of one position
 // Slot layout: tgt[s * (1 + K) + 0] = context of slot s, tgt[s * (1 + K) + 1 + k] = negative k;
 // -1 where the pair does not exist or the negative equals the context (masked).
-// W points at the walk (global or shared), c = W[i] >= 0.  Returns the number of pairs in the low
-// 8 bits and the number of masked negatives above them (identical on every lane).  dump_* (nullable) are this position's rows of the dump arrays.
+// W points at the walk (global or shared), c = W[i] >= 0.  Returns, identical on every lane, the
+// number of pairs in bits 0..7, the number of masked negatives in bits 8..19 and, from bit 20, the
+// number of ids that were refused: walk entries other than -1 and alias cells that name no row
+// of the tables (they are treated as absent).  dump_* (nullable) are this position's rows of the
+// dump arrays.
 // flags & PAIR_FWD keeps only contexts that come later in the walk (edge sampling of LINE);
 // flags & PAIR_SHRINK draws the window of this position, w_i = 1 + mulhi(word, w) uniform on
 // 1..w (word2vec's shrinking window), and keeps the contexts within w_i.  Slots and the keying
@@ -378,17 +385,21 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
     int w_i = w;
     if (flags & PAIR_SHRINK) w_i = 1 + (int)__umulhi(draw(seed, id, (uint32_t)i, TAG_WINDOW, 0).x, (uint32_t)w);
     const int hp = K > 0 ? (K + 1) / 2 : 1;          // Philox blocks per slot (>= 1 work item)
-    int pairs = 0, masked = 0;
+    int pairs = 0, masked = 0, refused = 0;
     __syncwarp();                                    // earlier readers of tgt are done
     for (int it0 = 0; it0 < S * hp; it0 += 32) {
         const int it = it0 + lane;
         bool valid = false, hid0 = false, hid1 = false;
+        int bad = 0;                                 // ids this lane refused
         if (it < S * hp) {
             const int s = it / hp, m = it - s * hp;
             const int j = i - w + s + (s >= w ? 1 : 0);
             const bool in_window = j - i <= w_i && i - j <= w_i && !(fwd && s < w);   // fwd: only j > i
             int32_t ctx = (j >= 0 && j < L && in_window) ? W[j] : -1;
-            if ((uint32_t)ctx >= n_alias) ctx = -1;        // absent, or not a node of the tables
+            if ((uint32_t)ctx >= n_alias) {                // absent, or not a node of the tables
+                if (ctx != -1 && m == 0) bad = 1;
+                ctx = -1;
+            }
             valid = ctx >= 0;
             if (m == 0) {
                 tgt[s * T1] = ctx;
@@ -405,12 +416,12 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
                     const uint32_t j0 = __umulhi(r.x, n_alias);
                     const uint64_t e0 = ld_random(alias + j0);
                     n0 = r.y < (uint32_t)e0 ? (int32_t)j0 : (int32_t)(e0 >> 32);
-                    if ((uint32_t)n0 >= n_alias) n0 = -1;      // a table entry that names no node
+                    if ((uint32_t)n0 >= n_alias) { n0 = -1; ++bad; }   // a table entry that names no node
                     if (two) {
                         const uint32_t j1 = __umulhi(r.z, n_alias);
                         const uint64_t e1 = ld_random(alias + j1);
                         n1 = r.w < (uint32_t)e1 ? (int32_t)j1 : (int32_t)(e1 >> 32);
-                        if ((uint32_t)n1 >= n_alias) n1 = -1;
+                        if ((uint32_t)n1 >= n_alias) { n1 = -1; ++bad; }
                     }
                 }
                 if (dump_negs) {
@@ -426,9 +437,13 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
         }
         pairs += __popc(__ballot_sync(0xffffffffu, valid));
         masked += __popc(__ballot_sync(0xffffffffu, hid0)) + __popc(__ballot_sync(0xffffffffu, hid1));
+        if (__any_sync(0xffffffffu, bad != 0)) {           // rare: a corrupt walk buffer or alias table
+            for (int o = 16; o > 0; o >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, o);
+            refused += bad;
+        }
     }
     __syncwarp();
-    return pairs | (masked << 8);
+    return pairs | (masked << 8) | (refused << 20);
 }
 
 __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int lane,
@@ -449,7 +464,8 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     int32_t L, int32_t w, int32_t K, const uint64_t *__restrict__ alias,
                     uint32_t n_alias, float lr, uint64_t seed, double *loss_out,
                     unsigned long long *pairs_out, int32_t *dump_pairs, int32_t *dump_negs,
-                    unsigned long long *ticket, int fwd, unsigned long long *masked_out)
+                    unsigned long long *ticket, int fwd, unsigned long long *masked_out,
+                    unsigned long long *refused_out)
 {
     using G = RowGeom<DIM, T, NARROW>;
     constexpr int FPL = G::FPL, LPR = G::LPR, NG = G::NG;
@@ -466,7 +482,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     int32_t *Wbuf = smem + wi * (wpt * L + SL);
     int32_t *tgt = Wbuf + wpt * L;
     double loss_acc = 0.0;
-    unsigned long long pair_acc = 0, masked_acc = 0;
+    unsigned long long pair_acc = 0, masked_acc = 0, refused_acc = 0;
 
     for (;;) {
         unsigned long long tk = 0;
@@ -485,11 +501,16 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             const int32_t c = W[i];
             int32_t *dp = dump_pairs ? dump_pairs + ((a * L + i) * S) * 2 : nullptr;
             int32_t *dn = dump_negs ? dump_negs + ((a * L + i) * S) * (int64_t)K : nullptr;
-            if ((uint32_t)c >= n_alias) { dump_empty_position(S, K, lane, dp, dn); continue; }   // -1 or no such row
+            if ((uint32_t)c >= n_alias) {                 // -1 or no such row
+                if (c != -1) ++refused_acc;
+                dump_empty_position(S, K, lane, dp, dn);
+                continue;
+            }
             const int packed = build_targets(W, L, i, w, K, seed, id, alias, n_alias, c, tgt, lane,
                                              dp, dn, fwd);
             const int pairs = packed & 0xFF;
-            masked_acc += (unsigned long long)(packed >> 8);
+            masked_acc += (unsigned long long)((packed >> 8) & 0xFFF);
+            refused_acc += (unsigned long long)((unsigned)packed >> 20);
             if (pairs == 0) continue;
             pair_acc += (unsigned long long)pairs;
             const Row<FPL> u = grow_load<DIM, T, NARROW>(w_in, c, sub);     // every group holds the center row
@@ -567,36 +588,34 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
         if (loss_out && pair_acc) atomicAdd(loss_out, loss_acc);
         if (pairs_out && pair_acc) atomicAdd(pairs_out, pair_acc);
         if (masked_out && masked_acc) atomicAdd(masked_out, masked_acc);
+        if (refused_out && refused_acc) atomicAdd(refused_out, refused_acc);
     }
 }
 
 // ---------------------------------------------------------------- synchronous mode
-// Pass 1: one warp per position.  Writes, for slot index x = pos * SL + slot:
-//   keys[x] = destination row of w_out (or `invalid`), gbuf[x] = coefficient g,
-// and per position: keys[n_slots + pos] = n_nodes + center (or `invalid`),
-// GU[pos] = sum g * v (gradient of the center row), loss_pos, pairs_pos.
-// MODE 0: everything.  MODE 1: keys only (no table is read; used by the momentum step to learn
-// which rows the batch will touch before it reads them).  MODE 2: everything but the keys.
-template <int DIM, typename T, int MODE>
+// Part A: one warp per position, no table is read.  The targets of a position are written as a
+// dense list - its contexts first, then its unmasked negatives, each in slot order - into a
+// segment of SLP = 2^shift >= SL entries: keys[pos << shift + k] = destination row of w_out for
+// k < n_all, `invalid` = 2 n_nodes behind them (*n_out counts the valid ones of the whole batch:
+// that is where the center keys begin once sorted).  Per position: tinfo[pos] = n_ctx | n_all << 16,
+// keys[n_slots + pos] = n_nodes + center (or `invalid` when the position forms no pair) and
+// pairs_pos[pos] = pairs | masked negatives << 8 | refused ids << 20.  (A power-of-two stride
+// turns "which position does contribution idx belong to" into a shift in the apply passes.)
 __global__ void __launch_bounds__(SGNS_WARPS * 32)
-sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out,
-                 const int32_t *__restrict__ walks, int64_t n_pos, int64_t walk_id_base, int32_t L,
-                 int32_t w, int32_t K, const uint64_t *__restrict__ alias, uint32_t n_alias,
-                 uint32_t n_nodes, uint64_t seed, uint32_t *__restrict__ keys,
-                 float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos,
-                 int32_t *__restrict__ pairs_pos, int32_t *dump_pairs, int32_t *dump_negs, int fwd)
+sgns_targets_kernel(const int32_t *__restrict__ walks, int64_t n_pos, int64_t walk_id_base, int32_t L,
+                    int32_t w, int32_t K, const uint64_t *__restrict__ alias, uint32_t n_alias,
+                    uint32_t n_nodes, uint64_t seed, int32_t shift, uint32_t *__restrict__ keys,
+                    uint32_t *__restrict__ tinfo, int32_t *__restrict__ pairs_pos,
+                    uint32_t *__restrict__ n_out, int32_t *dump_pairs, int32_t *dump_negs, int fwd)
 {
-    constexpr int FPL = RowGeom<DIM, T>::FPL, LPR = RowGeom<DIM, T>::LPR, NG = RowGeom<DIM, T>::NG;
-    constexpr int CH = TCH * NG;
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
-    const int grp = lane / LPR, sub = lane % LPR;
-    const int S = 2 * w, T1 = 1 + K, SL = S * T1;
+    const int S = 2 * w, T1 = 1 + K, SL = S * T1, SLP = 1 << shift;
     int32_t *tgt = smem + wi * SL;
     const uint32_t invalid = 2u * n_nodes;
-    const int64_t n_slots = n_pos * SL;
+    const int64_t n_slots = n_pos << shift;
     const int64_t n_warps = (int64_t)gridDim.x * SGNS_WARPS;
-
+    const unsigned below = (1u << lane) - 1u;
     for (int64_t pos = (int64_t)blockIdx.x * SGNS_WARPS + wi; pos < n_pos; pos += n_warps) {
         const int64_t a = pos / L;
         const int32_t i = (int32_t)(pos - a * L);
@@ -604,76 +623,168 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out,
         const int32_t c = W[i];
         int32_t *dp = dump_pairs ? dump_pairs + (pos * S) * 2 : nullptr;
         int32_t *dn = dump_negs ? dump_negs + (pos * S) * (int64_t)K : nullptr;
-        uint32_t *kp = keys + pos * SL;
-        float *gp = gbuf + pos * SL;
-        Row<FPL> acc;
-#pragma unroll
-        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
-        float loss = 0.f;
-        int pairs = 0;
-        __syncwarp();
+        uint32_t *kp = keys + (pos << shift);
         int packed = 0;
+        __syncwarp();
         if ((uint32_t)c < n_nodes) {                   // -1, or an id outside the tables: no pairs
             packed = build_targets(W, L, i, w, K, seed, (uint64_t)(walk_id_base + a), alias, n_alias,
                                    c, tgt, lane, dp, dn, fwd);
-            pairs = packed & 0xFF;
-        } else
-            dump_empty_position(S, K, lane, dp, dn);
-        if (pairs == 0) {
-            for (int x = lane; x < SL; x += 32) {
-                if (MODE != 2) kp[x] = invalid;
-                if (MODE != 1) gp[x] = 0.f;
-            }
-        } else if (MODE == 1) {
-            for (int x = lane; x < SL; x += 32) kp[x] = tgt[x] >= 0 ? (uint32_t)tgt[x] : invalid;
         } else {
-            const Row<FPL> u = grow_load<DIM>(w_in, c, sub);
-            int kk = 0;
-            for (int base = 0; base < SL; base += CH) {
-                int32_t ids[TCH];
-#pragma unroll
-                for (int k = 0; k < TCH; ++k) {
-                    const int t = base + k * NG + grp;
-                    ids[k] = t < SL ? tgt[t] : -1;
+            if (c != -1) packed = 1 << 20;             // one refused id
+            dump_empty_position(S, K, lane, dp, dn);
+        }
+        int n_ctx = 0, n_all = 0;
+        if ((packed & 0xFF) != 0) {
+#pragma unroll 1
+            for (int pass = 0; pass < 2; ++pass) {     // contexts, then negatives
+                for (int x0 = 0; x0 < SL; x0 += 32) {
+                    const int x = x0 + lane;
+                    const int32_t v = x < SL ? tgt[x] : -1;
+                    const bool take = v >= 0 && ((x % T1 == 0) == (pass == 0));
+                    const unsigned m = __ballot_sync(0xffffffffu, take);
+                    if (take) kp[n_all + __popc(m & below)] = (uint32_t)v;
+                    n_all += __popc(m);
                 }
-                Row<FPL> rows[TCH];
-                float f[TCH];
+                if (pass == 0) n_ctx = n_all;
+            }
+        }
+        for (int x = n_all + lane; x < SLP; x += 32) kp[x] = invalid;
+        if (lane == 0) {
+            keys[n_slots + pos] = n_ctx > 0 ? n_nodes + (uint32_t)c : invalid;
+            tinfo[pos] = (uint32_t)n_ctx | ((uint32_t)n_all << 16);
+            pairs_pos[pos] = packed;
+            if (n_all) atomicAdd(n_out, (uint32_t)n_all);   // integer: the total does not depend on order
+        }
+    }
+}
+
+// Sums of G rows at once.  v[q] is this lane's partial sum of row q.  The first log2(G) butterfly
+// steps exchange half of the values each (a lane keeps the rows whose index bit equals its lane
+// bit), the remaining steps add the one value left.  Afterwards the lanes whose index shares the
+// top log2(G) bits, r = lane >> (5 - log2 G), all hold the complete sum of row r.
+template <int G>
+__device__ __forceinline__ float reduce_rows(float (&v)[G], int lane)
+{
+    int off = 16;
 #pragma unroll
-                for (int k = 0; k < TCH; ++k)
-                    if (ids[k] >= 0) rows[k] = grow_load<DIM>(w_out, ids[k], sub);
+    for (int h = G / 2; h >= 1; h >>= 1, off >>= 1) {
+        const bool upper = (lane & off) != 0;
 #pragma unroll
-                for (int k = 0; k < TCH; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
+        for (int j = 0; j < h; ++j) {
+            const float send = upper ? v[j] : v[j + h];
+            const float keep = upper ? v[j + h] : v[j];
+            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    float s = v[0];
+    for (; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    return s;
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *p)
+{
+    asm volatile("prefetch.global.L2 [%0];" :: "l"(p));
+}
+
+// Part B, coefficients: one warp per position, a whole warp per row (a lane holds DIM / 32
+// values), G target rows in flight.  Reads the dense target list that part A wrote; writes g per
+// list entry, the center-row gradient GU[pos] = sum g * v and the position's loss.  The kernel is
+// kept light - its pace is set by how many row reads are in flight and by instruction issue, not
+// by arithmetic: the dot products of G rows are reduced together; the sigmoid, which the
+// gradient needs at once, is evaluated per group of G rows on all lanes; the softplus of the
+// loss is put off until every lane holds the argument of one entry (32 entries per evaluation);
+// while a group is worked on, the rows of the next one are already on their way into L2.
+template <int DIM, typename T>
+__global__ void __launch_bounds__(256, (DIM <= 64 ? 4 : 3))
+sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out, int64_t n_pos, int32_t shift,
+                 uint32_t n_nodes, const uint32_t *__restrict__ keys, const uint32_t *__restrict__ tinfo,
+                 float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos)
+{
+    constexpr int FPL = DIM / 32;
+    constexpr int G = FPL <= 4 ? 8 : 4;                 // rows in flight
+    constexpr int SH = FPL <= 4 ? 2 : 3;                // lanes [r << SH, (r + 1) << SH) hold the sum of row r
+    constexpr int QUAD = 1 << SH;                       // = 32 / G, also the groups per 32 entries
+    constexpr int ROW_BYTES = DIM * (int)sizeof(T);
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t n_slots = n_pos << shift;
+    for (int64_t pos = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); pos < n_pos;
+         pos += n_warps) {
+        const uint32_t info = tinfo[pos];
+        const int n_ctx = (int)(info & 0xFFFFu), n = (int)(info >> 16);
+        float loss = 0.f;
+        if (n > 0) {                                    // the position forms pairs (same on every lane)
+            const uint32_t *kp = keys + (pos << shift);
+            float *gp = gbuf + (pos << shift);
+            uint32_t id = lane < n ? kp[lane] : 0u;     // entries [k0, k0 + 32) of the list, one per lane
+            const Row<FPL> u = row_load<FPL>(w_in, (int64_t)(keys[n_slots + pos] - n_nodes), lane);
+            Row<FPL> acc;
 #pragma unroll
-                for (int k = 0; k < TCH; ++k) f[k] = group_sum<LPR>(f[k]);
-                const int my_t = base + sub * NG + grp;
-                const bool mine = sub < TCH && my_t < SL;
-                int my_kt = kk + (sub < TCH ? sub * NG + grp : 0);
-                while (my_kt >= T1) my_kt -= T1;
-                const int32_t my_id = mine ? tgt[my_t] : -1;
-                const float my_g = lane_coefficient<TCH>(f, sub, my_id, my_kt == 0, loss);
-                if (mine) {
-                    if (MODE != 2) kp[my_t] = my_id >= 0 ? (uint32_t)my_id : invalid;
-                    gp[my_t] = my_g;
-                }
+            for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+            // the first group's rows: one 128-byte line per lane, as far as the rows go
+            {
+                const uint32_t id0 = __shfl_sync(0xffffffffu, id, (lane * 128 / ROW_BYTES) & 31);
+                if (lane * 128 < G * ROW_BYTES && lane * 128 / ROW_BYTES < n)
+                    prefetch_l2((const char *)(w_out + (int64_t)id0 * DIM) + lane * 128 % ROW_BYTES);
+            }
+            for (int k0 = 0; k0 < n; k0 += 32) {
+                const uint32_t id_next = k0 + 32 + lane < n ? kp[k0 + 32 + lane] : 0u;
+                float my_z = 0.f;                       // softplus argument of the entry this lane keeps
+                bool my_has = false;
+                const int m = n - k0 < 32 ? n - k0 : 32;  // entries of this stretch
+                int g0 = 0;
+#pragma unroll 1
+                for (; g0 + G <= m; g0 += G) {            // full groups of G rows
+                    Row<FPL> rows[G];
+                    float f[G];
 #pragma unroll
-                for (int k = 0; k < TCH; ++k) {
-                    const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + k);
-                    if (ids[k] >= 0) {
+                    for (int q = 0; q < G; ++q)
+                        rows[q] = row_load<FPL>(w_out, (int64_t)__shfl_sync(0xffffffffu, id, g0 + q), lane);
+                    {   // next group's rows towards L2: lane l asks for line l of the group's G rows
+                        const int e = g0 + G + lane * 128 / ROW_BYTES;         // entry within [k0, k0 + 64)
+                        const uint32_t idn = g0 + 2 * G <= 32 ? __shfl_sync(0xffffffffu, id, e & 31)
+                                                              : __shfl_sync(0xffffffffu, id_next, e & 31);
+                        if (lane * 128 < G * ROW_BYTES && k0 + e < n)
+                            prefetch_l2((const char *)(w_out + (int64_t)idn * DIM) + lane * 128 % ROW_BYTES);
+                    }
 #pragma unroll
-                        for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g, rows[k].v[j], acc.v[j]);
+                    for (int q = 0; q < G; ++q) f[q] = row_dot<FPL>(u, rows[q]);
+                    const float fr = reduce_rows<G>(f, lane);
+                    const int kk = k0 + g0 + (lane >> SH);   // the entry whose sum this lane holds
+                    const bool is_ctx = kk < n_ctx;     // contexts come first in the list
+                    const float z = is_ctx ? -fr : fr;  // term: softplus(z); g = +-sigmoid(z)
+                    const float e = expf(-fabsf(z));
+                    const float rr = 1.0f / (1.0f + e);
+                    const float sig = z >= 0.f ? rr : e * rr;
+                    const float g = is_ctx ? -sig : sig;
+                    if ((lane & (QUAD - 1)) == ((g0 / G) & (QUAD - 1))) { my_z = z; my_has = true; }
+                    if ((lane & (QUAD - 1)) == 0) gp[kk] = g;
+#pragma unroll
+                    for (int q = 0; q < G; ++q) {
+                        const float gq = __shfl_sync(0xffffffffu, g, q << SH);
+#pragma unroll
+                        for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(gq, rows[q].v[j], acc.v[j]);
                     }
                 }
-                kk += CH;
-                while (kk >= T1) kk -= T1;
+#pragma unroll 1
+                for (; g0 < m; ++g0) {                    // the last few entries of the list, one at a time
+                    const Row<FPL> row = row_load<FPL>(w_out, (int64_t)__shfl_sync(0xffffffffu, id, g0), lane);
+                    const float fr = warp_sum(row_dot<FPL>(u, row));
+                    const bool is_ctx = k0 + g0 < n_ctx;
+                    float sig, sp;
+                    sigmoid_softplus(is_ctx ? -fr : fr, sig, sp);
+                    const float g = is_ctx ? -sig : sig;
+                    if (lane == 0) { gp[k0 + g0] = g; loss += sp; }
+#pragma unroll
+                    for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g, row.v[j], acc.v[j]);
+                }
+                if (my_has) loss += fmaxf(my_z, 0.f) + log1pf(expf(-fabsf(my_z)));
+                id = id_next;
             }
+            row_store<FPL>(GU, pos, lane, acc);         // fp32 scratch, natural column order
         }
-        loss = warp_sum(loss);                     // lane-local shares, fixed butterfly order
-        sum_over_groups<LPR, FPL>(acc);                 // fixed order as well
-        if (MODE != 1 && grp == 0) grow_store_f32<DIM, T>(GU, pos, sub, acc);
-        if (lane == 0) {
-            if (MODE != 2) keys[n_slots + pos] = pairs > 0 ? n_nodes + (uint32_t)c : invalid;
-            if (MODE != 1) { loss_pos[pos] = (double)loss; pairs_pos[pos] = packed; }   // pairs | masked << 8
-        }
+        loss = warp_sum(loss);                          // lane-local shares, fixed butterfly order
+        if (lane == 0) loss_pos[pos] = (double)loss;
     }
 }
 
@@ -831,7 +942,7 @@ momentum_stamp_kernel(int32_t *__restrict__ last, int64_t n_rows, int32_t iter)
 // RUN_CUT rows in a chain (a hub row of a 512-walk batch collects thousands).  A run that lies
 // inside one block of RUN_CUT positions is finished here.  Otherwise its first piece leaves a
 // partial sum in tail_part[block], each later piece in lead_part[block], and
-// sgns_apply_out_fixup_kernel adds the pieces in block order and writes the row.
+// the last launch of the step (finish_cut_runs) adds the pieces in block order and writes the row.
 constexpr int RUN_CUT = 256;
 
 template <int FPL, typename T>
@@ -839,7 +950,7 @@ __global__ void __launch_bounds__(256, 2)
 sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
                       const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
                       const uint32_t *__restrict__ vals, const float *__restrict__ gbuf,
-                      uint32_t n_keys, uint32_t n_nodes, int32_t SL, float lr,
+                      uint32_t n_keys, uint32_t n_nodes, int32_t shift, float lr,
                       double *__restrict__ lead_part, double *__restrict__ tail_part, MomState ms)
 {
     // One warp per block of RUN_CUT sorted positions.  The 32 lanes fetch the metadata of 32
@@ -889,7 +1000,7 @@ sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
             c = 0;
             if (key < n_nodes) {
                 g = gbuf[idx];
-                c = walks[idx / (uint32_t)SL];
+                c = walks[idx >> shift];                   // contribution idx belongs to position idx >> shift
             }
         };
         uint32_t my_key, key1, idx0, idx1;
@@ -948,21 +1059,184 @@ sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
     }
 }
 
-// One warp per block of RUN_CUT sorted positions: if a run starts in the block and continues
-// past its end, add its pieces (tail of this block, then the leading pieces of the following
-// blocks while they carry the same key) and write the row.
-template <int FPL, typename T>
-__global__ void __launch_bounds__(256)
-sgns_apply_out_fixup_kernel(T *__restrict__ w_out, const uint32_t *__restrict__ keys,
-                            uint32_t n_keys, uint32_t n_nodes, float lr,
-                            const double *__restrict__ lead_part, const double *__restrict__ tail_part,
-                            MomState ms)
+// row += x where nobody else adds to the row during this launch: one reduction per value, so the
+// result does not depend on timing, and the row never has to travel to the SM.
+template <int FPL>
+__device__ __forceinline__ void row_red_add(float *__restrict__ tab, int64_t r, int lane, const Row<FPL> &x)
 {
+    float *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 1) {
+        atomicAdd(p + lane, x.v[0]);
+    } else if constexpr (FPL == 2) {
+        atomicAdd(reinterpret_cast<float2 *>(p) + lane, make_float2(x.v[0], x.v[1]));
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q)
+            atomicAdd(reinterpret_cast<float4 *>(p) + q * 32 + lane,
+                      make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
+    }
+}
+
+// Pass 3 for fp32 tables and plain SGD.  Same walk over the sorted contributions as
+// sgns_apply_out_kernel (one warp per block of RUN_CUT positions, runs cut at block boundaries
+// and finished by the last launch of the step), made light so that many warps are resident:
+//  - a run is summed in fp32, in index order, by the warp that owns its block: at most RUN_CUT
+//    terms; the pieces of a longer run are added up in fp64 by the fix-up;
+//  - the output row is not read: the finished sum goes out as ONE reduction per value,
+//    row += -lr * sum.  Every row is owned by exactly one run, so this is the only addition the
+//    row receives in the step and the result bits do not depend on scheduling;
+//  - while a group of G center rows is added, the next group is already on its way into L1.
+template <int FPL>
+__global__ void __launch_bounds__(256, (FPL <= 2 ? 4 : 3))
+sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
+                          const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
+                          const uint32_t *__restrict__ vals, const float *__restrict__ gbuf,
+                          uint32_t n_keys, uint32_t n_nodes, int32_t shift, float lr,
+                          double *__restrict__ lead_part, double *__restrict__ tail_part)
+{
+    constexpr int G = FPL <= 4 ? 8 : 4;
+    constexpr int ROW_BYTES = FPL * 32 * 4;
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t n_blocks = ((int64_t)n_keys + RUN_CUT - 1) / RUN_CUT;
-    for (int64_t b = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); b + 1 < n_blocks;
+    for (int64_t b = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); b < n_blocks;
          b += n_warps) {
+        const int64_t base = b * RUN_CUT;
+        const int64_t end = base + RUN_CUT < (int64_t)n_keys ? base + RUN_CUT : (int64_t)n_keys;
+        uint32_t carry_key = base > 0 ? keys[base - 1] : 0xFFFFFFFFu;     // key before the block
+        bool have = false, lead = false;                 // a run is open / it began before this block
+        uint32_t cur_key = 0;
+        Row<FPL> acc;
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+        if (carry_key < n_nodes && keys[base] == carry_key) { have = true; lead = true; cur_key = carry_key; }
+
+        auto store_part = [&](double *part) {
+            double *dst = part + b * (int64_t)(FPL * 32);
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) dst[j * 32 + lane] = (double)acc.v[j];
+        };
+        auto close_inner = [&]() {                       // the run ends inside the block
+            if (lead) {
+                store_part(lead_part);
+            } else {
+                Row<FPL> d;
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) d.v[j] = -lr * acc.v[j];
+                row_red_add<FPL>(w_out, (int64_t)cur_key, lane, d);
+            }
+        };
+
+        // metadata of a chunk: sorted key and contribution index, then coefficient and center node
+        // (two dependent reads), fetched two chunks / one chunk ahead of the rows that need them
+        auto link1 = [&](int64_t i, uint32_t &key, uint32_t &idx) {
+            key = i < end ? keys[i] : 0xFFFFFFFFu;
+            idx = i < end ? vals[i] : 0u;
+        };
+        auto link2 = [&](uint32_t key, uint32_t idx, float &g, int32_t &c) {
+            g = 0.f;
+            c = 0;
+            if (key < n_nodes) {
+                g = gbuf[idx];
+                c = walks[idx >> shift];                  // contribution idx belongs to position idx >> shift
+            }
+        };
+        uint32_t my_key, key1, idx0, idx1;
+        float g;
+        int32_t c;
+        link1(base + lane, my_key, idx0);
+        link1(base + 32 + lane, key1, idx1);
+        link2(my_key, idx0, g, c);
+        for (int64_t s0 = base; s0 < end; s0 += 32) {
+            uint32_t key2, idx2;
+            link1(s0 + 64 + lane, key2, idx2);
+            float g1;
+            int32_t c1;
+            link2(key1, idx1, g1, c1);
+            const bool usable = my_key < n_nodes;                     // sorted: usable lanes are a prefix
+            uint32_t before = __shfl_up_sync(0xffffffffu, my_key, 1);
+            if (lane == 0) before = carry_key;
+            carry_key = __shfl_sync(0xffffffffu, my_key, 31);
+            const unsigned hmask = __ballot_sync(0xffffffffu, usable && my_key != before);
+            const int n = __popc(__ballot_sync(0xffffffffu, usable));
+            // G contributions at a time: their center rows are loaded together, then added in
+            // index order; where the head mask has a bit the run before ends and a new one starts
+            auto add_one = [&](int i, float gq, const Row<FPL> &row) {
+                if ((hmask >> i) & 1u) {                              // a run starts here (same on every lane)
+                    if (have) close_inner();
+                    have = true;
+                    lead = false;
+                    cur_key = __shfl_sync(0xffffffffu, my_key, i);
+#pragma unroll
+                    for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(gq, row.v[j], acc.v[j]);
+            };
+            // lane l asks for line l of the G rows that follow group q0: the rest of this chunk, or
+            // (behind the last group) the start of the next chunk, whose metadata is there by then
+            auto prefetch_next = [&](int q0) {
+                const int x = lane * 128 / ROW_BYTES;
+                int32_t cn;
+                bool there;
+                if (q0 + 2 * G <= 32) {
+                    cn = __shfl_sync(0xffffffffu, c, (q0 + G + x) & 31);
+                    there = q0 + G + x < n;
+                } else {
+                    cn = __shfl_sync(0xffffffffu, c1, x & 31);
+                    there = n == 32;                                  // unusable entries carry row 0
+                }
+                if (lane * 128 < G * ROW_BYTES && there)
+                    asm volatile("prefetch.global.L1 [%0];" ::
+                                 "l"((const char *)(w_in + (int64_t)cn * (FPL * 32)) + lane * 128 % ROW_BYTES));
+            };
+            int q0 = 0;
+#pragma unroll 1
+            for (; q0 + G <= n; q0 += G) {
+                Row<FPL> ru[G];
+#pragma unroll
+                for (int q = 0; q < G; ++q)
+                    ru[q] = row_load<FPL>(w_in, (int64_t)__shfl_sync(0xffffffffu, c, q0 + q), lane);
+                prefetch_next(q0);
+#pragma unroll
+                for (int q = 0; q < G; ++q) add_one(q0 + q, __shfl_sync(0xffffffffu, g, q0 + q), ru[q]);
+            }
+#pragma unroll 1
+            for (; q0 < n; ++q0) {                                    // only where the output-row keys end
+                const Row<FPL> r1 = row_load<FPL>(w_in, (int64_t)__shfl_sync(0xffffffffu, c, q0), lane);
+                add_one(q0, __shfl_sync(0xffffffffu, g, q0), r1);
+            }
+            if (n < 32) break;                                        // the rest is not ours
+            my_key = key1; g = g1; c = c1;
+            key1 = key2; idx1 = idx2;
+        }
+        if (have) {
+            const bool goes_on = end < (int64_t)n_keys && keys[end] == cur_key;
+            if (goes_on && !lead) store_part(tail_part);              // first piece of a cut run
+            else close_inner();                                       // (a middle piece is a lead piece)
+        }
+    }
+}
+
+// The last launch of a step does three independent jobs at once, by block role, instead of three
+// small launches one after another (each of them too small to fill the device):
+//   blocks [0, in_blocks)                      pass 4: the input rows of the centers,
+//   blocks [in_blocks, in_blocks + fix_blocks) the output rows whose runs were cut at block boundaries,
+//   the last block                             the fixed-order sums of losses and counters.
+//
+// Cut runs: one warp per block of RUN_CUT sorted positions: if a run starts in the block and
+// continues past its end, add its pieces (tail of this block, then the leading pieces of the
+// following blocks while they carry the same key) and write the row.
+template <int FPL, typename T>
+__device__ __forceinline__ void finish_cut_runs(int64_t warp, int64_t n_warps, T *__restrict__ w_out,
+                                                const uint32_t *__restrict__ keys, uint32_t n_keys,
+                                                uint32_t n_nodes, float lr,
+                                                const double *__restrict__ lead_part,
+                                                const double *__restrict__ tail_part, const MomState &ms)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t n_blocks = ((int64_t)n_keys + RUN_CUT - 1) / RUN_CUT;
+    for (int64_t b = warp; b + 1 < n_blocks; b += n_warps) {
         const int64_t last = (b + 1) * RUN_CUT - 1;                  // last position of block b
         const uint32_t key = keys[last];
         if (key >= n_nodes || keys[last + 1] != key) continue;       // nothing crosses this boundary
@@ -983,38 +1257,20 @@ sgns_apply_out_fixup_kernel(T *__restrict__ w_out, const uint32_t *__restrict__ 
 
 // Pass 4, keys in [n_nodes, 2 n_nodes): u_row -= lr * sum of the positions' GU rows.
 // The center keys sort behind every output-row key and before the invalid ones, so they form one
-// stretch of at most n_pos sorted positions.  Every warp finds where that stretch starts (a
-// search over keys that stay in L2) and then takes ONE position of it: if a run of equal keys
-// starts there, the warp sums the run's GU rows in index order and writes the row.  (A warp per 32
-// sorted positions left the whole pass to the few hundred warps whose chunk held center keys.)
+// stretch of at most n_pos sorted positions, and it starts at position *n_out: part A counted
+// the output-row keys it wrote.  Every warp takes ONE position of the stretch: if a run of equal
+// keys starts there, the warp sums the run's GU rows in index order and writes the row.
 template <int FPL, typename T>
-__global__ void __launch_bounds__(256)
-sgns_apply_in_kernel(T *__restrict__ w_in, const float *__restrict__ GU,
-                     const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals,
-                     uint32_t n_keys, uint32_t n_nodes, uint32_t n_slots, uint32_t n_pos, float lr,
-                     MomState ms)
+__device__ __forceinline__ void finish_input_rows(int64_t warp, int64_t n_warps, T *__restrict__ w_in,
+                                                  const float *__restrict__ GU,
+                                                  const uint32_t *__restrict__ keys,
+                                                  const uint32_t *__restrict__ vals, uint32_t n_keys,
+                                                  uint32_t n_nodes, uint32_t n_slots, uint32_t n_pos,
+                                                  int64_t first, float lr, const MomState &ms)
 {
     constexpr int U = FPL <= 4 ? 8 : 4;
     const int lane = threadIdx.x & 31;
-    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    // first sorted position whose key is not an output row: 32-way search, the lanes probe 32
-    // evenly spaced positions per step (5 round trips for 2^25 keys instead of 25)
-    int64_t first = 0;
-    {
-        int64_t lo = 0, hi = n_keys;                               // answer in [lo, hi]
-        while (hi - lo > 32) {
-            const int64_t step = (hi - lo + 31) / 32;
-            const int64_t p = lo + (int64_t)(lane + 1) * step - 1;  // last position of slice `lane`
-            const bool below = p < hi && keys[p] < n_nodes;         // the whole slice is below
-            const int full = __popc(__ballot_sync(0xffffffffu, below));   // sorted: a prefix of lanes
-            lo += (int64_t)full * step;
-            if (lo + step < hi) hi = lo + step;
-        }
-        const bool below = lo + lane < hi && keys[lo + lane] < n_nodes;
-        first = lo + __popc(__ballot_sync(0xffffffffu, below));
-    }
-    for (int64_t wi = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); wi < (int64_t)n_pos;
-         wi += n_warps) {
+    for (int64_t wi = warp; wi < (int64_t)n_pos; wi += n_warps) {
         const int64_t i = first + wi;
         if (i >= (int64_t)n_keys) break;
         const uint32_t key = keys[i];
@@ -1050,29 +1306,114 @@ sgns_apply_in_kernel(T *__restrict__ w_in, const float *__restrict__ GU,
     }
 }
 
-// Fixed-order reduction of the per-position losses and pair counts (one block).
-__global__ void __launch_bounds__(1024)
-sgns_reduce_kernel(const double *__restrict__ loss_pos, const int32_t *__restrict__ pairs_pos,
-                   int64_t n_pos, double *loss_out, long long *pairs_out, unsigned long long *masked_out)
+// Pass 4 for fp32 tables and plain SGD: one warp per 32 sorted center positions.  The lanes fetch
+// the metadata of the 32 positions at once and the GU rows G at a time; a run (the positions of
+// one center node) is summed in index order by the warp whose chunk holds its first position -
+// reading on past the chunk's end in the rare case that the run does - and goes out as one
+// reduction per value, row += -lr * sum, the only addition that row receives in the step.
+template <int FPL>
+__device__ __forceinline__ void finish_input_rows_sgd(int64_t warp, int64_t n_warps, float *__restrict__ w_in,
+                                                      const float *__restrict__ GU,
+                                                      const uint32_t *__restrict__ keys,
+                                                      const uint32_t *__restrict__ vals, uint32_t n_keys,
+                                                      uint32_t n_nodes, uint32_t n_slots, uint32_t n_pos,
+                                                      int64_t first, float lr)
 {
-    __shared__ double sl[1024];
-    __shared__ long long sp[1024], sm[1024];
+    constexpr int G = FPL <= 4 ? 8 : 4;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_chunks = ((int64_t)n_pos + 31) / 32;
+    for (int64_t ch = warp; ch < n_chunks; ch += n_warps) {
+        const int64_t i0 = first + ch * 32;
+        if (i0 >= (int64_t)n_keys) break;
+        const int64_t i = i0 + lane;
+        const uint32_t key = i < (int64_t)n_keys ? keys[i] : 0xFFFFFFFFu;
+        const bool usable = key >= n_nodes && key < 2u * n_nodes;    // sorted: usable lanes are a prefix
+        const uint32_t pos = usable ? vals[i] - n_slots : 0u;
+        uint32_t before = __shfl_up_sync(0xffffffffu, key, 1);
+        if (lane == 0) before = i0 > 0 ? keys[i0 - 1] : 0xFFFFFFFFu;
+        const unsigned hmask = __ballot_sync(0xffffffffu, usable && key != before);
+        const int n = __popc(__ballot_sync(0xffffffffu, usable));
+        if (hmask == 0) { if (n < 32) break; else continue; }        // no run starts in this chunk
+        bool have = false;
+        uint32_t cur_key = 0;
+        Row<FPL> acc;
+#pragma unroll
+        for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+        auto close = [&]() {
+            Row<FPL> d;
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) d.v[j] = -lr * acc.v[j];
+            row_red_add<FPL>(w_in, (int64_t)(cur_key - n_nodes), lane, d);
+        };
+        auto add_one = [&](int q, const Row<FPL> &row) {
+            if ((hmask >> q) & 1u) {
+                if (have) close();
+                have = true;
+                cur_key = __shfl_sync(0xffffffffu, key, q);
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < FPL; ++j) acc.v[j] += row.v[j];
+        };
+        int q0 = __ffs(hmask) - 1;                                    // entries before it belong to an earlier run
+#pragma unroll 1
+        for (; q0 + G <= n; q0 += G) {
+            Row<FPL> r[G];
+#pragma unroll
+            for (int q = 0; q < G; ++q)
+                r[q] = row_load<FPL>(GU, (int64_t)__shfl_sync(0xffffffffu, pos, q0 + q), lane);
+#pragma unroll
+            for (int q = 0; q < G; ++q) add_one(q0 + q, r[q]);
+        }
+#pragma unroll 1
+        for (; q0 < n; ++q0) {
+            const Row<FPL> r1 = row_load<FPL>(GU, (int64_t)__shfl_sync(0xffffffffu, pos, q0), lane);
+            add_one(q0, r1);
+        }
+        if (n == 32) {                                                // the last run may go on past the chunk
+            for (int64_t y = i0 + 32; y < (int64_t)n_keys && keys[y] == cur_key; ++y) {
+                const Row<FPL> r1 = row_load<FPL>(GU, (int64_t)(vals[y] - n_slots), lane);
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) acc.v[j] += r1.v[j];
+            }
+        }
+        close();
+        if (n < 32) break;
+    }
+}
+
+// Fixed-order reduction of the per-position losses and counters by one block of 256 threads:
+// thread t adds positions t, t + 256, ... in that order, then a binary tree over the threads.
+__device__ __forceinline__ void finish_sums(const double *__restrict__ loss_pos,
+                                            const int32_t *__restrict__ pairs_pos, int64_t n_pos,
+                                            double *loss_out, long long *pairs_out,
+                                            unsigned long long *masked_out, unsigned long long *refused_out)
+{
+    __shared__ double sl[256];
+    __shared__ long long sp[256], sm[256];
+    __shared__ unsigned int sr[256];
     double l = 0.0;
     long long p = 0, m = 0;
-    for (int64_t x = threadIdx.x; x < n_pos; x += 1024) {
+    unsigned int r = 0;
+    for (int64_t x = threadIdx.x; x < n_pos; x += 256) {
+        const int32_t packed = pairs_pos[x];             // pairs | masked negatives << 8 | refused ids << 20
         l += loss_pos[x];
-        p += pairs_pos[x] & 0xFF;                        // pairs | masked negatives << 8
-        m += pairs_pos[x] >> 8;
+        p += packed & 0xFF;
+        m += (packed >> 8) & 0xFFF;
+        r += (unsigned)packed >> 20;
     }
     sl[threadIdx.x] = l;
     sp[threadIdx.x] = p;
     sm[threadIdx.x] = m;
+    sr[threadIdx.x] = r;
     __syncthreads();
-    for (int o = 512; o > 0; o >>= 1) {
+    for (int o = 128; o > 0; o >>= 1) {
         if (threadIdx.x < o) {
             sl[threadIdx.x] += sl[threadIdx.x + o];
             sp[threadIdx.x] += sp[threadIdx.x + o];
             sm[threadIdx.x] += sm[threadIdx.x + o];
+            sr[threadIdx.x] += sr[threadIdx.x + o];
         }
         __syncthreads();
     }
@@ -1080,6 +1421,48 @@ sgns_reduce_kernel(const double *__restrict__ loss_pos, const int32_t *__restric
         if (loss_out) *loss_out += sl[0];
         if (pairs_out) *pairs_out += sp[0];
         if (masked_out) *masked_out += (unsigned long long)sm[0];
+        if (refused_out && sr[0]) atomicAdd(refused_out, (unsigned long long)sr[0]);
+    }
+}
+
+struct FinishArgs {
+    const uint32_t *keys, *vals, *n_out;
+    const float *GU;
+    const double *lead_part, *tail_part, *loss_pos;
+    const int32_t *pairs_pos;
+    uint32_t n_keys, n_nodes, n_slots, n_pos;
+    float lr;
+    int in_blocks, fix_blocks;
+    int light;                    // fp32 tables and plain SGD: input rows by reductions
+    double *loss_out;
+    long long *pairs_out;
+    unsigned long long *masked_out, *refused_out;
+};
+
+template <int FPL, typename T>
+__global__ void __launch_bounds__(256)
+sgns_finish_kernel(T *__restrict__ w_in, T *__restrict__ w_out, FinishArgs fa, MomState ms_in, MomState ms_out)
+{
+    const int wpb = blockDim.x >> 5;
+    const int b = (int)blockIdx.x;
+    if (b < fa.in_blocks) {
+        const int64_t warp = (int64_t)b * wpb + (threadIdx.x >> 5), n_warps = (int64_t)fa.in_blocks * wpb;
+        if constexpr (std::is_same<T, float>::value) {
+            if (fa.light) {
+                finish_input_rows_sgd<FPL>(warp, n_warps, w_in, fa.GU, fa.keys, fa.vals, fa.n_keys, fa.n_nodes,
+                                           fa.n_slots, fa.n_pos, (int64_t)*fa.n_out, fa.lr);
+                return;
+            }
+        }
+        finish_input_rows<FPL, T>(warp, n_warps, w_in, fa.GU, fa.keys, fa.vals, fa.n_keys, fa.n_nodes,
+                                  fa.n_slots, fa.n_pos, (int64_t)*fa.n_out, fa.lr, ms_in);
+    } else if (b < fa.in_blocks + fa.fix_blocks) {
+        finish_cut_runs<FPL, T>((int64_t)(b - fa.in_blocks) * wpb + (threadIdx.x >> 5),
+                                (int64_t)fa.fix_blocks * wpb, w_out, fa.keys, fa.n_keys, fa.n_nodes, fa.lr,
+                                fa.lead_part, fa.tail_part, ms_out);
+    } else {
+        finish_sums(fa.loss_pos, fa.pairs_pos, (int64_t)fa.n_pos, fa.loss_out, fa.pairs_out, fa.masked_out,
+                    fa.refused_out);
     }
 }
 
@@ -1099,6 +1482,8 @@ struct SgnsArgs {
     int32_t *dump_pairs, *dump_negs;
     int fwd;                      // PAIR_* flags of build_targets
     unsigned long long *masked;   // nullable: masked negatives are ADDED
+    int prepared;                 // >= 0: scratch set in which part A of this batch already ran
+    unsigned long long *refused;  // nullable: ids treated as absent because they name no row are ADDED
 };
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
@@ -1125,7 +1510,7 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
     kern<<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
         (T *)a.w_in, (T *)a.w_out, a.walks, a.n_walks, a.walk_id_base, a.L, a.w, a.K, a.alias,
         (uint32_t)a.n_nodes, a.lr, a.seed, a.loss, (unsigned long long *)a.pairs, a.dump_pairs,
-        a.dump_negs, ticket, a.fwd, a.masked);
+        a.dump_negs, ticket, a.fwd, a.masked, a.refused);
     GS_CUDA_TRY(cudaGetLastError());
     return GS_OK;
 }
@@ -1164,11 +1549,130 @@ struct MomHost {
     int64_t step;
 };
 
+// Scratch of one synchronous step.  By default it comes from the growing per-device cache, which
+// holds two sets so that part A of one batch can run while part B of the batch before it is
+// still reading its own; a caller that must not allocate hands in a fixed block instead
+// (gs_sgns_step_static), and a batch that does not fit it is refused.
+struct FixedScratch {
+    unsigned char *ptr;
+    size_t bytes;
+};
+
+struct SyncScratch {
+    uint32_t *keys;               // part A: destination row per slot, then one center key per position
+    uint32_t *keysB, *valsB, *keysC, *valsC, *counts;   // sort buffers
+    uint32_t *ks, *vs;            // where the sorted keys / contribution indices end up (B or C)
+    float *gbuf, *GU;
+    double *loss_pos;
+    int32_t *pairs_pos;
+    uint32_t *tinfo;              // per position: contexts | all targets << 16 of its dense list
+    uint32_t *n_out;              // output-row keys of the batch (one counter)
+    double *lead_part, *tail_part;
+    int64_t n_pos, n_slots, n_keys, n_cut;
+    int SL, shift, bits;          // a position's list occupies 2^shift >= SL entries
+};
+
+// Lays the arrays of one step out in `base` (nullptr: sizes only).  Returns the bytes needed.
+static size_t sync_layout(const SgnsArgs &a, unsigned char *base, SyncScratch *out)
+{
+    SyncScratch s;
+    s.SL = 2 * a.w * (1 + a.K);
+    s.shift = bit_length((uint64_t)s.SL - 1);            // smallest power of two >= SL
+    s.n_pos = a.n_walks * a.L;
+    s.n_slots = s.n_pos << s.shift;
+    s.n_keys = s.n_slots + s.n_pos;
+    s.n_cut = (s.n_keys + RUN_CUT - 1) / RUN_CUT;
+    s.bits = bit_length(2ull * (uint64_t)a.n_nodes);
+    const size_t b_keys = align_up(sizeof(uint32_t) * (size_t)s.n_keys);
+    const size_t b_g = align_up(sizeof(float) * (size_t)s.n_slots);
+    const size_t b_gu = align_up(sizeof(float) * (size_t)s.n_pos * a.dim);
+    const size_t b_loss = align_up(sizeof(double) * (size_t)s.n_pos);
+    const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)s.n_pos);
+    const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)s.n_keys));
+    const size_t b_part = align_up(sizeof(double) * (size_t)s.n_cut * a.dim);
+    unsigned char *p = base;
+    s.keys = (uint32_t *)p; p += b_keys;
+    s.keysB = (uint32_t *)p; p += b_keys;
+    s.valsB = (uint32_t *)p; p += b_keys;
+    s.keysC = (uint32_t *)p; p += b_keys;
+    s.valsC = (uint32_t *)p; p += b_keys;
+    s.gbuf = (float *)p; p += b_g;
+    s.GU = (float *)p; p += b_gu;
+    s.loss_pos = (double *)p; p += b_loss;
+    s.pairs_pos = (int32_t *)p; p += b_pairs;
+    s.tinfo = (uint32_t *)p; p += b_pairs;
+    s.n_out = (uint32_t *)p; p += 256;
+    s.counts = (uint32_t *)p; p += b_cnt;
+    s.lead_part = (double *)p; p += b_part;
+    s.tail_part = (double *)p; p += b_part;
+    // the sort alternates B, C, B, ...: an odd number of passes ends in B
+    const int passes = (s.bits + 7) / 8;
+    s.ks = (passes & 1) ? s.keysB : s.keysC;
+    s.vs = (passes & 1) ? s.valsB : s.valsC;
+    if (out) *out = s;
+    return (size_t)(p - base);
+}
+
+// Finds the scratch of set `set` (0 or 1) of the current device, or the caller's fixed block.
+static gs_status sync_scratch(const SgnsArgs &a, int set, const FixedScratch *fixed, SyncScratch *out)
+{
+    SyncScratch probe;
+    const size_t need = sync_layout(a, nullptr, &probe);
+    if (probe.n_keys > ((int64_t)1 << 30)) {
+        set_error("deterministic step: %lld slots exceed 2^30; use smaller batches", (long long)probe.n_keys);
+        return GS_ERR_UNSUPPORTED;
+    }
+    void *ws = nullptr;
+    if (fixed) {
+        if (need > fixed->bytes) {
+            set_error("gs_sgns_step_static: this batch needs %zu bytes of scratch, the fixed array has %zu; "
+                      "pass fewer walks per call or use gs_sgns_step", need, fixed->bytes);
+            return GS_ERR_UNSUPPORTED;
+        }
+        // Every byte that is read is written first by the pass before it (keys and pair counts
+        // by the targets pass for all slots; digit counts by the histogram pass for all tiles;
+        // g, GU and losses by the coefficient pass wherever the apply passes read them; the
+        // partial sums of cut runs by the apply pass before the fix-up pass reads exactly
+        // those), so nothing left over from an earlier call can leak in.
+        ws = fixed->ptr;
+    } else {
+        gs_status s = workspace_get(set ? WS_SGNS1 : WS_SGNS, need, &ws);
+        if (s != GS_OK) return s;
+    }
+    sync_layout(a, (unsigned char *)ws, out);
+    return GS_OK;
+}
+
+// Part A of the synchronous step (no table is read): targets and keys of every slot, sorted.
+static gs_status sync_prepare(const SgnsArgs &a, int set, const FixedScratch *fixed, cudaStream_t st)
+{
+    SyncScratch sc;
+    gs_status s = sync_scratch(a, set, fixed, &sc);
+    if (s != GS_OK) return s;
+    const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * sc.SL;
+    int64_t blocks = (sc.n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
+    if (blocks > (int64_t)sm_count() * 16) blocks = (int64_t)sm_count() * 16;
+    GS_CUDA_TRY(cudaMemsetAsync(sc.n_out, 0, sizeof(uint32_t), st));
+    sgns_targets_kernel<<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
+        a.walks, sc.n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias, (uint32_t)a.n_nodes,
+        (uint32_t)a.n_nodes, a.seed, sc.shift, sc.keys, sc.tinfo, sc.pairs_pos, sc.n_out, a.dump_pairs,
+        a.dump_negs, a.fwd);
+    GS_CUDA_TRY(cudaGetLastError());
+    uint32_t *ks = nullptr, *vs = nullptr;
+    radix_sort_pairs(sc.keys, sc.keysB, sc.valsB, sc.keysC, sc.valsC, (uint32_t)sc.n_keys, sc.bits,
+                     sc.counts, st, &ks, &vs);
+    GS_CUDA_TRY(cudaGetLastError());
+    if (ks != sc.ks || vs != sc.vs) { set_error("internal: sort result buffer mismatch"); return GS_ERR_CUDA; }
+    return GS_OK;
+}
+
+// Part B: coefficients from the entry tables, then the apply passes over the sorted contributions.
 template <int DIM, typename T>
-static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const MomHost *mom = nullptr)
+static gs_status sync_update(const SgnsArgs &a, int set, const FixedScratch *fixed, cudaStream_t st,
+                             const MomHost *mom)
 {
     T *w_in = (T *)a.w_in, *w_out = (T *)a.w_out;
-    constexpr int FPL = DIM / 32;                        // the apply passes use a whole warp per row
+    constexpr int FPL = DIM / 32;                        // the passes use a whole warp per row
     MomState ms_in = { nullptr, nullptr, 0.f, 0 }, ms_out = { nullptr, nullptr, 0.f, 0 };
     const bool adam = mom && mom->v_in;
     if (adam) {
@@ -1176,94 +1680,80 @@ static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const Mom
         const double c2 = 1.0 - pow((double)mom->b2, (double)mom->step);
         ms_in = MomState{ mom->m_in, nullptr, mom->mu, 0, mom->v_in, mom->b2, mom->eps, c1, c2 };
         ms_out = MomState{ mom->m_out, nullptr, mom->mu, 0, mom->v_out, mom->b2, mom->eps, c1, c2 };
-        mom = nullptr;                                   // no lazy catch-up: the plain order of passes
     } else if (mom) {
         ms_in = MomState{ mom->m_in, mom->last_in, mom->mu, mom->iter + 1 };
         ms_out = MomState{ mom->m_out, mom->last_out, mom->mu, mom->iter + 1 };
     }
-    const int SL = 2 * a.w * (1 + a.K);
-    const int64_t n_pos = a.n_walks * a.L;
-    const int64_t n_slots = n_pos * SL;
-    const int64_t n_keys = n_slots + n_pos;
-    if (n_keys > ((int64_t)1 << 30)) {
-        set_error("deterministic step: %lld slots exceed 2^30; use smaller batches",
-                  (long long)n_keys);
-        return GS_ERR_UNSUPPORTED;
-    }
-    // scratch carve-up
-    const size_t b_keys = align_up(sizeof(uint32_t) * (size_t)n_keys);
-    const size_t b_g = align_up(sizeof(float) * (size_t)n_slots);
-    const size_t b_gu = align_up(sizeof(float) * (size_t)n_pos * a.dim);
-    const size_t b_loss = align_up(sizeof(double) * (size_t)n_pos);
-    const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)n_pos);
-    const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)n_keys));
-    const int64_t n_cut = (n_keys + RUN_CUT - 1) / RUN_CUT;
-    const size_t b_part = align_up(sizeof(double) * (size_t)n_cut * a.dim);
-    void *ws = nullptr;
-    gs_status s = workspace_get(WS_SGNS, 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt + 2 * b_part, &ws);
+    SyncScratch sc;
+    gs_status s = sync_scratch(a, set, fixed, &sc);
     if (s != GS_OK) return s;
-    char *p = (char *)ws;
-    uint32_t *keysA = (uint32_t *)p; p += b_keys;
-    uint32_t *keysB = (uint32_t *)p; p += b_keys;
-    uint32_t *valsA = (uint32_t *)p; p += b_keys;
-    uint32_t *valsB = (uint32_t *)p; p += b_keys;
-    float *gbuf = (float *)p; p += b_g;
-    float *GU = (float *)p; p += b_gu;
-    double *loss_pos = (double *)p; p += b_loss;
-    int32_t *pairs_pos = (int32_t *)p; p += b_pairs;
-    uint32_t *counts = (uint32_t *)p; p += b_cnt;
-    double *lead_part = (double *)p; p += b_part;
-    double *tail_part = (double *)p;
-
-    const size_t coef_smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
-    int64_t coef_blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
-    if (coef_blocks > (int64_t)sm_count() * 16) coef_blocks = (int64_t)sm_count() * 16;
-#define GS_COEF(MODE)                                                                              \
-    sgns_coef_kernel<DIM, T, MODE><<<(unsigned)coef_blocks, SGNS_WARPS * 32, coef_smem, st>>>(         \
-        w_in, w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias, (uint32_t)a.n_nodes, \
-        (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos, a.dump_pairs, a.dump_negs, a.fwd)
-    if (mom) GS_COEF(1); else GS_COEF(0);            // with momentum: the keys first, no table reads
-    GS_CUDA_TRY(cudaGetLastError());
-    uint32_t *ks = nullptr, *vs = nullptr;
-    radix_sort_pairs(keysA, valsA, keysB, valsB, (uint32_t)n_keys,
-                     bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
-    GS_CUDA_TRY(cudaGetLastError());
-    if (mom) {
-        // bring every row the batch touches up to iteration `iter`, then compute the coefficients
-        int64_t cb = (n_keys + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 8 * 8;
+    if (mom && !adam) {
+        // lazy momentum: bring every row the batch touches up to iteration `iter` before it is read
+        int64_t cb = (sc.n_keys + 255) / 256;
         if (cb > (int64_t)sm_count() * 64) cb = (int64_t)sm_count() * 64;
         if constexpr (sizeof(T) == 4)
             momentum_catchup_kernel<FPL><<<(unsigned)cb, 256, 0, st>>>(
-                w_in, w_out, ms_in, ms_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, mom->iter);
-        GS_CUDA_TRY(cudaGetLastError());
-        GS_COEF(2);
+                w_in, w_out, ms_in, ms_out, sc.ks, (uint32_t)sc.n_keys, (uint32_t)a.n_nodes, a.lr, mom->iter);
         GS_CUDA_TRY(cudaGetLastError());
     }
-#undef GS_COEF
     {
-        const int64_t cap = (int64_t)sm_count() * 8 * 8;
-        sgns_apply_out_kernel<FPL, T><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-            w_in, w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
-            lead_part, tail_part, ms_out);
-        GS_CUDA_TRY(cudaGetLastError());
-        if (n_cut > 1) {
-            sgns_apply_out_fixup_kernel<FPL, T><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-                w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part, ms_out);
-            GS_CUDA_TRY(cudaGetLastError());
-        }
-        int64_t in_blocks = (n_pos + 7) / 8;                    // one warp per center position
-        if (in_blocks > cap) in_blocks = cap;
-        sgns_apply_in_kernel<FPL, T><<<(unsigned)in_blocks, 256, 0, st>>>(
-            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, (uint32_t)n_pos,
-            a.lr, ms_in);
+        int64_t blocks = (sc.n_pos + 7) / 8;             // one warp per position
+        if (blocks > cap) blocks = cap;
+        sgns_coef_kernel<DIM, T><<<(unsigned)blocks, 256, 0, st>>>(
+            w_in, w_out, sc.n_pos, sc.shift, (uint32_t)a.n_nodes, sc.keys, sc.tinfo, sc.gbuf, sc.GU, sc.loss_pos);
         GS_CUDA_TRY(cudaGetLastError());
     }
-    if (a.loss || a.pairs || a.masked) {
-        sgns_reduce_kernel<<<1, 1024, 0, st>>>(loss_pos, pairs_pos, n_pos, a.loss,
-                                               (long long *)a.pairs, a.masked);
+    {
+        const unsigned out_blocks = (unsigned)((sc.n_cut + 7) / 8);
+        bool light = false;
+        if constexpr (sizeof(T) == 4) light = !mom;      // fp32 tables, plain SGD
+        if (light) {
+            if constexpr (sizeof(T) == 4)
+                sgns_apply_out_sgd_kernel<FPL><<<out_blocks, 256, 0, st>>>(
+                    w_in, w_out, a.walks, sc.ks, sc.vs, sc.gbuf, (uint32_t)sc.n_keys, (uint32_t)a.n_nodes,
+                    sc.shift, a.lr, sc.lead_part, sc.tail_part);
+        } else {
+            sgns_apply_out_kernel<FPL, T><<<out_blocks, 256, 0, st>>>(
+                w_in, w_out, a.walks, sc.ks, sc.vs, sc.gbuf, (uint32_t)sc.n_keys, (uint32_t)a.n_nodes, sc.shift,
+                a.lr, sc.lead_part, sc.tail_part, ms_out);
+        }
+        GS_CUDA_TRY(cudaGetLastError());
+    }
+    {
+        // last launch: input rows, cut runs of output rows, sums - independent jobs, by block role
+        bool light = false;
+        if constexpr (sizeof(T) == 4) light = !mom;      // fp32 tables, plain SGD
+        // input rows: one warp per center position, or (light) per 32 sorted center positions
+        int64_t in_blocks = light ? (sc.n_pos + 255) / 256 : (sc.n_pos + 7) / 8;
+        if (in_blocks > cap) in_blocks = cap;
+        int64_t fix_blocks = sc.n_cut > 1 ? (sc.n_cut + 7) / 8 : 0;
+        if (fix_blocks > cap) fix_blocks = cap;
+        const bool sums = a.loss || a.pairs || a.masked || a.refused;
+        FinishArgs fa = { sc.ks, sc.vs, sc.n_out, sc.GU, sc.lead_part, sc.tail_part, sc.loss_pos, sc.pairs_pos,
+                          (uint32_t)sc.n_keys, (uint32_t)a.n_nodes, (uint32_t)sc.n_slots, (uint32_t)sc.n_pos,
+                          a.lr, (int)in_blocks, (int)fix_blocks, light ? 1 : 0, a.loss, (long long *)a.pairs,
+                          a.masked, a.refused };
+        sgns_finish_kernel<FPL, T><<<(unsigned)(in_blocks + fix_blocks + (sums ? 1 : 0)), 256, 0, st>>>(
+            w_in, w_out, fa, ms_in, ms_out);
         GS_CUDA_TRY(cudaGetLastError());
     }
     return GS_OK;
+}
+
+// One synchronous step.  a.prepared >= 0: part A of this batch has already run into that scratch
+// set (gs_sgns_epoch does that on its walk stream); otherwise both parts run here, in order.
+template <int DIM, typename T>
+static gs_status run_deterministic(const SgnsArgs &a, cudaStream_t st, const MomHost *mom = nullptr,
+                                   const FixedScratch *fixed = nullptr)
+{
+    int set = a.prepared;
+    if (set < 0) {
+        set = 0;
+        gs_status s = sync_prepare(a, set, fixed, st);
+        if (s != GS_OK) return s;
+    }
+    return sync_update<DIM, T>(a, set, fixed, st, mom);
 }
 
 static int pair_flags_of(int32_t mode)
@@ -1285,11 +1775,11 @@ gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, con
                     int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                     const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                     int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
-                    unsigned long long *masked)
+                    unsigned long long *masked, int prepared)
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked };
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
     mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     switch (dim) {
         case 32: return run_mode<32, float>(a, mode, st);
@@ -1307,11 +1797,11 @@ gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, c
                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                         const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                         int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
-                        unsigned long long *masked)
+                        unsigned long long *masked, int prepared)
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked };
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
     mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     switch (dim) {
         case 64: return run_mode<64, __half>(a, mode, st);
@@ -1328,11 +1818,11 @@ gs_status sgns_step_bf16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, 
                          int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                          const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                          int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
-                         unsigned long long *masked)
+                         unsigned long long *masked, int prepared)
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked };
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
     mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
     switch (dim) {
         case 64: return run_mode<64, __nv_bfloat16>(a, mode, st);
@@ -1348,11 +1838,11 @@ gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_ou
                              int32_t *last_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                              int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                              const uint64_t *alias, float lr, float mu, int32_t iter, uint64_t seed,
-                             double *loss, int64_t *pairs, cudaStream_t st)
+                             double *loss, int64_t *pairs, cudaStream_t st, int prepared)
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, nullptr, nullptr, 0, nullptr };
+                   seed, loss, pairs, nullptr, nullptr, 0, nullptr, prepared, refused_counter() };
     MomHost mom = { m_in, m_out, last_in, last_out, mu, iter, nullptr, nullptr, 0.f, 0.f, 0 };
     switch (dim) {
         case 32: return run_deterministic<32, float>(a, st, &mom);
@@ -1369,11 +1859,12 @@ gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, fl
                          float *v_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                          int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                          const uint64_t *alias, float lr, float b1, float b2, float eps, int64_t step,
-                         uint64_t seed, int32_t pair_mode, double *loss, int64_t *pairs, cudaStream_t st)
+                         uint64_t seed, int32_t pair_mode, double *loss, int64_t *pairs, cudaStream_t st,
+                         int prepared)
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, nullptr, nullptr, pair_flags_of(pair_mode), nullptr };
+                   seed, loss, pairs, nullptr, nullptr, pair_flags_of(pair_mode), nullptr, prepared, refused_counter() };
     MomHost mom = { m_in, m_out, nullptr, nullptr, b1, 0, v_in, v_out, b2, eps, step };
     switch (dim) {
         case 32: return run_deterministic<32, float>(a, st, &mom);
@@ -1384,6 +1875,20 @@ gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, fl
             set_error("dim %d not supported (32, 64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;
     }
+}
+
+// Part A of the synchronous step for the epoch driver: lists and sorts the contributions of a
+// batch into scratch set `set` (0 or 1) without reading a table, so that it can run on another
+// stream while the batch before it is still being applied.  The step functions above then take
+// prepared = set.
+gs_status sgns_prepare_sync(int64_t n_nodes, int32_t dim, const int32_t *walks, int64_t n_walks,
+                            int64_t walk_id_base, int32_t L, int32_t w, int32_t K, const uint64_t *alias,
+                            uint64_t seed, int32_t pair_mode, int set, cudaStream_t st)
+{
+    if (n_walks == 0) return GS_OK;
+    SgnsArgs a = { nullptr, nullptr, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, 0.f,
+                   seed, nullptr, nullptr, nullptr, nullptr, pair_flags_of(pair_mode), nullptr, -1, nullptr };
+    return sync_prepare(a, set, nullptr, st);
 }
 
 gs_status momentum_flush(float *w, float *m, int32_t *last, int64_t n_rows, int32_t dim, float lr,
@@ -1434,89 +1939,6 @@ static gs_status static_scratch_address(unsigned char **out)
     return GS_OK;
 }
 
-// Same kernels and the same order of launches as run_deterministic, with the scratch
-// carved out of the fixed array instead of the growing per-device cache.
-template <int DIM>
-static gs_status run_deterministic_static(const SgnsArgs &a, unsigned char *scratch, cudaStream_t st)
-{
-    constexpr int FPL = DIM / 32;
-    float *w_in = (float *)a.w_in, *w_out = (float *)a.w_out;
-    const int SL = 2 * a.w * (1 + a.K);
-    const int64_t n_pos = a.n_walks * a.L;
-    const int64_t n_slots = n_pos * SL;
-    const int64_t n_keys = n_slots + n_pos;
-    const size_t b_keys = align_up(sizeof(uint32_t) * (size_t)n_keys);
-    const size_t b_g = align_up(sizeof(float) * (size_t)n_slots);
-    const size_t b_gu = align_up(sizeof(float) * (size_t)n_pos * a.dim);
-    const size_t b_loss = align_up(sizeof(double) * (size_t)n_pos);
-    const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)n_pos);
-    const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)n_keys));
-    const int64_t n_cut = (n_keys + RUN_CUT - 1) / RUN_CUT;
-    const size_t b_part = align_up(sizeof(double) * (size_t)n_cut * a.dim);
-    const size_t need = 4 * b_keys + b_g + b_gu + b_loss + b_pairs + b_cnt + 2 * b_part;
-    if (n_keys > ((int64_t)1 << 30) || need > (size_t)GS_STATIC_SCRATCH_BYTES) {
-        set_error("gs_sgns_step_static: this batch needs %zu bytes of scratch, the fixed array has %u; "
-                  "pass fewer walks per call or use gs_sgns_step", need, GS_STATIC_SCRATCH_BYTES);
-        return GS_ERR_UNSUPPORTED;
-    }
-    // Every byte that is read below is written first by the pass before it (keys, g, GU, loss
-    // and pair counts by the coefficient pass for all slots; digit counts by the histogram
-    // pass for all tiles; the partial sums of cut runs by the apply pass before the fix-up
-    // pass reads exactly those), so nothing left over from an earlier call can leak in.
-    char *p = (char *)scratch;
-    uint32_t *keysA = (uint32_t *)p; p += b_keys;
-    uint32_t *keysB = (uint32_t *)p; p += b_keys;
-    uint32_t *valsA = (uint32_t *)p; p += b_keys;
-    uint32_t *valsB = (uint32_t *)p; p += b_keys;
-    float *gbuf = (float *)p; p += b_g;
-    float *GU = (float *)p; p += b_gu;
-    double *loss_pos = (double *)p; p += b_loss;
-    int32_t *pairs_pos = (int32_t *)p; p += b_pairs;
-    uint32_t *counts = (uint32_t *)p; p += b_cnt;
-    double *lead_part = (double *)p; p += b_part;
-    double *tail_part = (double *)p;
-    {
-        const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * SL;
-        int64_t blocks = (n_pos + SGNS_WARPS - 1) / SGNS_WARPS;
-        const int64_t cap = (int64_t)sm_count() * 16;
-        if (blocks > cap) blocks = cap;
-        sgns_coef_kernel<DIM, float, 0><<<(unsigned)blocks, SGNS_WARPS * 32, smem, st>>>(
-            w_in, w_out, a.walks, n_pos, a.walk_id_base, a.L, a.w, a.K, a.alias,
-            (uint32_t)a.n_nodes, (uint32_t)a.n_nodes, a.seed, keysA, gbuf, GU, loss_pos, pairs_pos,
-            a.dump_pairs, a.dump_negs, a.fwd);
-        GS_CUDA_TRY(cudaGetLastError());
-    }
-    uint32_t *ks = nullptr, *vs = nullptr;
-    radix_sort_pairs(keysA, valsA, keysB, valsB, (uint32_t)n_keys,
-                     bit_length(2ull * (uint64_t)a.n_nodes), counts, st, &ks, &vs);
-    GS_CUDA_TRY(cudaGetLastError());
-    {
-        const int64_t cap = (int64_t)sm_count() * 8 * 8;
-        sgns_apply_out_kernel<FPL, float><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-            w_in, w_out, a.walks, ks, vs, gbuf, (uint32_t)n_keys, (uint32_t)a.n_nodes, SL, a.lr,
-            lead_part, tail_part, MomState{ nullptr, nullptr, 0.f, 0 });
-        GS_CUDA_TRY(cudaGetLastError());
-        if (n_cut > 1) {
-            sgns_apply_out_fixup_kernel<FPL, float><<<(unsigned)((n_cut + 7) / 8), 256, 0, st>>>(
-                w_out, ks, (uint32_t)n_keys, (uint32_t)a.n_nodes, a.lr, lead_part, tail_part,
-                MomState{ nullptr, nullptr, 0.f, 0 });
-            GS_CUDA_TRY(cudaGetLastError());
-        }
-        int64_t in_blocks = (n_pos + 7) / 8;                    // one warp per center position
-        if (in_blocks > cap) in_blocks = cap;
-        sgns_apply_in_kernel<FPL, float><<<(unsigned)in_blocks, 256, 0, st>>>(
-            w_in, GU, ks, vs, (uint32_t)n_keys, (uint32_t)a.n_nodes, (uint32_t)n_slots, (uint32_t)n_pos,
-            a.lr, MomState{ nullptr, nullptr, 0.f, 0 });
-        GS_CUDA_TRY(cudaGetLastError());
-    }
-    if (a.loss || a.pairs || a.masked) {
-        sgns_reduce_kernel<<<1, 1024, 0, st>>>(loss_pos, pairs_pos, n_pos, a.loss,
-                                               (long long *)a.pairs, a.masked);
-        GS_CUDA_TRY(cudaGetLastError());
-    }
-    return GS_OK;
-}
-
 }  // namespace gs
 
 extern "C" gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t dim,
@@ -1543,13 +1965,15 @@ extern "C" gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t 
     gs_status s = static_scratch_address(&scratch);
     if (s != GS_OK) return s;
     SgnsArgs a = { d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len, window,
-                   n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr, 0, nullptr };
+                   n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr, 0, nullptr, -1,
+                   nullptr /* this entry point touches no library-owned memory but its array */ };
     cudaStream_t st = (cudaStream_t)stream;
+    const FixedScratch fixed = { scratch, (size_t)GS_STATIC_SCRATCH_BYTES };
     switch (dim) {
-        case 32: return run_deterministic_static<32>(a, scratch, st);
-        case 64: return run_deterministic_static<64>(a, scratch, st);
-        case 128: return run_deterministic_static<128>(a, scratch, st);
-        case 256: return run_deterministic_static<256>(a, scratch, st);
+        case 32: return run_deterministic<32, float>(a, st, nullptr, &fixed);
+        case 64: return run_deterministic<64, float>(a, st, nullptr, &fixed);
+        case 128: return run_deterministic<128, float>(a, st, nullptr, &fixed);
+        case 256: return run_deterministic<256, float>(a, st, nullptr, &fixed);
         default:
             set_error("dim %d not supported (32, 64, 128, 256)", dim);
             return GS_ERR_UNSUPPORTED;

@@ -1,4 +1,4 @@
-// Stable least-significant-digit radix sort of (key, value) pairs, 8 bits per
+// Stable least-significant-digit radix sort of (key, value) pairs, at most 8 bits per
 // pass.  It groups the gradient contributions of a synchronous SGNS step by
 // destination row while keeping contributions of one row in index order, which
 // is what makes the summation order (and so the result bits) fixed.
@@ -16,8 +16,8 @@ constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 2048 keys per block
 constexpr int RADIX = 256;
 
 __global__ void __launch_bounds__(SORT_THREADS)
-sort_hist_kernel(const uint32_t *__restrict__ keys, uint32_t n, int shift, uint32_t n_tiles,
-                 uint32_t *__restrict__ counts)
+sort_hist_kernel(const uint32_t *__restrict__ keys, uint32_t n, int shift, uint32_t mask,
+                 uint32_t n_tiles, uint32_t *__restrict__ counts)
 {
     __shared__ uint32_t h[RADIX];
     h[threadIdx.x] = 0;
@@ -26,7 +26,7 @@ sort_hist_kernel(const uint32_t *__restrict__ keys, uint32_t n, int shift, uint3
 #pragma unroll
     for (int r = 0; r < SORT_ITEMS; ++r) {
         const uint32_t i = base + r * SORT_THREADS + threadIdx.x;
-        if (i < n) atomicAdd(&h[(keys[i] >> shift) & (RADIX - 1)], 1u);
+        if (i < n) atomicAdd(&h[(keys[i] >> shift) & mask], 1u);
     }
     __syncthreads();
     counts[threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
@@ -69,7 +69,7 @@ template <bool IOTA>
 __global__ void __launch_bounds__(SORT_THREADS)
 sort_scatter_kernel(const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in,
                     uint32_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out, uint32_t n,
-                    int shift, uint32_t n_tiles, const uint32_t *__restrict__ offsets,
+                    int shift, uint32_t mask, uint32_t n_tiles, const uint32_t *__restrict__ offsets,
                     const uint32_t *__restrict__ totals)
 {
     constexpr int WARPS = SORT_THREADS / 32;
@@ -105,7 +105,7 @@ sort_scatter_kernel(const uint32_t *__restrict__ keys_in, const uint32_t *__rest
         const bool ok = i < n;
         key[r] = ok ? keys_in[i] : 0u;
         val[r] = ok ? (IOTA ? i : vals_in[i]) : 0u;
-        const uint32_t d = ok ? ((key[r] >> shift) & (RADIX - 1)) : RADIX;   // RADIX = absent
+        const uint32_t d = ok ? ((key[r] >> shift) & mask) : RADIX;   // RADIX = absent
         const unsigned peers = __match_any_sync(0xffffffffu, d);
         const int leader = __ffs(peers) - 1;
         uint32_t before = 0;
@@ -133,7 +133,7 @@ sort_scatter_kernel(const uint32_t *__restrict__ keys_in, const uint32_t *__rest
     for (int r = 0; r < SORT_ITEMS; ++r) {
         const uint32_t i = base + r * 32 + lane;
         if (i < n) {
-            const uint32_t dst = cnt[wi][(key[r] >> shift) & (RADIX - 1)] + loc[r];
+            const uint32_t dst = cnt[wi][(key[r] >> shift) & mask] + loc[r];
             keys_out[dst] = key[r];
             vals_out[dst] = val[r];
         }
@@ -146,34 +146,49 @@ size_t sort_counts_bytes(uint32_t n)
     return sizeof(uint32_t) * ((size_t)RADIX * (n_tiles ? n_tiles : 1) + RADIX);   // + digit totals
 }
 
-// Sorts n pairs by the low `bits` bits of the key.  The first pass takes value i for
-// item i (no input value array).  Buffers A hold the input; on return *keys_sorted /
-// *vals_sorted point at whichever of A / B holds the result.  Returns launches made.
-int radix_sort_pairs(uint32_t *keysA, uint32_t *valsA, uint32_t *keysB, uint32_t *valsB,
-                     uint32_t n, int bits, uint32_t *counts, cudaStream_t st,
+// Digit widths of the passes: ceil(bits / 8) passes of equal width (21-bit keys sort as 7 + 7 + 7,
+// not 8 + 8 + 5: the same number of passes with a smaller scatter fan-out in each).
+static int digit_width(int bits)
+{
+    const int passes = (bits + 7) / 8;
+    return passes ? (bits + passes - 1) / passes : 8;
+}
+
+// Sorts n pairs by the low `bits` bits of the key.  The first pass reads keys_src, which is left
+// untouched, and takes value i for item i (there is no input value array); the passes then
+// alternate between buffers B and C.  On return *keys_sorted / *vals_sorted point at whichever of
+// B / C holds the result.  Returns launches made.
+int radix_sort_pairs(const uint32_t *keys_src, uint32_t *keysB, uint32_t *valsB, uint32_t *keysC,
+                     uint32_t *valsC, uint32_t n, int bits, uint32_t *counts, cudaStream_t st,
                      uint32_t **keys_sorted, uint32_t **vals_sorted)
 {
     const uint32_t n_tiles = (n + SORT_TILE - 1) / SORT_TILE;
-    uint32_t *kin = keysA, *vin = valsA, *kout = keysB, *vout = valsB;
+    const uint32_t *kin = keys_src, *vin = nullptr;
+    uint32_t *kout = keysB, *vout = valsB;
     uint32_t *totals = counts + (size_t)RADIX * (n_tiles ? n_tiles : 1);
     int launches = 0;
     bool first = true;
-    for (int shift = 0; shift < bits && n > 0; shift += 8) {
-        sort_hist_kernel<<<n_tiles, SORT_THREADS, 0, st>>>(kin, n, shift, n_tiles, counts);
+    if (bits < 1) bits = 1;                                  // at least one pass: the result lives in B
+    const int width = digit_width(bits);
+    for (int shift = 0; shift < bits && n > 0; shift += width) {
+        const uint32_t mask = (1u << width) - 1u;
+        sort_hist_kernel<<<n_tiles, SORT_THREADS, 0, st>>>(kin, n, shift, mask, n_tiles, counts);
         sort_scan_kernel<<<RADIX, 256, 0, st>>>(counts, n_tiles, totals);
         if (first)
             sort_scatter_kernel<true><<<n_tiles, SORT_THREADS, 0, st>>>(kin, vin, kout, vout, n,
-                                                                        shift, n_tiles, counts, totals);
+                                                                        shift, mask, n_tiles, counts, totals);
         else
             sort_scatter_kernel<false><<<n_tiles, SORT_THREADS, 0, st>>>(kin, vin, kout, vout, n,
-                                                                         shift, n_tiles, counts, totals);
+                                                                         shift, mask, n_tiles, counts, totals);
         launches += 3;
+        kin = kout;
+        vin = vout;
+        kout = kout == keysB ? keysC : keysB;
+        vout = vout == valsB ? valsC : valsB;
         first = false;
-        uint32_t *t = kin; kin = kout; kout = t;
-        t = vin; vin = vout; vout = t;
     }
-    *keys_sorted = kin;
-    *vals_sorted = vin;
+    *keys_sorted = const_cast<uint32_t *>(kin);
+    *vals_sorted = const_cast<uint32_t *>(vin);
     return launches;
 }
 

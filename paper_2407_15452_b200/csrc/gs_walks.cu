@@ -4,8 +4,9 @@
 // flight, not from per-walk parallelism: both samplers run one walk per THREAD.  The walk index
 // makes a uniform transition one random 16-byte read; the node2vec sampler flattens rejection
 // rounds and transitions into one loop and answers its neighbour test from a hashed edge set.
-// The kernels that give G lanes to a walk (speculative rejection rounds, first accepted round
-// wins) and the nested-loop kernel are kept for comparison behind gs_tune_node2vec_group.
+// The kernel that gives G lanes to a walk (speculative rejection rounds, first accepted round
+// wins) serves odd walk lengths and unaligned outputs, and any walk when gs_tune_node2vec_group
+// asks for it.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -209,7 +210,8 @@ __global__ void __launch_bounds__(256)
 uniform_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
                     const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
                     int64_t walk_id_base, int32_t L, uint64_t seed,
-                    int32_t *__restrict__ walks, unsigned long long *steps_out)
+                    int32_t *__restrict__ walks, unsigned long long *steps_out,
+                    unsigned long long *refused_out)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     unsigned int my_steps = 0;
@@ -217,6 +219,7 @@ uniform_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ co
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
         const bool bad = (uint64_t)(uint32_t)cur >= (uint64_t)n_nodes;   // start outside the graph: empty walk
+        if (bad && refused_out) atomicAdd(refused_out, 1ull);
         int32_t *W = walks + i * (int64_t)L;
         W[0] = bad ? -1 : cur;
         int32_t t = 0;
@@ -246,7 +249,8 @@ __global__ void __launch_bounds__(256, 6)
 uniform_walk_vec_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
                         const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
                         int64_t walk_id_base, int32_t L, uint64_t seed,
-                        int32_t *__restrict__ walks, unsigned long long *steps_out)
+                        int32_t *__restrict__ walks, unsigned long long *steps_out,
+                    unsigned long long *refused_out)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int quads = L >> 2;
@@ -255,6 +259,7 @@ uniform_walk_vec_kernel(const OffT *__restrict__ off, const int32_t *__restrict_
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
         bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
+        if (!alive && refused_out) atomicAdd(refused_out, 1ull);
         int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
         int4 pend = make_int4(0, 0, 0, 0);
         for (int q = 0; q < quads; ++q) {
@@ -328,7 +333,8 @@ __global__ void __launch_bounds__(256, 6)
 uniform_walk_index_kernel(const OffT *__restrict__ off, const int4 *__restrict__ rec,
                           const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
                           int64_t walk_id_base, int32_t L, uint64_t seed,
-                          int32_t *__restrict__ walks, unsigned long long *steps_out)
+                          int32_t *__restrict__ walks, unsigned long long *steps_out,
+                    unsigned long long *refused_out)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int quads = L >> 2;
@@ -337,6 +343,7 @@ uniform_walk_index_kernel(const OffT *__restrict__ off, const int4 *__restrict__
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
         bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
+        if (!alive && refused_out) atomicAdd(refused_out, 1ull);
         int64_t o0 = 0;
         uint32_t deg = 0;
         if (alive) {
@@ -378,7 +385,7 @@ uniform_walk_index_kernel(const OffT *__restrict__ off, const int4 *__restrict__
 
 gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
                                int64_t base, int32_t L, uint64_t seed, int32_t *walks,
-                               unsigned long long *steps, cudaStream_t st)
+                               unsigned long long *steps, unsigned long long *refused, cudaStream_t st)
 {
     if (n_walks == 0) return GS_OK;
     const int threads = 256;
@@ -388,16 +395,17 @@ gs_status launch_uniform_walks(const gs_graph *g, const int32_t *starts, int64_t
     const bool vec = (L % 4 == 0) && (((uintptr_t)walks & 15) == 0);
 #define GS_UW(KERNEL, T)                                                                        \
     KERNEL<T><<<(unsigned)blocks, threads, 0, st>>>((const T *)g->d_offsets, g->d_cols, starts, \
-                                                    g->n_nodes, n_walks, base, L, seed, walks, steps)
+                                                    g->n_nodes, n_walks, base, L, seed, walks, steps, \
+                                                    refused)
     if (vec && g->d_edge_rec) {
         if (g->offsets64)
             uniform_walk_index_kernel<int64_t><<<(unsigned)blocks, threads, 0, st>>>(
                 (const int64_t *)g->d_offsets, g->d_edge_rec, starts, g->n_nodes, n_walks, base, L,
-                seed, walks, steps);
+                seed, walks, steps, refused);
         else
             uniform_walk_index_kernel<int32_t><<<(unsigned)blocks, threads, 0, st>>>(
                 (const int32_t *)g->d_offsets, g->d_edge_rec, starts, g->n_nodes, n_walks, base, L,
-                seed, walks, steps);
+                seed, walks, steps, refused);
     } else if (g->offsets64) { if (vec) GS_UW(uniform_walk_vec_kernel, int64_t); else GS_UW(uniform_walk_kernel, int64_t); }
     else { if (vec) GS_UW(uniform_walk_vec_kernel, int32_t); else GS_UW(uniform_walk_kernel, int32_t); }
 #undef GS_UW
@@ -496,7 +504,8 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
                      const int32_t *__restrict__ starts, int64_t n_nodes, int64_t n_walks,
                      int64_t walk_id_base, int32_t L, uint64_t seed, N2VThresholds T,
                      int32_t max_rounds, int32_t *__restrict__ walks,
-                     unsigned long long *steps_out, unsigned long long *caps_out)
+                     unsigned long long *steps_out, unsigned long long *caps_out,
+                     unsigned long long *refused_out)
 {
     const int lane = threadIdx.x & 31;
     const int sub = lane % G;                       // round offset inside the group
@@ -516,6 +525,7 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
         int64_t p0 = 0, p1 = 0;                     // adjacency range of prev
         int32_t *W = walks + i * (int64_t)L;
         const bool bad = (uint64_t)(uint32_t)cur >= (uint64_t)n_nodes;   // same for the whole group
+        if (sub == 0 && bad && refused_out) atomicAdd(refused_out, 1ull);
         if (sub == 0) W[0] = bad ? -1 : cur;
         int32_t t = 0;
         for (; !bad && t + 1 < L; ++t) {
@@ -566,110 +576,17 @@ node2vec_walk_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
     if (caps_out && my_caps) atomicAdd(caps_out, (unsigned long long)my_caps);
 }
 
-// One walk per thread, nested loops (walks in flight matter more than lanes
-// per walk).  Rejection rounds run one after another; the state carries the adjacency range of
-// the current and of the previous node, so a round costs one random read (the proposal) plus,
-// when the draw falls between the two class thresholds, a binary search in adj(prev).  With the
-// walk index the proposal's record already holds the next node's range; without it the range
-// is read from the offsets at the start of the next transition.  Entries leave 32 bytes at a
-// time.  Needs L % 4 == 0 and a 16-byte aligned output.
-template <typename OffT, bool INDEX, bool HASH>
-__global__ void __launch_bounds__(256, 4)
-node2vec_thread_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
-                       const int4 *__restrict__ rec, const unsigned long long *__restrict__ edge_set,
-                       unsigned long long edge_mask, const int32_t *__restrict__ starts,
-                       int64_t n_nodes, int64_t n_walks, int64_t walk_id_base, int32_t L,
-                       uint64_t seed, N2VThresholds T, int32_t max_rounds,
-                       int32_t *__restrict__ walks, unsigned long long *steps_out,
-                       unsigned long long *caps_out)
-{
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const int quads = L >> 2;
-    const unsigned long long t_lo = T.t_near < T.t_far ? T.t_near : T.t_far;
-    const unsigned long long t_hi = T.t_near < T.t_far ? T.t_far : T.t_near;
-    unsigned int my_steps = 0, my_caps = 0;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_walks; i += stride) {
-        const uint64_t id = (uint64_t)(walk_id_base + i);
-        int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
-        bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
-        int64_t o0 = 0;
-        uint32_t deg = 0;
-        if (alive) {
-            o0 = ld_random(off + cur);
-            deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0);
-        }
-        int32_t prev = -1;
-        int64_t p0 = 0, p1 = 0;
-        int4 *W4 = reinterpret_cast<int4 *>(walks + i * (int64_t)L);
-        int4 pend = make_int4(0, 0, 0, 0);
-        for (int q = 0; q < quads; ++q) {
-            int32_t v[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int e = 4 * q + k;                       // entry index, transition t = e - 1
-                if (e > 0 && alive) {
-                    if (deg == 0) {
-                        alive = false;
-                    } else {
-                        int32_t x = -1;
-                        uint32_t xdeg = 0;
-                        int64_t xoff = 0;
-                        const int32_t rounds = e == 1 ? 1 : max_rounds;
-                        bool acc = false;
-                        for (int32_t sr = 0; sr < rounds && !acc; ++sr) {
-                            const uint4 r = draw(seed, id, (uint32_t)(e - 1), TAG_NODE2VEC, (uint32_t)sr);
-                            const int64_t at = o0 + (int64_t)__umulhi(r.x, deg);
-                            if (INDEX) {
-                                const int4 rc = ld_random(rec + at);
-                                x = rc.x;
-                                xdeg = (uint32_t)rc.y;
-                                xoff = (int64_t)(((uint64_t)(uint32_t)rc.w << 32) | (uint32_t)rc.z);
-                            } else {
-                                x = ld_random(col + at);
-                            }
-                            const unsigned long long r1 = r.y;
-                            if (e == 1) acc = true;            // first transition: uniform
-                            else if (x == prev) acc = r1 < T.t_prev;
-                            else if (r1 < t_lo) acc = true;
-                            else if (r1 >= t_hi) acc = false;
-                            else {
-                                const bool near = HASH ? edge_set_contains(edge_set, edge_mask, prev, x)
-                                                       : row_contains(col, p0, p1, x);
-                                acc = r1 < (near ? T.t_near : T.t_far);
-                            }
-                        }
-                        if (!acc) ++my_caps;                   // cap reached: keep the last proposal
-                        prev = cur; p0 = o0; p1 = o0 + deg;
-                        cur = x;
-                        if (INDEX) { o0 = xoff; deg = xdeg; }
-                        else { o0 = ld_random(off + cur); deg = (uint32_t)((int64_t)ld_random(off + cur + 1) - o0); }
-                        ++my_steps;
-                    }
-                }
-                v[k] = alive ? cur : -1;
-            }
-            const int4 now = make_int4(v[0], v[1], v[2], v[3]);
-            if (q & 1) { W4[q - 1] = pend; W4[q] = now; }
-            else if (q == quads - 1) W4[q] = now;
-            else pend = now;
-        }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        my_steps += __shfl_xor_sync(0xffffffffu, my_steps, o);
-        my_caps += __shfl_xor_sync(0xffffffffu, my_caps, o);
-    }
-    if ((threadIdx.x & 31) == 0) {
-        if (steps_out && my_steps) atomicAdd(steps_out, (unsigned long long)my_steps);
-        if (caps_out && my_caps) atomicAdd(caps_out, (unsigned long long)my_caps);
-    }
-}
-
-// One walk per thread again, but with the rejection rounds and the transitions of a walk flattened
-// into ONE loop: every trip of the loop is one round of whatever transition the lane is at.  In the
-// kernel above a lane that has accepted waits until the slowest lane of its warp has (the number of
-// rounds is geometric, so the slowest of 32 needs about three times the mean); here it starts its
-// next transition at once, and the memory system sees a request from every lane on every trip.
-// Finished entries collect in shared memory, eight per thread, and leave as two 16-byte stores.
+// One walk per thread (walks in flight matter more than lanes per walk), with the rejection rounds
+// and the transitions of a walk flattened into ONE loop: every trip of the loop is one round of
+// whatever transition the lane is at.  With nested loops a lane that has accepted waits until the
+// slowest lane of its warp has (the number of rounds is geometric, so the slowest of 32 needs
+// about three times the mean); here it starts its next transition at once, and the memory system
+// sees a request from every lane on every trip.  The state carries the adjacency range of the
+// current and of the previous node, so a round costs one random read (the proposal) plus, when
+// the draw falls between the two class thresholds, one membership test of adj(prev).  With the
+// walk index the proposal's record already holds the next node's range.  Finished entries
+// collect in shared memory, eight per thread, and leave as two 16-byte stores.  Needs
+// L % 4 == 0 and a 16-byte aligned output.
 template <typename OffT, bool INDEX, bool HASH>
 __global__ void __launch_bounds__(256, 4)
 node2vec_flat_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ col,
@@ -678,7 +595,7 @@ node2vec_flat_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
                      int64_t n_nodes, int64_t n_walks, int64_t walk_id_base, int32_t L,
                      uint64_t seed, N2VThresholds T, int32_t max_rounds,
                      int32_t *__restrict__ walks, unsigned long long *steps_out,
-                     unsigned long long *caps_out)
+                     unsigned long long *caps_out, unsigned long long *refused_out)
 {
     __shared__ int32_t buf[8][256];                        // buf[j][thread]: conflict-free
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -690,6 +607,7 @@ node2vec_flat_kernel(const OffT *__restrict__ off, const int32_t *__restrict__ c
         const uint64_t id = (uint64_t)(walk_id_base + i);
         int32_t cur = starts ? __ldg(starts + i) : (int32_t)(id % (uint64_t)n_nodes);
         bool alive = (uint64_t)(uint32_t)cur < (uint64_t)n_nodes;        // start outside the graph: empty walk
+        if (!alive && refused_out) atomicAdd(refused_out, 1ull);
         int64_t o0 = 0;
         uint32_t deg = 0;
         if (alive) {
@@ -787,7 +705,7 @@ template <typename OffT, int G>
 static void launch_n2v(const gs_graph *g, const int32_t *starts, int64_t n_walks, int64_t base,
                        int32_t L, uint64_t seed, const N2VThresholds &T, int32_t max_rounds,
                        int32_t *walks, unsigned long long *steps, unsigned long long *caps,
-                       cudaStream_t st)
+                       unsigned long long *refused, cudaStream_t st)
 {
     const int threads = 256;
     const int64_t per_block = threads / G;
@@ -796,34 +714,27 @@ static void launch_n2v(const gs_graph *g, const int32_t *starts, int64_t n_walks
     if (blocks > cap) blocks = cap;
     node2vec_walk_kernel<OffT, G><<<(unsigned)blocks, threads, 0, st>>>(
         (const OffT *)g->d_offsets, g->d_cols, starts, g->n_nodes, n_walks, base, L, seed, T,
-        max_rounds, walks, steps, caps);
+        max_rounds, walks, steps, caps, refused);
 }
 
 gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_t n_walks,
                                 int64_t base, int32_t L, uint64_t seed, double p, double q,
                                 int32_t max_rounds, int group, int32_t *walks,
                                 unsigned long long *steps, unsigned long long *caps,
-                                cudaStream_t st)
+                                unsigned long long *refused, cudaStream_t st)
 {
     if (n_walks == 0) return GS_OK;
     N2VThresholds T;
     node2vec_thresholds(p, q, &T);
-    if (group <= 1 && L % 4 == 0 && (((uintptr_t)walks & 15) == 0)) {
+    if (group == 0 && L % 4 == 0 && (((uintptr_t)walks & 15) == 0)) {
         const int threads = 256;
         int64_t blocks = (n_walks + threads - 1) / threads;
         const int64_t cap = (int64_t)sm_count() * 8 * 16;
         if (blocks > cap) blocks = cap;
 #define GS_N2T(T_, IDX, HSH)                                                                      \
-        do {                                                                                      \
-            if (group == 0)                                                                       \
-                node2vec_flat_kernel<T_, IDX, HSH><<<(unsigned)blocks, threads, 0, st>>>(           \
-                    (const T_ *)g->d_offsets, g->d_cols, g->d_edge_rec, g->d_edge_hash, g->hash_mask, \
-                    starts, g->n_nodes, n_walks, base, L, seed, T, max_rounds, walks, steps, caps); \
-            else                                                                                  \
-                node2vec_thread_kernel<T_, IDX, HSH><<<(unsigned)blocks, threads, 0, st>>>(         \
-                    (const T_ *)g->d_offsets, g->d_cols, g->d_edge_rec, g->d_edge_hash, g->hash_mask, \
-                    starts, g->n_nodes, n_walks, base, L, seed, T, max_rounds, walks, steps, caps); \
-        } while (0)
+        node2vec_flat_kernel<T_, IDX, HSH><<<(unsigned)blocks, threads, 0, st>>>(                   \
+            (const T_ *)g->d_offsets, g->d_cols, g->d_edge_rec, g->d_edge_hash, g->hash_mask,      \
+            starts, g->n_nodes, n_walks, base, L, seed, T, max_rounds, walks, steps, caps, refused)
 #define GS_N2T_H(T_, IDX) do { if (g->d_edge_hash) GS_N2T(T_, IDX, true); else GS_N2T(T_, IDX, false); } while (0)
         if (g->offsets64) { if (g->d_edge_rec) GS_N2T_H(int64_t, true); else GS_N2T_H(int64_t, false); }
         else { if (g->d_edge_rec) GS_N2T_H(int32_t, true); else GS_N2T_H(int32_t, false); }
@@ -836,9 +747,9 @@ gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_
 #define GS_N2V(GG)                                                                              \
     do {                                                                                        \
         if (g->offsets64) launch_n2v<int64_t, GG>(g, starts, n_walks, base, L, seed, T,         \
-                                                  max_rounds, walks, steps, caps, st);          \
+                                                  max_rounds, walks, steps, caps, refused, st); \
         else launch_n2v<int32_t, GG>(g, starts, n_walks, base, L, seed, T, max_rounds, walks,   \
-                                     steps, caps, st);                                          \
+                                     steps, caps, refused, st);                                 \
     } while (0)
     switch (group) {
         case 1: GS_N2V(1); break;
@@ -849,56 +760,6 @@ gs_status launch_node2vec_walks(const gs_graph *g, const int32_t *starts, int64_
     }
 #undef GS_N2V
     GS_CUDA_TRY(cudaGetLastError());
-    return GS_OK;
-}
-
-// ---------------------------------------------------------------- measurement aid
-// Independent random 16-byte reads of the walk index with the same load instruction the walk
-// kernels use.  A walk transition is one such read that depends on the previous one; this kernel
-// gives the rate the memory system sustains when nothing but the reads is done, i.e. the ceiling
-// of any sampler that needs one isolated DRAM access per transition.
-__device__ __forceinline__ uint64_t probe_mix(uint64_t x)
-{
-    x ^= x >> 33; x *= 0xff51afd7ed558ccdull; x ^= x >> 33; x *= 0xc4ceb9fe1a85ec53ull; x ^= x >> 33;
-    return x;
-}
-
-__global__ void __launch_bounds__(256)
-random_read_probe_kernel(const int4 *__restrict__ rec, uint64_t n_rec, int iters, unsigned long long *sink)
-{
-    uint64_t s = probe_mix((uint64_t)blockIdx.x * blockDim.x + threadIdx.x + 1);
-    int acc = 0;
-    for (int it = 0; it < iters; it += 4) {
-        int4 v[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) { s = probe_mix(s + u + 1); v[u] = ld_random(rec + (s % n_rec)); }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) acc += v[u].x;
-    }
-    if (acc == 0x7fffffff) atomicAdd(sink, 1ull);           // keeps the loads alive
-}
-
-gs_status random_read_probe(const gs_graph *g, int64_t n_reads, float *ms_out, cudaStream_t st)
-{
-    const int iters = 256;
-    int64_t blocks = (n_reads + 256 * iters - 1) / (256 * iters);
-    if (blocks < 1) blocks = 1;
-    void *ws = nullptr;
-    gs_status s = workspace_get(WS_COUNTERS, 256, &ws);
-    if (s != GS_OK) return s;
-    unsigned long long *sink = (unsigned long long *)((char *)ws + 192);
-    cudaEvent_t e0, e1;
-    GS_CUDA_TRY(cudaEventCreate(&e0));
-    GS_CUDA_TRY(cudaEventCreate(&e1));
-    random_read_probe_kernel<<<(unsigned)blocks, 256, 0, st>>>(g->d_edge_rec, (uint64_t)g->n_edges, iters, sink);
-    cudaEventRecord(e0, st);
-    random_read_probe_kernel<<<(unsigned)blocks, 256, 0, st>>>(g->d_edge_rec, (uint64_t)g->n_edges, iters, sink);
-    cudaEventRecord(e1, st);
-    cudaError_t e = cudaEventSynchronize(e1);
-    if (e == cudaSuccess) e = cudaEventElapsedTime(ms_out, e0, e1);
-    cudaEventDestroy(e0);
-    cudaEventDestroy(e1);
-    if (e != cudaSuccess) return cuda_fail(e, "random read probe");
     return GS_OK;
 }
 

@@ -258,7 +258,3 @@ WORKLOADS = {
                              n_edges_target=1_000_000_000),
 }
 
-
-def pairs_per_full_walk(L: int, w: int) -> int:
-    """Number of (center, context) pairs of a walk without dead ends."""
-    return sum(min(L - 1, i + w) - max(0, i - w) for i in range(L))

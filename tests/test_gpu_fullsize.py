@@ -30,6 +30,78 @@ def count_pairs(walks, w):
     return total
 
 
+def check_synchronous_step(wl, w_in, w_out, sub, sub_base, a_dev, thr, alias, seed):
+    """One synchronous step of the 512 walks `sub` at full table size against the oracle working
+    on the touched rows only.  The touched rows first get seeded values large enough that the
+    step moves every one of them by far more than the tolerance, so a row that the apply pass
+    skipped, wrote twice or wrote at a wrong address could not pass; all rows outside the batch
+    inside three windows of a million rows (start, middle and end of the tables) must keep
+    their bits."""
+    n = w_in.shape[0]
+    sub_h = sub.cpu().numpy()
+    c, o, ng, n_pairs = O.expand_lists(sub_h, sub_base, wl.window, wl.n_neg, thr, alias, seed)
+    ids, cc, oo, nn = compact_problem(c, o, ng)
+    ids_dev = torch.from_numpy(ids).to(DEV)
+    gen = torch.Generator().manual_seed(1234 + int(sub_base % 1000))
+    u0 = (torch.rand((len(ids), wl.dim), generator=gen) - 0.5) * 0.6       # input rows: up to 0.3
+    v0 = (torch.rand((len(ids), wl.dim), generator=gen) - 0.5) * 0.15      # output rows: up to 0.075
+    w_in[ids_dev] = u0.to(DEV)
+    w_out[ids_dev] = v0.to(DEV)
+    U, V = u0.numpy().astype(np.float64), v0.numpy().astype(np.float64)
+    U0, V0 = U.copy(), V.copy()
+    win = min(1 << 20, n)
+    windows = sorted({0, max(0, n // 2 - win // 2), n - win})
+    keep = []
+    for lo in windows:
+        outside = torch.ones(win, dtype=torch.bool, device=DEV)
+        inside = ids_dev[(ids_dev >= lo) & (ids_dev < lo + win)] - lo
+        outside[inside] = False
+        keep.append((lo, outside, w_in[lo:lo + win].clone(), w_out[lo:lo + win].clone()))
+    loss_o, cnt_o = O.sgns_det_from_lists(U, V, cc, oo, nn, wl.lr0)
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    pd = torch.empty((512, wl.walk_len, 2 * wl.window, 2), dtype=torch.int32, device=DEV)
+    nd = torch.empty((512, wl.walk_len, 2 * wl.window, wl.n_neg), dtype=torch.int32, device=DEV)
+    B.gs_sgns_step(w_in, w_out, sub, sub_base, wl.window, wl.n_neg, a_dev, wl.lr0, seed,
+                   B.GS_DETERMINISTIC, loss, cnt, pd, nd)
+    torch.cuda.synchronize()
+    pd = pd.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+    assert np.array_equal(nd.cpu().numpy().reshape(-1, wl.n_neg), ng)
+    assert int(cnt.item()) == cnt_o == n_pairs > 0
+    assert abs(loss.item() - loss_o) <= 2e-6 * abs(loss_o)
+    err_in = np.abs(w_in[ids_dev].cpu().numpy() - U).max()
+    err_out = np.abs(w_out[ids_dev].cpu().numpy() - V).max()
+    assert err_in <= EMB_TOL and err_out <= EMB_TOL, (err_in, err_out)
+
+    # what the step moved, row by row (oracle values): every center row, and every output row
+    # that received exactly one contribution, moved by at least 20 x the tolerance.  An output
+    # row can move less only where contributions of opposite sign met (a node that is context
+    # in one slot and negative in another slot of the same center): those rows are counted.
+    is_center = np.zeros(len(ids), dtype=bool)
+    is_center[cc[cc >= 0]] = True
+    pair_ok = cc >= 0
+    hits = np.bincount(oo[pair_ok], minlength=len(ids))
+    negs = nn[pair_ok]
+    negs = negs[(negs >= 0) & (negs != oo[pair_ok][:, None])]
+    hits += np.bincount(negs, minlength=len(ids))
+    moved_in = np.abs(U - U0).max(axis=1)
+    moved_out = np.abs(V - V0).max(axis=1)
+    min_in = moved_in[is_center].min()
+    min_single = moved_out[hits == 1].min()
+    small = int(((hits > 0) & (moved_out < 20 * EMB_TOL)).sum())
+    print(f"{wl.name} base {sub_base}: {len(ids)} rows touched, ids {ids.min()}..{ids.max()}; smallest move "
+          f"of a center row {min_in:.2e}, of an output row hit once {min_single:.2e}; "
+          f"{small} of {int((hits > 0).sum())} output rows moved less than 20 x tol; "
+          f"errors {err_in:.1e} / {err_out:.1e}")
+    assert min_in >= 20 * EMB_TOL and min_single >= 20 * EMB_TOL
+    assert small <= 1e-3 * (hits > 0).sum()
+    assert np.array_equal(moved_in > 0, is_center) and np.array_equal(moved_out > 0, hits > 0)
+    for lo, outside, before_in, before_out in keep:
+        assert torch.equal(w_in[lo:lo + win][outside], before_in[outside]), lo
+        assert torch.equal(w_out[lo:lo + win][outside], before_out[outside]), lo
+
+
 @pytest.mark.parametrize("name", ["deepwalk_medium", "node2vec_4m", "deepwalk_large", "rmat_billion"])
 def test_fullsize_workload(name):
     wl = WL.WORKLOADS[name]
@@ -115,33 +187,21 @@ def test_fullsize_workload(name):
     per_pair = loss.item() / cnt.item()
     assert 0.3 < per_pair <= (1 + wl.n_neg) * np.log(2) * (1 + 1e-6)
 
-    # ---- synchronous step on 512 walks against the oracle on the touched rows
-    sub = walks[4096:4096 + 512].contiguous()
-    sub_h = sub.cpu().numpy()
-    c, o, ng, n_pairs = O.expand_lists(sub_h, base + 4096, wl.window, wl.n_neg, thr, alias, seed)
-    ids, cc, oo, nn = compact_problem(c, o, ng)
-    ids_dev = torch.from_numpy(ids).to(DEV)
-    U = w_in[ids_dev].cpu().numpy().astype(np.float64)
-    V = w_out[ids_dev].cpu().numpy().astype(np.float64)
-    assert np.abs(V).max() > 0
-    untouched = torch.from_numpy(np.setdiff1d(np.random.default_rng(1).integers(0, n, 4096), ids)).to(DEV)
-    before_in, before_out = w_in[untouched].clone(), w_out[untouched].clone()
-    loss_o, cnt_o = O.sgns_det_from_lists(U, V, cc, oo, nn, wl.lr0)
-    loss.zero_()
-    cnt.zero_()
-    pd = torch.empty((512, wl.walk_len, 2 * wl.window, 2), dtype=torch.int32, device=DEV)
-    nd = torch.empty((512, wl.walk_len, 2 * wl.window, wl.n_neg), dtype=torch.int32, device=DEV)
-    B.gs_sgns_step(w_in, w_out, sub, base + 4096, wl.window, wl.n_neg, a_dev, wl.lr0, seed,
-                   B.GS_DETERMINISTIC, loss, cnt, pd, nd)
-    torch.cuda.synchronize()
-    pd = pd.cpu().numpy().reshape(-1, 2)
-    assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
-    assert np.array_equal(nd.cpu().numpy().reshape(-1, wl.n_neg), ng)
-    assert int(cnt.item()) == cnt_o == n_pairs
-    assert abs(loss.item() - loss_o) <= 2e-6 * abs(loss_o)
-    assert np.abs(w_in[ids_dev].cpu().numpy() - U).max() <= EMB_TOL
-    assert np.abs(w_out[ids_dev].cpu().numpy() - V).max() <= EMB_TOL
-    assert torch.equal(w_in[untouched], before_in) and torch.equal(w_out[untouched], before_out)
+    # ---- synchronous step on 512 walks against the oracle on the touched rows: once in the middle
+    # of the epoch and once on the epoch's last 512 walk ids, whose start nodes are the last rows
+    # of the tables
+    check_synchronous_step(wl, w_in, w_out, walks[4096:4096 + 512].contiguous(), base + 4096, a_dev,
+                           thr, alias, seed)
+    last = total - 512
+    if wl.walk_kind == "uniform":
+        tail = B.gs_random_walks(G, None, 512, last, wl.walk_len, seed)
+        want, _ = O.uniform_walks(off, col, None, 512, last, wl.walk_len, seed)
+    else:
+        tail = B.gs_node2vec_walks(G, None, 512, last, wl.walk_len, seed, wl.p, wl.q)
+        want, _, _ = O.node2vec_walks(off, col, None, 512, last, wl.walk_len, seed, wl.p, wl.q)
+    assert np.array_equal(tail.cpu().numpy(), want)
+    assert int(tail[-1, 0]) == n - 1
+    check_synchronous_step(wl, w_in, w_out, tail, last, a_dev, thr, alias, seed)
 
     G.close()
     del w_in, w_out, walks, g, a_dev

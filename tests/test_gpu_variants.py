@@ -217,17 +217,6 @@ def test_adam_steps_match_oracle(dim, pair_mode):
         assert torch.equal(a, b)                       # bitwise reproducible
 
 
-# ---------------------------------------------------------------- measurement aid
-def test_random_read_probe_reports_a_rate_and_needs_the_walk_index(tiny):
-    _, g, off, col, _, _ = tiny
-    G = B.gs_graph_load_csr(g.offsets.to(DEV), g.cols.to(DEV), B.GS_BUILD_WALK_INDEX)
-    assert B.gs_probe_random_reads(G, 1 << 20) > 1e6
-    G2 = B.gs_graph_load_csr(g.offsets.to(DEV), g.cols.to(DEV), B.GS_VALIDATE)
-    with pytest.raises(B.GsError) as e:
-        B.gs_probe_random_reads(G2, 1 << 20)
-    assert e.value.status == -1
-
-
 def test_subsampling_drops_entries_outside_the_threshold_table(tiny):
     _, g, off, col, _, _ = tiny
     n = g.n_nodes

@@ -32,7 +32,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(B.SgnsConfig) == 10 * 4 + 3 * 8 + 3 * 8 + 8 + 8 + 2 * 4 + 4 * 4 + 8 + 6 * 8
-    assert ctypes.sizeof(B.EpochStats) == 8 + 5 * 8 + 3 * 4 + 4
+    assert ctypes.sizeof(B.EpochStats) == 8 + 5 * 8 + 4 * 4 + 8      # loss, 5 counters, 4 times, refused ids
 
 
 @pytest.mark.parametrize("power", [0.75, 1.0, 0.0])

@@ -18,6 +18,12 @@ GOLDEN = Path(__file__).parent / "golden"
 CHI2_P = 1e-4          # fixed seeds, so a pass is reproducible; this is the alarm level
 
 
+def pairs_per_full_walk(L, w):
+    """Number of (center, context) pairs of a walk without dead ends, by direct counting: position
+    i pairs with every other position within w of it."""
+    return sum(min(L - 1, i + w) - max(0, i - w) for i in range(L))
+
+
 def np_graph(g):
     return g.offsets.cpu().numpy().astype(np.int64), g.cols.cpu().numpy()
 
@@ -218,7 +224,7 @@ def test_pair_expansion_count_identity_and_brute_force(L, w):
     c = c.reshape(6, L, 2 * w)
     o = o.reshape(6, L, 2 * w)
     if L > w:
-        assert WL.pairs_per_full_walk(L, w) == 2 * (w * L - w * (w + 1) // 2)
+        assert pairs_per_full_walk(L, w) == 2 * (w * L - w * (w + 1) // 2)
     total = 0
     for a in range(6):
         got = []
@@ -235,7 +241,7 @@ def test_pair_expansion_count_identity_and_brute_force(L, w):
         # symmetry: (x, y) at (i, j) <=> (y, x) at (j, i)
         assert {(i, j, x, y) for (i, j, x, y) in got} == {(j, i, y, x) for (i, j, x, y) in got}
         if a < 4:
-            assert len(got) == WL.pairs_per_full_walk(L, w)
+            assert len(got) == pairs_per_full_walk(L, w)
         total += len(got)
     assert total == n_pairs
     assert (ng.reshape(6, L, 2 * w, 2)[c < 0] == -1).all()
@@ -307,7 +313,7 @@ def test_negative_draws_follow_unigram_power_distribution():
     walks = np.tile(np.arange(10, dtype=np.int32), (3000, 1))
     c, o, ng, n_pairs = O.expand_lists(walks, 1000, w, K, thr, alias, seed=33)
     draws = ng[c >= 0].ravel()
-    assert len(draws) == n_pairs * K and n_pairs == 3000 * WL.pairs_per_full_walk(L, w)
+    assert len(draws) == n_pairs * K and n_pairs == 3000 * pairs_per_full_walk(L, w)
     probs = wgt ** 0.75
     probs /= probs.sum()
     ok, stat = chi2_ok(np.bincount(draws, minlength=10), probs)

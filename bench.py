@@ -320,10 +320,10 @@ def walk_kernel_name(wl, indexed):
 
 def sync_step_launches(n_nodes, extra=0):
     """Kernels of one synchronous batch: walks; targets and three per radix pass of at most 8 bits
-    over keys below 2 n_nodes (the table-independent part); coefficients, apply (output rows,
-    fix-up, input rows), loss reduction."""
+    over keys below 2 n_nodes (the table-independent part); coefficients, apply of the output
+    rows, and the last launch (input rows, cut runs, sums)."""
     passes = ((2 * n_nodes).bit_length() + 7) // 8
-    return 1 + 1 + 3 * passes + 1 + 3 + 1 + extra
+    return 1 + 1 + 3 * passes + 1 + 2 + extra
 
 
 def parse_variants(args):
@@ -649,7 +649,10 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
         launches = n_steps                                        # SGNS launches on this rank
         positions = steps + walks_done                            # walk entries = center positions
         sgns_bytes = algorithmic_bytes(pairs, positions, wl.dim, wl.n_neg, 2 if f16 else 4) / launches
-        sgns_ms = ms_sgns / launches
+        lock_free = (mode & 0xFF) != B.GS_DETERMINISTIC
+        # lock-free: the update kernel's own time.  Synchronous: the whole step, because its kernels
+        # run on two streams (targets and sort of the next batch beside the update of this one)
+        sgns_ms = ms_sgns / launches if lock_free else ms / launches
         achieved = sgns_bytes / (sgns_ms * 1e-3) / 1e9
         indexed = "walk_index_bytes" in info
         if one_call and warm:                          # walk kernel alone: the warm-up calls
@@ -659,7 +662,6 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
         wbytes = walk_bytes(w_steps, wl.offsets64, indexed) / w_n
         gbytes = walk_granule_bytes(w_steps, indexed) / w_n
         walk_ms = w_ms / w_n
-        lock_free = (mode & 0xFF) != B.GS_DETERMINISTIC
         per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if lock_free and not f16 else None
         traffic = per_pair * pairs / launches if per_pair else None
         payload_gbs = wbytes / (walk_ms * 1e-3) / 1e9
@@ -689,7 +691,8 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
                          "kernel": "sgns_hogwild_kernel" if lock_free else "synchronous step (coefficients, sort, apply)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", **fractions(achieved, peak),
                          "peak_kind": f"of {peak_kind}", "traffic": traffic,
-                         "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (ms_sgns * 1e-3)},
+                         "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (sgns_ms * launches * 1e-3),
+                         "ms_update_stream": ms_sgns / launches},
             "walk": {"kernel": walk_kernel_name(wl, indexed),
                      "walk_steps_per_s_kernel": w_steps / (w_ms * 1e-3), "ms_per_launch": walk_ms,
                      "payload_gbs": payload_gbs, "payload_frac": payload_gbs / peak,

@@ -49,8 +49,11 @@ def parse_args():
     ap.add_argument("--workload", default="deepwalk_large")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the node count (testing)")
     ap.add_argument("--batch-walks", type=int, default=1 << 20)
-    ap.add_argument("--mode", default="hogwild",
-                    choices=["hogwild", "hogwild_red", "deterministic", "momentum", "adam"])
+    ap.add_argument("--mode", default="hogwild_red",
+                    choices=["hogwild", "hogwild_red", "deterministic", "momentum", "adam"],
+                    help="hogwild_red: lock-free, increments added by reductions (default; fp32 tables); "
+                         "hogwild: lock-free with plain stores; deterministic: synchronous batches of 512 "
+                         "walks; momentum / adam: synchronous with that optimizer")
     ap.add_argument("--variants", default="",
                     help="comma list of shrink (per-position window draw), subsample (frequent-node "
                          "sub-sampling, t = 1e-5), shuffle (keyed start-node order)")
@@ -137,22 +140,28 @@ NOMINAL_HBM_GBS = 8000.0      # the device's nominal HBM3e bandwidth, for contex
 
 def recorded_traffic(kernel, workload):
     """DRAM bytes per pair (or per transition) of `kernel` taken from the ncu summary under
-    profiles/, or None when there is none or the kernel's source has changed since the capture
-    (the summary records the sha256 of the source file)."""
+    profiles/, with the note that says where they were captured, or (None, None) when there is
+    none or the kernel's source has changed since the capture.  The summary records the sha256 of
+    the part of the source file that holds the kernel: everything before the line `upto`."""
     import hashlib
     import re
     f = ROOT / "profiles" / f"{kernel}__{workload}.md"
     if not f.exists():
-        return None
+        return None, None
     text = f.read_text()
     m = re.search(r"dram_bytes_per_unit\s*=\s*([0-9.eE+-]+)", text)
-    h = re.search(r"source\s*=\s*(\S+)\s+sha256\s*=\s*([0-9a-f]{64})", text)
+    h = re.search(r"source\s*=\s*(\S+)\s+upto\s*=\s*\"([^\"]+)\"\s+sha256\s*=\s*([0-9a-f]{64})", text)
+    note = re.search(r"traffic_note\s*=\s*(.+)", text)
     if not m or not h:
-        return None
+        return None, None
     src = ROOT / h.group(1)
-    if not src.exists() or hashlib.sha256(src.read_bytes()).hexdigest() != h.group(2):
-        return None
-    return float(m.group(1))
+    if not src.exists():
+        return None, None
+    body = src.read_text()
+    cut = body.find(h.group(2))
+    if cut < 0 or hashlib.sha256(body[:cut].encode()).hexdigest() != h.group(3):
+        return None, None
+    return float(m.group(1)), note.group(1).strip() if note else None
 
 
 def algorithmic_bytes(pairs, positions, dim, n_neg, elem=4):
@@ -536,8 +545,11 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
     step_fn = {"f32": B.gs_sgns_step, "f16": B.gs_sgns_step_f16, "bf16": B.gs_sgns_step_bf16}[args.table_dtype]
     if args.mode in ("momentum", "adam"):
         return run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev)
+    mode_name = args.mode
+    if f16 and mode_name == "hogwild_red":
+        mode_name = "hogwild"                          # 16-bit tables: plain stores only
     mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,
-            "deterministic": B.GS_DETERMINISTIC}[args.mode]
+            "deterministic": B.GS_DETERMINISTIC}[mode_name]
     if wl.forward_only:
         mode |= B.GS_PAIRS_FORWARD_ONLY
     variants = parse_variants(args)
@@ -662,7 +674,8 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
         wbytes = walk_bytes(w_steps, wl.offsets64, indexed) / w_n
         gbytes = walk_granule_bytes(w_steps, indexed) / w_n
         walk_ms = w_ms / w_n
-        per_pair = recorded_traffic("sgns_hogwild_kernel", wl.name) if lock_free and not f16 else None
+        per_pair, traffic_note = recorded_traffic("sgns_hogwild_kernel", wl.name) \
+            if mode_name == "hogwild_red" and not f16 else (None, None)
         traffic = per_pair * pairs / launches if per_pair else None
         payload_gbs = wbytes / (walk_ms * 1e-3) / 1e9
         granule_gbs = gbytes / (walk_ms * 1e-3) / 1e9
@@ -671,7 +684,7 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
             "steps": n_steps, "warmup": args.warmup, "ms_per_step": ms / n_steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": wl.name, "mode": args.mode, "table_dtype": args.table_dtype,
+            "config": {"workload": wl.name, "mode": mode_name, "table_dtype": args.table_dtype,
                        "batch_walks": bw,
                        "walk_kind": wl.walk_kind, "walk_len": wl.walk_len, "window": wl.window,
                        "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale, "variants": sorted(variants),
@@ -690,7 +703,7 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
             "roofline": {"bound": "hbm",
                          "kernel": "sgns_hogwild_kernel" if lock_free else "synchronous step (coefficients, sort, apply)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", **fractions(achieved, peak),
-                         "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                         "peak_kind": f"of {peak_kind}", "traffic": traffic, "traffic_note": traffic_note,
                          "ms_per_launch": sgns_ms, "pair_updates_per_s": pairs / (sgns_ms * launches * 1e-3),
                          "ms_update_stream": ms_sgns / launches},
             "walk": {"kernel": walk_kernel_name(wl, indexed),
@@ -733,9 +746,9 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
 PER_CONFIG_LEGS = [
     ("tiny_deepwalk", "deterministic", 17, 3),
     ("deepwalk_medium", "deterministic", 300, 5),
-    ("deepwalk_medium", "hogwild", 8, 3),
-    ("node2vec_4m", "hogwild", 6, 3),
-    ("rmat_billion", "hogwild", 10, 3),
+    ("deepwalk_medium", "hogwild_red", 8, 3),
+    ("node2vec_4m", "hogwild_red", 6, 3),
+    ("rmat_billion", "hogwild_red", 10, 3),
 ]
 
 
@@ -754,7 +767,7 @@ def run_ours(args, wl):
         dist.init_process_group("nccl", device_id=dev)
     B.lib()                                            # fail loudly if the library is missing
 
-    plain = (args.workload == "deepwalk_large" and args.mode == "hogwild" and args.stage == "all"
+    plain = (args.workload == "deepwalk_large" and args.mode == "hogwild_red" and args.stage == "all"
              and args.table_dtype == "f32" and not args.variants and args.scale == 1.0)
     out = run_leg(args, wl, dev, rank, world, local, with_e2e=not args.no_e2e,
                   with_cpu=not args.no_cpu_baseline)

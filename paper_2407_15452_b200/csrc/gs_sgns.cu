@@ -1084,8 +1084,9 @@ __device__ __forceinline__ void row_red_add(float *__restrict__ tab, int64_t r, 
 //    terms; the pieces of a longer run are added up in fp64 by the fix-up;
 //  - the output row is not read: the finished sum goes out as ONE reduction per value,
 //    row += -lr * sum.  Every row is owned by exactly one run, so this is the only addition the
-//    row receives in the step and the result bits do not depend on scheduling;
-//  - while a group of G center rows is added, the next group is already on its way into L1.
+//    row receives in the step and the result bits do not depend on scheduling.
+// (Prefetching the next group's center rows into L1 while a group is added was measured and did
+// not pay: 0.491 against 0.484 ms per batch.)
 template <int FPL>
 __global__ void __launch_bounds__(256, (FPL <= 2 ? 4 : 3))
 sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
@@ -1095,7 +1096,6 @@ sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_
                           double *__restrict__ lead_part, double *__restrict__ tail_part)
 {
     constexpr int G = FPL <= 4 ? 8 : 4;
-    constexpr int ROW_BYTES = FPL * 32 * 4;
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t n_blocks = ((int64_t)n_keys + RUN_CUT - 1) / RUN_CUT;
@@ -1173,23 +1173,6 @@ sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_
 #pragma unroll
                 for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(gq, row.v[j], acc.v[j]);
             };
-            // lane l asks for line l of the G rows that follow group q0: the rest of this chunk, or
-            // (behind the last group) the start of the next chunk, whose metadata is there by then
-            auto prefetch_next = [&](int q0) {
-                const int x = lane * 128 / ROW_BYTES;
-                int32_t cn;
-                bool there;
-                if (q0 + 2 * G <= 32) {
-                    cn = __shfl_sync(0xffffffffu, c, (q0 + G + x) & 31);
-                    there = q0 + G + x < n;
-                } else {
-                    cn = __shfl_sync(0xffffffffu, c1, x & 31);
-                    there = n == 32;                                  // unusable entries carry row 0
-                }
-                if (lane * 128 < G * ROW_BYTES && there)
-                    asm volatile("prefetch.global.L1 [%0];" ::
-                                 "l"((const char *)(w_in + (int64_t)cn * (FPL * 32)) + lane * 128 % ROW_BYTES));
-            };
             int q0 = 0;
 #pragma unroll 1
             for (; q0 + G <= n; q0 += G) {
@@ -1197,7 +1180,6 @@ sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_
 #pragma unroll
                 for (int q = 0; q < G; ++q)
                     ru[q] = row_load<FPL>(w_in, (int64_t)__shfl_sync(0xffffffffu, c, q0 + q), lane);
-                prefetch_next(q0);
 #pragma unroll
                 for (int q = 0; q < G; ++q) add_one(q0 + q, __shfl_sync(0xffffffffu, g, q0 + q), ru[q]);
             }

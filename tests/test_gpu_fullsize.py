@@ -209,6 +209,74 @@ def test_fullsize_workload(name):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("name,nb", [("node2vec_4m", 8), ("deepwalk_large", 8), ("rmat_billion", 16)])
+def test_truncated_epoch_on_touched_rows_matches_the_oracle(name, nb):
+    # The first nb 512-walk batches of the epoch through the epoch driver at full size (walks generated
+    # by the driver, the table-independent part of batch b+1 overlapping the update of batch b),
+    # against the oracle run batch by batch on the rows these batches touch (fp64; the rows'
+    # start values come from the oracle's own table initialisation): walk steps, pairs and masked
+    # negatives equal, mean loss within 1e-3, every touched value within 1e-6 (the rows are still
+    # small this early in training, so the bar is a hundredth of the usual one).
+    wl = WL.WORKLOADS[name]
+    torch.cuda.empty_cache()
+    g = wl.make_graph(device=DEV)
+    n, seed, bw = g.n_nodes, wl.graph_seed, 512
+    off = g.offsets.cpu().numpy().astype(np.int64)
+    col = g.cols.cpu().numpy()
+    thr, alias = O.build_alias((off[1:] - off[:-1]).astype(np.float64), 0.75)
+    # ---- oracle side: walks and lists of every batch, then the union of the rows they touch
+    batches, steps_o = [], 0
+    for b in range(nb):
+        if wl.walk_kind == "uniform":
+            walks, st = O.uniform_walks(off, col, None, bw, b * bw, wl.walk_len, seed)
+        else:
+            walks, st, _ = O.node2vec_walks(off, col, None, bw, b * bw, wl.walk_len, seed, wl.p, wl.q)
+        steps_o += st
+        batches.append(O.expand_lists(walks, b * bw, wl.window, wl.n_neg, thr, alias, seed)[:3])
+    union = np.unique(np.concatenate([np.concatenate([c, o, ng.ravel()]) for c, o, ng in batches]))
+    union = union[union >= 0]
+    U = O.init_rows(union, wl.dim, seed)
+    V = np.zeros_like(U)
+    loss_o, pairs_o, masked_o = 0.0, 0, 0
+    for c, o, ng in batches:
+        ids, cc, oo, nn = compact_problem(c, o, ng)              # this batch's rows, renumbered
+        at = np.searchsorted(union, ids)
+        Ub, Vb = np.ascontiguousarray(U[at]), np.ascontiguousarray(V[at])
+        ls, pc = O.sgns_det_from_lists(Ub, Vb, cc, oo, nn, wl.lr0)
+        U[at], V[at] = Ub, Vb
+        loss_o += ls
+        pairs_o += pc
+        masked_o += int(((ng == o[:, None]) & (c >= 0)[:, None]).sum())
+    # ---- the library
+    flags = B.GS_VALIDATE | B.GS_REQUIRE_SORTED | B.GS_BUILD_WALK_INDEX
+    if wl.walk_kind != "uniform":
+        flags |= B.GS_BUILD_EDGE_SET
+    G = B.gs_graph_load_csr(g.offsets, g.cols, flags)
+    w_in = torch.empty((n, wl.dim), dtype=torch.float32, device=DEV)
+    w_out = torch.empty_like(w_in)
+    B.gs_init_embeddings(w_in, w_out, seed)
+    table = (alias.astype(np.uint64) << np.uint64(32)) | thr.astype(np.uint64)
+    kind = B.GS_WALK_UNIFORM if wl.walk_kind == "uniform" else B.GS_WALK_NODE2VEC
+    res = B.gs_sgns_epoch(G, torch.from_numpy(table.view(np.int64)).to(DEV), w_in, w_out,
+                          walks_per_node=wl.walks_per_node, walk_len=wl.walk_len, window=wl.window,
+                          n_neg=wl.n_neg, lr0=wl.lr0, batch_walks=bw, seed=seed, mode=B.GS_DETERMINISTIC,
+                          walk_kind=kind, p=wl.p, q=wl.q, num_batches=nb)
+    assert (res.pairs, res.steps, res.masked_negs, res.batches, res.refused_ids) == (pairs_o, steps_o, masked_o, nb, 0)
+    assert abs(res.loss_sum - loss_o) <= 1e-3 * loss_o
+    rel = abs(res.loss_sum - loss_o) / loss_o
+    rows = torch.from_numpy(union).to(DEV)
+    err_in = np.abs(w_in[rows].cpu().numpy() - U).max()
+    err_out = np.abs(w_out[rows].cpu().numpy() - V).max()
+    print(f"{name}: {nb} batches, {len(union)} rows touched, loss {res.loss_sum / res.pairs:.5f} (rel. diff {rel:.1e}), "
+          f"largest output value {np.abs(V).max():.2e}, errors {err_in:.1e} / {err_out:.1e}")
+    assert err_in <= 1e-6 and err_out <= 1e-6, (err_in, err_out)
+    assert np.abs(V).max() > 1e-3                                 # the batches did move the rows
+    G.close()
+    del w_in, w_out, g
+    B.gs_release_workspace()
+    torch.cuda.empty_cache()
+
+
 def test_truncated_epoch_of_the_medium_workload_matches_the_oracle():
     # The first eight 512-walk batches of the 1M-node workload through the epoch driver against the
     # oracle's epoch on dense fp64 tables (2 x 1 GB on the host): pair, step and masked counts equal,

@@ -387,15 +387,31 @@ def test_lock_free_single_walk_equals_sequential_oracle(dim):
     w_in0, w_out0 = random_tables(n, dim, 5)
     U, V = w_in0.numpy().astype(np.float64), w_out0.numpy().astype(np.float64)
     loss_o, cnt_o = O.sgns_seq_from_lists(U, V, c, o, ng, 2 * w, 0.05)
+    # rows that occur more than once among the targets of ONE position (a negative drawn twice, or
+    # equal to another slot's context): the kernel loads a chunk of targets before it stores any, so
+    # such a row - and the center row of that position - may differ from strictly sequential SGD
+    S = 2 * w
+    repeated, their_centers = set(), set()
+    for p0 in range(0, len(c), S):
+        targets = []
+        for e in range(p0, p0 + S):
+            if c[e] >= 0:
+                targets.append(int(o[e]))
+                targets += [int(t) for t in ng[e] if t >= 0 and t != o[e]]
+        dup = {t for t in targets if targets.count(t) > 1}
+        if dup:
+            repeated |= dup
+            their_centers.add(int(c[p0:p0 + S].max()))
     for mode in (B.GS_HOGWILD, B.GS_HOGWILD_RED):
         w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
         loss, cnt, _, _ = run_step(w_in, w_out, torch.from_numpy(walk).to(DEV), 0, w, K,
                                    alias_to_device(thr, alias), 0.05, 12, mode, dump=False)
         assert cnt == cnt_o and abs(loss - loss_o) < 1e-5 * abs(loss_o)
-        # negatives may repeat across the chunk of one position; allow those few rows to differ
         diff_in = np.abs(w_in.cpu().numpy() - U).max(axis=1)
         diff_out = np.abs(w_out.cpu().numpy() - V).max(axis=1)
-        assert (diff_in > 1e-5).sum() <= 2 and (diff_out > 1e-5).sum() <= 4
+        assert set(np.nonzero(diff_out > 1e-5)[0].tolist()) <= repeated, (repeated, np.nonzero(diff_out > 1e-5))
+        assert set(np.nonzero(diff_in > 1e-5)[0].tolist()) <= their_centers
+        assert len(repeated) <= 4                      # the case stays almost free of repeats
         assert np.abs(V - w_out0.numpy()).max() > 1e-3
 
 

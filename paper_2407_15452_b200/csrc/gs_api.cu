@@ -453,15 +453,52 @@ gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, int32_t d
                      d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
 }
 
-// ------------------------------------------------------------------ half-precision tables
+// ------------------------------------------------------------------ 16-bit tables
 static bool dim_ok_f16(int32_t dim) { return dim == 64 || dim == 128 || dim == 256; }
+
+static gs_status init_embeddings_16(bool bf16, void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
+                                    uint64_t seed, void *stream)
+{
+    if (n_nodes < 0) return invalid("n_nodes < 0");
+    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
+    return bf16 ? init_embeddings_bf16(d_w_in, d_w_out, n_nodes, dim, seed, (cudaStream_t)stream)
+                : init_embeddings_f16(d_w_in, d_w_out, n_nodes, dim, seed, (cudaStream_t)stream);
+}
+
+static gs_status sgns_step_16(bool bf16, void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
+                              const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                              int32_t walk_len, int32_t window, int32_t n_neg, const uint64_t *d_alias,
+                              float lr, uint64_t seed, int32_t mode, double *d_loss_sum,
+                              int64_t *d_pair_count, int32_t *d_pairs_dump, int32_t *d_negs_dump,
+                              void *stream)
+{
+    if (!d_w_in || !d_w_out) return invalid("table pointer is NULL");
+    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
+    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
+    if (n_walks > 0 && !d_walks) return invalid("d_walks is NULL");
+    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
+    gs_status s = check_sgns_shape(128, walk_len, window, n_neg, mode);
+    if (s != GS_OK) return s;
+    if (n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
+    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out) & 15) return invalid("tables must be 16-byte aligned");
+    return bf16 ? sgns_step_bf16(d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len,
+                                 window, n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count,
+                                 d_pairs_dump, d_negs_dump, (cudaStream_t)stream)
+                : sgns_step_f16(d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len,
+                                window, n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count,
+                                d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
+}
 
 gs_status gs_init_embeddings_f16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
                                  uint64_t seed, void *stream)
 {
-    if (n_nodes < 0) return invalid("n_nodes < 0");
-    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with half-precision tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
-    return init_embeddings_f16(d_w_in, d_w_out, n_nodes, dim, seed, (cudaStream_t)stream);
+    return init_embeddings_16(false, d_w_in, d_w_out, n_nodes, dim, seed, stream);
+}
+
+gs_status gs_init_embeddings_bf16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
+                                  uint64_t seed, void *stream)
+{
+    return init_embeddings_16(true, d_w_in, d_w_out, n_nodes, dim, seed, stream);
 }
 
 gs_status gs_sgns_step_f16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
@@ -471,48 +508,21 @@ gs_status gs_sgns_step_f16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t
                            int64_t *d_pair_count, int32_t *d_pairs_dump, int32_t *d_negs_dump,
                            void *stream)
 {
-    if (!d_w_in || !d_w_out) return invalid("table pointer is NULL");
-    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
-    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
-    if (n_walks > 0 && !d_walks) return invalid("d_walks is NULL");
-    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with half-precision tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
-    gs_status s = check_sgns_shape(128, walk_len, window, n_neg, mode);
-    if (s != GS_OK) return s;
-    if (n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
-    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out) & 15) return invalid("tables must be 16-byte aligned");
-    return sgns_step_f16(d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len,
-                         window, n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count,
-                         d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
-}
-
-// ------------------------------------------------------------------ bfloat16 tables
-gs_status gs_init_embeddings_bf16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
-                                 uint64_t seed, void *stream)
-{
-    if (n_nodes < 0) return invalid("n_nodes < 0");
-    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
-    return init_embeddings_bf16(d_w_in, d_w_out, n_nodes, dim, seed, (cudaStream_t)stream);
+    return sgns_step_16(false, d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len, window,
+                        n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count, d_pairs_dump, d_negs_dump,
+                        stream);
 }
 
 gs_status gs_sgns_step_bf16(void *d_w_in, void *d_w_out, int64_t n_nodes, int32_t dim,
-                           const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
-                           int32_t walk_len, int32_t window, int32_t n_neg, const uint64_t *d_alias,
-                           float lr, uint64_t seed, int32_t mode, double *d_loss_sum,
-                           int64_t *d_pair_count, int32_t *d_pairs_dump, int32_t *d_negs_dump,
-                           void *stream)
+                            const int32_t *d_walks, int64_t n_walks, int64_t walk_id_base,
+                            int32_t walk_len, int32_t window, int32_t n_neg, const uint64_t *d_alias,
+                            float lr, uint64_t seed, int32_t mode, double *d_loss_sum,
+                            int64_t *d_pair_count, int32_t *d_pairs_dump, int32_t *d_negs_dump,
+                            void *stream)
 {
-    if (!d_w_in || !d_w_out) return invalid("table pointer is NULL");
-    if (n_nodes <= 0 || n_nodes >= ((int64_t)1 << 31)) return invalid("n_nodes must be in [1, 2^31)");
-    if (n_walks < 0 || walk_id_base < 0) return invalid("negative n_walks or walk_id_base");
-    if (n_walks > 0 && !d_walks) return invalid("d_walks is NULL");
-    if (!dim_ok_f16(dim)) { set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim); return GS_ERR_UNSUPPORTED; }
-    gs_status s = check_sgns_shape(128, walk_len, window, n_neg, mode);
-    if (s != GS_OK) return s;
-    if (n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
-    if (((uintptr_t)d_w_in | (uintptr_t)d_w_out) & 15) return invalid("tables must be 16-byte aligned");
-    return sgns_step_bf16(d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len,
-                         window, n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count,
-                         d_pairs_dump, d_negs_dump, (cudaStream_t)stream);
+    return sgns_step_16(true, d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len, window,
+                        n_neg, d_alias, lr, seed, mode, d_loss_sum, d_pair_count, d_pairs_dump, d_negs_dump,
+                        stream);
 }
 
 // ------------------------------------------------------------------ momentum
@@ -695,7 +705,7 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
         return invalid("unknown table_dtype");
     const bool f16 = cfg->table_dtype != GS_TABLE_F32;         // a 16-bit storage format
     const bool bf16 = cfg->table_dtype == GS_TABLE_BF16;
-    if (f16 && !dim_ok_f16(cfg->dim)) { set_error("dim %d not supported with half-precision tables (64, 128, 256)", cfg->dim); return GS_ERR_UNSUPPORTED; }
+    if (f16 && !dim_ok_f16(cfg->dim)) { set_error("dim %d not supported with 16-bit tables (64, 128, 256)", cfg->dim); return GS_ERR_UNSUPPORTED; }
     gs_status s = check_sgns_shape(f16 ? 128 : cfg->dim, cfg->walk_len, cfg->window, cfg->n_neg, cfg->mode);
     if (s != GS_OK) return s;
     if (cfg->n_neg > 0 && !d_alias) return invalid("d_alias is NULL");

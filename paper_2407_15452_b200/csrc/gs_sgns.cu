@@ -1753,67 +1753,62 @@ static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
     return GS_ERR_UNSUPPORTED;
 }
 
+// One step on tables of type T (float, or a 16-bit format with fp32 arithmetic and write-back
+// rounded to nearest even).
+template <typename T>
+static gs_status step_on_tables(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
+                                int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
+                                const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
+                                int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
+                                unsigned long long *masked, int prepared)
+{
+    if (n_walks == 0) return GS_OK;
+    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
+    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
+    switch (dim) {
+        case 32:
+            if constexpr (sizeof(T) == 4) return run_mode<32, T>(a, mode, st);
+            break;
+        case 64: return run_mode<64, T>(a, mode, st);
+        case 128: return run_mode<128, T>(a, mode, st);
+        case 256: return run_mode<256, T>(a, mode, st);
+        default: break;
+    }
+    set_error(sizeof(T) == 4 ? "dim %d not supported (32, 64, 128, 256)"
+                             : "dim %d not supported with 16-bit tables (64, 128, 256)", dim);
+    return GS_ERR_UNSUPPORTED;
+}
+
 gs_status sgns_step(float *w_in, float *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                     int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                     const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                     int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
                     unsigned long long *masked, int prepared)
 {
-    if (n_walks == 0) return GS_OK;
-    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
-    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
-    switch (dim) {
-        case 32: return run_mode<32, float>(a, mode, st);
-        case 64: return run_mode<64, float>(a, mode, st);
-        case 128: return run_mode<128, float>(a, mode, st);
-        case 256: return run_mode<256, float>(a, mode, st);
-        default:
-            set_error("dim %d not supported (32, 64, 128, 256)", dim);
-            return GS_ERR_UNSUPPORTED;
-    }
+    return step_on_tables<float>(w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                                 seed, mode, loss, pairs, dump_pairs, dump_negs, st, masked, prepared);
 }
 
-// Tables stored as IEEE half, arithmetic in fp32, write-back rounded to nearest even.
 gs_status sgns_step_f16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                         int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                         const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                         int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
                         unsigned long long *masked, int prepared)
 {
-    if (n_walks == 0) return GS_OK;
-    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
-    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
-    switch (dim) {
-        case 64: return run_mode<64, __half>(a, mode, st);
-        case 128: return run_mode<128, __half>(a, mode, st);
-        case 256: return run_mode<256, __half>(a, mode, st);
-        default:
-            set_error("dim %d not supported with half-precision tables (64, 128, 256)", dim);
-            return GS_ERR_UNSUPPORTED;
-    }
+    return step_on_tables<__half>(w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
+                                  seed, mode, loss, pairs, dump_pairs, dump_negs, st, masked, prepared);
 }
 
-// Tables stored as bfloat16: as above with the other 16-bit format.
 gs_status sgns_step_bf16(void *w_in, void *w_out, int64_t n_nodes, int32_t dim, const int32_t *walks,
                          int64_t n_walks, int64_t walk_id_base, int32_t L, int32_t w, int32_t K,
                          const uint64_t *alias, float lr, uint64_t seed, int32_t mode, double *loss,
                          int64_t *pairs, int32_t *dump_pairs, int32_t *dump_negs, cudaStream_t st,
                          unsigned long long *masked, int prepared)
 {
-    if (n_walks == 0) return GS_OK;
-    SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
-    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
-    switch (dim) {
-        case 64: return run_mode<64, __nv_bfloat16>(a, mode, st);
-        case 128: return run_mode<128, __nv_bfloat16>(a, mode, st);
-        case 256: return run_mode<256, __nv_bfloat16>(a, mode, st);
-        default:
-            set_error("dim %d not supported with 16-bit tables (64, 128, 256)", dim);
-            return GS_ERR_UNSUPPORTED;
-    }
+    return step_on_tables<__nv_bfloat16>(w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K,
+                                         alias, lr, seed, mode, loss, pairs, dump_pairs, dump_negs, st,
+                                         masked, prepared);
 }
 
 gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_out, int32_t *last_in,

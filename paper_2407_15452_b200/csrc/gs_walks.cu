@@ -90,8 +90,28 @@ gs_status validate_csr(const gs_graph *g, bool check_sorted, cudaStream_t st,
 }
 
 // ------------------------------------------------------------------ table init
+// Four start values of a row: (u - 0.5) / dim with u = (word >> 8) * 2^-24, stored in the table's
+// type (16-bit formats: rounded to nearest even).
+__device__ __forceinline__ void store_quad(float *w, int64_t x, float a, float b, float c, float d)
+{
+    reinterpret_cast<float4 *>(w)[x] = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store_quad(__half *w, int64_t x, float a, float b, float c, float d)
+{
+    __half2 *p = reinterpret_cast<__half2 *>(w) + 2 * x;
+    p[0] = __floats2half2_rn(a, b);
+    p[1] = __floats2half2_rn(c, d);
+}
+__device__ __forceinline__ void store_quad(__nv_bfloat16 *w, int64_t x, float a, float b, float c, float d)
+{
+    __nv_bfloat162 *p = reinterpret_cast<__nv_bfloat162 *>(w) + 2 * x;
+    p[0] = __floats2bfloat162_rn(a, b);
+    p[1] = __floats2bfloat162_rn(c, d);
+}
+
+template <typename T>
 __global__ void __launch_bounds__(256)
-init_rows_kernel(float *__restrict__ w, int64_t n_rows, int32_t dim, uint64_t seed)
+init_rows_kernel(T *__restrict__ w, int64_t n_rows, int32_t dim, uint64_t seed)
 {
     const int32_t quads = dim >> 2;
     const int64_t total = n_rows * quads;
@@ -101,105 +121,45 @@ init_rows_kernel(float *__restrict__ w, int64_t n_rows, int32_t dim, uint64_t se
         const int64_t row = x / quads;
         const uint32_t qd = (uint32_t)(x - row * quads);
         const uint4 r = draw(seed, (uint64_t)row, qd, TAG_INIT, 0);
-        float4 v;
-        v.x = ((float)(r.x >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        v.y = ((float)(r.y >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        v.z = ((float)(r.z >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        v.w = ((float)(r.w >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        reinterpret_cast<float4 *>(w)[x] = v;
+        store_quad(w, x, ((float)(r.x >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d,
+                   ((float)(r.y >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d,
+                   ((float)(r.z >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d,
+                   ((float)(r.w >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d);
     }
 }
 
-// Same start values rounded to IEEE half (round to nearest even).
-__global__ void __launch_bounds__(256)
-init_rows_f16_kernel(__half *__restrict__ w, int64_t n_rows, int32_t dim, uint64_t seed)
-{
-    const int32_t quads = dim >> 2;
-    const int64_t total = n_rows * quads;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const float inv_d = 1.0f / (float)dim;
-    for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < total; x += stride) {
-        const int64_t row = x / quads;
-        const uint32_t qd = (uint32_t)(x - row * quads);
-        const uint4 r = draw(seed, (uint64_t)row, qd, TAG_INIT, 0);
-        const float a = ((float)(r.x >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        const float b = ((float)(r.y >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        const float c = ((float)(r.z >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        const float d = ((float)(r.w >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        __half2 *p = reinterpret_cast<__half2 *>(w) + 2 * x;
-        p[0] = __floats2half2_rn(a, b);
-        p[1] = __floats2half2_rn(c, d);
-    }
-}
-
-// ... and rounded to bfloat16 (round to nearest even).
-__global__ void __launch_bounds__(256)
-init_rows_bf16_kernel(__nv_bfloat16 *__restrict__ w, int64_t n_rows, int32_t dim, uint64_t seed)
-{
-    const int32_t quads = dim >> 2;
-    const int64_t total = n_rows * quads;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const float inv_d = 1.0f / (float)dim;
-    for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < total; x += stride) {
-        const int64_t row = x / quads;
-        const uint32_t qd = (uint32_t)(x - row * quads);
-        const uint4 r = draw(seed, (uint64_t)row, qd, TAG_INIT, 0);
-        const float a = ((float)(r.x >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        const float b = ((float)(r.y >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        const float c = ((float)(r.z >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        const float d = ((float)(r.w >> 8) * (1.0f / 16777216.0f) - 0.5f) * inv_d;
-        __nv_bfloat162 *p = reinterpret_cast<__nv_bfloat162 *>(w) + 2 * x;
-        p[0] = __floats2bfloat162_rn(a, b);
-        p[1] = __floats2bfloat162_rn(c, d);
-    }
-}
-
-gs_status init_embeddings_bf16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
-                               cudaStream_t st)
+template <typename T>
+static gs_status init_tables(T *w_in, T *w_out, int64_t n, int32_t dim, uint64_t seed, cudaStream_t st)
 {
     if (w_in && n > 0) {
         const int64_t total = n * (dim >> 2);
         int64_t blocks = (total + 255) / 256;
         const int64_t cap = (int64_t)sm_count() * 32;
         if (blocks > cap) blocks = cap;
-        init_rows_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((__nv_bfloat16 *)w_in, n, dim, seed);
+        init_rows_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(w_in, n, dim, seed);
         GS_CUDA_TRY(cudaGetLastError());
     }
     if (w_out && n > 0)
-        GS_CUDA_TRY(cudaMemsetAsync(w_out, 0, sizeof(__nv_bfloat16) * (size_t)n * (size_t)dim, st));
-    return GS_OK;
-}
-
-gs_status init_embeddings_f16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
-                              cudaStream_t st)
-{
-    if (w_in && n > 0) {
-        const int64_t total = n * (dim >> 2);
-        int64_t blocks = (total + 255) / 256;
-        const int64_t cap = (int64_t)sm_count() * 32;
-        if (blocks > cap) blocks = cap;
-        init_rows_f16_kernel<<<(unsigned)blocks, 256, 0, st>>>((__half *)w_in, n, dim, seed);
-        GS_CUDA_TRY(cudaGetLastError());
-    }
-    if (w_out && n > 0)
-        GS_CUDA_TRY(cudaMemsetAsync(w_out, 0, sizeof(__half) * (size_t)n * (size_t)dim, st));
+        GS_CUDA_TRY(cudaMemsetAsync(w_out, 0, sizeof(T) * (size_t)n * (size_t)dim, st));
     return GS_OK;
 }
 
 gs_status init_embeddings(float *w_in, float *w_out, int64_t n, int32_t dim, uint64_t seed,
                           cudaStream_t st)
 {
-    if (w_in && n > 0) {
-        const int64_t total = n * (dim >> 2);
-        int64_t blocks = (total + 255) / 256;
-        const int64_t cap = (int64_t)sm_count() * 32;
-        if (blocks > cap) blocks = cap;
-        init_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(w_in, n, dim, seed);
-        GS_CUDA_TRY(cudaGetLastError());
-    }
-    if (w_out && n > 0)
-        GS_CUDA_TRY(cudaMemsetAsync(w_out, 0, sizeof(float) * (size_t)n * (size_t)dim, st));
-    return GS_OK;
+    return init_tables<float>(w_in, w_out, n, dim, seed, st);
+}
+
+gs_status init_embeddings_f16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
+                              cudaStream_t st)
+{
+    return init_tables<__half>((__half *)w_in, (__half *)w_out, n, dim, seed, st);
+}
+
+gs_status init_embeddings_bf16(void *w_in, void *w_out, int64_t n, int32_t dim, uint64_t seed,
+                               cudaStream_t st)
+{
+    return init_tables<__nv_bfloat16>((__nv_bfloat16 *)w_in, (__nv_bfloat16 *)w_out, n, dim, seed, st);
 }
 
 // ------------------------------------------------------------------ uniform walks

@@ -64,7 +64,7 @@ void gso_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
 
 /* Stream tags: which consumer of random words a counter belongs to. */
 enum { TAG_UNIFORM_WALK = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4,
-       TAG_WINDOW = 5, TAG_SUBSAMPLE = 6, TAG_SHUFFLE = 7 };
+       TAG_WINDOW = 5, TAG_SUBSAMPLE = 6, TAG_SHUFFLE = 7, TAG_ROUND_SYNC = 8, TAG_ROUND_LOCKFREE = 9 };
 
 /* Keying shared (as a published convention, not as code) with the GPU path:
  * key = 64-bit seed; counter = (id low, id high, step, tag<<24 | sub). */
@@ -574,12 +574,107 @@ void gso_round_bf16(double *x, int64_t n)
     for (int64_t i = 0; i < n; ++i) x[i] = rnb16(x[i]);
 }
 
+/* ------------------------------------------------------------------------
+ * Stochastic rounding to a 16-bit format (Section 4.2 of the paper keeps its production tables in
+ * 16 bits; with round-to-nearest an increment below half a unit in the last place is lost every
+ * time, with stochastic rounding it survives in expectation).
+ *
+ * The decision is taken on the fp32 value xf = float(x).  Let lo and hi be the neighbours of |xf|
+ * in the format (lo towards zero; fmt 0: binary16, 11 significant bits, spacing never below
+ * 2^-24; fmt 1: bfloat16, 8 significant bits, spacing never below 2^-133), frac = (|xf| - lo) /
+ * (hi - lo) in [0, 1) and thr = floor(frac * 2^16).  The result is hi when the 16-bit dither u16
+ * is below thr, else lo, with the sign of xf; a value that is representable never moves; a
+ * magnitude beyond the largest finite value of the format, or a step up from it, gives that
+ * largest value (no infinities are produced).
+ * ---------------------------------------------------------------------- */
+static double sr16(double x, int fmt, uint32_t u16)
+{
+    const float xf = (float)x;
+    if (xf == 0.0f || isnan(xf)) return (double)xf;
+    const int p = fmt ? 8 : 11;
+    const int qmin = fmt ? -133 : -24;
+    const double maxv = fmt ? 3.3895313892515355e38 : 65504.0;
+    const double ax = fabs((double)xf);
+    double r;
+    if (ax >= maxv) {
+        r = maxv;
+    } else {
+        int e;
+        frexp(ax, &e);                       /* ax = m * 2^e, 0.5 <= m < 1 */
+        int q = e - p;                       /* spacing 2^q keeps p significant bits */
+        if (q < qmin) q = qmin;
+        const double scaled = ldexp(ax, -q); /* exact */
+        const double lo = floor(scaled);
+        const uint32_t thr = (uint32_t)floor((scaled - lo) * 65536.0);
+        r = ldexp(lo + (u16 < thr ? 1.0 : 0.0), q);
+        if (r > maxv) r = maxv;
+    }
+    return xf < 0.0f ? -r : r;
+}
+
+void gso_round_sr(double *x, int64_t n, int fmt, const uint32_t *u16)
+{
+    for (int64_t i = 0; i < n; ++i) x[i] = sr16(x[i], fmt, u16[i] & 0xFFFFu);
+}
+
+/* The dither of column j of one row-write event.  An event has one Philox block r[0..3]; the
+ * 16-bit dithers of its columns come from a cheap mix of those words (the finalizer of
+ * MurmurHash3, a bijection of 32-bit words, so distinct inputs give distinct outputs): columns
+ * 2k and 2k+1 take the upper and lower half of
+ *   mix(r[k & 3] ^ 0x9E3779B9 * (k / 4 + 1) ^ 0x85EBCA77 * salt),
+ * `salt` telling apart the rows that share an event (lock-free mode). */
+static uint32_t mix32(uint32_t h)
+{
+    h ^= h >> 16; h *= 0x85EBCA6Bu; h ^= h >> 13; h *= 0xC2B2AE35u; h ^= h >> 16;
+    return h;
+}
+
+static uint32_t dither16(const uint32_t r[4], uint32_t salt, int32_t j)
+{
+    const uint32_t k = (uint32_t)j >> 1;
+    const uint32_t h = mix32(r[k & 3u] ^ (0x9E3779B9u * ((k >> 2) + 1u)) ^ (0x85EBCA77u * salt));
+    return (j & 1) ? (h & 0xFFFFu) : (h >> 16);
+}
+
+void gso_dither16(const uint32_t r[4], uint32_t salt, int32_t d, uint32_t *out)
+{
+    for (int32_t j = 0; j < d; ++j) out[j] = dither16(r, salt, j);
+}
+
+/* Event of the synchronous mode: row `row` of table `table` (0 input, 1 output) written by the
+ * step whose first walk id is walk_id_base: block (id = row | table << 32, step = low word of
+ * walk_id_base, TAG_ROUND_SYNC, sub = bits 32..55 of walk_id_base), salt 0. */
+static void sync_round_event(uint64_t seed, int64_t row, uint32_t table, int64_t walk_id_base, uint32_t r[4])
+{
+    draw4(seed, (uint64_t)row | ((uint64_t)table << 32), (uint32_t)((uint64_t)walk_id_base & 0xFFFFFFFFu),
+          TAG_ROUND_SYNC, (uint32_t)(((uint64_t)walk_id_base >> 32) & 0xFFFFFFu), r);
+}
+
+/* Rounds every value of X[n_rows][d] stochastically as the synchronous step writes it (a value
+ * that is representable already - every value of a row the step did not touch - stays). */
+void gso_round_sr_rows(double *X, int64_t n_rows, int32_t d, int fmt, uint64_t seed, uint32_t table,
+                       int64_t walk_id_base)
+{
+    for (int64_t row = 0; row < n_rows; ++row) {
+        uint32_t r[4];
+        sync_round_event(seed, row, table, walk_id_base, r);
+        for (int32_t j = 0; j < d; ++j)
+            X[row * d + j] = sr16(X[row * d + j], fmt, dither16(r, 0u, j));
+    }
+}
+
 /* Sequential per-pair SGD as gso_sgns_seq_from_lists, on tables whose values are kept in a
  * 16-bit format (fmt 0: binary16, 1: bfloat16): each updated output row and each updated center
  * row is rounded when written. */
+typedef struct {          /* stochastic write-back of the lock-free schedule (NULL: to nearest) */
+    uint64_t seed;
+    int64_t walk_id_base;
+    int32_t L;            /* walk length: slot e belongs to position e / S, walk (e / S) / L */
+} sr_keys;
+
 static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
                             const int32_t *centers, const int32_t *contexts, const int32_t *negs,
-                            double lr, int fmt, double *loss_sum, int64_t *pair_count);
+                            double lr, int fmt, const sr_keys *sr, double *loss_sum, int64_t *pair_count);
 
 int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
                                 int64_t n_slots, int32_t S, int32_t K,
@@ -587,7 +682,7 @@ int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
                                 const int32_t *negs, double lr,
                                 double *loss_sum, int64_t *pair_count)
 {
-    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 0, loss_sum, pair_count);
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 0, NULL, loss_sum, pair_count);
 }
 
 int gso_sgns_seq_bf16_from_lists(double *U, double *V, int32_t d,
@@ -596,12 +691,25 @@ int gso_sgns_seq_bf16_from_lists(double *U, double *V, int32_t d,
                                  const int32_t *negs, double lr,
                                  double *loss_sum, int64_t *pair_count)
 {
-    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 1, loss_sum, pair_count);
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 1, NULL, loss_sum, pair_count);
+}
+
+/* Same with stochastic write-back.  Event of the lock-free mode: the rows written while position
+ * i of walk `id` is worked on share the block (id, step = i, TAG_ROUND_LOCKFREE, sub 0); a target
+ * row takes salt = 1 + its index in the position's target list (slot * (1 + K) for the context of
+ * a slot, + 1 + k for its negative k), the center row salt 0x10000. */
+int gso_sgns_seq_sr_from_lists(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
+                               const int32_t *centers, const int32_t *contexts, const int32_t *negs,
+                               double lr, int fmt, uint64_t seed, int64_t walk_id_base, int32_t L,
+                               double *loss_sum, int64_t *pair_count)
+{
+    sr_keys sr = { seed, walk_id_base, L };
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, fmt, &sr, loss_sum, pair_count);
 }
 
 static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
                             const int32_t *centers, const int32_t *contexts, const int32_t *negs,
-                            double lr, int fmt, double *loss_sum, int64_t *pair_count)
+                            double lr, int fmt, const sr_keys *sr, double *loss_sum, int64_t *pair_count)
 {
     double *acc = (double *)malloc(sizeof(double) * (size_t)d);
     if (!acc) return -1;
@@ -609,6 +717,12 @@ static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, in
     int64_t pairs = 0;
     for (int64_t base = 0; base < n_slots; base += S) {
         int64_t c = -1;
+        uint32_t ev[4] = { 0, 0, 0, 0 };
+        if (sr) {
+            const int64_t pos = base / S;
+            draw4(sr->seed, (uint64_t)(sr->walk_id_base + pos / sr->L), (uint32_t)(pos % sr->L),
+                  TAG_ROUND_LOCKFREE, 0, ev);
+        }
         for (int32_t j = 0; j < d; ++j) acc[j] = 0.0;
         for (int32_t sg = 0; sg < S && base + sg < n_slots; ++sg) {
             int64_t e = base + sg;
@@ -624,16 +738,18 @@ static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, in
                 double f = dot(u, v, d);
                 double g = (k < 0) ? sigmoid(f) - 1.0 : sigmoid(f);
                 loss += (k < 0) ? softplus(-f) : softplus(f);
+                const uint32_t salt = 1u + (uint32_t)(sg * (1 + K) + (k + 1));
                 for (int32_t j = 0; j < d; ++j) {
                     acc[j] += g * v[j];
-                    v[j] = fmt ? rnb16(v[j] - lr * g * u[j]) : rn16(v[j] - lr * g * u[j]);
+                    const double nv = v[j] - lr * g * u[j];
+                    v[j] = sr ? sr16(nv, fmt, dither16(ev, salt, j)) : (fmt ? rnb16(nv) : rn16(nv));
                 }
             }
         }
         if (c >= 0)
             for (int32_t j = 0; j < d; ++j) {
                 double nv = U[c * d + j] - lr * acc[j];
-                U[c * d + j] = fmt ? rnb16(nv) : rn16(nv);
+                U[c * d + j] = sr ? sr16(nv, fmt, dither16(ev, 0x10000u, j)) : (fmt ? rnb16(nv) : rn16(nv));
             }
     }
     free(acc);

@@ -303,6 +303,62 @@ def sgns_seq_f16_from_lists(U, V, centers, contexts, negs, S, lr):
     return float(loss.value), int(cnt.value)
 
 
+def round_sr(x, fmt, u16):
+    """In place: every value rounded stochastically to binary16 (fmt 0) or bfloat16 (fmt 1) with the
+    given 16-bit dithers (one per value)."""
+    assert x.dtype == np.float64 and x.flags.c_contiguous
+    u = np.ascontiguousarray(u16, dtype=np.uint32)
+    assert u.size == x.size
+    lib().gso_round_sr(_p(x, ctypes.c_double), ctypes.c_int64(x.size), ctypes.c_int32(fmt), _p(u, ctypes.c_uint32))
+    return x
+
+
+def dither16(words, salt, d):
+    """The 16-bit dithers of the d columns of a row-write event with Philox block `words`."""
+    r = np.ascontiguousarray(words, dtype=np.uint32)
+    out = np.empty(d, dtype=np.uint32)
+    lib().gso_dither16(_p(r, ctypes.c_uint32), ctypes.c_uint32(salt), ctypes.c_int32(d), _p(out, ctypes.c_uint32))
+    return out
+
+
+def round_sr_rows(X, fmt, seed, table, walk_id_base):
+    """In place: table X (0 input, 1 output) as the synchronous step with stochastic write-back
+    leaves it: every value rounded with the dither of its (row, column) for that step."""
+    assert X.dtype == np.float64 and X.flags.c_contiguous
+    lib().gso_round_sr_rows(_p(X, ctypes.c_double), ctypes.c_int64(X.shape[0]), ctypes.c_int32(X.shape[1]),
+                            ctypes.c_int32(fmt), ctypes.c_uint64(seed), ctypes.c_uint32(table),
+                            ctypes.c_int64(walk_id_base))
+    return X
+
+
+def sgns_det_sr_from_lists(U, V, centers, contexts, negs, lr, fmt, seed, walk_id_base):
+    """Synchronous step on 16-bit-valued tables with stochastic write-back: full-precision step,
+    then every written value rounded stochastically (rows that are not written hold representable
+    values, which never move)."""
+    out = sgns_det_from_lists(U, V, centers, contexts, negs, lr)
+    round_sr_rows(U, fmt, seed, 0, walk_id_base)
+    round_sr_rows(V, fmt, seed, 1, walk_id_base)
+    return out
+
+
+def sgns_seq_sr_from_lists(U, V, centers, contexts, negs, S, lr, fmt, seed, walk_id_base, L):
+    """Sequential per-pair SGD on 16-bit-valued tables with stochastic write-back, in place."""
+    d = U.shape[1]
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    K = negs.shape[1]
+    loss = ctypes.c_double(0.0)
+    cnt = ctypes.c_int64(0)
+    rc = lib().gso_sgns_seq_sr_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int32(d),
+        ctypes.c_int64(len(centers)), ctypes.c_int32(S), ctypes.c_int32(K),
+        _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32),
+        ctypes.c_double(lr), ctypes.c_int32(fmt), ctypes.c_uint64(seed), ctypes.c_int64(walk_id_base),
+        ctypes.c_int32(L), ctypes.byref(loss), ctypes.byref(cnt))
+    if rc != 0:
+        raise MemoryError("oracle accumulator")
+    return float(loss.value), int(cnt.value)
+
+
 def keep_thresholds(weights, t):
     """Sub-sampling thresholds: keep(v) = min(1, sqrt(t / f(v))) as uint32 (0xFFFFFFFF = always)."""
     wgt = np.ascontiguousarray(weights, dtype=np.float64)

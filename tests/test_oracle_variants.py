@@ -251,3 +251,176 @@ def test_touched_rows_and_adam_step_on_lists():
     GU, GV, _, _ = O.sgns_grad_from_lists(U0, V0, c, o, ng)
     moved = np.abs(GV) > 1e-6                                     # step 1: lr * sign(g)
     assert np.allclose((V - V0)[moved], -0.01 * np.sign(GV[moved]), atol=1e-6)
+
+
+# ---------------------------------------------------------------- stochastic rounding to 16 bits
+def neighbours_f16(x32):
+    """(lo, hi) of |x32| among the binary16 values, lo towards zero, by numpy's own conversion and
+    nextafter; hi is inf above the largest finite value."""
+    ax = np.abs(x32.astype(np.float64))
+    a = np.abs(x32).astype(np.float16)                       # to nearest
+    lo = np.where(a.astype(np.float64) <= ax, a, np.nextafter(a, np.float16(0)))
+    hi = np.nextafter(lo, np.float16(np.inf))
+    return lo.astype(np.float64), hi.astype(np.float64)
+
+
+def neighbours_bf16(x32):
+    """(lo, hi) of |x32| among the bfloat16 values: the upper 16 bits of the fp32 pattern."""
+    bits = np.abs(x32).view(np.uint32)
+    lo = (bits & np.uint32(0xFFFF0000)).view(np.float32).astype(np.float64)
+    hi = ((bits & np.uint32(0xFFFF0000)) + np.uint32(0x10000)).view(np.float32).astype(np.float64)
+    return lo, hi
+
+
+def sample_values(rng, n, fmt):
+    mags = rng.uniform(-30, 12, n) if fmt == 0 else rng.uniform(-120, 100, n)   # includes binary16 subnormals
+    return (rng.choice([-1.0, 1.0], n) * rng.uniform(1, 2, n) * 2.0 ** mags).astype(np.float32)
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_stochastic_rounding_picks_a_neighbour_with_the_right_threshold(fmt):
+    rng = np.random.default_rng(3 + fmt)
+    x = sample_values(rng, 20000, fmt)
+    lo, hi = (neighbours_f16 if fmt == 0 else neighbours_bf16)(x)
+    finite = np.isfinite(hi)
+    ax = np.abs(x.astype(np.float64))
+    frac = np.where(finite & (hi > lo), (ax - lo) / np.where(finite & (hi > lo), hi - lo, 1.0), 0.0)
+    thr = np.floor(frac * 65536.0).astype(np.int64)
+    assert ((frac >= 0) & (frac < 1)).all() and (thr[frac > 0] >= 0).all()
+    sign = np.sign(x.astype(np.float64))
+    for u in (np.zeros_like(thr), np.maximum(thr - 1, 0), thr, np.full_like(thr, 65535), rng.integers(0, 65536, len(thr))):
+        got = O.round_sr(x.astype(np.float64), fmt, u.astype(np.uint32))
+        want = sign * np.where((u < thr) & finite, hi, lo)
+        assert np.array_equal(got, want)
+    # representable values never move, whatever the dither
+    rep = lo[lo > 0] * sign[lo > 0]
+    for u in (0, 1, 40000, 65535):
+        assert np.array_equal(O.round_sr(rep.copy(), fmt, np.full(len(rep), u, dtype=np.uint32)), rep)
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_stochastic_rounding_is_unbiased_and_saturates(fmt):
+    # over all 65536 dithers the mean is lo + (hi - lo) * thr / 2^16: within one 2^-16 of the spacing of x
+    rng = np.random.default_rng(8)
+    u_all = np.arange(65536, dtype=np.uint32)
+    for x in sample_values(rng, 12, fmt):
+        lo, hi = (neighbours_f16 if fmt == 0 else neighbours_bf16)(np.array([x], dtype=np.float32))
+        got = O.round_sr(np.full(65536, float(x)), fmt, u_all)
+        assert set(np.unique(np.abs(got))) <= {lo[0], hi[0]}
+        assert abs(got.mean() - float(x)) <= (hi[0] - lo[0]) / 65536.0 + 1e-300
+        ups = int((np.abs(got) == hi[0]).sum()) if hi[0] > lo[0] else 0
+        assert ups == int(np.floor((abs(float(x)) - lo[0]) / (hi[0] - lo[0]) * 65536.0))
+    # an exact tie goes up for exactly half of the dithers
+    tie = 1.0 + (2.0 ** -11 if fmt == 0 else 2.0 ** -8)
+    got = O.round_sr(np.full(65536, tie), fmt, u_all)
+    assert int((got > 1.0).sum()) == 32768 and np.array_equal(got > 1.0, u_all < 32768)
+    # beyond the largest finite value, and a step up from it: the largest finite value, never inf
+    top = 65504.0 if fmt == 0 else float(np.array([0x7F7F0000], dtype=np.uint32).view(np.float32)[0])
+    edge = np.array([top, -top, top * (1 + 2.0 ** -13), 1e39, -1e39, np.inf])
+    for u in (0, 65535):
+        got = O.round_sr(edge.copy(), fmt, np.full(len(edge), u, dtype=np.uint32))
+        assert np.array_equal(got, [top, -top, top, top, -top, top])
+    # symmetric in the sign
+    x = sample_values(rng, 500, fmt).astype(np.float64)
+    u = rng.integers(0, 65536, len(x)).astype(np.uint32)
+    assert np.array_equal(O.round_sr(x.copy(), fmt, u), -O.round_sr(-x, fmt, u))
+
+
+def test_dithers_of_a_row_write_are_keyed_well_spread_and_distinct():
+    rng = np.random.default_rng(1)
+    counts = np.zeros(64)
+    for _ in range(400):
+        r = rng.integers(0, 2 ** 32, 4, dtype=np.uint64).astype(np.uint32)
+        salt = int(rng.integers(0, 2 ** 17))
+        d = O.dither16(r, salt, 256)
+        assert np.array_equal(d, O.dither16(r, salt, 256)) and d.max() < 65536      # a function of its key
+        assert not np.array_equal(d, O.dither16(r, salt + 1, 256))                  # the salt matters
+        r2 = r.copy()
+        r2[2] ^= 1
+        assert not np.array_equal(d, O.dither16(r2, salt, 256))                     # so does every word
+        # columns 2k and 2k+1 are the halves of one mixed word, and the mixed words of a row are
+        # pairwise distinct (the mix is a bijection and the columns feed it distinct inputs
+        # unless two of the four words happen to collide, which random words do not)
+        words = (d[0::2].astype(np.uint64) << np.uint64(16)) | d[1::2].astype(np.uint64)
+        assert len(np.unique(words)) == len(words)
+        counts += np.bincount(d >> 10, minlength=64)
+    assert chi2_uniform_ok(counts)
+
+
+def sync_event(seed, row, table, base):
+    return O.philox4x32_10([row & 0xFFFFFFFF, table, base & 0xFFFFFFFF, (8 << 24) | ((base >> 32) & 0xFFFFFF)],
+                           [seed & 0xFFFFFFFF, seed >> 32])
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_synchronous_step_with_stochastic_write_back(fmt):
+    # the step is the full-precision step followed by ONE stochastic rounding of every written value,
+    # keyed by (row, table, first walk id of the step): re-assembled here from the Philox block,
+    # the dithers and the rounding of single values
+    off, col, thr, alias, walks = tiny_setup(n_walks=40, L=12)
+    n, d, seed, base = len(off) - 1, 32, 77, (5 << 32) + 40
+    c, o, ng, _ = O.expand_lists(walks, base, 3, 2, thr, alias, seed)
+    rng = np.random.default_rng(2)
+    rnd = O.round_f16 if fmt == 0 else O.round_bf16
+    U0 = rnd(rng.uniform(-0.3, 0.3, (n, d)))
+    V0 = rnd(rng.uniform(-0.3, 0.3, (n, d)))
+    Ue, Ve = U0.copy(), V0.copy()
+    O.sgns_det_from_lists(Ue, Ve, c, o, ng, 0.05)                        # exact step
+    U, V = U0.copy(), V0.copy()
+    O.sgns_det_sr_from_lists(U, V, c, o, ng, 0.05, fmt, seed, base)
+    for X, Xe, X0, table in ((U, Ue, U0, 0), (V, Ve, V0, 1)):
+        touched = np.nonzero((Xe != X0).any(axis=1))[0]
+        assert len(touched) > 50
+        assert np.array_equal(np.delete(X, touched, axis=0), np.delete(X0, touched, axis=0))   # others keep their bits
+        for row in touched[:40]:
+            u = O.dither16(sync_event(seed, int(row), table, base), 0, d)
+            assert np.array_equal(X[row], O.round_sr(Xe[row].copy(), fmt, u))
+    # another step (another first walk id) or another seed rounds differently; the same key repeats
+    U2, V2 = U0.copy(), V0.copy()
+    O.sgns_det_sr_from_lists(U2, V2, c, o, ng, 0.05, fmt, seed, base)
+    assert np.array_equal(U, U2) and np.array_equal(V, V2)
+    U3, V3 = U0.copy(), V0.copy()
+    O.sgns_det_sr_from_lists(U3, V3, c, o, ng, 0.05, fmt, seed + 1, base)
+    assert not np.array_equal(V, V3)
+    # unbiased where to-nearest is not: mean over seeds against the exact value
+    rows = np.nonzero((Ve != V0).any(axis=1))[0][:8]
+    acc = np.zeros((len(rows), d))
+    n_seeds = 300
+    for s in range(n_seeds):
+        Us, Vs = U0.copy(), V0.copy()
+        O.sgns_det_sr_from_lists(Us, Vs, c, o, ng, 0.05, fmt, 1000 + s, base)
+        acc += Vs[rows]
+    spacing = np.abs(Ve[rows]) * 2.0 ** (-10 if fmt == 0 else -7)         # at most one unit in the last place
+    assert (np.abs(acc / n_seeds - Ve[rows]) <= 4 * 0.5 * spacing / np.sqrt(n_seeds) + 1e-9).all()
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_sequential_mode_with_stochastic_write_back_keys_every_write(fmt):
+    # one walk, no negatives: the first pair of position 0 writes the context row and, after the
+    # position's last pair, the center row - with the block (walk id, position, tag 9), salt 1 + index
+    # in the position's target list for the target and 0x10000 for the center
+    n, d, L, w, seed, base = 50, 16, 4, 1, 9, 1234
+    walk = np.array([[3, 7, 11, 15]], dtype=np.int32)
+    thr, alias = O.build_alias(np.ones(n), 1.0)
+    c, o, ng, _ = O.expand_lists(walk, base, w, 0, thr, alias, seed)
+    rng = np.random.default_rng(4)
+    rnd = O.round_f16 if fmt == 0 else O.round_bf16
+    U0, V0 = rnd(rng.uniform(-0.4, 0.4, (n, d))), rnd(rng.uniform(-0.4, 0.4, (n, d)))
+    U, V = U0.copy(), V0.copy()
+    O.sgns_seq_sr_from_lists(U, V, c, o, ng, 2 * w, 0.1, fmt, seed, base, L)
+    # position 0 has one pair: (3, 7) in slot 1 (the later context); K = 0, so its list index is 1
+    ev = O.philox4x32_10([base & 0xFFFFFFFF, base >> 32, 0, 9 << 24], [seed, 0])
+    f = float(U0[3] @ V0[7])
+    g = 1.0 / (1.0 + np.exp(-f)) - 1.0
+    want_v = O.round_sr(V0[7] - 0.1 * g * U0[3], fmt, O.dither16(ev, 1 + 1, d))
+    want_u = O.round_sr(U0[3] - 0.1 * g * V0[7], fmt, O.dither16(ev, 0x10000, d))
+    assert np.array_equal(U[3], want_u)
+    # row 7 is written again by position 2 (center 11): undo nothing, compare after position 0 only
+    Ua, Va = U0.copy(), V0.copy()
+    O.sgns_seq_sr_from_lists(Ua, Va, c[:2], o[:2], ng[:2], 2 * w, 0.1, fmt, seed, base, L)
+    assert np.array_equal(Va[7], want_v) and np.array_equal(Ua[3], want_u)
+    # with dithers that never round up the result is truncation; the mode differs from to-nearest
+    Ub, Vb = U0.copy(), V0.copy()
+    (O.sgns_seq_f16_from_lists if fmt == 0 else O.sgns_seq_bf16_from_lists)(Ub, Vb, c, o, ng, 2 * w, 0.1)
+    assert not np.array_equal(V, Vb)
+    assert np.abs(V - Vb).max() <= np.abs(Vb).max() * 2.0 ** (-9 if fmt == 0 else -6)

@@ -59,6 +59,8 @@ def parse_args():
                          "sub-sampling, t = 1e-5), shuffle (keyed start-node order)")
     ap.add_argument("--table-dtype", default="f32", choices=["f32", "f16", "bf16"],
                     help="storage type of the embedding tables (arithmetic is fp32 either way)")
+    ap.add_argument("--round", default="nearest", choices=["nearest", "stochastic"],
+                    help="write-back rounding of 16-bit tables")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample-walks", type=int, default=16384)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -555,6 +557,10 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
     variants = parse_variants(args)
     if "shrink" in variants:
         mode |= B.GS_WINDOW_SHRINK
+    if args.round == "stochastic":
+        if not f16:
+            raise SystemExit("--round stochastic needs --table-dtype f16 or bf16")
+        mode |= B.GS_ROUND_STOCHASTIC
     keep_thr = keep_thresholds_device(g, dev) if "subsample" in variants else None
     kind = B.GS_WALK_UNIFORM if wl.walk_kind == "uniform" else B.GS_WALK_NODE2VEC
     total_walks = n * wl.walks_per_node
@@ -685,7 +691,7 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": wl.name, "mode": mode_name, "table_dtype": args.table_dtype,
-                       "batch_walks": bw,
+                       "round": args.round if f16 else None, "batch_walks": bw,
                        "walk_kind": wl.walk_kind, "walk_len": wl.walk_len, "window": wl.window,
                        "n_neg": wl.n_neg, "dim": wl.dim, "scale": args.scale, "variants": sorted(variants),
                        "l2": "tables (2 x n x dim x 4 B) and CSR far exceed the 126 MB L2; no flush"

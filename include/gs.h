@@ -34,6 +34,7 @@
  *      tag 5 window draw  : id = walk id, step = position i
  *      tag 6 sub-sampling : id = walk id, step = position t
  *      tag 7 start shuffle: id = right half | epoch << 32, step = Feistel round
+ *      tag 8, 9 dithers of the stochastic write-back (GS_ROUND_STOCHASTIC)
  *  - A 32-bit word r is mapped to [0, n) as (r * n) >> 32.
  */
 #ifndef GS_H
@@ -185,6 +186,21 @@ GS_API gs_status gs_node2vec_walks(const gs_graph *g, const int32_t *d_starts,
                                      /* weights near contexts more.  Slots and the keying of  */
                                      /* the negatives stay those of the full window.  (The    */
                                      /* paper's runs use a fixed window, Section 4.)          */
+
+#define GS_ROUND_STOCHASTIC   0x400   /* OR into `mode`, 16-bit tables only (gs_sgns_step_f16 / _bf16, and  */
+                                     /* gs_sgns_epoch with such tables): written values are rounded to    */
+                                     /* one of their two neighbours in the table's format, upwards in      */
+                                     /* magnitude with probability (|x| - lo) / (hi - lo) taken to 16     */
+                                     /* bits, instead of to the nearest.  An increment below half a unit  */
+                                     /* in the last place then survives in expectation.  (Section 4.2:    */
+                                     /* the production tables are 16-bit; the rounding is this library's.) */
+                                     /* Dithers: tag 8 (synchronous: block keyed by row | table << 32,    */
+                                     /* step = low word of walk_id_base, sub = its bits 32..55) or tag 9  */
+                                     /* (lock-free: block keyed by walk id, step = position; a target row */
+                                     /* takes salt 1 + its index in the position's target list, the       */
+                                     /* center row 0x10000); columns 2k, 2k+1 take the halves of          */
+                                     /* mix(word[k & 3] ^ 0x9E3779B9 (k/4 + 1) ^ 0x85EBCA77 salt).        */
+                                     /* GS_ERR_UNSUPPORTED with fp32 tables.                              */
 
 /*
  * One SGNS update over a batch of walks: skip-gram with negative sampling on

@@ -483,6 +483,11 @@ def sgns_epoch(off, col, thr, alias, U, V, *, walks_per_node, L, w, K, lr0, sche
             ls, pc = sgns_det_f16_from_lists(U, V, c, o, ng, lr)
         elif mode == "det_bf16":
             ls, pc = sgns_det_bf16_from_lists(U, V, c, o, ng, lr)
+        elif mode in ("det_sr_f16", "det_sr_bf16"):    # 16-bit tables, stochastic write-back
+            ls, pc = sgns_det_sr_from_lists(U, V, c, o, ng, lr, 0 if mode == "det_sr_f16" else 1, seed, base)
+        elif mode in ("seq_sr_f16", "seq_sr_bf16"):
+            ls, pc = sgns_seq_sr_from_lists(U, V, c, o, ng, 2 * w, lr, 0 if mode == "seq_sr_f16" else 1,
+                                            seed, base, L)
         else:
             ls, pc = sgns_seq_from_lists(U, V, c, o, ng, 2 * w, lr)
         loss_sum += ls

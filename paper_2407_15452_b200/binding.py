@@ -22,6 +22,7 @@ GS_VALIDATE, GS_REQUIRE_SORTED, GS_BUILD_WALK_INDEX, GS_BUILD_EDGE_SET = 1, 2, 4
 GS_DETERMINISTIC, GS_HOGWILD, GS_HOGWILD_RED = 0, 1, 2
 GS_PAIRS_FORWARD_ONLY = 0x100
 GS_WINDOW_SHRINK = 0x200
+GS_ROUND_STOCHASTIC = 0x400
 GS_WALK_UNIFORM, GS_WALK_NODE2VEC = 0, 1
 GS_LR_CONSTANT, GS_LR_LINEAR = 0, 1
 GS_TABLE_F32, GS_TABLE_F16, GS_TABLE_BF16 = 0, 1, 2

@@ -427,7 +427,7 @@ static gs_status check_sgns_shape(int32_t dim, int32_t L, int32_t w, int32_t K, 
     if (w < 1 || w > 32) { set_error("window %d outside [1, 32]", w); return GS_ERR_UNSUPPORTED; }
     if (K < 0 || K > 32) { set_error("n_neg %d outside [0, 32]", K); return GS_ERR_UNSUPPORTED; }
     if (2 * w * (1 + K) > 512) { set_error("2*window*(1+n_neg) = %d exceeds 512", 2 * w * (1 + K)); return GS_ERR_UNSUPPORTED; }
-    const int32_t base_mode = mode & ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
+    const int32_t base_mode = mode & ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK | GS_ROUND_STOCHASTIC);
     if (base_mode != GS_DETERMINISTIC && base_mode != GS_HOGWILD && base_mode != GS_HOGWILD_RED)
         return invalid("unknown mode");
     return GS_OK;
@@ -709,6 +709,7 @@ gs_status gs_sgns_epoch(const gs_graph *g, const uint64_t *d_alias, void *d_w_in
     gs_status s = check_sgns_shape(f16 ? 128 : cfg->dim, cfg->walk_len, cfg->window, cfg->n_neg, cfg->mode);
     if (s != GS_OK) return s;
     if (cfg->n_neg > 0 && !d_alias) return invalid("d_alias is NULL");
+    if ((cfg->mode & GS_ROUND_STOCHASTIC) && !f16) { set_error("GS_ROUND_STOCHASTIC applies to 16-bit tables"); return GS_ERR_UNSUPPORTED; }
     if (cfg->walks_per_node < 1 || cfg->batch_walks < 1) return invalid("walks_per_node and batch_walks must be >= 1");
     if (cfg->walk_kind != GS_WALK_UNIFORM && cfg->walk_kind != GS_WALK_NODE2VEC) return invalid("unknown walk_kind");
     if (cfg->lr_schedule != GS_LR_CONSTANT && cfg->lr_schedule != GS_LR_LINEAR) return invalid("unknown lr_schedule");

@@ -54,7 +54,8 @@ namespace gs {
 
 // ---- Philox4x32-10 ---------------------------------------------------------------
 enum : uint32_t { TAG_UNIFORM = 1, TAG_NODE2VEC = 2, TAG_NEGATIVE = 3, TAG_INIT = 4,
-                  TAG_WINDOW = 5, TAG_SUBSAMPLE = 6, TAG_SHUFFLE = 7 };
+                  TAG_WINDOW = 5, TAG_SUBSAMPLE = 6, TAG_SHUFFLE = 7, TAG_ROUND_SYNC = 8,
+                  TAG_ROUND_LOCKFREE = 9 };
 
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k)
 {

@@ -305,6 +305,108 @@ __device__ __forceinline__ void grow_store(T *__restrict__ tab, int64_t r, int s
         p[q * G::LPR + sub] = pack16(x.v + G::PER16 * q, (const T *)nullptr);
 }
 
+// ---------------------------------------------------------------- stochastic write-back (16-bit tables)
+// A value is rounded to one of its two neighbours in the table's format, upwards (in magnitude)
+// with probability (|x| - lo) / (hi - lo) taken to 16 bits: up iff the 16-bit dither is below
+// floor(frac * 2^16).  Representable values never move; nothing becomes infinite (a magnitude
+// beyond the largest finite value, or a step up from it, gives the largest finite value).
+__device__ __forceinline__ uint32_t sr_bits(float x, uint32_t u16, const __nv_bfloat16 *)
+{
+    // bfloat16 is the upper half of the fp32 pattern: the dropped 16 bits ARE frac * 2^16
+    const uint32_t bits = __float_as_uint(x);
+    uint32_t r = (bits >> 16) + (u16 < (bits & 0xFFFFu) ? 1u : 0u);
+    if ((r & 0x7FFFu) >= 0x7F80u) r = (r & 0x8000u) | 0x7F7Fu;
+    return r;
+}
+__device__ __forceinline__ uint32_t sr_bits(float x, uint32_t u16, const __half *)
+{
+    const float ax = fabsf(x);
+    const uint32_t abits = __float_as_uint(ax);
+    const uint32_t sign = (__float_as_uint(x) >> 16) & 0x8000u;
+    if (abits >= 0x38800000u && abits < 0x477FE000u) {
+        // normal range of binary16 (2^-14 <= |x| < 65504): 13 fraction bits are dropped, so they
+        // are frac * 2^13; the upper bits, with the exponent re-biased, are the neighbour towards zero
+        uint32_t h = (abits >> 13) - 0x1C000u;
+        h += u16 < ((abits & 0x1FFFu) << 3) ? 1u : 0u;
+        return sign | (h >= 0x7C00u ? 0x7BFFu : h);
+    }
+    if (!(ax < 65504.0f)) return sign | 0x7BFFu;
+    const __half lo_h = __float2half_rz(ax);                       // neighbour towards zero
+    const uint32_t lb = __half_as_ushort(lo_h);
+    const float lo = __half2float(lo_h);
+    const float hi = __half2float(__ushort_as_half((unsigned short)(lb + 1u)));
+    const float frac = (ax - lo) * __frcp_rn(hi - lo);             // both exact: hi - lo is a power of two
+    return sign | (lb + (u16 < (uint32_t)(frac * 65536.0f) ? 1u : 0u));
+}
+
+__device__ __forceinline__ uint32_t mix32(uint32_t h)
+{
+    h ^= h >> 16; h *= 0x85EBCA6Bu; h ^= h >> 13; h *= 0xC2B2AE35u; h ^= h >> 16;
+    return h;
+}
+
+// Dithers of columns 2k (upper half of the result) and 2k + 1 (lower half) of a row-write event
+// with Philox block ev; salt_term = 0x85EBCA77 * salt tells apart the rows that share an event.
+__device__ __forceinline__ uint32_t dither_pair(const uint4 &ev, uint32_t salt_term, uint32_t k)
+{
+    const uint32_t sel = k & 3u;
+    const uint32_t w = sel == 0 ? ev.x : sel == 1 ? ev.y : sel == 2 ? ev.z : ev.w;
+    return mix32(w ^ (0x9E3779B9u * ((k >> 2) + 1u)) ^ salt_term);
+}
+
+// Two consecutive columns 2k, 2k + 1 rounded stochastically and packed (low half: column 2k).
+template <typename T>
+__device__ __forceinline__ uint32_t sr_pack2(float a, float b, const uint4 &ev, uint32_t salt_term, uint32_t k)
+{
+    const uint32_t h = dither_pair(ev, salt_term, k);
+    return sr_bits(a, h >> 16, (const T *)nullptr) | (sr_bits(b, h & 0xFFFFu, (const T *)nullptr) << 16);
+}
+
+// grow_store with stochastic rounding (16-bit tables): lane `sub` holds, for access q, the 8
+// columns from (q * LPR + sub) * 8.
+template <int DIM, typename T, bool NARROW = false>
+__device__ __forceinline__ void grow_store_sr(T *__restrict__ tab, int64_t r, int sub,
+                                              const Row<RowGeom<DIM, T, NARROW>::FPL> &x, const uint4 &ev,
+                                              uint32_t salt_term)
+{
+    using G = RowGeom<DIM, T, NARROW>;
+    static_assert(sizeof(T) == 2, "stochastic write-back is for 16-bit tables");
+    uint4 *p = reinterpret_cast<uint4 *>(tab + r * (int64_t)DIM);
+#pragma unroll
+    for (int q = 0; q < G::FPL / G::PER16; ++q) {
+        const uint32_t k0 = (uint32_t)(q * G::LPR + sub) * 4u;     // first column pair of this access
+        const float *v = x.v + G::PER16 * q;
+        uint4 t;
+        t.x = sr_pack2<T>(v[0], v[1], ev, salt_term, k0);
+        t.y = sr_pack2<T>(v[2], v[3], ev, salt_term, k0 + 1);
+        t.z = sr_pack2<T>(v[4], v[5], ev, salt_term, k0 + 2);
+        t.w = sr_pack2<T>(v[6], v[7], ev, salt_term, k0 + 3);
+        p[q * G::LPR + sub] = t;
+    }
+}
+
+// row_store (whole warp per row) with stochastic rounding: lane holds, for piece q, the 4 columns
+// from (q * 32 + lane) * 4 (FPL = 2: columns 2 lane and 2 lane + 1).
+template <int FPL, typename T>
+__device__ __forceinline__ void row_store_sr(T *__restrict__ tab, int64_t r, int lane, const Row<FPL> &x,
+                                             const uint4 &ev)
+{
+    static_assert(sizeof(T) == 2, "stochastic write-back is for 16-bit tables");
+    T *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 2) {
+        reinterpret_cast<uint32_t *>(p)[lane] = sr_pack2<T>(x.v[0], x.v[1], ev, 0u, (uint32_t)lane);
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q) {
+            const uint32_t k0 = (uint32_t)(q * 32 + lane) * 2u;
+            uint2 t;
+            t.x = sr_pack2<T>(x.v[4 * q], x.v[4 * q + 1], ev, 0u, k0);
+            t.y = sr_pack2<T>(x.v[4 * q + 2], x.v[4 * q + 3], ev, 0u, k0 + 1);
+            reinterpret_cast<uint2 *>(p)[q * 32 + lane] = t;
+        }
+    }
+}
+
 // Stores a row held in the geometry of a T table into an fp32 scratch row (natural column order).
 template <int DIM, typename T>
 __device__ __forceinline__ void grow_store_f32(float *__restrict__ tab, int64_t r, int sub,
@@ -457,7 +559,7 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
 // walks covered by one ticket of the lock-free kernel (host and device agree on the buffer size)
 __host__ __device__ __forceinline__ int hogwild_walks_per_ticket(int L) { return L <= 16 ? 32 / L : 1; }
 
-template <int DIM, typename T, bool RED, int MINB, int TC, bool NARROW>
+template <int DIM, typename T, bool RED, int MINB, int TC, bool NARROW, bool SR = false>
 __global__ void __launch_bounds__(SGNS_WARPS * 32, MINB)
 sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                     const int32_t *__restrict__ walks, int64_t n_walks, int64_t walk_id_base,
@@ -513,6 +615,10 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             refused_acc += (unsigned long long)((unsigned)packed >> 20);
             if (pairs == 0) continue;
             pair_acc += (unsigned long long)pairs;
+            // stochastic write-back: the rows written while this position is worked on share one
+            // Philox block; a target takes salt 1 + its index in the list, the center row 0x10000
+            uint4 ev = make_uint4(0u, 0u, 0u, 0u);
+            if (SR) ev = draw(seed, id, (uint32_t)i, TAG_ROUND_LOCKFREE, 0);
             const Row<FPL> u = grow_load<DIM, T, NARROW>(w_in, c, sub);     // every group holds the center row
             Row<FPL> acc;                                        // this group's share of its gradient
 #pragma unroll
@@ -559,6 +665,9 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                                 rows[k].v[j] += delta.v[j];
                             }
                             if (RED) grow_red_add<DIM, NARROW>(w_out, ids[k], sub, delta);
+                            else if constexpr (SR)
+                                grow_store_sr<DIM, T, NARROW>(w_out, ids[k], sub, rows[k], ev,
+                                                              0x85EBCA77u * (uint32_t)(base + k * NG + grp + 1));
                             else grow_store<DIM, T, NARROW>(w_out, ids[k], sub, rows[k]);
                         }
                     }
@@ -577,7 +686,9 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                 Row<FPL> now = grow_load<DIM, T, NARROW>(w_in, c, sub);
 #pragma unroll
                 for (int j = 0; j < FPL; ++j) now.v[j] += delta.v[j];
-                if (grp == 0) grow_store<DIM, T, NARROW>(w_in, c, sub, now);
+                if constexpr (SR) {
+                    if (grp == 0) grow_store_sr<DIM, T, NARROW>(w_in, c, sub, now, ev, 0x85EBCA77u * 0x10000u);
+                } else if (grp == 0) grow_store<DIM, T, NARROW>(w_in, c, sub, now);
             }
             loss_acc += (double)loss;
         }
@@ -806,6 +917,10 @@ struct MomState {
     float *v;
     float b2, eps;
     double c1, c2;
+    // stochastic write-back of a 16-bit table in the synchronous mode (sr != 0): the event of row r
+    // is the block (r | sr_table << 32, sr_step, TAG_ROUND_SYNC, sr_sub), key sr_seed
+    uint32_t sr, sr_table, sr_step, sr_sub;
+    uint64_t sr_seed;
 };
 
 template <int FPL, typename T>
@@ -841,6 +956,14 @@ __device__ __forceinline__ void write_updated_row(T *__restrict__ tab, int64_t r
     } else {
 #pragma unroll
         for (int j = 0; j < FPL; ++j) row.v[j] = (float)((double)row.v[j] - (double)lr * acc[j]);
+    }
+    if constexpr (sizeof(T) == 2) {
+        if (ms.sr) {
+            const uint4 ev = draw(ms.sr_seed, (uint64_t)r | ((uint64_t)ms.sr_table << 32), ms.sr_step,
+                                  TAG_ROUND_SYNC, ms.sr_sub);
+            row_store_sr<FPL, T>(tab, r, lane, row, ev);
+            return;
+        }
     }
     row_store<FPL>(tab, r, lane, row);
 }
@@ -1466,16 +1589,17 @@ struct SgnsArgs {
     unsigned long long *masked;   // nullable: masked negatives are ADDED
     int prepared;                 // >= 0: scratch set in which part A of this batch already ran
     unsigned long long *refused;  // nullable: ids treated as absent because they name no row are ADDED
+    int sr;                       // 16-bit tables: stochastic write-back instead of round to nearest
 };
 
 static int bit_length(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
-template <int DIM, typename T, bool RED, int MINB, int TC = TCH, bool NARROW = false>
+template <int DIM, typename T, bool RED, int MINB, int TC = TCH, bool NARROW = false, bool SR = false>
 static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
     const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(hogwild_walks_per_ticket(a.L) * a.L + SL);
-    auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB, TC, NARROW>;
+    auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB, TC, NARROW, SR>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -1502,6 +1626,10 @@ static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 template <int DIM, typename T, bool RED>
 static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
+    if constexpr (sizeof(T) == 2) {
+        if (a.sr && !RED)                   // stochastic write-back: the dithers need registers
+            return run_hogwild_b<DIM, T, false, 4, 3, false, true>(a, st);
+    }
     if constexpr (std::is_same<T, __nv_bfloat16>::value)   // 6 blocks would spill; 5 blocks of 96 registers
         return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL > 8 ? 4 : 5), 3>(a, st);
     else if constexpr (sizeof(T) == 2)       // half rows: 3 rows per group in flight, 6 blocks (measured)
@@ -1666,6 +1794,15 @@ static gs_status sync_update(const SgnsArgs &a, int set, const FixedScratch *fix
         ms_in = MomState{ mom->m_in, mom->last_in, mom->mu, mom->iter + 1 };
         ms_out = MomState{ mom->m_out, mom->last_out, mom->mu, mom->iter + 1 };
     }
+    if (a.sr) {
+        for (MomState *ms : { &ms_in, &ms_out }) {
+            ms->sr = 1;
+            ms->sr_table = ms == &ms_out ? 1u : 0u;
+            ms->sr_step = (uint32_t)((uint64_t)a.walk_id_base & 0xFFFFFFFFu);
+            ms->sr_sub = (uint32_t)(((uint64_t)a.walk_id_base >> 32) & 0xFFFFFFu);
+            ms->sr_seed = a.seed;
+        }
+    }
     SyncScratch sc;
     gs_status s = sync_scratch(a, set, fixed, &sc);
     if (s != GS_OK) return s;
@@ -1764,8 +1901,13 @@ static gs_status step_on_tables(void *w_in, void *w_out, int64_t n_nodes, int32_
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter() };
-    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK);
+                   seed, loss, pairs, dump_pairs, dump_negs, pair_flags_of(mode), masked, prepared, refused_counter(),
+                   (mode & GS_ROUND_STOCHASTIC) ? 1 : 0 };
+    if (a.sr && sizeof(T) != 2) {
+        set_error("GS_ROUND_STOCHASTIC applies to 16-bit tables");
+        return GS_ERR_UNSUPPORTED;
+    }
+    mode &= ~(GS_PAIRS_FORWARD_ONLY | GS_WINDOW_SHRINK | GS_ROUND_STOCHASTIC);
     switch (dim) {
         case 32:
             if constexpr (sizeof(T) == 4) return run_mode<32, T>(a, mode, st);
@@ -1819,7 +1961,7 @@ gs_status sgns_step_momentum(float *w_in, float *w_out, float *m_in, float *m_ou
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, nullptr, nullptr, 0, nullptr, prepared, refused_counter() };
+                   seed, loss, pairs, nullptr, nullptr, 0, nullptr, prepared, refused_counter(), 0 };
     MomHost mom = { m_in, m_out, last_in, last_out, mu, iter, nullptr, nullptr, 0.f, 0.f, 0 };
     switch (dim) {
         case 32: return run_deterministic<32, float>(a, st, &mom);
@@ -1841,7 +1983,7 @@ gs_status sgns_step_adam(float *w_in, float *w_out, float *m_in, float *v_in, fl
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { w_in, w_out, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, lr,
-                   seed, loss, pairs, nullptr, nullptr, pair_flags_of(pair_mode), nullptr, prepared, refused_counter() };
+                   seed, loss, pairs, nullptr, nullptr, pair_flags_of(pair_mode), nullptr, prepared, refused_counter(), 0 };
     MomHost mom = { m_in, m_out, nullptr, nullptr, b1, 0, v_in, v_out, b2, eps, step };
     switch (dim) {
         case 32: return run_deterministic<32, float>(a, st, &mom);
@@ -1864,7 +2006,7 @@ gs_status sgns_prepare_sync(int64_t n_nodes, int32_t dim, const int32_t *walks, 
 {
     if (n_walks == 0) return GS_OK;
     SgnsArgs a = { nullptr, nullptr, n_nodes, dim, walks, n_walks, walk_id_base, L, w, K, alias, 0.f,
-                   seed, nullptr, nullptr, nullptr, nullptr, pair_flags_of(pair_mode), nullptr, -1, nullptr };
+                   seed, nullptr, nullptr, nullptr, nullptr, pair_flags_of(pair_mode), nullptr, -1, nullptr, 0 };
     return sync_prepare(a, set, nullptr, st);
 }
 
@@ -1943,7 +2085,7 @@ extern "C" gs_status gs_sgns_step_static(float *d_w_in, float *d_w_out, int64_t 
     if (s != GS_OK) return s;
     SgnsArgs a = { d_w_in, d_w_out, n_nodes, dim, d_walks, n_walks, walk_id_base, walk_len, window,
                    n_neg, d_alias, lr, seed, d_loss_sum, d_pair_count, nullptr, nullptr, 0, nullptr, -1,
-                   nullptr /* this entry point touches no library-owned memory but its array */ };
+                   nullptr /* this entry point touches no library-owned memory but its array */, 0 };
     cudaStream_t st = (cudaStream_t)stream;
     const FixedScratch fixed = { scratch, (size_t)GS_STATIC_SCRATCH_BYTES };
     switch (dim) {

@@ -70,9 +70,11 @@ def parse_args():
     ap.add_argument("--no-edge-set", action="store_true",
                     help="node2vec: membership in adj(prev) by binary search instead of the hashed edge set")
     ap.add_argument("--n2v-lanes", type=int, default=None,
-                    help="node2vec kernel: 0 flattened loop, 1 nested loops, 2..32 lanes per walk")
+                    help="node2vec kernel: 0 one lane per walk, flattened loop (default); 1, 2, 4, 8, 32: the "
+                         "generic kernel with that many lanes per walk")
     ap.add_argument("--stage", default="all", choices=["all", "walks"],
-                    help="'walks' times the walk sampler alone (no tables are allocated)")
+                    help="'walks' times the walk sampler alone (no tables are allocated); 'row-updates' measures "
+                         "the device's ceiling for random row read-modify-write (no workload is built)")
     ap.add_argument("--no-per-config", action="store_true",
                     help="skip the short legs over the other workloads that the default run adds")
     ap.add_argument("--cpu-workers", type=int, default=0,
@@ -371,6 +373,52 @@ def probe_random_reads(n_records, n_reads, dev):
     if rc != 0 or ms.value <= 0:
         return None
     return done.value / (ms.value * 1e-3)
+
+
+def run_row_update_probe(args):
+    """The ceiling of the update kernels' access pattern, measured with the benchmark's own probe
+    library: rows of 256 bytes (dim 128 in a 16-bit format) and 512 bytes (dim 128 in fp32) of a 4 GB
+    table visited at random, each read and written back, nothing computed.  One JSON line."""
+    import ctypes
+    import torch
+    so = ROOT / "libbench_probe.so"
+    if not so.exists():
+        raise SystemExit("libbench_probe.so is missing: run python -m paper_2407_15452_b200.build")
+    lib = ctypes.CDLL(str(so))
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    table_bytes, n_visits = 4 << 30, 1 << 23
+    table = torch.zeros(table_bytes // 4, dtype=torch.int32, device=dev)
+    peak, peak_kind = measured_peak_gbs()
+    rows_out = []
+    for row_bytes in (256, 512):
+        n_rows = table_bytes // row_bytes
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(12345)
+        ids = torch.randint(0, n_rows, (n_visits,), dtype=torch.int32, device=dev, generator=gen)
+        for write in (0, 1):
+            best = None
+            for in_flight in (3, 6):
+                for bps in (4, 8, 16):
+                    ms = ctypes.c_float(0.0)
+                    rc = lib.bench_probe_row_updates(
+                        ctypes.c_void_p(table.data_ptr()), ctypes.c_int64(n_rows), ctypes.c_int32(row_bytes),
+                        ctypes.c_void_p(ids.data_ptr()), ctypes.c_int64(n_visits), ctypes.c_int32(in_flight),
+                        ctypes.c_int32(bps), ctypes.c_int32(write), ctypes.byref(ms),
+                        ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+                    if rc != 0 or ms.value <= 0:
+                        raise SystemExit(f"bench_probe_row_updates failed with CUDA error {rc}")
+                    gbs = n_visits * row_bytes * (2 if write else 1) / (ms.value * 1e-3) / 1e9
+                    if best is None or gbs > best["gbs"]:
+                        best = {"row_bytes": row_bytes, "write_back": bool(write), "gbs": gbs,
+                                "rows_per_s": n_visits / (ms.value * 1e-3), "accesses_in_flight": in_flight,
+                                "blocks_per_sm": bps, "frac_of_copy_rate": gbs / peak}
+            rows_out.append(best)
+    print(json.dumps({"metric": "row_update_ceiling", "unit": "GB/s", "n_gpus": 1, "data": "synthetic",
+                      "config": {"stage": "row-updates", "table_bytes": table_bytes, "visits": n_visits,
+                                 "note": "best over 3 or 6 accesses in flight per warp and 4, 8, 16 blocks of "
+                                         "4 warps per SM; one warm-up and one timed launch each"},
+                      "peak": peak, "peak_kind": f"of {peak_kind}", "results": rows_out}))
 
 
 # ---------------------------------------------------------------------------- walk sampler alone
@@ -803,6 +851,8 @@ def main():
     args = parse_args()
     from paper_2407_15452_b200.workloads import WORKLOADS
     wl = WORKLOADS[args.workload]
+    if args.stage == "row-updates" and args.impl != "reference":
+        return run_row_update_probe(args)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

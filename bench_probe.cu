@@ -10,6 +10,19 @@
 // d_records: device buffer of n_records 16-byte records (contents do not matter).  n_reads is
 // rounded up to a multiple of 65,536 (*h_reads_done).  The kernel runs twice; the second run is
 // timed with events on `stream` (*h_ms_out).  Waits for completion.  Returns 0, or a cudaError_t.
+//
+// A second probe gives the ceiling of the update kernels' access pattern: rows of 256 or 512
+// bytes of a table, visited at random, each read and written back (16 bytes per lane, the rows of
+// a warp's chunk in flight together), with nothing computed in between.
+//
+//   int bench_probe_row_updates(void *d_table, int64_t n_rows, int32_t row_bytes, const int32_t *d_ids,
+//                               int64_t n_visits, int32_t rows_in_flight, int32_t blocks_per_sm,
+//                               int32_t write_back, float *h_ms_out, void *stream)
+//
+// d_table: n_rows rows of row_bytes (256 or 512) bytes, 16-byte aligned; its contents change when
+// write_back != 0.  d_ids: n_visits row ids in [0, n_rows) (checked on the device: others are
+// skipped).  rows_in_flight: 3 or 6 accesses of a warp in flight (6 or 12 rows of 256 bytes, 3 or
+// 6 of 512).  One warm-up launch, one timed one.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -44,7 +57,81 @@ random_read_kernel(const int4 *__restrict__ rec, uint64_t n_rec, int iters, unsi
     if (acc == 0x7fffffff) atomicAdd(sink, 1ull);           // keeps the loads alive
 }
 
+// LPR lanes per row (16 bytes per lane), G accesses in flight per warp: G * 32 / LPR rows
+template <int LPR, int G>
+__global__ void __launch_bounds__(128)
+row_update_kernel(uint4 *tab, int64_t n_rows, const int32_t *__restrict__ ids, int64_t n, int write_back,
+                  unsigned long long *sink)
+{
+    constexpr int NG = 32 / LPR, CH = G * NG;
+    const int lane = threadIdx.x & 31, grp = lane / LPR, sub = lane % LPR;
+    const int64_t warp = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5), nw = (int64_t)gridDim.x * 4;
+    uint32_t acc = 0;
+    for (int64_t i = warp * CH; i < n; i += nw * CH) {
+        uint4 r[G];
+        int64_t id[G];
+#pragma unroll
+        for (int q = 0; q < G; ++q) {
+            const int64_t e = i + q * NG + grp;
+            id[q] = e < n ? (int64_t)ids[e] : -1;
+            if (id[q] >= n_rows) id[q] = -1;
+        }
+#pragma unroll
+        for (int q = 0; q < G; ++q)
+            if (id[q] >= 0) r[q] = tab[id[q] * LPR + sub];
+#pragma unroll
+        for (int q = 0; q < G; ++q)
+            if (id[q] >= 0) {
+                acc += r[q].x;
+                if (write_back) { r[q].x += 1u; r[q].y ^= 3u; tab[id[q] * LPR + sub] = r[q]; }
+            }
+    }
+    if (acc == 0x7fffffffu) atomicAdd(sink, 1ull);           // keeps the loads alive
+}
+
 }  // namespace
+
+extern "C" __attribute__((visibility("default")))
+int bench_probe_row_updates(void *d_table, int64_t n_rows, int32_t row_bytes, const int32_t *d_ids,
+                            int64_t n_visits, int32_t rows_in_flight, int32_t blocks_per_sm,
+                            int32_t write_back, float *h_ms_out, void *stream)
+{
+    if (!d_table || !d_ids || !h_ms_out || n_rows < 1 || n_visits < 1 || ((uintptr_t)d_table & 15) ||
+        (row_bytes != 256 && row_bytes != 512) || (rows_in_flight != 3 && rows_in_flight != 6) ||
+        blocks_per_sm < 1 || blocks_per_sm > 16)
+        return (int)cudaErrorInvalidValue;
+    cudaStream_t st = (cudaStream_t)stream;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return (int)e;
+    unsigned long long *sink = nullptr;
+    e = cudaMalloc(&sink, sizeof(*sink));
+    if (e != cudaSuccess) return (int)e;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    e = cudaMemsetAsync(sink, 0, sizeof(*sink), st);
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    if (e == cudaSuccess) {
+        const unsigned blocks = (unsigned)(sms * blocks_per_sm);
+        for (int run = 0; run < 2; ++run) {
+            if (run == 1) cudaEventRecord(e0, st);
+            uint4 *t = (uint4 *)d_table;
+            if (row_bytes == 256 && rows_in_flight == 3) row_update_kernel<16, 3><<<blocks, 128, 0, st>>>(t, n_rows, d_ids, n_visits, write_back, sink);
+            else if (row_bytes == 256) row_update_kernel<16, 6><<<blocks, 128, 0, st>>>(t, n_rows, d_ids, n_visits, write_back, sink);
+            else if (rows_in_flight == 3) row_update_kernel<32, 3><<<blocks, 128, 0, st>>>(t, n_rows, d_ids, n_visits, write_back, sink);
+            else row_update_kernel<32, 6><<<blocks, 128, 0, st>>>(t, n_rows, d_ids, n_visits, write_back, sink);
+        }
+        cudaEventRecord(e1, st);
+        e = cudaEventSynchronize(e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(h_ms_out, e0, e1);
+        if (e == cudaSuccess) e = cudaGetLastError();
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(sink);
+    return (int)e;
+}
 
 extern "C" __attribute__((visibility("default")))
 int bench_probe_random_reads(const void *d_records, int64_t n_records, int64_t n_reads,

@@ -36,6 +36,8 @@ int radix_sort_pairs(const uint32_t *keys_src, uint32_t *keysB, uint32_t *valsB,
                      uint32_t **keys_sorted, uint32_t **vals_sorted);
 size_t sort_counts_bytes(uint32_t n);
 
+constexpr bool HOGWILD_PREFETCH = true;
+constexpr int HOGWILD_PF_DIST = 2;   // chunks between a prefetch and the loads that use it
 constexpr int TCH = 6;            // target rows in flight per row group (3 for half rows, see run_hogwild)
 constexpr int SGNS_WARPS = 4;     // warps per block
 
@@ -186,28 +188,6 @@ __device__ __forceinline__ void sigmoid_softplus(float z, float &sig, float &sp)
     sp = fmaxf(z, 0.f) + log1pf(e);
 }
 
-// The dot products f[0..TCH) of a chunk are known to every lane.  Lane k < TCH evaluates the
-// transcendentals of target k only (the other lanes idle through those few instructions):
-// for a context (label 1) the term is softplus(-f) and g = sigmoid(f) - 1 = -sigmoid(-f); for a
-// negative softplus(f) and g = sigmoid(f).  Returns this lane's g (0 for an absent target) and
-// adds its loss term to `loss`.
-template <int N>
-__device__ __forceinline__ float lane_coefficient(const float (&f)[N], int lane, int32_t my_id,
-                                                  bool my_is_ctx, float &loss)
-{
-    float mf = f[0];
-#pragma unroll
-    for (int k = 1; k < N; ++k) mf = lane == k ? f[k] : mf;
-    float g = 0.f;
-    if (lane < N && my_id >= 0) {
-        float sig, sp;
-        sigmoid_softplus(my_is_ctx ? -mf : mf, sig, sp);
-        g = my_is_ctx ? -sig : sig;
-        loss += sp;
-    }
-    return g;
-}
-
 __device__ __forceinline__ double warp_sum_double(double s)
 {
 #pragma unroll
@@ -310,33 +290,31 @@ __device__ __forceinline__ void grow_store(T *__restrict__ tab, int64_t r, int s
 // with probability (|x| - lo) / (hi - lo) taken to 16 bits: up iff the 16-bit dither is below
 // floor(frac * 2^16).  Representable values never move; nothing becomes infinite (a magnitude
 // beyond the largest finite value, or a step up from it, gives the largest finite value).
+// Both formats use the same carry: with frac held as an integer in the low bits of a word whose upper
+// bits are the neighbour towards zero, "dither < frac" is the carry of frac + (all ones - dither)
+// into the upper bits, so one addition both decides and rounds (a carry into the exponent is the
+// step to the next binade).  The value is clamped to the largest finite value first.
 __device__ __forceinline__ uint32_t sr_bits(float x, uint32_t u16, const __nv_bfloat16 *)
 {
     // bfloat16 is the upper half of the fp32 pattern: the dropped 16 bits ARE frac * 2^16
-    const uint32_t bits = __float_as_uint(x);
-    uint32_t r = (bits >> 16) + (u16 < (bits & 0xFFFFu) ? 1u : 0u);
-    if ((r & 0x7FFFu) >= 0x7F80u) r = (r & 0x8000u) | 0x7F7Fu;
-    return r;
+    const float big = __uint_as_float(0x7F7F0000u);                 // largest finite bfloat16
+    const uint32_t bits = __float_as_uint(fminf(fmaxf(x, -big), big));
+    return (bits + (u16 ^ 0xFFFFu)) >> 16;
 }
 __device__ __forceinline__ uint32_t sr_bits(float x, uint32_t u16, const __half *)
 {
-    const float ax = fabsf(x);
+    const float ax = fminf(fabsf(x), 65504.0f);
     const uint32_t abits = __float_as_uint(ax);
     const uint32_t sign = (__float_as_uint(x) >> 16) & 0x8000u;
-    if (abits >= 0x38800000u && abits < 0x477FE000u) {
-        // normal range of binary16 (2^-14 <= |x| < 65504): 13 fraction bits are dropped, so they
-        // are frac * 2^13; the upper bits, with the exponent re-biased, are the neighbour towards zero
-        uint32_t h = (abits >> 13) - 0x1C000u;
-        h += u16 < ((abits & 0x1FFFu) << 3) ? 1u : 0u;
-        return sign | (h >= 0x7C00u ? 0x7BFFu : h);
-    }
-    if (!(ax < 65504.0f)) return sign | 0x7BFFu;
-    const __half lo_h = __float2half_rz(ax);                       // neighbour towards zero
-    const uint32_t lb = __half_as_ushort(lo_h);
-    const float lo = __half2float(lo_h);
-    const float hi = __half2float(__ushort_as_half((unsigned short)(lb + 1u)));
-    const float frac = (ax - lo) * __frcp_rn(hi - lo);             // both exact: hi - lo is a power of two
-    return sign | (lb + (u16 < (uint32_t)(frac * 65536.0f) ? 1u : 0u));
+    // normal range of binary16 (|x| >= 2^-14): 13 fraction bits are dropped, so they are
+    // frac * 2^13 and the dither's upper 13 bits decide; the upper bits, exponent re-biased, are the
+    // neighbour towards zero
+    const uint32_t h_normal = ((abits + ((u16 >> 3) ^ 0x1FFFu)) >> 13) - 0x1C000u;
+    // below 2^-14 the spacing is 2^-24: |x| * 2^40, truncated, holds the neighbour in its upper
+    // and frac * 2^16 in its lower 16 bits (the product is exact)
+    const uint32_t fixed = __float2uint_rz(ax * 1099511627776.0f);
+    const uint32_t h_small = (fixed + (u16 ^ 0xFFFFu)) >> 16;
+    return sign | (abits >= 0x38800000u ? h_normal : h_small);
 }
 
 __device__ __forceinline__ uint32_t mix32(uint32_t h)
@@ -442,13 +420,66 @@ template <int DIM, bool NARROW>
 __device__ __forceinline__ void grow_red_add(__nv_bfloat16 *, int64_t, int,
                                              const Row<RowGeom<DIM, __nv_bfloat16, NARROW>::FPL> &) {}
 
-// sum over the LPR lanes that hold one row (identical bits on each of them)
-template <int LPR>
-__device__ __forceinline__ float group_sum(float s)
+// Sums of N values over the LPR lanes of a row group in about half the shuffles of N separate
+// butterflies.  While more than one value is left, a step pairs the values up and a lane keeps,
+// of each pair, the one its lane bit selects (odd index: bit set) and sends the other; a value
+// without a partner is added the plain way.  In the end every lane holds the complete sum of ONE
+// value, f[0]: lane `sub` that of value group_value<LPR, N>(sub).  Value k is complete on lane
+// group_owner<LPR, N>(k) and on the lanes that differ from it in bits no pairing of k used.
+template <int O, int CNT, int N>
+__device__ __forceinline__ void group_reduce_step(float (&f)[N], int sub)
 {
+    if constexpr (O >= 1) {
+        if constexpr (CNT > 1) {
+            const bool up = (sub & O) != 0;
 #pragma unroll
-    for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    return s;
+            for (int i = 0; i < CNT / 2; ++i) {
+                const float send = up ? f[2 * i] : f[2 * i + 1];
+                const float keep = up ? f[2 * i + 1] : f[2 * i];
+                f[i] = keep + __shfl_xor_sync(0xffffffffu, send, O);
+            }
+            if constexpr ((CNT & 1) != 0)
+                f[CNT / 2] = f[CNT - 1] + __shfl_xor_sync(0xffffffffu, f[CNT - 1], O);
+        } else {
+            f[0] += __shfl_xor_sync(0xffffffffu, f[0], O);
+        }
+        group_reduce_step<O / 2, (CNT + 1) / 2, N>(f, sub);
+    }
+}
+
+template <int LPR, int N>
+__device__ __forceinline__ float group_reduce(float (&f)[N], int sub)
+{
+    static_assert(N <= LPR, "a row group sums at most as many values as it has lanes");
+    group_reduce_step<LPR / 2, N, N>(f, sub);
+    return f[0];
+}
+
+// lane bits that the pairings on the way of value k used (mask) and their values on the lanes
+// that end up with value k (owner)
+template <int LPR, int N>
+__host__ __device__ constexpr int group_owner(int k, bool want_mask = false)
+{
+    int own = 0, mask = 0, cnt = N, slot = k;
+    for (int o = LPR / 2; o >= 1 && cnt > 1; o >>= 1) {
+        if ((slot | 1) < cnt) {                      // this value has a partner at this step
+            mask |= o;
+            if (slot & 1) own |= o;
+        }
+        slot >>= 1;
+        cnt = (cnt + 1) / 2;
+    }
+    return want_mask ? mask : own;
+}
+
+template <int LPR, int N>
+__device__ __forceinline__ int group_value(int sub)
+{
+    int k = 0;
+#pragma unroll
+    for (int q = 1; q < N; ++q)
+        if ((sub & group_owner<LPR, N>(q, true)) == group_owner<LPR, N>(q)) k = q;
+    return k;
 }
 
 // add up the per-group copies of a row held by the NG = 32 / LPR groups of a warp
@@ -460,6 +491,11 @@ __device__ __forceinline__ void sum_over_groups(Row<FPL> &x)
 #pragma unroll
         for (int j = 0; j < FPL; ++j) x.v[j] += __shfl_xor_sync(0xffffffffu, x.v[j], o);
     }
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *p)
+{
+    asm volatile("prefetch.global.L2 [%0];" :: "l"(p));
 }
 
 // ---------------------------------------------------------------- target list of one position
@@ -572,6 +608,10 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     using G = RowGeom<DIM, T, NARROW>;
     constexpr int FPL = G::FPL, LPR = G::LPR, NG = G::NG;
     constexpr int CH = TC * NG;                          // targets per chunk
+    // 16-bit tables: few bytes are in flight per warp (CH rows of 128 to 512 bytes), so the rows of
+    // a later chunk are asked into L2 ahead of time, one 128-byte line per lane
+    constexpr int LINES = G::BYTES >= 128 ? G::BYTES / 128 : 1;
+    constexpr int PF_LINES = (sizeof(T) == 2 && HOGWILD_PREFETCH && CH * LINES <= 32) ? CH * LINES : 0;
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int grp = lane / LPR, sub = lane % LPR;
@@ -581,6 +621,11 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     // walks, up to 16 when walks are short (LINE: two nodes), so that the round trips of the
     // ticket and of the walk entries are paid once per 32 entries and not once per pair.
     const int wpt = hogwild_walks_per_ticket(L);
+    // of every chunk this lane evaluates target my_k of its group, list entry base + my_off; the
+    // lanes that hold the same sum evaluate it too, and one of them (my_owner) counts its loss
+    const int my_k = group_value<LPR, TC>(sub);
+    const int my_off = my_k * NG + grp;
+    const bool my_owner = sub == (sub & group_owner<LPR, TC>(my_k, true));
     int32_t *Wbuf = smem + wi * (wpt * L + SL);
     int32_t *tgt = Wbuf + wpt * L;
     double loss_acc = 0.0;
@@ -623,8 +668,23 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             Row<FPL> acc;                                        // this group's share of its gradient
 #pragma unroll
             for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
-            float loss = 0.f;                            // this lane's share of the position's loss
-            int kk = 0;                                  // base mod T1, tracked incrementally
+            // The loss term of a target is softplus(z) = max(z, 0) + log(1 + e^-|z|) with z = -f for
+            // a context and f for a negative.  A lane adds up the first part and multiplies the
+            // second parts (each in [1, 2]); the logarithm is taken once per position.
+            float sp_lin = 0.f, sp_prod = 1.f;
+            int my_kt = my_off;                          // (list index of this lane's target) mod (1 + K)
+            while (my_kt >= T1) my_kt -= T1;
+            // the rows of a later chunk on their way into L2 while the ones before it are worked
+            // on: lane l asks for line l of the chunk's CH rows
+            auto prefetch_chunk = [&](int first) {
+                const int e = first + lane / LINES;
+                const int32_t idn = lane < PF_LINES && e < SL ? tgt[e] : -1;
+                if (idn >= 0) prefetch_l2((const char *)(w_out + (int64_t)idn * DIM) + (lane % LINES) * 128);
+            };
+            if constexpr (PF_LINES > 0) {
+#pragma unroll
+                for (int d = 1; d < HOGWILD_PF_DIST; ++d) prefetch_chunk(d * CH);
+            }
             for (int base = 0; base < SL; base += CH) {
                 // target k of group grp is list entry base + k * NG + grp
                 int32_t ids[TC];
@@ -641,20 +701,27 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
 #pragma unroll
                     for (int k = 0; k < TC; ++k)
                         if (ids[k] >= 0) rows[k] = grow_load<DIM, T, NARROW>(w_out, ids[k], sub);
+                    if constexpr (PF_LINES > 0) prefetch_chunk(base + HOGWILD_PF_DIST * CH);
 #pragma unroll
                     for (int k = 0; k < TC; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
-#pragma unroll
-                    for (int k = 0; k < TC; ++k) f[k] = group_sum<LPR>(f[k]);
-                    // lane `sub` of a group evaluates the group's target `sub`
-                    const int my_t = base + sub * NG + grp;
-                    const bool mine = sub < TC && my_t < SL;
-                    int my_kt = kk + (sub < TC ? sub * NG + grp : 0);
-                    while (my_kt >= T1) my_kt -= T1;
-                    const int32_t my_id = mine ? tgt[my_t] : -1;
-                    const float my_g = lane_coefficient<TC>(f, sub, my_id, my_kt == 0, loss);
+                    // the dot products of the chunk, reduced together: this lane ends up with
+                    // that of target my_k of its group and evaluates its coefficient.  For a
+                    // context (label 1) g = sigmoid(f) - 1 = -sigmoid(-f), for a negative sigmoid(f).
+                    const float fs = group_reduce<LPR, TC>(f, sub);
+                    const bool ctx = my_kt == 0;
+                    const float z = ctx ? -fs : fs;
+                    const float e = __expf(-fabsf(z));
+                    const float r = __fdividef(1.0f, 1.0f + e);
+                    const float sig = z >= 0.f ? r : e * r;
+                    const float my_g = ctx ? -sig : sig;
+                    const int my_t = base + my_off;
+                    if (my_owner && my_t < SL && tgt[my_t] >= 0) {
+                        sp_lin += fmaxf(z, 0.f);
+                        sp_prod *= 1.0f + e;
+                    }
 #pragma unroll
                     for (int k = 0; k < TC; ++k) {
-                        const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + k);
+                        const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + group_owner<LPR, TC>(k));
                         if (ids[k] >= 0) {
                             const float step = -lr * g;
                             Row<FPL> delta;
@@ -671,10 +738,14 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
                             else grow_store<DIM, T, NARROW>(w_out, ids[k], sub, rows[k]);
                         }
                     }
+                    if (sp_prod > 1e30f) { sp_lin += logf(sp_prod); sp_prod = 1.f; }
+                } else if constexpr (PF_LINES > 0) {
+                    prefetch_chunk(base + HOGWILD_PF_DIST * CH);
                 }
-                kk += CH;
-                while (kk >= T1) kk -= T1;
+                my_kt += CH;
+                while (my_kt >= T1) my_kt -= T1;
             }
+            const float loss = sp_lin + logf(sp_prod);   // this lane's share of the position's loss
             // center row: add the accumulated increment to the row as it is now
             sum_over_groups<LPR, FPL>(acc);
             Row<FPL> delta;
@@ -790,11 +861,6 @@ __device__ __forceinline__ float reduce_rows(float (&v)[G], int lane)
     float s = v[0];
     for (; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
     return s;
-}
-
-__device__ __forceinline__ void prefetch_l2(const void *p)
-{
-    asm volatile("prefetch.global.L2 [%0];" :: "l"(p));
 }
 
 // Part B, coefficients: one warp per position, a whole warp per row (a lane holds DIM / 32
@@ -1628,12 +1694,10 @@ static gs_status run_hogwild(const SgnsArgs &a, cudaStream_t st)
 {
     if constexpr (sizeof(T) == 2) {
         if (a.sr && !RED)                   // stochastic write-back: the dithers need registers
-            return run_hogwild_b<DIM, T, false, 4, 3, false, true>(a, st);
+            return run_hogwild_b<DIM, T, false, 5, 3, false, true>(a, st);
     }
-    if constexpr (std::is_same<T, __nv_bfloat16>::value)   // 6 blocks would spill; 5 blocks of 96 registers
-        return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL > 8 ? 4 : 5), 3>(a, st);
-    else if constexpr (sizeof(T) == 2)       // half rows: 3 rows per group in flight, 6 blocks (measured)
-        return run_hogwild_b<DIM, T, RED, (RowGeom<DIM, T>::FPL > 8 ? 4 : 6), 3>(a, st);
+    if constexpr (sizeof(T) == 2)            // 16-bit rows: 3 rows per group in flight, 5 blocks of 96 registers
+        return run_hogwild_b<DIM, T, RED, 5, 3>(a, st);
     else {
         // few targets per position (fewer than two wide chunks): 16 bytes per lane, one chunk
         // of TCH rows per row group, so that chunks are full

@@ -72,7 +72,7 @@ def parse_args():
     ap.add_argument("--n2v-lanes", type=int, default=None,
                     help="node2vec kernel: 0 one lane per walk, flattened loop (default); 1, 2, 4, 8, 32: the "
                          "generic kernel with that many lanes per walk")
-    ap.add_argument("--stage", default="all", choices=["all", "walks"],
+    ap.add_argument("--stage", default="all", choices=["all", "walks", "row-updates"],
                     help="'walks' times the walk sampler alone (no tables are allocated); 'row-updates' measures "
                          "the device's ceiling for random row read-modify-write (no workload is built)")
     ap.add_argument("--no-per-config", action="store_true",

@@ -36,7 +36,6 @@ int radix_sort_pairs(const uint32_t *keys_src, uint32_t *keysB, uint32_t *valsB,
                      uint32_t **keys_sorted, uint32_t **vals_sorted);
 size_t sort_counts_bytes(uint32_t n);
 
-constexpr bool HOGWILD_PREFETCH = true;
 constexpr int HOGWILD_PF_DIST = 2;   // chunks between a prefetch and the loads that use it
 constexpr int TCH = 6;            // target rows in flight per row group (3 for half rows, see run_hogwild)
 constexpr int SGNS_WARPS = 4;     // warps per block
@@ -207,8 +206,8 @@ template <int DIM, typename T = float, bool NARROW = false> struct RowGeom {
     // lanes per row: 16 bytes per lane for half tables and for fp32 rows of 128 bytes; fp32 rows
     // of 256 and 512 bytes give a lane 32 bytes (8 and 16 lanes per row, 4 and 2 rows per
     // warp-wide access), which halves the per-row instruction overhead: measured +5 % on the
-    // dim-64 workload and +4 % / +10 % on the 50M-node / 1M-node dim-128 workloads.  Half rows
-    // of 256 bytes run 13 % slower that way (16 values per lane cost a resident block).
+    // dim-64 workload and +4 % / +10 % on the 50M-node / 1M-node dim-128 workloads.  16-bit rows
+    // of 256 bytes run 2 to 10 % slower that way (16 values per lane cost resident warps).
     // NARROW keeps 16 bytes per lane for those rows too: with few targets per position (LINE: one
     // pair per walk) wide chunks stay half empty and the narrow layout is 20 % faster.
     static constexpr int LPR = !NARROW && sizeof(T) == 4 && (BYTES == 256 || BYTES == 512)
@@ -381,23 +380,6 @@ __device__ __forceinline__ void row_store_sr(T *__restrict__ tab, int64_t r, int
             t.x = sr_pack2<T>(x.v[4 * q], x.v[4 * q + 1], ev, 0u, k0);
             t.y = sr_pack2<T>(x.v[4 * q + 2], x.v[4 * q + 3], ev, 0u, k0 + 1);
             reinterpret_cast<uint2 *>(p)[q * 32 + lane] = t;
-        }
-    }
-}
-
-// Stores a row held in the geometry of a T table into an fp32 scratch row (natural column order).
-template <int DIM, typename T>
-__device__ __forceinline__ void grow_store_f32(float *__restrict__ tab, int64_t r, int sub,
-                                               const Row<RowGeom<DIM, T>::FPL> &x)
-{
-    using G = RowGeom<DIM, T>;
-    float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
-#pragma unroll
-    for (int q = 0; q < G::FPL / G::PER16; ++q) {
-#pragma unroll
-        for (int e = 0; e < G::PER16 / 4; ++e) {
-            const float *v = x.v + G::PER16 * q + 4 * e;
-            p[(q * G::LPR + sub) * (G::PER16 / 4) + e] = make_float4(v[0], v[1], v[2], v[3]);
         }
     }
 }
@@ -611,7 +593,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     // 16-bit tables: few bytes are in flight per warp (CH rows of 128 to 512 bytes), so the rows of
     // a later chunk are asked into L2 ahead of time, one 128-byte line per lane
     constexpr int LINES = G::BYTES >= 128 ? G::BYTES / 128 : 1;
-    constexpr int PF_LINES = (sizeof(T) == 2 && HOGWILD_PREFETCH && CH * LINES <= 32) ? CH * LINES : 0;
+    constexpr int PF_LINES = (sizeof(T) == 2 && CH * LINES <= 32) ? CH * LINES : 0;
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int grp = lane / LPR, sub = lane % LPR;

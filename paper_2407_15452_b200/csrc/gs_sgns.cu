@@ -481,7 +481,8 @@ __device__ __forceinline__ void prefetch_l2(const void *p)
 }
 
 // ---------------------------------------------------------------- target list of one position
-// Slot layout: tgt[s * (1 + K) + 0] = context of slot s, tgt[s * (1 + K) + 1 + k] = negative k;
+// Slot layout: tgt[s * (1 + K) + 0] = context of slot s with bit 31 set (TARGET_IS_CONTEXT; node ids
+// stay below 2^31 - 1, so no entry collides with -1), tgt[s * (1 + K) + 1 + k] = negative k;
 // -1 where the pair does not exist or the negative equals the context (masked).
 // W points at the walk (global or shared), c = W[i] >= 0.  Returns, identical on every lane, the
 // number of pairs in bits 0..7, the number of masked negatives in bits 8..19 and, from bit 20, the
@@ -493,6 +494,7 @@ __device__ __forceinline__ void prefetch_l2(const void *p)
 // 1..w (word2vec's shrinking window), and keeps the contexts within w_i.  Slots and the keying
 // of the negatives stay those of the full window.
 enum { PAIR_FWD = 1, PAIR_SHRINK = 2 };
+constexpr uint32_t TARGET_IS_CONTEXT = 0x80000000u;
 
 __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_t i, int32_t w,
                                              int32_t K, uint64_t seed, uint64_t id,
@@ -522,7 +524,7 @@ __device__ __forceinline__ int build_targets(const int32_t *W, int32_t L, int32_
             }
             valid = ctx >= 0;
             if (m == 0) {
-                tgt[s * T1] = ctx;
+                tgt[s * T1] = valid ? (int32_t)((uint32_t)ctx | TARGET_IS_CONTEXT) : -1;
                 if (dump_pairs) {
                     dump_pairs[2 * s] = valid ? c : -1;
                     dump_pairs[2 * s + 1] = ctx;
@@ -573,6 +575,30 @@ __device__ __forceinline__ void dump_empty_position(int32_t S, int32_t K, int la
     if (dump_negs) for (int x = lane; x < S * K; x += 32) dump_negs[x] = -1;
 }
 
+// Closes the gaps of a target list in place, keeping the order: afterwards tgt[0 .. n) are the
+// entries other than -1 (returned: n, identical on every lane).  orig (nullable) receives the
+// index each kept entry had in the slot layout.
+__device__ __forceinline__ int compact_targets(int32_t *tgt, int SL, int lane, int32_t *orig)
+{
+    const unsigned below = (1u << lane) - 1u;
+    int n = 0;
+    for (int x0 = 0; x0 < SL; x0 += 32) {
+        const int x = x0 + lane;
+        const int32_t v = x < SL ? tgt[x] : -1;
+        // every lane has read its entry before any lane writes: the ballot needs all of them, and
+        // the writes go to places at or below the ones just read
+        const unsigned m = __ballot_sync(0xffffffffu, v != -1);
+        if (v != -1) {
+            const int at = n + __popc(m & below);
+            tgt[at] = v;
+            if (orig) orig[at] = x;
+        }
+        n += __popc(m);
+    }
+    __syncwarp();
+    return n;
+}
+
 // ---------------------------------------------------------------- lock-free kernel
 // walks covered by one ticket of the lock-free kernel (host and device agree on the buffer size)
 __host__ __device__ __forceinline__ int hogwild_walks_per_ticket(int L) { return L <= 16 ? 32 / L : 1; }
@@ -597,7 +623,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     extern __shared__ int32_t smem[];
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int grp = lane / LPR, sub = lane % LPR;
-    const int S = 2 * w, T1 = 1 + K, SL = S * T1;
+    const int S = 2 * w, SL = S * (1 + K);
     // Walks differ in length (dead ends), so warps draw walks from a shared ticket counter
     // instead of taking a fixed share.  A ticket covers `wpt` consecutive walks: one for ordinary
     // walks, up to 16 when walks are short (LINE: two nodes), so that the round trips of the
@@ -608,7 +634,7 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
     const int my_k = group_value<LPR, TC>(sub);
     const int my_off = my_k * NG + grp;
     const bool my_owner = sub == (sub & group_owner<LPR, TC>(my_k, true));
-    int32_t *Wbuf = smem + wi * (wpt * L + SL);
+    int32_t *Wbuf = smem + wi * (wpt * L + (SR ? 2 : 1) * SL);   // SR: + the slot index of every list entry
     int32_t *tgt = Wbuf + wpt * L;
     double loss_acc = 0.0;
     unsigned long long pair_acc = 0, masked_acc = 0, refused_acc = 0;
@@ -642,8 +668,10 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             refused_acc += (unsigned long long)((unsigned)packed >> 20);
             if (pairs == 0) continue;
             pair_acc += (unsigned long long)pairs;
+            // the list without its gaps: chunks are full but for the last one
+            const int n_tgt = compact_targets(tgt, SL, lane, SR ? tgt + SL : nullptr);
             // stochastic write-back: the rows written while this position is worked on share one
-            // Philox block; a target takes salt 1 + its index in the list, the center row 0x10000
+            // Philox block; a target takes salt 1 + its index in the slot layout, the center row 0x10000
             uint4 ev = make_uint4(0u, 0u, 0u, 0u);
             if (SR) ev = draw(seed, id, (uint32_t)i, TAG_ROUND_LOCKFREE, 0);
             const Row<FPL> u = grow_load<DIM, T, NARROW>(w_in, c, sub);     // every group holds the center row
@@ -654,78 +682,73 @@ sgns_hogwild_kernel(T *__restrict__ w_in, T *__restrict__ w_out,
             // a context and f for a negative.  A lane adds up the first part and multiplies the
             // second parts (each in [1, 2]); the logarithm is taken once per position.
             float sp_lin = 0.f, sp_prod = 1.f;
-            int my_kt = my_off;                          // (list index of this lane's target) mod (1 + K)
-            while (my_kt >= T1) my_kt -= T1;
             // the rows of a later chunk on their way into L2 while the ones before it are worked
             // on: lane l asks for line l of the chunk's CH rows
             auto prefetch_chunk = [&](int first) {
                 const int e = first + lane / LINES;
-                const int32_t idn = lane < PF_LINES && e < SL ? tgt[e] : -1;
-                if (idn >= 0) prefetch_l2((const char *)(w_out + (int64_t)idn * DIM) + (lane % LINES) * 128);
+                if (lane < PF_LINES && e < n_tgt) {
+                    const int64_t idn = (int64_t)((uint32_t)tgt[e] & ~TARGET_IS_CONTEXT);
+                    prefetch_l2((const char *)(w_out + idn * DIM) + (lane % LINES) * 128);
+                }
             };
             if constexpr (PF_LINES > 0) {
 #pragma unroll
                 for (int d = 1; d < HOGWILD_PF_DIST; ++d) prefetch_chunk(d * CH);
             }
-            for (int base = 0; base < SL; base += CH) {
-                // target k of group grp is list entry base + k * NG + grp
+            for (int base = 0; base < n_tgt; base += CH) {
+                // target k of group grp is list entry base + k * NG + grp (-1: past the end)
                 int32_t ids[TC];
-                bool any = false;
 #pragma unroll
                 for (int k = 0; k < TC; ++k) {
                     const int t = base + k * NG + grp;
-                    ids[k] = t < SL ? tgt[t] : -1;
-                    any |= ids[k] >= 0;
+                    ids[k] = t < n_tgt ? tgt[t] : -1;
                 }
-                if (__any_sync(0xffffffffu, any)) {
-                    Row<FPL> rows[TC];
-                    float f[TC];
+                Row<FPL> rows[TC];
+                float f[TC];
 #pragma unroll
-                    for (int k = 0; k < TC; ++k)
-                        if (ids[k] >= 0) rows[k] = grow_load<DIM, T, NARROW>(w_out, ids[k], sub);
-                    if constexpr (PF_LINES > 0) prefetch_chunk(base + HOGWILD_PF_DIST * CH);
+                for (int k = 0; k < TC; ++k)
+                    if (ids[k] != -1)
+                        rows[k] = grow_load<DIM, T, NARROW>(w_out, (int64_t)((uint32_t)ids[k] & ~TARGET_IS_CONTEXT), sub);
+                if constexpr (PF_LINES > 0) prefetch_chunk(base + HOGWILD_PF_DIST * CH);
 #pragma unroll
-                    for (int k = 0; k < TC; ++k) f[k] = ids[k] >= 0 ? row_dot<FPL>(u, rows[k]) : 0.f;
-                    // the dot products of the chunk, reduced together: this lane ends up with
-                    // that of target my_k of its group and evaluates its coefficient.  For a
-                    // context (label 1) g = sigmoid(f) - 1 = -sigmoid(-f), for a negative sigmoid(f).
-                    const float fs = group_reduce<LPR, TC>(f, sub);
-                    const bool ctx = my_kt == 0;
-                    const float z = ctx ? -fs : fs;
-                    const float e = __expf(-fabsf(z));
-                    const float r = __fdividef(1.0f, 1.0f + e);
-                    const float sig = z >= 0.f ? r : e * r;
-                    const float my_g = ctx ? -sig : sig;
-                    const int my_t = base + my_off;
-                    if (my_owner && my_t < SL && tgt[my_t] >= 0) {
-                        sp_lin += fmaxf(z, 0.f);
-                        sp_prod *= 1.0f + e;
-                    }
+                for (int k = 0; k < TC; ++k) f[k] = ids[k] != -1 ? row_dot<FPL>(u, rows[k]) : 0.f;
+                // the dot products of the chunk, reduced together: this lane ends up with that of
+                // target my_k of its group and evaluates its coefficient.  For a context
+                // (label 1) g = sigmoid(f) - 1 = -sigmoid(-f), for a negative sigmoid(f).
+                const float fs = group_reduce<LPR, TC>(f, sub);
+                const int my_t = base + my_off;
+                const int32_t my_e = my_t < n_tgt ? tgt[my_t] : -1;
+                const bool ctx = my_e < 0;               // bit 31 (an absent entry's g is not used)
+                const float z = ctx ? -fs : fs;
+                const float e = __expf(-fabsf(z));
+                const float r = __fdividef(1.0f, 1.0f + e);
+                const float sig = z >= 0.f ? r : e * r;
+                const float my_g = ctx ? -sig : sig;
+                if (my_owner && my_e != -1) {
+                    sp_lin += fmaxf(z, 0.f);
+                    sp_prod *= 1.0f + e;
+                }
 #pragma unroll
-                    for (int k = 0; k < TC; ++k) {
-                        const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + group_owner<LPR, TC>(k));
-                        if (ids[k] >= 0) {
-                            const float step = -lr * g;
-                            Row<FPL> delta;
+                for (int k = 0; k < TC; ++k) {
+                    const float g = __shfl_sync(0xffffffffu, my_g, grp * LPR + group_owner<LPR, TC>(k));
+                    if (ids[k] != -1) {
+                        const int64_t row = (int64_t)((uint32_t)ids[k] & ~TARGET_IS_CONTEXT);
+                        const float step = -lr * g;
+                        Row<FPL> delta;
 #pragma unroll
-                            for (int j = 0; j < FPL; ++j) {
-                                acc.v[j] = fmaf(g, rows[k].v[j], acc.v[j]);
-                                delta.v[j] = step * u.v[j];
-                                rows[k].v[j] += delta.v[j];
-                            }
-                            if (RED) grow_red_add<DIM, NARROW>(w_out, ids[k], sub, delta);
-                            else if constexpr (SR)
-                                grow_store_sr<DIM, T, NARROW>(w_out, ids[k], sub, rows[k], ev,
-                                                              0x85EBCA77u * (uint32_t)(base + k * NG + grp + 1));
-                            else grow_store<DIM, T, NARROW>(w_out, ids[k], sub, rows[k]);
+                        for (int j = 0; j < FPL; ++j) {
+                            acc.v[j] = fmaf(g, rows[k].v[j], acc.v[j]);
+                            delta.v[j] = step * u.v[j];
+                            rows[k].v[j] += delta.v[j];
                         }
+                        if (RED) grow_red_add<DIM, NARROW>(w_out, row, sub, delta);
+                        else if constexpr (SR)
+                            grow_store_sr<DIM, T, NARROW>(w_out, row, sub, rows[k], ev,
+                                                          0x85EBCA77u * (uint32_t)(tgt[SL + base + k * NG + grp] + 1));
+                        else grow_store<DIM, T, NARROW>(w_out, row, sub, rows[k]);
                     }
-                    if (sp_prod > 1e30f) { sp_lin += logf(sp_prod); sp_prod = 1.f; }
-                } else if constexpr (PF_LINES > 0) {
-                    prefetch_chunk(base + HOGWILD_PF_DIST * CH);
                 }
-                my_kt += CH;
-                while (my_kt >= T1) my_kt -= T1;
+                if (sp_prod > 1e30f) { sp_lin += logf(sp_prod); sp_prod = 1.f; }
             }
             const float loss = sp_lin + logf(sp_prod);   // this lane's share of the position's loss
             // center row: add the accumulated increment to the row as it is now
@@ -804,9 +827,9 @@ sgns_targets_kernel(const int32_t *__restrict__ walks, int64_t n_pos, int64_t wa
                 for (int x0 = 0; x0 < SL; x0 += 32) {
                     const int x = x0 + lane;
                     const int32_t v = x < SL ? tgt[x] : -1;
-                    const bool take = v >= 0 && ((x % T1 == 0) == (pass == 0));
+                    const bool take = v != -1 && ((v < 0) == (pass == 0));   // bit 31: a context
                     const unsigned m = __ballot_sync(0xffffffffu, take);
-                    if (take) kp[n_all + __popc(m & below)] = (uint32_t)v;
+                    if (take) kp[n_all + __popc(m & below)] = (uint32_t)v & ~TARGET_IS_CONTEXT;
                     n_all += __popc(m);
                 }
                 if (pass == 0) n_ctx = n_all;
@@ -1646,7 +1669,7 @@ template <int DIM, typename T, bool RED, int MINB, int TC = TCH, bool NARROW = f
 static gs_status run_hogwild_b(const SgnsArgs &a, cudaStream_t st)
 {
     const int SL = 2 * a.w * (1 + a.K);
-    const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(hogwild_walks_per_ticket(a.L) * a.L + SL);
+    const size_t smem = sizeof(int32_t) * (size_t)SGNS_WARPS * (size_t)(hogwild_walks_per_ticket(a.L) * a.L + (SR ? 2 : 1) * SL);
     auto kern = sgns_hogwild_kernel<DIM, T, RED, MINB, TC, NARROW, SR>;
     if (smem > 48 * 1024)
         GS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

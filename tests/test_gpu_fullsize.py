@@ -332,3 +332,99 @@ def test_truncated_epoch_of_the_medium_workload_matches_the_oracle():
     assert np.abs(V).max() > 1e-3
     G.close()
     B.gs_release_workspace()
+
+
+@pytest.mark.parametrize("fmt", ["f16", "bf16"])
+def test_16bit_tables_at_the_largest_table_size(fmt):
+    # Tables of the 50M-node workload stored in a 16-bit format: 12.8 GB each, so the byte offset of
+    # a row passes 2^32 after a third of the table.  Start values checked on sampled rows across the
+    # whole table; a synchronous step of the epoch's last 512 walks (their start nodes are the last
+    # rows) against the oracle on the touched rows, seeded so that the step moves them: every value
+    # within one unit of the format and all but a few per cent bit-equal, rows outside the batch in
+    # three windows of a million rows keep their bits; then the whole batch through the lock-free
+    # kernel: pair count and a loss in the expected range.
+    wl = WL.WORKLOADS["deepwalk_large"]
+    torch.cuda.empty_cache()
+    tdt = torch.float16 if fmt == "f16" else torch.bfloat16
+    init = B.gs_init_embeddings_f16 if fmt == "f16" else B.gs_init_embeddings_bf16
+    step = B.gs_sgns_step_f16 if fmt == "f16" else B.gs_sgns_step_bf16
+    rnd = O.round_f16 if fmt == "f16" else O.round_bf16
+    det = O.sgns_det_f16_from_lists if fmt == "f16" else O.sgns_det_bf16_from_lists
+    frac_bits = 10 if fmt == "f16" else 7
+
+    def unit(x):                                    # spacing of the format at |x| (normal range)
+        return 2.0 ** (np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -14))) - frac_bits)
+
+    g = wl.make_graph(device=DEV)
+    n, seed = g.n_nodes, wl.graph_seed
+    off = g.offsets.cpu().numpy().astype(np.int64)
+    col = g.cols.cpu().numpy()
+    thr, alias = O.build_alias((off[1:] - off[:-1]).astype(np.float64), 0.75)
+    table = (alias.astype(np.uint64) << np.uint64(32)) | thr.astype(np.uint64)
+    a_dev = torch.from_numpy(table.view(np.int64)).to(DEV)
+    G = B.gs_graph_load_csr(g.offsets, g.cols, B.GS_VALIDATE | B.GS_REQUIRE_SORTED | B.GS_BUILD_WALK_INDEX)
+    w_in = torch.empty((n, wl.dim), dtype=tdt, device=DEV)
+    w_out = torch.empty_like(w_in)
+    assert w_in.numel() * 2 > 1 << 33
+    init(w_in, w_out, seed)
+    probe = np.concatenate([np.random.default_rng(1).integers(0, n, 61), [0, n // 3 + 1, n - 1]])
+    got = w_in[torch.from_numpy(probe).to(DEV)].float().cpu().numpy().astype(np.float64)
+    assert np.array_equal(got, rnd(O.init_rows(probe, wl.dim, seed)))
+
+    total = n * wl.walks_per_node
+    last = total - 512
+    tail = B.gs_random_walks(G, None, 512, last, wl.walk_len, seed)
+    tail_h = tail.cpu().numpy()
+    want, _ = O.uniform_walks(off, col, None, 512, last, wl.walk_len, seed)
+    assert np.array_equal(tail_h, want) and int(tail_h[-1, 0]) == n - 1
+    c, o, ng, n_pairs = O.expand_lists(tail_h, last, wl.window, wl.n_neg, thr, alias, seed)
+    ids, cc, oo, nn = compact_problem(c, o, ng)
+    assert ids.max() == n - 1 and (ids > n // 3).any()
+    ids_dev = torch.from_numpy(ids).to(DEV)
+    gen = torch.Generator().manual_seed(99)
+    u0 = ((torch.rand((len(ids), wl.dim), generator=gen) - 0.5) * 0.6).to(tdt)
+    v0 = ((torch.rand((len(ids), wl.dim), generator=gen) - 0.5) * 0.15).to(tdt)
+    w_in[ids_dev] = u0.to(DEV)
+    w_out[ids_dev] = v0.to(DEV)
+    U, V = u0.float().numpy().astype(np.float64), v0.float().numpy().astype(np.float64)
+    U0, V0 = U.copy(), V.copy()
+    win = 1 << 20
+    keep = []
+    for lo in (0, n // 2 - win // 2, n - win):
+        outside = torch.ones(win, dtype=torch.bool, device=DEV)
+        outside[ids_dev[(ids_dev >= lo) & (ids_dev < lo + win)] - lo] = False
+        keep.append((lo, outside, w_in[lo:lo + win].clone(), w_out[lo:lo + win].clone()))
+    lr = 4 * wl.lr0                                  # so that most written values change in 16 bits
+    loss_o, cnt_o = det(U, V, cc, oo, nn, lr)
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    step(w_in, w_out, tail, last, wl.window, wl.n_neg, a_dev, lr, seed, B.GS_DETERMINISTIC, loss, cnt)
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == cnt_o == n_pairs > 0
+    assert abs(loss.item() - loss_o) <= 2e-6 * abs(loss_o)
+    for name, tab, want_rows, before in (("in", w_in, U, U0), ("out", w_out, V, V0)):
+        got = tab[ids_dev].float().cpu().numpy().astype(np.float64)
+        diff = np.abs(got - want_rows)
+        assert (diff <= unit(want_rows) * 1.0001 + 1e-6).all(), (name, float((diff / unit(want_rows)).max()))
+        assert np.mean(diff > 0) <= 0.02, (name, float(np.mean(diff > 0)))
+        touched = (want_rows != before).any(axis=1)
+        assert np.mean((got != before)[touched]) > 0.5, name      # the step is not lost in the rounding
+    for lo, outside, before_in, before_out in keep:
+        assert torch.equal(w_in[lo:lo + win][outside], before_in[outside]), lo
+        assert torch.equal(w_out[lo:lo + win][outside], before_out[outside]), lo
+    del keep
+
+    bw = 1 << 20
+    base = ((total // bw) // 2) * bw
+    walks = B.gs_random_walks(G, None, bw, base, wl.walk_len, seed)
+    loss.zero_()
+    cnt.zero_()
+    step(w_in, w_out, walks, base, wl.window, wl.n_neg, a_dev, wl.lr0, seed, B.GS_HOGWILD, loss, cnt)
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == count_pairs(walks, wl.window)
+    assert 0.3 < loss.item() / cnt.item() <= (1 + wl.n_neg) * np.log(2) * (1 + 1e-3)
+    assert bool(torch.isfinite(w_out[ids_dev].float()).all())
+    G.close()
+    del w_in, w_out, walks, g, a_dev
+    B.gs_release_workspace()
+    torch.cuda.empty_cache()

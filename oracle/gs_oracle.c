@@ -674,7 +674,7 @@ typedef struct {          /* stochastic write-back of the lock-free schedule (NU
 
 static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
                             const int32_t *centers, const int32_t *contexts, const int32_t *negs,
-                            double lr, int fmt, const sr_keys *sr, double *loss_sum, int64_t *pair_count);
+                            double lr, int fmt, const sr_keys *sr, int red, double *loss_sum, int64_t *pair_count);
 
 int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
                                 int64_t n_slots, int32_t S, int32_t K,
@@ -682,7 +682,7 @@ int gso_sgns_seq_f16_from_lists(double *U, double *V, int32_t d,
                                 const int32_t *negs, double lr,
                                 double *loss_sum, int64_t *pair_count)
 {
-    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 0, NULL, loss_sum, pair_count);
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 0, NULL, 0, loss_sum, pair_count);
 }
 
 int gso_sgns_seq_bf16_from_lists(double *U, double *V, int32_t d,
@@ -691,7 +691,7 @@ int gso_sgns_seq_bf16_from_lists(double *U, double *V, int32_t d,
                                  const int32_t *negs, double lr,
                                  double *loss_sum, int64_t *pair_count)
 {
-    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 1, NULL, loss_sum, pair_count);
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, 1, NULL, 0, loss_sum, pair_count);
 }
 
 /* Same with stochastic write-back.  Event of the lock-free mode: the rows written while position
@@ -704,12 +704,24 @@ int gso_sgns_seq_sr_from_lists(double *U, double *V, int32_t d, int64_t n_slots,
                                double *loss_sum, int64_t *pair_count)
 {
     sr_keys sr = { seed, walk_id_base, L };
-    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, fmt, &sr, loss_sum, pair_count);
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, fmt, &sr, 0, loss_sum, pair_count);
+}
+
+/* Same order of pairs, but the tables are changed the way Section 3.2 describes the exchange
+ * between trainer and storage: the trainer sends an INCREMENT and the storage adds it.  With a
+ * 16-bit table both the increment and the sum exist in the table's format only: the increment is
+ * rounded to the format (nearest even), the addition of the two 16-bit values is exact and its
+ * result is rounded to the format once more.  fmt 0: binary16, 1: bfloat16. */
+int gso_sgns_seq_add16_from_lists(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
+                                  const int32_t *centers, const int32_t *contexts, const int32_t *negs,
+                                  double lr, int fmt, double *loss_sum, int64_t *pair_count)
+{
+    return sgns_seq_rounded(U, V, d, n_slots, S, K, centers, contexts, negs, lr, fmt, NULL, 1, loss_sum, pair_count);
 }
 
 static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, int32_t S, int32_t K,
                             const int32_t *centers, const int32_t *contexts, const int32_t *negs,
-                            double lr, int fmt, const sr_keys *sr, double *loss_sum, int64_t *pair_count)
+                            double lr, int fmt, const sr_keys *sr, int red, double *loss_sum, int64_t *pair_count)
 {
     double *acc = (double *)malloc(sizeof(double) * (size_t)d);
     if (!acc) return -1;
@@ -741,6 +753,11 @@ static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, in
                 const uint32_t salt = 1u + (uint32_t)(sg * (1 + K) + (k + 1));
                 for (int32_t j = 0; j < d; ++j) {
                     acc[j] += g * v[j];
+                    if (red) {                       /* increment in the format, then the sum in the format */
+                        const double inc = fmt ? rnb16(-lr * g * u[j]) : rn16(-lr * g * u[j]);
+                        v[j] = fmt ? rnb16(v[j] + inc) : rn16(v[j] + inc);
+                        continue;
+                    }
                     const double nv = v[j] - lr * g * u[j];
                     v[j] = sr ? sr16(nv, fmt, dither16(ev, salt, j)) : (fmt ? rnb16(nv) : rn16(nv));
                 }
@@ -748,6 +765,11 @@ static int sgns_seq_rounded(double *U, double *V, int32_t d, int64_t n_slots, in
         }
         if (c >= 0)
             for (int32_t j = 0; j < d; ++j) {
+                if (red) {
+                    const double inc = fmt ? rnb16(-lr * acc[j]) : rn16(-lr * acc[j]);
+                    U[c * d + j] = fmt ? rnb16(U[c * d + j] + inc) : rn16(U[c * d + j] + inc);
+                    continue;
+                }
                 double nv = U[c * d + j] - lr * acc[j];
                 U[c * d + j] = sr ? sr16(nv, fmt, dither16(ev, 0x10000u, j)) : (fmt ? rnb16(nv) : rn16(nv));
             }

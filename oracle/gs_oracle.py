@@ -303,6 +303,24 @@ def sgns_seq_f16_from_lists(U, V, centers, contexts, negs, S, lr):
     return float(loss.value), int(cnt.value)
 
 
+def sgns_seq_add16_from_lists(U, V, centers, contexts, negs, S, lr, fmt):
+    """Sequential per-pair SGD on 16-bit-valued tables where every change is an increment rounded
+    to the format and added in the format (fmt 0: binary16, 1: bfloat16), in place."""
+    d = U.shape[1]
+    centers, contexts, negs = _i32(centers), _i32(contexts), _i32(negs)
+    K = negs.shape[1]
+    loss = ctypes.c_double(0.0)
+    cnt = ctypes.c_int64(0)
+    rc = lib().gso_sgns_seq_add16_from_lists(
+        _p(U, ctypes.c_double), _p(V, ctypes.c_double), ctypes.c_int32(d),
+        ctypes.c_int64(len(centers)), ctypes.c_int32(S), ctypes.c_int32(K),
+        _p(centers, ctypes.c_int32), _p(contexts, ctypes.c_int32), _p(negs, ctypes.c_int32),
+        ctypes.c_double(lr), ctypes.c_int32(fmt), ctypes.byref(loss), ctypes.byref(cnt))
+    if rc != 0:
+        raise MemoryError("oracle accumulator")
+    return float(loss.value), int(cnt.value)
+
+
 def round_sr(x, fmt, u16):
     """In place: every value rounded stochastically to binary16 (fmt 0) or bfloat16 (fmt 1) with the
     given 16-bit dithers (one per value)."""

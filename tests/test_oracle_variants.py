@@ -424,3 +424,98 @@ def test_sequential_mode_with_stochastic_write_back_keys_every_write(fmt):
     (O.sgns_seq_f16_from_lists if fmt == 0 else O.sgns_seq_bf16_from_lists)(Ub, Vb, c, o, ng, 2 * w, 0.1)
     assert not np.array_equal(V, Vb)
     assert np.abs(V - Vb).max() <= np.abs(Vb).max() * 2.0 ** (-9 if fmt == 0 else -6)
+
+
+# ---- increments rounded to the format and added in the format (Section 3.2: the trainer sends
+# increments, the storage adds them), sequential order
+def _round_to_bits(x, bits):
+    """Nearest-even rounding of float64 values to `bits` significant bits (normal range), written
+    with frexp / rint / ldexp: independent of the oracle's C code."""
+    m, e = np.frexp(np.asarray(x, dtype=np.float64))
+    return np.ldexp(np.rint(m * 2.0 ** bits), e - bits)
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_increment_and_add_rounds_twice_where_the_plain_write_back_rounds_once(fmt):
+    # One pair, dimension 1, no negative: context value 1.0, center value 2^-10.  The learning rate
+    # is chosen so that the context's increment is a hair above HALF a unit of 1.0 in the format:
+    # written back in one rounding, 1 + inc goes up to the next value; sent as an increment, inc is
+    # first rounded to exactly half a unit, the sum is a tie, and ties go to the even neighbour 1.0.
+    import math
+    bits = 11 if fmt == 0 else 8                      # significant bits of the format
+    half_unit = 2.0 ** -bits                          # half the spacing just above 1.0
+    u, v = 2.0 ** -10, 1.0
+    g = 1.0 / (1.0 + math.exp(-u * v)) - 1.0          # context: sigmoid(f) - 1
+    lr = half_unit * (1.0 + 2.0 ** -19) / (-g * u)
+    assert abs(-lr * g * u / half_unit - 1.0 - 2.0 ** -19) < 1e-12
+    c = np.array([0], dtype=np.int32)
+    o = np.array([1], dtype=np.int32)
+    ng = np.array([[-1]], dtype=np.int32)
+    seq16 = O.sgns_seq_f16_from_lists if fmt == 0 else O.sgns_seq_bf16_from_lists
+
+    def tables():
+        return np.array([[u], [0.0]]), np.array([[0.0], [v]])
+    U1, V1 = tables()
+    seq16(U1, V1, c, o, ng, 1, lr)
+    assert V1[1, 0] == 1.0 + 2.0 * half_unit          # one rounding: up
+    U2, V2 = tables()
+    loss, cnt = O.sgns_seq_add16_from_lists(U2, V2, c, o, ng, 1, lr, fmt)
+    assert cnt == 1 and abs(loss - math.log1p(math.exp(-u * v))) < 1e-15
+    assert V2[1, 0] == 1.0                            # two roundings: the tie goes to even
+    # the center row: its increment -lr * g * v = inc / u is representable after rounding, and so is the sum here
+    inc_u = _round_to_bits(-lr * g * v, bits)
+    assert U2[0, 0] == _round_to_bits(u + inc_u, bits)
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_increment_and_add_is_the_full_precision_step_rounded_as_increment_then_as_sum(fmt):
+    # One position whose targets are all different rows: every row is written once, so the clause
+    # must equal  round(old + round(new_full - old))  with new_full from the full-precision sequential
+    # step and the rounding done here with frexp / rint (binary16 also with numpy's conversion).
+    bits = 11 if fmt == 0 else 8
+    rng = np.random.default_rng(17 + fmt)
+    n, d, S, K = 64, 24, 6, 3
+    ids = rng.permutation(n)
+    c = np.full(S, ids[0], dtype=np.int32)
+    o = ids[1:1 + S].astype(np.int32)
+    ng = ids[1 + S:1 + S + S * K].reshape(S, K).astype(np.int32)
+    c[4], o[4], ng[4] = -1, -1, -1                     # a slot without a pair
+    ng[2, 1] = -1                                      # an absent negative
+    U0 = _round_to_bits(rng.uniform(-0.5, 0.5, (n, d)), bits)
+    V0 = _round_to_bits(rng.uniform(-0.5, 0.5, (n, d)), bits)
+    lr = 0.05
+    Uf, Vf = U0.copy(), V0.copy()
+    loss_f, cnt_f = O.sgns_seq_from_lists(Uf, Vf, c, o, ng, S, lr)
+    U, V = U0.copy(), V0.copy()
+    loss, cnt = O.sgns_seq_add16_from_lists(U, V, c, o, ng, S, lr, fmt)
+    assert cnt == cnt_f == S - 1 and abs(loss - loss_f) < 1e-12
+    want_U = _round_to_bits(U0 + _round_to_bits(Uf - U0, bits), bits)
+    want_V = _round_to_bits(V0 + _round_to_bits(Vf - V0, bits), bits)
+    # new_full - old carries fp64 rounding of about 1e-17, far from deciding a rounding here
+    assert np.array_equal(U, want_U) and np.array_equal(V, want_V)
+    touched = np.concatenate([[ids[0]], o[o >= 0], ng[ng >= 0]])
+    assert (V != V0).any(axis=1).sum() == len(touched) - 1 and (U != U0).any(axis=1).sum() == 1
+    if fmt == 0:                                       # numpy has binary16: round with its conversion as well
+        h = lambda x: x.astype(np.float16).astype(np.float64)
+        assert np.array_equal(V, h(V0 + h(Vf - V0))) and np.array_equal(U, h(U0 + h(Uf - U0)))
+    # and it is not the single rounding: some values differ from the plain 16-bit write-back
+    U1, V1 = U0.copy(), V0.copy()
+    (O.sgns_seq_f16_from_lists if fmt == 0 else O.sgns_seq_bf16_from_lists)(U1, V1, c, o, ng, S, lr)
+    assert np.abs(V1 - V).max() <= 2.0 ** (1 - bits) and (V1 != V).any()
+
+
+def test_increment_and_add_drops_increments_below_half_a_unit_of_the_stored_value():
+    # The same tiny increment sent 200 times (one position with 200 slots that name the same context,
+    # so the center row stays as it is meanwhile): each is below half a unit of the stored value, so
+    # a table that adds in its own format never moves, while the increments add up to more than a unit.
+    c = np.zeros(200, dtype=np.int32)
+    o = np.ones(200, dtype=np.int32)
+    ng = np.full((200, 1), -1, dtype=np.int32)
+    U = np.array([[2.0 ** -12], [0.0]])
+    V = np.array([[0.0], [1.0]])
+    lr = 0.05                                          # increment about 0.05 * 0.5 * 2^-12 = 6e-6; half a unit of 1.0 is 4.9e-4
+    O.sgns_seq_add16_from_lists(U, V, c, o, ng, 200, lr, 0)
+    assert V[1, 0] == 1.0
+    Uf, Vf = np.array([[2.0 ** -12], [0.0]]), np.array([[0.0], [1.0]])
+    O.sgns_seq_from_lists(Uf, Vf, c, o, ng, 200, lr)
+    assert Vf[1, 0] - 1.0 > 1e-3

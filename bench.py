@@ -51,7 +51,7 @@ def parse_args():
     ap.add_argument("--batch-walks", type=int, default=1 << 20)
     ap.add_argument("--mode", default="hogwild_red",
                     choices=["hogwild", "hogwild_red", "deterministic", "momentum", "adam"],
-                    help="hogwild_red: lock-free, increments added by reductions (default; fp32 tables); "
+                    help="hogwild_red: lock-free, increments added by reductions (default); "
                          "hogwild: lock-free with plain stores; deterministic: synchronous batches of 512 "
                          "walks; momentum / adam: synchronous with that optimizer")
     ap.add_argument("--variants", default="",
@@ -596,8 +596,8 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
     if args.mode in ("momentum", "adam"):
         return run_momentum(args, wl, g, G, alias, w_in, w_out, info, dev)
     mode_name = args.mode
-    if f16 and mode_name == "hogwild_red":
-        mode_name = "hogwild"                          # 16-bit tables: plain stores only
+    if f16 and mode_name == "hogwild_red" and args.round == "stochastic":
+        mode_name = "hogwild"                          # the reduction unit rounds to nearest only
     mode = {"hogwild": B.GS_HOGWILD, "hogwild_red": B.GS_HOGWILD_RED,
             "deterministic": B.GS_DETERMINISTIC}[mode_name]
     if wl.forward_only:

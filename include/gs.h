@@ -338,10 +338,15 @@ GS_API gs_status gs_momentum_flush(float *d_w, float *d_m, int32_t *d_last, int6
  * 128 values in 256 GB, Section 4.2).  d_w_in / d_w_out hold IEEE half values,
  * [n_nodes][dim] row-major, dim in {64, 128, 256}.  Every row is widened to
  * fp32 when read, all arithmetic is as in gs_sgns_step, and a written row is
- * rounded to nearest-even half.  Row traffic halves; increments far below half
- * an ulp of the stored value are lost (no stochastic rounding).
- * Modes: GS_DETERMINISTIC (bitwise reproducible) and GS_HOGWILD;
- * GS_HOGWILD_RED returns GS_ERR_UNSUPPORTED.  Other arguments as gs_sgns_step.
+ * rounded to nearest-even half (or stochastically, GS_ROUND_STOCHASTIC).  Row
+ * traffic halves; to nearest, increments far below half a unit in the last
+ * place of the stored value are lost.
+ * Modes: GS_DETERMINISTIC (bitwise reproducible), GS_HOGWILD, and
+ * GS_HOGWILD_RED: there every change is sent as an INCREMENT rounded to the
+ * table's format and the reduction unit adds it in that format (a second
+ * rounding to nearest; Section 3.2: trainers send increments, the storage adds
+ * them), so no update is lost to a race; GS_ROUND_STOCHASTIC cannot be combined
+ * with it (GS_ERR_UNSUPPORTED).  Other arguments as gs_sgns_step.
  * gs_init_embeddings_f16 writes the start values of gs_init_embeddings rounded
  * to half.
  */

@@ -384,23 +384,37 @@ __device__ __forceinline__ void row_store_sr(T *__restrict__ tab, int64_t r, int
     }
 }
 
-// row += x as reductions (fp32 tables only)
-template <int DIM, bool NARROW>
-__device__ __forceinline__ void grow_red_add(float *__restrict__ tab, int64_t r, int sub,
-                                             const Row<RowGeom<DIM, float, NARROW>::FPL> &x)
+// row += x as reductions.  fp32 tables: 16 bytes of fp32 increments per instruction.  16-bit
+// tables: the increment is rounded to the table's format (nearest even) and the reduction unit
+// adds it there in that format (one more rounding), 16 bytes = 8 values per instruction.
+__device__ __forceinline__ void red_add_16bytes(__half *p, const uint4 &v)
 {
-    constexpr int FPL = RowGeom<DIM, float, NARROW>::FPL, LPR = RowGeom<DIM, float, NARROW>::LPR;
-    float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
-#pragma unroll
-    for (int q = 0; q < FPL / 4; ++q)
-        atomicAdd(p + q * LPR + sub,
-                  make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
+    asm volatile("red.global.add.noftz.v4.f16x2 [%0], {%1, %2, %3, %4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
-template <int DIM, bool NARROW>
-__device__ __forceinline__ void grow_red_add(__half *, int64_t, int, const Row<RowGeom<DIM, __half, NARROW>::FPL> &) {}
-template <int DIM, bool NARROW>
-__device__ __forceinline__ void grow_red_add(__nv_bfloat16 *, int64_t, int,
-                                             const Row<RowGeom<DIM, __nv_bfloat16, NARROW>::FPL> &) {}
+__device__ __forceinline__ void red_add_16bytes(__nv_bfloat16 *p, const uint4 &v)
+{
+    asm volatile("red.global.add.noftz.v4.bf16x2 [%0], {%1, %2, %3, %4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+template <int DIM, bool NARROW, typename T>
+__device__ __forceinline__ void grow_red_add(T *__restrict__ tab, int64_t r, int sub,
+                                             const Row<RowGeom<DIM, T, NARROW>::FPL> &x)
+{
+    using G = RowGeom<DIM, T, NARROW>;
+    if constexpr (sizeof(T) == 4) {
+        float4 *p = reinterpret_cast<float4 *>(tab + r * (int64_t)DIM);
+#pragma unroll
+        for (int q = 0; q < G::FPL / 4; ++q)
+            atomicAdd(p + q * G::LPR + sub,
+                      make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
+    } else {
+        T *p = tab + r * (int64_t)DIM;
+#pragma unroll
+        for (int q = 0; q < G::FPL / G::PER16; ++q)
+            red_add_16bytes(p + (q * G::LPR + sub) * G::PER16, pack16(x.v + G::PER16 * q, (const T *)nullptr));
+    }
+}
 
 // Sums of N values over the LPR lanes of a row group in about half the shuffles of N separate
 // butterflies.  While more than one value is left, a step pairs the values up and a lane keeps,
@@ -1954,9 +1968,11 @@ static gs_status run_mode(const SgnsArgs &a, int mode, cudaStream_t st)
 {
     if (mode == GS_DETERMINISTIC) return run_deterministic<DIM, T>(a, st);
     if (mode == GS_HOGWILD) return run_hogwild<DIM, T, false>(a, st);
-    if constexpr (sizeof(T) == 4) return run_hogwild<DIM, T, true>(a, st);
-    set_error("GS_HOGWILD_RED is not available for 16-bit tables");
-    return GS_ERR_UNSUPPORTED;
+    if (a.sr) {                     // the reduction unit rounds to nearest
+        set_error("GS_ROUND_STOCHASTIC is not available with GS_HOGWILD_RED");
+        return GS_ERR_UNSUPPORTED;
+    }
+    return run_hogwild<DIM, T, true>(a, st);
 }
 
 // One step on tables of type T (float, or a 16-bit format with fp32 arithmetic and write-back

@@ -163,8 +163,8 @@ def test_half_tables_reject_what_they_do_not_support(tiny):
         B.gs_sgns_step_f16(w32, w32.clone(), walks, 0, 2, 2, a_dev, 0.1, 0, B.GS_HOGWILD)
     assert e.value.status == -6
     w = torch.zeros((g.n_nodes, 64), dtype=torch.float16, device=DEV)
-    with pytest.raises(B.GsError) as e:
-        B.gs_sgns_step_f16(w, w.clone(), walks, 0, 2, 2, a_dev, 0.1, 0, B.GS_HOGWILD_RED)
+    with pytest.raises(B.GsError) as e:                    # the reduction unit rounds to nearest only
+        B.gs_sgns_step_f16(w, w.clone(), walks, 0, 2, 2, a_dev, 0.1, 0, B.GS_HOGWILD_RED | B.GS_ROUND_STOCHASTIC)
     assert e.value.status == -6
 
 

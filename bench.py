@@ -794,15 +794,17 @@ def run_leg(args, wl, dev, rank, world, local, with_e2e, with_cpu):
     return out
 
 
-# The default run's short legs: (workload, mode, steps, warm-up).  The synchronous mode takes
-# batches of 512 walks, so its legs run a few hundred steps inside one call of the epoch driver;
-# the tiny workload is its whole epoch (20 batches).
+# The default run's short legs: (workload, mode, steps, warm-up, table type).  The synchronous mode
+# takes batches of 512 walks, so its legs run a few hundred steps inside one call of the epoch
+# driver; the tiny workload is its whole epoch (20 batches).  The last leg is the headline workload
+# with half-precision tables (the storage type of the paper's production run, Section 4.2).
 PER_CONFIG_LEGS = [
-    ("tiny_deepwalk", "deterministic", 17, 3),
-    ("deepwalk_medium", "deterministic", 300, 5),
-    ("deepwalk_medium", "hogwild_red", 8, 3),
-    ("node2vec_4m", "hogwild_red", 6, 3),
-    ("rmat_billion", "hogwild_red", 10, 3),
+    ("tiny_deepwalk", "deterministic", 17, 3, "f32"),
+    ("deepwalk_medium", "deterministic", 300, 5, "f32"),
+    ("deepwalk_medium", "hogwild_red", 8, 3, "f32"),
+    ("node2vec_4m", "hogwild_red", 6, 3, "f32"),
+    ("rmat_billion", "hogwild_red", 10, 3, "f32"),
+    ("deepwalk_large", "hogwild_red", 8, 3, "f16"),
 ]
 
 
@@ -827,17 +829,17 @@ def run_ours(args, wl):
                   with_cpu=not args.no_cpu_baseline)
     if out is not None and plain and world == 1 and not args.no_per_config:
         legs = {}
-        for name, mode, steps, warmup in PER_CONFIG_LEGS:
+        for name, mode, steps, warmup, tdt in PER_CONFIG_LEGS:
             from paper_2407_15452_b200.workloads import WORKLOADS
             largs = argparse.Namespace(**{**vars(args), "workload": name, "mode": mode, "steps": steps,
-                                          "warmup": warmup, "batch_walks": 1 << 20})
+                                          "warmup": warmup, "batch_walks": 1 << 20, "table_dtype": tdt})
             t0 = time.time()
             r = run_leg(largs, WORKLOADS[name], dev, rank, world, local, with_e2e=False, with_cpu=False)
-            legs[f"{name}/{mode}"] = {
+            legs[f"{name}/{mode}" + ("" if tdt == "f32" else f"/{tdt}")] = {
                 "pair_updates_per_s": r["value"], "walk_steps_per_s": r["walk_steps_per_s"],
                 "ms_per_step": r["ms_per_step"], "steps": r["steps"], "warmup": r["warmup"],
                 "batch_walks": r["config"]["batch_walks"], "mean_loss": r["mean_loss"],
-                "gpu_launches": r["gpu_launches"], "n_nodes": r["config"]["n_nodes"],
+                "gpu_launches": r["gpu_launches"], "table_dtype": tdt, "n_nodes": r["config"]["n_nodes"],
                 "n_edges": r["config"]["n_edges"], "roofline": r["roofline"], "walk": r["walk"],
                 "clocks": r["clocks"], "leg_s": round(time.time() - t0, 1)}
         out["per_config"] = legs

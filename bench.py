@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="deepwalk_large")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the node count (testing)")
+    ap.add_argument("--dim", type=int, default=None, choices=[32, 64, 128, 256],
+                    help="embedding dimension instead of the workload's own (a sweep over the embedding "
+                         "size, as in the paper's Fig. 11); named in config.dim")
     ap.add_argument("--batch-walks", type=int, default=1 << 20)
     ap.add_argument("--mode", default="hogwild_red",
                     choices=["hogwild", "hogwild_red", "deterministic", "momentum", "adam"],
@@ -824,7 +827,7 @@ def run_ours(args, wl):
     B.lib()                                            # fail loudly if the library is missing
 
     plain = (args.workload == "deepwalk_large" and args.mode == "hogwild_red" and args.stage == "all"
-             and args.table_dtype == "f32" and not args.variants and args.scale == 1.0)
+             and args.table_dtype == "f32" and not args.variants and args.scale == 1.0 and args.dim is None)
     out = run_leg(args, wl, dev, rank, world, local, with_e2e=not args.no_e2e,
                   with_cpu=not args.no_cpu_baseline)
     if out is not None and plain and world == 1 and not args.no_per_config:
@@ -853,6 +856,9 @@ def main():
     args = parse_args()
     from paper_2407_15452_b200.workloads import WORKLOADS
     wl = WORKLOADS[args.workload]
+    if args.dim is not None:
+        import dataclasses
+        wl = dataclasses.replace(wl, dim=args.dim)
     if args.stage == "row-updates" and args.impl != "reference":
         return run_row_update_probe(args)
     if args.impl == "reference":

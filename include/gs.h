@@ -271,7 +271,7 @@ GS_API gs_status gs_sgns_step(float *d_w_in, float *d_w_out, int64_t n_nodes, in
  *
  * Limit: the batch must need at most 32 MiB of scratch,
  *   slots = n_walks * walk_len * (P + 1), P = 2*window*(1+n_neg) rounded up to a power of two
- *   bytes ~ (24 + dim/16) * slots + n_walks * walk_len * (4*dim + 16)  (+ < 1 % for the sort)
+ *   bytes ~ (25 + dim/16) * slots + n_walks * walk_len * (4*dim + 16)  (+ < 1 % for the sort)
  * e.g. up to about 300 walks of length 40 with window 5, 5 negatives, dim 128.
  * Larger batches are rejected with GS_ERR_UNSUPPORTED and a message that
  * states the bytes needed; nothing is launched in that case.

@@ -859,6 +859,52 @@ sgns_targets_kernel(const int32_t *__restrict__ walks, int64_t n_pos, int64_t wa
     }
 }
 
+// row += x where nobody else adds to the row during this launch: one reduction per value, so the
+// result does not depend on timing, and the row never has to travel to the SM.
+template <int FPL>
+__device__ __forceinline__ void row_red_add(float *__restrict__ tab, int64_t r, int lane, const Row<FPL> &x)
+{
+    float *p = tab + r * (int64_t)(FPL * 32);
+    if constexpr (FPL == 1) {
+        atomicAdd(p + lane, x.v[0]);
+    } else if constexpr (FPL == 2) {
+        atomicAdd(reinterpret_cast<float2 *>(p) + lane, make_float2(x.v[0], x.v[1]));
+    } else {
+#pragma unroll
+        for (int q = 0; q < FPL / 4; ++q)
+            atomicAdd(reinterpret_cast<float4 *>(p) + q * 32 + lane,
+                      make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
+    }
+}
+
+// Part A, last launch: output rows that receive exactly ONE contribution in this batch (a run of
+// length one in the sorted keys; half of the rows, a quarter of the contributions on a graph of
+// 10^6 nodes).  No other contribution reads or changes such a row, so the coefficient pass, which
+// has the center row in registers, can add its increment at once and the apply pass can skip it:
+// single[idx] = 1 for the coefficient pass, and bit 31 of the sorted contribution index for the
+// apply pass (indices stay below 2^30).
+constexpr uint32_t SINGLE_RUN = 0x80000000u;
+// The shortcut pays where most runs have one entry, i.e. where the tables have many more rows than
+// a batch has list entries (measured with 1.3e6 entries per batch: 5 % slower at 1e6 rows, 9 % slower
+// at 2e6, 13 % faster at 5e6, 14 % faster at 5e7); the step marks them from this ratio of rows
+// per list entry on.
+constexpr int64_t SINGLE_MIN_NODES_PER_ENTRY = 3;
+
+__global__ void __launch_bounds__(256)
+sgns_mark_single_kernel(const uint32_t *__restrict__ keys, uint32_t *__restrict__ vals, uint32_t n_keys,
+                        uint32_t n_nodes, uint8_t *__restrict__ single)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (int64_t)n_keys; i += stride) {
+        const uint32_t key = keys[i];
+        if (key >= n_nodes) continue;                    // a center key or an empty slot
+        const bool alone = (i == 0 || keys[i - 1] != key) && (i + 1 >= (int64_t)n_keys || keys[i + 1] != key);
+        const uint32_t idx = vals[i];
+        single[idx] = alone ? 1 : 0;
+        if (alone) vals[i] = idx | SINGLE_RUN;
+    }
+}
+
 // Sums of G rows at once.  v[q] is this lane's partial sum of row q.  The first log2(G) butterfly
 // steps exchange half of the values each (a lane keeps the rows whose index bit equals its lane
 // bit), the remaining steps add the one value left.  Afterwards the lanes whose index shares the
@@ -890,11 +936,15 @@ __device__ __forceinline__ float reduce_rows(float (&v)[G], int lane)
 // gradient needs at once, is evaluated per group of G rows on all lanes; the softplus of the
 // loss is put off until every lane holds the argument of one entry (32 entries per evaluation);
 // while a group is worked on, the rows of the next one are already on their way into L2.
-template <int DIM, typename T>
+// SINGLE (fp32 tables, plain SGD): an output row that receives only this contribution in the
+// batch gets its increment -lr g u here, as one reduction per value (nobody else reads or changes
+// the row in this batch, so the step stays synchronous and its bits do not depend on timing).
+template <int DIM, typename T, bool SINGLE>
 __global__ void __launch_bounds__(256, (DIM <= 64 ? 4 : 3))
-sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out, int64_t n_pos, int32_t shift,
+sgns_coef_kernel(const T *__restrict__ w_in, T *w_out, int64_t n_pos, int32_t shift,
                  uint32_t n_nodes, const uint32_t *__restrict__ keys, const uint32_t *__restrict__ tinfo,
-                 float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos)
+                 float *__restrict__ gbuf, float *__restrict__ GU, double *__restrict__ loss_pos,
+                 const uint8_t *__restrict__ single, float lr)
 {
     constexpr int FPL = DIM / 32;
     constexpr int G = FPL <= 4 ? 8 : 4;                 // rows in flight
@@ -913,7 +963,16 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out, int64_
             const uint32_t *kp = keys + (pos << shift);
             float *gp = gbuf + (pos << shift);
             uint32_t id = lane < n ? kp[lane] : 0u;     // entries [k0, k0 + 32) of the list, one per lane
+            const uint8_t *alone_p = single + (pos << shift);
+            uint32_t alone = 0u;                        // ... and whether the entry is its row's only one
+            if constexpr (SINGLE) alone = lane < n ? alone_p[lane] : 0u;
             const Row<FPL> u = row_load<FPL>(w_in, (int64_t)(keys[n_slots + pos] - n_nodes), lane);
+            auto add_at_once = [&](uint32_t row, float g) {
+                Row<FPL> d;
+#pragma unroll
+                for (int j = 0; j < FPL; ++j) d.v[j] = -lr * (g * u.v[j]);
+                if constexpr (sizeof(T) == 4) row_red_add<FPL>(w_out, (int64_t)row, lane, d);
+            };
             Row<FPL> acc;
 #pragma unroll
             for (int j = 0; j < FPL; ++j) acc.v[j] = 0.f;
@@ -925,6 +984,9 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out, int64_
             }
             for (int k0 = 0; k0 < n; k0 += 32) {
                 const uint32_t id_next = k0 + 32 + lane < n ? kp[k0 + 32 + lane] : 0u;
+                uint32_t alone_next = 0u;
+                if constexpr (SINGLE) alone_next = k0 + 32 + lane < n ? alone_p[k0 + 32 + lane] : 0u;
+                const unsigned alone_mask = __ballot_sync(0xffffffffu, alone != 0u);
                 float my_z = 0.f;                       // softplus argument of the entry this lane keeps
                 bool my_has = false;
                 const int m = n - k0 < 32 ? n - k0 : 32;  // entries of this stretch
@@ -960,6 +1022,9 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out, int64_
                         const float gq = __shfl_sync(0xffffffffu, g, q << SH);
 #pragma unroll
                         for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(gq, rows[q].v[j], acc.v[j]);
+                        if constexpr (SINGLE) {
+                            if ((alone_mask >> (g0 + q)) & 1u) add_at_once(__shfl_sync(0xffffffffu, id, g0 + q), gq);
+                        }
                     }
                 }
 #pragma unroll 1
@@ -973,9 +1038,13 @@ sgns_coef_kernel(const T *__restrict__ w_in, const T *__restrict__ w_out, int64_
                     if (lane == 0) { gp[k0 + g0] = g; loss += sp; }
 #pragma unroll
                     for (int j = 0; j < FPL; ++j) acc.v[j] = fmaf(g, row.v[j], acc.v[j]);
+                    if constexpr (SINGLE) {
+                        if ((alone_mask >> g0) & 1u) add_at_once(__shfl_sync(0xffffffffu, id, g0), g);
+                    }
                 }
                 if (my_has) loss += fmaxf(my_z, 0.f) + log1pf(expf(-fabsf(my_z)));
                 id = id_next;
+                alone = alone_next;
             }
             row_store<FPL>(GU, pos, lane, acc);         // fp32 scratch, natural column order
         }
@@ -1201,7 +1270,7 @@ sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
         // chunk never wait for it.
         auto link1 = [&](int64_t i, uint32_t &key, uint32_t &idx) {
             key = i < end ? keys[i] : 0xFFFFFFFFu;
-            idx = i < end ? vals[i] : 0u;
+            idx = i < end ? vals[i] & ~SINGLE_RUN : 0u;    // this pass treats one-entry runs like the others
         };
         auto link2 = [&](uint32_t key, uint32_t idx, float &g, int32_t &c) {
             g = 0.f;
@@ -1267,24 +1336,6 @@ sgns_apply_out_kernel(const T *__restrict__ w_in, T *__restrict__ w_out,
     }
 }
 
-// row += x where nobody else adds to the row during this launch: one reduction per value, so the
-// result does not depend on timing, and the row never has to travel to the SM.
-template <int FPL>
-__device__ __forceinline__ void row_red_add(float *__restrict__ tab, int64_t r, int lane, const Row<FPL> &x)
-{
-    float *p = tab + r * (int64_t)(FPL * 32);
-    if constexpr (FPL == 1) {
-        atomicAdd(p + lane, x.v[0]);
-    } else if constexpr (FPL == 2) {
-        atomicAdd(reinterpret_cast<float2 *>(p) + lane, make_float2(x.v[0], x.v[1]));
-    } else {
-#pragma unroll
-        for (int q = 0; q < FPL / 4; ++q)
-            atomicAdd(reinterpret_cast<float4 *>(p) + q * 32 + lane,
-                      make_float4(x.v[4 * q], x.v[4 * q + 1], x.v[4 * q + 2], x.v[4 * q + 3]));
-    }
-}
-
 // Pass 3 for fp32 tables and plain SGD.  Same walk over the sorted contributions as
 // sgns_apply_out_kernel (one warp per block of RUN_CUT positions, runs cut at block boundaries
 // and finished by the last launch of the step), made light so that many warps are resident:
@@ -1295,7 +1346,8 @@ __device__ __forceinline__ void row_red_add(float *__restrict__ tab, int64_t r, 
 //    row receives in the step and the result bits do not depend on scheduling.
 // (Prefetching the next group's center rows into L1 while a group is added was measured and did
 // not pay: 0.491 against 0.484 ms per batch.)
-template <int FPL>
+// MARKED: part A marked the runs of one entry and the coefficient pass has added them already.
+template <int FPL, bool MARKED>
 __global__ void __launch_bounds__(256, (FPL <= 2 ? 4 : 3))
 sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_out,
                           const int32_t *__restrict__ walks, const uint32_t *__restrict__ keys,
@@ -1341,10 +1393,12 @@ sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_
             key = i < end ? keys[i] : 0xFFFFFFFFu;
             idx = i < end ? vals[i] : 0u;
         };
+        // (a run of one entry, marked in bit 31 of its index, was added by the coefficient pass:
+        // nothing of it is fetched here)
         auto link2 = [&](uint32_t key, uint32_t idx, float &g, int32_t &c) {
             g = 0.f;
             c = 0;
-            if (key < n_nodes) {
+            if (key < n_nodes && !(MARKED && (idx & SINGLE_RUN))) {
                 g = gbuf[idx];
                 c = walks[idx >> shift];                  // contribution idx belongs to position idx >> shift
             }
@@ -1366,12 +1420,18 @@ sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_
             if (lane == 0) before = carry_key;
             carry_key = __shfl_sync(0xffffffffu, my_key, 31);
             const unsigned hmask = __ballot_sync(0xffffffffu, usable && my_key != before);
+            unsigned smask = 0u;                                      // runs of one entry, done already
+            if constexpr (MARKED) smask = __ballot_sync(0xffffffffu, usable && (idx0 & SINGLE_RUN) != 0u);
             const int n = __popc(__ballot_sync(0xffffffffu, usable));
             // G contributions at a time: their center rows are loaded together, then added in
             // index order; where the head mask has a bit the run before ends and a new one starts
             auto add_one = [&](int i, float gq, const Row<FPL> &row) {
                 if ((hmask >> i) & 1u) {                              // a run starts here (same on every lane)
                     if (have) close_inner();
+                    if constexpr (MARKED) {
+                        have = false;
+                        if ((smask >> i) & 1u) return;                // ... and is over: done by the coefficient pass
+                    }
                     have = true;
                     lead = false;
                     cur_key = __shfl_sync(0xffffffffu, my_key, i);
@@ -1384,20 +1444,31 @@ sgns_apply_out_sgd_kernel(const float *__restrict__ w_in, float *__restrict__ w_
             int q0 = 0;
 #pragma unroll 1
             for (; q0 + G <= n; q0 += G) {
+                if constexpr (MARKED) {
+                    if (((smask >> q0) & ((1u << G) - 1u)) == (1u << G) - 1u) {   // G one-entry runs in a row
+                        if (have) close_inner();
+                        have = false;
+                        continue;
+                    }
+                }
                 Row<FPL> ru[G];
 #pragma unroll
                 for (int q = 0; q < G; ++q)
-                    ru[q] = row_load<FPL>(w_in, (int64_t)__shfl_sync(0xffffffffu, c, q0 + q), lane);
+                    if (!MARKED || !((smask >> (q0 + q)) & 1u))
+                        ru[q] = row_load<FPL>(w_in, (int64_t)__shfl_sync(0xffffffffu, c, q0 + q), lane);
 #pragma unroll
                 for (int q = 0; q < G; ++q) add_one(q0 + q, __shfl_sync(0xffffffffu, g, q0 + q), ru[q]);
             }
 #pragma unroll 1
             for (; q0 < n; ++q0) {                                    // only where the output-row keys end
-                const Row<FPL> r1 = row_load<FPL>(w_in, (int64_t)__shfl_sync(0xffffffffu, c, q0), lane);
+                Row<FPL> r1;
+                if (!MARKED || !((smask >> q0) & 1u))
+                    r1 = row_load<FPL>(w_in, (int64_t)__shfl_sync(0xffffffffu, c, q0), lane);
                 add_one(q0, __shfl_sync(0xffffffffu, g, q0), r1);
             }
             if (n < 32) break;                                        // the rest is not ours
             my_key = key1; g = g1; c = c1;
+            if constexpr (MARKED) idx0 = idx1;
             key1 = key2; idx1 = idx2;
         }
         if (have) {
@@ -1760,6 +1831,8 @@ struct SyncScratch {
     int32_t *pairs_pos;
     uint32_t *tinfo;              // per position: contexts | all targets << 16 of its dense list
     uint32_t *n_out;              // output-row keys of the batch (one counter)
+    uint8_t *single;              // per list entry: the only contribution to its output row in this batch
+    bool mark;                    // one-entry runs are marked (and added by the coefficient pass)
     double *lead_part, *tail_part;
     int64_t n_pos, n_slots, n_keys, n_cut;
     int SL, shift, bits;          // a position's list occupies 2^shift >= SL entries
@@ -1776,6 +1849,7 @@ static size_t sync_layout(const SgnsArgs &a, unsigned char *base, SyncScratch *o
     s.n_keys = s.n_slots + s.n_pos;
     s.n_cut = (s.n_keys + RUN_CUT - 1) / RUN_CUT;
     s.bits = bit_length(2ull * (uint64_t)a.n_nodes);
+    s.mark = (int64_t)a.n_nodes >= SINGLE_MIN_NODES_PER_ENTRY * s.n_slots;
     const size_t b_keys = align_up(sizeof(uint32_t) * (size_t)s.n_keys);
     const size_t b_g = align_up(sizeof(float) * (size_t)s.n_slots);
     const size_t b_gu = align_up(sizeof(float) * (size_t)s.n_pos * a.dim);
@@ -1783,6 +1857,7 @@ static size_t sync_layout(const SgnsArgs &a, unsigned char *base, SyncScratch *o
     const size_t b_pairs = align_up(sizeof(int32_t) * (size_t)s.n_pos);
     const size_t b_cnt = align_up(sort_counts_bytes((uint32_t)s.n_keys));
     const size_t b_part = align_up(sizeof(double) * (size_t)s.n_cut * a.dim);
+    const size_t b_single = align_up((size_t)s.n_slots);
     unsigned char *p = base;
     s.keys = (uint32_t *)p; p += b_keys;
     s.keysB = (uint32_t *)p; p += b_keys;
@@ -1796,6 +1871,7 @@ static size_t sync_layout(const SgnsArgs &a, unsigned char *base, SyncScratch *o
     s.tinfo = (uint32_t *)p; p += b_pairs;
     s.n_out = (uint32_t *)p; p += 256;
     s.counts = (uint32_t *)p; p += b_cnt;
+    s.single = (uint8_t *)p; p += b_single;
     s.lead_part = (double *)p; p += b_part;
     s.tail_part = (double *)p; p += b_part;
     // the sort alternates B, C, B, ...: an odd number of passes ends in B
@@ -1824,6 +1900,7 @@ static gs_status sync_scratch(const SgnsArgs &a, int set, const FixedScratch *fi
         }
         // Every byte that is read is written first by the pass before it (keys and pair counts
         // by the targets pass for all slots; digit counts by the histogram pass for all tiles;
+        // the marks of one-entry runs by the marking pass for every list entry that exists;
         // g, GU and losses by the coefficient pass wherever the apply passes read them; the
         // partial sums of cut runs by the apply pass before the fix-up pass reads exactly
         // those), so nothing left over from an earlier call can leak in.
@@ -1856,6 +1933,13 @@ static gs_status sync_prepare(const SgnsArgs &a, int set, const FixedScratch *fi
                      sc.counts, st, &ks, &vs);
     GS_CUDA_TRY(cudaGetLastError());
     if (ks != sc.ks || vs != sc.vs) { set_error("internal: sort result buffer mismatch"); return GS_ERR_CUDA; }
+    if (sc.mark) {
+        int64_t mb = (sc.n_keys + 255) / 256;
+        if (mb > (int64_t)sm_count() * 16) mb = (int64_t)sm_count() * 16;
+        sgns_mark_single_kernel<<<(unsigned)mb, 256, 0, st>>>(sc.ks, sc.vs, (uint32_t)sc.n_keys,
+                                                              (uint32_t)a.n_nodes, sc.single);
+        GS_CUDA_TRY(cudaGetLastError());
+    }
     return GS_OK;
 }
 
@@ -1902,8 +1986,18 @@ static gs_status sync_update(const SgnsArgs &a, int set, const FixedScratch *fix
     {
         int64_t blocks = (sc.n_pos + 7) / 8;             // one warp per position
         if (blocks > cap) blocks = cap;
-        sgns_coef_kernel<DIM, T><<<(unsigned)blocks, 256, 0, st>>>(
-            w_in, w_out, sc.n_pos, sc.shift, (uint32_t)a.n_nodes, sc.keys, sc.tinfo, sc.gbuf, sc.GU, sc.loss_pos);
+        bool light = false;
+        if constexpr (sizeof(T) == 4) light = !mom;      // fp32 tables, plain SGD
+        if (light && sc.mark) {
+            if constexpr (sizeof(T) == 4)
+                sgns_coef_kernel<DIM, T, true><<<(unsigned)blocks, 256, 0, st>>>(
+                    w_in, w_out, sc.n_pos, sc.shift, (uint32_t)a.n_nodes, sc.keys, sc.tinfo, sc.gbuf, sc.GU,
+                    sc.loss_pos, sc.single, a.lr);
+        } else {
+            sgns_coef_kernel<DIM, T, false><<<(unsigned)blocks, 256, 0, st>>>(
+                w_in, w_out, sc.n_pos, sc.shift, (uint32_t)a.n_nodes, sc.keys, sc.tinfo, sc.gbuf, sc.GU,
+                sc.loss_pos, sc.single, a.lr);
+        }
         GS_CUDA_TRY(cudaGetLastError());
     }
     {
@@ -1911,10 +2005,16 @@ static gs_status sync_update(const SgnsArgs &a, int set, const FixedScratch *fix
         bool light = false;
         if constexpr (sizeof(T) == 4) light = !mom;      // fp32 tables, plain SGD
         if (light) {
-            if constexpr (sizeof(T) == 4)
-                sgns_apply_out_sgd_kernel<FPL><<<out_blocks, 256, 0, st>>>(
-                    w_in, w_out, a.walks, sc.ks, sc.vs, sc.gbuf, (uint32_t)sc.n_keys, (uint32_t)a.n_nodes,
-                    sc.shift, a.lr, sc.lead_part, sc.tail_part);
+            if constexpr (sizeof(T) == 4) {
+                if (sc.mark)
+                    sgns_apply_out_sgd_kernel<FPL, true><<<out_blocks, 256, 0, st>>>(
+                        w_in, w_out, a.walks, sc.ks, sc.vs, sc.gbuf, (uint32_t)sc.n_keys, (uint32_t)a.n_nodes,
+                        sc.shift, a.lr, sc.lead_part, sc.tail_part);
+                else
+                    sgns_apply_out_sgd_kernel<FPL, false><<<out_blocks, 256, 0, st>>>(
+                        w_in, w_out, a.walks, sc.ks, sc.vs, sc.gbuf, (uint32_t)sc.n_keys, (uint32_t)a.n_nodes,
+                        sc.shift, a.lr, sc.lead_part, sc.tail_part);
+            }
         } else {
             sgns_apply_out_kernel<FPL, T><<<out_blocks, 256, 0, st>>>(
                 w_in, w_out, a.walks, sc.ks, sc.vs, sc.gbuf, (uint32_t)sc.n_keys, (uint32_t)a.n_nodes, sc.shift,

@@ -332,6 +332,64 @@ def test_limits_of_the_supported_shapes(tiny, dim, L, w, K, n_walks):
         assert e.value.status == -6
 
 
+@pytest.mark.parametrize("dim", [32, 64, 128, 256])
+def test_deterministic_step_where_most_output_rows_receive_one_contribution(dim):
+    # 300,000 rows and a batch of 40 short walks: the tables have far more rows than the batch has
+    # list entries, the regime of large graphs, in which the step adds the increment of a row that
+    # receives a single contribution straight from the coefficient pass.  The power-law graph makes
+    # both kinds of rows occur (hubs collect several contributions).  Oracle on the touched rows.
+    wl = WL.WORKLOADS["deepwalk_medium"]
+    g = wl.make_graph(scale=0.3)
+    n = g.n_nodes
+    off, col = np_graph(g)
+    thr, alias = degree_alias(off)
+    L, w, K, n_walks, base, seed, lr = 10, 3, 4, 40, 12345, 6, 0.05
+    walks, _ = O.uniform_walks(off, col, None, n_walks, base, L, seed)
+    walks[3, L // 2:] = -1
+    c, o, ng, n_pairs = O.expand_lists(walks, base, w, K, thr, alias, seed)
+    ids, cc, oo, nn = compact_problem(c, o, ng)
+    assert n >= 3 * n_walks * L * 32                   # rows per (padded) list entry: the shortcut is on
+    pair_ok = cc >= 0
+    hits = np.bincount(oo[pair_ok], minlength=len(ids))
+    negs = nn[pair_ok]
+    hits += np.bincount(negs[(negs >= 0) & (negs != oo[pair_ok][:, None])], minlength=len(ids))
+    assert (hits == 1).sum() > 100 and (hits > 1).sum() > 20 and hits.max() >= 4
+    w_in0, w_out0 = random_tables(n, dim, 11)
+    U = w_in0[torch.from_numpy(ids)].numpy().astype(np.float64)
+    V = w_out0[torch.from_numpy(ids)].numpy().astype(np.float64)
+    V0 = V.copy()
+    loss_o, cnt_o = O.sgns_det_from_lists(U, V, cc, oo, nn, lr)
+    a_dev = alias_to_device(thr, alias)
+    w_in, w_out = w_in0.to(DEV), w_out0.to(DEV)
+    loss, cnt, pd, nd = run_step(w_in, w_out, torch.from_numpy(walks).to(DEV), base, w, K, a_dev, lr, seed,
+                                 B.GS_DETERMINISTIC)
+    pd = pd.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(pd[:, 0], c) and np.array_equal(pd[:, 1], o)
+    assert np.array_equal(nd.cpu().numpy().reshape(-1, K), ng)
+    assert cnt == cnt_o == n_pairs and abs(loss - loss_o) <= 2e-6 * abs(loss_o)
+    ids_dev = torch.from_numpy(ids).to(DEV)
+    assert np.abs(w_in[ids_dev].cpu().numpy() - U).max() <= EMB_TOL
+    got_out = w_out[ids_dev].cpu().numpy()
+    assert np.abs(got_out - V).max() <= EMB_TOL
+    # every output row that the lists name moved, whether it was hit once or several times, by much
+    # more than the tolerance; every row outside the batch kept its bits
+    moved = np.abs(V - V0).max(axis=1)
+    assert (moved[hits == 1] > 20 * EMB_TOL).all() and (moved[hits > 1] > 20 * EMB_TOL).all()
+    assert np.array_equal(np.abs(got_out - V0).max(axis=1) > 0, hits > 0)
+    outside = torch.ones(n, dtype=torch.bool)
+    outside[torch.from_numpy(ids)] = False
+    assert torch.equal(w_in.cpu()[outside], w_in0[outside]) and torch.equal(w_out.cpu()[outside], w_out0[outside])
+    # bitwise reproducible, and the allocation-free entry point gives the same bits
+    for step in (B.gs_sgns_step, B.gs_sgns_step_static):
+        w_in2, w_out2 = w_in0.to(DEV), w_out0.to(DEV)
+        if step is B.gs_sgns_step:
+            step(w_in2, w_out2, torch.from_numpy(walks).to(DEV), base, w, K, a_dev, lr, seed, B.GS_DETERMINISTIC)
+        else:
+            step(w_in2, w_out2, torch.from_numpy(walks).to(DEV), base, w, K, a_dev, lr, seed)
+        torch.cuda.synchronize()
+        assert torch.equal(w_in, w_in2) and torch.equal(w_out, w_out2)
+
+
 def test_deterministic_step_hub_rows_with_thousands_of_contributions():
     # a star: every walk alternates hub / leaf, so one output row collects most contributions
     n = 400
